@@ -1,0 +1,216 @@
+/*
+ * planfront_oracle.h -- CPU reference ("oracle") for batched MoE parallel-plan scoring.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This is the plain, slow, candidate-by-candidate definition of
+ * what the scoring path computes: fp64 for every floating quantity, int64 for every byte and
+ * token count, a full sort for top-k.  It shares no code with the CUDA library and must never
+ * be linked, imported or called from the product path; only the tests, the smoke check and
+ * the benchmark's CPU-baseline leg use it.
+ *
+ * What it follows (paper sections):
+ *   - plan tuple and its axes ............ Sec. 3.1 (intermediate representation)
+ *   - predicate order: emit dry-run rules first, memory gate second ... Sec. 3.3, Fig. 2
+ *   - rule list (unmapped schedule class, layer-count divisibility, overlap preconditions,
+ *     serving dp == ep, missing kernels) . Sec. 4 "Emitters", Fig. 2, Sec. 5 RQ1
+ *   - memory gate, 0.9 usable fraction, expert-DP optimizer shards ... Sec. 2.1, Sec. 5 RQ1
+ *   - analytic (closed-form) scorer and the list-scheduling simulator . Sec. 3.2
+ *   - realization tax, throughput / (1 + frac) ........................ Sec. 3.2, Table "tax"
+ *   - calibration domain m_range [64, 8192], "extrapolated" flag ...... Sec. 3 (P4), Appendix
+ *   - top-k invariant (every returned plan passes the predicate) ...... Sec. 3.3
+ * The paper prints no equations; where it is silent the reading taken is stated beside each
+ * formula in planfront_oracle.c.
+ *
+ * Pins (what fixes this file to something other than itself) live in the CPU tests:
+ * printed memory numbers (72 GB budget, 21.59 GB expert optimizer state, the 10.8 / 21.59 GB
+ * ep8 -> ep4 -> ep2 increments), the tax rule, rule outcomes the paper states (27 layers vs
+ * pp*v, serving dp != ep, DualPipe unmapped), the 1F1B bubble closed form, the interleaved
+ * closed form, brute-force enumeration of the tiny space, and monotonicity invariants.
+ * PARITY UNPINNED: absolute throughputs (the paper's cost constants are not published), the
+ * DualPipe analytic closed form and its startup divisor, and the serving time model.
+ */
+#ifndef PLANFRONT_ORACLE_H
+#define PLANFRONT_ORACLE_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define ORC_MAX_SCHED 8
+#define ORC_MAX_KERN 16
+#define ORC_NBUCKET 8
+#define ORC_MAX_AXES 10
+#define ORC_MAX_RANKS 32   /* simulator domain: pp <= 32 */
+#define ORC_MAX_V 8        /* simulator domain: virtual stages per rank <= 8 */
+#define ORC_SIM_WINDOW 64  /* simulated microbatches per step at most */
+
+/* reason codes (first failing rule, in this order) */
+enum {
+    ORC_FEASIBLE = 0,
+    ORC_R_WORLD = 1,
+    ORC_R_TP = 2,
+    ORC_R_EP = 3,
+    ORC_R_BATCH = 4,
+    ORC_R_VSTAGE = 5,
+    ORC_R_LAYERS = 6,
+    ORC_R_MICROBATCH = 7,
+    ORC_R_KERNEL_MISSING = 8,
+    ORC_R_UNMAPPED_SCHEDULE = 9,
+    ORC_R_OVERLAP_PRECOND = 10,
+    ORC_R_MEMORY = 11,
+    ORC_FLAG_EXTRAPOLATED = 0x80
+};
+
+enum { ORC_KIND_1F1B = 0, ORC_KIND_INTERLEAVED = 1, ORC_KIND_DUALPIPE = 2 };
+enum { ORC_REC_NONE = 0, ORC_REC_SELECTIVE = 1, ORC_REC_FULL = 2 };
+enum { ORC_SIM_OK = 0, ORC_SIM_UNSUPPORTED = 1, ORC_SIM_STALL = 2 };
+
+typedef struct {
+    int64_t L, H, nh, nkv, hd;
+    int64_t attn_kind; /* 0 MHA/GQA, 1 MLA */
+    int64_t kv_latent, rope_dim;
+    int64_t E, K, F, S, Fs;
+    int64_t seq, vocab;
+    int64_t wb, gb, ob, ab; /* bytes: weight, gradient, optimizer state per parameter, activation */
+    int64_t n_mats;         /* matrices per expert FFN (3 = gate, up, down) */
+    int64_t count_embeddings;
+} orc_model_t;
+
+typedef struct {
+    int64_t G;            /* GPUs per node */
+    int64_t budget_bytes; /* usable HBM per GPU (caller: 0.9 x capacity) */
+    int64_t reserved_bytes;
+    int64_t caps; /* bit 0: fp8, bit 1: device-initiated communication */
+    double peak_flops, hbm_bw, bw_intra, bw_inter, alpha_intra, alpha_inter;
+} orc_cluster_t;
+
+typedef struct {
+    int64_t phase;      /* 0 train, 1 serve */
+    int64_t gbs;        /* train: sequences per step */
+    int64_t world;      /* serve: the cluster's world size */
+    int64_t n_scen;     /* serve: number of (prompt, output) scenarios */
+    const int64_t *scen_P;
+    const int64_t *scen_O;
+} orc_workload_t;
+
+typedef struct {
+    double eff_dense, bwd_factor, dp_overlap_frac, dualpipe_startup_div, step_overhead;
+} orc_consts_t;
+
+typedef struct {
+    int64_t kind, overlap, mapped;
+    double hide_frac, sched_ovh;
+} orc_sched_t;
+
+typedef struct {
+    int64_t needs_caps, avail_mask, is_native, wbytes;
+    double dtype_mult, eff[ORC_NBUCKET], patch_ovh;
+} orc_kern_t;
+
+typedef struct {
+    int64_t ep_scope;   /* 0: ep | dp, 1: ep | dp*tp */
+    int64_t layer_mode; /* 0: L mod (pp*v) == 0, 2: balanced uneven split, pp*v <= L */
+    int64_t tp_max, world_min, world_max;
+    int64_t enforce_realizability;
+} orc_rules_t;
+
+/* axis value lists, least-significant digit first.
+ * train: kv, rec, sched, mb, v, ep, pp, tp, dp, world   (10 axes)
+ * serve: kv, chunk, batch, dpa, ep, tp, scen             (7 axes) */
+typedef struct {
+    int64_t n_axes;
+    int64_t len[ORC_MAX_AXES];
+    const int64_t *val[ORC_MAX_AXES];
+} orc_axes_t;
+
+typedef struct {
+    orc_model_t model;
+    orc_cluster_t cluster;
+    orc_workload_t workload;
+    orc_consts_t consts;
+    int64_t n_sched;
+    orc_sched_t sched[ORC_MAX_SCHED];
+    int64_t n_kern;
+    orc_kern_t kern[ORC_MAX_KERN];
+    orc_rules_t rules;
+    orc_axes_t axes;
+} orc_problem_t;
+
+/* candidate-independent model constants (exact integers) */
+typedef struct {
+    int64_t dk, P_attn, P_rt, P_e, P_sh, P_dl, P_emb;
+    int64_t a_attn, a_fix, a_ffn, a_full, a_sel, a_ckpt;
+    int64_t f_attn, f_rt, f_sh, f_dense, f_exp, f_head;
+} orc_derived_t;
+
+/* everything computed for one candidate; unfilled parts stay 0 */
+typedef struct {
+    /* decoded tuple (train names; serve: chunk->mb slot unused, see fields below) */
+    int64_t kv, rec, sched, mb, v, ep, pp, tp, dp, world;
+    int64_t chunk, batch, dpa, scen; /* serve */
+    /* derived integers */
+    int64_t kind, ov, v_eff, m, t, Q, Lc, Ls, edp, m_e, bucket, bucket_pre;
+    /* memory terms */
+    int64_t N_dense, N_exp, bytes_w, bytes_g, bytes_o_dense, bytes_o_expert, bytes_o, bytes_a, mem;
+    /* time terms */
+    double cF, cB, rc, tpc, a2a, xF, xB, F_l, B_l, headF, F, B, p, T_pipe, T_dp, T_opt, T_step;
+    double T_dec, T_pre; /* serve */
+    double tput_unpriced, tput;
+    int64_t reason;
+} orc_detail_t;
+
+int64_t orc_budget_bytes(int64_t hbm_bytes); /* floor(0.9 * capacity), in integers */
+void orc_derive(const orc_model_t *m, orc_derived_t *d);
+uint64_t orc_space_size(const orc_problem_t *pb);
+
+/* score one candidate: fills detail (may be NULL); returns the reason byte */
+int orc_eval(const orc_problem_t *pb, uint64_t idx, orc_detail_t *detail);
+
+/* score [first, first+count); any output may be NULL; uses OpenMP threads when n_threads > 1.
+ * returns the number of threads actually used */
+int orc_score_range(const orc_problem_t *pb, uint64_t first, uint64_t count, uint8_t *reason,
+                    double *tput, int64_t *mem, int n_threads);
+
+/* top-k among entries with (reason & 0x7f) == 0, by (tput desc, idx asc): full sort.
+ * idx[i] = first + i for the dense arrays given.  returns the number written (<= k) */
+uint64_t orc_topk(const uint8_t *reason, const double *tput, uint64_t first, uint64_t count,
+                  uint64_t k, uint64_t *out_idx, double *out_score);
+/* same, over an explicit index list (re-ranking of survivors) */
+uint64_t orc_topk_list(const uint64_t *idx, const double *score, uint64_t n, uint64_t k,
+                       uint64_t *out_idx, double *out_score);
+
+/* survivors: the s_max best feasible candidates inside the simulator domain, sorted by idx */
+uint64_t orc_select_survivors(const orc_problem_t *pb, const uint8_t *reason, const double *tput,
+                              uint64_t first, uint64_t count, uint64_t s_max, uint64_t *out_idx);
+
+/* --- simulator tier --- */
+/* op encoding for per-rank orders: bit 0 = backward, bit 1 = direction (DualPipe), bits 2..9 =
+ * virtual stage / position q, bits 10.. = microbatch j */
+#define ORC_OP(q, j, dir, isb) ((int32_t)(((j) << 10) | ((q) << 2) | ((dir) << 1) | (isb)))
+#define ORC_OP_ISB(o) ((o) & 1)
+#define ORC_OP_DIR(o) (((o) >> 1) & 1)
+#define ORC_OP_Q(o) (((o) >> 2) & 255)
+#define ORC_OP_J(o) ((o) >> 10)
+
+/* per-rank static order; out[rank*stride .. ] receives n_ops ops; returns ops per rank, <0 on error
+ * kind 0: 1F1B (v ignored), 1: interleaved (m % pp == 0), 2: DualPipe-style (pp == 1 or even, m even) */
+int orc_schedule_order(int kind, int pp, int v, int m, int32_t *out, int stride);
+
+/* evaluate a fixed order with per-stage durations; returns makespan, <0 on stall.
+ * Fq/Bq have Q entries (Q = pp*v; DualPipe: pp).  p = cross-rank latency */
+double orc_makespan(int kind, int pp, int v, int m, const double *Fq, const double *Bq, double p);
+
+uint32_t orc_mix32(uint32_t x);
+double orc_jitter(uint32_t seed, uint64_t idx, int q, int is_backward);
+
+/* simulate one survivor; returns status; *tput_sim receives the priced simulated throughput */
+int orc_simulate(const orc_problem_t *pb, uint64_t idx, uint32_t seed, double *tput_sim,
+                 double *T_pipe_sim);
+int orc_simulate_list(const orc_problem_t *pb, const uint64_t *idx, uint64_t n, uint32_t seed,
+                      double *tput_sim, uint8_t *status, int n_threads);
+
+#ifdef __cplusplus
+}
+#endif
+#endif
