@@ -1,0 +1,266 @@
+/*
+ * planfront.h -- C ABI of the B200 plan-scoring library (libplanfront.so).
+ *
+ * The library scores every candidate of a mixed-radix plan space on one GPU:
+ *   (model spec, modeled-cluster spec, plan-axis ranges, kernel/overhead tables)
+ *     -> (feasibility reason, predicted tokens/s/GPU, peak memory per GPU, top-k plan indices),
+ * then re-ranks the best survivors with a per-candidate pipeline-schedule simulation.
+ * This is the search loop of the paper's three-tier optimizer (Sec. 3.3) with its realizability
+ * predicate (Sec. 3.3, Fig. 2), dual-fidelity cost model (Sec. 3.2) and realization tax (Sec. 3.2),
+ * evaluated for all candidates at once instead of one Python call per plan.
+ *
+ * Conventions
+ *   - plain C, no exceptions; every call returns an int32 status (PF_OK = 0, negative = error).
+ *   - "d_" pointers are DEVICE pointers owned by the caller; everything else is HOST memory.
+ *   - the library allocates no output or workspace memory: the caller passes raw pointers and sizes.
+ *     (pf_plan_create allocates a few KB of device memory for the plan's constant tables, freed by
+ *     pf_plan_destroy.)
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  All device work is
+ *     enqueued on it and the calls do not synchronize; results are valid once the stream has been
+ *     synchronized by the caller.  pf_search_host is the exception: it takes host buffers and returns
+ *     after its copies have completed.
+ *   - spec structs are copied by pf_plan_create; the caller may free them afterwards.
+ *   - a handle may be used from one thread at a time, on the device that was current at create.
+ *   - candidates are addressed by a linear index: idx = sum_a digit_a * prod_{b<a} len_b, axes listed
+ *     least-significant first.  train axes: kv, rec, sched, mb, v, ep, pp, tp, dp, world;
+ *     serve axes: kv, chunk, batch, dpa, ep, tp, scen.  An axis value list {0} for dp / world / v means
+ *     "derived" (dp = world/(tp*pp); world = tp*pp*dp; v = 2 for interleaved schedules, else 1).
+ */
+#ifndef PLANFRONT_H
+#define PLANFRONT_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define PF_VERSION 100
+#define PF_MAX_AXES 10
+#define PF_MAX_AXIS_LEN 4096
+#define PF_MAX_SCHED 8
+#define PF_MAX_KERN 16
+#define PF_NBUCKET 8
+#define PF_K_MAX 1024         /* largest top-k */
+#define PF_MAX_SCEN 4096
+#define PF_SIM_MAX_RANKS 32   /* simulator domain: pp <= 32 (one lane per pipeline rank) */
+#define PF_SIM_MAX_V 8        /* simulator domain: virtual stages per rank <= 8 */
+#define PF_SIM_WINDOW 64      /* simulated microbatches per step at most */
+#define PF_MAX_COUNT (1ull << 32) /* pf_score / pf_select_survivors take count < PF_MAX_COUNT per call */
+
+/* status codes */
+enum {
+    PF_OK = 0,
+    PF_EINVAL = -1,       /* NULL required pointer, inconsistent spec, k out of range */
+    PF_ERANGE = -2,       /* axis length 0 or too long, space size >= 2^63, range outside the space */
+    PF_EWORKSPACE = -3,   /* workspace too small or misaligned (needs 256-byte alignment) */
+    PF_ECUDA = -4,        /* a CUDA runtime call failed; see pf_last_cuda_error() */
+    PF_EUNSUPPORTED = -5  /* the call does not apply to this plan's phase */
+};
+
+/* per-candidate reason byte: 0 = feasible, else the FIRST failing rule in this order (the predicate's
+ * fixed order: structural checks, emit dry-run rules, memory gate last -- Sec. 3.3, Fig. 2).
+ * Bit 7 is OR-ed into a feasible candidate whose tokens-per-expert lies outside the calibration
+ * domain [64, 8192] ("extrapolated", Sec. 3 principle P4). */
+enum {
+    PF_FEASIBLE = 0,
+    PF_R_WORLD = 1,
+    PF_R_TP = 2,
+    PF_R_EP = 3,
+    PF_R_BATCH = 4,
+    PF_R_VSTAGE = 5,
+    PF_R_LAYERS = 6,
+    PF_R_MICROBATCH = 7,
+    PF_R_KERNEL_MISSING = 8,
+    PF_R_UNMAPPED_SCHEDULE = 9,
+    PF_R_OVERLAP_PRECOND = 10,
+    PF_R_MEMORY = 11,
+    PF_FLAG_EXTRAPOLATED = 0x80
+};
+
+enum { PF_KIND_1F1B = 0, PF_KIND_INTERLEAVED = 1, PF_KIND_DUALPIPE = 2 };
+enum { PF_REC_NONE = 0, PF_REC_SELECTIVE = 1, PF_REC_FULL = 2 };
+enum { PF_PHASE_TRAIN = 0, PF_PHASE_SERVE = 1 };
+enum { PF_CAP_FP8 = 1, PF_CAP_DEVICE_COMM = 2 };
+/* per-survivor simulator status */
+enum { PF_SIM_OK = 0, PF_SIM_UNSUPPORTED = 1, PF_SIM_STALL = 2 };
+
+typedef struct {
+    int32_t L, H, nh, nkv, hd;
+    int32_t attn_kind;            /* 0 MHA/GQA, 1 MLA (compressed KV) */
+    int32_t kv_latent, rope_dim;  /* MLA only */
+    int32_t E, K, F, S, Fs;       /* routed experts, top-k, expert FFN, shared experts, shared FFN */
+    int32_t seq, vocab;
+    int32_t wb, gb, ob, ab;       /* bytes per weight / gradient / optimizer state per param / activation */
+    int32_t n_mats;               /* matrices per expert FFN (3 = gate, up, down) */
+    int32_t count_embeddings;     /* 0/1: embedding + head counted in memory */
+} pf_model_t;
+
+typedef struct {
+    int32_t G;                    /* GPUs per node */
+    uint32_t caps;                /* PF_CAP_* bits the modeled cluster has */
+    int64_t budget_bytes;         /* usable HBM per GPU: the memory gate rejects mem > budget (Sec. 5 RQ1) */
+    int64_t reserved_bytes;       /* added to every candidate's memory */
+    float peak_flops, hbm_bw, bw_intra, bw_inter, alpha_intra, alpha_inter;
+} pf_cluster_t;
+
+typedef struct {
+    int32_t phase;                /* PF_PHASE_* */
+    int32_t n_scen;               /* serve: number of (prompt, output) length scenarios */
+    int64_t gbs;                  /* train: sequences per step */
+    int64_t world;                /* serve: world size of the modeled cluster */
+    const int32_t *scen_P;        /* host, n_scen entries */
+    const int32_t *scen_O;
+} pf_workload_t;
+
+typedef struct {
+    int32_t n_axes;               /* 10 (train) or 7 (serve) */
+    int32_t len[PF_MAX_AXES];     /* 1 .. PF_MAX_AXIS_LEN */
+    const int32_t *val[PF_MAX_AXES]; /* host value lists */
+} pf_axes_t;
+
+typedef struct {
+    int32_t kind;                 /* PF_KIND_* */
+    int32_t overlap;              /* expert all-to-all overlapped with compute */
+    int32_t mapped;               /* 0: the toolchain cannot emit this class (Sec. 2.1) */
+    float hide_frac;              /* hidden fraction of the all-to-all when overlapped (alpha-table) */
+    float sched_ovh;              /* realization overhead, applied as tput / (1 + ovh) when overlap = 1 */
+} pf_sched_t;
+
+typedef struct {
+    uint32_t needs_caps;          /* PF_CAP_* bits the variant needs */
+    uint32_t avail_mask;          /* bit b: the autotune report has an entry for tokens-per-expert bucket b */
+    int32_t is_native;            /* 1: the engine's own kernel, pays no patch overhead */
+    int32_t wbytes;               /* expert weight bytes per parameter in serving (2 bf16, 1 fp8) */
+    float dtype_mult;             /* peak multiplier of the variant's dtype (1 bf16, 2 fp8) */
+    float eff[PF_NBUCKET];        /* efficiency per bucket: m_e <128, 128.., 256.., ... , >=8192 */
+    float patch_ovh;              /* realization tax, applied as tput / (1 + ovh) when !is_native */
+} pf_kern_t;
+
+typedef struct {
+    float eff_dense, bwd_factor, dp_overlap_frac, dualpipe_startup_div, step_overhead;
+    int32_t n_sched;
+    pf_sched_t sched[PF_MAX_SCHED];
+    int32_t n_kern;
+    pf_kern_t kern[PF_MAX_KERN];
+} pf_tables_t;
+
+typedef struct {
+    int32_t ep_scope;             /* 0: ep | dp (EP inside DP, Sec. 4), 1: ep | dp*tp */
+    int32_t layer_mode;           /* 0: L mod (pp*v) == 0 (Fig. 2), 2: balanced uneven split, pp*v <= L */
+    int32_t tp_max;
+    int32_t world_min, world_max;
+    int32_t enforce_realizability; /* 0: unconstrained mode, dry-run rules 9-10 skipped (Sec. 3.3) */
+} pf_rules_t;
+
+typedef struct {
+    int32_t kv, rec, sched, mb, v, ep, pp, tp, dp, world; /* train (dp/world as listed, before derivation) */
+    int32_t chunk, batch, dpa, scen;                      /* serve */
+} pf_tuple_t;
+
+typedef struct pf_plan pf_plan_t;
+
+int pf_version(void);
+const char *pf_strerror(int status);
+const char *pf_reason_str(uint8_t reason);
+/* text of the last CUDA error seen by this thread's library calls ("" if none) */
+const char *pf_last_cuda_error(void);
+
+/* Build a plan space (Sec. 3.1: one normalized tuple carries every knob; Sec. 3.3: enumeration).
+ * Validates the specs, derives the candidate-independent constants (parameter, activation and FLOP
+ * counts per layer; radices; schedule-order tables for the simulator) and uploads them.
+ * Errors: PF_EINVAL (NULL pointer, phase/axis-count mismatch, table index out of range, both dp and
+ * world derived), PF_ERANGE (axis length, value range, space size), PF_ECUDA. */
+int pf_plan_create(const pf_model_t *model, const pf_cluster_t *cluster, const pf_workload_t *workload,
+                   const pf_axes_t *axes, const pf_tables_t *tables, const pf_rules_t *rules, pf_plan_t **out);
+void pf_plan_destroy(pf_plan_t *plan);
+uint64_t pf_plan_size(const pf_plan_t *plan); /* N = product of axis lengths */
+/* host helper: linear index -> axis values (no rule is applied).  PF_ERANGE if idx >= N. */
+int pf_decode(const pf_plan_t *plan, uint64_t idx, pf_tuple_t *out);
+
+/* Score candidates [first, first+count): decode -> realizability rules -> memory gate -> analytic step
+ * time -> priced throughput (Sec. 3.2-3.3), and reduce to the k best feasible ones by (tput descending,
+ * index ascending) (Sec. 3.3: every returned plan passes the predicate).
+ *   d_reason[count] uint8, d_tput[count] float (tokens/s/GPU, 0 when infeasible), d_mem[count] int64
+ *   (bytes; 0 when a rule before the memory gate failed) -- each may be NULL (not written); element i
+ *   belongs to candidate first+i.
+ *   k = 0 skips the top-k; otherwise 1 <= k <= PF_K_MAX and d_topk_idx[k] (uint64, UINT64_MAX in unused
+ *   slots), d_topk_score[k] (float, 0 in unused slots), d_topk_count[1] (uint32) are required.
+ *   d_workspace: at least pf_score_workspace(plan, count, k) bytes, 256-byte aligned, contents ignored.
+ * count < PF_MAX_COUNT per call; larger spaces are scored in chunks and merged with pf_topk_merge.
+ * Errors: PF_EINVAL, PF_ERANGE, PF_EWORKSPACE, PF_ECUDA (launch failure). */
+size_t pf_score_workspace(const pf_plan_t *plan, uint64_t count, uint32_t k);
+int pf_score(pf_plan_t *plan, uint64_t first, uint64_t count, uint8_t *d_reason, float *d_tput, int64_t *d_mem,
+             uint32_t k, uint64_t *d_topk_idx, float *d_topk_score, uint32_t *d_topk_count, void *d_workspace,
+             size_t workspace_bytes, void *stream);
+
+/* Merge two top-k lists (as written by pf_score / pf_simulate, each sorted, with device counts) into the k
+ * best of their union, same ordering rule.  Used to combine chunks or shards of one space.  The output
+ * may alias neither input.  Errors: PF_EINVAL (k out of range, NULL). */
+int pf_topk_merge(uint32_t k, const uint64_t *d_idx_a, const float *d_score_a, const uint32_t *d_count_a,
+                  const uint64_t *d_idx_b, const float *d_score_b, const uint32_t *d_count_b,
+                  uint64_t *d_idx_out, float *d_score_out, uint32_t *d_count_out, void *stream);
+
+/* Survivor selection for the schedule tier (Sec. 3.3: the top-ranked layouts are refined with the
+ * simulator; here the short list is the s_max best instead of ten): among candidates of
+ * [first, first+count) that are feasible ((reason & 0x7f) == 0) and inside the simulator's domain
+ * (training plan, pp <= PF_SIM_MAX_RANKS, virtual stages <= PF_SIM_MAX_V), the s_max best by
+ * (tput descending, index ascending), written as absolute indices in ASCENDING index order.
+ *   d_reason / d_tput: the dense outputs of pf_score for the same range (required).
+ *   d_surv_idx[s_max] uint64, d_surv_count[1] uint64 (= min(s_max, eligible)).
+ * Errors: PF_EINVAL, PF_ERANGE, PF_EWORKSPACE, PF_EUNSUPPORTED (serving plan), PF_ECUDA. */
+size_t pf_select_workspace(const pf_plan_t *plan, uint64_t count, uint64_t s_max);
+int pf_select_survivors(pf_plan_t *plan, uint64_t first, uint64_t count, const uint8_t *d_reason,
+                        const float *d_tput, uint64_t s_max, uint64_t *d_surv_idx, uint64_t *d_surv_count,
+                        void *d_workspace, size_t workspace_bytes, void *stream);
+
+/* Simulator tier (Sec. 3.2: the list-scheduling timeline is the higher-fidelity scorer used to refine
+ * schedules).  For each of the n candidates listed in d_surv_idx (n may also be given on the device:
+ * if d_n is not NULL the kernel uses min(n, *d_n)): per-stage forward/backward durations from the
+ * analytic terms with an exact balanced layer split, +-10% multiplicative jitter from a counter hash
+ * of (jitter_seed, idx, stage, F/B), evaluation of the schedule's fixed per-rank order (1F1B,
+ * interleaved, DualPipe-style) with cross-rank latency, steady-state extension beyond PF_SIM_WINDOW
+ * microbatches, then the same step terms and pricing as pf_score.
+ *   d_tput_sim[n] float, d_sim_status[n] uint8 (PF_SIM_*) -- each may be NULL.
+ *   top-k outputs as in pf_score, ranking by (tput_sim descending, index ascending); entries past
+ *   min(n, *d_n) are ignored.  An infeasible candidate scores 0 with status PF_SIM_UNSUPPORTED; a
+ *   feasible one outside the domain keeps its analytic score with PF_SIM_UNSUPPORTED.
+ * Errors: PF_EINVAL, PF_EWORKSPACE, PF_EUNSUPPORTED (serving plan), PF_ECUDA. */
+size_t pf_simulate_workspace(const pf_plan_t *plan, uint64_t n, uint32_t k);
+int pf_simulate(pf_plan_t *plan, const uint64_t *d_surv_idx, uint64_t n, const uint64_t *d_n,
+                uint32_t jitter_seed, float *d_tput_sim, uint8_t *d_sim_status, uint32_t k,
+                uint64_t *d_topk_idx, float *d_topk_score, uint32_t *d_topk_count, void *d_workspace,
+                size_t workspace_bytes, void *stream);
+
+/* Host helper (no GPU): the DualPipe-style per-rank op order the simulator uses for pipeline depth pp
+ * (1 or even, <= PF_SIM_MAX_RANKS) and m microbatches (even, 2..PF_SIM_WINDOW).  The order is defined by a
+ * nominal list scheduling (forward 1 tick, backward 2 ticks, zero latency; ready op with the smallest
+ * (ready time, backward first, microbatch, direction); a forward at position q waits while pp - q
+ * microbatches of its direction are in flight on the rank).  The paper names the schedule class only
+ * (Sec. 3.1); this order is this library's definition of it.
+ * out_ops[pp][2*m]: op = (microbatch << 2) | (direction << 1) | is_backward; direction 0 places position q
+ * on rank q, direction 1 on rank pp-1-q; each direction carries m/2 microbatches.
+ * Errors: PF_EINVAL (shape outside the domain, NULL). */
+int pf_dualpipe_order(int pp, int m, uint8_t *out_ops);
+
+/* Whole search with HOST result buffers (the call a user without device code makes): scores the full
+ * space, returns the analytic top-k and -- for training plans with s_max > 0 -- the simulator-refined
+ * top-k_sim over the s_max best survivors.  Dense per-candidate outputs are copied back only for the
+ * non-NULL h_* pointers (N elements each).  d_workspace must hold pf_search_workspace() bytes of DEVICE
+ * memory (it carries the dense arrays, the survivor list and the per-kernel workspaces).
+ * Returns after all copies have completed.  Errors as the calls above. */
+size_t pf_search_workspace(const pf_plan_t *plan, uint32_t k, uint64_t s_max, uint32_t k_sim);
+int pf_search_host(pf_plan_t *plan, uint32_t k, uint64_t s_max, uint32_t k_sim, uint32_t jitter_seed,
+                   uint8_t *h_reason, float *h_tput, int64_t *h_mem, uint64_t *h_topk_idx, float *h_topk_score,
+                   uint32_t *h_topk_count, uint64_t *h_sim_topk_idx, float *h_sim_topk_score,
+                   uint32_t *h_sim_topk_count, uint64_t *h_surv_count, void *d_workspace,
+                   size_t workspace_bytes, void *stream);
+
+/* Number of kernels this library has launched in this process (for launch accounting in benchmarks). */
+uint64_t pf_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif

@@ -1,0 +1,361 @@
+"""Thin ctypes binding over libplanfront.so: argument marshalling only.
+
+Every step of the path (decode, rules, memory, cost, pricing, top-k, survivor selection, simulation) runs in
+the library's CUDA kernels.  PyTorch provides device memory and the current stream, nothing else.  There is
+no CPU fallback: if the library is missing or no CUDA device is present, the calls raise.
+
+Function names mirror the C ABI declared in include/planfront.h.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(HERE, "libplanfront.so")
+
+MAX_AXES, MAX_SCHED, MAX_KERN, NBUCKET, K_MAX = 10, 8, 16, 8, 1024
+PF_OK, PF_EINVAL, PF_ERANGE, PF_EWORKSPACE, PF_ECUDA, PF_EUNSUPPORTED = 0, -1, -2, -3, -4, -5
+UINT64_MAX = 0xFFFFFFFFFFFFFFFF
+
+EXPORTS = ("pf_version", "pf_strerror", "pf_reason_str", "pf_last_cuda_error", "pf_plan_create", "pf_plan_destroy",
+           "pf_plan_size", "pf_decode", "pf_score_workspace", "pf_score", "pf_topk_merge", "pf_select_workspace",
+           "pf_select_survivors", "pf_simulate_workspace", "pf_simulate", "pf_search_workspace", "pf_search_host",
+           "pf_launch_count", "pf_dualpipe_order")
+
+i32, u32, i64, u64, f32 = C.c_int32, C.c_uint32, C.c_int64, C.c_uint64, C.c_float
+
+
+class PfModel(C.Structure):
+    _fields_ = [(n, i32) for n in ("L", "H", "nh", "nkv", "hd", "attn_kind", "kv_latent", "rope_dim", "E", "K", "F",
+                                   "S", "Fs", "seq", "vocab", "wb", "gb", "ob", "ab", "n_mats", "count_embeddings")]
+
+
+class PfCluster(C.Structure):
+    _fields_ = [("G", i32), ("caps", u32), ("budget_bytes", i64), ("reserved_bytes", i64)] + \
+               [(n, f32) for n in ("peak_flops", "hbm_bw", "bw_intra", "bw_inter", "alpha_intra", "alpha_inter")]
+
+
+class PfWorkload(C.Structure):
+    _fields_ = [("phase", i32), ("n_scen", i32), ("gbs", i64), ("world", i64),
+                ("scen_P", C.POINTER(i32)), ("scen_O", C.POINTER(i32))]
+
+
+class PfAxes(C.Structure):
+    _fields_ = [("n_axes", i32), ("len", i32 * MAX_AXES), ("val", C.POINTER(i32) * MAX_AXES)]
+
+
+class PfSched(C.Structure):
+    _fields_ = [("kind", i32), ("overlap", i32), ("mapped", i32), ("hide_frac", f32), ("sched_ovh", f32)]
+
+
+class PfKern(C.Structure):
+    _fields_ = [("needs_caps", u32), ("avail_mask", u32), ("is_native", i32), ("wbytes", i32),
+                ("dtype_mult", f32), ("eff", f32 * NBUCKET), ("patch_ovh", f32)]
+
+
+class PfTables(C.Structure):
+    _fields_ = [(n, f32) for n in ("eff_dense", "bwd_factor", "dp_overlap_frac", "dualpipe_startup_div",
+                                   "step_overhead")] + \
+               [("n_sched", i32), ("sched", PfSched * MAX_SCHED), ("n_kern", i32), ("kern", PfKern * MAX_KERN)]
+
+
+class PfRules(C.Structure):
+    _fields_ = [(n, i32) for n in ("ep_scope", "layer_mode", "tp_max", "world_min", "world_max",
+                                   "enforce_realizability")]
+
+
+class PfTuple(C.Structure):
+    _fields_ = [(n, i32) for n in ("kv", "rec", "sched", "mb", "v", "ep", "pp", "tp", "dp", "world", "chunk",
+                                   "batch", "dpa", "scen")]
+
+
+class PlanfrontError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        self.status = status
+        super().__init__(what)
+
+
+_lib = None
+
+
+def load_library(path: str | None = None):
+    """dlopen libplanfront.so and declare the signatures.  Raises if the library has not been built."""
+    global _lib
+    if _lib is not None and path is None:
+        return _lib
+    path = path or LIB_PATH
+    if not os.path.exists(path):
+        raise PlanfrontError(PF_EINVAL, f"{path} not found: build it with `python -m paper_2607_18631_b200.build`")
+    L = C.CDLL(path)
+    vp, sz = C.c_void_p, C.c_size_t
+    L.pf_version.restype = C.c_int
+    L.pf_strerror.restype = C.c_char_p
+    L.pf_strerror.argtypes = [C.c_int]
+    L.pf_reason_str.restype = C.c_char_p
+    L.pf_reason_str.argtypes = [C.c_uint8]
+    L.pf_last_cuda_error.restype = C.c_char_p
+    L.pf_plan_create.restype = C.c_int
+    L.pf_plan_create.argtypes = [C.POINTER(PfModel), C.POINTER(PfCluster), C.POINTER(PfWorkload), C.POINTER(PfAxes),
+                                 C.POINTER(PfTables), C.POINTER(PfRules), C.POINTER(vp)]
+    L.pf_plan_destroy.restype = None
+    L.pf_plan_destroy.argtypes = [vp]
+    L.pf_plan_size.restype = u64
+    L.pf_plan_size.argtypes = [vp]
+    L.pf_decode.restype = C.c_int
+    L.pf_decode.argtypes = [vp, u64, C.POINTER(PfTuple)]
+    L.pf_score_workspace.restype = sz
+    L.pf_score_workspace.argtypes = [vp, u64, u32]
+    L.pf_score.restype = C.c_int
+    L.pf_score.argtypes = [vp, u64, u64, vp, vp, vp, u32, vp, vp, vp, vp, sz, vp]
+    L.pf_topk_merge.restype = C.c_int
+    L.pf_topk_merge.argtypes = [u32, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
+    L.pf_select_workspace.restype = sz
+    L.pf_select_workspace.argtypes = [vp, u64, u64]
+    L.pf_select_survivors.restype = C.c_int
+    L.pf_select_survivors.argtypes = [vp, u64, u64, vp, vp, u64, vp, vp, vp, sz, vp]
+    L.pf_simulate_workspace.restype = sz
+    L.pf_simulate_workspace.argtypes = [vp, u64, u32]
+    L.pf_simulate.restype = C.c_int
+    L.pf_simulate.argtypes = [vp, vp, u64, vp, u32, vp, vp, u32, vp, vp, vp, vp, sz, vp]
+    L.pf_search_workspace.restype = sz
+    L.pf_search_workspace.argtypes = [vp, u32, u64, u32]
+    L.pf_search_host.restype = C.c_int
+    L.pf_search_host.argtypes = [vp, u32, u64, u32, u32, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    L.pf_launch_count.restype = u64
+    L.pf_dualpipe_order.restype = C.c_int
+    L.pf_dualpipe_order.argtypes = [C.c_int, C.c_int, vp]
+    if path == LIB_PATH:
+        _lib = L
+    return L
+
+
+def _check(status: int, what: str):
+    if status != PF_OK:
+        L = load_library()
+        msg = L.pf_strerror(status).decode()
+        if status == PF_ECUDA:
+            msg += " (" + L.pf_last_cuda_error().decode() + ")"
+        raise PlanfrontError(status, f"{what}: {msg}")
+
+
+def pf_version() -> int:
+    return int(load_library().pf_version())
+
+
+def pf_strerror(status: int) -> str:
+    return load_library().pf_strerror(status).decode()
+
+
+def pf_reason_str(reason: int) -> str:
+    return load_library().pf_reason_str(reason).decode()
+
+
+def pf_launch_count() -> int:
+    return int(load_library().pf_launch_count())
+
+
+def pf_dualpipe_order(pp: int, m: int):
+    """Host helper, needs no GPU: per-rank op order as lists of (position, microbatch, direction, is_backward)."""
+    out = np.zeros(pp * 2 * m, dtype=np.uint8)
+    _check(load_library().pf_dualpipe_order(pp, m, out.ctypes.data_as(C.c_void_p)), "pf_dualpipe_order")
+    res = []
+    for r in range(pp):
+        ops = out[r * 2 * m:(r + 1) * 2 * m]
+        res.append([((pp - 1 - r) if (int(o) >> 1) & 1 else r, int(o) >> 2, (int(o) >> 1) & 1, int(o) & 1)
+                    for o in ops])
+    return res
+
+
+def _torch():
+    import torch
+    if not torch.cuda.is_available():
+        raise PlanfrontError(PF_ECUDA, "no CUDA device: the plan-scoring path has no CPU fallback")
+    return torch
+
+
+def _dptr(t):
+    return C.c_void_p(t.data_ptr()) if t is not None else None
+
+
+def _stream_ptr(torch, stream=None):
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return C.c_void_p(s.cuda_stream)
+
+
+class Plan:
+    """A plan space on the current CUDA device (pf_plan_create / pf_plan_destroy)."""
+
+    def __init__(self, cfg: dict):
+        torch = _torch()
+        self._L = load_library()
+        self.cfg = cfg
+        self._keep = []
+        m = PfModel(**{n: int(cfg["model"][n]) for n, _ in PfModel._fields_})
+        c = cfg["cluster"]
+        cl = PfCluster(G=int(c["G"]), caps=int(c["caps"]), budget_bytes=int(c["budget_bytes"]),
+                       reserved_bytes=int(c["reserved_bytes"]),
+                       **{n: float(c[n]) for n in ("peak_flops", "hbm_bw", "bw_intra", "bw_inter", "alpha_intra",
+                                                   "alpha_inter")})
+        w = cfg["workload"]
+        sp = np.asarray(w.get("scen_P", []), dtype=np.int32)
+        so = np.asarray(w.get("scen_O", []), dtype=np.int32)
+        self._keep += [sp, so]
+        wl = PfWorkload(phase=int(cfg["phase"]), n_scen=len(sp), gbs=int(w.get("gbs", 0)), world=int(w.get("world", 0)),
+                        scen_P=sp.ctypes.data_as(C.POINTER(i32)), scen_O=so.ctypes.data_as(C.POINTER(i32)))
+        ax = PfAxes()
+        ax.n_axes = len(cfg["axes"])
+        for a, (_, vals) in enumerate(cfg["axes"]):
+            arr = np.asarray(vals, dtype=np.int32)
+            self._keep.append(arr)
+            ax.len[a] = len(arr)
+            ax.val[a] = arr.ctypes.data_as(C.POINTER(i32))
+        tb = PfTables(**{n: float(cfg["consts"][n]) for n in ("eff_dense", "bwd_factor", "dp_overlap_frac",
+                                                               "dualpipe_startup_div", "step_overhead")})
+        tb.n_sched = len(cfg["sched"])
+        for i, s in enumerate(cfg["sched"]):
+            tb.sched[i] = PfSched(kind=int(s["kind"]), overlap=int(s["overlap"]), mapped=int(s["mapped"]),
+                                  hide_frac=float(s["hide_frac"]), sched_ovh=float(s["sched_ovh"]))
+        tb.n_kern = len(cfg["kern"])
+        for i, k in enumerate(cfg["kern"]):
+            kk = PfKern(needs_caps=int(k["needs_caps"]), avail_mask=int(k["avail_mask"]), is_native=int(k["is_native"]),
+                        wbytes=int(k["wbytes"]), dtype_mult=float(k["dtype_mult"]), patch_ovh=float(k["patch_ovh"]))
+            for b in range(NBUCKET):
+                kk.eff[b] = float(k["eff"][b])
+            tb.kern[i] = kk
+        ru = PfRules(**{n: int(cfg["rules"][n]) for n, _ in PfRules._fields_})
+        h = C.c_void_p()
+        _check(self._L.pf_plan_create(C.byref(m), C.byref(cl), C.byref(wl), C.byref(ax), C.byref(tb), C.byref(ru),
+                                      C.byref(h)), "pf_plan_create")
+        self._h = h
+        self.size = int(self._L.pf_plan_size(h))
+        self.device = torch.device("cuda", torch.cuda.current_device())
+
+    def close(self):
+        if getattr(self, "_h", None):
+            self._L.pf_plan_destroy(self._h)
+            self._h = None
+
+    def __del__(self):  # pragma: no cover
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # ---- pf_decode
+    def decode(self, idx: int) -> dict:
+        t = PfTuple()
+        _check(self._L.pf_decode(self._h, idx, C.byref(t)), "pf_decode")
+        return {n: getattr(t, n) for n, _ in PfTuple._fields_}
+
+    # ---- pf_score
+    def score_workspace(self, count: int, k: int) -> int:
+        return int(self._L.pf_score_workspace(self._h, count, k))
+
+    def score(self, first: int = 0, count: int | None = None, k: int = 0, reason=None, tput=None, mem=None,
+              topk_idx=None, topk_score=None, topk_count=None, workspace=None, stream=None, dense: bool = True):
+        """Enqueue pf_score.  Missing output tensors are allocated here (dense ones only if dense=True);
+        returns a dict of the tensors used.  Does not synchronize."""
+        torch = _torch()
+        if count is None:
+            count = self.size - first
+        dev = self.device
+        if dense:
+            reason = torch.empty(count, dtype=torch.uint8, device=dev) if reason is None else reason
+            tput = torch.empty(count, dtype=torch.float32, device=dev) if tput is None else tput
+            mem = torch.empty(count, dtype=torch.int64, device=dev) if mem is None else mem
+        if k > 0:
+            topk_idx = torch.empty(k, dtype=torch.int64, device=dev) if topk_idx is None else topk_idx
+            topk_score = torch.empty(k, dtype=torch.float32, device=dev) if topk_score is None else topk_score
+            topk_count = torch.empty(1, dtype=torch.int32, device=dev) if topk_count is None else topk_count
+        if workspace is None:
+            workspace = torch.empty(self.score_workspace(count, k), dtype=torch.uint8, device=dev)
+        _check(self._L.pf_score(self._h, first, count, _dptr(reason), _dptr(tput), _dptr(mem), k, _dptr(topk_idx),
+                                _dptr(topk_score), _dptr(topk_count), _dptr(workspace), workspace.numel(),
+                                _stream_ptr(torch, stream)), "pf_score")
+        return dict(reason=reason, tput=tput, mem=mem, topk_idx=topk_idx, topk_score=topk_score,
+                    topk_count=topk_count, workspace=workspace)
+
+    # ---- pf_select_survivors
+    def select_workspace(self, count: int, s_max: int) -> int:
+        return int(self._L.pf_select_workspace(self._h, count, s_max))
+
+    def select_survivors(self, reason, tput, s_max: int, first: int = 0, surv_idx=None, surv_count=None,
+                         workspace=None, stream=None):
+        torch = _torch()
+        count = reason.numel()
+        dev = self.device
+        surv_idx = torch.empty(max(s_max, 1), dtype=torch.int64, device=dev) if surv_idx is None else surv_idx
+        surv_count = torch.empty(1, dtype=torch.int64, device=dev) if surv_count is None else surv_count
+        if workspace is None:
+            workspace = torch.empty(self.select_workspace(count, s_max), dtype=torch.uint8, device=dev)
+        _check(self._L.pf_select_survivors(self._h, first, count, _dptr(reason), _dptr(tput), s_max, _dptr(surv_idx),
+                                           _dptr(surv_count), _dptr(workspace), workspace.numel(),
+                                           _stream_ptr(torch, stream)), "pf_select_survivors")
+        return dict(surv_idx=surv_idx, surv_count=surv_count, workspace=workspace)
+
+    # ---- pf_simulate
+    def simulate_workspace(self, n: int, k: int) -> int:
+        return int(self._L.pf_simulate_workspace(self._h, n, k))
+
+    def simulate(self, surv_idx, n: int, jitter_seed: int, k: int = 0, d_n=None, tput_sim=None, sim_status=None,
+                 topk_idx=None, topk_score=None, topk_count=None, workspace=None, stream=None, dense: bool = True):
+        torch = _torch()
+        dev = self.device
+        if dense:
+            tput_sim = torch.empty(max(n, 1), dtype=torch.float32, device=dev) if tput_sim is None else tput_sim
+            sim_status = torch.empty(max(n, 1), dtype=torch.uint8, device=dev) if sim_status is None else sim_status
+        if k > 0:
+            topk_idx = torch.empty(k, dtype=torch.int64, device=dev) if topk_idx is None else topk_idx
+            topk_score = torch.empty(k, dtype=torch.float32, device=dev) if topk_score is None else topk_score
+            topk_count = torch.empty(1, dtype=torch.int32, device=dev) if topk_count is None else topk_count
+        if workspace is None:
+            workspace = torch.empty(self.simulate_workspace(n, k), dtype=torch.uint8, device=dev)
+        _check(self._L.pf_simulate(self._h, _dptr(surv_idx), n, _dptr(d_n), jitter_seed, _dptr(tput_sim),
+                                   _dptr(sim_status), k, _dptr(topk_idx), _dptr(topk_score), _dptr(topk_count),
+                                   _dptr(workspace), workspace.numel(), _stream_ptr(torch, stream)), "pf_simulate")
+        return dict(tput_sim=tput_sim, sim_status=sim_status, topk_idx=topk_idx, topk_score=topk_score,
+                    topk_count=topk_count, workspace=workspace)
+
+    # ---- pf_search_host
+    def search_workspace(self, k: int, s_max: int, k_sim: int) -> int:
+        return int(self._L.pf_search_workspace(self._h, k, s_max, k_sim))
+
+    def search_host(self, k: int, s_max: int, k_sim: int, jitter_seed: int, workspace, h_reason=None, h_tput=None,
+                    h_mem=None, stream=None):
+        """pf_search_host with numpy / pinned-torch HOST buffers for the dense outputs (each may be None).
+        Returns a dict of numpy results; synchronous."""
+        torch = _torch()
+
+        def hptr(x):
+            if x is None:
+                return None
+            return C.c_void_p(x.data_ptr()) if hasattr(x, "data_ptr") else x.ctypes.data_as(C.c_void_p)
+        ti = np.empty(max(k, 1), dtype=np.uint64)
+        ts = np.empty(max(k, 1), dtype=np.float32)
+        tc = np.zeros(1, dtype=np.uint32)
+        si = np.empty(max(k_sim, 1), dtype=np.uint64)
+        ss = np.empty(max(k_sim, 1), dtype=np.float32)
+        sc = np.zeros(1, dtype=np.uint32)
+        nsurv = np.zeros(1, dtype=np.uint64)
+        _check(self._L.pf_search_host(self._h, k, s_max, k_sim, jitter_seed, hptr(h_reason), hptr(h_tput), hptr(h_mem),
+                                      hptr(ti), hptr(ts), hptr(tc), hptr(si), hptr(ss), hptr(sc), hptr(nsurv),
+                                      _dptr(workspace), workspace.numel(), _stream_ptr(torch, stream)),
+               "pf_search_host")
+        return dict(topk_idx=ti[:tc[0]], topk_score=ts[:tc[0]], sim_topk_idx=si[:sc[0]], sim_topk_score=ss[:sc[0]],
+                    n_survivors=int(nsurv[0]))
+
+
+def pf_topk_merge(k: int, idx_a, score_a, count_a, idx_b, score_b, count_b, stream=None):
+    """Merge two device top-k lists; returns (idx, score, count) device tensors."""
+    torch = _torch()
+    dev = idx_a.device
+    oi = torch.empty(k, dtype=torch.int64, device=dev)
+    os_ = torch.empty(k, dtype=torch.float32, device=dev)
+    oc = torch.empty(1, dtype=torch.int32, device=dev)
+    _check(load_library().pf_topk_merge(k, _dptr(idx_a), _dptr(score_a), _dptr(count_a), _dptr(idx_b), _dptr(score_b),
+                                        _dptr(count_b), _dptr(oi), _dptr(os_), _dptr(oc), _stream_ptr(torch, stream)),
+           "pf_topk_merge")
+    return oi, os_, oc

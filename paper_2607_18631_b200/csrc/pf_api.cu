@@ -1,0 +1,356 @@
+// pf_api.cu -- handle life cycle, validation, host-side derivation of the candidate-independent constants,
+// status strings.  Host code only.
+#include <atomic>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+
+#include "pf_internal.cuh"
+
+namespace pf {
+
+static thread_local char g_cuda_msg[256] = "";
+static std::atomic<uint64_t> g_launches{0};
+
+void set_cuda_error(cudaError_t e, const char *where)
+{
+    snprintf(g_cuda_msg, sizeof(g_cuda_msg), "%s: %s", where, cudaGetErrorString(e));
+}
+void count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
+
+}  // namespace pf
+
+using pf::DevPlan;
+
+namespace pf {
+int build_sim_tables(pf_plan_t *p);  // pf_simulate.cu: schedule-order tables for the simulator
+void free_sim_tables(pf_plan_t *p);
+}
+
+extern "C" int pf_version(void) { return PF_VERSION; }
+
+extern "C" const char *pf_last_cuda_error(void) { return pf::g_cuda_msg; }
+
+extern "C" uint64_t pf_launch_count(void) { return pf::g_launches.load(); }
+
+extern "C" const char *pf_strerror(int status)
+{
+    switch (status) {
+    case PF_OK: return "ok";
+    case PF_EINVAL: return "invalid argument";
+    case PF_ERANGE: return "value out of range";
+    case PF_EWORKSPACE: return "workspace too small or misaligned";
+    case PF_ECUDA: return "CUDA error";
+    case PF_EUNSUPPORTED: return "not supported for this plan";
+    default: return "unknown status";
+    }
+}
+
+extern "C" const char *pf_reason_str(uint8_t reason)
+{
+    switch (reason & 0x7f) {
+    case PF_FEASIBLE: return (reason & PF_FLAG_EXTRAPOLATED) ? "feasible (extrapolated)" : "feasible";
+    case PF_R_WORLD: return "world size does not match the parallel degrees";
+    case PF_R_TP: return "tensor-parallel degree not admissible";
+    case PF_R_EP: return "expert-parallel degree not admissible";
+    case PF_R_BATCH: return "global batch not divisible by dp * microbatch";
+    case PF_R_VSTAGE: return "virtual-stage count does not fit the schedule class";
+    case PF_R_LAYERS: return "layer count does not divide the pipeline depth";
+    case PF_R_MICROBATCH: return "microbatch count does not fit the schedule order";
+    case PF_R_KERNEL_MISSING: return "kernel variant missing for this expert shape or hardware";
+    case PF_R_UNMAPPED_SCHEDULE: return "schedule class has no realization in the toolchain";
+    case PF_R_OVERLAP_PRECOND: return "overlap precondition violated";
+    case PF_R_MEMORY: return "memory_infeasible";
+    default: return "unknown reason";
+    }
+}
+
+// Per-layer parameter, activation and FLOP counts (exact int64 on the host).
+static void derive_model(const pf_model_t &m, DevPlan &d)
+{
+    const long long H = m.H, nh = m.nh, nkv = m.nkv, hd = m.hd, ab = m.ab;
+    const long long lat = m.kv_latent, rope = m.rope_dim;
+    const bool mla = m.attn_kind != 0;
+    d.dk = mla ? (int)(lat + rope) : m.hd;
+    const long long q_proj = H * nh * hd, o_proj = nh * hd * H;
+    if (!mla)
+        d.P_attn = q_proj + 2 * H * nkv * hd + o_proj;
+    else
+        d.P_attn = q_proj + H * (lat + rope) + lat * nh * 2 * hd + o_proj;
+    d.P_rt = H * (long long)m.E;
+    d.P_e = (long long)m.n_mats * H * m.F;
+    d.P_sh = (long long)m.S * m.n_mats * H * m.Fs;
+    d.P_dl = d.P_attn + d.P_sh;
+    d.P_emb = m.count_embeddings ? (long long)m.vocab * H : 0;
+
+    const long long qkv = mla ? nh * hd + lat + rope + 2 * nh * hd : (nh + 2 * nkv) * hd;
+    const long long a_attn = ab * (2 * H + qkv + nh * hd);
+    const long long a_fix = ab * 2 * H + 4ll * m.E + ab * m.K * H + ab * H;
+    const long long a_ffn = ab * 3 * ((long long)m.K * m.F + (long long)m.S * m.Fs);
+    d.a_full = a_attn + a_fix + a_ffn;
+    d.a_sel = a_attn + a_fix;
+    d.a_ckpt = ab * H;
+
+    const long long f_attn = 2 * d.P_attn + 2ll * m.seq * nh * d.dk;
+    const long long f_rt = 2 * H * (long long)m.E;
+    const long long f_sh = 2 * d.P_sh;
+    d.f_dense = (float)(f_attn + f_rt + f_sh);
+    d.f_exp = (float)(2ll * m.K * d.P_e);
+    d.f_head = (float)(2ll * m.vocab * H);
+    d.f_sh = (float)f_sh;
+}
+
+static bool positive(std::initializer_list<long long> xs)
+{
+    for (long long x : xs)
+        if (x <= 0) return false;
+    return true;
+}
+
+extern "C" int pf_plan_create(const pf_model_t *model, const pf_cluster_t *cluster, const pf_workload_t *workload,
+                              const pf_axes_t *axes, const pf_tables_t *tables, const pf_rules_t *rules,
+                              pf_plan_t **out)
+{
+    if (!model || !cluster || !workload || !axes || !tables || !rules || !out) return PF_EINVAL;
+    *out = nullptr;
+    const int phase = workload->phase;
+    if (phase != PF_PHASE_TRAIN && phase != PF_PHASE_SERVE) return PF_EINVAL;
+    const int want_axes = phase == PF_PHASE_TRAIN ? 10 : 7;
+    if (axes->n_axes != want_axes) return PF_EINVAL;
+    if (tables->n_sched < 1 || tables->n_sched > PF_MAX_SCHED || tables->n_kern < 1 || tables->n_kern > PF_MAX_KERN)
+        return PF_EINVAL;
+    const pf_model_t &M = *model;
+    if (!positive({M.L, M.H, M.nh, M.hd, M.E, M.K, M.F, M.seq, M.vocab, M.wb, M.gb, M.ob, M.ab, M.n_mats}))
+        return PF_EINVAL;
+    if (M.S < 0 || (M.S > 0 && M.Fs <= 0) || M.K > M.E) return PF_EINVAL;
+    if (M.attn_kind == 0 ? M.nkv <= 0 : (M.kv_latent <= 0 || M.rope_dim < 0)) return PF_EINVAL;
+    if (cluster->G <= 0 || cluster->budget_bytes < 0 || cluster->reserved_bytes < 0) return PF_EINVAL;
+    if (!(cluster->peak_flops > 0) || !(cluster->hbm_bw > 0) || !(cluster->bw_intra > 0) || !(cluster->bw_inter > 0))
+        return PF_EINVAL;
+    if (!(tables->eff_dense > 0) || !(tables->dualpipe_startup_div > 0)) return PF_EINVAL;
+    if (phase == PF_PHASE_TRAIN && workload->gbs <= 0) return PF_EINVAL;
+    if (phase == PF_PHASE_SERVE) {
+        if (workload->world <= 0 || workload->n_scen < 1 || workload->n_scen > PF_MAX_SCEN) return PF_EINVAL;
+        if (!workload->scen_P || !workload->scen_O) return PF_EINVAL;
+        for (int i = 0; i < workload->n_scen; i++)
+            if (workload->scen_P[i] < 1 || workload->scen_O[i] < 1) return PF_ERANGE;
+    }
+
+    // axes: lengths, packed values, space size
+    int total_vals = 0;
+    uint64_t N = 1;
+    for (int a = 0; a < want_axes; a++) {
+        int len = axes->len[a];
+        if (len < 1 || len > PF_MAX_AXIS_LEN) return PF_ERANGE;
+        if (!axes->val[a]) return PF_EINVAL;
+        if (N > (UINT64_MAX >> 1) / (uint64_t)len) return PF_ERANGE;  // keep N < 2^63
+        N *= (uint64_t)len;
+        total_vals += len;
+    }
+    // value ranges per axis
+    auto in_range = [&](int a, long long lo, long long hi) {
+        for (int i = 0; i < axes->len[a]; i++)
+            if (axes->val[a][i] < lo || axes->val[a][i] > hi) return false;
+        return true;
+    };
+    const long long kDeg = 1 << 20;  // largest parallel degree / world size the integer paths are sized for
+    bool dp_derived = false, world_derived = false;
+    if (phase == PF_PHASE_TRAIN) {
+        if (!in_range(0, 0, tables->n_kern - 1) || !in_range(1, 0, 2) || !in_range(2, 0, tables->n_sched - 1))
+            return PF_EINVAL;
+        if (!in_range(3, 1, 1 << 16) || !in_range(4, 0, 255)) return PF_ERANGE;
+        if (!in_range(5, 1, kDeg) || !in_range(6, 1, kDeg) || !in_range(7, 1, kDeg)) return PF_ERANGE;
+        if (!in_range(8, 0, kDeg) || !in_range(9, 0, kDeg)) return PF_ERANGE;
+        // "derived" is a whole-axis statement: the list {0}
+        for (int a = 8; a <= 9; a++) {
+            bool has0 = false;
+            for (int i = 0; i < axes->len[a]; i++) has0 |= axes->val[a][i] == 0;
+            if (has0 && axes->len[a] != 1) return PF_EINVAL;
+            (a == 8 ? dp_derived : world_derived) = has0;
+        }
+        if (dp_derived && world_derived) return PF_EINVAL;
+        {
+            bool has0 = false;
+            for (int i = 0; i < axes->len[4]; i++) has0 |= axes->val[4][i] == 0;
+            if (has0 && axes->len[4] != 1) return PF_EINVAL;
+        }
+        for (int s = 0; s < tables->n_sched; s++)
+            if (tables->sched[s].kind < 0 || tables->sched[s].kind > 2) return PF_EINVAL;
+    } else {
+        if (!in_range(0, 0, tables->n_kern - 1)) return PF_EINVAL;
+        if (!in_range(1, 1, 1 << 20) || !in_range(2, 1, 1 << 20) || !in_range(3, 0, 1)) return PF_ERANGE;
+        if (!in_range(4, 1, kDeg) || !in_range(5, 1, kDeg)) return PF_ERANGE;
+        if (!in_range(6, 0, workload->n_scen - 1)) return PF_EINVAL;
+    }
+    for (int i = 0; i < tables->n_kern; i++) {
+        const pf_kern_t &k = tables->kern[i];
+        if (!(k.dtype_mult > 0) || k.wbytes < 1) return PF_EINVAL;
+        for (int b = 0; b < PF_NBUCKET; b++)
+            if (!(k.eff[b] > 0)) return PF_EINVAL;
+    }
+
+    pf_plan_t *p = new (std::nothrow) pf_plan_t;
+    if (!p) return PF_EINVAL;
+    memset(p, 0, sizeof(*p));
+    DevPlan &d = p->dev;
+    p->size = N;
+    d.phase = phase;
+    d.n_axes = want_axes;
+
+    // packed values
+    p->h_vals = (int32_t *)malloc(sizeof(int32_t) * (size_t)total_vals);
+    int off = 0;
+    for (int a = 0; a < want_axes; a++) {
+        p->axis_len[a] = axes->len[a];
+        d.radix[a] = (uint32_t)axes->len[a];
+        d.val_off[a] = off;
+        memcpy(p->h_vals + off, axes->val[a], sizeof(int32_t) * (size_t)axes->len[a]);
+        off += axes->len[a];
+    }
+
+    // slab = longest axis prefix whose product stays under a size that still leaves a few blocks per SM
+    cudaDeviceProp prop;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess) {
+        pf::set_cuda_error(cudaGetLastError(), "pf_plan_create: device query");
+        free(p->h_vals);
+        delete p;
+        return PF_ECUDA;
+    }
+    p->device = dev;
+    p->sm_count = prop.multiProcessorCount;
+    uint64_t target = N / (uint64_t)(4 * p->sm_count);
+    if (target < 256) target = 256;
+    if (target > pf::kSlabMax) target = pf::kSlabMax;
+    uint64_t slab = 1;
+    int n_inner = 0;
+    while (n_inner < want_axes && slab * d.radix[n_inner] <= target) {
+        slab *= d.radix[n_inner];
+        n_inner++;
+    }
+    d.n_inner = n_inner;
+    d.slab = (uint32_t)slab;
+    for (int a = 0; a < want_axes; a++) {
+        // ceil(2^32 / r): exact quotient by multiply-high for n < 2^32 / r, and n <= slab * ... <= 2^14
+        d.magic[a] = d.radix[a] == 1 ? 0u : (uint32_t)(((1ull << 32) + d.radix[a] - 1) / d.radix[a]);
+    }
+    // leading rules whose axes are all outer (train: R1 tp,pp,dp,world; R2 tp; R3 ep,dp,tp; R4 dp,mb;
+    // serve: R1 tp,dpa,ep; R2 tp; R3 ep,tp,dpa; R4 dpa,batch,ep)
+    if (phase == PF_PHASE_TRAIN)
+        d.n_pre_rules = n_inner <= 3 ? 4 : n_inner <= 5 ? 3 : n_inner <= 6 ? 2 : 0;
+    else
+        d.n_pre_rules = n_inner <= 2 ? 4 : n_inner <= 3 ? 3 : 0;
+
+    // model, cluster, workload, tables
+    d.L = M.L; d.H = M.H; d.nh = M.nh; d.nkv = M.nkv; d.hd = M.hd; d.attn_kind = M.attn_kind;
+    d.kv_latent = M.kv_latent; d.rope_dim = M.rope_dim; d.E = M.E; d.K = M.K; d.F = M.F; d.S = M.S; d.Fs = M.Fs;
+    d.seq = M.seq; d.vocab = M.vocab; d.wb = M.wb; d.gb = M.gb; d.ob = M.ob; d.ab = M.ab;
+    d.count_embeddings = M.count_embeddings ? 1 : 0;
+    derive_model(M, d);
+    d.G = cluster->G; d.caps = cluster->caps;
+    d.budget_bytes = cluster->budget_bytes; d.reserved_bytes = cluster->reserved_bytes;
+    d.peak_flops = cluster->peak_flops; d.hbm_bw = cluster->hbm_bw;
+    d.bw_intra = cluster->bw_intra; d.bw_inter = cluster->bw_inter;
+    d.alpha_intra = cluster->alpha_intra; d.alpha_inter = cluster->alpha_inter;
+    d.gbs = workload->gbs; d.world = workload->world; d.n_scen = phase == PF_PHASE_SERVE ? workload->n_scen : 0;
+    d.eff_dense = tables->eff_dense; d.bwd_factor = tables->bwd_factor; d.dp_overlap_frac = tables->dp_overlap_frac;
+    d.dualpipe_startup_div = tables->dualpipe_startup_div; d.step_overhead = tables->step_overhead;
+    d.ep_scope = rules->ep_scope ? 1 : 0; d.layer_mode = rules->layer_mode; d.tp_max = rules->tp_max;
+    d.world_min = rules->world_min; d.world_max = rules->world_max;
+    d.enforce = rules->enforce_realizability ? 1 : 0;
+    d.n_sched = tables->n_sched; d.n_kern = tables->n_kern;
+    for (int s = 0; s < tables->n_sched; s++) {
+        d.sched[s].kind = tables->sched[s].kind; d.sched[s].overlap = tables->sched[s].overlap ? 1 : 0;
+        d.sched[s].mapped = tables->sched[s].mapped ? 1 : 0;
+        d.sched[s].hide_frac = tables->sched[s].hide_frac; d.sched[s].sched_ovh = tables->sched[s].sched_ovh;
+    }
+    for (int i = 0; i < tables->n_kern; i++) {
+        const pf_kern_t &k = tables->kern[i];
+        d.kern[i].needs_caps = k.needs_caps; d.kern[i].avail_mask = k.avail_mask;
+        d.kern[i].is_native = k.is_native ? 1 : 0; d.kern[i].wbytes = k.wbytes;
+        d.kern[i].dtype_mult = k.dtype_mult; d.kern[i].patch_ovh = k.patch_ovh;
+        for (int b = 0; b < PF_NBUCKET; b++) d.kern[i].eff[b] = k.eff[b];
+    }
+
+    // can the rule arithmetic stay in 32 bits?  (largest products the rules form)
+    auto axis_max = [&](int a) {
+        long long m = 0;
+        for (int i = 0; i < axes->len[a]; i++) m = axes->val[a][i] > m ? axes->val[a][i] : m;
+        return m;
+    };
+    const long long lim = (1ll << 31) - 1;
+    bool wide = false;
+    if (phase == PF_PHASE_TRAIN) {
+        long long mb = axis_max(3), ep = axis_max(5), pp = axis_max(6), tp = axis_max(7);
+        long long dp = dp_derived ? axis_max(9) : axis_max(8);
+        long long world = world_derived ? tp * pp * dp : axis_max(9);
+        wide |= tp * pp > lim || tp * pp * dp > lim || world > lim || dp * tp > lim || dp * mb > lim;
+        wide |= workload->gbs > lim || mb * M.seq > lim || mb * M.seq * M.K > lim / (ep > 0 ? ep : 1);
+        wide |= (long long)M.E * tp > lim || pp * 256 > lim;
+    } else {
+        long long C = axis_max(1), B = axis_max(2), ep = axis_max(4), tp = axis_max(5);
+        wide |= tp * ep > lim || B * M.K > lim || C * M.K > lim || workload->world > lim;
+    }
+    d.wide = wide ? 1 : 0;
+
+    // device copies
+    cudaError_t e = cudaMalloc((void **)&p->d_vals, sizeof(int32_t) * (size_t)total_vals);
+    if (e == cudaSuccess)
+        e = cudaMemcpy(p->d_vals, p->h_vals, sizeof(int32_t) * (size_t)total_vals, cudaMemcpyHostToDevice);
+    if (e == cudaSuccess && phase == PF_PHASE_SERVE) {
+        size_t n = (size_t)workload->n_scen;
+        e = cudaMalloc((void **)&p->d_scen, sizeof(int32_t) * 2 * n);
+        if (e == cudaSuccess) e = cudaMemcpy(p->d_scen, workload->scen_P, sizeof(int32_t) * n, cudaMemcpyHostToDevice);
+        if (e == cudaSuccess)
+            e = cudaMemcpy(p->d_scen + n, workload->scen_O, sizeof(int32_t) * n, cudaMemcpyHostToDevice);
+    }
+    if (e != cudaSuccess) {
+        pf::set_cuda_error(e, "pf_plan_create: upload");
+        pf_plan_destroy(p);
+        return PF_ECUDA;
+    }
+    if (phase == PF_PHASE_TRAIN) {
+        int rc = pf::build_sim_tables(p);
+        if (rc != PF_OK) {
+            pf_plan_destroy(p);
+            return rc;
+        }
+    }
+    *out = p;
+    return PF_OK;
+}
+
+extern "C" void pf_plan_destroy(pf_plan_t *p)
+{
+    if (!p) return;
+    pf::free_sim_tables(p);
+    if (p->d_vals) cudaFree(p->d_vals);
+    if (p->d_scen) cudaFree(p->d_scen);
+    free(p->h_vals);
+    delete p;
+}
+
+extern "C" uint64_t pf_plan_size(const pf_plan_t *p) { return p ? p->size : 0; }
+
+extern "C" int pf_decode(const pf_plan_t *p, uint64_t idx, pf_tuple_t *out)
+{
+    if (!p || !out) return PF_EINVAL;
+    if (idx >= p->size) return PF_ERANGE;
+    int32_t v[PF_MAX_AXES] = {0};
+    uint64_t rem = idx;
+    for (int a = 0; a < p->dev.n_axes; a++) {
+        uint64_t r = p->dev.radix[a];
+        v[a] = p->h_vals[p->dev.val_off[a] + (int)(rem % r)];
+        rem /= r;
+    }
+    memset(out, 0, sizeof(*out));
+    if (p->dev.phase == PF_PHASE_TRAIN) {
+        out->kv = v[0]; out->rec = v[1]; out->sched = v[2]; out->mb = v[3]; out->v = v[4];
+        out->ep = v[5]; out->pp = v[6]; out->tp = v[7]; out->dp = v[8]; out->world = v[9];
+    } else {
+        out->kv = v[0]; out->chunk = v[1]; out->batch = v[2]; out->dpa = v[3];
+        out->ep = v[4]; out->tp = v[5]; out->scen = v[6];
+    }
+    return PF_OK;
+}

@@ -1,0 +1,195 @@
+// pf_internal.cuh -- device-side plan description, handle layout and block top-k utilities shared by the
+// translation units of libplanfront.so.  Nothing here is part of the public ABI.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "planfront.h"
+
+namespace pf {
+
+constexpr int kThreads = 256;        // threads per block of the scoring kernel
+constexpr int kTopkCap = 2048;       // shared-memory candidate buffer per block (2 * PF_K_MAX)
+constexpr int kMergeGroup = 32;      // lists merged per block in one merge pass
+constexpr uint32_t kSlabMax = 16384; // upper bound on candidates per slab (inner-axis product)
+
+struct DevSched {
+    int kind, overlap, mapped;
+    float hide_frac, sched_ovh;
+};
+
+struct DevKern {
+    uint32_t needs_caps, avail_mask;
+    int is_native, wbytes;
+    float dtype_mult, patch_ovh;
+    float eff[PF_NBUCKET];
+};
+
+// Everything a kernel needs about the plan space except the axis value lists (global memory).
+// Passed by value as a __grid_constant__ kernel parameter, so uniform reads come from the constant bank.
+struct DevPlan {
+    // --- index space
+    int phase, n_axes;
+    int n_inner;          // axes [0, n_inner) vary inside a slab, the rest select the slab
+    int n_pre_rules;      // leading rules that depend on outer axes only (checked once per slab)
+    uint32_t slab;        // candidates per slab = product of inner radices (<= kSlabMax)
+    uint32_t radix[PF_MAX_AXES];
+    uint32_t magic[PF_MAX_AXES];   // ceil(2^32 / radix) for the inner axes: q = umulhi(n, magic)
+    int val_off[PF_MAX_AXES];      // offset of each axis' value list in the packed value array
+    int wide;                      // 1: rule arithmetic needs 64-bit integers
+    // --- model (Sec. 3.1) and host-derived per-layer constants
+    int L, H, nh, nkv, hd, attn_kind, kv_latent, rope_dim, E, K, F, S, Fs, seq, vocab;
+    int wb, gb, ob, ab, count_embeddings;
+    int dk;
+    long long P_attn, P_rt, P_e, P_sh, P_dl, P_emb;
+    long long a_full, a_sel, a_ckpt;
+    float f_dense, f_exp, f_head, f_sh;   // forward FLOPs per token (per layer; head once), rounded to fp32 once
+    // --- modeled cluster
+    int G;
+    uint32_t caps;
+    long long budget_bytes, reserved_bytes;
+    float peak_flops, hbm_bw, bw_intra, bw_inter, alpha_intra, alpha_inter;
+    // --- workload
+    long long gbs, world;
+    int n_scen;
+    // --- cost constants, rules, tables
+    float eff_dense, bwd_factor, dp_overlap_frac, dualpipe_startup_div, step_overhead;
+    int ep_scope, layer_mode, tp_max, world_min, world_max, enforce;
+    int n_sched, n_kern;
+    DevSched sched[PF_MAX_SCHED];
+    DevKern kern[PF_MAX_KERN];
+};
+
+}  // namespace pf
+
+// The opaque handle of the C ABI.
+struct pf_plan {
+    pf::DevPlan dev;
+    uint64_t size;                 // N
+    int device;
+    int sm_count;
+    // host copies
+    int32_t *h_vals;               // packed axis value lists
+    int32_t axis_len[PF_MAX_AXES];
+    // device buffers owned by the handle
+    int32_t *d_vals;               // packed axis value lists
+    int32_t *d_scen;               // serve: P[n_scen] then O[n_scen]
+    // simulator order tables (built lazily by the simulator unit)
+    void *sim_tables;
+};
+
+namespace pf {
+
+// ------------------------------------------------------------------ error plumbing (host)
+void set_cuda_error(cudaError_t e, const char *where);
+void count_launch();
+#define PF_CUDA_TRY(expr, where)                        \
+    do {                                                \
+        cudaError_t e__ = (expr);                       \
+        if (e__ != cudaSuccess) {                       \
+            pf::set_cuda_error(e__, where);             \
+            return PF_ECUDA;                            \
+        }                                               \
+    } while (0)
+
+// ------------------------------------------------------------------ keys
+// A ranked candidate is one 64-bit key: (fp32 score bits << 32) | (0xFFFFFFFF - rel), rel = position in
+// the call's range (< 2^32 - 1).  Scores are positive floats, so unsigned key order = (score descending,
+// index ascending) when sorted descending.  Key 0 = empty slot.
+__device__ __forceinline__ unsigned long long make_key(float score, uint32_t rel)
+{
+    return ((unsigned long long)__float_as_uint(score) << 32) | (unsigned long long)(0xFFFFFFFFu - rel);
+}
+__device__ __forceinline__ float key_score(unsigned long long key) { return __uint_as_float((uint32_t)(key >> 32)); }
+__device__ __forceinline__ uint32_t key_rel(unsigned long long key) { return 0xFFFFFFFFu - (uint32_t)key; }
+
+// ------------------------------------------------------------------ block top-k in shared memory
+// buf[kTopkCap] holds candidate keys, *count the number of valid ones, *thr the current admission
+// threshold (the k-th best key once k are held, else 0).  All functions are block-collective unless
+// noted; the block may have any multiple of 32 threads.
+
+// Descending bitonic sort of buf[0, kTopkCap) in shared memory.
+__device__ inline void tk_sort_desc(unsigned long long *buf)
+{
+    const int tid = threadIdx.x, nt = blockDim.x;
+    for (int size = 2; size <= kTopkCap; size <<= 1) {
+        for (int stride = size >> 1; stride > 0; stride >>= 1) {
+            __syncthreads();
+            for (int i = tid; i < kTopkCap / 2; i += nt) {
+                int lo = 2 * i - (i & (stride - 1));  // element with the stride bit clear
+                int hi = lo + stride;
+                bool desc = ((lo & size) == 0);       // direction of this bitonic block
+                unsigned long long a = buf[lo], b = buf[hi];
+                bool swap = desc ? (a < b) : (a > b);
+                if (swap) {
+                    buf[lo] = b;
+                    buf[hi] = a;
+                }
+            }
+        }
+    }
+    __syncthreads();
+}
+
+// Keep the best k: sort, clamp the count, refresh the threshold.
+__device__ inline void tk_prune(unsigned long long *buf, int *count, unsigned long long *thr, int k)
+{
+    __syncthreads();
+    int c = *count;
+    if (c > kTopkCap) c = kTopkCap;
+    for (int i = c + threadIdx.x; i < kTopkCap; i += blockDim.x) buf[i] = 0ull;
+    tk_sort_desc(buf);
+    if (threadIdx.x == 0) {
+        int n = c < k ? c : k;
+        *count = n;
+        *thr = (n == k) ? buf[k - 1] : 0ull;
+    }
+    __syncthreads();
+}
+
+// Append this thread's key if it beats the threshold.  Warp-collective (all 32 lanes must call); the
+// caller guarantees room for one key per thread of the block.
+__device__ __forceinline__ void tk_push(unsigned long long *buf, int *count, unsigned long long thr, bool has,
+                                        unsigned long long key)
+{
+    bool take = has && key > thr;
+    unsigned mask = __ballot_sync(0xFFFFFFFFu, take);
+    if (mask == 0) return;
+    int lane = threadIdx.x & 31;
+    int leader = __ffs(mask) - 1;
+    int base = 0;
+    if (lane == leader) base = atomicAdd(count, __popc(mask));
+    base = __shfl_sync(0xFFFFFFFFu, base, leader);
+    if (take) {
+        int pos = base + __popc(mask & ((1u << lane) - 1u));
+        if (pos < kTopkCap) buf[pos] = key;
+    }
+}
+
+// host: workspace layout of one top-k reduction with `nblocks` producers
+struct TopkLayout {
+    size_t off_ctrl, off_lists_a, off_lists_b, total;
+    int n_b;  // lists after the first merge pass
+};
+inline TopkLayout topk_layout(int nblocks, uint32_t k)
+{
+    TopkLayout l;
+    size_t kk = k ? k : 1;
+    l.off_ctrl = 0;
+    l.off_lists_a = 256;
+    size_t a = ((size_t)nblocks * kk * 8 + 255) & ~(size_t)255;
+    l.n_b = (nblocks + kMergeGroup - 1) / kMergeGroup;
+    size_t b = ((size_t)l.n_b * kk * 8 + 255) & ~(size_t)255;
+    l.off_lists_b = l.off_lists_a + a;
+    l.total = l.off_lists_b + b;
+    return l;
+}
+
+// host: merge `n_lists` per-block key lists (k keys each, zero padded) down to the final outputs.
+// idx_map (device, may be NULL): final index = idx_map[rel] instead of first + rel.
+int launch_topk_reduce(unsigned long long *d_lists_a, unsigned long long *d_lists_b, int n_lists, uint32_t k,
+                       uint64_t first, const uint64_t *d_idx_map, uint64_t *d_topk_idx, float *d_topk_score,
+                       uint32_t *d_topk_count, cudaStream_t st);
+
+}  // namespace pf

@@ -1,0 +1,449 @@
+// pf_score.cu -- the scoring kernel (decode -> rules -> memory -> cost -> price -> block top-k), the top-k
+// merge kernels, and their C entry points.
+//
+// Work decomposition.  The index space is cut into slabs: one slab = all combinations of the `n_inner`
+// fastest-varying axes (<= 16384 candidates) for one combination of the remaining (outer) axes.  A
+// persistent grid (a few blocks per SM) pulls slab numbers from an atomic counter.  For each slab one
+// thread decodes the outer digits and evaluates the leading rules that depend on outer axes only; when one
+// of them fails the whole slab has the same reason and the block just streams constant bytes into the
+// dense outputs with 16-byte stores.  Otherwise each thread takes candidates slab_base + j, decodes the
+// inner digits with multiply-high divisions and runs the remaining rules, the memory model and the cost
+// model in registers.  Feasible candidates are offered to a shared-memory top-k buffer; each block writes
+// its k best keys at the end and a small merge kernel reduces the per-block lists.
+#include "pf_eval.cuh"
+
+namespace pf {
+
+struct ScoreArgs {
+    uint64_t first, count;          // range of this call
+    uint64_t slab_lo;               // number of the first slab that intersects the range
+    uint32_t n_slabs;               // slabs intersecting the range
+    uint32_t k;
+    uint8_t *reason;
+    float *tput;
+    long long *mem;
+    unsigned long long *lists;      // [gridDim.x][k] keys, zero padded
+    unsigned int *slab_counter;     // zeroed before launch
+    const int32_t *vals;            // packed axis value lists
+    const int32_t *scen;            // serve: P[n_scen], O[n_scen]
+};
+
+struct SlabInfo {
+    uint32_t slab;                  // slab number relative to slab_lo, or 0xFFFFFFFF when the queue is empty
+    int pre_reason;                 // != 0: every candidate of the slab fails this rule
+    int outer[PF_MAX_AXES];         // values of the outer axes (entries [n_inner, n_axes))
+};
+
+// Fill n bytes at p with byte b using 16-byte streaming stores where alignment allows.  Block-collective.
+__device__ __forceinline__ void block_fill(uint8_t *p, uint64_t n, uint32_t b)
+{
+    const uint32_t tid = threadIdx.x, nt = blockDim.x;
+    uint64_t head = (16 - ((uintptr_t)p & 15)) & 15;
+    if (head > n) head = n;
+    for (uint64_t i = tid; i < head; i += nt) p[i] = (uint8_t)b;
+    const uint32_t w = b * 0x01010101u;
+    const uint4 v = make_uint4(w, w, w, w);
+    uint4 *q = reinterpret_cast<uint4 *>(p + head);
+    const uint64_t nv = (n - head) >> 4;
+    for (uint64_t i = tid; i < nv; i += nt) __stcs(q + i, v);
+    const uint64_t done = head + (nv << 4);
+    for (uint64_t i = done + tid; i < n; i += nt) p[i] = (uint8_t)b;
+}
+
+template <typename RI>
+__global__ void __launch_bounds__(kThreads) score_kernel(const __grid_constant__ DevPlan P, const ScoreArgs A)
+{
+    __shared__ unsigned long long s_buf[kTopkCap];
+    __shared__ int s_count;
+    __shared__ unsigned long long s_thr;
+    __shared__ SlabInfo s_slab;
+
+    const int tid = threadIdx.x;
+    const bool train = P.phase == PF_PHASE_TRAIN;
+    const bool want_topk = A.k > 0;
+    if (tid == 0) {
+        s_count = 0;
+        s_thr = 0ull;
+    }
+    // iterations that may still append without overflowing the buffer (one key per thread per iteration)
+    int room_iters = kTopkCap / kThreads;
+    unsigned long long thr = 0ull;
+
+    for (;;) {
+        __syncthreads();  // previous slab fully consumed before s_slab is overwritten
+        if (tid == 0) {
+            uint32_t s = atomicAdd(A.slab_counter, 1u);
+            SlabInfo si;
+            si.slab = s < A.n_slabs ? s : 0xFFFFFFFFu;
+            si.pre_reason = 0;
+            if (s < A.n_slabs) {
+                uint64_t o = A.slab_lo + s;
+                for (int a = P.n_inner; a < P.n_axes; a++) {
+                    uint64_t r = P.radix[a];
+                    uint64_t q = o / r;
+                    si.outer[a] = __ldg(A.vals + P.val_off[a] + (int)(o - q * r));
+                    o = q;
+                }
+                if (P.n_pre_rules > 0) {
+                    if (train) {
+                        TrainTuple c;
+                        c.mb = P.n_inner <= 3 ? si.outer[3] : 1;
+                        c.ep = P.n_inner <= 5 ? si.outer[5] : 1;
+                        c.pp = si.outer[6]; c.tp = si.outer[7]; c.dp = si.outer[8]; c.world = si.outer[9];
+                        RI dp, world;
+                        int r = train_layout_rules<RI>(P, c, 1, P.n_pre_rules < 3 ? P.n_pre_rules : 3, dp, world);
+                        if (r == 0 && P.n_pre_rules >= 4) {
+                            RI dpmb = dp * (RI)c.mb;
+                            if (((RI)P.gbs) % dpmb != 0) r = PF_R_BATCH;
+                        }
+                        si.pre_reason = r;
+                    } else {
+                        ServeTuple c;
+                        c.batch = P.n_inner <= 2 ? si.outer[2] : 1;
+                        c.dpa = si.outer[3]; c.ep = si.outer[4]; c.tp = si.outer[5];
+                        si.pre_reason = serve_layout_rules<RI>(P, c, 1, P.n_pre_rules >= 4);
+                    }
+                }
+            }
+            s_slab = si;
+        }
+        __syncthreads();
+        if (s_slab.slab == 0xFFFFFFFFu) break;
+
+        // candidate range of this slab clipped to the call's range
+        const uint64_t slab_no = A.slab_lo + s_slab.slab;
+        const uint64_t base = slab_no * (uint64_t)P.slab;
+        const uint64_t lo = base > A.first ? base : A.first;
+        const uint64_t end_slab = base + P.slab, end_call = A.first + A.count;
+        const uint64_t hi = end_slab < end_call ? end_slab : end_call;
+        const uint64_t rel0 = lo - A.first;  // offset of the first candidate in the dense outputs
+        const uint32_t n = (uint32_t)(hi - lo);
+
+        if (s_slab.pre_reason != 0) {
+            if (A.reason) block_fill(A.reason + rel0, n, (uint32_t)s_slab.pre_reason);
+            if (A.tput) block_fill(reinterpret_cast<uint8_t *>(A.tput + rel0), (uint64_t)n * 4, 0u);
+            if (A.mem) block_fill(reinterpret_cast<uint8_t *>(A.mem + rel0), (uint64_t)n * 8, 0u);
+            continue;
+        }
+
+        const uint32_t j0 = (uint32_t)(lo - base);
+        const int first_rule = P.n_pre_rules + 1;
+        for (uint32_t it = 0; it < n; it += kThreads) {
+            const uint32_t i = it + tid;
+            const bool active = i < n;
+            int reason = 0;
+            float tput = 0.f;
+            long long mem = 0;
+            if (active) {
+                // inner digits by multiply-high division (exact: j * radix < 2^32)
+                uint32_t rem = j0 + i;
+                int v[PF_MAX_AXES];
+#pragma unroll
+                for (int a = 0; a < PF_MAX_AXES; a++) {
+                    if (a < P.n_inner) {
+                        uint32_t r = P.radix[a];
+                        uint32_t q = r == 1u ? rem : __umulhi(rem, P.magic[a]);
+                        v[a] = __ldg(A.vals + P.val_off[a] + (int)(rem - q * r));
+                        rem = q;
+                    } else {
+                        v[a] = a < P.n_axes ? s_slab.outer[a] : 0;
+                    }
+                }
+                if (train) {
+                    TrainTuple c;
+                    c.kv = v[0]; c.rec = v[1]; c.s = v[2]; c.mb = v[3]; c.v = v[4];
+                    c.ep = v[5]; c.pp = v[6]; c.tp = v[7]; c.dp = v[8]; c.world = v[9];
+                    RI dp, world;
+                    reason = train_layout_rules<RI>(P, c, first_rule, 3, dp, world);
+                    if (reason == 0) {
+                        TrainDerived<RI> D;
+                        reason = train_plan_rules<RI>(P, c, dp, world, first_rule, D);
+                        if (reason == 0) {
+                            TrainMem M;
+                            train_memory<RI>(P, c, D, M);
+                            mem = M.mem;
+                            if (mem > P.budget_bytes) {
+                                reason = PF_R_MEMORY;
+                            } else {
+                                TrainTimes T;
+                                train_times<RI>(P, c, D, M, T);
+                                tput = train_price<RI>(P, c, D, T, train_pipe_analytic<RI>(P, c, D, T));
+                                if (D.m_e < (RI)64 || D.m_e > (RI)8192) reason = PF_FLAG_EXTRAPOLATED;
+                            }
+                        }
+                    }
+                } else {
+                    ServeTuple c;
+                    c.kv = v[0]; c.chunk = v[1]; c.batch = v[2]; c.dpa = v[3]; c.ep = v[4]; c.tp = v[5]; c.scen = v[6];
+                    ServeOut so;
+                    serve_eval<RI>(P, c, first_rule, __ldg(A.scen + c.scen), __ldg(A.scen + P.n_scen + c.scen), so);
+                    reason = so.reason;
+                    tput = so.tput;
+                    mem = so.mem;
+                }
+                const uint64_t o = rel0 + i;
+                if (A.reason) A.reason[o] = (uint8_t)reason;
+                if (A.tput) A.tput[o] = tput;
+                if (A.mem) A.mem[o] = mem;
+            }
+            if (want_topk) {
+                if (room_iters == 0) {
+                    __syncthreads();
+                    if (s_count > kTopkCap - kThreads) tk_prune(s_buf, &s_count, &s_thr, (int)A.k);
+                    room_iters = (kTopkCap - s_count) / kThreads;
+                    thr = s_thr;
+                    __syncthreads();
+                }
+                const bool feasible = active && (reason & 0x7f) == 0;
+                tk_push(s_buf, &s_count, thr, feasible, make_key(tput, (uint32_t)(rel0 + i)));
+                room_iters--;
+            }
+        }
+    }
+
+    if (want_topk) {
+        tk_prune(s_buf, &s_count, &s_thr, (int)A.k);
+        unsigned long long *out = A.lists + (size_t)blockIdx.x * A.k;
+        const int c = s_count;
+        for (int i = tid; i < (int)A.k; i += kThreads) out[i] = i < c ? s_buf[i] : 0ull;
+    }
+}
+
+// ------------------------------------------------------------------ merging per-block lists
+
+struct MergeArgs {
+    const unsigned long long *in;   // [n_lists][k]
+    unsigned long long *out;        // [gridDim.x][k] when not final
+    int n_lists;
+    uint32_t k;
+    int group;                      // lists per block
+    int final;                      // 1: write idx / score / count instead of keys (gridDim.x must be 1)
+    uint64_t first;
+    const uint64_t *idx_map;        // NULL: idx = first + rel; else idx = idx_map[rel]
+    uint64_t *topk_idx;
+    float *topk_score;
+    uint32_t *topk_count;
+};
+
+__global__ void __launch_bounds__(kThreads) merge_kernel(const MergeArgs A)
+{
+    __shared__ unsigned long long s_buf[kTopkCap];
+    __shared__ int s_count;
+    __shared__ unsigned long long s_thr;
+    const int tid = threadIdx.x, k = (int)A.k;
+    if (tid == 0) {
+        s_count = 0;
+        s_thr = 0ull;
+    }
+    __syncthreads();
+    const int l0 = blockIdx.x * A.group;
+    const int l1 = min(l0 + A.group, A.n_lists);
+    // each input list holds at most k keys; the buffer takes kTopkCap / k lists between prunes
+    const int per_round = max(1, (kTopkCap - k) / k);
+    for (int l = l0; l < l1; l += per_round) {
+        const int le = min(l + per_round, l1);
+        const int base = s_count;
+        const int total = (le - l) * k;
+        for (int i = tid; i < total; i += kThreads) {
+            unsigned long long key = A.in[(size_t)l * k + i];
+            s_buf[base + i] = key;  // zeros (empty slots) sort to the end
+        }
+        __syncthreads();
+        if (tid == 0) s_count = base + total;
+        tk_prune(s_buf, &s_count, &s_thr, k);
+        // drop trailing empties from the count
+        if (tid == 0) {
+            int c = s_count;
+            while (c > 0 && s_buf[c - 1] == 0ull) c--;
+            s_count = c;
+        }
+        __syncthreads();
+    }
+    const int c = s_count;
+    if (!A.final) {
+        unsigned long long *out = A.out + (size_t)blockIdx.x * k;
+        for (int i = tid; i < k; i += kThreads) out[i] = i < c ? s_buf[i] : 0ull;
+    } else {
+        for (int i = tid; i < k; i += kThreads) {
+            if (i < c) {
+                unsigned long long key = s_buf[i];
+                uint32_t rel = key_rel(key);
+                A.topk_idx[i] = A.idx_map ? A.idx_map[rel] : A.first + rel;
+                A.topk_score[i] = key_score(key);
+            } else {
+                A.topk_idx[i] = UINT64_MAX;
+                A.topk_score[i] = 0.f;
+            }
+        }
+        if (tid == 0) *A.topk_count = (uint32_t)c;
+    }
+}
+
+int launch_topk_reduce(unsigned long long *d_lists_a, unsigned long long *d_lists_b, int n_lists, uint32_t k,
+                       uint64_t first, const uint64_t *d_idx_map, uint64_t *d_topk_idx, float *d_topk_score,
+                       uint32_t *d_topk_count, cudaStream_t st)
+{
+    unsigned long long *in = d_lists_a, *out = d_lists_b;
+    for (;;) {
+        MergeArgs m;
+        m.in = in; m.out = out; m.n_lists = n_lists; m.k = k; m.group = kMergeGroup;
+        m.first = first; m.idx_map = d_idx_map;
+        m.topk_idx = d_topk_idx; m.topk_score = d_topk_score; m.topk_count = d_topk_count;
+        int n_out = (n_lists + kMergeGroup - 1) / kMergeGroup;
+        m.final = n_out == 1;
+        merge_kernel<<<n_out, kThreads, 0, st>>>(m);
+        count_launch();
+        PF_CUDA_TRY(cudaGetLastError(), "merge_kernel launch");
+        if (n_out == 1) break;
+        n_lists = n_out;
+        unsigned long long *t = in; in = out; out = t;
+    }
+    return PF_OK;
+}
+
+// ------------------------------------------------------------------ merge of two finished top-k lists
+
+struct Merge2Args {
+    uint32_t k;
+    const uint64_t *idx_a, *idx_b;
+    const float *sc_a, *sc_b;
+    const uint32_t *cnt_a, *cnt_b;
+    uint64_t *idx_out;
+    float *sc_out;
+    uint32_t *cnt_out;
+};
+
+// (score descending, index ascending) on explicit pairs; empty slots (idx = UINT64_MAX) last
+__device__ __forceinline__ bool pair_before(uint32_t sa, uint64_t ia, uint32_t sb, uint64_t ib)
+{
+    if (ia == UINT64_MAX || ib == UINT64_MAX) return ib == UINT64_MAX && ia != UINT64_MAX;
+    if (sa != sb) return sa > sb;
+    return ia < ib;
+}
+
+__global__ void __launch_bounds__(kThreads) merge2_kernel(const Merge2Args A)
+{
+    __shared__ uint32_t s_sc[kTopkCap];
+    __shared__ uint64_t s_ix[kTopkCap];
+    const int tid = threadIdx.x, k = (int)A.k;
+    const int na = min((int)*A.cnt_a, k), nb = min((int)*A.cnt_b, k);
+    for (int i = tid; i < kTopkCap; i += kThreads) {
+        uint32_t s = 0;
+        uint64_t x = UINT64_MAX;
+        if (i < na) {
+            s = __float_as_uint(A.sc_a[i]);
+            x = A.idx_a[i];
+        } else if (i >= k && i - k < nb) {
+            s = __float_as_uint(A.sc_b[i - k]);
+            x = A.idx_b[i - k];
+        }
+        s_sc[i] = s;
+        s_ix[i] = x;
+    }
+    for (int size = 2; size <= kTopkCap; size <<= 1)
+        for (int stride = size >> 1; stride > 0; stride >>= 1) {
+            __syncthreads();
+            for (int i = tid; i < kTopkCap / 2; i += kThreads) {
+                int lo = 2 * i - (i & (stride - 1)), hi = lo + stride;
+                bool fwd = (lo & size) == 0;
+                uint32_t sa = s_sc[lo], sb = s_sc[hi];
+                uint64_t ia = s_ix[lo], ib = s_ix[hi];
+                bool swap = fwd ? pair_before(sb, ib, sa, ia) : pair_before(sa, ia, sb, ib);
+                if (swap) {
+                    s_sc[lo] = sb; s_sc[hi] = sa;
+                    s_ix[lo] = ib; s_ix[hi] = ia;
+                }
+            }
+        }
+    __syncthreads();
+    // duplicates (the same candidate in both lists) would be adjacent; the inputs are shards of one space,
+    // so none are expected and none are removed
+    const int n = min(na + nb, k);
+    for (int i = tid; i < k; i += kThreads) {
+        A.idx_out[i] = i < n ? s_ix[i] : UINT64_MAX;
+        A.sc_out[i] = i < n ? __uint_as_float(s_sc[i]) : 0.f;
+    }
+    if (tid == 0) *A.cnt_out = (uint32_t)n;
+}
+
+static int grid_for(const pf_plan_t *p, uint64_t n_slabs)
+{
+    uint64_t g = (uint64_t)p->sm_count * 4;
+    if (g > n_slabs) g = n_slabs;
+    return g < 1 ? 1 : (int)g;
+}
+
+static void slab_span(const pf_plan_t *p, uint64_t first, uint64_t count, uint64_t &slab_lo, uint64_t &n_slabs)
+{
+    const uint64_t S = p->dev.slab;
+    slab_lo = first / S;
+    uint64_t slab_hi = (first + count + S - 1) / S;
+    n_slabs = slab_hi - slab_lo;
+}
+
+}  // namespace pf
+
+using namespace pf;
+
+extern "C" size_t pf_score_workspace(const pf_plan_t *p, uint64_t count, uint32_t k)
+{
+    if (!p || count == 0) return 256;
+    uint64_t slab_lo, n_slabs;
+    slab_span(p, 0, count + p->dev.slab, slab_lo, n_slabs);  // any alignment of `first`
+    return topk_layout(grid_for(p, n_slabs), k).total;
+}
+
+extern "C" int pf_score(pf_plan_t *p, uint64_t first, uint64_t count, uint8_t *d_reason, float *d_tput,
+                        int64_t *d_mem, uint32_t k, uint64_t *d_topk_idx, float *d_topk_score,
+                        uint32_t *d_topk_count, void *d_workspace, size_t workspace_bytes, void *stream)
+{
+    if (!p) return PF_EINVAL;
+    if (k > PF_K_MAX) return PF_EINVAL;
+    if (k > 0 && (!d_topk_idx || !d_topk_score || !d_topk_count)) return PF_EINVAL;
+    if (count == 0 || count >= PF_MAX_COUNT) return PF_ERANGE;
+    if (first >= p->size || count > p->size - first) return PF_ERANGE;
+    if (!d_workspace || ((uintptr_t)d_workspace & 255) != 0) return PF_EWORKSPACE;
+    if (workspace_bytes < pf_score_workspace(p, count, k)) return PF_EWORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+
+    uint64_t slab_lo, n_slabs;
+    slab_span(p, first, count, slab_lo, n_slabs);
+    const int grid = grid_for(p, n_slabs);
+    const TopkLayout lay = topk_layout(grid, k);
+    uint8_t *ws = (uint8_t *)d_workspace;
+
+    ScoreArgs a;
+    a.first = first; a.count = count; a.slab_lo = slab_lo; a.n_slabs = (uint32_t)n_slabs; a.k = k;
+    a.reason = d_reason; a.tput = d_tput; a.mem = (long long *)d_mem;
+    a.lists = (unsigned long long *)(ws + lay.off_lists_a);
+    a.slab_counter = (unsigned int *)(ws + lay.off_ctrl);
+    a.vals = p->d_vals; a.scen = p->d_scen;
+    PF_CUDA_TRY(cudaMemsetAsync(a.slab_counter, 0, 256, st), "pf_score: counter reset");
+    if (p->dev.wide)
+        score_kernel<unsigned long long><<<grid, kThreads, 0, st>>>(p->dev, a);
+    else
+        score_kernel<uint32_t><<<grid, kThreads, 0, st>>>(p->dev, a);
+    count_launch();
+    PF_CUDA_TRY(cudaGetLastError(), "score_kernel launch");
+    if (k > 0)
+        return launch_topk_reduce(a.lists, (unsigned long long *)(ws + lay.off_lists_b), grid, k, first, nullptr,
+                                  d_topk_idx, d_topk_score, d_topk_count, st);
+    return PF_OK;
+}
+
+extern "C" int pf_topk_merge(uint32_t k, const uint64_t *d_idx_a, const float *d_score_a, const uint32_t *d_count_a,
+                             const uint64_t *d_idx_b, const float *d_score_b, const uint32_t *d_count_b,
+                             uint64_t *d_idx_out, float *d_score_out, uint32_t *d_count_out, void *stream)
+{
+    if (k < 1 || k > PF_K_MAX) return PF_EINVAL;
+    if (!d_idx_a || !d_score_a || !d_count_a || !d_idx_b || !d_score_b || !d_count_b || !d_idx_out || !d_score_out ||
+        !d_count_out)
+        return PF_EINVAL;
+    Merge2Args a;
+    a.k = k; a.idx_a = d_idx_a; a.idx_b = d_idx_b; a.sc_a = d_score_a; a.sc_b = d_score_b;
+    a.cnt_a = d_count_a; a.cnt_b = d_count_b; a.idx_out = d_idx_out; a.sc_out = d_score_out; a.cnt_out = d_count_out;
+    merge2_kernel<<<1, kThreads, 0, (cudaStream_t)stream>>>(a);
+    count_launch();
+    PF_CUDA_TRY(cudaGetLastError(), "merge2_kernel launch");
+    return PF_OK;
+}

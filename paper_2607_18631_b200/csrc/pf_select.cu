@@ -1,0 +1,347 @@
+// pf_select.cu -- survivor selection for the schedule tier (Sec. 3.3: the best analytic candidates are
+// refined with the simulator).  Exact top-S by (score descending, index ascending), emitted in ascending
+// index order, as a two-level radix select on the fp32 score bits followed by an ordered compaction:
+//   hist(hi 16 bits) -> scan -> hist(lo 16 bits inside the threshold bin) -> scan -> per-block counts ->
+//   block-offset scan -> ordered write.
+// Every pass reads the reason bytes with 16-byte loads and touches a score only where the candidate is
+// feasible, so a sparse space costs little more than one byte per candidate per pass.
+#include "pf_internal.cuh"
+
+namespace pf {
+
+constexpr int kSelThreads = 256;
+constexpr int kBins = 65536;
+
+struct SelCtrl {
+    unsigned long long total;     // eligible candidates
+    unsigned long long above1;    // eligible with hi16 > b1
+    unsigned long long n_gt;      // eligible with score bits > threshold
+    unsigned long long need_eq;   // how many of the == threshold ones are taken (smallest indices)
+    unsigned long long target;    // S
+    uint32_t b1, thr_bits;
+    int take_all;
+};
+
+struct SelArgs {
+    uint64_t first, count, s_max;
+    const uint8_t *reason;
+    const float *tput;
+    unsigned int *hist1, *hist2;      // kBins each
+    SelCtrl *ctrl;
+    unsigned long long *blk_gt, *blk_eq;  // per block counts, then exclusive prefixes
+    uint64_t *surv_idx, *surv_count;
+    uint64_t chunk;                   // candidates per block (multiple of 16)
+};
+
+// eligibility beyond feasibility: the simulator's domain (pp <= 32 ranks, <= 8 virtual stages per rank)
+__device__ __forceinline__ bool in_sim_domain(const DevPlan &P, const int32_t *vals, uint64_t idx)
+{
+    int s = 0, v = 0, pp = 0;
+    uint64_t rem = idx;
+#pragma unroll
+    for (int a = 0; a < 7; a++) {
+        uint64_t r = P.radix[a];
+        uint64_t q = rem / r;
+        int d = (int)(rem - q * r);
+        rem = q;
+        if (a == 2) s = __ldg(vals + P.val_off[2] + d);
+        if (a == 4) v = __ldg(vals + P.val_off[4] + d);
+        if (a == 6) pp = __ldg(vals + P.val_off[6] + d);
+    }
+    int v_eff = v == 0 ? (P.sched[s].kind == PF_KIND_INTERLEAVED ? 2 : 1) : v;
+    return pp <= PF_SIM_MAX_RANKS && v_eff <= PF_SIM_MAX_V;
+}
+
+// 16 reason bytes starting at element e (may run past count: missing ones read as 0xFF = infeasible)
+__device__ __forceinline__ uint4 load_reason16(const uint8_t *reason, uint64_t e, uint64_t count)
+{
+    if (e + 16 <= count && (((uintptr_t)(reason + e)) & 15) == 0) return __ldg(reinterpret_cast<const uint4 *>(reason + e));
+    uint32_t w[4] = {0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu};
+    for (int i = 0; i < 16; i++)
+        if (e + i < count) {
+            uint32_t b = reason[e + i];
+            w[i >> 2] = (w[i >> 2] & ~(0xFFu << (8 * (i & 3)))) | (b << (8 * (i & 3)));
+        }
+    return make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+// bit i set: byte i of the 16 has (b & 0x7f) == 0
+__device__ __forceinline__ uint32_t feasible_mask16(uint4 r)
+{
+    uint32_t w[4] = {r.x, r.y, r.z, r.w};
+    uint32_t m = 0;
+#pragma unroll
+    for (int i = 0; i < 4; i++) {
+        uint32_t x = w[i] & 0x7F7F7F7Fu;
+#pragma unroll
+        for (int b = 0; b < 4; b++)
+            if (((x >> (8 * b)) & 0xFFu) == 0) m |= 1u << (4 * i + b);
+    }
+    return m;
+}
+
+// Visit the eligible candidates of a block's chunk in ascending order: f(rel, score_bits).
+template <typename F>
+__device__ __forceinline__ void for_each_eligible16(const DevPlan &P, const int32_t *vals, const SelArgs &A,
+                                                    uint64_t e, F f)
+{
+    uint32_t m = feasible_mask16(load_reason16(A.reason, e, A.count));
+    while (m) {
+        int i = __ffs(m) - 1;
+        m &= m - 1;
+        uint64_t rel = e + i;
+        if (in_sim_domain(P, vals, A.first + rel)) f(rel, __float_as_uint(__ldg(A.tput + rel)));
+    }
+}
+
+__global__ void __launch_bounds__(kSelThreads) sel_hist_kernel(const __grid_constant__ DevPlan P, const SelArgs A,
+                                                                const int32_t *vals, int pass)
+{
+    const uint64_t lo = (uint64_t)blockIdx.x * A.chunk;
+    const uint64_t hi = min(lo + A.chunk, A.count);
+    if (pass == 1 && A.ctrl->take_all) return;
+    const uint32_t b1 = pass == 1 ? A.ctrl->b1 : 0;
+    for (uint64_t e = lo + (uint64_t)threadIdx.x * 16; e < hi; e += (uint64_t)kSelThreads * 16) {
+        for_each_eligible16(P, vals, A, e, [&](uint64_t, uint32_t bits) {
+            if (pass == 0)
+                atomicAdd(A.hist1 + (bits >> 16), 1u);
+            else if ((bits >> 16) == b1)
+                atomicAdd(A.hist2 + (bits & 0xFFFFu), 1u);
+        });
+    }
+}
+
+// One block of 1024 threads: find the bin (scanning from the top) where the running count reaches the target.
+__global__ void __launch_bounds__(1024) sel_scan_kernel(const SelArgs A, int pass)
+{
+    __shared__ unsigned long long s_sum[1024];
+    __shared__ unsigned long long s_suffix[1025];
+    const int tid = threadIdx.x;
+    SelCtrl *c = A.ctrl;
+    if (pass == 1 && c->take_all) return;
+    const unsigned int *hist = pass == 0 ? A.hist1 : A.hist2;
+    constexpr int per = kBins / 1024;
+    // thread t owns bins [t*per, (t+1)*per)
+    unsigned long long mine = 0;
+    for (int i = 0; i < per; i++) mine += hist[tid * per + i];
+    s_sum[tid] = mine;
+    __syncthreads();
+    if (tid == 0) {
+        unsigned long long run = 0;
+        s_suffix[1024] = 0;
+        for (int t = 1023; t >= 0; t--) {
+            run += s_sum[t];
+            s_suffix[t] = run;  // count in bins >= t*per
+        }
+    }
+    __syncthreads();
+    const unsigned long long total = s_suffix[0];
+    unsigned long long target;
+    if (pass == 0) {
+        target = A.s_max;
+        if (tid == 0) {
+            c->total = total;
+            c->target = target;
+            c->take_all = total <= target ? 1 : 0;
+            if (total <= target) {
+                c->thr_bits = 0;
+                c->n_gt = total;
+                c->need_eq = 0;
+            }
+        }
+        if (total <= target) return;
+    } else {
+        target = c->target - c->above1;
+    }
+    // the owner of the crossing: suffix above me < target <= suffix including me
+    const unsigned long long above = s_suffix[tid + 1];
+    if (above < target && above + mine >= target) {
+        unsigned long long run = above;
+        for (int i = per - 1; i >= 0; i--) {
+            unsigned int h = hist[tid * per + i];
+            if (run + h >= target) {
+                uint32_t bin = (uint32_t)(tid * per + i);
+                if (pass == 0) {
+                    c->b1 = bin;
+                    c->above1 = run;
+                } else {
+                    c->thr_bits = (c->b1 << 16) | bin;
+                    c->n_gt = c->above1 + run;
+                    c->need_eq = c->target - (c->above1 + run);
+                }
+                break;
+            }
+            run += h;
+        }
+    }
+}
+
+__global__ void __launch_bounds__(kSelThreads) sel_count_kernel(const __grid_constant__ DevPlan P, const SelArgs A,
+                                                                 const int32_t *vals)
+{
+    __shared__ unsigned long long s_gt, s_eq;
+    if (threadIdx.x == 0) s_gt = s_eq = 0;
+    __syncthreads();
+    const uint64_t lo = (uint64_t)blockIdx.x * A.chunk;
+    const uint64_t hi = min(lo + A.chunk, A.count);
+    const uint32_t thr = A.ctrl->thr_bits;
+    const bool all = A.ctrl->take_all != 0;
+    unsigned int gt = 0, eq = 0;
+    for (uint64_t e = lo + (uint64_t)threadIdx.x * 16; e < hi; e += (uint64_t)kSelThreads * 16) {
+        for_each_eligible16(P, vals, A, e, [&](uint64_t, uint32_t bits) {
+            if (all || bits > thr) gt++;
+            else if (bits == thr) eq++;
+        });
+    }
+    if (gt) atomicAdd(&s_gt, (unsigned long long)gt);
+    if (eq) atomicAdd(&s_eq, (unsigned long long)eq);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        A.blk_gt[blockIdx.x] = s_gt;
+        A.blk_eq[blockIdx.x] = s_eq;
+    }
+}
+
+// exclusive prefix over blocks (one thread: a few hundred entries) + the survivor count
+__global__ void sel_blockscan_kernel(const SelArgs A, int nblocks)
+{
+    if (threadIdx.x != 0 || blockIdx.x != 0) return;
+    unsigned long long g = 0, q = 0;
+    for (int b = 0; b < nblocks; b++) {
+        unsigned long long cg = A.blk_gt[b], ce = A.blk_eq[b];
+        A.blk_gt[b] = g;
+        A.blk_eq[b] = q;
+        g += cg;
+        q += ce;
+    }
+    const SelCtrl *c = A.ctrl;
+    *A.surv_count = c->take_all ? c->total : c->target;
+}
+
+// Ordered write: position of an admitted candidate = (# taken "greater" before it) + min(# "equal" before it, need_eq)
+__global__ void __launch_bounds__(kSelThreads) sel_write_kernel(const __grid_constant__ DevPlan P, const SelArgs A,
+                                                                 const int32_t *vals)
+{
+    __shared__ unsigned int s_gt[kSelThreads], s_eq[kSelThreads];
+    __shared__ unsigned long long s_run_gt, s_run_eq;
+    const int tid = threadIdx.x;
+    const uint64_t lo = (uint64_t)blockIdx.x * A.chunk;
+    const uint64_t hi = min(lo + A.chunk, A.count);
+    const uint32_t thr = A.ctrl->thr_bits;
+    const bool all = A.ctrl->take_all != 0;
+    const unsigned long long need_eq = all ? 0ull : A.ctrl->need_eq;
+    if (tid == 0) {
+        s_run_gt = A.blk_gt[blockIdx.x];
+        s_run_eq = A.blk_eq[blockIdx.x];
+    }
+    __syncthreads();
+    for (uint64_t tile = lo; tile < hi; tile += (uint64_t)kSelThreads * 16) {
+        const uint64_t e = tile + (uint64_t)tid * 16;
+        unsigned int gt = 0, eq = 0;
+        if (e < hi)
+            for_each_eligible16(P, vals, A, e, [&](uint64_t, uint32_t bits) {
+                if (all || bits > thr) gt++;
+                else if (bits == thr) eq++;
+            });
+        s_gt[tid] = gt;
+        s_eq[tid] = eq;
+        __syncthreads();
+        // exclusive scan by one warp-free loop would serialize 256 steps; do a simple Hillis-Steele scan
+        for (int off = 1; off < kSelThreads; off <<= 1) {
+            unsigned int ag = tid >= off ? s_gt[tid - off] : 0, ae = tid >= off ? s_eq[tid - off] : 0;
+            __syncthreads();
+            s_gt[tid] += ag;
+            s_eq[tid] += ae;
+            __syncthreads();
+        }
+        unsigned long long my_gt = s_run_gt + (s_gt[tid] - gt);
+        unsigned long long my_eq = s_run_eq + (s_eq[tid] - eq);
+        if (e < hi && (gt | eq))
+            for_each_eligible16(P, vals, A, e, [&](uint64_t rel, uint32_t bits) {
+                if (all || bits > thr) {
+                    unsigned long long pos = my_gt + (my_eq < need_eq ? my_eq : need_eq);
+                    A.surv_idx[pos] = A.first + rel;
+                    my_gt++;
+                } else if (bits == thr) {
+                    if (my_eq < need_eq) A.surv_idx[my_gt + my_eq] = A.first + rel;
+                    my_eq++;
+                }
+            });
+        __syncthreads();
+        if (tid == kSelThreads - 1) {
+            s_run_gt += s_gt[tid];
+            s_run_eq += s_eq[tid];
+        }
+        __syncthreads();
+    }
+}
+
+struct SelLayout {
+    size_t off_ctrl, off_hist1, off_hist2, off_gt, off_eq, total;
+    int nblocks;
+    uint64_t chunk;
+};
+
+static SelLayout sel_layout(const pf_plan_t *p, uint64_t count)
+{
+    SelLayout l;
+    uint64_t nb = (uint64_t)p->sm_count * 4;
+    uint64_t chunk = (count + nb - 1) / nb;
+    chunk = (chunk + 4095) & ~(uint64_t)4095;  // whole tiles of 256 threads x 16 candidates
+    if (chunk == 0) chunk = 4096;
+    l.chunk = chunk;
+    l.nblocks = (int)((count + chunk - 1) / chunk);
+    if (l.nblocks < 1) l.nblocks = 1;
+    l.off_ctrl = 0;
+    l.off_hist1 = 256;
+    l.off_hist2 = l.off_hist1 + kBins * 4;
+    l.off_gt = l.off_hist2 + kBins * 4;
+    size_t per = (((size_t)p->sm_count * 4 + 1) * 8 + 255) & ~(size_t)255;
+    l.off_eq = l.off_gt + per;
+    l.total = l.off_eq + per;
+    return l;
+}
+
+}  // namespace pf
+
+using namespace pf;
+
+extern "C" size_t pf_select_workspace(const pf_plan_t *p, uint64_t count, uint64_t s_max)
+{
+    (void)s_max;
+    if (!p) return 0;
+    return sel_layout(p, count).total;
+}
+
+extern "C" int pf_select_survivors(pf_plan_t *p, uint64_t first, uint64_t count, const uint8_t *d_reason,
+                                   const float *d_tput, uint64_t s_max, uint64_t *d_surv_idx, uint64_t *d_surv_count,
+                                   void *d_workspace, size_t workspace_bytes, void *stream)
+{
+    if (!p || !d_reason || !d_tput || !d_surv_idx || !d_surv_count) return PF_EINVAL;
+    if (p->dev.phase != PF_PHASE_TRAIN) return PF_EUNSUPPORTED;
+    if (count == 0 || count >= PF_MAX_COUNT || s_max == 0) return PF_ERANGE;
+    if (first >= p->size || count > p->size - first) return PF_ERANGE;
+    const SelLayout lay = sel_layout(p, count);
+    if (!d_workspace || ((uintptr_t)d_workspace & 255) != 0 || workspace_bytes < lay.total) return PF_EWORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    uint8_t *ws = (uint8_t *)d_workspace;
+    SelArgs a;
+    a.first = first; a.count = count; a.s_max = s_max; a.reason = d_reason; a.tput = d_tput;
+    a.ctrl = (SelCtrl *)(ws + lay.off_ctrl);
+    a.hist1 = (unsigned int *)(ws + lay.off_hist1);
+    a.hist2 = (unsigned int *)(ws + lay.off_hist2);
+    a.blk_gt = (unsigned long long *)(ws + lay.off_gt);
+    a.blk_eq = (unsigned long long *)(ws + lay.off_eq);
+    a.surv_idx = d_surv_idx; a.surv_count = d_surv_count; a.chunk = lay.chunk;
+    PF_CUDA_TRY(cudaMemsetAsync(ws, 0, lay.off_gt, st), "pf_select_survivors: clear");
+    sel_hist_kernel<<<lay.nblocks, kSelThreads, 0, st>>>(p->dev, a, p->d_vals, 0);
+    sel_scan_kernel<<<1, 1024, 0, st>>>(a, 0);
+    sel_hist_kernel<<<lay.nblocks, kSelThreads, 0, st>>>(p->dev, a, p->d_vals, 1);
+    sel_scan_kernel<<<1, 1024, 0, st>>>(a, 1);
+    sel_count_kernel<<<lay.nblocks, kSelThreads, 0, st>>>(p->dev, a, p->d_vals);
+    sel_blockscan_kernel<<<1, 32, 0, st>>>(a, lay.nblocks);
+    sel_write_kernel<<<lay.nblocks, kSelThreads, 0, st>>>(p->dev, a, p->d_vals);
+    for (int i = 0; i < 7; i++) count_launch();
+    PF_CUDA_TRY(cudaGetLastError(), "pf_select_survivors launch");
+    return PF_OK;
+}

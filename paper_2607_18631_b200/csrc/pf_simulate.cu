@@ -1,0 +1,592 @@
+// pf_simulate.cu -- simulator tier: one warp per survivor, one lane per pipeline rank (Sec. 3.2: the
+// list-scheduling timeline refines the schedules the closed form only approximates).
+//
+// Each lane walks its rank's fixed op order (1F1B and interleaved orders are generated on the fly from
+// counters; the DualPipe-style order comes from a host-built table) and computes
+//   end(op) = max(end of the rank's previous op, end(dependency) + latency) + duration.
+// A forward of stage q needs the forward of stage q-1 of the same microbatch, a backward of stage q needs
+// the backward of stage q+1; the op's own forward is already behind the lane's clock.  Within one stage,
+// forwards (and backwards) finish in microbatch order, so "is the dependency done" is a per-stage counter
+// compare and the end-time arrays in shared memory never need clearing.  Lanes advance in lock step with
+// __syncwarp between rounds; a round in which no lane advances ends the candidate with PF_SIM_STALL, so
+// the loop is bounded by the op count.
+#include <cstdlib>
+#include <cstring>
+#include <vector>
+
+#include "pf_eval.cuh"
+
+namespace pf {
+
+constexpr int kSimMaxWarps = 16;        // warps per block at most (each simulates one candidate at a time)
+constexpr int kSimSmemBudget = 200 * 1024;  // dynamic shared memory a block may take
+
+// DualPipe-style order tables: for every (pp, m) in the domain a byte string per rank,
+// op = (j << 2) | (dir << 1) | is_backward, 2*m ops per rank.
+struct SimTables {
+    uint8_t *d_ops;                 // device copy of all tables
+    int32_t *d_offset;              // [33][33]: offset of table (pp, m/2), -1 if absent
+    std::vector<int32_t> h_offset;
+    size_t bytes;
+};
+
+// Host: nominal list scheduling that DEFINES the DualPipe-style order (F = 1 tick, B = 2 ticks, zero
+// latency).  At every event time each idle rank starts the ready op with the smallest
+// (ready time, backward before forward, microbatch, direction); a forward at position q may start only
+// while fewer than pp - q microbatches of its direction are in flight on the rank.  Within one
+// (rank, direction, F/B) stream ops become ready in microbatch order, so only the four stream heads of a
+// rank compete.
+static bool build_dualpipe_table(int pp, int m, uint8_t *out /* [pp][2m] */)
+{
+    const int n = m / 2;
+    // done_at[type][dir][q][j]: nominal completion tick, -1 while not started
+    std::vector<int> done_at((size_t)4 * pp * n, -1);
+    auto at = [&](int b, int d, int q, int j) -> int & { return done_at[(((size_t)b * 2 + d) * pp + q) * n + j]; };
+    std::vector<int> head((size_t)pp * 4, 0);  // next microbatch per (rank, dir, type)
+    std::vector<int> live((size_t)pp * 2, 0), free_at(pp, 0), len(pp, 0);
+    int remaining = 4 * pp * n, now = 0;
+    while (remaining > 0) {
+        for (int r = 0; r < pp; r++) {
+            if (free_at[r] > now) continue;
+            int best_b = -1, best_d = 0, best_j = 0, best_q = 0, best_ready = 0;
+            for (int d = 0; d < 2; d++) {
+                const int q = d ? pp - 1 - r : r;
+                for (int b = 1; b >= 0; b--) {
+                    const int j = head[(r * 2 + d) * 2 + b];
+                    if (j >= n) continue;
+                    int ready = 0;
+                    if (b == 0) {
+                        if (q > 0) {
+                            int e = at(0, d, q - 1, j);
+                            if (e < 0 || e > now) continue;
+                            ready = e;
+                        }
+                        if (live[r * 2 + d] >= pp - q) continue;
+                    } else {
+                        int e = at(0, d, q, j);
+                        if (e < 0 || e > now) continue;
+                        ready = e;
+                        if (q < pp - 1) {
+                            int e2 = at(1, d, q + 1, j);
+                            if (e2 < 0 || e2 > now) continue;
+                            ready = e2 > ready ? e2 : ready;
+                        }
+                    }
+                    bool better;
+                    if (best_b < 0) better = true;
+                    else if (ready != best_ready) better = ready < best_ready;
+                    else if (b != best_b) better = b > best_b;
+                    else if (j != best_j) better = j < best_j;
+                    else better = d < best_d;
+                    if (better) best_b = b, best_d = d, best_j = j, best_q = q, best_ready = ready;
+                }
+            }
+            if (best_b < 0) continue;
+            const int fin = now + (best_b ? 2 : 1);
+            at(best_b, best_d, best_q, best_j) = fin;
+            free_at[r] = fin;
+            head[(r * 2 + best_d) * 2 + best_b]++;
+            live[r * 2 + best_d] += best_b ? -1 : 1;
+            out[(size_t)r * 2 * m + len[r]++] = (uint8_t)((best_j << 2) | (best_d << 1) | best_b);
+            remaining--;
+        }
+        int next = -1;
+        for (int r = 0; r < pp; r++)
+            if (free_at[r] > now && (next < 0 || free_at[r] < next)) next = free_at[r];
+        if (next < 0) return remaining == 0;  // nothing running and nothing ready: would never finish
+        now = next;
+    }
+    return true;
+}
+
+// Called once by pf_plan_create for training plans: builds and uploads the order tables.
+int build_sim_tables(pf_plan_t *p)
+{
+    if (p->sim_tables) return PF_OK;
+    SimTables *t = new SimTables;
+    t->d_ops = nullptr;
+    t->d_offset = nullptr;
+    t->h_offset.assign(33 * 33, -1);
+    std::vector<uint8_t> ops;
+    // only if the plan has a DualPipe-class schedule; depths from the pp axis (1 or even, <= 32)
+    bool any_dual = false;
+    for (int s = 0; s < p->dev.n_sched; s++) any_dual |= p->dev.sched[s].kind == PF_KIND_DUALPIPE;
+    if (any_dual && p->dev.phase == PF_PHASE_TRAIN) {
+        const int32_t *pps = p->h_vals + p->dev.val_off[6];
+        for (int i = 0; i < p->axis_len[6]; i++) {
+            const int pp = pps[i];
+            if (pp > PF_SIM_MAX_RANKS || (pp > 1 && (pp & 1))) continue;
+            if (t->h_offset[pp * 33 + 1] >= 0) continue;
+            for (int n = 1; n <= PF_SIM_WINDOW / 2; n++) {
+                const int m = 2 * n;
+                size_t off = ops.size();
+                ops.resize(off + (size_t)pp * 2 * m);
+                if (!build_dualpipe_table(pp, m, ops.data() + off)) {
+                    delete t;
+                    return PF_EINVAL;
+                }
+                t->h_offset[pp * 33 + n] = (int32_t)off;
+            }
+        }
+    }
+    t->bytes = ops.size();
+    cudaError_t e = cudaMalloc((void **)&t->d_offset, sizeof(int32_t) * 33 * 33);
+    if (e == cudaSuccess)
+        e = cudaMemcpy(t->d_offset, t->h_offset.data(), sizeof(int32_t) * 33 * 33, cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaMalloc((void **)&t->d_ops, ops.size() ? ops.size() : 16);
+    if (e == cudaSuccess && !ops.empty()) e = cudaMemcpy(t->d_ops, ops.data(), ops.size(), cudaMemcpyHostToDevice);
+    if (e != cudaSuccess) {
+        set_cuda_error(e, "simulator tables");
+        if (t->d_offset) cudaFree(t->d_offset);
+        if (t->d_ops) cudaFree(t->d_ops);
+        delete t;
+        return PF_ECUDA;
+    }
+    p->sim_tables = t;
+    return PF_OK;
+}
+
+void free_sim_tables(pf_plan_t *p)
+{
+    SimTables *t = (SimTables *)p->sim_tables;
+    if (!t) return;
+    if (t->d_offset) cudaFree(t->d_offset);
+    if (t->d_ops) cudaFree(t->d_ops);
+    delete t;
+    p->sim_tables = nullptr;
+}
+
+// ------------------------------------------------------------------ device
+
+__device__ __forceinline__ uint32_t mix32(uint32_t x)
+{
+    x ^= x >> 16;
+    x *= 0x7feb352du;
+    x ^= x >> 15;
+    x *= 0x846ca68bu;
+    x ^= x >> 16;
+    return x;
+}
+
+// multiplicative jitter in [0.9, 1.1): counter hash of (seed, candidate, stage, F/B)
+__device__ __forceinline__ float jitter(uint32_t seed_mixed, uint64_t idx, int q, int is_b)
+{
+    uint32_t h = mix32(seed_mixed ^ (uint32_t)idx);
+    h = mix32(h ^ (uint32_t)(idx >> 32));
+    h = mix32(h ^ (uint32_t)(2 * q + is_b));
+    float u = (float)(h >> 8) * (1.0f / 16777216.0f);
+    return 0.9f + 0.2f * u;
+}
+
+struct SimArgs {
+    const uint64_t *surv;
+    uint64_t n;
+    const uint64_t *d_n;            // optional device-side count
+    uint32_t seed;
+    float *tput_sim;
+    uint8_t *status;
+    unsigned int *counter;          // work queue, zeroed before launch
+    const int32_t *vals;
+    const uint8_t *dual_ops;
+    const int32_t *dual_off;
+    int q_max;                      // stages per candidate at most (plan-wide)
+};
+
+// per-warp shared memory: endF[q_max*64], endB[q_max*64], durF[q_max], durB[q_max], cntF[q_max*2], cntB[q_max*2]
+__host__ __device__ inline size_t sim_warp_floats(int q_max) { return (size_t)q_max * (2 * PF_SIM_WINDOW + 2 + 4); }
+
+template <typename RI>
+__global__ void __launch_bounds__(kSimMaxWarps * 32) simulate_kernel(const __grid_constant__ DevPlan P, const SimArgs A)
+{
+    extern __shared__ float s_mem[];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    float *base = s_mem + (size_t)warp * sim_warp_floats(A.q_max);
+    // end times and per-stage completion counters are written by one lane and read by its neighbours
+    // within a round: volatile accesses plus a block-level fence between "value" and "counter" keep the
+    // pair ordered
+    volatile float *endF = base;
+    volatile float *endB = endF + (size_t)A.q_max * PF_SIM_WINDOW;
+    float *durF = base + (size_t)2 * A.q_max * PF_SIM_WINDOW;
+    float *durB = durF + A.q_max;
+    volatile int *cntF = reinterpret_cast<int *>(durB + A.q_max);
+    volatile int *cntB = cntF + 2 * A.q_max;
+
+    uint64_t n = A.n;
+    if (A.d_n) {
+        uint64_t dn = *A.d_n;
+        n = dn < n ? dn : n;
+    }
+    const uint32_t seed_mixed = mix32(A.seed + 0x9e3779b9u);
+
+    for (;;) {
+        unsigned int w = 0;
+        if (lane == 0) w = atomicAdd(A.counter, 1u);
+        w = __shfl_sync(0xFFFFFFFFu, w, 0);
+        if ((uint64_t)w >= n) break;
+        const uint64_t idx = A.surv[w];
+
+        // ---- every lane re-derives the candidate (uniform across the warp)
+        TrainTuple c;
+        {
+            int v[PF_MAX_AXES];
+            uint64_t rem = idx;
+#pragma unroll
+            for (int a = 0; a < PF_MAX_AXES; a++) {
+                uint64_t r = P.radix[a];
+                uint64_t q = rem / r;
+                v[a] = __ldg(A.vals + P.val_off[a] + (int)(rem - q * r));
+                rem = q;
+            }
+            c.kv = v[0]; c.rec = v[1]; c.s = v[2]; c.mb = v[3]; c.v = v[4];
+            c.ep = v[5]; c.pp = v[6]; c.tp = v[7]; c.dp = v[8]; c.world = v[9];
+        }
+        RI dp, world;
+        TrainDerived<RI> D;
+        TrainMem M;
+        int reason = train_layout_rules<RI>(P, c, 1, 3, dp, world);
+        if (reason == 0) reason = train_plan_rules<RI>(P, c, dp, world, 1, D);
+        if (reason == 0) {
+            train_memory<RI>(P, c, D, M);
+            if (M.mem > P.budget_bytes) reason = PF_R_MEMORY;
+        }
+        if (reason != 0) {
+            if (lane == 0) {
+                if (A.tput_sim) A.tput_sim[w] = 0.f;
+                if (A.status) A.status[w] = PF_SIM_UNSUPPORTED;
+            }
+            continue;
+        }
+        TrainTimes T;
+        train_times<RI>(P, c, D, M, T);
+        const int pp = c.pp, v = D.v_eff, kind = D.kind;
+        if (pp > PF_SIM_MAX_RANKS || v > PF_SIM_MAX_V) {
+            if (lane == 0) {
+                if (A.tput_sim) A.tput_sim[w] = train_price<RI>(P, c, D, T, train_pipe_analytic<RI>(P, c, D, T));
+                if (A.status) A.status[w] = PF_SIM_UNSUPPORTED;
+            }
+            continue;
+        }
+        const bool dual = kind == PF_KIND_DUALPIPE;
+        const int Q = dual ? pp : pp * v;
+        // simulated window
+        const long long m = (long long)D.m;
+        int m_sim = m < PF_SIM_WINDOW ? (int)m : PF_SIM_WINDOW;
+        if (kind == PF_KIND_INTERLEAVED) m_sim = (m_sim / pp) * pp;
+        const int nj = dual ? m_sim / 2 : m_sim;  // microbatches per stage stream
+
+        // ---- stage durations: balanced layer split, head on the last stage, jitter
+        __syncwarp();
+        const int L_lo = P.L / Q, L_rem = P.L - L_lo * Q;
+        for (int q = lane; q < Q; q += 32) {
+            const float nq = (float)(L_lo + (q < L_rem ? 1 : 0));
+            const bool last = q == Q - 1;
+            durF[q] = (nq * T.F_l + (last ? T.headF : 0.f)) * jitter(seed_mixed, idx, q, 0);
+            durB[q] = (nq * T.B_l + (last ? P.bwd_factor * T.headF : 0.f)) * jitter(seed_mixed, idx, q, 1);
+        }
+        for (int i = lane; i < 2 * Q; i += 32) {
+            cntF[i] = 0;
+            cntB[i] = 0;
+        }
+        __syncwarp();
+
+        // ---- per-lane order state
+        const bool rank_active = lane < pp;
+        const int U = dual ? 2 * nj : nj * (kind == PF_KIND_INTERLEAVED ? v : 1);  // forward units of this rank
+        int warm;
+        if (kind == PF_KIND_INTERLEAVED)
+            warm = min(2 * (pp - lane - 1) + (v - 1) * pp, U);
+        else
+            warm = min(pp - lane - 1, U);
+        // forward / backward unit cursors as (group, chunk slot, slot-in-group) without divisions
+        int nF = 0, nB = 0;               // units issued
+        int fg = 0, fc = 0, fw = 0;       // forward cursor: microbatch = fg*pp + fw, chunk = fc
+        int bg = 0, bc = 0, bw = 0;       // backward cursor: chunk = v-1-bc
+        const uint8_t *dops = nullptr;
+        bool stalled = false;
+        if (dual) {
+            const int off = __ldg(A.dual_off + pp * 33 + nj);
+            if (off < 0) stalled = true;  // no table for this shape: report instead of reading out of bounds
+            else dops = A.dual_ops + off + (size_t)lane * 2 * m_sim;
+        }
+        float clock = 0.f;
+        const int total_ops = (rank_active && !stalled) ? 2 * U : 0;
+        int done_ops = 0;
+
+        for (;;) {
+            bool progressed = false;
+            // up to 4 ops per round keep the lanes that run ahead from waiting on the barrier
+#pragma unroll 1
+            for (int rep = 0; rep < 4 && done_ops < total_ops; rep++) {
+                int isb, d = 0, q, j;
+                if (dual) {
+                    const uint8_t op = __ldg(dops + done_ops);
+                    isb = op & 1;
+                    d = (op >> 1) & 1;
+                    j = op >> 2;
+                    q = d ? pp - 1 - lane : lane;
+                } else {
+                    isb = !(nF < warm || (nF < U && nF - warm == nB));
+                    if (!isb) {
+                        j = fg * pp + fw;
+                        q = fc * pp + lane;
+                    } else {
+                        j = bg * pp + bw;
+                        q = (v - 1 - bc) * pp + lane;
+                    }
+                    if (kind == PF_KIND_1F1B) {
+                        j = isb ? nB : nF;
+                        q = lane;
+                    }
+                }
+                const int sidx = d * Q + q;          // stage stream (direction-major for DualPipe)
+                float dep = 0.f;
+                bool ready = true;
+                if (!isb) {
+                    if (q > 0) {
+                        ready = cntF[sidx - 1] > j;
+                        if (ready) {
+                            __threadfence_block();
+                            dep = endF[(size_t)(sidx - 1) * nj + j] + T.p;
+                        }
+                    }
+                } else {
+                    if (q < Q - 1) {
+                        ready = cntB[sidx + 1] > j;
+                        if (ready) {
+                            __threadfence_block();
+                            dep = endB[(size_t)(sidx + 1) * nj + j] + T.p;
+                        }
+                    }
+                }
+                if (!ready) break;
+                const float fin = fmaxf(clock, dep) + (isb ? durB[q] : durF[q]);
+                clock = fin;
+                if (!isb) {
+                    endF[(size_t)sidx * nj + j] = fin;
+                    __threadfence_block();
+                    cntF[sidx] = j + 1;
+                    nF++;
+                    if (++fw == pp) {
+                        fw = 0;
+                        if (++fc == v) fc = 0, fg++;
+                    }
+                } else {
+                    endB[(size_t)sidx * nj + j] = fin;
+                    __threadfence_block();
+                    cntB[sidx] = j + 1;
+                    nB++;
+                    if (++bw == pp) {
+                        bw = 0;
+                        if (++bc == v) bc = 0, bg++;
+                    }
+                }
+                done_ops++;
+                progressed = true;
+            }
+            __syncwarp();
+            const unsigned pending = __ballot_sync(0xFFFFFFFFu, done_ops < total_ops);
+            if (pending == 0) break;
+            if (!__any_sync(0xFFFFFFFFu, progressed)) {
+                stalled = true;
+                break;
+            }
+        }
+
+        // ---- makespan, steady-state extension beyond the window, pricing
+        float work = 0.f;
+        if (rank_active) {
+            if (dual) {
+                work = 0.5f * (durF[lane] + durB[lane] + durF[pp - 1 - lane] + durB[pp - 1 - lane]);
+            } else {
+                const int vv = kind == PF_KIND_INTERLEAVED ? v : 1;
+                for (int cc = 0; cc < vv; cc++) work += durF[cc * pp + lane] + durB[cc * pp + lane];
+            }
+        }
+        float span = rank_active ? clock : 0.f;
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+            span = fmaxf(span, __shfl_xor_sync(0xFFFFFFFFu, span, off));
+            work = fmaxf(work, __shfl_xor_sync(0xFFFFFFFFu, work, off));
+        }
+        if (lane == 0) {
+            float tput = 0.f;
+            if (!stalled) {
+                float T_pipe = span;
+                if (m > m_sim) T_pipe += (float)(m - m_sim) * work;
+                tput = train_price<RI>(P, c, D, T, T_pipe);
+            }
+            if (A.tput_sim) A.tput_sim[w] = tput;
+            if (A.status) A.status[w] = stalled ? PF_SIM_STALL : PF_SIM_OK;
+        }
+        __syncwarp();
+    }
+}
+
+// ------------------------------------------------------------------ top-k over a dense score array
+// position in the list is the tie-break (equal to index order for lists from pf_select_survivors)
+
+struct DenseTopkArgs {
+    const float *score;
+    uint64_t n;
+    const uint64_t *d_n;
+    uint32_t k;
+    unsigned long long *lists;
+};
+
+__global__ void __launch_bounds__(kThreads) dense_topk_kernel(const DenseTopkArgs A)
+{
+    __shared__ unsigned long long s_buf[kTopkCap];
+    __shared__ int s_count;
+    __shared__ unsigned long long s_thr;
+    const int tid = threadIdx.x;
+    if (tid == 0) {
+        s_count = 0;
+        s_thr = 0ull;
+    }
+    __syncthreads();
+    uint64_t n = A.n;
+    if (A.d_n) {
+        uint64_t dn = *A.d_n;
+        n = dn < n ? dn : n;
+    }
+    int room = kTopkCap / kThreads;
+    unsigned long long thr = 0ull;
+    for (uint64_t base = (uint64_t)blockIdx.x * kThreads; base < n; base += (uint64_t)gridDim.x * kThreads) {
+        if (room == 0) {
+            __syncthreads();
+            if (s_count > kTopkCap - kThreads) tk_prune(s_buf, &s_count, &s_thr, (int)A.k);
+            room = (kTopkCap - s_count) / kThreads;
+            thr = s_thr;
+            __syncthreads();
+        }
+        const uint64_t i = base + tid;
+        const float s = i < n ? A.score[i] : 0.f;
+        tk_push(s_buf, &s_count, thr, s > 0.f, make_key(s, (uint32_t)i));
+        room--;
+    }
+    tk_prune(s_buf, &s_count, &s_thr, (int)A.k);
+    unsigned long long *out = A.lists + (size_t)blockIdx.x * A.k;
+    const int c = s_count;
+    for (int i = tid; i < (int)A.k; i += kThreads) out[i] = i < c ? s_buf[i] : 0ull;
+}
+
+struct SimLayout {
+    size_t off_counter, off_scores, off_topk, total;
+    int topk_blocks;
+    TopkLayout tk;
+};
+
+static SimLayout sim_layout(const pf_plan_t *p, uint64_t n, uint32_t k)
+{
+    SimLayout l;
+    l.off_counter = 0;
+    l.off_scores = 256;
+    size_t sc = ((size_t)(n ? n : 1) * 4 + 255) & ~(size_t)255;
+    l.off_topk = l.off_scores + sc;
+    uint64_t tb = (n + kThreads - 1) / kThreads;
+    uint64_t cap = (uint64_t)p->sm_count * 2;
+    l.topk_blocks = (int)(tb < 1 ? 1 : (tb > cap ? cap : tb));
+    l.tk = topk_layout(l.topk_blocks, k);
+    l.total = l.off_topk + (k ? l.tk.total : 0);
+    return l;
+}
+
+// plan-wide bound on stages per candidate inside the simulator's domain
+static int plan_q_max(const pf_plan_t *p)
+{
+    int pp_max = 1, v_max = 1;
+    const int32_t *pps = p->h_vals + p->dev.val_off[6];
+    for (int i = 0; i < p->axis_len[6]; i++)
+        if (pps[i] <= PF_SIM_MAX_RANKS && pps[i] > pp_max) pp_max = pps[i];
+    const int32_t *vs = p->h_vals + p->dev.val_off[4];
+    for (int i = 0; i < p->axis_len[4]; i++) {
+        int v = vs[i] == 0 ? 2 : vs[i];
+        if (v <= PF_SIM_MAX_V && v > v_max) v_max = v;
+    }
+    long long q = (long long)pp_max * v_max;
+    if (q > p->dev.L) q = p->dev.L;  // the layer rule admits pp*v <= L only
+    if (q < pp_max) q = pp_max;
+    return (int)q;
+}
+
+}  // namespace pf
+
+using namespace pf;
+
+extern "C" int pf_dualpipe_order(int pp, int m, uint8_t *out_ops)
+{
+    if (!out_ops || pp < 1 || pp > PF_SIM_MAX_RANKS || (pp > 1 && (pp & 1)) || m < 2 || (m & 1) || m > PF_SIM_WINDOW)
+        return PF_EINVAL;
+    return build_dualpipe_table(pp, m, out_ops) ? PF_OK : PF_EINVAL;
+}
+
+extern "C" size_t pf_simulate_workspace(const pf_plan_t *p, uint64_t n, uint32_t k)
+{
+    if (!p) return 0;
+    return sim_layout(p, n, k).total;
+}
+
+extern "C" int pf_simulate(pf_plan_t *p, const uint64_t *d_surv_idx, uint64_t n, const uint64_t *d_n,
+                           uint32_t jitter_seed, float *d_tput_sim, uint8_t *d_sim_status, uint32_t k,
+                           uint64_t *d_topk_idx, float *d_topk_score, uint32_t *d_topk_count, void *d_workspace,
+                           size_t workspace_bytes, void *stream)
+{
+    if (!p || !d_surv_idx) return PF_EINVAL;
+    if (p->dev.phase != PF_PHASE_TRAIN) return PF_EUNSUPPORTED;
+    if (k > PF_K_MAX) return PF_EINVAL;
+    if (k > 0 && (!d_topk_idx || !d_topk_score || !d_topk_count)) return PF_EINVAL;
+    if (n >= PF_MAX_COUNT) return PF_ERANGE;
+    const SimLayout lay = sim_layout(p, n, k);
+    if (!d_workspace || ((uintptr_t)d_workspace & 255) != 0 || workspace_bytes < lay.total) return PF_EWORKSPACE;
+    if (!p->sim_tables) return PF_EINVAL;
+    const SimTables *tab = (const SimTables *)p->sim_tables;
+    cudaStream_t st = (cudaStream_t)stream;
+    uint8_t *ws = (uint8_t *)d_workspace;
+    float *scores = d_tput_sim ? d_tput_sim : (float *)(ws + lay.off_scores);
+
+    SimArgs a;
+    a.surv = d_surv_idx; a.n = n; a.d_n = d_n; a.seed = jitter_seed;
+    a.tput_sim = scores; a.status = d_sim_status;
+    a.counter = (unsigned int *)(ws + lay.off_counter);
+    a.vals = p->d_vals; a.dual_ops = tab->d_ops; a.dual_off = tab->d_offset;
+    a.q_max = plan_q_max(p);
+    // as many warps per block as the shared-memory budget allows (each warp holds one candidate's timeline)
+    const size_t per_warp = sim_warp_floats(a.q_max) * sizeof(float);
+    int warps = (int)(kSimSmemBudget / per_warp);
+    warps = warps < 1 ? 1 : (warps > kSimMaxWarps ? kSimMaxWarps : warps);
+    const size_t smem = (size_t)warps * per_warp;
+    if (smem > 227 * 1024) return PF_EUNSUPPORTED;
+    const int kSimThreads = warps * 32;
+    PF_CUDA_TRY(cudaMemsetAsync(a.counter, 0, 256, st), "pf_simulate: counter reset");
+    if (n > 0) {
+        uint64_t want = (n + warps - 1) / warps;
+        int per_sm = (int)((size_t)(227 * 1024) / (smem + 1024));
+        per_sm = per_sm < 1 ? 1 : (per_sm > 4 ? 4 : per_sm);
+        uint64_t cap = (uint64_t)p->sm_count * per_sm;
+        int grid = (int)(want < cap ? want : cap);
+        if (p->dev.wide) {
+            PF_CUDA_TRY(cudaFuncSetAttribute(simulate_kernel<unsigned long long>,
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem),
+                        "simulate_kernel smem");
+            simulate_kernel<unsigned long long><<<grid, kSimThreads, smem, st>>>(p->dev, a);
+        } else {
+            PF_CUDA_TRY(cudaFuncSetAttribute(simulate_kernel<uint32_t>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)smem),
+                        "simulate_kernel smem");
+            simulate_kernel<uint32_t><<<grid, kSimThreads, smem, st>>>(p->dev, a);
+        }
+        count_launch();
+        PF_CUDA_TRY(cudaGetLastError(), "simulate_kernel launch");
+    }
+    if (k > 0) {
+        DenseTopkArgs t;
+        t.score = scores; t.n = n; t.d_n = d_n; t.k = k;
+        t.lists = (unsigned long long *)(ws + lay.off_topk + lay.tk.off_lists_a);
+        dense_topk_kernel<<<lay.topk_blocks, kThreads, 0, st>>>(t);
+        count_launch();
+        PF_CUDA_TRY(cudaGetLastError(), "dense_topk_kernel launch");
+        return launch_topk_reduce(t.lists, (unsigned long long *)(ws + lay.off_topk + lay.tk.off_lists_b),
+                                  lay.topk_blocks, k, 0, d_surv_idx, d_topk_idx, d_topk_score, d_topk_count, st);
+    }
+    return PF_OK;
+}
