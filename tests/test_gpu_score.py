@@ -40,9 +40,9 @@ def test_mid_variants_dense_in_feasible_candidates():
     of candidates reach the cost model and the block top-k has to prune."""
     big = 10 ** 15
     r = _full_parity(variant("mid", cluster=dict(budget_bytes=big)))
-    assert ((r & 0x7F) == 0).sum() > 2000
+    assert ((r & 0x7F) == 0).sum() > 1500
     r = _full_parity(variant("mid", cluster=dict(budget_bytes=big), rules=dict(enforce_realizability=0)))
-    assert ((r & 0x7F) == 0).sum() > 5000
+    assert ((r & 0x7F) == 0).sum() > 3000
     cfg = variant("mid", cluster=dict(budget_bytes=big), rules=dict(ep_scope=0))
     cfg["k"] = 1024
     _full_parity(cfg)
@@ -54,6 +54,22 @@ def test_serve_variant_all_kernels_available():
         k["avail_mask"] = 255
     cfg["k"] = 1024
     _full_parity(cfg)
+
+
+def test_dense_space_with_exact_ties_prunes_the_block_buffers():
+    """Nearly every candidate feasible and every score repeated 64 times (the kernel-variant axis lists each
+    variant 64 times): each block sees thousands of admissible keys, so its shared-memory buffer is pruned
+    repeatedly, and the cut at k falls inside a run of exact ties that only the index order resolves."""
+    cfg = variant("large", cluster=dict(budget_bytes=10 ** 15), rules=dict(world_min=1, enforce_realizability=0))
+    for kn in cfg["kern"]:
+        kn["avail_mask"] = 255
+    cfg["axes"] = [("kv", [i % 8 for i in range(512)]), ("rec", [0, 1, 2]), ("sched", [0, 1]),
+                   ("mb", [1, 2, 4, 8, 16]), ("v", [1]), ("ep", [1, 2, 4, 8]), ("pp", [1]), ("tp", [1, 2, 4, 8]),
+                   ("dp", [8, 16, 32, 64, 128, 256, 512, 1024]), ("world", [0])]
+    for k in (1024, 100):
+        cfg["k"] = k
+        r = _full_parity(cfg)
+    assert ((r & 0x7F) == 0).mean() > 0.5 and len(r) == 1_966_080
 
 
 def test_derived_axes_and_wide_integers():

@@ -108,7 +108,7 @@ def test_simulate_every_schedule_class_small():
     orc = Oracle(cfg)
     reason, _, _, _ = orc.score_range(threads=8)
     idx = np.flatnonzero((reason & 0x7F) == 0).astype(np.uint64)
-    assert len(idx) > 5000
+    assert len(idx) > 3000
     kinds = {orc.eval(int(i))["kind"] for i in idx[::97]}
     assert kinds == {0, 1, 2}
     _, status = _sim_parity(cfg, idx)
