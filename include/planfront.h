@@ -257,6 +257,16 @@ int pf_search_host(pf_plan_t *plan, uint32_t k, uint64_t s_max, uint32_t k_sim, 
                    uint32_t *h_sim_topk_count, uint64_t *h_surv_count, void *d_workspace,
                    size_t workspace_bytes, void *stream);
 
+/* Optional device timing of the library's own kernels, by class, for roofline accounting (the paper has
+ * no counterpart).  While enabled, every call brackets the launches of each class with a CUDA event pair
+ * on the caller's stream; pf_timing_read waits for the recorded events, adds the elapsed times (ms) and
+ * kernel counts per class into ms[PF_T_CLASSES] / kernels[PF_T_CLASSES], and forgets them.
+ * PF_T_SCORE: the scoring kernel; PF_T_TOPK: top-k list kernels (merge passes, dense top-k);
+ * PF_T_SELECT: the survivor-selection kernels; PF_T_SIMULATE: the simulator kernel. */
+enum { PF_T_SCORE = 0, PF_T_TOPK = 1, PF_T_SELECT = 2, PF_T_SIMULATE = 3, PF_T_CLASSES = 4 };
+int pf_timing_enable(pf_plan_t *plan, int on);
+int pf_timing_read(pf_plan_t *plan, float *ms, uint32_t *kernels);
+
 /* Number of kernels this library has launched in this process (for launch accounting in benchmarks). */
 uint64_t pf_launch_count(void);
 

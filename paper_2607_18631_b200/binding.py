@@ -23,7 +23,8 @@ UINT64_MAX = 0xFFFFFFFFFFFFFFFF
 EXPORTS = ("pf_version", "pf_strerror", "pf_reason_str", "pf_last_cuda_error", "pf_plan_create", "pf_plan_destroy",
            "pf_plan_size", "pf_decode", "pf_score_workspace", "pf_score", "pf_topk_merge", "pf_select_workspace",
            "pf_select_survivors", "pf_simulate_workspace", "pf_simulate", "pf_search_workspace", "pf_search_host",
-           "pf_launch_count", "pf_dualpipe_order")
+           "pf_launch_count", "pf_dualpipe_order", "pf_timing_enable", "pf_timing_read")
+T_CLASSES = ("score", "topk", "select", "simulate")
 
 i32, u32, i64, u64, f32 = C.c_int32, C.c_uint32, C.c_int64, C.c_uint64, C.c_float
 
@@ -125,6 +126,10 @@ def load_library(path: str | None = None):
     L.pf_search_host.restype = C.c_int
     L.pf_search_host.argtypes = [vp, u32, u64, u32, u32, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     L.pf_launch_count.restype = u64
+    L.pf_timing_enable.restype = C.c_int
+    L.pf_timing_enable.argtypes = [vp, C.c_int]
+    L.pf_timing_read.restype = C.c_int
+    L.pf_timing_read.argtypes = [vp, vp, vp]
     L.pf_dualpipe_order.restype = C.c_int
     L.pf_dualpipe_order.argtypes = [C.c_int, C.c_int, vp]
     if path == LIB_PATH:
@@ -243,6 +248,18 @@ class Plan:
             self.close()
         except Exception:
             pass
+
+    # ---- pf_timing_enable / pf_timing_read
+    def timing_enable(self, on: bool = True):
+        _check(self._L.pf_timing_enable(self._h, 1 if on else 0), "pf_timing_enable")
+
+    def timing_read(self) -> dict:
+        """{class: (milliseconds, kernels)} accumulated since the last read; waits for the recorded events."""
+        ms = np.zeros(len(T_CLASSES), dtype=np.float32)
+        nk = np.zeros(len(T_CLASSES), dtype=np.uint32)
+        _check(self._L.pf_timing_read(self._h, ms.ctypes.data_as(C.c_void_p), nk.ctypes.data_as(C.c_void_p)),
+               "pf_timing_read")
+        return {n: (float(ms[i]), int(nk[i])) for i, n in enumerate(T_CLASSES)}
 
     # ---- pf_decode
     def decode(self, idx: int) -> dict:

@@ -5,6 +5,7 @@
 #include <cstdlib>
 #include <cstring>
 #include <new>
+#include <vector>
 
 #include "pf_internal.cuh"
 
@@ -18,6 +19,48 @@ void set_cuda_error(cudaError_t e, const char *where)
     snprintf(g_cuda_msg, sizeof(g_cuda_msg), "%s: %s", where, cudaGetErrorString(e));
 }
 void count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
+
+struct TimingRec {
+    int cls, n_kernels;
+    cudaEvent_t a, b;
+};
+struct Timing {
+    bool on = false;
+    std::vector<TimingRec> recs;
+    std::vector<cudaEvent_t> pool;
+    cudaEvent_t get()
+    {
+        if (!pool.empty()) {
+            cudaEvent_t e = pool.back();
+            pool.pop_back();
+            return e;
+        }
+        cudaEvent_t e = nullptr;
+        cudaEventCreate(&e);
+        return e;
+    }
+};
+
+void timing_begin(pf_plan_t *p, int cls, cudaStream_t st)
+{
+    Timing *t = (Timing *)p->timing;
+    if (!t || !t->on) return;
+    TimingRec r;
+    r.cls = cls;
+    r.n_kernels = 0;
+    r.a = t->get();
+    r.b = t->get();
+    cudaEventRecord(r.a, st);
+    t->recs.push_back(r);
+}
+
+void timing_end(pf_plan_t *p, int cls, int n_kernels, cudaStream_t st)
+{
+    Timing *t = (Timing *)p->timing;
+    if (!t || !t->on || t->recs.empty() || t->recs.back().cls != cls) return;
+    t->recs.back().n_kernels = n_kernels;
+    cudaEventRecord(t->recs.back().b, st);
+}
 
 }  // namespace pf
 
@@ -321,9 +364,45 @@ extern "C" int pf_plan_create(const pf_model_t *model, const pf_cluster_t *clust
     return PF_OK;
 }
 
+extern "C" int pf_timing_enable(pf_plan_t *p, int on)
+{
+    if (!p) return PF_EINVAL;
+    if (!p->timing) p->timing = new pf::Timing;
+    ((pf::Timing *)p->timing)->on = on != 0;
+    return PF_OK;
+}
+
+extern "C" int pf_timing_read(pf_plan_t *p, float *ms, uint32_t *kernels)
+{
+    if (!p || !ms || !kernels) return PF_EINVAL;
+    for (int i = 0; i < PF_T_CLASSES; i++) ms[i] = 0.f, kernels[i] = 0;
+    pf::Timing *t = (pf::Timing *)p->timing;
+    if (!t) return PF_OK;
+    for (auto &r : t->recs) {
+        float x = 0.f;
+        PF_CUDA_TRY(cudaEventSynchronize(r.b), "pf_timing_read");
+        PF_CUDA_TRY(cudaEventElapsedTime(&x, r.a, r.b), "pf_timing_read");
+        ms[r.cls] += x;
+        kernels[r.cls] += (uint32_t)r.n_kernels;
+        t->pool.push_back(r.a);
+        t->pool.push_back(r.b);
+    }
+    t->recs.clear();
+    return PF_OK;
+}
+
 extern "C" void pf_plan_destroy(pf_plan_t *p)
 {
     if (!p) return;
+    if (p->timing) {
+        pf::Timing *t = (pf::Timing *)p->timing;
+        for (auto &r : t->recs) {
+            cudaEventDestroy(r.a);
+            cudaEventDestroy(r.b);
+        }
+        for (auto e : t->pool) cudaEventDestroy(e);
+        delete t;
+    }
     pf::free_sim_tables(p);
     if (p->d_vals) cudaFree(p->d_vals);
     if (p->d_scen) cudaFree(p->d_scen);

@@ -11,7 +11,6 @@ namespace pf {
 
 constexpr int kThreads = 256;        // threads per block of the scoring kernel
 constexpr int kTopkCap = 2048;       // shared-memory candidate buffer per block (2 * PF_K_MAX)
-constexpr int kMergeGroup = 32;      // lists merged per block in one merge pass
 constexpr uint32_t kSlabMax = 16384; // upper bound on candidates per slab (inner-axis product)
 
 struct DevSched {
@@ -75,8 +74,10 @@ struct pf_plan {
     // device buffers owned by the handle
     int32_t *d_vals;               // packed axis value lists
     int32_t *d_scen;               // serve: P[n_scen] then O[n_scen]
-    // simulator order tables (built lazily by the simulator unit)
+    // simulator order tables (built at create for training plans)
     void *sim_tables;
+    // optional per-kernel-class event timing (pf_timing_enable)
+    void *timing;
 };
 
 namespace pf {
@@ -84,6 +85,9 @@ namespace pf {
 // ------------------------------------------------------------------ error plumbing (host)
 void set_cuda_error(cudaError_t e, const char *where);
 void count_launch();
+// event pair around the launches of one kernel class; no-ops unless pf_timing_enable(plan, 1)
+void timing_begin(pf_plan_t *p, int cls, cudaStream_t st);
+void timing_end(pf_plan_t *p, int cls, int n_kernels, cudaStream_t st);
 #define PF_CUDA_TRY(expr, where)                        \
     do {                                                \
         cudaError_t e__ = (expr);                       \
@@ -109,14 +113,14 @@ __device__ __forceinline__ uint32_t key_rel(unsigned long long key) { return 0xF
 // threshold (the k-th best key once k are held, else 0).  All functions are block-collective unless
 // noted; the block may have any multiple of 32 threads.
 
-// Descending bitonic sort of buf[0, kTopkCap) in shared memory.
-__device__ inline void tk_sort_desc(unsigned long long *buf)
+// Descending bitonic sort of buf[0, n_sort) in shared memory; n_sort a power of two <= kTopkCap.
+__device__ inline void tk_sort_desc(unsigned long long *buf, int n_sort)
 {
     const int tid = threadIdx.x, nt = blockDim.x;
-    for (int size = 2; size <= kTopkCap; size <<= 1) {
+    for (int size = 2; size <= n_sort; size <<= 1) {
         for (int stride = size >> 1; stride > 0; stride >>= 1) {
             __syncthreads();
-            for (int i = tid; i < kTopkCap / 2; i += nt) {
+            for (int i = tid; i < n_sort / 2; i += nt) {
                 int lo = 2 * i - (i & (stride - 1));  // element with the stride bit clear
                 int hi = lo + stride;
                 bool desc = ((lo & size) == 0);       // direction of this bitonic block
@@ -132,20 +136,33 @@ __device__ inline void tk_sort_desc(unsigned long long *buf)
     __syncthreads();
 }
 
-// Keep the best k: sort, clamp the count, refresh the threshold.
+// Keep the best k: sort what is held (padded to a power of two), clamp the count, refresh the threshold.
 __device__ inline void tk_prune(unsigned long long *buf, int *count, unsigned long long *thr, int k)
 {
     __syncthreads();
     int c = *count;
     if (c > kTopkCap) c = kTopkCap;
-    for (int i = c + threadIdx.x; i < kTopkCap; i += blockDim.x) buf[i] = 0ull;
-    tk_sort_desc(buf);
+    int n_sort = 32;
+    while (n_sort < c) n_sort <<= 1;
+    for (int i = c + threadIdx.x; i < n_sort; i += blockDim.x) buf[i] = 0ull;
+    tk_sort_desc(buf, n_sort);
     if (threadIdx.x == 0) {
         int n = c < k ? c : k;
         *count = n;
         *thr = (n == k) ? buf[k - 1] : 0ull;
     }
     __syncthreads();
+}
+
+// Append the block's held keys (after tk_prune: sorted, *count of them) to a compact global key list.
+// s_base: one shared int of scratch.  Block-collective.
+__device__ inline void tk_flush(const unsigned long long *buf, int c, int *s_base, unsigned long long *out_keys,
+                                unsigned int *out_count)
+{
+    if (threadIdx.x == 0) *s_base = c > 0 ? (int)atomicAdd(out_count, (unsigned int)c) : 0;
+    __syncthreads();
+    unsigned long long *out = out_keys + *s_base;
+    for (int i = threadIdx.x; i < c; i += blockDim.x) out[i] = buf[i];
 }
 
 // Append this thread's key if it beats the threshold.  Warp-collective (all 32 lanes must call); the
@@ -167,29 +184,33 @@ __device__ __forceinline__ void tk_push(unsigned long long *buf, int *count, uns
     }
 }
 
-// host: workspace layout of one top-k reduction with `nblocks` producers
+// host: workspace layout of one top-k reduction whose producers append at most n_keys_max keys in total.
+// ctrl is 256 bytes of uint32: [0] producer work counter, [1] keys in list A, [2] keys in list B, [3] spare.
+constexpr int kReduceSeg = 32768;    // keys one block of the reduce kernel walks through
+constexpr int kReduceThreads = 1024;
 struct TopkLayout {
-    size_t off_ctrl, off_lists_a, off_lists_b, total;
-    int n_b;  // lists after the first merge pass
+    size_t off_ctrl, off_keys_a, off_keys_b, total;
 };
-inline TopkLayout topk_layout(int nblocks, uint32_t k)
+inline TopkLayout topk_layout(uint64_t n_keys_max, uint32_t k)
 {
     TopkLayout l;
     size_t kk = k ? k : 1;
+    if (n_keys_max < kk) n_keys_max = kk;
     l.off_ctrl = 0;
-    l.off_lists_a = 256;
-    size_t a = ((size_t)nblocks * kk * 8 + 255) & ~(size_t)255;
-    l.n_b = (nblocks + kMergeGroup - 1) / kMergeGroup;
-    size_t b = ((size_t)l.n_b * kk * 8 + 255) & ~(size_t)255;
-    l.off_lists_b = l.off_lists_a + a;
-    l.total = l.off_lists_b + b;
+    l.off_keys_a = 256;
+    size_t a = ((size_t)n_keys_max * 8 + 255) & ~(size_t)255;
+    size_t blocks = (n_keys_max + kReduceSeg - 1) / kReduceSeg;
+    size_t b = (blocks * kk * 8 + 255) & ~(size_t)255;
+    l.off_keys_b = l.off_keys_a + a;
+    l.total = l.off_keys_b + b;
     return l;
 }
 
-// host: merge `n_lists` per-block key lists (k keys each, zero padded) down to the final outputs.
+// host: reduce a compact key list (device count in ctrl[1], at most n_keys_max keys) to the final outputs.
 // idx_map (device, may be NULL): final index = idx_map[rel] instead of first + rel.
-int launch_topk_reduce(unsigned long long *d_lists_a, unsigned long long *d_lists_b, int n_lists, uint32_t k,
-                       uint64_t first, const uint64_t *d_idx_map, uint64_t *d_topk_idx, float *d_topk_score,
-                       uint32_t *d_topk_count, cudaStream_t st);
+// Returns the number of kernels launched through *n_kernels.
+int launch_topk_reduce(void *d_workspace, const TopkLayout &lay, uint64_t n_keys_max, uint32_t k, uint64_t first,
+                       const uint64_t *d_idx_map, uint64_t *d_topk_idx, float *d_topk_score, uint32_t *d_topk_count,
+                       cudaStream_t st, int *n_kernels);
 
 }  // namespace pf

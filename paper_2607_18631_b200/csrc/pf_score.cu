@@ -22,7 +22,8 @@ struct ScoreArgs {
     uint8_t *reason;
     float *tput;
     long long *mem;
-    unsigned long long *lists;      // [gridDim.x][k] keys, zero padded
+    unsigned long long *keys;       // compact list of the blocks' best keys
+    unsigned int *key_count;        // its length (zeroed before launch)
     unsigned int *slab_counter;     // zeroed before launch
     const int32_t *vals;            // packed axis value lists
     const int32_t *scen;            // serve: P[n_scen], O[n_scen]
@@ -57,6 +58,7 @@ __global__ void __launch_bounds__(kThreads) score_kernel(const __grid_constant__
     __shared__ int s_count;
     __shared__ unsigned long long s_thr;
     __shared__ SlabInfo s_slab;
+    __shared__ int s_base;
 
     const int tid = threadIdx.x;
     const bool train = P.phase == PF_PHASE_TRAIN;
@@ -203,21 +205,19 @@ __global__ void __launch_bounds__(kThreads) score_kernel(const __grid_constant__
 
     if (want_topk) {
         tk_prune(s_buf, &s_count, &s_thr, (int)A.k);
-        unsigned long long *out = A.lists + (size_t)blockIdx.x * A.k;
-        const int c = s_count;
-        for (int i = tid; i < (int)A.k; i += kThreads) out[i] = i < c ? s_buf[i] : 0ull;
+        tk_flush(s_buf, s_count, &s_base, A.keys, A.key_count);
     }
 }
 
-// ------------------------------------------------------------------ merging per-block lists
+// ------------------------------------------------------------------ reducing a compact key list
 
-struct MergeArgs {
-    const unsigned long long *in;   // [n_lists][k]
-    unsigned long long *out;        // [gridDim.x][k] when not final
-    int n_lists;
+struct ReduceArgs {
+    const unsigned long long *in;   // compact keys
+    const unsigned int *in_count;
+    unsigned long long *out;        // compact keys of the next pass (when not final)
+    unsigned int *out_count;
     uint32_t k;
-    int group;                      // lists per block
-    int final;                      // 1: write idx / score / count instead of keys (gridDim.x must be 1)
+    int final;                      // 1: write idx / score / count (gridDim.x == 1)
     uint64_t first;
     const uint64_t *idx_map;        // NULL: idx = first + rel; else idx = idx_map[rel]
     uint64_t *topk_idx;
@@ -225,46 +225,37 @@ struct MergeArgs {
     uint32_t *topk_count;
 };
 
-__global__ void __launch_bounds__(kThreads) merge_kernel(const MergeArgs A)
+// Block b walks keys [b*kReduceSeg, (b+1)*kReduceSeg) of the input in buffer-sized rounds, keeping the k best.
+__global__ void __launch_bounds__(kReduceThreads) reduce_kernel(const ReduceArgs A)
 {
     __shared__ unsigned long long s_buf[kTopkCap];
     __shared__ int s_count;
     __shared__ unsigned long long s_thr;
+    __shared__ int s_base;
     const int tid = threadIdx.x, k = (int)A.k;
+    const unsigned int n = *A.in_count;
+    unsigned int pos = blockIdx.x * (unsigned int)kReduceSeg;
+    const unsigned int hi = min(pos + (unsigned int)kReduceSeg, n);
+    if (pos >= hi && !A.final) return;
     if (tid == 0) {
         s_count = 0;
         s_thr = 0ull;
     }
     __syncthreads();
-    const int l0 = blockIdx.x * A.group;
-    const int l1 = min(l0 + A.group, A.n_lists);
-    // each input list holds at most k keys; the buffer takes kTopkCap / k lists between prunes
-    const int per_round = max(1, (kTopkCap - k) / k);
-    for (int l = l0; l < l1; l += per_round) {
-        const int le = min(l + per_round, l1);
-        const int base = s_count;
-        const int total = (le - l) * k;
-        for (int i = tid; i < total; i += kThreads) {
-            unsigned long long key = A.in[(size_t)l * k + i];
-            s_buf[base + i] = key;  // zeros (empty slots) sort to the end
-        }
+    while (pos < hi) {
+        const int held = s_count;
+        const int take = min((unsigned int)(kTopkCap - held), hi - pos);
+        for (int i = tid; i < take; i += kReduceThreads) s_buf[held + i] = A.in[pos + i];
+        pos += take;
         __syncthreads();
-        if (tid == 0) s_count = base + total;
+        if (tid == 0) s_count = held + take;
         tk_prune(s_buf, &s_count, &s_thr, k);
-        // drop trailing empties from the count
-        if (tid == 0) {
-            int c = s_count;
-            while (c > 0 && s_buf[c - 1] == 0ull) c--;
-            s_count = c;
-        }
-        __syncthreads();
     }
     const int c = s_count;
     if (!A.final) {
-        unsigned long long *out = A.out + (size_t)blockIdx.x * k;
-        for (int i = tid; i < k; i += kThreads) out[i] = i < c ? s_buf[i] : 0ull;
+        tk_flush(s_buf, c, &s_base, A.out, A.out_count);
     } else {
-        for (int i = tid; i < k; i += kThreads) {
+        for (int i = tid; i < k; i += kReduceThreads) {
             if (i < c) {
                 unsigned long long key = s_buf[i];
                 uint32_t rel = key_rel(key);
@@ -279,26 +270,33 @@ __global__ void __launch_bounds__(kThreads) merge_kernel(const MergeArgs A)
     }
 }
 
-int launch_topk_reduce(unsigned long long *d_lists_a, unsigned long long *d_lists_b, int n_lists, uint32_t k,
-                       uint64_t first, const uint64_t *d_idx_map, uint64_t *d_topk_idx, float *d_topk_score,
-                       uint32_t *d_topk_count, cudaStream_t st)
+int launch_topk_reduce(void *d_workspace, const TopkLayout &lay, uint64_t n_keys_max, uint32_t k, uint64_t first,
+                       const uint64_t *d_idx_map, uint64_t *d_topk_idx, float *d_topk_score, uint32_t *d_topk_count,
+                       cudaStream_t st, int *n_kernels)
 {
-    unsigned long long *in = d_lists_a, *out = d_lists_b;
-    for (;;) {
-        MergeArgs m;
-        m.in = in; m.out = out; m.n_lists = n_lists; m.k = k; m.group = kMergeGroup;
-        m.first = first; m.idx_map = d_idx_map;
-        m.topk_idx = d_topk_idx; m.topk_score = d_topk_score; m.topk_count = d_topk_count;
-        int n_out = (n_lists + kMergeGroup - 1) / kMergeGroup;
-        m.final = n_out == 1;
-        merge_kernel<<<n_out, kThreads, 0, st>>>(m);
+    uint8_t *ws = (uint8_t *)d_workspace;
+    unsigned int *ctrl = (unsigned int *)(ws + lay.off_ctrl);
+    unsigned long long *in = (unsigned long long *)(ws + lay.off_keys_a);
+    unsigned long long *out = (unsigned long long *)(ws + lay.off_keys_b);
+    int in_slot = 1, out_slot = 2;
+    *n_kernels = 0;
+    for (int pass = 0; pass < 3; pass++) {
+        const uint64_t blocks = (n_keys_max + kReduceSeg - 1) / kReduceSeg;
+        ReduceArgs r;
+        r.in = in; r.in_count = ctrl + in_slot; r.out = out; r.out_count = ctrl + out_slot;
+        r.k = k; r.final = blocks <= 1; r.first = first; r.idx_map = d_idx_map;
+        r.topk_idx = d_topk_idx; r.topk_score = d_topk_score; r.topk_count = d_topk_count;
+        reduce_kernel<<<(unsigned int)(blocks < 1 ? 1 : blocks), kReduceThreads, 0, st>>>(r);
         count_launch();
-        PF_CUDA_TRY(cudaGetLastError(), "merge_kernel launch");
-        if (n_out == 1) break;
-        n_lists = n_out;
+        (*n_kernels)++;
+        PF_CUDA_TRY(cudaGetLastError(), "reduce_kernel launch");
+        if (r.final) return PF_OK;
+        n_keys_max = blocks * k;
         unsigned long long *t = in; in = out; out = t;
+        in_slot = out_slot;
+        out_slot = 3;   // a third pass would need n_keys_max > 32768 * 32768 / k: never with k <= 1024 lists
     }
-    return PF_OK;
+    return PF_EINVAL;
 }
 
 // ------------------------------------------------------------------ merge of two finished top-k lists
@@ -390,7 +388,7 @@ extern "C" size_t pf_score_workspace(const pf_plan_t *p, uint64_t count, uint32_
     if (!p || count == 0) return 256;
     uint64_t slab_lo, n_slabs;
     slab_span(p, 0, count + p->dev.slab, slab_lo, n_slabs);  // any alignment of `first`
-    return topk_layout(grid_for(p, n_slabs), k).total;
+    return topk_layout((uint64_t)grid_for(p, n_slabs) * k, k).total;
 }
 
 extern "C" int pf_score(pf_plan_t *p, uint64_t first, uint64_t count, uint8_t *d_reason, float *d_tput,
@@ -409,25 +407,33 @@ extern "C" int pf_score(pf_plan_t *p, uint64_t first, uint64_t count, uint8_t *d
     uint64_t slab_lo, n_slabs;
     slab_span(p, first, count, slab_lo, n_slabs);
     const int grid = grid_for(p, n_slabs);
-    const TopkLayout lay = topk_layout(grid, k);
+    const TopkLayout lay = topk_layout((uint64_t)grid * k, k);
     uint8_t *ws = (uint8_t *)d_workspace;
 
     ScoreArgs a;
     a.first = first; a.count = count; a.slab_lo = slab_lo; a.n_slabs = (uint32_t)n_slabs; a.k = k;
     a.reason = d_reason; a.tput = d_tput; a.mem = (long long *)d_mem;
-    a.lists = (unsigned long long *)(ws + lay.off_lists_a);
+    a.keys = (unsigned long long *)(ws + lay.off_keys_a);
     a.slab_counter = (unsigned int *)(ws + lay.off_ctrl);
+    a.key_count = a.slab_counter + 1;
     a.vals = p->d_vals; a.scen = p->d_scen;
     PF_CUDA_TRY(cudaMemsetAsync(a.slab_counter, 0, 256, st), "pf_score: counter reset");
+    timing_begin(p, PF_T_SCORE, st);
     if (p->dev.wide)
         score_kernel<unsigned long long><<<grid, kThreads, 0, st>>>(p->dev, a);
     else
         score_kernel<uint32_t><<<grid, kThreads, 0, st>>>(p->dev, a);
     count_launch();
+    timing_end(p, PF_T_SCORE, 1, st);
     PF_CUDA_TRY(cudaGetLastError(), "score_kernel launch");
-    if (k > 0)
-        return launch_topk_reduce(a.lists, (unsigned long long *)(ws + lay.off_lists_b), grid, k, first, nullptr,
-                                  d_topk_idx, d_topk_score, d_topk_count, st);
+    if (k > 0) {
+        timing_begin(p, PF_T_TOPK, st);
+        int nk = 0;
+        int rc = launch_topk_reduce(ws, lay, (uint64_t)grid * k, k, first, nullptr, d_topk_idx, d_topk_score,
+                                    d_topk_count, st, &nk);
+        timing_end(p, PF_T_TOPK, nk, st);
+        return rc;
+    }
     return PF_OK;
 }
 

@@ -111,31 +111,51 @@ __global__ void __launch_bounds__(kSelThreads) sel_hist_kernel(const __grid_cons
     }
 }
 
+// Block-wide inclusive prefix sum over 1024 threads (warp shuffles, then the warp totals).
+__device__ __forceinline__ unsigned long long block_prefix_1024(unsigned long long x, unsigned long long *s_warp)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        unsigned long long y = __shfl_up_sync(0xFFFFFFFFu, x, off);
+        if (lane >= off) x += y;
+    }
+    if (lane == 31) s_warp[warp] = x;
+    __syncthreads();
+    if (warp == 0) {
+        unsigned long long t = s_warp[lane];
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            unsigned long long y = __shfl_up_sync(0xFFFFFFFFu, t, off);
+            if (lane >= off) t += y;
+        }
+        s_warp[lane] = t;
+    }
+    __syncthreads();
+    if (warp > 0) x += s_warp[warp - 1];
+    __syncthreads();
+    return x;
+}
+
 // One block of 1024 threads: find the bin (scanning from the top) where the running count reaches the target.
 __global__ void __launch_bounds__(1024) sel_scan_kernel(const SelArgs A, int pass)
 {
-    __shared__ unsigned long long s_sum[1024];
-    __shared__ unsigned long long s_suffix[1025];
+    __shared__ unsigned long long s_warp[32];
+    __shared__ unsigned long long s_total;
     const int tid = threadIdx.x;
     SelCtrl *c = A.ctrl;
     if (pass == 1 && c->take_all) return;
     const unsigned int *hist = pass == 0 ? A.hist1 : A.hist2;
     constexpr int per = kBins / 1024;
-    // thread t owns bins [t*per, (t+1)*per)
+    // thread t owns bins [(1023-t)*per, (1024-t)*per): thread 0 holds the TOP bins, so an inclusive prefix
+    // over threads counts from the top
+    const int my_lo = (1023 - tid) * per;
     unsigned long long mine = 0;
-    for (int i = 0; i < per; i++) mine += hist[tid * per + i];
-    s_sum[tid] = mine;
+    for (int i = 0; i < per; i++) mine += hist[my_lo + i];
+    const unsigned long long incl = block_prefix_1024(mine, s_warp);
+    if (tid == 1023) s_total = incl;
     __syncthreads();
-    if (tid == 0) {
-        unsigned long long run = 0;
-        s_suffix[1024] = 0;
-        for (int t = 1023; t >= 0; t--) {
-            run += s_sum[t];
-            s_suffix[t] = run;  // count in bins >= t*per
-        }
-    }
-    __syncthreads();
-    const unsigned long long total = s_suffix[0];
+    const unsigned long long total = s_total;
     unsigned long long target;
     if (pass == 0) {
         target = A.s_max;
@@ -153,14 +173,14 @@ __global__ void __launch_bounds__(1024) sel_scan_kernel(const SelArgs A, int pas
     } else {
         target = c->target - c->above1;
     }
-    // the owner of the crossing: suffix above me < target <= suffix including me
-    const unsigned long long above = s_suffix[tid + 1];
-    if (above < target && above + mine >= target) {
+    // the owner of the crossing: count above my bins < target <= count including them
+    const unsigned long long above = incl - mine;
+    if (above < target && incl >= target) {
         unsigned long long run = above;
         for (int i = per - 1; i >= 0; i--) {
-            unsigned int h = hist[tid * per + i];
+            unsigned int h = hist[my_lo + i];
             if (run + h >= target) {
-                uint32_t bin = (uint32_t)(tid * per + i);
+                uint32_t bin = (uint32_t)(my_lo + i);
                 if (pass == 0) {
                     c->b1 = bin;
                     c->above1 = run;
@@ -202,20 +222,34 @@ __global__ void __launch_bounds__(kSelThreads) sel_count_kernel(const __grid_con
     }
 }
 
-// exclusive prefix over blocks (one thread: a few hundred entries) + the survivor count
-__global__ void sel_blockscan_kernel(const SelArgs A, int nblocks)
+// exclusive prefix over the per-block counts (tiles of 1024 blocks with a carry) + the survivor count
+__global__ void __launch_bounds__(1024) sel_blockscan_kernel(const SelArgs A, int nblocks)
 {
-    if (threadIdx.x != 0 || blockIdx.x != 0) return;
-    unsigned long long g = 0, q = 0;
-    for (int b = 0; b < nblocks; b++) {
-        unsigned long long cg = A.blk_gt[b], ce = A.blk_eq[b];
-        A.blk_gt[b] = g;
-        A.blk_eq[b] = q;
-        g += cg;
-        q += ce;
+    __shared__ unsigned long long s_warp[32];
+    __shared__ unsigned long long s_carry_g, s_carry_e;
+    const int tid = threadIdx.x;
+    if (tid == 0) s_carry_g = s_carry_e = 0;
+    __syncthreads();
+    for (int base = 0; base < nblocks; base += 1024) {
+        const int b = base + tid;
+        const unsigned long long cg = b < nblocks ? A.blk_gt[b] : 0, ce = b < nblocks ? A.blk_eq[b] : 0;
+        const unsigned long long ig = block_prefix_1024(cg, s_warp);
+        const unsigned long long ie = block_prefix_1024(ce, s_warp);
+        if (b < nblocks) {
+            A.blk_gt[b] = s_carry_g + ig - cg;
+            A.blk_eq[b] = s_carry_e + ie - ce;
+        }
+        __syncthreads();
+        if (tid == 1023) {
+            s_carry_g += ig;
+            s_carry_e += ie;
+        }
+        __syncthreads();
     }
-    const SelCtrl *c = A.ctrl;
-    *A.surv_count = c->take_all ? c->total : c->target;
+    if (tid == 0) {
+        const SelCtrl *c = A.ctrl;
+        *A.surv_count = c->take_all ? c->total : c->target;
+    }
 }
 
 // Ordered write: position of an admitted candidate = (# taken "greater" before it) + min(# "equal" before it, need_eq)
@@ -334,13 +368,15 @@ extern "C" int pf_select_survivors(pf_plan_t *p, uint64_t first, uint64_t count,
     a.blk_eq = (unsigned long long *)(ws + lay.off_eq);
     a.surv_idx = d_surv_idx; a.surv_count = d_surv_count; a.chunk = lay.chunk;
     PF_CUDA_TRY(cudaMemsetAsync(ws, 0, lay.off_gt, st), "pf_select_survivors: clear");
+    timing_begin(p, PF_T_SELECT, st);
     sel_hist_kernel<<<lay.nblocks, kSelThreads, 0, st>>>(p->dev, a, p->d_vals, 0);
     sel_scan_kernel<<<1, 1024, 0, st>>>(a, 0);
     sel_hist_kernel<<<lay.nblocks, kSelThreads, 0, st>>>(p->dev, a, p->d_vals, 1);
     sel_scan_kernel<<<1, 1024, 0, st>>>(a, 1);
     sel_count_kernel<<<lay.nblocks, kSelThreads, 0, st>>>(p->dev, a, p->d_vals);
-    sel_blockscan_kernel<<<1, 32, 0, st>>>(a, lay.nblocks);
+    sel_blockscan_kernel<<<1, 1024, 0, st>>>(a, lay.nblocks);
     sel_write_kernel<<<lay.nblocks, kSelThreads, 0, st>>>(p->dev, a, p->d_vals);
+    timing_end(p, PF_T_SELECT, 7, st);
     for (int i = 0; i < 7; i++) count_launch();
     PF_CUDA_TRY(cudaGetLastError(), "pf_select_survivors launch");
     return PF_OK;

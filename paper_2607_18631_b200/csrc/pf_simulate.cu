@@ -19,7 +19,6 @@
 namespace pf {
 
 constexpr int kSimMaxWarps = 16;        // warps per block at most (each simulates one candidate at a time)
-constexpr int kSimSmemBudget = 200 * 1024;  // dynamic shared memory a block may take
 
 // DualPipe-style order tables: for every (pp, m) in the domain a byte string per rank,
 // op = (j << 2) | (dir << 1) | is_backward, 2*m ops per rank.
@@ -108,9 +107,11 @@ int build_sim_tables(pf_plan_t *p)
     t->d_offset = nullptr;
     t->h_offset.assign(33 * 33, -1);
     std::vector<uint8_t> ops;
-    // only if the plan has a DualPipe-class schedule; depths from the pp axis (1 or even, <= 32)
+    // only if a DualPipe-class schedule can pass the dry-run rules (mapped, or unconstrained mode);
+    // depths from the pp axis (1 or even, <= 32)
     bool any_dual = false;
-    for (int s = 0; s < p->dev.n_sched; s++) any_dual |= p->dev.sched[s].kind == PF_KIND_DUALPIPE;
+    for (int s = 0; s < p->dev.n_sched; s++)
+        any_dual |= p->dev.sched[s].kind == PF_KIND_DUALPIPE && (p->dev.sched[s].mapped || !p->dev.enforce);
     if (any_dual && p->dev.phase == PF_PHASE_TRAIN) {
         const int32_t *pps = p->h_vals + p->dev.val_off[6];
         for (int i = 0; i < p->axis_len[6]; i++) {
@@ -178,6 +179,9 @@ __device__ __forceinline__ float jitter(uint32_t seed_mixed, uint64_t idx, int q
     return 0.9f + 0.2f * u;
 }
 
+constexpr int kSimClasses = 7;          // timeline sizes 256 << c entries (stage streams x microbatches)
+__host__ __device__ inline int sim_class_entries(int c) { return 256 << c; }
+
 struct SimArgs {
     const uint64_t *surv;
     uint64_t n;
@@ -185,44 +189,96 @@ struct SimArgs {
     uint32_t seed;
     float *tput_sim;
     uint8_t *status;
-    unsigned int *counter;          // work queue, zeroed before launch
+    unsigned int *work;             // [kSimClasses] work-queue heads, zeroed before launch
+    unsigned int *cls_count;        // [kSimClasses] list lengths, zeroed before the classify kernel
+    uint32_t *cls_list;             // [kSimClasses][n] positions in surv, grouped by timeline size
     const int32_t *vals;
     const uint8_t *dual_ops;
     const int32_t *dual_off;
     int q_max;                      // stages per candidate at most (plan-wide)
+    int cls;                        // class this launch serves
 };
 
-// per-warp shared memory: endF[q_max*64], endB[q_max*64], durF[q_max], durB[q_max], cntF[q_max*2], cntB[q_max*2]
-__host__ __device__ inline size_t sim_warp_floats(int q_max) { return (size_t)q_max * (2 * PF_SIM_WINDOW + 2 + 4); }
+// Pre-pass: one thread per survivor computes how many timeline entries its simulation needs and files the
+// survivor under the smallest class that holds them, so each class can run with as many warps per SM as its
+// shared-memory footprint allows.  Entries that cannot be simulated (outside the domain, malformed) go to
+// class 0, where the simulator kernel rejects them before touching the timeline.
+template <typename RI>
+__global__ void __launch_bounds__(256) sim_classify_kernel(const __grid_constant__ DevPlan P, const SimArgs A)
+{
+    uint64_t n = A.n;
+    if (A.d_n) {
+        uint64_t dn = *A.d_n;
+        n = dn < n ? dn : n;
+    }
+    const uint64_t w = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    int cls = -1;
+    if (w < n) {
+        uint64_t rem = A.surv[w];
+        int v[PF_MAX_AXES];
+#pragma unroll
+        for (int a = 0; a < PF_MAX_AXES; a++) {
+            uint64_t r = P.radix[a];
+            uint64_t q = rem / r;
+            v[a] = __ldg(A.vals + P.val_off[a] + (int)(rem - q * r));
+            rem = q;
+        }
+        const int s = v[2], mb = v[3], vv = v[4], pp = v[6], tp = v[7];
+        RI dp = (RI)v[8];
+        if (v[8] == 0) dp = (RI)v[9] / ((RI)tp * (RI)pp);
+        const int kind = P.sched[s].kind;
+        const int v_eff = vv == 0 ? (kind == PF_KIND_INTERLEAVED ? 2 : 1) : vv;
+        cls = 0;
+        const RI dpmb = dp * (RI)mb;
+        if (dpmb != 0 && pp <= PF_SIM_MAX_RANKS && v_eff <= PF_SIM_MAX_V) {
+            RI m = (RI)P.gbs / dpmb;
+            int m_sim = m < (RI)PF_SIM_WINDOW ? (int)m : PF_SIM_WINDOW;
+            if (kind == PF_KIND_INTERLEAVED) m_sim = (m_sim / pp) * pp;
+            const int streams = kind == PF_KIND_DUALPIPE ? pp : pp * v_eff;  // DualPipe: 2 directions x m/2
+            const int entries = streams * m_sim;
+            while (cls < kSimClasses - 1 && sim_class_entries(cls) < entries) cls++;
+            if (sim_class_entries(cls) < entries || streams > A.q_max) cls = 0;   // cannot be a feasible plan
+        }
+    }
+    // warp-aggregated append per class
+    for (int c = 0; c < kSimClasses; c++) {
+        const unsigned mask = __ballot_sync(0xFFFFFFFFu, cls == c);
+        if (mask == 0) continue;
+        const int lane = threadIdx.x & 31, leader = __ffs(mask) - 1;
+        unsigned int base = 0;
+        if (lane == leader) base = atomicAdd(A.cls_count + c, (unsigned int)__popc(mask));
+        base = __shfl_sync(0xFFFFFFFFu, base, leader);
+        if (cls == c) A.cls_list[(size_t)c * A.n + base + __popc(mask & ((1u << lane) - 1u))] = (uint32_t)w;
+    }
+}
+
+// per-warp shared memory of class c: endF[E], endB[E], durF[q_max], durB[q_max]
+__host__ __device__ inline size_t sim_warp_floats(int entries, int q_max) { return (size_t)2 * entries + 2 * q_max; }
 
 template <typename RI>
 __global__ void __launch_bounds__(kSimMaxWarps * 32) simulate_kernel(const __grid_constant__ DevPlan P, const SimArgs A)
 {
     extern __shared__ float s_mem[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    float *base = s_mem + (size_t)warp * sim_warp_floats(A.q_max);
-    // end times and per-stage completion counters are written by one lane and read by its neighbours
-    // within a round: volatile accesses plus a block-level fence between "value" and "counter" keep the
-    // pair ordered
+    const int E = sim_class_entries(A.cls);
+    float *base = s_mem + (size_t)warp * sim_warp_floats(E, A.q_max);
+    // End times are written by the lane that owns the stage and polled by its neighbour: one 32-bit word per
+    // op, negative while the op has not finished, so a single volatile load answers "done, and when".
     volatile float *endF = base;
-    volatile float *endB = endF + (size_t)A.q_max * PF_SIM_WINDOW;
-    float *durF = base + (size_t)2 * A.q_max * PF_SIM_WINDOW;
+    volatile float *endB = base + E;
+    float *durF = base + 2 * (size_t)E;
     float *durB = durF + A.q_max;
-    volatile int *cntF = reinterpret_cast<int *>(durB + A.q_max);
-    volatile int *cntB = cntF + 2 * A.q_max;
 
-    uint64_t n = A.n;
-    if (A.d_n) {
-        uint64_t dn = *A.d_n;
-        n = dn < n ? dn : n;
-    }
+    const unsigned int n_cls = A.cls_count[A.cls];
+    const uint32_t *list = A.cls_list + (size_t)A.cls * A.n;
     const uint32_t seed_mixed = mix32(A.seed + 0x9e3779b9u);
 
     for (;;) {
-        unsigned int w = 0;
-        if (lane == 0) w = atomicAdd(A.counter, 1u);
-        w = __shfl_sync(0xFFFFFFFFu, w, 0);
-        if ((uint64_t)w >= n) break;
+        unsigned int wi = 0;
+        if (lane == 0) wi = atomicAdd(A.work + A.cls, 1u);
+        wi = __shfl_sync(0xFFFFFFFFu, wi, 0);
+        if (wi >= n_cls) break;
+        const uint32_t w = list[wi];
         const uint64_t idx = A.surv[w];
 
         // ---- every lane re-derives the candidate (uniform across the warp)
@@ -272,20 +328,25 @@ __global__ void __launch_bounds__(kSimMaxWarps * 32) simulate_kernel(const __gri
         const long long m = (long long)D.m;
         int m_sim = m < PF_SIM_WINDOW ? (int)m : PF_SIM_WINDOW;
         if (kind == PF_KIND_INTERLEAVED) m_sim = (m_sim / pp) * pp;
-        const int nj = dual ? m_sim / 2 : m_sim;  // microbatches per stage stream
+        const int nj = dual ? m_sim / 2 : m_sim;      // microbatches per stage stream
+        const int n_entries = (dual ? 2 * Q : Q) * nj;
+        bool stalled = n_entries > E || Q > A.q_max;  // filed under a class that cannot hold it: never for a
+                                                      // feasible plan, reported instead of overrunning
 
-        // ---- stage durations: balanced layer split, head on the last stage, jitter
+        // ---- stage durations (balanced layer split, head on the last stage, jitter) and cleared timeline
         __syncwarp();
-        const int L_lo = P.L / Q, L_rem = P.L - L_lo * Q;
-        for (int q = lane; q < Q; q += 32) {
-            const float nq = (float)(L_lo + (q < L_rem ? 1 : 0));
-            const bool last = q == Q - 1;
-            durF[q] = (nq * T.F_l + (last ? T.headF : 0.f)) * jitter(seed_mixed, idx, q, 0);
-            durB[q] = (nq * T.B_l + (last ? P.bwd_factor * T.headF : 0.f)) * jitter(seed_mixed, idx, q, 1);
-        }
-        for (int i = lane; i < 2 * Q; i += 32) {
-            cntF[i] = 0;
-            cntB[i] = 0;
+        if (!stalled) {
+            const int L_lo = P.L / Q, L_rem = P.L - L_lo * Q;
+            for (int q = lane; q < Q; q += 32) {
+                const float nq = (float)(L_lo + (q < L_rem ? 1 : 0));
+                const bool last = q == Q - 1;
+                durF[q] = (nq * T.F_l + (last ? T.headF : 0.f)) * jitter(seed_mixed, idx, q, 0);
+                durB[q] = (nq * T.B_l + (last ? P.bwd_factor * T.headF : 0.f)) * jitter(seed_mixed, idx, q, 1);
+            }
+            for (int i = lane; i < n_entries; i += 32) {
+                endF[i] = -1.f;
+                endB[i] = -1.f;
+            }
         }
         __syncwarp();
 
@@ -297,13 +358,11 @@ __global__ void __launch_bounds__(kSimMaxWarps * 32) simulate_kernel(const __gri
             warm = min(2 * (pp - lane - 1) + (v - 1) * pp, U);
         else
             warm = min(pp - lane - 1, U);
-        // forward / backward unit cursors as (group, chunk slot, slot-in-group) without divisions
         int nF = 0, nB = 0;               // units issued
-        int fg = 0, fc = 0, fw = 0;       // forward cursor: microbatch = fg*pp + fw, chunk = fc
-        int bg = 0, bc = 0, bw = 0;       // backward cursor: chunk = v-1-bc
+        int fc = 0, fw = 0, fg = 0;       // forward cursor: microbatch = fg*pp + fw, chunk = fc
+        int bc = 0, bw = 0, bg = 0;       // backward cursor: chunk = v-1-bc
         const uint8_t *dops = nullptr;
-        bool stalled = false;
-        if (dual) {
+        if (dual && !stalled) {
             const int off = __ldg(A.dual_off + pp * 33 + nj);
             if (off < 0) stalled = true;  // no table for this shape: report instead of reading out of bounds
             else dops = A.dual_ops + off + (size_t)lane * 2 * m_sim;
@@ -311,10 +370,11 @@ __global__ void __launch_bounds__(kSimMaxWarps * 32) simulate_kernel(const __gri
         float clock = 0.f;
         const int total_ops = (rank_active && !stalled) ? 2 * U : 0;
         int done_ops = 0;
+        int rounds = 0;
+        bool moved = false;
 
         for (;;) {
-            bool progressed = false;
-            // up to 4 ops per round keep the lanes that run ahead from waiting on the barrier
+            // up to 4 ops per round keep the lanes that run ahead from waiting on the vote
 #pragma unroll 1
             for (int rep = 0; rep < 4 && done_ops < total_ops; rep++) {
                 int isb, d = 0, q, j;
@@ -324,56 +384,41 @@ __global__ void __launch_bounds__(kSimMaxWarps * 32) simulate_kernel(const __gri
                     d = (op >> 1) & 1;
                     j = op >> 2;
                     q = d ? pp - 1 - lane : lane;
+                } else if (kind == PF_KIND_1F1B) {
+                    isb = !(nF < warm || (nF < U && nF - warm == nB));
+                    j = isb ? nB : nF;
+                    q = lane;
                 } else {
                     isb = !(nF < warm || (nF < U && nF - warm == nB));
-                    if (!isb) {
-                        j = fg * pp + fw;
-                        q = fc * pp + lane;
-                    } else {
-                        j = bg * pp + bw;
-                        q = (v - 1 - bc) * pp + lane;
-                    }
-                    if (kind == PF_KIND_1F1B) {
-                        j = isb ? nB : nF;
-                        q = lane;
-                    }
+                    j = isb ? bg * pp + bw : fg * pp + fw;
+                    q = (isb ? v - 1 - bc : fc) * pp + lane;
                 }
                 const int sidx = d * Q + q;          // stage stream (direction-major for DualPipe)
                 float dep = 0.f;
-                bool ready = true;
                 if (!isb) {
                     if (q > 0) {
-                        ready = cntF[sidx - 1] > j;
-                        if (ready) {
-                            __threadfence_block();
-                            dep = endF[(size_t)(sidx - 1) * nj + j] + T.p;
-                        }
+                        dep = endF[(sidx - 1) * nj + j];
+                        if (dep < 0.f) break;
+                        dep += T.p;
                     }
                 } else {
                     if (q < Q - 1) {
-                        ready = cntB[sidx + 1] > j;
-                        if (ready) {
-                            __threadfence_block();
-                            dep = endB[(size_t)(sidx + 1) * nj + j] + T.p;
-                        }
+                        dep = endB[(sidx + 1) * nj + j];
+                        if (dep < 0.f) break;
+                        dep += T.p;
                     }
                 }
-                if (!ready) break;
                 const float fin = fmaxf(clock, dep) + (isb ? durB[q] : durF[q]);
                 clock = fin;
                 if (!isb) {
-                    endF[(size_t)sidx * nj + j] = fin;
-                    __threadfence_block();
-                    cntF[sidx] = j + 1;
+                    endF[sidx * nj + j] = fin;
                     nF++;
                     if (++fw == pp) {
                         fw = 0;
                         if (++fc == v) fc = 0, fg++;
                     }
                 } else {
-                    endB[(size_t)sidx * nj + j] = fin;
-                    __threadfence_block();
-                    cntB[sidx] = j + 1;
+                    endB[sidx * nj + j] = fin;
                     nB++;
                     if (++bw == pp) {
                         bw = 0;
@@ -381,20 +426,22 @@ __global__ void __launch_bounds__(kSimMaxWarps * 32) simulate_kernel(const __gri
                     }
                 }
                 done_ops++;
-                progressed = true;
+                moved = true;
             }
-            __syncwarp();
-            const unsigned pending = __ballot_sync(0xFFFFFFFFu, done_ops < total_ops);
-            if (pending == 0) break;
-            if (!__any_sync(0xFFFFFFFFu, progressed)) {
-                stalled = true;
-                break;
+            if (!__any_sync(0xFFFFFFFFu, done_ops < total_ops)) break;
+            // bounded wait: every 64 rounds some lane must have advanced
+            if ((++rounds & 63) == 0) {
+                if (!__any_sync(0xFFFFFFFFu, moved)) {
+                    stalled = true;
+                    break;
+                }
+                moved = false;
             }
         }
 
         // ---- makespan, steady-state extension beyond the window, pricing
         float work = 0.f;
-        if (rank_active) {
+        if (rank_active && !stalled) {
             if (dual) {
                 work = 0.5f * (durF[lane] + durB[lane] + durF[pp - 1 - lane] + durB[pp - 1 - lane]);
             } else {
@@ -430,7 +477,8 @@ struct DenseTopkArgs {
     uint64_t n;
     const uint64_t *d_n;
     uint32_t k;
-    unsigned long long *lists;
+    unsigned long long *keys;
+    unsigned int *key_count;
 };
 
 __global__ void __launch_bounds__(kThreads) dense_topk_kernel(const DenseTopkArgs A)
@@ -438,6 +486,7 @@ __global__ void __launch_bounds__(kThreads) dense_topk_kernel(const DenseTopkArg
     __shared__ unsigned long long s_buf[kTopkCap];
     __shared__ int s_count;
     __shared__ unsigned long long s_thr;
+    __shared__ int s_base;
     const int tid = threadIdx.x;
     if (tid == 0) {
         s_count = 0;
@@ -465,28 +514,30 @@ __global__ void __launch_bounds__(kThreads) dense_topk_kernel(const DenseTopkArg
         room--;
     }
     tk_prune(s_buf, &s_count, &s_thr, (int)A.k);
-    unsigned long long *out = A.lists + (size_t)blockIdx.x * A.k;
-    const int c = s_count;
-    for (int i = tid; i < (int)A.k; i += kThreads) out[i] = i < c ? s_buf[i] : 0ull;
+    tk_flush(s_buf, s_count, &s_base, A.keys, A.key_count);
 }
 
 struct SimLayout {
-    size_t off_counter, off_scores, off_topk, total;
+    size_t off_ctrl, off_lists, off_scores, off_topk, total;
     int topk_blocks;
+    uint64_t topk_keys_max;
     TopkLayout tk;
 };
 
 static SimLayout sim_layout(const pf_plan_t *p, uint64_t n, uint32_t k)
 {
     SimLayout l;
-    l.off_counter = 0;
-    l.off_scores = 256;
-    size_t sc = ((size_t)(n ? n : 1) * 4 + 255) & ~(size_t)255;
-    l.off_topk = l.off_scores + sc;
+    const size_t nn = (size_t)(n ? n : 1);
+    l.off_ctrl = 0;                       // work[kSimClasses], cls_count[kSimClasses]
+    l.off_lists = 256;
+    l.off_scores = l.off_lists + (((size_t)kSimClasses * nn * 4 + 255) & ~(size_t)255);
+    l.off_topk = l.off_scores + ((nn * 4 + 255) & ~(size_t)255);
     uint64_t tb = (n + kThreads - 1) / kThreads;
     uint64_t cap = (uint64_t)p->sm_count * 2;
     l.topk_blocks = (int)(tb < 1 ? 1 : (tb > cap ? cap : tb));
-    l.tk = topk_layout(l.topk_blocks, k);
+    l.topk_keys_max = (uint64_t)l.topk_blocks * (k ? k : 1);
+    if (l.topk_keys_max > nn) l.topk_keys_max = nn < (k ? k : 1) ? (k ? k : 1) : nn;
+    l.tk = topk_layout(l.topk_keys_max, k);
     l.total = l.off_topk + (k ? l.tk.total : 0);
     return l;
 }
@@ -507,6 +558,42 @@ static int plan_q_max(const pf_plan_t *p)
     if (q > p->dev.L) q = p->dev.L;  // the layer rule admits pp*v <= L only
     if (q < pp_max) q = pp_max;
     return (int)q;
+}
+
+template <typename RI>
+static int launch_simulate(pf_plan_t *p, SimArgs a, uint64_t n, cudaStream_t st, int *n_kernels)
+{
+    *n_kernels = 0;
+    sim_classify_kernel<RI><<<(unsigned int)((n + 255) / 256), 256, 0, st>>>(p->dev, a);
+    count_launch();
+    (*n_kernels)++;
+    PF_CUDA_TRY(cudaGetLastError(), "sim_classify_kernel launch");
+    PF_CUDA_TRY(cudaFuncSetAttribute(simulate_kernel<RI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)(227 * 1024)),
+                "simulate_kernel smem");
+    // one launch per timeline-size class that the plan can produce
+    const int entries_max = a.q_max * PF_SIM_WINDOW;
+    for (int c = 0; c < kSimClasses; c++) {
+        if (c > 0 && sim_class_entries(c - 1) >= entries_max) break;
+        const size_t per_warp = sim_warp_floats(sim_class_entries(c), a.q_max) * sizeof(float);
+        if (per_warp > 227 * 1024) return PF_EUNSUPPORTED;
+        // blocks of up to 16 warps, at least two blocks per SM where the footprint allows
+        int warps = (int)((size_t)(110 * 1024) / per_warp);
+        if (warps < 1) warps = (int)((size_t)(227 * 1024) / per_warp);
+        warps = warps < 1 ? 1 : (warps > kSimMaxWarps ? kSimMaxWarps : warps);
+        const size_t smem = (size_t)warps * per_warp;
+        int per_sm = (int)((size_t)(227 * 1024) / (smem + 1024));
+        per_sm = per_sm < 1 ? 1 : (per_sm > 4 ? 4 : per_sm);
+        const uint64_t want = (n + warps - 1) / warps;
+        const uint64_t cap = (uint64_t)p->sm_count * per_sm;
+        const int grid = (int)(want < cap ? want : cap);
+        a.cls = c;
+        simulate_kernel<RI><<<grid, warps * 32, smem, st>>>(p->dev, a);
+        count_launch();
+        (*n_kernels)++;
+        PF_CUDA_TRY(cudaGetLastError(), "simulate_kernel launch");
+    }
+    return PF_OK;
 }
 
 }  // namespace pf
@@ -539,6 +626,7 @@ extern "C" int pf_simulate(pf_plan_t *p, const uint64_t *d_surv_idx, uint64_t n,
     const SimLayout lay = sim_layout(p, n, k);
     if (!d_workspace || ((uintptr_t)d_workspace & 255) != 0 || workspace_bytes < lay.total) return PF_EWORKSPACE;
     if (!p->sim_tables) return PF_EINVAL;
+    int rc = PF_OK;
     const SimTables *tab = (const SimTables *)p->sim_tables;
     cudaStream_t st = (cudaStream_t)stream;
     uint8_t *ws = (uint8_t *)d_workspace;
@@ -547,46 +635,37 @@ extern "C" int pf_simulate(pf_plan_t *p, const uint64_t *d_surv_idx, uint64_t n,
     SimArgs a;
     a.surv = d_surv_idx; a.n = n; a.d_n = d_n; a.seed = jitter_seed;
     a.tput_sim = scores; a.status = d_sim_status;
-    a.counter = (unsigned int *)(ws + lay.off_counter);
+    a.work = (unsigned int *)(ws + lay.off_ctrl);
+    a.cls_count = a.work + kSimClasses;
+    a.cls_list = (uint32_t *)(ws + lay.off_lists);
     a.vals = p->d_vals; a.dual_ops = tab->d_ops; a.dual_off = tab->d_offset;
     a.q_max = plan_q_max(p);
-    // as many warps per block as the shared-memory budget allows (each warp holds one candidate's timeline)
-    const size_t per_warp = sim_warp_floats(a.q_max) * sizeof(float);
-    int warps = (int)(kSimSmemBudget / per_warp);
-    warps = warps < 1 ? 1 : (warps > kSimMaxWarps ? kSimMaxWarps : warps);
-    const size_t smem = (size_t)warps * per_warp;
-    if (smem > 227 * 1024) return PF_EUNSUPPORTED;
-    const int kSimThreads = warps * 32;
-    PF_CUDA_TRY(cudaMemsetAsync(a.counter, 0, 256, st), "pf_simulate: counter reset");
+    a.cls = 0;
+    PF_CUDA_TRY(cudaMemsetAsync(ws + lay.off_ctrl, 0, 256, st), "pf_simulate: counter reset");
     if (n > 0) {
-        uint64_t want = (n + warps - 1) / warps;
-        int per_sm = (int)((size_t)(227 * 1024) / (smem + 1024));
-        per_sm = per_sm < 1 ? 1 : (per_sm > 4 ? 4 : per_sm);
-        uint64_t cap = (uint64_t)p->sm_count * per_sm;
-        int grid = (int)(want < cap ? want : cap);
-        if (p->dev.wide) {
-            PF_CUDA_TRY(cudaFuncSetAttribute(simulate_kernel<unsigned long long>,
-                                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem),
-                        "simulate_kernel smem");
-            simulate_kernel<unsigned long long><<<grid, kSimThreads, smem, st>>>(p->dev, a);
-        } else {
-            PF_CUDA_TRY(cudaFuncSetAttribute(simulate_kernel<uint32_t>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             (int)smem),
-                        "simulate_kernel smem");
-            simulate_kernel<uint32_t><<<grid, kSimThreads, smem, st>>>(p->dev, a);
-        }
-        count_launch();
-        PF_CUDA_TRY(cudaGetLastError(), "simulate_kernel launch");
+        int nk = 0;
+        timing_begin(p, PF_T_SIMULATE, st);
+        rc = p->dev.wide ? launch_simulate<unsigned long long>(p, a, n, st, &nk)
+                         : launch_simulate<uint32_t>(p, a, n, st, &nk);
+        timing_end(p, PF_T_SIMULATE, nk, st);
+        if (rc != PF_OK) return rc;
     }
     if (k > 0) {
+        uint8_t *tws = ws + lay.off_topk;
+        PF_CUDA_TRY(cudaMemsetAsync(tws + lay.tk.off_ctrl, 0, 256, st), "pf_simulate: top-k reset");
         DenseTopkArgs t;
         t.score = scores; t.n = n; t.d_n = d_n; t.k = k;
-        t.lists = (unsigned long long *)(ws + lay.off_topk + lay.tk.off_lists_a);
+        t.keys = (unsigned long long *)(tws + lay.tk.off_keys_a);
+        t.key_count = (unsigned int *)(tws + lay.tk.off_ctrl) + 1;
+        timing_begin(p, PF_T_TOPK, st);
         dense_topk_kernel<<<lay.topk_blocks, kThreads, 0, st>>>(t);
         count_launch();
         PF_CUDA_TRY(cudaGetLastError(), "dense_topk_kernel launch");
-        return launch_topk_reduce(t.lists, (unsigned long long *)(ws + lay.off_topk + lay.tk.off_lists_b),
-                                  lay.topk_blocks, k, 0, d_surv_idx, d_topk_idx, d_topk_score, d_topk_count, st);
+        int nk = 0;
+        rc = launch_topk_reduce(tws, lay.tk, lay.topk_keys_max, k, 0, d_surv_idx, d_topk_idx, d_topk_score,
+                                d_topk_count, st, &nk);
+        timing_end(p, PF_T_TOPK, nk + 1, st);
+        return rc;
     }
     return PF_OK;
 }

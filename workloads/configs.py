@@ -136,8 +136,8 @@ def _serve():
     )
 
 
-def _large(enforce: int):
-    _, eff, patch, sovh, masks = table_draws(0, 8, 4, 0.9)
+def _large(enforce: int, seed: int = 0):
+    _, eff, patch, sovh, masks = table_draws(seed, 8, 4, 0.9)
     p2 = [1 << i for i in range(11)]
     return dict(
         name="large" if enforce else "large_unconstrained", phase=0, k=1024,
@@ -157,9 +157,11 @@ def _large(enforce: int):
     )
 
 
-def make_config(name: str) -> dict:
+def make_config(name: str, seed: int = 0) -> dict:
     """Return a fresh config dict.  'large_unconstrained' is 'large' with the dry-run rules off
-    (the paper's unconstrained search mode), used by the simulator tier."""
+    (the paper's unconstrained search mode), used by the simulator tier.  `seed` re-draws the tables of
+    the large spaces (independent problems of the same shape, one per GPU in a multi-GPU benchmark);
+    the other spaces keep their fixed seeds."""
     if name == "tiny":
         return _tiny()
     if name == "mid":
@@ -167,9 +169,9 @@ def make_config(name: str) -> dict:
     if name == "serve":
         return _serve()
     if name == "large":
-        return _large(1)
+        return _large(1, seed)
     if name == "large_unconstrained":
-        return _large(0)
+        return _large(0, seed)
     raise KeyError(name)
 
 
