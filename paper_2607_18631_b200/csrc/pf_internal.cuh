@@ -154,15 +154,22 @@ __device__ inline void tk_prune(unsigned long long *buf, int *count, unsigned lo
     __syncthreads();
 }
 
-// Append the block's held keys (after tk_prune: sorted, *count of them) to a compact global key list.
-// s_base: one shared int of scratch.  Block-collective.
-__device__ inline void tk_flush(const unsigned long long *buf, int c, int *s_base, unsigned long long *out_keys,
-                                unsigned int *out_count)
+// Append the block's held keys that are >= min_key (after tk_prune: sorted, c of them) to a compact global
+// key list.  s_base: two shared ints of scratch.  Block-collective.
+__device__ inline void tk_flush(const unsigned long long *buf, int c, unsigned long long min_key, int *s_base,
+                                unsigned long long *out_keys, unsigned int *out_count)
 {
-    if (threadIdx.x == 0) *s_base = c > 0 ? (int)atomicAdd(out_count, (unsigned int)c) : 0;
+    if (threadIdx.x == 0) s_base[1] = 0;
     __syncthreads();
-    unsigned long long *out = out_keys + *s_base;
-    for (int i = threadIdx.x; i < c; i += blockDim.x) out[i] = buf[i];
+    // the buffer is sorted descending: the cut is the last position whose key is still >= min_key
+    for (int i = threadIdx.x; i < c; i += blockDim.x)
+        if (buf[i] >= min_key && (i + 1 == c || buf[i + 1] < min_key)) s_base[1] = i + 1;
+    __syncthreads();
+    const int keep = s_base[1];
+    if (threadIdx.x == 0) s_base[0] = keep > 0 ? (int)atomicAdd(out_count, (unsigned int)keep) : 0;
+    __syncthreads();
+    unsigned long long *out = out_keys + s_base[0];
+    for (int i = threadIdx.x; i < keep; i += blockDim.x) out[i] = buf[i];
 }
 
 // Append this thread's key if it beats the threshold.  Warp-collective (all 32 lanes must call); the
@@ -185,7 +192,8 @@ __device__ __forceinline__ void tk_push(unsigned long long *buf, int *count, uns
 }
 
 // host: workspace layout of one top-k reduction whose producers append at most n_keys_max keys in total.
-// ctrl is 256 bytes of uint32: [0] producer work counter, [1] keys in list A, [2] keys in list B, [3] spare.
+// ctrl is 256 bytes: uint32 [0] producer work counter, [1] keys in list A, [2] keys in list B, [3] spare;
+// uint64 at byte 16: the producers' shared admission threshold (largest k-th key any block has reached).
 constexpr int kReduceSeg = 32768;    // keys one block of the reduce kernel walks through
 constexpr int kReduceThreads = 1024;
 struct TopkLayout {

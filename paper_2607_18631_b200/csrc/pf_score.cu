@@ -24,6 +24,7 @@ struct ScoreArgs {
     long long *mem;
     unsigned long long *keys;       // compact list of the blocks' best keys
     unsigned int *key_count;        // its length (zeroed before launch)
+    unsigned long long *g_thr;      // largest k-th key any block has reached (zeroed before launch)
     unsigned int *slab_counter;     // zeroed before launch
     const int32_t *vals;            // packed axis value lists
     const int32_t *scen;            // serve: P[n_scen], O[n_scen]
@@ -58,7 +59,8 @@ __global__ void __launch_bounds__(kThreads) score_kernel(const __grid_constant__
     __shared__ int s_count;
     __shared__ unsigned long long s_thr;
     __shared__ SlabInfo s_slab;
-    __shared__ int s_base;
+    __shared__ int s_base[2];
+    __shared__ unsigned long long s_gthr;   // snapshot of the grid-wide threshold, refreshed once per slab
 
     const int tid = threadIdx.x;
     const bool train = P.phase == PF_PHASE_TRAIN;
@@ -75,6 +77,7 @@ __global__ void __launch_bounds__(kThreads) score_kernel(const __grid_constant__
         __syncthreads();  // previous slab fully consumed before s_slab is overwritten
         if (tid == 0) {
             uint32_t s = atomicAdd(A.slab_counter, 1u);
+            s_gthr = want_topk ? *reinterpret_cast<volatile unsigned long long *>(A.g_thr) : 0ull;
             SlabInfo si;
             si.slab = s < A.n_slabs ? s : 0xFFFFFFFFu;
             si.pre_reason = 0;
@@ -191,9 +194,13 @@ __global__ void __launch_bounds__(kThreads) score_kernel(const __grid_constant__
             if (want_topk) {
                 if (room_iters == 0) {
                     __syncthreads();
-                    if (s_count > kTopkCap - kThreads) tk_prune(s_buf, &s_count, &s_thr, (int)A.k);
+                    if (s_count > kTopkCap - kThreads) {
+                        tk_prune(s_buf, &s_count, &s_thr, (int)A.k);
+                        // a block's k-th key bounds the global k-th from below: share it
+                        if (tid == 0 && s_thr != 0ull) atomicMax(A.g_thr, s_thr);
+                    }
                     room_iters = (kTopkCap - s_count) / kThreads;
-                    thr = s_thr;
+                    thr = s_thr > s_gthr ? s_thr : s_gthr;
                     __syncthreads();
                 }
                 const bool feasible = active && (reason & 0x7f) == 0;
@@ -205,7 +212,12 @@ __global__ void __launch_bounds__(kThreads) score_kernel(const __grid_constant__
 
     if (want_topk) {
         tk_prune(s_buf, &s_count, &s_thr, (int)A.k);
-        tk_flush(s_buf, s_count, &s_base, A.keys, A.key_count);
+        if (tid == 0) {
+            if (s_thr != 0ull) atomicMax(A.g_thr, s_thr);
+            s_thr = *reinterpret_cast<volatile unsigned long long *>(A.g_thr);
+        }
+        __syncthreads();
+        tk_flush(s_buf, s_count, s_thr, s_base, A.keys, A.key_count);
     }
 }
 
@@ -225,35 +237,38 @@ struct ReduceArgs {
     uint32_t *topk_count;
 };
 
-// Block b walks keys [b*kReduceSeg, (b+1)*kReduceSeg) of the input in buffer-sized rounds, keeping the k best.
+// Block b walks keys [b*kReduceSeg, (b+1)*kReduceSeg) of the input one tile at a time, admitting only keys
+// above its running k-th best, and keeps the k best.
 __global__ void __launch_bounds__(kReduceThreads) reduce_kernel(const ReduceArgs A)
 {
     __shared__ unsigned long long s_buf[kTopkCap];
     __shared__ int s_count;
     __shared__ unsigned long long s_thr;
-    __shared__ int s_base;
+    __shared__ int s_base[2];
     const int tid = threadIdx.x, k = (int)A.k;
     const unsigned int n = *A.in_count;
-    unsigned int pos = blockIdx.x * (unsigned int)kReduceSeg;
-    const unsigned int hi = min(pos + (unsigned int)kReduceSeg, n);
-    if (pos >= hi && !A.final) return;
+    const unsigned int lo = blockIdx.x * (unsigned int)kReduceSeg;
+    const unsigned int hi = min(lo + (unsigned int)kReduceSeg, n);
+    if (lo >= hi && !A.final) return;
     if (tid == 0) {
         s_count = 0;
         s_thr = 0ull;
     }
     __syncthreads();
-    while (pos < hi) {
-        const int held = s_count;
-        const int take = min((unsigned int)(kTopkCap - held), hi - pos);
-        for (int i = tid; i < take; i += kReduceThreads) s_buf[held + i] = A.in[pos + i];
-        pos += take;
+    unsigned long long thr = 0ull;
+    for (unsigned int pos = lo; pos < hi; pos += kReduceThreads) {
         __syncthreads();
-        if (tid == 0) s_count = held + take;
-        tk_prune(s_buf, &s_count, &s_thr, k);
+        if (s_count > kTopkCap - kReduceThreads) tk_prune(s_buf, &s_count, &s_thr, k);
+        thr = s_thr;
+        __syncthreads();
+        const unsigned int i = pos + tid;
+        const unsigned long long key = i < hi ? A.in[i] : 0ull;
+        tk_push(s_buf, &s_count, thr, key != 0ull, key);
     }
+    tk_prune(s_buf, &s_count, &s_thr, k);
     const int c = s_count;
     if (!A.final) {
-        tk_flush(s_buf, c, &s_base, A.out, A.out_count);
+        tk_flush(s_buf, c, 0ull, s_base, A.out, A.out_count);
     } else {
         for (int i = tid; i < k; i += kReduceThreads) {
             if (i < c) {
@@ -416,6 +431,7 @@ extern "C" int pf_score(pf_plan_t *p, uint64_t first, uint64_t count, uint8_t *d
     a.keys = (unsigned long long *)(ws + lay.off_keys_a);
     a.slab_counter = (unsigned int *)(ws + lay.off_ctrl);
     a.key_count = a.slab_counter + 1;
+    a.g_thr = (unsigned long long *)(ws + lay.off_ctrl + 16);
     a.vals = p->d_vals; a.scen = p->d_scen;
     PF_CUDA_TRY(cudaMemsetAsync(a.slab_counter, 0, 256, st), "pf_score: counter reset");
     timing_begin(p, PF_T_SCORE, st);

@@ -85,7 +85,13 @@ template <typename F>
 __device__ __forceinline__ void for_each_eligible16(const DevPlan &P, const int32_t *vals, const SelArgs &A,
                                                     uint64_t e, F f)
 {
-    uint32_t m = feasible_mask16(load_reason16(A.reason, e, A.count));
+    const uint4 r = load_reason16(A.reason, e, A.count);
+    // any byte with its low 7 bits clear?  (zero-byte test on the masked words; most groups have none)
+    const uint32_t x0 = r.x & 0x7F7F7F7Fu, x1 = r.y & 0x7F7F7F7Fu, x2 = r.z & 0x7F7F7F7Fu, x3 = r.w & 0x7F7F7F7Fu;
+    const uint32_t z = ((x0 - 0x01010101u) & ~x0) | ((x1 - 0x01010101u) & ~x1) | ((x2 - 0x01010101u) & ~x2) |
+                       ((x3 - 0x01010101u) & ~x3);
+    if ((z & 0x80808080u) == 0) return;
+    uint32_t m = feasible_mask16(r);
     while (m) {
         int i = __ffs(m) - 1;
         m &= m - 1;
@@ -277,10 +283,11 @@ __global__ void __launch_bounds__(kSelThreads) sel_write_kernel(const __grid_con
                 if (all || bits > thr) gt++;
                 else if (bits == thr) eq++;
             });
+        if (!__syncthreads_or((int)(gt | eq))) continue;   // nothing eligible in this tile (the common case)
         s_gt[tid] = gt;
         s_eq[tid] = eq;
         __syncthreads();
-        // exclusive scan by one warp-free loop would serialize 256 steps; do a simple Hillis-Steele scan
+        // inclusive Hillis-Steele scan of the per-thread counts
         for (int off = 1; off < kSelThreads; off <<= 1) {
             unsigned int ag = tid >= off ? s_gt[tid - off] : 0, ae = tid >= off ? s_eq[tid - off] : 0;
             __syncthreads();

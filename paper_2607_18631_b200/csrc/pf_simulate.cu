@@ -196,7 +196,8 @@ struct SimArgs {
     const uint8_t *dual_ops;
     const int32_t *dual_off;
     int q_max;                      // stages per candidate at most (plan-wide)
-    int cls;                        // class this launch serves
+    int cls_hi;                     // largest class the plan can produce
+    int pool_floats;                // dynamic shared memory of a block, in floats
 };
 
 // Pre-pass: one thread per survivor computes how many timeline entries its simulation needs and files the
@@ -255,27 +256,35 @@ __global__ void __launch_bounds__(256) sim_classify_kernel(const __grid_constant
 // per-warp shared memory of class c: endF[E], endB[E], durF[q_max], durB[q_max]
 __host__ __device__ inline size_t sim_warp_floats(int entries, int q_max) { return (size_t)2 * entries + 2 * q_max; }
 
+// One launch serves every class, largest timelines first (the longest simulations start earliest).  A block
+// owns a fixed pool of shared memory; for class c as many of its warps as fit (pool / footprint) pull
+// candidates from that class' queue, the others wait at the barrier that separates two classes.
 template <typename RI>
 __global__ void __launch_bounds__(kSimMaxWarps * 32) simulate_kernel(const __grid_constant__ DevPlan P, const SimArgs A)
 {
     extern __shared__ float s_mem[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int E = sim_class_entries(A.cls);
-    float *base = s_mem + (size_t)warp * sim_warp_floats(E, A.q_max);
+    const uint32_t seed_mixed = mix32(A.seed + 0x9e3779b9u);
+
+    for (int cls = A.cls_hi; cls >= 0; cls--) {
+    const unsigned int n_cls = A.cls_count[cls];
+    if (n_cls == 0) continue;
+    const int E = sim_class_entries(cls);
+    const int per_warp = (int)sim_warp_floats(E, A.q_max);
+    const int active_warps = min((int)(blockDim.x >> 5), A.pool_floats / per_warp);
+    if (warp < active_warps) {
+    float *base = s_mem + (size_t)warp * per_warp;
     // End times are written by the lane that owns the stage and polled by its neighbour: one 32-bit word per
     // op, negative while the op has not finished, so a single volatile load answers "done, and when".
     volatile float *endF = base;
     volatile float *endB = base + E;
     float *durF = base + 2 * (size_t)E;
     float *durB = durF + A.q_max;
-
-    const unsigned int n_cls = A.cls_count[A.cls];
-    const uint32_t *list = A.cls_list + (size_t)A.cls * A.n;
-    const uint32_t seed_mixed = mix32(A.seed + 0x9e3779b9u);
+    const uint32_t *list = A.cls_list + (size_t)cls * A.n;
 
     for (;;) {
         unsigned int wi = 0;
-        if (lane == 0) wi = atomicAdd(A.work + A.cls, 1u);
+        if (lane == 0) wi = atomicAdd(A.work + cls, 1u);
         wi = __shfl_sync(0xFFFFFFFFu, wi, 0);
         if (wi >= n_cls) break;
         const uint32_t w = list[wi];
@@ -358,9 +367,10 @@ __global__ void __launch_bounds__(kSimMaxWarps * 32) simulate_kernel(const __gri
             warm = min(2 * (pp - lane - 1) + (v - 1) * pp, U);
         else
             warm = min(pp - lane - 1, U);
-        int nF = 0, nB = 0;               // units issued
-        int fc = 0, fw = 0, fg = 0;       // forward cursor: microbatch = fg*pp + fw, chunk = fc
-        int bc = 0, bw = 0, bg = 0;       // backward cursor: chunk = v-1-bc
+        // unit cursors (1F1B is the one-chunk case): microbatch = g*pp + w, chunk = c (backward: v-1-c)
+        int nF = 0, nB = 0;
+        int fc = 0, fw = 0, fg = 0;
+        int bc = 0, bw = 0, bg = 0;
         const uint8_t *dops = nullptr;
         if (dual && !stalled) {
             const int off = __ldg(A.dual_off + pp * 33 + nj);
@@ -372,61 +382,47 @@ __global__ void __launch_bounds__(kSimMaxWarps * 32) simulate_kernel(const __gri
         int done_ops = 0;
         int rounds = 0;
         bool moved = false;
+        const float lat = T.p;
 
+        // One op per lane per round at most; the body is branch-free apart from the "not ready" exit, so the
+        // lanes of a warp stay converged and a round costs one shared-memory poll plus one vote.
         for (;;) {
-            // up to 4 ops per round keep the lanes that run ahead from waiting on the vote
-#pragma unroll 1
-            for (int rep = 0; rep < 4 && done_ops < total_ops; rep++) {
+            if (done_ops < total_ops) {
                 int isb, d = 0, q, j;
                 if (dual) {
-                    const uint8_t op = __ldg(dops + done_ops);
+                    const uint32_t op = __ldg(dops + done_ops);
                     isb = op & 1;
                     d = (op >> 1) & 1;
                     j = op >> 2;
                     q = d ? pp - 1 - lane : lane;
-                } else if (kind == PF_KIND_1F1B) {
-                    isb = !(nF < warm || (nF < U && nF - warm == nB));
-                    j = isb ? nB : nF;
-                    q = lane;
                 } else {
                     isb = !(nF < warm || (nF < U && nF - warm == nB));
-                    j = isb ? bg * pp + bw : fg * pp + fw;
-                    q = (isb ? v - 1 - bc : fc) * pp + lane;
+                    const int cw = isb ? bw : fw, cc = isb ? bc : fc, cg = isb ? bg : fg;
+                    j = cg * pp + cw;
+                    q = (isb ? v - 1 - cc : cc) * pp + lane;
                 }
-                const int sidx = d * Q + q;          // stage stream (direction-major for DualPipe)
-                float dep = 0.f;
-                if (!isb) {
-                    if (q > 0) {
-                        dep = endF[(sidx - 1) * nj + j];
-                        if (dep < 0.f) break;
-                        dep += T.p;
+                const int sidx = d * Q + q;                  // stage stream (direction-major for DualPipe)
+                const bool has_dep = isb ? (q < Q - 1) : (q > 0);
+                const int nb = has_dep ? (isb ? sidx + 1 : sidx - 1) : sidx;
+                volatile float *in = isb ? endB : endF;
+                const float e = in[nb * nj + j];
+                const float dur = (isb ? durB : durF)[q];
+                if (!has_dep || e >= 0.f) {
+                    const float fin = fmaxf(clock, has_dep ? e + lat : 0.f) + dur;
+                    clock = fin;
+                    in[sidx * nj + j] = fin;
+                    if (!dual) {
+                        int w_ = (isb ? bw : fw) + 1, c_ = isb ? bc : fc, g_ = isb ? bg : fg;
+                        if (w_ == pp) {
+                            w_ = 0;
+                            if (++c_ == v) c_ = 0, g_++;
+                        }
+                        if (isb) bw = w_, bc = c_, bg = g_, nB++;
+                        else fw = w_, fc = c_, fg = g_, nF++;
                     }
-                } else {
-                    if (q < Q - 1) {
-                        dep = endB[(sidx + 1) * nj + j];
-                        if (dep < 0.f) break;
-                        dep += T.p;
-                    }
+                    done_ops++;
+                    moved = true;
                 }
-                const float fin = fmaxf(clock, dep) + (isb ? durB[q] : durF[q]);
-                clock = fin;
-                if (!isb) {
-                    endF[sidx * nj + j] = fin;
-                    nF++;
-                    if (++fw == pp) {
-                        fw = 0;
-                        if (++fc == v) fc = 0, fg++;
-                    }
-                } else {
-                    endB[sidx * nj + j] = fin;
-                    nB++;
-                    if (++bw == pp) {
-                        bw = 0;
-                        if (++bc == v) bc = 0, bg++;
-                    }
-                }
-                done_ops++;
-                moved = true;
             }
             if (!__any_sync(0xFFFFFFFFu, done_ops < total_ops)) break;
             // bounded wait: every 64 rounds some lane must have advanced
@@ -467,6 +463,9 @@ __global__ void __launch_bounds__(kSimMaxWarps * 32) simulate_kernel(const __gri
         }
         __syncwarp();
     }
+    }  // active warps of this class
+    __syncthreads();  // the next class lays the pool out differently
+    }  // classes
 }
 
 // ------------------------------------------------------------------ top-k over a dense score array
@@ -486,7 +485,7 @@ __global__ void __launch_bounds__(kThreads) dense_topk_kernel(const DenseTopkArg
     __shared__ unsigned long long s_buf[kTopkCap];
     __shared__ int s_count;
     __shared__ unsigned long long s_thr;
-    __shared__ int s_base;
+    __shared__ int s_base[2];
     const int tid = threadIdx.x;
     if (tid == 0) {
         s_count = 0;
@@ -514,7 +513,7 @@ __global__ void __launch_bounds__(kThreads) dense_topk_kernel(const DenseTopkArg
         room--;
     }
     tk_prune(s_buf, &s_count, &s_thr, (int)A.k);
-    tk_flush(s_buf, s_count, &s_base, A.keys, A.key_count);
+    tk_flush(s_buf, s_count, 0ull, s_base, A.keys, A.key_count);
 }
 
 struct SimLayout {
@@ -571,28 +570,24 @@ static int launch_simulate(pf_plan_t *p, SimArgs a, uint64_t n, cudaStream_t st,
     PF_CUDA_TRY(cudaFuncSetAttribute(simulate_kernel<RI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      (int)(227 * 1024)),
                 "simulate_kernel smem");
-    // one launch per timeline-size class that the plan can produce
+    // largest class the plan can produce, and a pool that holds at least one such timeline
     const int entries_max = a.q_max * PF_SIM_WINDOW;
-    for (int c = 0; c < kSimClasses; c++) {
-        if (c > 0 && sim_class_entries(c - 1) >= entries_max) break;
-        const size_t per_warp = sim_warp_floats(sim_class_entries(c), a.q_max) * sizeof(float);
-        if (per_warp > 227 * 1024) return PF_EUNSUPPORTED;
-        // blocks of up to 16 warps, at least two blocks per SM where the footprint allows
-        int warps = (int)((size_t)(110 * 1024) / per_warp);
-        if (warps < 1) warps = (int)((size_t)(227 * 1024) / per_warp);
-        warps = warps < 1 ? 1 : (warps > kSimMaxWarps ? kSimMaxWarps : warps);
-        const size_t smem = (size_t)warps * per_warp;
-        int per_sm = (int)((size_t)(227 * 1024) / (smem + 1024));
-        per_sm = per_sm < 1 ? 1 : (per_sm > 4 ? 4 : per_sm);
-        const uint64_t want = (n + warps - 1) / warps;
-        const uint64_t cap = (uint64_t)p->sm_count * per_sm;
-        const int grid = (int)(want < cap ? want : cap);
-        a.cls = c;
-        simulate_kernel<RI><<<grid, warps * 32, smem, st>>>(p->dev, a);
-        count_launch();
-        (*n_kernels)++;
-        PF_CUDA_TRY(cudaGetLastError(), "simulate_kernel launch");
-    }
+    int cls_hi = 0;
+    while (cls_hi < kSimClasses - 1 && sim_class_entries(cls_hi) < entries_max) cls_hi++;
+    const size_t biggest = sim_warp_floats(sim_class_entries(cls_hi), a.q_max) * sizeof(float);
+    if (biggest > 227 * 1024) return PF_EUNSUPPORTED;
+    size_t pool = 72 * 1024;                         // three blocks per SM when the largest timeline allows
+    if (pool < biggest) pool = biggest;
+    int per_sm = (int)((size_t)(227 * 1024) / (pool + 1024));
+    per_sm = per_sm < 1 ? 1 : per_sm;
+    a.cls_hi = cls_hi;
+    a.pool_floats = (int)(pool / sizeof(float));
+    const uint64_t cap = (uint64_t)p->sm_count * per_sm;
+    const int grid = (int)(n < cap ? n : cap);
+    simulate_kernel<RI><<<grid, kSimMaxWarps * 32, pool, st>>>(p->dev, a);
+    count_launch();
+    (*n_kernels)++;
+    PF_CUDA_TRY(cudaGetLastError(), "simulate_kernel launch");
     return PF_OK;
 }
 
@@ -640,7 +635,8 @@ extern "C" int pf_simulate(pf_plan_t *p, const uint64_t *d_surv_idx, uint64_t n,
     a.cls_list = (uint32_t *)(ws + lay.off_lists);
     a.vals = p->d_vals; a.dual_ops = tab->d_ops; a.dual_off = tab->d_offset;
     a.q_max = plan_q_max(p);
-    a.cls = 0;
+    a.cls_hi = 0;
+    a.pool_floats = 0;
     PF_CUDA_TRY(cudaMemsetAsync(ws + lay.off_ctrl, 0, 256, st), "pf_simulate: counter reset");
     if (n > 0) {
         int nk = 0;
