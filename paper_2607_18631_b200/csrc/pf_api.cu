@@ -336,6 +336,21 @@ extern "C" int pf_plan_create(const pf_model_t *model, const pf_cluster_t *clust
         wide |= tp * ep > lim || B * M.K > lim || C * M.K > lim || workload->world > lim;
     }
     d.wide = wide ? 1 : 0;
+    // A feasible training plan has pp * v <= L (layer rule).  If no listed pp or v value that can pass that
+    // rule leaves the simulator's domain, survivor selection needs no per-candidate domain check.
+    d.sim_domain_all = 0;
+    if (phase == PF_PHASE_TRAIN) {
+        bool all_in = true;
+        for (int i = 0; i < axes->len[6]; i++) {
+            int pp = axes->val[6][i];
+            if (pp <= M.L && pp > PF_SIM_MAX_RANKS) all_in = false;
+        }
+        for (int i = 0; i < axes->len[4]; i++) {
+            int v = axes->val[4][i] == 0 ? 2 : axes->val[4][i];
+            if (v <= M.L && v > PF_SIM_MAX_V) all_in = false;
+        }
+        d.sim_domain_all = all_in ? 1 : 0;
+    }
 
     // device copies
     cudaError_t e = cudaMalloc((void **)&p->d_vals, sizeof(int32_t) * (size_t)total_vals);

@@ -37,6 +37,7 @@ struct DevPlan {
     uint32_t magic[PF_MAX_AXES];   // ceil(2^32 / radix) for the inner axes: q = umulhi(n, magic)
     int val_off[PF_MAX_AXES];      // offset of each axis' value list in the packed value array
     int wide;                      // 1: rule arithmetic needs 64-bit integers
+    int sim_domain_all;            // 1: every feasible candidate lies inside the simulator's domain
     // --- model (Sec. 3.1) and host-derived per-layer constants
     int L, H, nh, nkv, hd, attn_kind, kv_latent, rope_dim, E, K, F, S, Fs, seq, vocab;
     int wb, gb, ob, ab, count_embeddings;
@@ -114,12 +115,18 @@ __device__ __forceinline__ uint32_t key_rel(unsigned long long key) { return 0xF
 // noted; the block may have any multiple of 32 threads.
 
 // Descending bitonic sort of buf[0, n_sort) in shared memory; n_sort a power of two <= kTopkCap.
+// Thread i takes compare-exchange pairs i, i + blockDim, ...; for strides <= 32 the 32 pairs of a warp lie
+// in one 64-element window that no other warp touches, so those stages need only a warp barrier.  A block
+// barrier is used when a stage is wider than that or follows one that was.
 __device__ inline void tk_sort_desc(unsigned long long *buf, int n_sort)
 {
     const int tid = threadIdx.x, nt = blockDim.x;
+    int prev_stride = 64;  // whatever filled the buffer was block-wide
     for (int size = 2; size <= n_sort; size <<= 1) {
         for (int stride = size >> 1; stride > 0; stride >>= 1) {
-            __syncthreads();
+            if (stride > 32 || prev_stride > 32) __syncthreads();
+            else __syncwarp();
+            prev_stride = stride;
             for (int i = tid; i < n_sort / 2; i += nt) {
                 int lo = 2 * i - (i & (stride - 1));  // element with the stride bit clear
                 int hi = lo + stride;
@@ -194,7 +201,7 @@ __device__ __forceinline__ void tk_push(unsigned long long *buf, int *count, uns
 // host: workspace layout of one top-k reduction whose producers append at most n_keys_max keys in total.
 // ctrl is 256 bytes: uint32 [0] producer work counter, [1] keys in list A, [2] keys in list B, [3] spare;
 // uint64 at byte 16: the producers' shared admission threshold (largest k-th key any block has reached).
-constexpr int kReduceSeg = 32768;    // keys one block of the reduce kernel walks through
+constexpr int kReduceSeg = 8192;     // keys one block of the reduce kernel walks through
 constexpr int kReduceThreads = 1024;
 struct TopkLayout {
     size_t off_ctrl, off_keys_a, off_keys_b, total;

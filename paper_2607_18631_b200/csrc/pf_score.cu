@@ -295,7 +295,7 @@ int launch_topk_reduce(void *d_workspace, const TopkLayout &lay, uint64_t n_keys
     unsigned long long *out = (unsigned long long *)(ws + lay.off_keys_b);
     int in_slot = 1, out_slot = 2;
     *n_kernels = 0;
-    for (int pass = 0; pass < 3; pass++) {
+    for (int pass = 0; pass < 6; pass++) {
         const uint64_t blocks = (n_keys_max + kReduceSeg - 1) / kReduceSeg;
         ReduceArgs r;
         r.in = in; r.in_count = ctrl + in_slot; r.out = out; r.out_count = ctrl + out_slot;
@@ -308,8 +308,11 @@ int launch_topk_reduce(void *d_workspace, const TopkLayout &lay, uint64_t n_keys
         if (r.final) return PF_OK;
         n_keys_max = blocks * k;
         unsigned long long *t = in; in = out; out = t;
+        // counters rotate through ctrl[1..3]; the one about to be reused was consumed two passes ago
+        const int next = in_slot == 1 ? 3 : in_slot - 1;
         in_slot = out_slot;
-        out_slot = 3;   // a third pass would need n_keys_max > 32768 * 32768 / k: never with k <= 1024 lists
+        out_slot = next;
+        if (pass >= 1) PF_CUDA_TRY(cudaMemsetAsync(ctrl + out_slot, 0, 4, st), "reduce counter reset");
     }
     return PF_EINVAL;
 }

@@ -36,6 +36,7 @@ struct SelArgs {
 // eligibility beyond feasibility: the simulator's domain (pp <= 32 ranks, <= 8 virtual stages per rank)
 __device__ __forceinline__ bool in_sim_domain(const DevPlan &P, const int32_t *vals, uint64_t idx)
 {
+    if (P.sim_domain_all) return true;
     int s = 0, v = 0, pp = 0;
     uint64_t rem = idx;
 #pragma unroll
@@ -80,12 +81,12 @@ __device__ __forceinline__ uint32_t feasible_mask16(uint4 r)
     return m;
 }
 
-// Visit the eligible candidates of a block's chunk in ascending order: f(rel, score_bits).
+// Visit the eligible candidates of one group of 16 (reason bytes r, first element e) in ascending order:
+// f(rel, score_bits).
 template <typename F>
 __device__ __forceinline__ void for_each_eligible16(const DevPlan &P, const int32_t *vals, const SelArgs &A,
-                                                    uint64_t e, F f)
+                                                    uint64_t e, const uint4 r, F f)
 {
-    const uint4 r = load_reason16(A.reason, e, A.count);
     // any byte with its low 7 bits clear?  (zero-byte test on the masked words; most groups have none)
     const uint32_t x0 = r.x & 0x7F7F7F7Fu, x1 = r.y & 0x7F7F7F7Fu, x2 = r.z & 0x7F7F7F7Fu, x3 = r.w & 0x7F7F7F7Fu;
     const uint32_t z = ((x0 - 0x01010101u) & ~x0) | ((x1 - 0x01010101u) & ~x1) | ((x2 - 0x01010101u) & ~x2) |
@@ -100,6 +101,20 @@ __device__ __forceinline__ void for_each_eligible16(const DevPlan &P, const int3
     }
 }
 
+constexpr int kSelTiles = 16;                              // tiles of 256 x 16 candidates per block
+constexpr uint64_t kSelTile = (uint64_t)kSelThreads * 16;  // candidates per tile
+
+// Load this thread's group of every tile of the block's chunk before any of them is looked at, so the
+// reads of a chunk are all in flight together.
+__device__ __forceinline__ void load_chunk(const SelArgs &A, uint64_t lo, uint64_t hi, uint4 (&r)[kSelTiles])
+{
+#pragma unroll
+    for (int t = 0; t < kSelTiles; t++) {
+        const uint64_t e = lo + (uint64_t)t * kSelTile + (uint64_t)threadIdx.x * 16;
+        r[t] = e < hi ? load_reason16(A.reason, e, A.count) : make_uint4(~0u, ~0u, ~0u, ~0u);
+    }
+}
+
 __global__ void __launch_bounds__(kSelThreads) sel_hist_kernel(const __grid_constant__ DevPlan P, const SelArgs A,
                                                                 const int32_t *vals, int pass)
 {
@@ -107,8 +122,12 @@ __global__ void __launch_bounds__(kSelThreads) sel_hist_kernel(const __grid_cons
     const uint64_t hi = min(lo + A.chunk, A.count);
     if (pass == 1 && A.ctrl->take_all) return;
     const uint32_t b1 = pass == 1 ? A.ctrl->b1 : 0;
-    for (uint64_t e = lo + (uint64_t)threadIdx.x * 16; e < hi; e += (uint64_t)kSelThreads * 16) {
-        for_each_eligible16(P, vals, A, e, [&](uint64_t, uint32_t bits) {
+    uint4 r[kSelTiles];
+    load_chunk(A, lo, hi, r);
+#pragma unroll
+    for (int t = 0; t < kSelTiles; t++) {
+        const uint64_t e = lo + (uint64_t)t * kSelTile + (uint64_t)threadIdx.x * 16;
+        for_each_eligible16(P, vals, A, e, r[t], [&](uint64_t, uint32_t bits) {
             if (pass == 0)
                 atomicAdd(A.hist1 + (bits >> 16), 1u);
             else if ((bits >> 16) == b1)
@@ -205,7 +224,7 @@ __global__ void __launch_bounds__(1024) sel_scan_kernel(const SelArgs A, int pas
 __global__ void __launch_bounds__(kSelThreads) sel_count_kernel(const __grid_constant__ DevPlan P, const SelArgs A,
                                                                  const int32_t *vals)
 {
-    __shared__ unsigned long long s_gt, s_eq;
+    __shared__ unsigned int s_gt, s_eq;
     if (threadIdx.x == 0) s_gt = s_eq = 0;
     __syncthreads();
     const uint64_t lo = (uint64_t)blockIdx.x * A.chunk;
@@ -213,14 +232,18 @@ __global__ void __launch_bounds__(kSelThreads) sel_count_kernel(const __grid_con
     const uint32_t thr = A.ctrl->thr_bits;
     const bool all = A.ctrl->take_all != 0;
     unsigned int gt = 0, eq = 0;
-    for (uint64_t e = lo + (uint64_t)threadIdx.x * 16; e < hi; e += (uint64_t)kSelThreads * 16) {
-        for_each_eligible16(P, vals, A, e, [&](uint64_t, uint32_t bits) {
+    uint4 r[kSelTiles];
+    load_chunk(A, lo, hi, r);
+#pragma unroll
+    for (int t = 0; t < kSelTiles; t++) {
+        const uint64_t e = lo + (uint64_t)t * kSelTile + (uint64_t)threadIdx.x * 16;
+        for_each_eligible16(P, vals, A, e, r[t], [&](uint64_t, uint32_t bits) {
             if (all || bits > thr) gt++;
             else if (bits == thr) eq++;
         });
     }
-    if (gt) atomicAdd(&s_gt, (unsigned long long)gt);
-    if (eq) atomicAdd(&s_eq, (unsigned long long)eq);
+    if (gt) atomicAdd(&s_gt, gt);
+    if (eq) atomicAdd(&s_eq, eq);
     __syncthreads();
     if (threadIdx.x == 0) {
         A.blk_gt[blockIdx.x] = s_gt;
@@ -274,15 +297,17 @@ __global__ void __launch_bounds__(kSelThreads) sel_write_kernel(const __grid_con
         s_run_gt = A.blk_gt[blockIdx.x];
         s_run_eq = A.blk_eq[blockIdx.x];
     }
+    uint4 r[kSelTiles];
+    load_chunk(A, lo, hi, r);
     __syncthreads();
-    for (uint64_t tile = lo; tile < hi; tile += (uint64_t)kSelThreads * 16) {
-        const uint64_t e = tile + (uint64_t)tid * 16;
+#pragma unroll
+    for (int t = 0; t < kSelTiles; t++) {
+        const uint64_t e = lo + (uint64_t)t * kSelTile + (uint64_t)tid * 16;
         unsigned int gt = 0, eq = 0;
-        if (e < hi)
-            for_each_eligible16(P, vals, A, e, [&](uint64_t, uint32_t bits) {
-                if (all || bits > thr) gt++;
-                else if (bits == thr) eq++;
-            });
+        for_each_eligible16(P, vals, A, e, r[t], [&](uint64_t, uint32_t bits) {
+            if (all || bits > thr) gt++;
+            else if (bits == thr) eq++;
+        });
         if (!__syncthreads_or((int)(gt | eq))) continue;   // nothing eligible in this tile (the common case)
         s_gt[tid] = gt;
         s_eq[tid] = eq;
@@ -297,8 +322,8 @@ __global__ void __launch_bounds__(kSelThreads) sel_write_kernel(const __grid_con
         }
         unsigned long long my_gt = s_run_gt + (s_gt[tid] - gt);
         unsigned long long my_eq = s_run_eq + (s_eq[tid] - eq);
-        if (e < hi && (gt | eq))
-            for_each_eligible16(P, vals, A, e, [&](uint64_t rel, uint32_t bits) {
+        if (gt | eq)
+            for_each_eligible16(P, vals, A, e, r[t], [&](uint64_t rel, uint32_t bits) {
                 if (all || bits > thr) {
                     unsigned long long pos = my_gt + (my_eq < need_eq ? my_eq : need_eq);
                     A.surv_idx[pos] = A.first + rel;
@@ -326,10 +351,9 @@ struct SelLayout {
 static SelLayout sel_layout(const pf_plan_t *p, uint64_t count)
 {
     SelLayout l;
-    uint64_t nb = (uint64_t)p->sm_count * 4;
-    uint64_t chunk = (count + nb - 1) / nb;
-    chunk = (chunk + 4095) & ~(uint64_t)4095;  // whole tiles of 256 threads x 16 candidates
-    if (chunk == 0) chunk = 4096;
+    // contiguous chunks of 16 tiles (256 threads x 16 candidates each): many more blocks than SMs, so a
+    // chunk that happens to hold most of the feasible candidates does not hold up the rest
+    uint64_t chunk = (uint64_t)kSelTiles * kSelTile;
     l.chunk = chunk;
     l.nblocks = (int)((count + chunk - 1) / chunk);
     if (l.nblocks < 1) l.nblocks = 1;
@@ -337,7 +361,7 @@ static SelLayout sel_layout(const pf_plan_t *p, uint64_t count)
     l.off_hist1 = 256;
     l.off_hist2 = l.off_hist1 + kBins * 4;
     l.off_gt = l.off_hist2 + kBins * 4;
-    size_t per = (((size_t)p->sm_count * 4 + 1) * 8 + 255) & ~(size_t)255;
+    size_t per = (((size_t)l.nblocks + 1) * 8 + 255) & ~(size_t)255;
     l.off_eq = l.off_gt + per;
     l.total = l.off_eq + per;
     return l;

@@ -256,9 +256,134 @@ __global__ void __launch_bounds__(256) sim_classify_kernel(const __grid_constant
 // per-warp shared memory of class c: endF[E], endB[E], durF[q_max], durB[q_max]
 __host__ __device__ inline size_t sim_warp_floats(int entries, int q_max) { return (size_t)2 * entries + 2 * q_max; }
 
-// One launch serves every class, largest timelines first (the longest simulations start earliest).  A block
-// owns a fixed pool of shared memory; for class c as many of its warps as fit (pool / footprint) pull
-// candidates from that class' queue, the others wait at the barrier that separates two classes.
+// The three round loops.  In every round a lane runs at most its next op, and only if the op it waits for
+// has already published its end time; the body is branch-free apart from that test, so the lanes of a warp
+// stay converged and a round costs one shared-memory poll plus one vote.  Every 64 rounds some lane must
+// have advanced, otherwise the candidate is reported as stalled: the loops are bounded by the op count.
+struct SimLane {
+    float clock;
+    bool stalled;
+};
+
+#define PF_SIM_ROUND_END()                                               \
+    if (!__any_sync(0xFFFFFFFFu, done < total_ops)) break;               \
+    if ((++rounds & 63) == 0) {                                          \
+        if (!__any_sync(0xFFFFFFFFu, moved)) {                           \
+            st.stalled = true;                                           \
+            break;                                                       \
+        }                                                                \
+        moved = false;                                                   \
+    }
+
+// 1F1B: rank = stage = lane; `warm` forwards, then one forward / one backward, then the remaining backwards
+__device__ __forceinline__ void sim_rounds_1f1b(volatile float *endF, volatile float *endB, const float *durF,
+                                                const float *durB, int lane, int pp, int nj, int warm, int total_ops,
+                                                float lat, SimLane &st)
+{
+    const bool depF = lane > 0, depB = lane < pp - 1;
+    volatile float *inF = endF + (depF ? lane - 1 : lane) * nj, *inB = endB + (depB ? lane + 1 : lane) * nj;
+    volatile float *outF = endF + lane * nj, *outB = endB + lane * nj;
+    const float dF = lane < pp ? durF[lane] : 0.f, dB = lane < pp ? durB[lane] : 0.f;
+    int nF = 0, nB = 0, done = 0, rounds = 0;
+    bool moved = false;
+    float clock = 0.f;
+    for (;;) {
+        if (done < total_ops) {
+            const bool isb = !(nF < warm || (nF < nj && nF - warm == nB));
+            const int j = isb ? nB : nF;
+            const bool dep = isb ? depB : depF;
+            const float e = (isb ? inB : inF)[j];
+            if (!dep || e >= 0.f) {
+                clock = fmaxf(clock, dep ? e + lat : 0.f) + (isb ? dB : dF);
+                (isb ? outB : outF)[j] = clock;
+                nF += isb ? 0 : 1;
+                nB += isb ? 1 : 0;
+                done++;
+                moved = true;
+            }
+        }
+        PF_SIM_ROUND_END()
+    }
+    st.clock = clock;
+}
+
+// Interleaved: v chunks per rank; unit k of a rank is microbatch (k / (pp v)) pp + k mod pp of chunk
+// (k mod (pp v)) / pp, backward units walk the chunks downward; cursors advance without divisions
+__device__ __forceinline__ void sim_rounds_interleaved(volatile float *endF, volatile float *endB, const float *durF,
+                                                       const float *durB, int lane, int pp, int v, int nj, int U,
+                                                       int warm, int total_ops, float lat, SimLane &st)
+{
+    const int Q = pp * v;
+    int nF = 0, nB = 0, done = 0, rounds = 0;
+    int fw = 0, fc = 0, fg = 0, bw = 0, bc = 0, bg = 0;
+    bool moved = false;
+    float clock = 0.f;
+    for (;;) {
+        if (done < total_ops) {
+            const bool isb = !(nF < warm || (nF < U && nF - warm == nB));
+            const int cw = isb ? bw : fw, cc = isb ? bc : fc, cg = isb ? bg : fg;
+            const int j = cg * pp + cw;
+            const int q = (isb ? v - 1 - cc : cc) * pp + lane;
+            const bool dep = isb ? (q < Q - 1) : (q > 0);
+            const int nb = dep ? (isb ? q + 1 : q - 1) : q;
+            volatile float *arr = isb ? endB : endF;
+            const float e = arr[nb * nj + j];
+            const float dur = (isb ? durB : durF)[q];
+            if (!dep || e >= 0.f) {
+                clock = fmaxf(clock, dep ? e + lat : 0.f) + dur;
+                arr[q * nj + j] = clock;
+                int w_ = cw + 1, c_ = cc, g_ = cg;
+                if (w_ == pp) {
+                    w_ = 0;
+                    if (++c_ == v) c_ = 0, g_++;
+                }
+                if (isb) bw = w_, bc = c_, bg = g_, nB++;
+                else fw = w_, fc = c_, fg = g_, nF++;
+                done++;
+                moved = true;
+            }
+        }
+        PF_SIM_ROUND_END()
+    }
+    st.clock = clock;
+}
+
+// DualPipe-style: two directions; the per-rank order comes from the host-built table
+__device__ __forceinline__ void sim_rounds_dual(volatile float *endF, volatile float *endB, const float *durF,
+                                                const float *durB, int lane, int pp, int nj, const uint8_t *ops,
+                                                int total_ops, float lat, SimLane &st)
+{
+    int done = 0, rounds = 0;
+    bool moved = false;
+    float clock = 0.f;
+    for (;;) {
+        if (done < total_ops) {
+            const uint32_t op = __ldg(ops + done);
+            const bool isb = op & 1;
+            const int d = (op >> 1) & 1, j = op >> 2;
+            const int q = d ? pp - 1 - lane : lane;
+            const int sidx = d * pp + q;
+            const bool dep = isb ? (q < pp - 1) : (q > 0);
+            const int nb = dep ? (isb ? sidx + 1 : sidx - 1) : sidx;
+            volatile float *arr = isb ? endB : endF;
+            const float e = arr[nb * nj + j];
+            const float dur = (isb ? durB : durF)[q];
+            if (!dep || e >= 0.f) {
+                clock = fmaxf(clock, dep ? e + lat : 0.f) + dur;
+                arr[sidx * nj + j] = clock;
+                done++;
+                moved = true;
+            }
+        }
+        PF_SIM_ROUND_END()
+    }
+    st.clock = clock;
+}
+#undef PF_SIM_ROUND_END
+
+// One launch serves every class.  A block owns a fixed pool of shared memory; while it works on class c as
+// many of its warps as fit (pool / footprint) pull candidates from that class' queue, the others wait at the
+// barrier that separates two classes.
 template <typename RI>
 __global__ void __launch_bounds__(kSimMaxWarps * 32) simulate_kernel(const __grid_constant__ DevPlan P, const SimArgs A)
 {
@@ -266,9 +391,18 @@ __global__ void __launch_bounds__(kSimMaxWarps * 32) simulate_kernel(const __gri
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint32_t seed_mixed = mix32(A.seed + 0x9e3779b9u);
 
-    for (int cls = A.cls_hi; cls >= 0; cls--) {
+    // Blocks start on different classes (cyclic, staggered by block number) so that all classes are in
+    // progress at once; a class whose queue is already drained is skipped, decided once per block.
+    __shared__ int s_skip;
+    const int n_classes = A.cls_hi + 1;
+    for (int step = 0; step < n_classes; step++) {
+    const int cls = (A.cls_hi - (int)(blockIdx.x % n_classes) - step + 2 * n_classes) % n_classes;
     const unsigned int n_cls = A.cls_count[cls];
-    if (n_cls == 0) continue;
+    if (threadIdx.x == 0) s_skip = *reinterpret_cast<volatile unsigned int *>(A.work + cls) >= n_cls;
+    __syncthreads();
+    const bool skip = s_skip != 0;
+    __syncthreads();
+    if (skip) continue;
     const int E = sim_class_entries(cls);
     const int per_warp = (int)sim_warp_floats(E, A.q_max);
     const int active_warps = min((int)(blockDim.x >> 5), A.pool_floats / per_warp);
@@ -359,81 +493,30 @@ __global__ void __launch_bounds__(kSimMaxWarps * 32) simulate_kernel(const __gri
         }
         __syncwarp();
 
-        // ---- per-lane order state
+        // ---- walk the rank's order
         const bool rank_active = lane < pp;
         const int U = dual ? 2 * nj : nj * (kind == PF_KIND_INTERLEAVED ? v : 1);  // forward units of this rank
-        int warm;
-        if (kind == PF_KIND_INTERLEAVED)
-            warm = min(2 * (pp - lane - 1) + (v - 1) * pp, U);
-        else
-            warm = min(pp - lane - 1, U);
-        // unit cursors (1F1B is the one-chunk case): microbatch = g*pp + w, chunk = c (backward: v-1-c)
-        int nF = 0, nB = 0;
-        int fc = 0, fw = 0, fg = 0;
-        int bc = 0, bw = 0, bg = 0;
         const uint8_t *dops = nullptr;
         if (dual && !stalled) {
             const int off = __ldg(A.dual_off + pp * 33 + nj);
             if (off < 0) stalled = true;  // no table for this shape: report instead of reading out of bounds
             else dops = A.dual_ops + off + (size_t)lane * 2 * m_sim;
         }
-        float clock = 0.f;
         const int total_ops = (rank_active && !stalled) ? 2 * U : 0;
-        int done_ops = 0;
-        int rounds = 0;
-        bool moved = false;
-        const float lat = T.p;
-
-        // One op per lane per round at most; the body is branch-free apart from the "not ready" exit, so the
-        // lanes of a warp stay converged and a round costs one shared-memory poll plus one vote.
-        for (;;) {
-            if (done_ops < total_ops) {
-                int isb, d = 0, q, j;
-                if (dual) {
-                    const uint32_t op = __ldg(dops + done_ops);
-                    isb = op & 1;
-                    d = (op >> 1) & 1;
-                    j = op >> 2;
-                    q = d ? pp - 1 - lane : lane;
-                } else {
-                    isb = !(nF < warm || (nF < U && nF - warm == nB));
-                    const int cw = isb ? bw : fw, cc = isb ? bc : fc, cg = isb ? bg : fg;
-                    j = cg * pp + cw;
-                    q = (isb ? v - 1 - cc : cc) * pp + lane;
-                }
-                const int sidx = d * Q + q;                  // stage stream (direction-major for DualPipe)
-                const bool has_dep = isb ? (q < Q - 1) : (q > 0);
-                const int nb = has_dep ? (isb ? sidx + 1 : sidx - 1) : sidx;
-                volatile float *in = isb ? endB : endF;
-                const float e = in[nb * nj + j];
-                const float dur = (isb ? durB : durF)[q];
-                if (!has_dep || e >= 0.f) {
-                    const float fin = fmaxf(clock, has_dep ? e + lat : 0.f) + dur;
-                    clock = fin;
-                    in[sidx * nj + j] = fin;
-                    if (!dual) {
-                        int w_ = (isb ? bw : fw) + 1, c_ = isb ? bc : fc, g_ = isb ? bg : fg;
-                        if (w_ == pp) {
-                            w_ = 0;
-                            if (++c_ == v) c_ = 0, g_++;
-                        }
-                        if (isb) bw = w_, bc = c_, bg = g_, nB++;
-                        else fw = w_, fc = c_, fg = g_, nF++;
-                    }
-                    done_ops++;
-                    moved = true;
-                }
-            }
-            if (!__any_sync(0xFFFFFFFFu, done_ops < total_ops)) break;
-            // bounded wait: every 64 rounds some lane must have advanced
-            if ((++rounds & 63) == 0) {
-                if (!__any_sync(0xFFFFFFFFu, moved)) {
-                    stalled = true;
-                    break;
-                }
-                moved = false;
-            }
+        SimLane sl;
+        sl.clock = 0.f;
+        sl.stalled = stalled;
+        if (!stalled) {
+            if (kind == PF_KIND_1F1B)
+                sim_rounds_1f1b(endF, endB, durF, durB, lane, pp, nj, min(pp - lane - 1, U), total_ops, T.p, sl);
+            else if (kind == PF_KIND_INTERLEAVED)
+                sim_rounds_interleaved(endF, endB, durF, durB, lane, pp, v, nj, U,
+                                       min(2 * (pp - lane - 1) + (v - 1) * pp, U), total_ops, T.p, sl);
+            else
+                sim_rounds_dual(endF, endB, durF, durB, lane, pp, nj, dops, total_ops, T.p, sl);
         }
+        stalled = sl.stalled;
+        const float clock = sl.clock;
 
         // ---- makespan, steady-state extension beyond the window, pricing
         float work = 0.f;
@@ -567,15 +650,12 @@ static int launch_simulate(pf_plan_t *p, SimArgs a, uint64_t n, cudaStream_t st,
     count_launch();
     (*n_kernels)++;
     PF_CUDA_TRY(cudaGetLastError(), "sim_classify_kernel launch");
-    PF_CUDA_TRY(cudaFuncSetAttribute(simulate_kernel<RI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     (int)(227 * 1024)),
-                "simulate_kernel smem");
     // largest class the plan can produce, and a pool that holds at least one such timeline
     const int entries_max = a.q_max * PF_SIM_WINDOW;
     int cls_hi = 0;
     while (cls_hi < kSimClasses - 1 && sim_class_entries(cls_hi) < entries_max) cls_hi++;
     const size_t biggest = sim_warp_floats(sim_class_entries(cls_hi), a.q_max) * sizeof(float);
-    if (biggest > 227 * 1024) return PF_EUNSUPPORTED;
+    if (biggest > 226 * 1024) return PF_EUNSUPPORTED;   // 227 KB per block minus the kernel's static words
     size_t pool = 72 * 1024;                         // three blocks per SM when the largest timeline allows
     if (pool < biggest) pool = biggest;
     int per_sm = (int)((size_t)(227 * 1024) / (pool + 1024));
@@ -584,6 +664,8 @@ static int launch_simulate(pf_plan_t *p, SimArgs a, uint64_t n, cudaStream_t st,
     a.pool_floats = (int)(pool / sizeof(float));
     const uint64_t cap = (uint64_t)p->sm_count * per_sm;
     const int grid = (int)(n < cap ? n : cap);
+    PF_CUDA_TRY(cudaFuncSetAttribute(simulate_kernel<RI>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pool),
+                "simulate_kernel smem");
     simulate_kernel<RI><<<grid, kSimMaxWarps * 32, pool, st>>>(p->dev, a);
     count_launch();
     (*n_kernels)++;
