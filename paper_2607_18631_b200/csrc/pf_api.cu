@@ -278,6 +278,14 @@ extern "C" int pf_plan_create(const pf_model_t *model, const pf_cluster_t *clust
         // ceil(2^32 / r): exact quotient by multiply-high for n < 2^32 / r, and n <= slab * ... <= 2^14
         d.magic[a] = d.radix[a] == 1 ? 0u : (uint32_t)(((1ull << 32) + d.radix[a] - 1) / d.radix[a]);
     }
+    // Per-slab table of rules 4-7 (batch, virtual stages, layers, microbatches): they depend on the layout
+    // and on (sched, mb, v) only, so when the layout axes are all outer a slab evaluates them once per
+    // (sched, mb, v) combination instead of once per candidate.
+    d.tab_n[0] = d.tab_n[1] = d.tab_n[2] = 0;
+    if (phase == PF_PHASE_TRAIN && n_inner <= 5) {
+        uint64_t n2 = n_inner > 2 ? d.radix[2] : 1, n3 = n_inner > 3 ? d.radix[3] : 1, n4 = n_inner > 4 ? d.radix[4] : 1;
+        if (n2 * n3 * n4 <= 2048) d.tab_n[0] = (int)n2, d.tab_n[1] = (int)n3, d.tab_n[2] = (int)n4;
+    }
     // leading rules whose axes are all outer (train: R1 tp,pp,dp,world; R2 tp; R3 ep,dp,tp; R4 dp,mb;
     // serve: R1 tp,dpa,ep; R2 tp; R3 ep,tp,dpa; R4 dpa,batch,ep)
     if (phase == PF_PHASE_TRAIN)

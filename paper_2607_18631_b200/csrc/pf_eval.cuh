@@ -11,7 +11,17 @@ namespace pf {
 
 typedef long long i64;
 
-__device__ __forceinline__ i64 cdiv64(i64 a, i64 b) { return (a + b - 1) / b; }
+// ceil(a / b) for a >= 0, b >= 1.  Parallel degrees are almost always powers of two: those take a shift
+// (the branch is uniform wherever the degree is, i.e. across a slab), anything else the 64-bit division.
+__device__ __forceinline__ i64 cdiv64(i64 a, i64 b)
+{
+    if ((b & (b - 1)) == 0) return (a + b - 1) >> (63 - __clzll(b));
+    return (a + b - 1) / b;
+}
+
+// fp32 quotient by reciprocal-multiply (2 ulp): the step-time model tolerates 1e-4 relative, and its ~20
+// quotients per candidate are otherwise the largest block of instructions in the cost model
+__device__ __forceinline__ float fdiv(float a, float b) { return __fdividef(a, b); }
 
 // tokens-per-expert bucket over the calibration domain [64, 8192]: <128, 128.., 256.., ..., >= 8192
 template <typename RI>
@@ -39,13 +49,13 @@ __device__ __forceinline__ float t_allreduce(i64 n, float bytes, Link lk)
 {
     if (n <= 1) return 0.f;
     float fn = (float)n;
-    return 2.f * (fn - 1.f) / fn * bytes / lk.bw + 2.f * ceil_log2f(n) * lk.alpha;
+    return fdiv(2.f * (fn - 1.f) * bytes, fn * lk.bw) + 2.f * ceil_log2f(n) * lk.alpha;
 }
 __device__ __forceinline__ float t_alltoall(i64 n, float bytes, Link lk)
 {
     if (n <= 1) return 0.f;
     float fn = (float)n;
-    return (fn - 1.f) / fn * bytes / lk.bw + lk.alpha;
+    return fdiv((fn - 1.f) * bytes, fn * lk.bw) + lk.alpha;
 }
 
 // ------------------------------------------------------------------ training
@@ -94,10 +104,11 @@ __device__ __forceinline__ int train_layout_rules(const DevPlan &P, const TrainT
     return 0;
 }
 
-// Rules 4-10.  Returns 0 or the failing rule; fills D.
+// Rules 4-10 (up to last_rule; rules 4-7 look at sched, mb, v and the layout only).  Returns 0 or the failing
+// rule; fills D.
 template <typename RI>
 __device__ __forceinline__ int train_plan_rules(const DevPlan &P, const TrainTuple &c, RI dp, RI world, int first_rule,
-                                                TrainDerived<RI> &D)
+                                                TrainDerived<RI> &D, int last_rule = 10)
 {
     D.dp = dp;
     D.world = world;
@@ -135,6 +146,7 @@ __device__ __forceinline__ int train_plan_rules(const DevPlan &P, const TrainTup
         if ((m & 1) != 0) return PF_R_MICROBATCH;
         if (c.pp > 1 && (c.pp & 1) != 0) return PF_R_MICROBATCH;
     }
+    if (last_rule < 8) return 0;
     RI tps = P.ep_scope ? (RI)c.tp : (RI)1;
     D.edp = P.ep_scope ? dp * (RI)c.tp / (RI)c.ep : dp / (RI)c.ep;
     D.m_e = (D.t * (RI)P.K * (RI)c.ep) / ((RI)P.E * tps);
@@ -196,32 +208,32 @@ __device__ __forceinline__ void train_times(const DevPlan &P, const TrainTuple &
     const DevKern &kn = P.kern[c.kv];
     const float t = (float)D.t, tp = (float)c.tp;
     const float dense_rate = tp * P.peak_flops * P.eff_dense;
-    const float cD = t * P.f_dense / dense_rate;
-    const float cE = t * P.f_exp / (tp * P.peak_flops * kn.dtype_mult * kn.eff[D.bucket]);
+    const float cD = fdiv(t * P.f_dense, dense_rate);
+    const float cE = fdiv(t * P.f_exp, tp * P.peak_flops * kn.dtype_mult * kn.eff[D.bucket]);
     const float cF = cD + cE, cB = P.bwd_factor * cF;
     float rc = 0.f;
     if (c.rec == PF_REC_SELECTIVE)
-        rc = (2.f / 3.f) * (cE + t * P.f_sh / dense_rate);
+        rc = (2.f / 3.f) * (cE + fdiv(t * P.f_sh, dense_rate));
     else if (c.rec == PF_REC_FULL)
         rc = cF;
     const i64 act_bytes = (i64)P.ab * (i64)D.t * (i64)P.H;  // one activation tensor of the microbatch
     const float tpc = 2.f * t_allreduce(c.tp, (float)act_bytes, link_of(P, c.tp));
-    const float a2a = 2.f * t_alltoall(c.ep, (float)(act_bytes * P.K) / tp, link_of(P, (i64)c.tp * c.ep));
+    const float a2a = 2.f * t_alltoall(c.ep, fdiv((float)(act_bytes * P.K), tp), link_of(P, (i64)c.tp * c.ep));
     const float hid = D.ov ? P.sched[c.s].hide_frac * a2a : 0.f;
     const float xF = a2a - fminf(hid, cF);
     const float xB = a2a - fminf(hid, cB + rc);
     T.F_l = cF + tpc + xF;
     T.B_l = cB + rc + tpc + xB + (c.rec == PF_REC_FULL ? tpc + xF : 0.f);
-    T.headF = t * P.f_head / dense_rate;
+    T.headF = fdiv(t * P.f_head, dense_rate);
     T.p = 0.f;
     if (c.pp > 1) {
         Link lw = link_of(P, (i64)D.world);
-        T.p = (float)act_bytes / tp / lw.bw + lw.alpha;
+        T.p = fdiv((float)act_bytes, tp * lw.bw) + lw.alpha;
     }
     Link ldp = link_of(P, (i64)c.tp * (i64)D.dp);
     const float gw = (float)(P.gb + P.wb);
     T.T_dp = t_allreduce((i64)D.dp, gw * (float)M.N_dense, ldp) + t_allreduce((i64)D.edp, gw * (float)M.N_exp, ldp);
-    T.T_opt = 2.f * (float)M.bytes_o / P.hbm_bw;
+    T.T_opt = fdiv(2.f * (float)M.bytes_o, P.hbm_bw);
 }
 
 // tokens/s/GPU from a pipeline time, with the realization taxes of the plans that pay them
@@ -230,10 +242,10 @@ __device__ __forceinline__ float train_price(const DevPlan &P, const TrainTuple 
                                              const TrainTimes &T, float T_pipe)
 {
     const float T_step = T_pipe + (1.f - P.dp_overlap_frac) * T.T_dp + T.T_opt + P.step_overhead;
-    float tput = (float)(P.gbs * (i64)P.seq) / (T_step * (float)D.world);
+    float tput = fdiv((float)(P.gbs * (i64)P.seq), T_step * (float)D.world);
     const DevKern &kn = P.kern[c.kv];
-    if (!kn.is_native) tput = tput / (1.f + kn.patch_ovh);
-    if (D.ov) tput = tput / (1.f + P.sched[c.s].sched_ovh);
+    if (!kn.is_native) tput = fdiv(tput, 1.f + kn.patch_ovh);
+    if (D.ov) tput = fdiv(tput, 1.f + P.sched[c.s].sched_ovh);
     return tput;
 }
 
@@ -243,12 +255,12 @@ __device__ __forceinline__ float train_pipe_analytic(const DevPlan &P, const Tra
                                                      const TrainTimes &T)
 {
     const float pp = (float)c.pp, m = (float)D.m;
-    const float F = (float)D.Ls * T.F_l + T.headF / pp;
-    const float B = (float)D.Ls * T.B_l + P.bwd_factor * T.headF / pp;
+    const float F = (float)D.Ls * T.F_l + fdiv(T.headF, pp);
+    const float B = (float)D.Ls * T.B_l + P.bwd_factor * fdiv(T.headF, pp);
     if (D.kind == PF_KIND_1F1B) return (m + pp - 1.f) * (F + B) + 2.f * (pp - 1.f) * T.p;
     if (D.kind == PF_KIND_INTERLEAVED)
-        return (m + (pp - 1.f) / (float)D.v_eff) * (F + B) + 2.f * (float)(D.Q - 1) * T.p;
-    return m * (F + B) + fmaxf(pp - 2.f, 0.f) * B + (F + B) / P.dualpipe_startup_div + 2.f * (pp - 1.f) * T.p;
+        return (m + fdiv(pp - 1.f, (float)D.v_eff)) * (F + B) + 2.f * (float)(D.Q - 1) * T.p;
+    return m * (F + B) + fmaxf(pp - 2.f, 0.f) * B + fdiv(F + B, P.dualpipe_startup_div) + 2.f * (pp - 1.f) * T.p;
 }
 
 // ------------------------------------------------------------------ serving
@@ -335,29 +347,29 @@ __device__ __forceinline__ void serve_eval(const DevPlan &P, const ServeTuple &c
     const float P_dl = (float)P.P_dl;
     const float dense_rate = ftp * peak * P.eff_dense;
     const float ctx = Pf + Of * 0.5f;
-    const float attn_w = (float)(P.P_dl * P.wb) / ftp;
+    const float attn_w = fdiv((float)(P.P_dl * P.wb), ftp);
     const float e_loc = (float)(P.E / c.ep);
-    const float exp_unit = (float)(P.P_e * kn.wbytes) / (float)moe_tp;
+    const float exp_unit = fdiv((float)(P.P_e * kn.wbytes), (float)moe_tp);
     const float moe_rate = nen * peak * kn.dtype_mult;
     const float KH = (float)((i64)P.K * P.H);
     // decode
-    const float touched_d = fminf(e_loc, fmaxf(1.f, (float)((i64)c.batch * P.K) / (float)c.ep));
-    const float t_attn_d = fmaxf(bl * (2.f * P_dl + 4.f * ctx * nh * dk) / dense_rate, (attn_w + bl * ctx * (float)kv_tok) / hbm);
-    const float t_moe_d = fmaxf((float)c.batch * P.f_exp / (moe_rate * kn.eff[b]), touched_d * exp_unit / hbm);
+    const float touched_d = fminf(e_loc, fmaxf(1.f, fdiv((float)((i64)c.batch * P.K), (float)c.ep)));
+    const float t_attn_d = fmaxf(fdiv(bl * (2.f * P_dl + 4.f * ctx * nh * dk), dense_rate), fdiv(attn_w + bl * ctx * (float)kv_tok, hbm));
+    const float t_moe_d = fmaxf(fdiv((float)c.batch * P.f_exp, moe_rate * kn.eff[b]), fdiv(touched_d * exp_unit, hbm));
     const float t_com_d = c.dpa ? 2.f * t_alltoall(n_eng, (float)P.ab * bl * KH, lk)
                                 : 2.f * t_allreduce(c.tp, (float)((i64)P.ab * c.batch * P.H), lk);
     const float T_dec = Lf * (t_attn_d + t_moe_d + t_com_d) + P.step_overhead;
     // chunked prefill
     const int nc = (Pn + c.chunk - 1) / c.chunk;
-    const float cl = Pf / (float)nc;
-    const float touched_p = fminf(e_loc, fmaxf(1.f, cl * (float)P.K / (float)c.ep));
-    const float t_attn_p = fmaxf(cl * (2.f * P_dl + 4.f * (Pf * 0.5f) * nh * dk) / dense_rate, attn_w / hbm);
-    const float t_moe_p = fmaxf(cl * P.f_exp / (moe_rate * kn.eff[b_pre]), touched_p * exp_unit / hbm);
+    const float cl = fdiv(Pf, (float)nc);
+    const float touched_p = fminf(e_loc, fmaxf(1.f, fdiv(cl * (float)P.K, (float)c.ep)));
+    const float t_attn_p = fmaxf(fdiv(cl * (2.f * P_dl + 4.f * (Pf * 0.5f) * nh * dk), dense_rate), fdiv(attn_w, hbm));
+    const float t_moe_p = fmaxf(fdiv(cl * P.f_exp, moe_rate * kn.eff[b_pre]), fdiv(touched_p * exp_unit, hbm));
     const float t_com_p = c.dpa ? 2.f * t_alltoall(n_eng, (float)P.ab * cl * KH, lk)
                                 : 2.f * t_allreduce(c.tp, (float)P.ab * cl * (float)P.H, lk);
     const float T_pre = (float)nc * Lf * (t_attn_p + t_moe_p + t_com_p);
-    float tput = (float)((i64)c.batch * On) / (bl * T_pre + Of * T_dec) / nen;
-    if (!kn.is_native) tput = tput / (1.f + kn.patch_ovh);
+    float tput = fdiv((float)((i64)c.batch * On), (bl * T_pre + Of * T_dec) * nen);
+    if (!kn.is_native) tput = fdiv(tput, 1.f + kn.patch_ovh);
     out.tput = tput;
     out.reason = (m_e < (RI)64 || m_e > (RI)8192) ? PF_FLAG_EXTRAPOLATED : PF_FEASIBLE;
 }

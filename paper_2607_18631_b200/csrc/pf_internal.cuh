@@ -12,6 +12,7 @@ namespace pf {
 constexpr int kThreads = 256;        // threads per block of the scoring kernel
 constexpr int kTopkCap = 2048;       // shared-memory candidate buffer per block (2 * PF_K_MAX)
 constexpr uint32_t kSlabMax = 16384; // upper bound on candidates per slab (inner-axis product)
+constexpr int kInnerVals = 1024;     // inner-axis values the scoring kernel keeps in shared memory
 
 struct DevSched {
     int kind, overlap, mapped;
@@ -38,6 +39,8 @@ struct DevPlan {
     int val_off[PF_MAX_AXES];      // offset of each axis' value list in the packed value array
     int wide;                      // 1: rule arithmetic needs 64-bit integers
     int sim_domain_all;            // 1: every feasible candidate lies inside the simulator's domain
+    int tab_n[3];                  // per-slab rule table over the inner ones of (sched, mb, v); 0 = not used
+    uint32_t slab_mul;             // slabs are visited in the order (s * slab_mul) mod n_slabs
     // --- model (Sec. 3.1) and host-derived per-layer constants
     int L, H, nh, nkv, hd, attn_kind, kv_latent, rope_dim, E, K, F, S, Fs, seq, vocab;
     int wb, gb, ob, ab, count_embeddings;

@@ -18,6 +18,7 @@ struct ScoreArgs {
     uint64_t first, count;          // range of this call
     uint64_t slab_lo;               // number of the first slab that intersects the range
     uint32_t n_slabs;               // slabs intersecting the range
+    uint32_t slab_mul;              // visiting order: slab (s * slab_mul) mod n_slabs, slab_mul coprime to n_slabs
     uint32_t k;
     uint8_t *reason;
     float *tput;
@@ -53,14 +54,20 @@ __device__ __forceinline__ void block_fill(uint8_t *p, uint64_t n, uint32_t b)
 }
 
 template <typename RI>
-__global__ void __launch_bounds__(kThreads) score_kernel(const __grid_constant__ DevPlan P, const ScoreArgs A)
+__global__ void __launch_bounds__(kThreads, 4) score_kernel(const __grid_constant__ DevPlan P, const ScoreArgs A)
 {
     __shared__ unsigned long long s_buf[kTopkCap];
     __shared__ int s_count;
     __shared__ unsigned long long s_thr;
-    __shared__ SlabInfo s_slab;
+    __shared__ SlabInfo s_slabs[2];
     __shared__ int s_base[2];
     __shared__ unsigned long long s_gthr;   // snapshot of the grid-wide threshold, refreshed once per slab
+    __shared__ uint8_t s_tab[2048];         // rules 4-7 per (sched, mb, v) combination of the current slab
+    __shared__ int32_t s_vals[kInnerVals];  // value lists of the inner axes (the packed array's prefix)
+    __shared__ uint16_t s_pass[2048];       // table entries of the current slab that pass rules 4-7
+    __shared__ int s_np;
+    __shared__ int s_qn;                    // candidates of the current slab queued for the cost model
+    extern __shared__ uint16_t s_queue[];   // their positions in the slab (P.slab entries, training plans)
 
     const int tid = threadIdx.x;
     const bool train = P.phase == PF_PHASE_TRAIN;
@@ -73,47 +80,61 @@ __global__ void __launch_bounds__(kThreads) score_kernel(const __grid_constant__
     int room_iters = kTopkCap / kThreads;
     unsigned long long thr = 0ull;
 
-    for (;;) {
-        __syncthreads();  // previous slab fully consumed before s_slab is overwritten
-        if (tid == 0) {
-            uint32_t s = atomicAdd(A.slab_counter, 1u);
-            s_gthr = want_topk ? *reinterpret_cast<volatile unsigned long long *>(A.g_thr) : 0ull;
-            SlabInfo si;
-            si.slab = s < A.n_slabs ? s : 0xFFFFFFFFu;
-            si.pre_reason = 0;
-            if (s < A.n_slabs) {
-                uint64_t o = A.slab_lo + s;
-                for (int a = P.n_inner; a < P.n_axes; a++) {
-                    uint64_t r = P.radix[a];
-                    uint64_t q = o / r;
-                    si.outer[a] = __ldg(A.vals + P.val_off[a] + (int)(o - q * r));
-                    o = q;
-                }
-                if (P.n_pre_rules > 0) {
-                    if (train) {
-                        TrainTuple c;
-                        c.mb = P.n_inner <= 3 ? si.outer[3] : 1;
-                        c.ep = P.n_inner <= 5 ? si.outer[5] : 1;
-                        c.pp = si.outer[6]; c.tp = si.outer[7]; c.dp = si.outer[8]; c.world = si.outer[9];
-                        RI dp, world;
-                        int r = train_layout_rules<RI>(P, c, 1, P.n_pre_rules < 3 ? P.n_pre_rules : 3, dp, world);
-                        if (r == 0 && P.n_pre_rules >= 4) {
-                            RI dpmb = dp * (RI)c.mb;
-                            if (((RI)P.gbs) % dpmb != 0) r = PF_R_BATCH;
-                        }
-                        si.pre_reason = r;
-                    } else {
-                        ServeTuple c;
-                        c.batch = P.n_inner <= 2 ? si.outer[2] : 1;
-                        c.dpa = si.outer[3]; c.ep = si.outer[4]; c.tp = si.outer[5];
-                        si.pre_reason = serve_layout_rules<RI>(P, c, 1, P.n_pre_rules >= 4);
+    // The inner axes' value lists are read once per candidate: keep them in shared memory.  Under the
+    // store stream of the fill slabs a read that misses L1 waits thousands of cycles in L2.
+    const int n_inner_vals = P.n_inner < P.n_axes ? P.val_off[P.n_inner] : P.val_off[P.n_axes - 1] + (int)P.radix[P.n_axes - 1];
+    const bool vals_in_smem = n_inner_vals <= kInnerVals;
+    if (vals_in_smem)
+        for (int i = tid; i < n_inner_vals; i += kThreads) s_vals[i] = A.vals[i];
+    const int32_t *inner_vals = vals_in_smem ? s_vals : A.vals;
+    // Slab tickets are double-buffered: while the block works on one slab, thread 0 already draws and decodes
+    // the next one, so the queue round trip and the outer-digit divisions stay off the critical path.
+    auto fetch_slab = [&](SlabInfo &dst) {
+        uint32_t s = atomicAdd(A.slab_counter, 1u);
+        s_gthr = want_topk ? *reinterpret_cast<volatile unsigned long long *>(A.g_thr) : 0ull;
+        SlabInfo si;
+        // heavy (evaluated) and light (constant-fill) slabs cluster in index order; a multiplicative
+        // permutation interleaves them so that arithmetic and store traffic overlap on every SM
+        si.slab = s < A.n_slabs ? (uint32_t)(((uint64_t)s * A.slab_mul) % A.n_slabs) : 0xFFFFFFFFu;
+        si.pre_reason = 0;
+        if (s < A.n_slabs) {
+            uint64_t o = A.slab_lo + si.slab;
+            for (int a = P.n_inner; a < P.n_axes; a++) {
+                uint64_t r = P.radix[a];
+                uint64_t q = o / r;
+                si.outer[a] = __ldg(A.vals + P.val_off[a] + (int)(o - q * r));
+                o = q;
+            }
+            if (P.n_pre_rules > 0) {
+                if (train) {
+                    TrainTuple c;
+                    c.mb = P.n_inner <= 3 ? si.outer[3] : 1;
+                    c.ep = P.n_inner <= 5 ? si.outer[5] : 1;
+                    c.pp = si.outer[6]; c.tp = si.outer[7]; c.dp = si.outer[8]; c.world = si.outer[9];
+                    RI dp, world;
+                    int r = train_layout_rules<RI>(P, c, 1, P.n_pre_rules < 3 ? P.n_pre_rules : 3, dp, world);
+                    if (r == 0 && P.n_pre_rules >= 4) {
+                        RI dpmb = dp * (RI)c.mb;
+                        if (((RI)P.gbs) % dpmb != 0) r = PF_R_BATCH;
                     }
+                    si.pre_reason = r;
+                } else {
+                    ServeTuple c;
+                    c.batch = P.n_inner <= 2 ? si.outer[2] : 1;
+                    c.dpa = si.outer[3]; c.ep = si.outer[4]; c.tp = si.outer[5];
+                    si.pre_reason = serve_layout_rules<RI>(P, c, 1, P.n_pre_rules >= 4);
                 }
             }
-            s_slab = si;
         }
-        __syncthreads();
+        dst = si;
+    };
+    if (tid == 0) fetch_slab(s_slabs[0]);
+    __syncthreads();
+
+    for (int cur = 0;; cur ^= 1) {
+        const SlabInfo &s_slab = s_slabs[cur];
         if (s_slab.slab == 0xFFFFFFFFu) break;
+        if (tid == 0) fetch_slab(s_slabs[cur ^ 1]);
 
         // candidate range of this slab clipped to the call's range
         const uint64_t slab_no = A.slab_lo + s_slab.slab;
@@ -128,86 +149,245 @@ __global__ void __launch_bounds__(kThreads) score_kernel(const __grid_constant__
             if (A.reason) block_fill(A.reason + rel0, n, (uint32_t)s_slab.pre_reason);
             if (A.tput) block_fill(reinterpret_cast<uint8_t *>(A.tput + rel0), (uint64_t)n * 4, 0u);
             if (A.mem) block_fill(reinterpret_cast<uint8_t *>(A.mem + rel0), (uint64_t)n * 8, 0u);
+            __syncthreads();  // the next ticket is complete and this one no longer read
             continue;
         }
 
         const uint32_t j0 = (uint32_t)(lo - base);
         const int first_rule = P.n_pre_rules + 1;
-        for (uint32_t it = 0; it < n; it += kThreads) {
-            const uint32_t i = it + tid;
-            const bool active = i < n;
-            int reason = 0;
-            float tput = 0.f;
-            long long mem = 0;
-            if (active) {
-                // inner digits by multiply-high division (exact: j * radix < 2^32)
-                uint32_t rem = j0 + i;
-                int v[PF_MAX_AXES];
+        const bool use_tab = train && P.tab_n[0] > 0;
+        if (use_tab) {
+            const int n2 = P.tab_n[0], n3 = P.tab_n[1], n4 = P.tab_n[2];
+            for (int e = tid; e < n2 * n3 * n4; e += kThreads) {
+                const int d2 = e % n2, d3 = (e / n2) % n3, d4 = e / (n2 * n3);
+                TrainTuple c;
+                c.kv = 0; c.rec = 0;
+                c.s = P.n_inner > 2 ? inner_vals[P.val_off[2] + d2] : s_slab.outer[2];
+                c.mb = P.n_inner > 3 ? inner_vals[P.val_off[3] + d3] : s_slab.outer[3];
+                c.v = P.n_inner > 4 ? inner_vals[P.val_off[4] + d4] : s_slab.outer[4];
+                c.ep = s_slab.outer[5]; c.pp = s_slab.outer[6]; c.tp = s_slab.outer[7];
+                c.dp = s_slab.outer[8]; c.world = s_slab.outer[9];
+                RI dp, world;
+                int r = train_layout_rules<RI>(P, c, first_rule, 3, dp, world);
+                if (r == 0) {
+                    TrainDerived<RI> D;
+                    r = train_plan_rules<RI>(P, c, dp, world, first_rule, D, 7);
+                }
+                s_tab[e] = (uint8_t)r;
+            }
+            __syncthreads();
+        }
+        // inner digits by multiply-high division (exact: j * radix < 2^32)
+        auto decode_inner = [&](uint32_t j, int (&v)[PF_MAX_AXES], int (&dg)[5]) {
+            uint32_t rem = j;
 #pragma unroll
-                for (int a = 0; a < PF_MAX_AXES; a++) {
-                    if (a < P.n_inner) {
-                        uint32_t r = P.radix[a];
-                        uint32_t q = r == 1u ? rem : __umulhi(rem, P.magic[a]);
-                        v[a] = __ldg(A.vals + P.val_off[a] + (int)(rem - q * r));
-                        rem = q;
-                    } else {
-                        v[a] = a < P.n_axes ? s_slab.outer[a] : 0;
+            for (int a = 0; a < PF_MAX_AXES; a++) {
+                if (a < P.n_inner) {
+                    uint32_t r = P.radix[a];
+                    uint32_t q = r == 1u ? rem : __umulhi(rem, P.magic[a]);
+                    const int digit = (int)(rem - q * r);
+                    if (a < 5) dg[a] = digit;
+                    v[a] = inner_vals[P.val_off[a] + digit];
+                    rem = q;
+                } else {
+                    v[a] = a < P.n_axes ? s_slab.outer[a] : 0;
+                }
+            }
+        };
+        // offer a scored candidate to the block's top-k buffer (block-collective, once per iteration)
+        auto offer = [&](bool feasible, float tput, uint32_t rel) {
+            if (!want_topk) return;
+            if (room_iters == 0) {
+                __syncthreads();
+                if (s_count > kTopkCap - kThreads) {
+                    tk_prune(s_buf, &s_count, &s_thr, (int)A.k);
+                    // a block's k-th key bounds the global k-th from below: share it
+                    if (tid == 0 && s_thr != 0ull) atomicMax(A.g_thr, s_thr);
+                }
+                room_iters = (kTopkCap - s_count) / kThreads;
+                thr = s_thr > s_gthr ? s_thr : s_gthr;
+                __syncthreads();
+            }
+            tk_push(s_buf, &s_count, thr, feasible, make_key(tput, rel));
+            room_iters--;
+        };
+
+        if (train) {
+            if (tid == 0) {
+                s_qn = 0;
+                s_np = 0;
+            }
+            __syncthreads();
+            if (use_tab) {
+                // Phase 1a.  Candidates that share (sched, mb, v) are contiguous: a run of R = |kv| x |rec|
+                // indices.  A warp takes 32 table entries at a time; runs whose entry holds a failing rule are
+                // written at once, cooperatively and coalesced; passing entries are only listed.
+                const uint32_t n_combos = (uint32_t)(P.tab_n[0] * P.tab_n[1] * P.tab_n[2]);
+                const uint32_t R = P.slab / n_combos;
+                const int lane = tid & 31, warp = tid >> 5;
+                for (uint32_t cb = (uint32_t)warp * 32; cb < n_combos; cb += (kThreads / 32) * 32) {
+                    const uint32_t e = cb + lane;
+                    const int t = e < n_combos ? (int)s_tab[e] : 0xFF;
+                    const unsigned pm = __ballot_sync(0xFFFFFFFFu, t == 0);
+                    if (pm) {
+                        const int leader = __ffs(pm) - 1;
+                        int pb = 0;
+                        if (lane == leader) pb = atomicAdd(&s_np, __popc(pm));
+                        pb = __shfl_sync(0xFFFFFFFFu, pb, leader);
+                        if (t == 0) s_pass[pb + __popc(pm & ((1u << lane) - 1u))] = (uint16_t)e;
+                    }
+                    const uint32_t cnt = min(32u, n_combos - cb) * R;
+                    for (uint32_t xb = 0; xb < cnt; xb += 32) {
+                        const uint32_t x = xb + lane;
+                        const uint32_t run = min(x / R, 31u);
+                        const int r = __shfl_sync(0xFFFFFFFFu, t, (int)run);
+                        const uint32_t j = cb * R + x;
+                        if (x < cnt && r != 0 && j >= j0 && j < j0 + n) {
+                            const uint64_t o = rel0 + (j - j0);
+                            if (A.reason) A.reason[o] = (uint8_t)r;
+                            if (A.tput) A.tput[o] = 0.f;
+                            if (A.mem) A.mem[o] = 0;
+                        }
                     }
                 }
-                if (train) {
+                __syncthreads();
+                // Phase 1b.  The candidates of the passing entries, densely: kernel availability and the
+                // emit dry-run rules (8-10).  Rejected ones are written, the rest queued for the cost model.
+                const uint32_t total = (uint32_t)s_np * R;
+                for (uint32_t it = 0; it < total; it += kThreads) {
+                    const uint32_t x = it + tid;
+                    bool queued = false;
+                    uint32_t i = 0;
+                    if (x < total) {
+                        const uint32_t pe = x / R;
+                        const uint32_t j = (uint32_t)s_pass[pe] * R + (x - pe * R);
+                        if (j >= j0 && j < j0 + n) {
+                            i = j - j0;
+                            int v[PF_MAX_AXES], dg[5] = {0, 0, 0, 0, 0};
+                            decode_inner(j, v, dg);
+                            TrainTuple c;
+                            c.kv = v[0]; c.rec = v[1]; c.s = v[2]; c.mb = v[3]; c.v = v[4];
+                            c.ep = v[5]; c.pp = v[6]; c.tp = v[7]; c.dp = v[8]; c.world = v[9];
+                            RI dp, world;
+                            TrainDerived<RI> D;
+                            train_layout_rules<RI>(P, c, 4, 3, dp, world);   // derives dp / world only
+                            const int reason = train_plan_rules<RI>(P, c, dp, world, 4, D);
+                            if (reason != 0) {
+                                const uint64_t o = rel0 + i;
+                                if (A.reason) A.reason[o] = (uint8_t)reason;
+                                if (A.tput) A.tput[o] = 0.f;
+                                if (A.mem) A.mem[o] = 0;
+                            } else {
+                                queued = true;
+                            }
+                        }
+                    }
+                    const unsigned mask = __ballot_sync(0xFFFFFFFFu, queued);
+                    if (mask) {
+                        const int lane2 = tid & 31, leader = __ffs(mask) - 1;
+                        int qb = 0;
+                        if (lane2 == leader) qb = atomicAdd(&s_qn, __popc(mask));
+                        qb = __shfl_sync(0xFFFFFFFFu, qb, leader);
+                        if (queued) s_queue[qb + __popc(mask & ((1u << lane2) - 1u))] = (uint16_t)i;
+                    }
+                }
+            } else {
+            // Phase 1 without a rule table: integer rules for every candidate of the slab.  Rejected
+            // candidates are written at once; the ones that reach the memory gate are only queued, because
+            // they come in short runs and would leave most lanes of their warps idle.
+            for (uint32_t it = 0; it < n; it += kThreads) {
+                const uint32_t i = it + tid;
+                bool queued = false;
+                if (i < n) {
+                    int v[PF_MAX_AXES], dg[5] = {0, 0, 0, 0, 0};
+                    decode_inner(j0 + i, v, dg);
                     TrainTuple c;
                     c.kv = v[0]; c.rec = v[1]; c.s = v[2]; c.mb = v[3]; c.v = v[4];
                     c.ep = v[5]; c.pp = v[6]; c.tp = v[7]; c.dp = v[8]; c.world = v[9];
                     RI dp, world;
-                    reason = train_layout_rules<RI>(P, c, first_rule, 3, dp, world);
+                    int reason = train_layout_rules<RI>(P, c, first_rule, 3, dp, world);
                     if (reason == 0) {
                         TrainDerived<RI> D;
                         reason = train_plan_rules<RI>(P, c, dp, world, first_rule, D);
-                        if (reason == 0) {
-                            TrainMem M;
-                            train_memory<RI>(P, c, D, M);
-                            mem = M.mem;
-                            if (mem > P.budget_bytes) {
-                                reason = PF_R_MEMORY;
-                            } else {
-                                TrainTimes T;
-                                train_times<RI>(P, c, D, M, T);
-                                tput = train_price<RI>(P, c, D, T, train_pipe_analytic<RI>(P, c, D, T));
-                                if (D.m_e < (RI)64 || D.m_e > (RI)8192) reason = PF_FLAG_EXTRAPOLATED;
-                            }
-                        }
                     }
-                } else {
+                    if (reason != 0) {
+                        const uint64_t o = rel0 + i;
+                        if (A.reason) A.reason[o] = (uint8_t)reason;
+                        if (A.tput) A.tput[o] = 0.f;
+                        if (A.mem) A.mem[o] = 0;
+                    } else {
+                        queued = true;
+                    }
+                }
+                const unsigned mask = __ballot_sync(0xFFFFFFFFu, queued);
+                if (mask) {
+                    const int lane = tid & 31, leader = __ffs(mask) - 1;
+                    int qb = 0;
+                    if (lane == leader) qb = atomicAdd(&s_qn, __popc(mask));
+                    qb = __shfl_sync(0xFFFFFFFFu, qb, leader);
+                    if (queued) s_queue[qb + __popc(mask & ((1u << lane) - 1u))] = (uint16_t)i;
+                }
+            }
+            }
+            __syncthreads();
+            // Phase 2: memory model, gate, step time and pricing for the queued candidates, one per thread,
+            // every warp full.
+            const uint32_t qn = (uint32_t)s_qn;
+            for (uint32_t it = 0; it < qn; it += kThreads) {
+                const uint32_t qi = it + tid;
+                const bool active = qi < qn;
+                int reason = 0;
+                float tput = 0.f;
+                uint32_t i = 0;
+                if (active) {
+                    i = s_queue[qi];
+                    int v[PF_MAX_AXES], dg[5] = {0, 0, 0, 0, 0};
+                    decode_inner(j0 + i, v, dg);
+                    TrainTuple c;
+                    c.kv = v[0]; c.rec = v[1]; c.s = v[2]; c.mb = v[3]; c.v = v[4];
+                    c.ep = v[5]; c.pp = v[6]; c.tp = v[7]; c.dp = v[8]; c.world = v[9];
+                    RI dp, world;
+                    TrainDerived<RI> D;
+                    train_layout_rules<RI>(P, c, 4, 3, dp, world);      // derives dp / world only
+                    train_plan_rules<RI>(P, c, dp, world, 4, D);        // passed in phase 1: fills D
+                    TrainMem M;
+                    train_memory<RI>(P, c, D, M);
+                    if (M.mem > P.budget_bytes) {
+                        reason = PF_R_MEMORY;
+                    } else {
+                        TrainTimes T;
+                        train_times<RI>(P, c, D, M, T);
+                        tput = train_price<RI>(P, c, D, T, train_pipe_analytic<RI>(P, c, D, T));
+                        if (D.m_e < (RI)64 || D.m_e > (RI)8192) reason = PF_FLAG_EXTRAPOLATED;
+                    }
+                    const uint64_t o = rel0 + i;
+                    if (A.reason) A.reason[o] = (uint8_t)reason;
+                    if (A.tput) A.tput[o] = tput;
+                    if (A.mem) A.mem[o] = M.mem;
+                }
+                offer(active && (reason & 0x7f) == 0, tput, (uint32_t)(rel0 + i));
+            }
+        } else {
+            for (uint32_t it = 0; it < n; it += kThreads) {
+                const uint32_t i = it + tid;
+                const bool active = i < n;
+                ServeOut so;
+                so.reason = 0; so.tput = 0.f; so.mem = 0;
+                if (active) {
+                    int v[PF_MAX_AXES], dg[5] = {0, 0, 0, 0, 0};
+                    decode_inner(j0 + i, v, dg);
                     ServeTuple c;
                     c.kv = v[0]; c.chunk = v[1]; c.batch = v[2]; c.dpa = v[3]; c.ep = v[4]; c.tp = v[5]; c.scen = v[6];
-                    ServeOut so;
                     serve_eval<RI>(P, c, first_rule, __ldg(A.scen + c.scen), __ldg(A.scen + P.n_scen + c.scen), so);
-                    reason = so.reason;
-                    tput = so.tput;
-                    mem = so.mem;
+                    const uint64_t o = rel0 + i;
+                    if (A.reason) A.reason[o] = (uint8_t)so.reason;
+                    if (A.tput) A.tput[o] = so.tput;
+                    if (A.mem) A.mem[o] = so.mem;
                 }
-                const uint64_t o = rel0 + i;
-                if (A.reason) A.reason[o] = (uint8_t)reason;
-                if (A.tput) A.tput[o] = tput;
-                if (A.mem) A.mem[o] = mem;
-            }
-            if (want_topk) {
-                if (room_iters == 0) {
-                    __syncthreads();
-                    if (s_count > kTopkCap - kThreads) {
-                        tk_prune(s_buf, &s_count, &s_thr, (int)A.k);
-                        // a block's k-th key bounds the global k-th from below: share it
-                        if (tid == 0 && s_thr != 0ull) atomicMax(A.g_thr, s_thr);
-                    }
-                    room_iters = (kTopkCap - s_count) / kThreads;
-                    thr = s_thr > s_gthr ? s_thr : s_gthr;
-                    __syncthreads();
-                }
-                const bool feasible = active && (reason & 0x7f) == 0;
-                tk_push(s_buf, &s_count, thr, feasible, make_key(tput, (uint32_t)(rel0 + i)));
-                room_iters--;
+                offer(active && (so.reason & 0x7f) == 0, so.tput, (uint32_t)(rel0 + i));
             }
         }
+        __syncthreads();  // the next ticket is complete and this one no longer read
     }
 
     if (want_topk) {
@@ -430,6 +610,14 @@ extern "C" int pf_score(pf_plan_t *p, uint64_t first, uint64_t count, uint8_t *d
 
     ScoreArgs a;
     a.first = first; a.count = count; a.slab_lo = slab_lo; a.n_slabs = (uint32_t)n_slabs; a.k = k;
+    {
+        // a multiplier near 0.618 * n_slabs that is coprime to n_slabs: consecutive queue tickets land far apart
+        uint64_t n = n_slabs, m = (uint64_t)((double)n_slabs * 0.6180339887) | 1;
+        auto gcd = [](uint64_t x, uint64_t y) { while (y) { uint64_t t = x % y; x = y; y = t; } return x; };
+        while (m > 1 && gcd(m, n) != 1) m -= 2;
+        if (n <= 2 || m < 1) m = 1;
+        a.slab_mul = (uint32_t)m;
+    }
     a.reason = d_reason; a.tput = d_tput; a.mem = (long long *)d_mem;
     a.keys = (unsigned long long *)(ws + lay.off_keys_a);
     a.slab_counter = (unsigned int *)(ws + lay.off_ctrl);
@@ -437,11 +625,19 @@ extern "C" int pf_score(pf_plan_t *p, uint64_t first, uint64_t count, uint8_t *d
     a.g_thr = (unsigned long long *)(ws + lay.off_ctrl + 16);
     a.vals = p->d_vals; a.scen = p->d_scen;
     PF_CUDA_TRY(cudaMemsetAsync(a.slab_counter, 0, 256, st), "pf_score: counter reset");
+    const size_t queue_bytes = p->dev.phase == PF_PHASE_TRAIN ? (size_t)p->dev.slab * sizeof(uint16_t) : 0;
+    // static + dynamic shared memory passes the 48 KB default for large slabs: opt in
+    if (p->dev.wide)
+        PF_CUDA_TRY(cudaFuncSetAttribute(score_kernel<unsigned long long>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)queue_bytes), "score_kernel smem");
+    else
+        PF_CUDA_TRY(cudaFuncSetAttribute(score_kernel<uint32_t>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)queue_bytes), "score_kernel smem");
     timing_begin(p, PF_T_SCORE, st);
     if (p->dev.wide)
-        score_kernel<unsigned long long><<<grid, kThreads, 0, st>>>(p->dev, a);
+        score_kernel<unsigned long long><<<grid, kThreads, queue_bytes, st>>>(p->dev, a);
     else
-        score_kernel<uint32_t><<<grid, kThreads, 0, st>>>(p->dev, a);
+        score_kernel<uint32_t><<<grid, kThreads, queue_bytes, st>>>(p->dev, a);
     count_launch();
     timing_end(p, PF_T_SCORE, 1, st);
     PF_CUDA_TRY(cudaGetLastError(), "score_kernel launch");
