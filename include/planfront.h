@@ -195,6 +195,32 @@ int pf_score(pf_plan_t *plan, uint64_t first, uint64_t count, uint8_t *d_reason,
              uint32_t k, uint64_t *d_topk_idx, float *d_topk_score, uint32_t *d_topk_count, void *d_workspace,
              size_t workspace_bytes, void *stream);
 
+/* pf_score for callers that must not allocate device memory when they call it.  (The paper has no
+ * counterpart: this is a deployment convenience of this library.)
+ *
+ * Who needs it: code that runs where a device allocation is unavailable or forbidden -- a service whose
+ * whole device memory is handed to a pool at start-up, a latency-critical loop in which the implicit device
+ * synchronization of an allocation is not acceptable, a plugin that is given buffers by its host application
+ * and has no allocator of its own.  Such a caller can usually still provide the inputs and the result
+ * buffers, but has nowhere to take pf_score's workspace from.
+ *
+ * Same arguments and results as pf_score, minus the workspace: the scratch memory (work counters and the
+ * blocks' candidate key lists) lives in a fixed array of PF_STATIC_SCRATCH_BYTES inside the library's device
+ * image.  Every GPU that loads the library carries that array until the process exits.
+ *   - The call allocates nothing and frees nothing (no cudaMalloc / cudaFree, no allocating library routine).
+ *   - The FIRST call on each device looks up the array's device address (once per device, with that device
+ *     current); make that first call before any stream capture begins.
+ *   - All calls on one device share the one array, which keeps the previous call's contents; the call clears
+ *     the words that must start at zero.  Two calls whose device work overlaps (different streams, different
+ *     threads) race on it: issue them on one stream, or order them yourself.
+ *   - A request whose workspace need (pf_score_workspace) exceeds PF_STATIC_SCRATCH_BYTES is refused with
+ *     PF_EWORKSPACE before anything is launched; use pf_score with your own workspace for it.
+ * Errors: as pf_score; PF_ECUDA also if the address look-up fails. */
+#define PF_STATIC_SCRATCH_BYTES (4u << 20)
+int pf_score_static(pf_plan_t *plan, uint64_t first, uint64_t count, uint8_t *d_reason, float *d_tput,
+                    int64_t *d_mem, uint32_t k, uint64_t *d_topk_idx, float *d_topk_score, uint32_t *d_topk_count,
+                    void *stream);
+
 /* Merge two top-k lists (as written by pf_score / pf_simulate, each sorted, with device counts) into the k
  * best of their union, same ordering rule.  Used to combine chunks or shards of one space.  The output
  * may alias neither input.  Errors: PF_EINVAL (k out of range, NULL). */

@@ -23,7 +23,8 @@ UINT64_MAX = 0xFFFFFFFFFFFFFFFF
 EXPORTS = ("pf_version", "pf_strerror", "pf_reason_str", "pf_last_cuda_error", "pf_plan_create", "pf_plan_destroy",
            "pf_plan_size", "pf_decode", "pf_score_workspace", "pf_score", "pf_topk_merge", "pf_select_workspace",
            "pf_select_survivors", "pf_simulate_workspace", "pf_simulate", "pf_search_workspace", "pf_search_host",
-           "pf_launch_count", "pf_dualpipe_order", "pf_timing_enable", "pf_timing_read")
+           "pf_launch_count", "pf_dualpipe_order", "pf_timing_enable", "pf_timing_read", "pf_score_static")
+STATIC_SCRATCH_BYTES = 4 << 20
 T_CLASSES = ("score", "topk", "select", "simulate")
 
 i32, u32, i64, u64, f32 = C.c_int32, C.c_uint32, C.c_int64, C.c_uint64, C.c_float
@@ -111,6 +112,8 @@ def load_library(path: str | None = None):
     L.pf_score_workspace.argtypes = [vp, u64, u32]
     L.pf_score.restype = C.c_int
     L.pf_score.argtypes = [vp, u64, u64, vp, vp, vp, u32, vp, vp, vp, vp, sz, vp]
+    L.pf_score_static.restype = C.c_int
+    L.pf_score_static.argtypes = [vp, u64, u64, vp, vp, vp, u32, vp, vp, vp, vp]
     L.pf_topk_merge.restype = C.c_int
     L.pf_topk_merge.argtypes = [u32, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
     L.pf_select_workspace.restype = sz
@@ -294,6 +297,18 @@ class Plan:
                                 _stream_ptr(torch, stream)), "pf_score")
         return dict(reason=reason, tput=tput, mem=mem, topk_idx=topk_idx, topk_score=topk_score,
                     topk_count=topk_count, workspace=workspace)
+
+    # ---- pf_score_static
+    def score_static(self, reason, tput, mem, k: int, topk_idx, topk_score, topk_count, first: int = 0,
+                     count: int | None = None, stream=None):
+        """Enqueue pf_score_static: the caller passes every buffer, nothing is allocated here or in the library
+        (the scratch is the library's built-in array).  Does not synchronize."""
+        torch = _torch()
+        if count is None:
+            count = self.size - first
+        _check(self._L.pf_score_static(self._h, first, count, _dptr(reason), _dptr(tput), _dptr(mem), k,
+                                       _dptr(topk_idx), _dptr(topk_score), _dptr(topk_count),
+                                       _stream_ptr(torch, stream)), "pf_score_static")
 
     # ---- pf_select_survivors
     def select_workspace(self, count: int, s_max: int) -> int:

@@ -652,6 +652,46 @@ extern "C" int pf_score(pf_plan_t *p, uint64_t first, uint64_t count, uint8_t *d
     return PF_OK;
 }
 
+// ------------------------------------------------------------------ pf_score without a caller workspace
+// The scratch of pf_score_static: part of the device image, one copy per GPU that loads the library.
+// In host code this name is only a handle for cudaGetSymbolAddress, never a device address.
+static __device__ __align__(256) unsigned char g_static_scratch[PF_STATIC_SCRATCH_BYTES];
+
+#include <mutex>
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mu;
+void *g_static_ptr[kMaxDevices];   // device address of g_static_scratch, per device ordinal
+}  // namespace
+
+extern "C" int pf_score_static(pf_plan_t *p, uint64_t first, uint64_t count, uint8_t *d_reason, float *d_tput,
+                               int64_t *d_mem, uint32_t k, uint64_t *d_topk_idx, float *d_topk_score,
+                               uint32_t *d_topk_count, void *stream)
+{
+    if (!p) return PF_EINVAL;
+    if (k > PF_K_MAX) return PF_EINVAL;
+    if (count == 0 || count >= PF_MAX_COUNT) return PF_ERANGE;
+    // refuse what the fixed array cannot hold before touching the device
+    if (pf_score_workspace(p, count, k) > (size_t)PF_STATIC_SCRATCH_BYTES) return PF_EWORKSPACE;
+    int dev = -1;
+    PF_CUDA_TRY(cudaGetDevice(&dev), "pf_score_static: current device");
+    if (dev < 0 || dev >= kMaxDevices) return PF_EUNSUPPORTED;
+    void *scratch = nullptr;
+    {
+        // once per device, with that device current: ask the runtime where the array lives on it
+        std::lock_guard<std::mutex> lock(g_static_mu);
+        if (!g_static_ptr[dev]) {
+            void *ptr = nullptr;
+            PF_CUDA_TRY(cudaGetSymbolAddress(&ptr, g_static_scratch), "pf_score_static: scratch address");
+            g_static_ptr[dev] = ptr;
+        }
+        scratch = g_static_ptr[dev];
+    }
+    // pf_score clears the counters it needs at the start of every call; the rest is written before it is read
+    return pf_score(p, first, count, d_reason, d_tput, d_mem, k, d_topk_idx, d_topk_score, d_topk_count, scratch,
+                    (size_t)PF_STATIC_SCRATCH_BYTES, stream);
+}
+
 extern "C" int pf_topk_merge(uint32_t k, const uint64_t *d_idx_a, const float *d_score_a, const uint32_t *d_count_a,
                              const uint64_t *d_idx_b, const float *d_score_b, const uint32_t *d_count_b,
                              uint64_t *d_idx_out, float *d_score_out, uint32_t *d_count_out, void *stream)
