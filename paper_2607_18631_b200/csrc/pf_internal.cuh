@@ -117,36 +117,93 @@ __device__ __forceinline__ uint32_t key_rel(unsigned long long key) { return 0xF
 // threshold (the k-th best key once k are held, else 0).  All functions are block-collective unless
 // noted; the block may have any multiple of 32 threads.
 
-// Descending bitonic sort of buf[0, n_sort) in shared memory; n_sort a power of two <= kTopkCap.
-// Thread i takes compare-exchange pairs i, i + blockDim, ...; for strides <= 32 the 32 pairs of a warp lie
-// in one 64-element window that no other warp touches, so those stages need only a warp barrier.  A block
-// barrier is used when a stage is wider than that or follows one that was.
+// Descending bitonic sort of buf[0, n_sort); n_sort a power of two <= kTopkCap; buf has room for 64 keys at
+// least.  PAIRS = kTopkCap / 2 / blockDim.x.  Each thread owns adjacent elements (2p, 2p+1) for its pair
+// numbers p = tid, tid + blockDim, ...; a warp therefore owns a 64-element window.  All compare-exchanges
+// with stride <= 32 stay inside that window: they run on registers with warp shuffles.  Only the wider
+// strides (>= 64) go through shared memory with block barriers.
+template <int PAIRS>
 __device__ inline void tk_sort_desc(unsigned long long *buf, int n_sort)
 {
-    const int tid = threadIdx.x, nt = blockDim.x;
-    int prev_stride = 64;  // whatever filled the buffer was block-wide
-    for (int size = 2; size <= n_sort; size <<= 1) {
-        for (int stride = size >> 1; stride > 0; stride >>= 1) {
-            if (stride > 32 || prev_stride > 32) __syncthreads();
-            else __syncwarp();
-            prev_stride = stride;
-            for (int i = tid; i < n_sort / 2; i += nt) {
-                int lo = 2 * i - (i & (stride - 1));  // element with the stride bit clear
-                int hi = lo + stride;
-                bool desc = ((lo & size) == 0);       // direction of this bitonic block
-                unsigned long long a = buf[lo], b = buf[hi];
-                bool swap = desc ? (a < b) : (a > b);
-                if (swap) {
-                    buf[lo] = b;
-                    buf[hi] = a;
+    const int tid = threadIdx.x, nt = blockDim.x, lane = tid & 31;
+    const int n_eff = n_sort < 64 ? 64 : n_sort;   // whole warps take part; missing elements are zeros
+    unsigned long long r0[PAIRS], r1[PAIRS];
+    __syncthreads();
+#pragma unroll
+    for (int t = 0; t < PAIRS; t++) {
+        const int i0 = 2 * (tid + t * nt);
+        r0[t] = i0 < n_sort ? buf[i0] : 0ull;
+        r1[t] = i0 + 1 < n_sort ? buf[i0 + 1] : 0ull;
+    }
+    for (int size = 2; size <= n_eff; size <<= 1) {
+        int stride = size >> 1;
+        if (stride >= 64) {
+#pragma unroll
+            for (int t = 0; t < PAIRS; t++) {
+                const int i0 = 2 * (tid + t * nt);
+                if (i0 < n_eff) {
+                    buf[i0] = r0[t];
+                    buf[i0 + 1] = r1[t];
                 }
             }
+            for (; stride >= 64; stride >>= 1) {
+                __syncthreads();
+                for (int i = tid; i < n_eff / 2; i += nt) {
+                    const int lo = 2 * i - (i & (stride - 1)), hi = lo + stride;
+                    const bool desc = (lo & size) == 0;
+                    const unsigned long long a = buf[lo], b = buf[hi];
+                    if (desc ? (a < b) : (a > b)) {
+                        buf[lo] = b;
+                        buf[hi] = a;
+                    }
+                }
+            }
+            __syncthreads();
+#pragma unroll
+            for (int t = 0; t < PAIRS; t++) {
+                const int i0 = 2 * (tid + t * nt);
+                if (i0 < n_eff) {
+                    r0[t] = buf[i0];
+                    r1[t] = buf[i0 + 1];
+                }
+            }
+        }
+        for (; stride >= 1; stride >>= 1) {
+#pragma unroll
+            for (int t = 0; t < PAIRS; t++) {
+                const int i0 = 2 * (tid + t * nt);
+                if (i0 >= n_eff) continue;   // whole warps only: n_eff / 2 is a multiple of 32
+                const bool desc = (i0 & size) == 0;
+                if (stride == 1) {
+                    const unsigned long long a = r0[t], b = r1[t];
+                    if (desc ? (a < b) : (a > b)) {
+                        r0[t] = b;
+                        r1[t] = a;
+                    }
+                } else {
+                    const int lm = stride >> 1;
+                    const unsigned long long o0 = __shfl_xor_sync(0xFFFFFFFFu, r0[t], lm);
+                    const unsigned long long o1 = __shfl_xor_sync(0xFFFFFFFFu, r1[t], lm);
+                    const bool keep_max = ((lane & lm) == 0) == desc;
+                    r0[t] = keep_max ? (r0[t] > o0 ? r0[t] : o0) : (r0[t] < o0 ? r0[t] : o0);
+                    r1[t] = keep_max ? (r1[t] > o1 ? r1[t] : o1) : (r1[t] < o1 ? r1[t] : o1);
+                }
+            }
+        }
+    }
+#pragma unroll
+    for (int t = 0; t < PAIRS; t++) {
+        const int i0 = 2 * (tid + t * nt);
+        if (i0 < n_eff) {
+            buf[i0] = r0[t];
+            buf[i0 + 1] = r1[t];
         }
     }
     __syncthreads();
 }
 
 // Keep the best k: sort what is held (padded to a power of two), clamp the count, refresh the threshold.
+template <int PAIRS>
 __device__ inline void tk_prune(unsigned long long *buf, int *count, unsigned long long *thr, int k)
 {
     __syncthreads();
@@ -155,7 +212,7 @@ __device__ inline void tk_prune(unsigned long long *buf, int *count, unsigned lo
     int n_sort = 32;
     while (n_sort < c) n_sort <<= 1;
     for (int i = c + threadIdx.x; i < n_sort; i += blockDim.x) buf[i] = 0ull;
-    tk_sort_desc(buf, n_sort);
+    tk_sort_desc<PAIRS>(buf, n_sort);
     if (threadIdx.x == 0) {
         int n = c < k ? c : k;
         *count = n;

@@ -200,7 +200,7 @@ __global__ void __launch_bounds__(kThreads, 4) score_kernel(const __grid_constan
             if (room_iters == 0) {
                 __syncthreads();
                 if (s_count > kTopkCap - kThreads) {
-                    tk_prune(s_buf, &s_count, &s_thr, (int)A.k);
+                    tk_prune<kTopkCap / 2 / kThreads>(s_buf, &s_count, &s_thr, (int)A.k);
                     // a block's k-th key bounds the global k-th from below: share it
                     if (tid == 0 && s_thr != 0ull) atomicMax(A.g_thr, s_thr);
                 }
@@ -391,7 +391,7 @@ __global__ void __launch_bounds__(kThreads, 4) score_kernel(const __grid_constan
     }
 
     if (want_topk) {
-        tk_prune(s_buf, &s_count, &s_thr, (int)A.k);
+        tk_prune<kTopkCap / 2 / kThreads>(s_buf, &s_count, &s_thr, (int)A.k);
         if (tid == 0) {
             if (s_thr != 0ull) atomicMax(A.g_thr, s_thr);
             s_thr = *reinterpret_cast<volatile unsigned long long *>(A.g_thr);
@@ -409,6 +409,7 @@ struct ReduceArgs {
     unsigned long long *out;        // compact keys of the next pass (when not final)
     unsigned int *out_count;
     uint32_t k;
+    unsigned int seg;               // keys per block
     int final;                      // 1: write idx / score / count (gridDim.x == 1)
     uint64_t first;
     const uint64_t *idx_map;        // NULL: idx = first + rel; else idx = idx_map[rel]
@@ -417,8 +418,9 @@ struct ReduceArgs {
     uint32_t *topk_count;
 };
 
-// Block b walks keys [b*kReduceSeg, (b+1)*kReduceSeg) of the input one tile at a time, admitting only keys
-// above its running k-th best, and keeps the k best.
+// Block b walks keys [b*seg, (b+1)*seg) of the input one tile at a time, admitting only keys above its
+// running k-th best, and keeps the k best.  A tile's admissions are counted before they are appended, so the
+// buffer is pruned only when it would really overflow.
 __global__ void __launch_bounds__(kReduceThreads) reduce_kernel(const ReduceArgs A)
 {
     __shared__ unsigned long long s_buf[kTopkCap];
@@ -427,25 +429,27 @@ __global__ void __launch_bounds__(kReduceThreads) reduce_kernel(const ReduceArgs
     __shared__ int s_base[2];
     const int tid = threadIdx.x, k = (int)A.k;
     const unsigned int n = *A.in_count;
-    const unsigned int lo = blockIdx.x * (unsigned int)kReduceSeg;
-    const unsigned int hi = min(lo + (unsigned int)kReduceSeg, n);
+    const unsigned int lo = blockIdx.x * A.seg;
+    const unsigned int hi = min(lo + A.seg, n);
     if (lo >= hi && !A.final) return;
     if (tid == 0) {
         s_count = 0;
         s_thr = 0ull;
     }
     __syncthreads();
-    unsigned long long thr = 0ull;
     for (unsigned int pos = lo; pos < hi; pos += kReduceThreads) {
-        __syncthreads();
-        if (s_count > kTopkCap - kReduceThreads) tk_prune(s_buf, &s_count, &s_thr, k);
-        thr = s_thr;
-        __syncthreads();
         const unsigned int i = pos + tid;
         const unsigned long long key = i < hi ? A.in[i] : 0ull;
+        unsigned long long thr = s_thr;
+        const int takers = __syncthreads_count(key > thr);
+        if (s_count + takers > kTopkCap) {
+            tk_prune<kTopkCap / 2 / kReduceThreads>(s_buf, &s_count, &s_thr, k);
+            thr = s_thr;
+        }
         tk_push(s_buf, &s_count, thr, key != 0ull, key);
+        __syncthreads();
     }
-    tk_prune(s_buf, &s_count, &s_thr, k);
+    tk_prune<kTopkCap / 2 / kReduceThreads>(s_buf, &s_count, &s_thr, k);
     const int c = s_count;
     if (!A.final) {
         tk_flush(s_buf, c, 0ull, s_base, A.out, A.out_count);
@@ -475,24 +479,23 @@ int launch_topk_reduce(void *d_workspace, const TopkLayout &lay, uint64_t n_keys
     unsigned long long *out = (unsigned long long *)(ws + lay.off_keys_b);
     int in_slot = 1, out_slot = 2;
     *n_kernels = 0;
-    for (int pass = 0; pass < 6; pass++) {
-        const uint64_t blocks = (n_keys_max + kReduceSeg - 1) / kReduceSeg;
+    // pass 1 spreads a long list over blocks of kReduceSeg keys; whatever it leaves (at most k keys per
+    // block) is finished by one block
+    for (int pass = 0; pass < 2; pass++) {
+        const uint64_t blocks = pass == 0 ? (n_keys_max + kReduceSeg - 1) / kReduceSeg : 1;
         ReduceArgs r;
         r.in = in; r.in_count = ctrl + in_slot; r.out = out; r.out_count = ctrl + out_slot;
         r.k = k; r.final = blocks <= 1; r.first = first; r.idx_map = d_idx_map;
+        r.seg = blocks <= 1 ? 0xFFFFFFFFu : (unsigned int)kReduceSeg;
         r.topk_idx = d_topk_idx; r.topk_score = d_topk_score; r.topk_count = d_topk_count;
         reduce_kernel<<<(unsigned int)(blocks < 1 ? 1 : blocks), kReduceThreads, 0, st>>>(r);
         count_launch();
         (*n_kernels)++;
         PF_CUDA_TRY(cudaGetLastError(), "reduce_kernel launch");
         if (r.final) return PF_OK;
-        n_keys_max = blocks * k;
         unsigned long long *t = in; in = out; out = t;
-        // counters rotate through ctrl[1..3]; the one about to be reused was consumed two passes ago
-        const int next = in_slot == 1 ? 3 : in_slot - 1;
-        in_slot = out_slot;
-        out_slot = next;
-        if (pass >= 1) PF_CUDA_TRY(cudaMemsetAsync(ctrl + out_slot, 0, 4, st), "reduce counter reset");
+        in_slot = 2;
+        out_slot = 3;
     }
     return PF_EINVAL;
 }

@@ -585,7 +585,7 @@ __global__ void __launch_bounds__(kThreads) dense_topk_kernel(const DenseTopkArg
     for (uint64_t base = (uint64_t)blockIdx.x * kThreads; base < n; base += (uint64_t)gridDim.x * kThreads) {
         if (room == 0) {
             __syncthreads();
-            if (s_count > kTopkCap - kThreads) tk_prune(s_buf, &s_count, &s_thr, (int)A.k);
+            if (s_count > kTopkCap - kThreads) tk_prune<kTopkCap / 2 / kThreads>(s_buf, &s_count, &s_thr, (int)A.k);
             room = (kTopkCap - s_count) / kThreads;
             thr = s_thr;
             __syncthreads();
@@ -595,7 +595,7 @@ __global__ void __launch_bounds__(kThreads) dense_topk_kernel(const DenseTopkArg
         tk_push(s_buf, &s_count, thr, s > 0.f, make_key(s, (uint32_t)i));
         room--;
     }
-    tk_prune(s_buf, &s_count, &s_thr, (int)A.k);
+    tk_prune<kTopkCap / 2 / kThreads>(s_buf, &s_count, &s_thr, (int)A.k);
     tk_flush(s_buf, s_count, 0ull, s_base, A.keys, A.key_count);
 }
 
