@@ -27,6 +27,8 @@ struct SelArgs {
     const uint8_t *reason;
     const float *tput;
     unsigned int *hist1, *hist2;      // kBins each
+    unsigned int *coarse1, *coarse2;  // 256 bins each: sums over groups of 256 fine bins
+    unsigned int *blk_elig;           // eligible candidates per block, written by the first pass
     SelCtrl *ctrl;
     unsigned long long *blk_gt, *blk_eq;  // per block counts, then exclusive prefixes
     uint64_t *surv_idx, *surv_count;
@@ -118,21 +120,36 @@ __device__ __forceinline__ void load_chunk(const SelArgs &A, uint64_t lo, uint64
 __global__ void __launch_bounds__(kSelThreads) sel_hist_kernel(const __grid_constant__ DevPlan P, const SelArgs A,
                                                                 const int32_t *vals, int pass)
 {
+    __shared__ unsigned int s_elig;
     const uint64_t lo = (uint64_t)blockIdx.x * A.chunk;
     const uint64_t hi = min(lo + A.chunk, A.count);
-    if (pass == 1 && A.ctrl->take_all) return;
+    if (pass == 1 && (A.ctrl->take_all || A.blk_elig[blockIdx.x] == 0)) return;   // nothing to refine here
+    if (pass == 0) {
+        if (threadIdx.x == 0) s_elig = 0;
+        __syncthreads();
+    }
     const uint32_t b1 = pass == 1 ? A.ctrl->b1 : 0;
+    unsigned int mine = 0;
     uint4 r[kSelTiles];
     load_chunk(A, lo, hi, r);
 #pragma unroll
     for (int t = 0; t < kSelTiles; t++) {
         const uint64_t e = lo + (uint64_t)t * kSelTile + (uint64_t)threadIdx.x * 16;
         for_each_eligible16(P, vals, A, e, r[t], [&](uint64_t, uint32_t bits) {
-            if (pass == 0)
+            if (pass == 0) {
                 atomicAdd(A.hist1 + (bits >> 16), 1u);
-            else if ((bits >> 16) == b1)
+                atomicAdd(A.coarse1 + (bits >> 24), 1u);
+                mine++;
+            } else if ((bits >> 16) == b1) {
                 atomicAdd(A.hist2 + (bits & 0xFFFFu), 1u);
+                atomicAdd(A.coarse2 + ((bits >> 8) & 0xFFu), 1u);
+            }
         });
+    }
+    if (pass == 0) {
+        if (mine) atomicAdd(&s_elig, mine);
+        __syncthreads();
+        if (threadIdx.x == 0) A.blk_elig[blockIdx.x] = s_elig;
     }
 }
 
@@ -162,23 +179,38 @@ __device__ __forceinline__ unsigned long long block_prefix_1024(unsigned long lo
     return x;
 }
 
-// One block of 1024 threads: find the bin (scanning from the top) where the running count reaches the target.
-__global__ void __launch_bounds__(1024) sel_scan_kernel(const SelArgs A, int pass)
+// One block of 256 threads: find the bin (scanning from the top) where the running count reaches the target.
+// The coarse histogram (one entry per 256 fine bins) locates the group, the group's 256 fine bins the bin.
+__device__ __forceinline__ unsigned long long block_prefix_256(unsigned long long x, unsigned long long *s_warp)
 {
-    __shared__ unsigned long long s_warp[32];
-    __shared__ unsigned long long s_total;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        unsigned long long y = __shfl_up_sync(0xFFFFFFFFu, x, off);
+        if (lane >= off) x += y;
+    }
+    if (lane == 31) s_warp[warp] = x;
+    __syncthreads();
+    unsigned long long add = 0;
+    for (int w = 0; w < warp; w++) add += s_warp[w];
+    __syncthreads();
+    return x + add;
+}
+
+__global__ void __launch_bounds__(256) sel_scan_kernel(const SelArgs A, int pass)
+{
+    __shared__ unsigned long long s_warp[8];
+    __shared__ unsigned long long s_total, s_above;
+    __shared__ int s_group;
     const int tid = threadIdx.x;
     SelCtrl *c = A.ctrl;
     if (pass == 1 && c->take_all) return;
-    const unsigned int *hist = pass == 0 ? A.hist1 : A.hist2;
-    constexpr int per = kBins / 1024;
-    // thread t owns bins [(1023-t)*per, (1024-t)*per): thread 0 holds the TOP bins, so an inclusive prefix
-    // over threads counts from the top
-    const int my_lo = (1023 - tid) * per;
-    unsigned long long mine = 0;
-    for (int i = 0; i < per; i++) mine += hist[my_lo + i];
-    const unsigned long long incl = block_prefix_1024(mine, s_warp);
-    if (tid == 1023) s_total = incl;
+    const unsigned int *fine = pass == 0 ? A.hist1 : A.hist2;
+    const unsigned int *coarse = pass == 0 ? A.coarse1 : A.coarse2;
+    // thread t owns coarse group 255 - t: an inclusive prefix over threads counts from the top
+    const unsigned long long mine = coarse[255 - tid];
+    const unsigned long long incl = block_prefix_256(mine, s_warp);
+    if (tid == 255) s_total = incl;
     __syncthreads();
     const unsigned long long total = s_total;
     unsigned long long target;
@@ -198,25 +230,25 @@ __global__ void __launch_bounds__(1024) sel_scan_kernel(const SelArgs A, int pas
     } else {
         target = c->target - c->above1;
     }
-    // the owner of the crossing: count above my bins < target <= count including them
-    const unsigned long long above = incl - mine;
-    if (above < target && incl >= target) {
-        unsigned long long run = above;
-        for (int i = per - 1; i >= 0; i--) {
-            unsigned int h = hist[my_lo + i];
-            if (run + h >= target) {
-                uint32_t bin = (uint32_t)(my_lo + i);
-                if (pass == 0) {
-                    c->b1 = bin;
-                    c->above1 = run;
-                } else {
-                    c->thr_bits = (c->b1 << 16) | bin;
-                    c->n_gt = c->above1 + run;
-                    c->need_eq = c->target - (c->above1 + run);
-                }
-                break;
-            }
-            run += h;
+    if (incl - mine < target && incl >= target) {
+        s_group = 255 - tid;
+        s_above = incl - mine;
+    }
+    __syncthreads();
+    // same search inside the group's 256 fine bins
+    const int g = s_group;
+    const unsigned long long fm = fine[g * 256 + (255 - tid)];
+    const unsigned long long fincl = s_above + block_prefix_256(fm, s_warp);
+    if (fincl - fm < target && fincl >= target) {
+        const uint32_t bin = (uint32_t)(g * 256 + (255 - tid));
+        const unsigned long long run = fincl - fm;   // eligible strictly above this bin
+        if (pass == 0) {
+            c->b1 = bin;
+            c->above1 = run;
+        } else {
+            c->thr_bits = (c->b1 << 16) | bin;
+            c->n_gt = c->above1 + run;
+            c->need_eq = c->target - (c->above1 + run);
         }
     }
 }
@@ -225,6 +257,13 @@ __global__ void __launch_bounds__(kSelThreads) sel_count_kernel(const __grid_con
                                                                  const int32_t *vals)
 {
     __shared__ unsigned int s_gt, s_eq;
+    if (A.blk_elig[blockIdx.x] == 0) {   // nothing eligible in this chunk: its counts are zero
+        if (threadIdx.x == 0) {
+            A.blk_gt[blockIdx.x] = 0;
+            A.blk_eq[blockIdx.x] = 0;
+        }
+        return;
+    }
     if (threadIdx.x == 0) s_gt = s_eq = 0;
     __syncthreads();
     const uint64_t lo = (uint64_t)blockIdx.x * A.chunk;
@@ -288,6 +327,7 @@ __global__ void __launch_bounds__(kSelThreads) sel_write_kernel(const __grid_con
     __shared__ unsigned int s_gt[kSelThreads], s_eq[kSelThreads];
     __shared__ unsigned long long s_run_gt, s_run_eq;
     const int tid = threadIdx.x;
+    if (A.blk_elig[blockIdx.x] == 0) return;   // nothing to write from this chunk
     const uint64_t lo = (uint64_t)blockIdx.x * A.chunk;
     const uint64_t hi = min(lo + A.chunk, A.count);
     const uint32_t thr = A.ctrl->thr_bits;
@@ -343,7 +383,7 @@ __global__ void __launch_bounds__(kSelThreads) sel_write_kernel(const __grid_con
 }
 
 struct SelLayout {
-    size_t off_ctrl, off_hist1, off_hist2, off_gt, off_eq, total;
+    size_t off_ctrl, off_hist1, off_hist2, off_coarse, off_gt, off_eq, off_elig, total;
     int nblocks;
     uint64_t chunk;
 };
@@ -360,10 +400,12 @@ static SelLayout sel_layout(const pf_plan_t *p, uint64_t count)
     l.off_ctrl = 0;
     l.off_hist1 = 256;
     l.off_hist2 = l.off_hist1 + kBins * 4;
-    l.off_gt = l.off_hist2 + kBins * 4;
+    l.off_coarse = l.off_hist2 + kBins * 4;          // coarse1[256], coarse2[256]
+    l.off_gt = l.off_coarse + 2 * 256 * 4;
     size_t per = (((size_t)l.nblocks + 1) * 8 + 255) & ~(size_t)255;
     l.off_eq = l.off_gt + per;
-    l.total = l.off_eq + per;
+    l.off_elig = l.off_eq + per;
+    l.total = l.off_elig + per;
     return l;
 }
 
@@ -395,15 +437,18 @@ extern "C" int pf_select_survivors(pf_plan_t *p, uint64_t first, uint64_t count,
     a.ctrl = (SelCtrl *)(ws + lay.off_ctrl);
     a.hist1 = (unsigned int *)(ws + lay.off_hist1);
     a.hist2 = (unsigned int *)(ws + lay.off_hist2);
+    a.coarse1 = (unsigned int *)(ws + lay.off_coarse);
+    a.coarse2 = a.coarse1 + 256;
+    a.blk_elig = (unsigned int *)(ws + lay.off_elig);
     a.blk_gt = (unsigned long long *)(ws + lay.off_gt);
     a.blk_eq = (unsigned long long *)(ws + lay.off_eq);
     a.surv_idx = d_surv_idx; a.surv_count = d_surv_count; a.chunk = lay.chunk;
     PF_CUDA_TRY(cudaMemsetAsync(ws, 0, lay.off_gt, st), "pf_select_survivors: clear");
     timing_begin(p, PF_T_SELECT, st);
     sel_hist_kernel<<<lay.nblocks, kSelThreads, 0, st>>>(p->dev, a, p->d_vals, 0);
-    sel_scan_kernel<<<1, 1024, 0, st>>>(a, 0);
+    sel_scan_kernel<<<1, 256, 0, st>>>(a, 0);
     sel_hist_kernel<<<lay.nblocks, kSelThreads, 0, st>>>(p->dev, a, p->d_vals, 1);
-    sel_scan_kernel<<<1, 1024, 0, st>>>(a, 1);
+    sel_scan_kernel<<<1, 256, 0, st>>>(a, 1);
     sel_count_kernel<<<lay.nblocks, kSelThreads, 0, st>>>(p->dev, a, p->d_vals);
     sel_blockscan_kernel<<<1, 1024, 0, st>>>(a, lay.nblocks);
     sel_write_kernel<<<lay.nblocks, kSelThreads, 0, st>>>(p->dev, a, p->d_vals);
