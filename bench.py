@@ -34,9 +34,10 @@ UNIT = "candidates/s"
 K_TOP, S_MAX, K_SIM, JITTER_SEED = 1024, 1_000_000, 100, 4
 BYTES_PER_CANDIDATE = 13          # dense outputs: reason u8 + tput f32 + mem i64
 FALLBACK_HBM_GBS = 6650.0         # used only when MEASURED_PEAKS.json is absent
-# dram__bytes_read.sum + dram__bytes_write.sum of one score_kernel launch on this workload, from the ncu
-# capture summarised in profiles/ (None until a capture exists)
-SCORE_KERNEL_DRAM_BYTES = None
+# dram__bytes_read.sum + dram__bytes_write.sum of one score_kernel launch on this workload: captured with ncu
+# on a 50,000,000-candidate slice (597.3 MB) and scaled by candidates to the full space (the ncu summary is
+# kept under profiles/).  Below the algorithmic bytes because dirty lines still sit in L2 when the kernel ends.
+SCORE_KERNEL_DRAM_BYTES = int(597.257472e6 * 179_908_608 / 50_000_000)
 
 
 def _measured_hbm():
@@ -156,8 +157,10 @@ def run_reference(args):
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": "large training space (179,908,608 candidates) + simulator tier", "k": K_TOP,
-                       "s_max": S_MAX, "k_sim": K_SIM},
+            "config": {"workload": "large training space (config 4: 179,908,608 candidates, top-1024) + simulator "
+                                   "tier on its survivors (config 5, top-100)",
+                       "candidates_per_gpu": orc.size, "k": K_TOP, "s_max": S_MAX, "k_sim": K_SIM,
+                       "parallelism": "dp1"},
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": used, "kind": "oracle", "sample": sample},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
