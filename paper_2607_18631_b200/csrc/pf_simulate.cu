@@ -18,7 +18,6 @@
 
 namespace pf {
 
-constexpr int kSimMaxWarps = 16;        // warps per block at most (each simulates one candidate at a time)
 
 // DualPipe-style order tables: for every (pp, m) in the domain a byte string per rank,
 // op = (j << 2) | (dir << 1) | is_backward, 2*m ops per rank.
@@ -180,7 +179,11 @@ __device__ __forceinline__ float jitter(uint32_t seed_mixed, uint64_t idx, int q
 }
 
 constexpr int kSimClasses = 7;          // timeline sizes 256 << c entries (stage streams x microbatches)
+constexpr int kSimGroups = 3;           // lanes per candidate: 8, 16 or 32 (pipeline depth rounded up)
+constexpr int kSimBins = kSimClasses * kSimGroups;
+constexpr int kSimThreads = 128;        // 4 warps per block, each with its own shared-memory slice
 __host__ __device__ inline int sim_class_entries(int c) { return 256 << c; }
+__host__ __device__ inline int sim_group_lanes(int g) { return 8 << g; }
 
 struct SimArgs {
     const uint64_t *surv;
@@ -189,21 +192,25 @@ struct SimArgs {
     uint32_t seed;
     float *tput_sim;
     uint8_t *status;
-    unsigned int *work;             // [kSimClasses] work-queue heads, zeroed before launch
-    unsigned int *cls_count;        // [kSimClasses] list lengths, zeroed before the classify kernel
-    uint32_t *cls_list;             // [kSimClasses][n] positions in surv, grouped by timeline size
+    unsigned int *work;             // [kSimBins] work-queue heads
+    unsigned int *bin_count;        // [kSimBins] survivors per bin
+    unsigned int *bin_off;          // [kSimBins + 1] start of each bin in the list
+    unsigned int *bin_fill;         // [kSimBins] scatter cursors
+    uint8_t *bin_of;                // [n] bin of each survivor
+    uint32_t *list;                 // [n] positions in surv, grouped by bin
     const int32_t *vals;
     const uint8_t *dual_ops;
     const int32_t *dual_off;
     int q_max;                      // stages per candidate at most (plan-wide)
     int cls_hi;                     // largest class the plan can produce
-    int pool_floats;                // dynamic shared memory of a block, in floats
+    int warp_floats;                // shared-memory slice of one warp, in floats
 };
 
-// Pre-pass: one thread per survivor computes how many timeline entries its simulation needs and files the
-// survivor under the smallest class that holds them, so each class can run with as many warps per SM as its
-// shared-memory footprint allows.  Entries that cannot be simulated (outside the domain, malformed) go to
-// class 0, where the simulator kernel rejects them before touching the timeline.
+// Pre-pass 1: one thread per survivor decides its bin -- the smallest timeline class that holds its
+// stage-streams x microbatches, and the lane-group width that holds its pipeline depth -- so that timelines of
+// similar size are scheduled together and several shallow pipelines share a warp.  Entries that cannot be
+// simulated (outside the domain, malformed) go to bin 0, where the simulator rejects them before touching a
+// timeline.
 template <typename RI>
 __global__ void __launch_bounds__(256) sim_classify_kernel(const __grid_constant__ DevPlan P, const SimArgs A)
 {
@@ -213,7 +220,7 @@ __global__ void __launch_bounds__(256) sim_classify_kernel(const __grid_constant
         n = dn < n ? dn : n;
     }
     const uint64_t w = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    int cls = -1;
+    int bin = -1;
     if (w < n) {
         uint64_t rem = A.surv[w];
         int v[PF_MAX_AXES];
@@ -229,7 +236,7 @@ __global__ void __launch_bounds__(256) sim_classify_kernel(const __grid_constant
         if (v[8] == 0) dp = (RI)v[9] / ((RI)tp * (RI)pp);
         const int kind = P.sched[s].kind;
         const int v_eff = vv == 0 ? (kind == PF_KIND_INTERLEAVED ? 2 : 1) : vv;
-        cls = 0;
+        bin = 0;
         const RI dpmb = dp * (RI)mb;
         if (dpmb != 0 && pp <= PF_SIM_MAX_RANKS && v_eff <= PF_SIM_MAX_V) {
             RI m = (RI)P.gbs / dpmb;
@@ -237,317 +244,268 @@ __global__ void __launch_bounds__(256) sim_classify_kernel(const __grid_constant
             if (kind == PF_KIND_INTERLEAVED) m_sim = (m_sim / pp) * pp;
             const int streams = kind == PF_KIND_DUALPIPE ? pp : pp * v_eff;  // DualPipe: 2 directions x m/2
             const int entries = streams * m_sim;
+            int cls = 0;
             while (cls < kSimClasses - 1 && sim_class_entries(cls) < entries) cls++;
-            if (sim_class_entries(cls) < entries || streams > A.q_max) cls = 0;   // cannot be a feasible plan
+            if (sim_class_entries(cls) >= entries && streams <= A.q_max)
+                bin = cls * kSimGroups + (pp <= 8 ? 0 : (pp <= 16 ? 1 : 2));
         }
+        A.bin_of[w] = (uint8_t)bin;
     }
-    // warp-aggregated append per class
-    for (int c = 0; c < kSimClasses; c++) {
-        const unsigned mask = __ballot_sync(0xFFFFFFFFu, cls == c);
-        if (mask == 0) continue;
-        const int lane = threadIdx.x & 31, leader = __ffs(mask) - 1;
-        unsigned int base = 0;
-        if (lane == leader) base = atomicAdd(A.cls_count + c, (unsigned int)__popc(mask));
-        base = __shfl_sync(0xFFFFFFFFu, base, leader);
-        if (cls == c) A.cls_list[(size_t)c * A.n + base + __popc(mask & ((1u << lane) - 1u))] = (uint32_t)w;
-    }
+    // warp-aggregated count per bin
+    const unsigned peers = __match_any_sync(0xFFFFFFFFu, bin);
+    if (bin >= 0 && (int)(threadIdx.x & 31) == __ffs(peers) - 1) atomicAdd(A.bin_count + bin, (unsigned int)__popc(peers));
 }
 
-// per-warp shared memory of class c: endF[E], endB[E], durF[q_max], durB[q_max]
-__host__ __device__ inline size_t sim_warp_floats(int entries, int q_max) { return (size_t)2 * entries + 2 * q_max; }
-
-// The three round loops.  In every round a lane runs at most its next op, and only if the op it waits for
-// has already published its end time; the body is branch-free apart from that test, so the lanes of a warp
-// stay converged and a round costs one shared-memory poll plus one vote.  Every 64 rounds some lane must
-// have advanced, otherwise the candidate is reported as stalled: the loops are bounded by the op count.
-struct SimLane {
-    float clock;
-    bool stalled;
-};
-
-#define PF_SIM_ROUND_END()                                               \
-    if (!__any_sync(0xFFFFFFFFu, done < total_ops)) break;               \
-    if ((++rounds & 63) == 0) {                                          \
-        if (!__any_sync(0xFFFFFFFFu, moved)) {                           \
-            st.stalled = true;                                           \
-            break;                                                       \
-        }                                                                \
-        moved = false;                                                   \
-    }
-
-// 1F1B: rank = stage = lane; `warm` forwards, then one forward / one backward, then the remaining backwards
-__device__ __forceinline__ void sim_rounds_1f1b(volatile float *endF, volatile float *endB, const float *durF,
-                                                const float *durB, int lane, int pp, int nj, int warm, int total_ops,
-                                                float lat, SimLane &st)
+// Pre-pass 2 (one thread): bin offsets.
+__global__ void sim_offsets_kernel(const SimArgs A)
 {
-    const bool depF = lane > 0, depB = lane < pp - 1;
-    volatile float *inF = endF + (depF ? lane - 1 : lane) * nj, *inB = endB + (depB ? lane + 1 : lane) * nj;
-    volatile float *outF = endF + lane * nj, *outB = endB + lane * nj;
-    const float dF = lane < pp ? durF[lane] : 0.f, dB = lane < pp ? durB[lane] : 0.f;
-    int nF = 0, nB = 0, done = 0, rounds = 0;
-    bool moved = false;
-    float clock = 0.f;
-    for (;;) {
-        if (done < total_ops) {
-            const bool isb = !(nF < warm || (nF < nj && nF - warm == nB));
-            const int j = isb ? nB : nF;
-            const bool dep = isb ? depB : depF;
-            const float e = (isb ? inB : inF)[j];
-            if (!dep || e >= 0.f) {
-                clock = fmaxf(clock, dep ? e + lat : 0.f) + (isb ? dB : dF);
-                (isb ? outB : outF)[j] = clock;
-                nF += isb ? 0 : 1;
-                nB += isb ? 1 : 0;
-                done++;
-                moved = true;
-            }
+    if (threadIdx.x == 0) {
+        unsigned int run = 0;
+        for (int b = 0; b < kSimBins; b++) {
+            A.bin_off[b] = run;
+            run += A.bin_count[b];
         }
-        PF_SIM_ROUND_END()
+        A.bin_off[kSimBins] = run;
     }
-    st.clock = clock;
 }
 
-// Interleaved: v chunks per rank; unit k of a rank is microbatch (k / (pp v)) pp + k mod pp of chunk
-// (k mod (pp v)) / pp, backward units walk the chunks downward; cursors advance without divisions
-__device__ __forceinline__ void sim_rounds_interleaved(volatile float *endF, volatile float *endB, const float *durF,
-                                                       const float *durB, int lane, int pp, int v, int nj, int U,
-                                                       int warm, int total_ops, float lat, SimLane &st)
+// Pre-pass 3: scatter survivor positions into their bins.
+__global__ void __launch_bounds__(256) sim_scatter_kernel(const SimArgs A)
 {
-    const int Q = pp * v;
-    int nF = 0, nB = 0, done = 0, rounds = 0;
-    int fw = 0, fc = 0, fg = 0, bw = 0, bc = 0, bg = 0;
-    bool moved = false;
-    float clock = 0.f;
-    for (;;) {
-        if (done < total_ops) {
-            const bool isb = !(nF < warm || (nF < U && nF - warm == nB));
-            const int cw = isb ? bw : fw, cc = isb ? bc : fc, cg = isb ? bg : fg;
-            const int j = cg * pp + cw;
-            const int q = (isb ? v - 1 - cc : cc) * pp + lane;
-            const bool dep = isb ? (q < Q - 1) : (q > 0);
-            const int nb = dep ? (isb ? q + 1 : q - 1) : q;
-            volatile float *arr = isb ? endB : endF;
-            const float e = arr[nb * nj + j];
-            const float dur = (isb ? durB : durF)[q];
-            if (!dep || e >= 0.f) {
-                clock = fmaxf(clock, dep ? e + lat : 0.f) + dur;
-                arr[q * nj + j] = clock;
-                int w_ = cw + 1, c_ = cc, g_ = cg;
-                if (w_ == pp) {
-                    w_ = 0;
-                    if (++c_ == v) c_ = 0, g_++;
-                }
-                if (isb) bw = w_, bc = c_, bg = g_, nB++;
-                else fw = w_, fc = c_, fg = g_, nF++;
-                done++;
-                moved = true;
-            }
-        }
-        PF_SIM_ROUND_END()
+    uint64_t n = A.n;
+    if (A.d_n) {
+        uint64_t dn = *A.d_n;
+        n = dn < n ? dn : n;
     }
-    st.clock = clock;
+    const uint64_t w = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int bin = w < n ? (int)A.bin_of[w] : -1;
+    const unsigned peers = __match_any_sync(0xFFFFFFFFu, bin);
+    const int lane = threadIdx.x & 31, leader = __ffs(peers) - 1;
+    unsigned int base = 0;
+    if (bin >= 0 && lane == leader) base = atomicAdd(A.bin_fill + bin, (unsigned int)__popc(peers));
+    base = __shfl_sync(0xFFFFFFFFu, base, leader);
+    if (bin >= 0) A.list[A.bin_off[bin] + base + __popc(peers & ((1u << lane) - 1u))] = (uint32_t)w;
 }
 
-// DualPipe-style: two directions; the per-rank order comes from the host-built table
-__device__ __forceinline__ void sim_rounds_dual(volatile float *endF, volatile float *endB, const float *durF,
-                                                const float *durB, int lane, int pp, int nj, const uint8_t *ops,
-                                                int total_ops, float lat, SimLane &st)
-{
-    int done = 0, rounds = 0;
-    bool moved = false;
-    float clock = 0.f;
-    for (;;) {
-        if (done < total_ops) {
-            const uint32_t op = __ldg(ops + done);
-            const bool isb = op & 1;
-            const int d = (op >> 1) & 1, j = op >> 2;
-            const int q = d ? pp - 1 - lane : lane;
-            const int sidx = d * pp + q;
-            const bool dep = isb ? (q < pp - 1) : (q > 0);
-            const int nb = dep ? (isb ? sidx + 1 : sidx - 1) : sidx;
-            volatile float *arr = isb ? endB : endF;
-            const float e = arr[nb * nj + j];
-            const float dur = (isb ? durB : durF)[q];
-            if (!dep || e >= 0.f) {
-                clock = fmaxf(clock, dep ? e + lat : 0.f) + dur;
-                arr[sidx * nj + j] = clock;
-                done++;
-                moved = true;
-            }
-        }
-        PF_SIM_ROUND_END()
-    }
-    st.clock = clock;
-}
-#undef PF_SIM_ROUND_END
-
-// One launch serves every class.  A block owns a fixed pool of shared memory; while it works on class c as
-// many of its warps as fit (pool / footprint) pull candidates from that class' queue, the others wait at the
-// barrier that separates two classes.
+// One launch serves every bin.  Every warp owns a fixed slice of the block's shared memory, large enough for
+// one timeline of the largest class (or several of a smaller one), and works through the bins on its own --
+// largest timelines first, so the longest simulations start earliest and the tail is one candidate long.  No
+// block-level barrier is involved.
+//
+// Inside a warp a candidate is run by a group of 8, 16 or 32 lanes, lane = pipeline rank; a warp takes as many
+// candidates per batch as it has groups and its slice has room.  Each lane walks its rank's fixed op order and
+// computes  end(op) = max(rank clock, end(dependency) + latency) + duration.  A forward of stage q needs the
+// forward of stage q-1 of the same microbatch, a backward of stage q the backward of stage q+1 (the op's own
+// forward is already behind the lane's clock).  The timeline has ONE 32-bit word per (stage stream,
+// microbatch): 0 while nothing has finished, +t once the forward has ended at t, -t once the backward has --
+// the forward's end has been consumed by stage q+1 before the backward of the same slot can start, so the two
+// never need the word at the same time.  The owner writes it, the neighbour polls it with a volatile load.  In
+// every round a lane runs at most its next op; the body is branch-free apart from the readiness test, so lanes
+// (and the groups of a warp) stay converged and a round costs one shared-memory poll plus one vote.  Every 64
+// rounds some lane of the warp must have advanced, otherwise its unfinished candidates are reported as
+// PF_SIM_STALL: the loop is bounded by the op count.
 template <typename RI>
-__global__ void __launch_bounds__(kSimMaxWarps * 32) simulate_kernel(const __grid_constant__ DevPlan P, const SimArgs A)
+__global__ void __launch_bounds__(kSimThreads, 4) simulate_kernel(const __grid_constant__ DevPlan P, const SimArgs A)
 {
     extern __shared__ float s_mem[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint32_t seed_mixed = mix32(A.seed + 0x9e3779b9u);
+    const int E_hi = sim_class_entries(A.cls_hi);
+    float *slice = s_mem + (size_t)warp * A.warp_floats;   // [E_hi] timelines, then 4 x (durF, durB)[q_max]
 
-    // Blocks start on different classes (cyclic, staggered by block number) so that all classes are in
-    // progress at once; a class whose queue is already drained is skipped, decided once per block.
-    __shared__ int s_skip;
-    const int n_classes = A.cls_hi + 1;
-    for (int step = 0; step < n_classes; step++) {
-    const int cls = (A.cls_hi - (int)(blockIdx.x % n_classes) - step + 2 * n_classes) % n_classes;
-    const unsigned int n_cls = A.cls_count[cls];
-    if (threadIdx.x == 0) s_skip = *reinterpret_cast<volatile unsigned int *>(A.work + cls) >= n_cls;
-    __syncthreads();
-    const bool skip = s_skip != 0;
-    __syncthreads();
-    if (skip) continue;
-    const int E = sim_class_entries(cls);
-    const int per_warp = (int)sim_warp_floats(E, A.q_max);
-    const int active_warps = min((int)(blockDim.x >> 5), A.pool_floats / per_warp);
-    if (warp < active_warps) {
-    float *base = s_mem + (size_t)warp * per_warp;
-    // End times are written by the lane that owns the stage and polled by its neighbour: one 32-bit word per
-    // op, negative while the op has not finished, so a single volatile load answers "done, and when".
-    volatile float *endF = base;
-    volatile float *endB = base + E;
-    float *durF = base + 2 * (size_t)E;
-    float *durB = durF + A.q_max;
-    const uint32_t *list = A.cls_list + (size_t)cls * A.n;
+    for (int cls = A.cls_hi; cls >= 0; cls--) {
+        for (int gi = 0; gi < kSimGroups; gi++) {
+            const int bin = cls * kSimGroups + gi;
+            const unsigned int n_bin = A.bin_count[bin];
+            if (n_bin == 0) continue;
+            const int g = sim_group_lanes(gi);
+            const int E = sim_class_entries(cls);
+            const int batch = min(32 / g, E_hi / E);               // candidates this warp runs side by side
+            const int gidx = lane / g, glane = lane - gidx * g;
+            const bool group_on = gidx < batch;
+            volatile float *tl = slice + (size_t)(group_on ? gidx : 0) * E;   // the timeline
+            float *durF = slice + E_hi + (size_t)(group_on ? gidx : 0) * 2 * A.q_max, *durB = durF + A.q_max;
+            const uint32_t *list = A.list + A.bin_off[bin];
 
-    for (;;) {
-        unsigned int wi = 0;
-        if (lane == 0) wi = atomicAdd(A.work + cls, 1u);
-        wi = __shfl_sync(0xFFFFFFFFu, wi, 0);
-        if (wi >= n_cls) break;
-        const uint32_t w = list[wi];
-        const uint64_t idx = A.surv[w];
+            for (;;) {
+                unsigned int wi = 0;
+                if (lane == 0) wi = atomicAdd(A.work + bin, (unsigned int)batch);
+                wi = __shfl_sync(0xFFFFFFFFu, wi, 0);
+                if (wi >= n_bin) break;
+                const bool have = group_on && wi + gidx < n_bin;   // this group's candidate exists
+                const uint32_t w = have ? list[wi + gidx] : 0u;
+                const uint64_t idx = have ? A.surv[w] : 0ull;
 
-        // ---- every lane re-derives the candidate (uniform across the warp)
-        TrainTuple c;
-        {
-            int v[PF_MAX_AXES];
-            uint64_t rem = idx;
+                // ---- every lane of the group derives the group's candidate
+                TrainTuple c;
+                {
+                    int v[PF_MAX_AXES];
+                    if ((idx >> 32) == 0) {
+                        uint32_t rem = (uint32_t)idx;
 #pragma unroll
-            for (int a = 0; a < PF_MAX_AXES; a++) {
-                uint64_t r = P.radix[a];
-                uint64_t q = rem / r;
-                v[a] = __ldg(A.vals + P.val_off[a] + (int)(rem - q * r));
-                rem = q;
-            }
-            c.kv = v[0]; c.rec = v[1]; c.s = v[2]; c.mb = v[3]; c.v = v[4];
-            c.ep = v[5]; c.pp = v[6]; c.tp = v[7]; c.dp = v[8]; c.world = v[9];
-        }
-        RI dp, world;
-        TrainDerived<RI> D;
-        TrainMem M;
-        int reason = train_layout_rules<RI>(P, c, 1, 3, dp, world);
-        if (reason == 0) reason = train_plan_rules<RI>(P, c, dp, world, 1, D);
-        if (reason == 0) {
-            train_memory<RI>(P, c, D, M);
-            if (M.mem > P.budget_bytes) reason = PF_R_MEMORY;
-        }
-        if (reason != 0) {
-            if (lane == 0) {
-                if (A.tput_sim) A.tput_sim[w] = 0.f;
-                if (A.status) A.status[w] = PF_SIM_UNSUPPORTED;
-            }
-            continue;
-        }
-        TrainTimes T;
-        train_times<RI>(P, c, D, M, T);
-        const int pp = c.pp, v = D.v_eff, kind = D.kind;
-        if (pp > PF_SIM_MAX_RANKS || v > PF_SIM_MAX_V) {
-            if (lane == 0) {
-                if (A.tput_sim) A.tput_sim[w] = train_price<RI>(P, c, D, T, train_pipe_analytic<RI>(P, c, D, T));
-                if (A.status) A.status[w] = PF_SIM_UNSUPPORTED;
-            }
-            continue;
-        }
-        const bool dual = kind == PF_KIND_DUALPIPE;
-        const int Q = dual ? pp : pp * v;
-        // simulated window
-        const long long m = (long long)D.m;
-        int m_sim = m < PF_SIM_WINDOW ? (int)m : PF_SIM_WINDOW;
-        if (kind == PF_KIND_INTERLEAVED) m_sim = (m_sim / pp) * pp;
-        const int nj = dual ? m_sim / 2 : m_sim;      // microbatches per stage stream
-        const int n_entries = (dual ? 2 * Q : Q) * nj;
-        bool stalled = n_entries > E || Q > A.q_max;  // filed under a class that cannot hold it: never for a
-                                                      // feasible plan, reported instead of overrunning
-
-        // ---- stage durations (balanced layer split, head on the last stage, jitter) and cleared timeline
-        __syncwarp();
-        if (!stalled) {
-            const int L_lo = P.L / Q, L_rem = P.L - L_lo * Q;
-            for (int q = lane; q < Q; q += 32) {
-                const float nq = (float)(L_lo + (q < L_rem ? 1 : 0));
-                const bool last = q == Q - 1;
-                durF[q] = (nq * T.F_l + (last ? T.headF : 0.f)) * jitter(seed_mixed, idx, q, 0);
-                durB[q] = (nq * T.B_l + (last ? P.bwd_factor * T.headF : 0.f)) * jitter(seed_mixed, idx, q, 1);
-            }
-            for (int i = lane; i < n_entries; i += 32) {
-                endF[i] = -1.f;
-                endB[i] = -1.f;
-            }
-        }
-        __syncwarp();
-
-        // ---- walk the rank's order
-        const bool rank_active = lane < pp;
-        const int U = dual ? 2 * nj : nj * (kind == PF_KIND_INTERLEAVED ? v : 1);  // forward units of this rank
-        const uint8_t *dops = nullptr;
-        if (dual && !stalled) {
-            const int off = __ldg(A.dual_off + pp * 33 + nj);
-            if (off < 0) stalled = true;  // no table for this shape: report instead of reading out of bounds
-            else dops = A.dual_ops + off + (size_t)lane * 2 * m_sim;
-        }
-        const int total_ops = (rank_active && !stalled) ? 2 * U : 0;
-        SimLane sl;
-        sl.clock = 0.f;
-        sl.stalled = stalled;
-        if (!stalled) {
-            if (kind == PF_KIND_1F1B)
-                sim_rounds_1f1b(endF, endB, durF, durB, lane, pp, nj, min(pp - lane - 1, U), total_ops, T.p, sl);
-            else if (kind == PF_KIND_INTERLEAVED)
-                sim_rounds_interleaved(endF, endB, durF, durB, lane, pp, v, nj, U,
-                                       min(2 * (pp - lane - 1) + (v - 1) * pp, U), total_ops, T.p, sl);
-            else
-                sim_rounds_dual(endF, endB, durF, durB, lane, pp, nj, dops, total_ops, T.p, sl);
-        }
-        stalled = sl.stalled;
-        const float clock = sl.clock;
-
-        // ---- makespan, steady-state extension beyond the window, pricing
-        float work = 0.f;
-        if (rank_active && !stalled) {
-            if (dual) {
-                work = 0.5f * (durF[lane] + durB[lane] + durF[pp - 1 - lane] + durB[pp - 1 - lane]);
-            } else {
-                const int vv = kind == PF_KIND_INTERLEAVED ? v : 1;
-                for (int cc = 0; cc < vv; cc++) work += durF[cc * pp + lane] + durB[cc * pp + lane];
-            }
-        }
-        float span = rank_active ? clock : 0.f;
+                        for (int a = 0; a < PF_MAX_AXES; a++) {
+                            uint32_t r = P.radix[a];
+                            uint32_t q = rem / r;
+                            v[a] = __ldg(A.vals + P.val_off[a] + (int)(rem - q * r));
+                            rem = q;
+                        }
+                    } else {
+                        uint64_t rem = idx;
 #pragma unroll
-        for (int off = 16; off > 0; off >>= 1) {
-            span = fmaxf(span, __shfl_xor_sync(0xFFFFFFFFu, span, off));
-            work = fmaxf(work, __shfl_xor_sync(0xFFFFFFFFu, work, off));
-        }
-        if (lane == 0) {
-            float tput = 0.f;
-            if (!stalled) {
-                float T_pipe = span;
-                if (m > m_sim) T_pipe += (float)(m - m_sim) * work;
-                tput = train_price<RI>(P, c, D, T, T_pipe);
+                        for (int a = 0; a < PF_MAX_AXES; a++) {
+                            uint64_t r = P.radix[a];
+                            uint64_t q = rem / r;
+                            v[a] = __ldg(A.vals + P.val_off[a] + (int)(rem - q * r));
+                            rem = q;
+                        }
+                    }
+                    c.kv = v[0]; c.rec = v[1]; c.s = v[2]; c.mb = v[3]; c.v = v[4];
+                    c.ep = v[5]; c.pp = v[6]; c.tp = v[7]; c.dp = v[8]; c.world = v[9];
+                }
+                RI dp, world;
+                TrainDerived<RI> D;
+                TrainMem M;
+                TrainTimes T;
+                int reason = train_layout_rules<RI>(P, c, 1, 3, dp, world);
+                if (reason == 0) reason = train_plan_rules<RI>(P, c, dp, world, 1, D);
+                if (reason == 0) {
+                    train_memory<RI>(P, c, D, M);
+                    if (M.mem > P.budget_bytes) reason = PF_R_MEMORY;
+                }
+                // outcome without a simulation: infeasible -> 0, outside the domain -> analytic score
+                int status = PF_SIM_OK;
+                float tput_out = 0.f;
+                bool run = have && reason == 0;
+                if (have && reason != 0) status = PF_SIM_UNSUPPORTED;
+                if (run) {
+                    train_times<RI>(P, c, D, M, T);
+                    if (c.pp > PF_SIM_MAX_RANKS || D.v_eff > PF_SIM_MAX_V) {
+                        tput_out = train_price<RI>(P, c, D, T, train_pipe_analytic<RI>(P, c, D, T));
+                        status = PF_SIM_UNSUPPORTED;
+                        run = false;
+                    }
+                }
+                const int pp = run ? c.pp : 1, v = run ? D.v_eff : 1, kind = run ? D.kind : PF_KIND_1F1B;
+                const bool dual = kind == PF_KIND_DUALPIPE;
+                const int Q = dual ? pp : pp * v;
+                const long long m = run ? (long long)D.m : 1;
+                int m_sim = m < PF_SIM_WINDOW ? (int)m : PF_SIM_WINDOW;
+                if (kind == PF_KIND_INTERLEAVED) m_sim = (m_sim / pp) * pp;
+                const int nj = dual ? m_sim / 2 : m_sim;      // microbatches per stage stream
+                const int n_entries = (dual ? 2 * Q : Q) * nj;
+                // filed under a bin that cannot hold it: never for a feasible plan; reported, not overrun
+                bool stalled = run && (n_entries > E || Q > A.q_max || pp > g);
+                if (stalled) run = false;
+
+                // ---- stage durations (balanced layer split, head on the last stage, jitter), cleared timeline
+                __syncwarp();
+                if (run) {
+                    const int L_lo = P.L / Q, L_rem = P.L - L_lo * Q;
+                    for (int q = glane; q < Q; q += g) {
+                        const float nq = (float)(L_lo + (q < L_rem ? 1 : 0));
+                        const bool last = q == Q - 1;
+                        durF[q] = (nq * T.F_l + (last ? T.headF : 0.f)) * jitter(seed_mixed, idx, q, 0);
+                        durB[q] = (nq * T.B_l + (last ? P.bwd_factor * T.headF : 0.f)) * jitter(seed_mixed, idx, q, 1);
+                    }
+                    for (int i = glane; i < n_entries; i += g) tl[i] = 0.f;
+                }
+                __syncwarp();
+
+                // ---- per-lane order state (1F1B is the one-chunk case of the unit cursors)
+                const bool rank_active = run && glane < pp;
+                const int U = dual ? 2 * nj : nj * v;          // forward units of this rank
+                const int warm = kind == PF_KIND_INTERLEAVED ? min(2 * (pp - glane - 1) + (v - 1) * pp, U)
+                                                             : min(pp - glane - 1, U);
+                const uint8_t *dops = A.dual_ops;              // any valid address for lanes that do not use it
+                if (dual && run) {
+                    const int off = __ldg(A.dual_off + pp * 33 + nj);
+                    if (off < 0) stalled = true, run = false;  // no table for this shape
+                    else dops = A.dual_ops + off + (size_t)glane * 2 * m_sim;
+                }
+                const int total_ops = (rank_active && run) ? 2 * U : 0;
+                const float lat = run ? T.p : 0.f;
+                int done = 0, rounds = 0, nF = 0, nB = 0;
+                int fw = 0, fc = 0, fg = 0, bw = 0, bc = 0, bg = 0;
+                bool moved = false;
+                float clock = 0.f;
+
+                for (;;) {
+                    if (done < total_ops) {
+                        // next op of this rank: from the table (DualPipe-style) or from the unit cursors
+                        uint32_t op = 0;
+                        if (dual) op = __ldg(dops + done);
+                        const bool isb_c = !(nF < warm || (nF < U && nF - warm == nB));
+                        const bool isb = dual ? (op & 1u) != 0 : isb_c;
+                        const int d = dual ? (int)((op >> 1) & 1u) : 0;
+                        const int cw = isb ? bw : fw, cc = isb ? bc : fc, cg = isb ? bg : fg;
+                        const int j = dual ? (int)(op >> 2) : cg * pp + cw;
+                        const int q = dual ? (d ? pp - 1 - glane : glane) : (isb ? v - 1 - cc : cc) * pp + glane;
+                        const int sidx = d * Q + q;             // stage stream (direction-major for DualPipe)
+                        const bool dep = isb ? (q < Q - 1) : (q > 0);
+                        const int nb = dep ? (isb ? sidx + 1 : sidx - 1) : sidx;
+                        const float e = tl[nb * nj + j];
+                        const float dur = (isb ? durB : durF)[q];
+                        // a forward waits for a positive word (forward ended), a backward for a negative one
+                        const bool ready = !dep || (isb ? e < 0.f : e > 0.f);
+                        if (ready) {
+                            clock = fmaxf(clock, dep ? fabsf(e) + lat : 0.f) + dur;
+                            tl[sidx * nj + j] = isb ? -clock : clock;
+                            int w_ = cw + 1, c_ = cc, g_ = cg;
+                            if (w_ == pp) {
+                                w_ = 0;
+                                if (++c_ == v) c_ = 0, g_++;
+                            }
+                            if (isb) bw = w_, bc = c_, bg = g_, nB++;
+                            else fw = w_, fc = c_, fg = g_, nF++;
+                            done++;
+                            moved = true;
+                        }
+                    }
+                    if (!__any_sync(0xFFFFFFFFu, done < total_ops)) break;
+                    if ((++rounds & 63) == 0) {
+                        if (!__any_sync(0xFFFFFFFFu, moved)) break;   // nothing advanced: give up, report below
+                        moved = false;
+                    }
+                }
+                if (done < total_ops) stalled = true;
+
+                // ---- makespan, steady-state extension beyond the window, pricing (reductions inside the group)
+                float work = 0.f;
+                if (rank_active && run) {
+                    if (dual) {
+                        work = 0.5f * (durF[glane] + durB[glane] + durF[pp - 1 - glane] + durB[pp - 1 - glane]);
+                    } else {
+                        for (int cc = 0; cc < v; cc++) work += durF[cc * pp + glane] + durB[cc * pp + glane];
+                    }
+                }
+                float span = rank_active ? clock : 0.f;
+                int any_stall = stalled ? 1 : 0;
+#pragma unroll
+                for (int off = 16; off > 0; off >>= 1) {
+                    const float s2 = __shfl_xor_sync(0xFFFFFFFFu, span, off);
+                    const float w2 = __shfl_xor_sync(0xFFFFFFFFu, work, off);
+                    const int a2 = __shfl_xor_sync(0xFFFFFFFFu, any_stall, off);
+                    if (off < g) {
+                        span = fmaxf(span, s2);
+                        work = fmaxf(work, w2);
+                        any_stall |= a2;
+                    }
+                }
+                if (glane == 0 && have) {
+                    if (any_stall) {
+                        status = PF_SIM_STALL;
+                        tput_out = 0.f;
+                    } else if (run) {
+                        float T_pipe = span;
+                        if (m > m_sim) T_pipe += (float)(m - m_sim) * work;
+                        tput_out = train_price<RI>(P, c, D, T, T_pipe);
+                    }
+                    if (A.tput_sim) A.tput_sim[w] = tput_out;
+                    if (A.status) A.status[w] = (uint8_t)status;
+                }
+                __syncwarp();
             }
-            if (A.tput_sim) A.tput_sim[w] = tput;
-            if (A.status) A.status[w] = stalled ? PF_SIM_STALL : PF_SIM_OK;
-        }
-        __syncwarp();
-    }
-    }  // active warps of this class
-    __syncthreads();  // the next class lays the pool out differently
+        }  // lane-group widths
     }  // classes
 }
 
@@ -600,7 +558,7 @@ __global__ void __launch_bounds__(kThreads) dense_topk_kernel(const DenseTopkArg
 }
 
 struct SimLayout {
-    size_t off_ctrl, off_lists, off_scores, off_topk, total;
+    size_t off_ctrl, off_bin_of, off_list, off_scores, off_topk, total;
     int topk_blocks;
     uint64_t topk_keys_max;
     TopkLayout tk;
@@ -610,9 +568,10 @@ static SimLayout sim_layout(const pf_plan_t *p, uint64_t n, uint32_t k)
 {
     SimLayout l;
     const size_t nn = (size_t)(n ? n : 1);
-    l.off_ctrl = 0;                       // work[kSimClasses], cls_count[kSimClasses]
-    l.off_lists = 256;
-    l.off_scores = l.off_lists + (((size_t)kSimClasses * nn * 4 + 255) & ~(size_t)255);
+    l.off_ctrl = 0;                       // 512 B: work, bin_count, bin_off, bin_fill
+    l.off_bin_of = 512;
+    l.off_list = l.off_bin_of + ((nn + 255) & ~(size_t)255);
+    l.off_scores = l.off_list + ((nn * 4 + 255) & ~(size_t)255);
     l.off_topk = l.off_scores + ((nn * 4 + 255) & ~(size_t)255);
     uint64_t tb = (n + kThreads - 1) / kThreads;
     uint64_t cap = (uint64_t)p->sm_count * 2;
@@ -646,27 +605,30 @@ template <typename RI>
 static int launch_simulate(pf_plan_t *p, SimArgs a, uint64_t n, cudaStream_t st, int *n_kernels)
 {
     *n_kernels = 0;
-    sim_classify_kernel<RI><<<(unsigned int)((n + 255) / 256), 256, 0, st>>>(p->dev, a);
-    count_launch();
-    (*n_kernels)++;
-    PF_CUDA_TRY(cudaGetLastError(), "sim_classify_kernel launch");
-    // largest class the plan can produce, and a pool that holds at least one such timeline
+    const unsigned int nb = (unsigned int)((n + 255) / 256);
+    sim_classify_kernel<RI><<<nb, 256, 0, st>>>(p->dev, a);
+    sim_offsets_kernel<<<1, 32, 0, st>>>(a);
+    sim_scatter_kernel<<<nb, 256, 0, st>>>(a);
+    for (int i = 0; i < 3; i++) count_launch();
+    *n_kernels += 3;
+    PF_CUDA_TRY(cudaGetLastError(), "simulator pre-pass launch");
+    // largest class the plan can produce; a warp's slice holds one such timeline plus four duration tables
     const int entries_max = a.q_max * PF_SIM_WINDOW;
     int cls_hi = 0;
     while (cls_hi < kSimClasses - 1 && sim_class_entries(cls_hi) < entries_max) cls_hi++;
-    const size_t biggest = sim_warp_floats(sim_class_entries(cls_hi), a.q_max) * sizeof(float);
-    if (biggest > 226 * 1024) return PF_EUNSUPPORTED;   // 227 KB per block minus the kernel's static words
-    size_t pool = 72 * 1024;                         // three blocks per SM when the largest timeline allows
-    if (pool < biggest) pool = biggest;
+    const int warp_floats = sim_class_entries(cls_hi) + 4 * 2 * a.q_max;
+    const size_t pool = (size_t)(kSimThreads / 32) * warp_floats * sizeof(float);
+    if (pool > 226 * 1024) return PF_EUNSUPPORTED;
     int per_sm = (int)((size_t)(227 * 1024) / (pool + 1024));
-    per_sm = per_sm < 1 ? 1 : per_sm;
+    per_sm = per_sm < 1 ? 1 : (per_sm > 12 ? 12 : per_sm);
     a.cls_hi = cls_hi;
-    a.pool_floats = (int)(pool / sizeof(float));
+    a.warp_floats = warp_floats;
     const uint64_t cap = (uint64_t)p->sm_count * per_sm;
-    const int grid = (int)(n < cap ? n : cap);
+    const uint64_t want = (n + kSimThreads / 32 - 1) / (kSimThreads / 32);
+    const int grid = (int)(want < cap ? want : cap);
     PF_CUDA_TRY(cudaFuncSetAttribute(simulate_kernel<RI>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pool),
                 "simulate_kernel smem");
-    simulate_kernel<RI><<<grid, kSimMaxWarps * 32, pool, st>>>(p->dev, a);
+    simulate_kernel<RI><<<grid, kSimThreads, pool, st>>>(p->dev, a);
     count_launch();
     (*n_kernels)++;
     PF_CUDA_TRY(cudaGetLastError(), "simulate_kernel launch");
@@ -713,13 +675,16 @@ extern "C" int pf_simulate(pf_plan_t *p, const uint64_t *d_surv_idx, uint64_t n,
     a.surv = d_surv_idx; a.n = n; a.d_n = d_n; a.seed = jitter_seed;
     a.tput_sim = scores; a.status = d_sim_status;
     a.work = (unsigned int *)(ws + lay.off_ctrl);
-    a.cls_count = a.work + kSimClasses;
-    a.cls_list = (uint32_t *)(ws + lay.off_lists);
+    a.bin_count = a.work + kSimBins;
+    a.bin_off = a.bin_count + kSimBins;
+    a.bin_fill = a.bin_off + kSimBins + 1;
+    a.bin_of = ws + lay.off_bin_of;
+    a.list = (uint32_t *)(ws + lay.off_list);
     a.vals = p->d_vals; a.dual_ops = tab->d_ops; a.dual_off = tab->d_offset;
     a.q_max = plan_q_max(p);
     a.cls_hi = 0;
-    a.pool_floats = 0;
-    PF_CUDA_TRY(cudaMemsetAsync(ws + lay.off_ctrl, 0, 256, st), "pf_simulate: counter reset");
+    a.warp_floats = 0;
+    PF_CUDA_TRY(cudaMemsetAsync(ws + lay.off_ctrl, 0, 512, st), "pf_simulate: counter reset");
     if (n > 0) {
         int nk = 0;
         timing_begin(p, PF_T_SIMULATE, st);
