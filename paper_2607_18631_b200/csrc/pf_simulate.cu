@@ -180,7 +180,8 @@ __device__ __forceinline__ float jitter(uint32_t seed_mixed, uint64_t idx, int q
 
 constexpr int kSimClasses = 7;          // timeline sizes 256 << c entries (stage streams x microbatches)
 constexpr int kSimGroups = 3;           // lanes per candidate: 8, 16 or 32 (pipeline depth rounded up)
-constexpr int kSimBins = kSimClasses * kSimGroups;
+constexpr int kSimKinds = 3;            // schedule class: candidates of one batch share the round loop
+constexpr int kSimBins = kSimClasses * kSimGroups * kSimKinds;
 constexpr int kSimThreads = 128;        // 4 warps per block, each with its own shared-memory slice
 __host__ __device__ inline int sim_class_entries(int c) { return 256 << c; }
 __host__ __device__ inline int sim_group_lanes(int g) { return 8 << g; }
@@ -247,7 +248,7 @@ __global__ void __launch_bounds__(256) sim_classify_kernel(const __grid_constant
             int cls = 0;
             while (cls < kSimClasses - 1 && sim_class_entries(cls) < entries) cls++;
             if (sim_class_entries(cls) >= entries && streams <= A.q_max)
-                bin = cls * kSimGroups + (pp <= 8 ? 0 : (pp <= 16 ? 1 : 2));
+                bin = (cls * kSimGroups + (pp <= 8 ? 0 : (pp <= 16 ? 1 : 2))) * kSimKinds + kind;
         }
         A.bin_of[w] = (uint8_t)bin;
     }
@@ -287,6 +288,125 @@ __global__ void __launch_bounds__(256) sim_scatter_kernel(const SimArgs A)
     if (bin >= 0) A.list[A.bin_off[bin] + base + __popc(peers & ((1u << lane) - 1u))] = (uint32_t)w;
 }
 
+// The round loops, one per schedule class (all candidates of a batch share the class).  The timeline has one
+// 32-bit word per (stage stream, microbatch): 0 = nothing finished, +t = forward ended at t, -t = backward ended
+// at t.  In every round a lane runs at most its next op, and only if the word it depends on already carries the
+// right sign; the body is branch-free apart from that test.  Every 64 rounds some lane of the warp must have
+// advanced, otherwise the loop ends and the unfinished candidates are reported as stalled.
+#define PF_SIM_ROUND_END()                                               \
+    if (!__any_sync(0xFFFFFFFFu, done < total_ops)) break;               \
+    if ((++rounds & 63) == 0) {                                          \
+        if (!__any_sync(0xFFFFFFFFu, moved)) break;                      \
+        moved = false;                                                   \
+    }
+
+// 1F1B: rank = stage = lane; `warm` forwards, then one forward / one backward, then the remaining backwards
+__device__ __forceinline__ void sim_rounds_1f1b(volatile float *tl, const float *durF, const float *durB, int glane,
+                                                int pp, int nj, int warm, int total_ops, float lat, float &clock_out,
+                                                int &done_out)
+{
+    const bool depF = glane > 0, depB = glane < pp - 1;
+    volatile float *inF = tl + (depF ? glane - 1 : glane) * nj, *inB = tl + (depB ? glane + 1 : glane) * nj;
+    volatile float *out = tl + glane * nj;
+    const float dF = total_ops ? durF[glane] : 0.f, dB = total_ops ? durB[glane] : 0.f;
+    int nF = 0, nB = 0, done = 0, rounds = 0;
+    bool moved = false;
+    float clock = 0.f;
+    for (;;) {
+        if (done < total_ops) {
+            const bool isb = !(nF < warm || (nF < nj && nF - warm == nB));
+            const int j = isb ? nB : nF;
+            const bool dep = isb ? depB : depF;
+            const float e = (isb ? inB : inF)[j];
+            if (!dep || (isb ? e < 0.f : e > 0.f)) {
+                clock = fmaxf(clock, dep ? fabsf(e) + lat : 0.f) + (isb ? dB : dF);
+                out[j] = isb ? -clock : clock;
+                nF += isb ? 0 : 1;
+                nB += isb ? 1 : 0;
+                done++;
+                moved = true;
+            }
+        }
+        PF_SIM_ROUND_END()
+    }
+    clock_out = clock;
+    done_out = done;
+}
+
+// Interleaved: v chunks per rank; unit k of a rank is microbatch (k / (pp v)) pp + k mod pp of chunk
+// (k mod (pp v)) / pp, backward units walk the chunks downward; cursors advance without divisions
+__device__ __forceinline__ void sim_rounds_interleaved(volatile float *tl, const float *durF, const float *durB,
+                                                       int glane, int pp, int v, int nj, int U, int warm,
+                                                       int total_ops, float lat, float &clock_out, int &done_out)
+{
+    const int Q = pp * v;
+    int nF = 0, nB = 0, done = 0, rounds = 0;
+    int fw = 0, fc = 0, fg = 0, bw = 0, bc = 0, bg = 0;
+    bool moved = false;
+    float clock = 0.f;
+    for (;;) {
+        if (done < total_ops) {
+            const bool isb = !(nF < warm || (nF < U && nF - warm == nB));
+            const int cw = isb ? bw : fw, cc = isb ? bc : fc, cg = isb ? bg : fg;
+            const int j = cg * pp + cw;
+            const int q = (isb ? v - 1 - cc : cc) * pp + glane;
+            const bool dep = isb ? (q < Q - 1) : (q > 0);
+            const int nb = dep ? (isb ? q + 1 : q - 1) : q;
+            const float e = tl[nb * nj + j];
+            const float dur = (isb ? durB : durF)[q];
+            if (!dep || (isb ? e < 0.f : e > 0.f)) {
+                clock = fmaxf(clock, dep ? fabsf(e) + lat : 0.f) + dur;
+                tl[q * nj + j] = isb ? -clock : clock;
+                int w_ = cw + 1, c_ = cc, g_ = cg;
+                if (w_ == pp) {
+                    w_ = 0;
+                    if (++c_ == v) c_ = 0, g_++;
+                }
+                if (isb) bw = w_, bc = c_, bg = g_, nB++;
+                else fw = w_, fc = c_, fg = g_, nF++;
+                done++;
+                moved = true;
+            }
+        }
+        PF_SIM_ROUND_END()
+    }
+    clock_out = clock;
+    done_out = done;
+}
+
+// DualPipe-style: two directions; the per-rank order comes from the host-built table
+__device__ __forceinline__ void sim_rounds_dual(volatile float *tl, const float *durF, const float *durB, int glane,
+                                                int pp, int nj, const uint8_t *ops, int total_ops, float lat,
+                                                float &clock_out, int &done_out)
+{
+    int done = 0, rounds = 0;
+    bool moved = false;
+    float clock = 0.f;
+    for (;;) {
+        if (done < total_ops) {
+            const uint32_t op = __ldg(ops + done);
+            const bool isb = op & 1;
+            const int d = (op >> 1) & 1, j = op >> 2;
+            const int q = d ? pp - 1 - glane : glane;
+            const int sidx = d * pp + q;
+            const bool dep = isb ? (q < pp - 1) : (q > 0);
+            const int nb = dep ? (isb ? sidx + 1 : sidx - 1) : sidx;
+            const float e = tl[nb * nj + j];
+            const float dur = (isb ? durB : durF)[q];
+            if (!dep || (isb ? e < 0.f : e > 0.f)) {
+                clock = fmaxf(clock, dep ? fabsf(e) + lat : 0.f) + dur;
+                tl[sidx * nj + j] = isb ? -clock : clock;
+                done++;
+                moved = true;
+            }
+        }
+        PF_SIM_ROUND_END()
+    }
+    clock_out = clock;
+    done_out = done;
+}
+#undef PF_SIM_ROUND_END
+
 // One launch serves every bin.  Every warp owns a fixed slice of the block's shared memory, large enough for
 // one timeline of the largest class (or several of a smaller one), and works through the bins on its own --
 // largest timelines first, so the longest simulations start earliest and the tail is one candidate long.  No
@@ -314,8 +434,9 @@ __global__ void __launch_bounds__(kSimThreads, 4) simulate_kernel(const __grid_c
     float *slice = s_mem + (size_t)warp * A.warp_floats;   // [E_hi] timelines, then 4 x (durF, durB)[q_max]
 
     for (int cls = A.cls_hi; cls >= 0; cls--) {
-        for (int gi = 0; gi < kSimGroups; gi++) {
-            const int bin = cls * kSimGroups + gi;
+        for (int gk = 0; gk < kSimGroups * kSimKinds; gk++) {
+            const int gi = gk / kSimKinds, bin_kind = gk - gi * kSimKinds;
+            const int bin = (cls * kSimGroups + gi) * kSimKinds + bin_kind;
             const unsigned int n_bin = A.bin_count[bin];
             if (n_bin == 0) continue;
             const int g = sim_group_lanes(gi);
@@ -394,7 +515,7 @@ __global__ void __launch_bounds__(kSimThreads, 4) simulate_kernel(const __grid_c
                 const int nj = dual ? m_sim / 2 : m_sim;      // microbatches per stage stream
                 const int n_entries = (dual ? 2 * Q : Q) * nj;
                 // filed under a bin that cannot hold it: never for a feasible plan; reported, not overrun
-                bool stalled = run && (n_entries > E || Q > A.q_max || pp > g);
+                bool stalled = run && (n_entries > E || Q > A.q_max || pp > g || kind != bin_kind);
                 if (stalled) run = false;
 
                 // ---- stage durations (balanced layer split, head on the last stage, jitter), cleared timeline
@@ -424,49 +545,15 @@ __global__ void __launch_bounds__(kSimThreads, 4) simulate_kernel(const __grid_c
                 }
                 const int total_ops = (rank_active && run) ? 2 * U : 0;
                 const float lat = run ? T.p : 0.f;
-                int done = 0, rounds = 0, nF = 0, nB = 0;
-                int fw = 0, fc = 0, fg = 0, bw = 0, bc = 0, bg = 0;
-                bool moved = false;
+                // a batch's candidates share the schedule class of their bin: one specialised loop per class
+                int done = 0;
                 float clock = 0.f;
-
-                for (;;) {
-                    if (done < total_ops) {
-                        // next op of this rank: from the table (DualPipe-style) or from the unit cursors
-                        uint32_t op = 0;
-                        if (dual) op = __ldg(dops + done);
-                        const bool isb_c = !(nF < warm || (nF < U && nF - warm == nB));
-                        const bool isb = dual ? (op & 1u) != 0 : isb_c;
-                        const int d = dual ? (int)((op >> 1) & 1u) : 0;
-                        const int cw = isb ? bw : fw, cc = isb ? bc : fc, cg = isb ? bg : fg;
-                        const int j = dual ? (int)(op >> 2) : cg * pp + cw;
-                        const int q = dual ? (d ? pp - 1 - glane : glane) : (isb ? v - 1 - cc : cc) * pp + glane;
-                        const int sidx = d * Q + q;             // stage stream (direction-major for DualPipe)
-                        const bool dep = isb ? (q < Q - 1) : (q > 0);
-                        const int nb = dep ? (isb ? sidx + 1 : sidx - 1) : sidx;
-                        const float e = tl[nb * nj + j];
-                        const float dur = (isb ? durB : durF)[q];
-                        // a forward waits for a positive word (forward ended), a backward for a negative one
-                        const bool ready = !dep || (isb ? e < 0.f : e > 0.f);
-                        if (ready) {
-                            clock = fmaxf(clock, dep ? fabsf(e) + lat : 0.f) + dur;
-                            tl[sidx * nj + j] = isb ? -clock : clock;
-                            int w_ = cw + 1, c_ = cc, g_ = cg;
-                            if (w_ == pp) {
-                                w_ = 0;
-                                if (++c_ == v) c_ = 0, g_++;
-                            }
-                            if (isb) bw = w_, bc = c_, bg = g_, nB++;
-                            else fw = w_, fc = c_, fg = g_, nF++;
-                            done++;
-                            moved = true;
-                        }
-                    }
-                    if (!__any_sync(0xFFFFFFFFu, done < total_ops)) break;
-                    if ((++rounds & 63) == 0) {
-                        if (!__any_sync(0xFFFFFFFFu, moved)) break;   // nothing advanced: give up, report below
-                        moved = false;
-                    }
-                }
+                if (bin_kind == PF_KIND_1F1B)
+                    sim_rounds_1f1b(tl, durF, durB, glane, pp, nj, warm, total_ops, lat, clock, done);
+                else if (bin_kind == PF_KIND_INTERLEAVED)
+                    sim_rounds_interleaved(tl, durF, durB, glane, pp, v, nj, U, warm, total_ops, lat, clock, done);
+                else
+                    sim_rounds_dual(tl, durF, durB, glane, pp, nj, dops, total_ops, lat, clock, done);
                 if (done < total_ops) stalled = true;
 
                 // ---- makespan, steady-state extension beyond the window, pricing (reductions inside the group)
@@ -568,8 +655,8 @@ static SimLayout sim_layout(const pf_plan_t *p, uint64_t n, uint32_t k)
 {
     SimLayout l;
     const size_t nn = (size_t)(n ? n : 1);
-    l.off_ctrl = 0;                       // 512 B: work, bin_count, bin_off, bin_fill
-    l.off_bin_of = 512;
+    l.off_ctrl = 0;                       // 2 KB: work, bin_count, bin_off, bin_fill (kSimBins words each)
+    l.off_bin_of = 2048;
     l.off_list = l.off_bin_of + ((nn + 255) & ~(size_t)255);
     l.off_scores = l.off_list + ((nn * 4 + 255) & ~(size_t)255);
     l.off_topk = l.off_scores + ((nn * 4 + 255) & ~(size_t)255);
@@ -684,7 +771,7 @@ extern "C" int pf_simulate(pf_plan_t *p, const uint64_t *d_surv_idx, uint64_t n,
     a.q_max = plan_q_max(p);
     a.cls_hi = 0;
     a.warp_floats = 0;
-    PF_CUDA_TRY(cudaMemsetAsync(ws + lay.off_ctrl, 0, 512, st), "pf_simulate: counter reset");
+    PF_CUDA_TRY(cudaMemsetAsync(ws + lay.off_ctrl, 0, 2048, st), "pf_simulate: counter reset");
     if (n > 0) {
         int nk = 0;
         timing_begin(p, PF_T_SIMULATE, st);
