@@ -313,6 +313,8 @@ __device__ __forceinline__ void sim_rounds_1f1b(volatile float *tl, const float 
     bool moved = false;
     float clock = 0.f;
     for (;;) {
+#pragma unroll
+        for (int rep = 0; rep < 4; rep++)
         if (done < total_ops) {
             const bool isb = !(nF < warm || (nF < nj && nF - warm == nB));
             const int j = isb ? nB : nF;
@@ -345,6 +347,8 @@ __device__ __forceinline__ void sim_rounds_interleaved(volatile float *tl, const
     bool moved = false;
     float clock = 0.f;
     for (;;) {
+#pragma unroll
+        for (int rep = 0; rep < 4; rep++)
         if (done < total_ops) {
             const bool isb = !(nF < warm || (nF < U && nF - warm == nB));
             const int cw = isb ? bw : fw, cc = isb ? bc : fc, cg = isb ? bg : fg;
