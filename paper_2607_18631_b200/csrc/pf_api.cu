@@ -272,6 +272,11 @@ extern "C" int pf_plan_create(const pf_model_t *model, const pf_cluster_t *clust
         slab *= d.radix[n_inner];
         n_inner++;
     }
+    // a first axis longer than the target still makes a better slab than single candidates
+    if (n_inner == 0 && d.radix[0] <= pf::kSlabMax) {
+        slab = d.radix[0];
+        n_inner = 1;
+    }
     d.n_inner = n_inner;
     d.slab = (uint32_t)slab;
     for (int a = 0; a < want_axes; a++) {

@@ -185,3 +185,36 @@ def test_large_unconstrained_topk():
     compare_dense(res, reason, tput, mem)
     compare_topk(res, orc, reason, tput, first, 1024)
     plan.close()
+
+
+def test_degenerate_spaces():
+    """Edge shapes: a 4096-entry axis, single-entry axes everywhere else, a space with no feasible plan at all
+    (empty top-k, empty survivor list, empty simulation), k = 1."""
+    import torch
+    # (a) one long axis (the kernel-variant list repeated up to the axis limit), everything else fixed
+    cfg = variant("mid", cluster=dict(budget_bytes=10 ** 15))
+    cfg["axes"] = [("kv", [i % 4 for i in range(4096)]), ("rec", [1]), ("sched", [0]), ("mb", [2]), ("v", [1]),
+                   ("ep", [2]), ("pp", [2]), ("tp", [2]), ("dp", [2]), ("world", [8])]
+    cfg["k"] = 1
+    r = _full_parity(cfg)
+    assert len(r) == 4096 and ((r & 0x7F) == 0).sum() > 3000
+    # (b) a first axis longer than a slab may be: slabs degenerate to single candidates of the second axis
+    cfg = variant("tiny")
+    cfg["axes"][0] = ("kv", [i % 2 for i in range(3000)])
+    cfg["k"] = 7
+    _full_parity(cfg)
+    # (c) nothing feasible: budget of one byte
+    cfg = variant("mid", cluster=dict(budget_bytes=1))
+    plan, orc = _plan(cfg), Oracle(cfg)
+    reason, tput, mem, _ = orc.score_range(threads=8)
+    assert ((reason & 0x7F) == 0).sum() == 0
+    res = gpu_score(plan, k=128)
+    compare_dense(res, reason, tput, mem)
+    assert len(res["topk_idx"]) == 0
+    out = plan.score(k=0)
+    sel = plan.select_survivors(out["reason"], out["tput"], 1000)
+    sim = plan.simulate(sel["surv_idx"], 1000, 4, k=10, d_n=sel["surv_count"])
+    torch.cuda.synchronize()
+    assert int(sel["surv_count"].item()) == 0 and int(sim["topk_count"].item()) == 0
+    assert torch.all(sim["topk_idx"] == -1)
+    plan.close()
