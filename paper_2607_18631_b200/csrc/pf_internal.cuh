@@ -261,7 +261,7 @@ __device__ __forceinline__ void tk_push(unsigned long long *buf, int *count, uns
 // host: workspace layout of one top-k reduction whose producers append at most n_keys_max keys in total.
 // ctrl is 256 bytes: uint32 [0] producer work counter, [1] keys in list A, [2] keys in list B, [3] spare;
 // uint64 at byte 16: the producers' shared admission threshold (largest k-th key any block has reached).
-constexpr int kReduceSeg = 8192;     // keys one block of the reduce kernel walks through
+constexpr int kReduceSeg = 2048;     // keys one block of the reduce kernel walks through
 constexpr int kReduceThreads = 1024;
 struct TopkLayout {
     size_t off_ctrl, off_keys_a, off_keys_b, total;
