@@ -130,6 +130,10 @@ def lib():
         L.orc_topk_list.argtypes = [C.c_void_p, C.c_void_p, u64, u64, C.c_void_p, C.c_void_p]
         L.orc_select_survivors.restype = u64
         L.orc_select_survivors.argtypes = [PP, C.c_void_p, C.c_void_p, u64, u64, u64, C.c_void_p]
+        L.orc_serve_plan_count.restype = u64
+        L.orc_serve_plan_count.argtypes = [PP]
+        L.orc_aggregate_serving.restype = None
+        L.orc_aggregate_serving.argtypes = [PP, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.orc_schedule_order.restype = C.c_int
         L.orc_schedule_order.argtypes = [C.c_int, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_int]
         L.orc_makespan.restype = f64
@@ -265,6 +269,16 @@ class Oracle:
         os_ = np.zeros(k, dtype=np.float64)
         n = lib().orc_topk_list(_ptr(idx), _ptr(score), len(idx), k, _ptr(oi), _ptr(os_))
         return oi[:n], os_[:n]
+
+    def aggregate_serving(self, reason, tput):
+        """Per-plan (reason uint8[n_plans], tput float64[n_plans]) over all length scenarios."""
+        n = int(lib().orc_serve_plan_count(C.byref(self.pb)))
+        reason = np.ascontiguousarray(reason, dtype=np.uint8)
+        tput = np.ascontiguousarray(tput, dtype=np.float64)
+        pr = np.zeros(n, dtype=np.uint8)
+        pt = np.zeros(n, dtype=np.float64)
+        lib().orc_aggregate_serving(C.byref(self.pb), _ptr(reason), _ptr(tput), _ptr(pr), _ptr(pt))
+        return pr, pt
 
     def select_survivors(self, reason, tput, first: int, s_max: int):
         out = np.zeros(max(min(s_max, len(reason)), 1), dtype=np.uint64)

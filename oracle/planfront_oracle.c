@@ -568,6 +568,45 @@ uint64_t orc_select_survivors(const orc_problem_t *pb, const uint8_t *reason, co
     return n;
 }
 
+/* ------------------------------------------------------------------ serving: per-plan aggregate */
+
+uint64_t orc_serve_plan_count(const orc_problem_t *pb)
+{
+    const orc_axes_t *ax = &pb->axes;
+    return orc_space_size(pb) / (uint64_t)ax->len[ax->n_axes - 1];
+}
+
+void orc_aggregate_serving(const orc_problem_t *pb, const uint8_t *reason, const double *tput,
+                           uint8_t *plan_reason, double *plan_tput)
+{
+    const orc_axes_t *ax = &pb->axes;
+    const int64_t n_scen = ax->len[ax->n_axes - 1];
+    const uint64_t n_plans = orc_serve_plan_count(pb);
+    for (uint64_t p = 0; p < n_plans; p++) {
+        int first_fail = 0, flags = 0;
+        double tokens = 0.0, time = 0.0;
+        for (int64_t i = 0; i < n_scen; i++) {
+            uint64_t idx = p + n_plans * (uint64_t)i;
+            int r = reason[idx];
+            if ((r & 0x7f) != 0) {
+                if (!first_fail) first_fail = r & 0x7f;
+                continue;
+            }
+            flags |= r & ORC_FLAG_EXTRAPOLATED;
+            double O = (double)pb->workload.scen_O[ax->val[ax->n_axes - 1][i]];
+            tokens += O;          /* output tokens of one request of this scenario */
+            time += O / tput[idx]; /* and the GPU-seconds they take at this scenario's rate */
+        }
+        if (first_fail) {
+            plan_reason[p] = (uint8_t)first_fail;
+            plan_tput[p] = 0.0;
+        } else {
+            plan_reason[p] = (uint8_t)flags;
+            plan_tput[p] = tokens / time;
+        }
+    }
+}
+
 /* ------------------------------------------------------------------ schedule orders */
 
 static int order_1f1b(int pp, int m, int32_t *out, int stride)

@@ -184,6 +184,16 @@ uint64_t orc_topk_list(const uint64_t *idx, const double *score, uint64_t n, uin
 uint64_t orc_select_survivors(const orc_problem_t *pb, const uint8_t *reason, const double *tput,
                               uint64_t first, uint64_t count, uint64_t s_max, uint64_t *out_idx);
 
+/* --- serving: one score per plan over the whole length mix (Sec. 5 RQ3 ranks serving PLANS) ---
+ * The serving space lists every plan once per (prompt, output) scenario; the scenario axis is the most
+ * significant one, so candidate idx = plan + n_plans * scenario_digit.  A plan is feasible iff it is feasible
+ * in every scenario (its reason is that of the first failing scenario); its score is total output tokens over
+ * total time, which for per-scenario throughputs tput_i and output lengths O_i is the O-weighted harmonic mean
+ * sum(O_i) / sum(O_i / tput_i).  Bit 7 (extrapolated) is the OR over scenarios. */
+uint64_t orc_serve_plan_count(const orc_problem_t *pb);
+void orc_aggregate_serving(const orc_problem_t *pb, const uint8_t *reason, const double *tput,
+                           uint8_t *plan_reason, double *plan_tput);
+
 /* --- simulator tier --- */
 /* op encoding for per-rank orders: bit 0 = backward, bit 1 = direction (DualPipe), bits 2..9 =
  * virtual stage / position q, bits 10.. = microbatch j */

@@ -452,3 +452,77 @@ def test_survivors_are_best_feasible_sorted_by_index():
     assert set(s.tolist()) == set(top.tolist())
     allf = o.select_survivors(reason, tput, 0, 10 ** 6)
     assert len(allf) == int(((reason & 0x7F) == 0).sum())
+
+
+# ----------------------------------------------------------------------------- serving: one score per plan
+
+def test_serving_plan_aggregate_is_tokens_over_time():
+    """Sec. 5 RQ3 ranks serving plans, not (plan, request-shape) pairs.  The aggregate must equal total output
+    tokens over total time, rebuilt here from the per-scenario prefill / decode times, and must reduce to the
+    per-scenario score when the mix has one scenario or all scenarios score alike."""
+    cfg = variant("serve", cluster=dict(budget_bytes=10 ** 15))
+    for k in cfg["kern"]:
+        k["avail_mask"] = 255
+    # a small length mix keeps the per-candidate loop short
+    cfg["workload"]["scen_P"] = cfg["workload"]["scen_P"][:5]
+    cfg["workload"]["scen_O"] = cfg["workload"]["scen_O"][:5]
+    cfg["axes"][6] = ("scen", [0, 1, 2, 3, 4])
+    o = Oracle(cfg)
+    reason, tput, _, _ = o.score_range(threads=4)
+    pr, pt = o.aggregate_serving(reason, tput)
+    n_plans = o.size // 5
+    assert len(pr) == n_plans
+    checked = 0
+    for p in range(0, n_plans, 37):
+        ds = [o.eval(p + n_plans * i) for i in range(5)]
+        if any(d["reason"] & 0x7F for d in ds):
+            first = next(d["reason"] & 0x7F for d in ds if d["reason"] & 0x7F)
+            assert pr[p] == first and pt[p] == 0.0
+            continue
+        checked += 1
+        d0 = ds[0]
+        n_eng = d0["tp"] * d0["ep"] if d0["dpa"] else d0["tp"]
+        b_loc = d0["batch"] // d0["ep"] if d0["dpa"] else d0["batch"]
+        O = cfg["workload"]["scen_O"]
+        tokens = sum(d0["batch"] * O[i] for i in range(5))
+        time = sum(b_loc * ds[i]["T_pre"] + O[i] * ds[i]["T_dec"] for i in range(5))
+        want = tokens / time / n_eng
+        if not cfg["kern"][d0["kv"]]["is_native"]:
+            want /= 1 + cfg["kern"][d0["kv"]]["patch_ovh"]
+        assert pt[p] == pytest.approx(want, rel=1e-12)
+        per = [d["tput"] for d in ds]
+        assert min(per) * (1 - 1e-12) <= pt[p] <= max(per) * (1 + 1e-12)
+        assert pr[p] == (0x80 if any(d["reason"] & 0x80 for d in ds) else 0)
+    assert checked > 20
+    # one scenario: the aggregate is the scenario's own score
+    one = variant("serve", cluster=dict(budget_bytes=10 ** 15))
+    one["axes"][6] = ("scen", [3])
+    oo = Oracle(one)
+    r1, t1, _, _ = oo.score_range(threads=4)
+    pr1, pt1 = oo.aggregate_serving(r1, t1)
+    f = (r1 & 0x7F) == 0
+    np.testing.assert_allclose(pt1[f], t1[f], rtol=1e-15)
+    np.testing.assert_array_equal(pr1, r1)
+    # the same scenario listed three times: still the scenario's own score
+    rep = variant("serve", cluster=dict(budget_bytes=10 ** 15))
+    rep["axes"][6] = ("scen", [3, 3, 3])
+    orp = Oracle(rep)
+    r3, t3, _, _ = orp.score_range(threads=4)
+    pr3, pt3 = orp.aggregate_serving(r3, t3)
+    np.testing.assert_allclose(pt3[f], t1[f], rtol=1e-14)
+
+
+def test_serving_plan_is_infeasible_if_any_scenario_is():
+    """The KV cache grows with prompt + output length, so the memory gate can reject a plan for the long requests
+    only; such a plan cannot serve the mix."""
+    cfg = make_config("serve")
+    o = Oracle(cfg)
+    reason, tput, _, _ = o.score_range(threads=8)
+    pr, pt = o.aggregate_serving(reason, tput)
+    n_plans = o.size // 128
+    per = (reason.reshape(128, n_plans) & 0x7F)
+    any_bad = (per != 0).any(axis=0)
+    all_bad = (per != 0).all(axis=0)
+    assert (any_bad & ~all_bad).sum() > 0                      # mixed plans exist in this space
+    np.testing.assert_array_equal((pr & 0x7F) != 0, any_bad)
+    assert np.all(pt[any_bad] == 0) and np.all(pt[~any_bad] > 0)
