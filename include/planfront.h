@@ -259,6 +259,22 @@ int pf_simulate(pf_plan_t *plan, const uint64_t *d_surv_idx, uint64_t n, const u
                 uint64_t *d_topk_idx, float *d_topk_score, uint32_t *d_topk_count, void *d_workspace,
                 size_t workspace_bytes, void *stream);
 
+/* Serving plans ranked over the whole request-length mix (Sec. 5 RQ3 compares serving PLANS; the scored
+ * space lists every plan once per (prompt, output) scenario, scenario being the most significant axis, so
+ * candidate = plan + n_plans * scenario_digit and n_plans = N / len(scen axis)).
+ * Input: the dense d_reason / d_tput of pf_score over the WHOLE space (first = 0, count = N).
+ * Per plan: feasible iff feasible in every scenario, else the reason of the first failing scenario and score
+ * 0; score = total output tokens / total time = sum(O_i) / sum(O_i / tput_i) over the scenarios; bit 7
+ * (extrapolated) is the OR over scenarios.
+ *   d_plan_reason[n_plans] uint8, d_plan_tput[n_plans] float -- each may be NULL;
+ *   top-k over plans as in pf_score (k = 0 skips it), indices are plan numbers.
+ * Errors: PF_EINVAL, PF_EWORKSPACE, PF_EUNSUPPORTED (training plan), PF_ECUDA. */
+uint64_t pf_serve_plan_count(const pf_plan_t *plan);
+size_t pf_aggregate_workspace(const pf_plan_t *plan, uint32_t k);
+int pf_aggregate_serving(pf_plan_t *plan, const uint8_t *d_reason, const float *d_tput, uint8_t *d_plan_reason,
+                         float *d_plan_tput, uint32_t k, uint64_t *d_topk_idx, float *d_topk_score,
+                         uint32_t *d_topk_count, void *d_workspace, size_t workspace_bytes, void *stream);
+
 /* Host helper (no GPU): the DualPipe-style per-rank op order the simulator uses for pipeline depth pp
  * (1 or even, <= PF_SIM_MAX_RANKS) and m microbatches (even, 2..PF_SIM_WINDOW).  The order is defined by a
  * nominal list scheduling (forward 1 tick, backward 2 ticks, zero latency; ready op with the smallest
@@ -288,8 +304,9 @@ int pf_search_host(pf_plan_t *plan, uint32_t k, uint64_t s_max, uint32_t k_sim, 
  * on the caller's stream; pf_timing_read waits for the recorded events, adds the elapsed times (ms) and
  * kernel counts per class into ms[PF_T_CLASSES] / kernels[PF_T_CLASSES], and forgets them.
  * PF_T_SCORE: the scoring kernel; PF_T_TOPK: top-k list kernels (merge passes, dense top-k);
- * PF_T_SELECT: the survivor-selection kernels; PF_T_SIMULATE: the simulator kernel. */
-enum { PF_T_SCORE = 0, PF_T_TOPK = 1, PF_T_SELECT = 2, PF_T_SIMULATE = 3, PF_T_CLASSES = 4 };
+ * PF_T_SELECT: the survivor-selection kernels; PF_T_SIMULATE: the simulator kernels;
+ * PF_T_AGGREGATE: the per-plan serving aggregate. */
+enum { PF_T_SCORE = 0, PF_T_TOPK = 1, PF_T_SELECT = 2, PF_T_SIMULATE = 3, PF_T_AGGREGATE = 4, PF_T_CLASSES = 5 };
 int pf_timing_enable(pf_plan_t *plan, int on);
 int pf_timing_read(pf_plan_t *plan, float *ms, uint32_t *kernels);
 

@@ -23,9 +23,9 @@ UINT64_MAX = 0xFFFFFFFFFFFFFFFF
 EXPORTS = ("pf_version", "pf_strerror", "pf_reason_str", "pf_last_cuda_error", "pf_plan_create", "pf_plan_destroy",
            "pf_plan_size", "pf_decode", "pf_score_workspace", "pf_score", "pf_topk_merge", "pf_select_workspace",
            "pf_select_survivors", "pf_simulate_workspace", "pf_simulate", "pf_search_workspace", "pf_search_host",
-           "pf_launch_count", "pf_dualpipe_order", "pf_timing_enable", "pf_timing_read", "pf_score_static")
+           "pf_launch_count", "pf_dualpipe_order", "pf_timing_enable", "pf_timing_read", "pf_score_static", "pf_serve_plan_count", "pf_aggregate_workspace", "pf_aggregate_serving")
 STATIC_SCRATCH_BYTES = 4 << 20
-T_CLASSES = ("score", "topk", "select", "simulate")
+T_CLASSES = ("score", "topk", "select", "simulate", "aggregate")
 
 i32, u32, i64, u64, f32 = C.c_int32, C.c_uint32, C.c_int64, C.c_uint64, C.c_float
 
@@ -114,6 +114,12 @@ def load_library(path: str | None = None):
     L.pf_score.argtypes = [vp, u64, u64, vp, vp, vp, u32, vp, vp, vp, vp, sz, vp]
     L.pf_score_static.restype = C.c_int
     L.pf_score_static.argtypes = [vp, u64, u64, vp, vp, vp, u32, vp, vp, vp, vp]
+    L.pf_serve_plan_count.restype = u64
+    L.pf_serve_plan_count.argtypes = [vp]
+    L.pf_aggregate_workspace.restype = sz
+    L.pf_aggregate_workspace.argtypes = [vp, u32]
+    L.pf_aggregate_serving.restype = C.c_int
+    L.pf_aggregate_serving.argtypes = [vp, vp, vp, vp, vp, u32, vp, vp, vp, vp, sz, vp]
     L.pf_topk_merge.restype = C.c_int
     L.pf_topk_merge.argtypes = [u32, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
     L.pf_select_workspace.restype = sz
@@ -349,6 +355,31 @@ class Plan:
                                    _dptr(sim_status), k, _dptr(topk_idx), _dptr(topk_score), _dptr(topk_count),
                                    _dptr(workspace), workspace.numel(), _stream_ptr(torch, stream)), "pf_simulate")
         return dict(tput_sim=tput_sim, sim_status=sim_status, topk_idx=topk_idx, topk_score=topk_score,
+                    topk_count=topk_count, workspace=workspace)
+
+    # ---- pf_aggregate_serving
+    def serve_plan_count(self) -> int:
+        return int(self._L.pf_serve_plan_count(self._h))
+
+    def aggregate_serving(self, reason, tput, k: int = 0, plan_reason=None, plan_tput=None, topk_idx=None,
+                          topk_score=None, topk_count=None, workspace=None, stream=None):
+        """Enqueue pf_aggregate_serving on the dense outputs of a whole-space pf_score.  Does not synchronize."""
+        torch = _torch()
+        dev = self.device
+        n = self.serve_plan_count()
+        plan_reason = torch.empty(n, dtype=torch.uint8, device=dev) if plan_reason is None else plan_reason
+        plan_tput = torch.empty(n, dtype=torch.float32, device=dev) if plan_tput is None else plan_tput
+        if k > 0:
+            topk_idx = torch.empty(k, dtype=torch.int64, device=dev) if topk_idx is None else topk_idx
+            topk_score = torch.empty(k, dtype=torch.float32, device=dev) if topk_score is None else topk_score
+            topk_count = torch.empty(1, dtype=torch.int32, device=dev) if topk_count is None else topk_count
+        if workspace is None:
+            workspace = torch.empty(int(self._L.pf_aggregate_workspace(self._h, k)), dtype=torch.uint8, device=dev)
+        _check(self._L.pf_aggregate_serving(self._h, _dptr(reason), _dptr(tput), _dptr(plan_reason), _dptr(plan_tput),
+                                            k, _dptr(topk_idx), _dptr(topk_score), _dptr(topk_count),
+                                            _dptr(workspace), workspace.numel(), _stream_ptr(torch, stream)),
+               "pf_aggregate_serving")
+        return dict(plan_reason=plan_reason, plan_tput=plan_tput, topk_idx=topk_idx, topk_score=topk_score,
                     topk_count=topk_count, workspace=workspace)
 
     # ---- pf_search_host

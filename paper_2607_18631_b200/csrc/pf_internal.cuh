@@ -288,4 +288,16 @@ int launch_topk_reduce(void *d_workspace, const TopkLayout &lay, uint64_t n_keys
                        const uint64_t *d_idx_map, uint64_t *d_topk_idx, float *d_topk_score, uint32_t *d_topk_count,
                        cudaStream_t st, int *n_kernels);
 
+// host: top-k of a dense score array (entries with score <= 0 are skipped; ties go to the lower position).
+// The workspace is laid out by dense_topk_layout; idx_map as in launch_topk_reduce.
+struct DenseTopkLayout {
+    int blocks;
+    uint64_t keys_max;
+    TopkLayout tk;
+};
+DenseTopkLayout dense_topk_layout(int sm_count, uint64_t n, uint32_t k);
+int launch_dense_topk(const float *d_score, uint64_t n, const uint64_t *d_n, uint32_t k, const uint64_t *d_idx_map,
+                      void *d_workspace, const DenseTopkLayout &lay, uint64_t *d_topk_idx, float *d_topk_score,
+                      uint32_t *d_topk_count, cudaStream_t st, int *n_kernels);
+
 }  // namespace pf

@@ -648,11 +648,42 @@ __global__ void __launch_bounds__(kThreads) dense_topk_kernel(const DenseTopkArg
     tk_flush(s_buf, s_count, 0ull, s_base, A.keys, A.key_count);
 }
 
+DenseTopkLayout dense_topk_layout(int sm_count, uint64_t n, uint32_t k)
+{
+    DenseTopkLayout l;
+    const uint64_t nn = n ? n : 1, kk = k ? k : 1;
+    uint64_t tb = (n + kThreads - 1) / kThreads;
+    uint64_t cap = (uint64_t)sm_count * 2;
+    l.blocks = (int)(tb < 1 ? 1 : (tb > cap ? cap : tb));
+    l.keys_max = (uint64_t)l.blocks * kk;
+    if (l.keys_max > nn) l.keys_max = nn < kk ? kk : nn;
+    l.tk = topk_layout(l.keys_max, k);
+    return l;
+}
+
+int launch_dense_topk(const float *d_score, uint64_t n, const uint64_t *d_n, uint32_t k, const uint64_t *d_idx_map,
+                      void *d_workspace, const DenseTopkLayout &lay, uint64_t *d_topk_idx, float *d_topk_score,
+                      uint32_t *d_topk_count, cudaStream_t st, int *n_kernels)
+{
+    uint8_t *tws = (uint8_t *)d_workspace;
+    PF_CUDA_TRY(cudaMemsetAsync(tws + lay.tk.off_ctrl, 0, 256, st), "dense top-k: counter reset");
+    DenseTopkArgs t;
+    t.score = d_score; t.n = n; t.d_n = d_n; t.k = k;
+    t.keys = (unsigned long long *)(tws + lay.tk.off_keys_a);
+    t.key_count = (unsigned int *)(tws + lay.tk.off_ctrl) + 1;
+    dense_topk_kernel<<<lay.blocks, kThreads, 0, st>>>(t);
+    count_launch();
+    PF_CUDA_TRY(cudaGetLastError(), "dense_topk_kernel launch");
+    int nk = 0;
+    int rc = launch_topk_reduce(tws, lay.tk, lay.keys_max, k, 0, d_idx_map, d_topk_idx, d_topk_score, d_topk_count,
+                                st, &nk);
+    *n_kernels = nk + 1;
+    return rc;
+}
+
 struct SimLayout {
     size_t off_ctrl, off_bin_of, off_list, off_scores, off_topk, total;
-    int topk_blocks;
-    uint64_t topk_keys_max;
-    TopkLayout tk;
+    DenseTopkLayout dt;
 };
 
 static SimLayout sim_layout(const pf_plan_t *p, uint64_t n, uint32_t k)
@@ -664,13 +695,8 @@ static SimLayout sim_layout(const pf_plan_t *p, uint64_t n, uint32_t k)
     l.off_list = l.off_bin_of + ((nn + 255) & ~(size_t)255);
     l.off_scores = l.off_list + ((nn * 4 + 255) & ~(size_t)255);
     l.off_topk = l.off_scores + ((nn * 4 + 255) & ~(size_t)255);
-    uint64_t tb = (n + kThreads - 1) / kThreads;
-    uint64_t cap = (uint64_t)p->sm_count * 2;
-    l.topk_blocks = (int)(tb < 1 ? 1 : (tb > cap ? cap : tb));
-    l.topk_keys_max = (uint64_t)l.topk_blocks * (k ? k : 1);
-    if (l.topk_keys_max > nn) l.topk_keys_max = nn < (k ? k : 1) ? (k ? k : 1) : nn;
-    l.tk = topk_layout(l.topk_keys_max, k);
-    l.total = l.off_topk + (k ? l.tk.total : 0);
+    l.dt = dense_topk_layout(p->sm_count, n, k);
+    l.total = l.off_topk + (k ? l.dt.tk.total : 0);
     return l;
 }
 
@@ -785,20 +811,11 @@ extern "C" int pf_simulate(pf_plan_t *p, const uint64_t *d_surv_idx, uint64_t n,
         if (rc != PF_OK) return rc;
     }
     if (k > 0) {
-        uint8_t *tws = ws + lay.off_topk;
-        PF_CUDA_TRY(cudaMemsetAsync(tws + lay.tk.off_ctrl, 0, 256, st), "pf_simulate: top-k reset");
-        DenseTopkArgs t;
-        t.score = scores; t.n = n; t.d_n = d_n; t.k = k;
-        t.keys = (unsigned long long *)(tws + lay.tk.off_keys_a);
-        t.key_count = (unsigned int *)(tws + lay.tk.off_ctrl) + 1;
-        timing_begin(p, PF_T_TOPK, st);
-        dense_topk_kernel<<<lay.topk_blocks, kThreads, 0, st>>>(t);
-        count_launch();
-        PF_CUDA_TRY(cudaGetLastError(), "dense_topk_kernel launch");
         int nk = 0;
-        rc = launch_topk_reduce(tws, lay.tk, lay.topk_keys_max, k, 0, d_surv_idx, d_topk_idx, d_topk_score,
-                                d_topk_count, st, &nk);
-        timing_end(p, PF_T_TOPK, nk + 1, st);
+        timing_begin(p, PF_T_TOPK, st);
+        rc = launch_dense_topk(scores, n, d_n, k, d_surv_idx, ws + lay.off_topk, lay.dt, d_topk_idx, d_topk_score,
+                               d_topk_count, st, &nk);
+        timing_end(p, PF_T_TOPK, nk, st);
         return rc;
     }
     return PF_OK;
