@@ -229,3 +229,43 @@ def test_search_host_returns_the_same_results():
     np.testing.assert_array_equal(r2["topk_idx"], r["topk_idx"])
     np.testing.assert_array_equal(r2["sim_topk_idx"], r["sim_topk_idx"])
     plan.close()
+
+
+def test_one_million_survivors_sampled_parity():
+    """The simulator tier at its nominal size: with the memory gate lifted the unconstrained large space has
+    more than a million feasible plans, so select returns exactly 1e6 survivors.  The list is checked by its
+    invariants (ascending, feasible, none better left out) and 20,000 sampled simulations against the oracle."""
+    import torch
+    cfg = variant("large_unconstrained", cluster=dict(budget_bytes=10 ** 15))
+    plan, orc = _plan(cfg), Oracle(cfg)
+    out = plan.score(k=0)
+    sel = plan.select_survivors(out["reason"], out["tput"], 10 ** 6)
+    sim = plan.simulate(sel["surv_idx"], 10 ** 6, 4, k=100, d_n=sel["surv_count"])
+    torch.cuda.synchronize()
+    S = int(sel["surv_count"].item())
+    assert S == 10 ** 6
+    surv = sel["surv_idx"][:S].cpu().numpy().view(np.uint64)
+    assert np.all(np.diff(surv.astype(np.int64)) > 0)
+    reason = out["reason"].cpu().numpy()
+    tput = out["tput"].cpu().numpy()
+    assert np.all((reason[surv.astype(np.int64)] & 0x7F) == 0)
+    # nothing left out beats the worst survivor (the domain holds every feasible plan of this space)
+    taken = np.zeros(len(reason), dtype=bool)
+    taken[surv.astype(np.int64)] = True
+    feas = (reason & 0x7F) == 0
+    worst_in = tput[taken].min()
+    assert tput[feas & ~taken].max() <= worst_in
+    pick = np.sort(np.random.default_rng(0).choice(S, 20_000, replace=False))
+    ref, ref_st, _ = orc.simulate_list(surv[pick], 4, threads=64)
+    np.testing.assert_array_equal(sim["sim_status"][:S].cpu().numpy()[pick], ref_st)
+    np.testing.assert_allclose(sim["tput_sim"][:S].cpu().numpy()[pick], ref, rtol=TPUT_RTOL, atol=0)
+    # the re-ranked top-100 is sorted, drawn from the survivors, and consistent with the dense scores
+    k = int(sim["topk_count"].item())
+    assert k == 100
+    ti = sim["topk_idx"].cpu().numpy().view(np.uint64)[:k]
+    tsc = sim["topk_score"].cpu().numpy()[:k]
+    dense = sim["tput_sim"][:S].cpu().numpy()
+    order = np.lexsort((np.arange(S), -dense.astype(np.float64)))[:k]
+    np.testing.assert_array_equal(ti, surv[order])
+    np.testing.assert_array_equal(tsc, dense[order])
+    plan.close()
