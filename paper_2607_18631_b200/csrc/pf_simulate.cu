@@ -1,15 +1,19 @@
-// pf_simulate.cu -- simulator tier: one warp per survivor, one lane per pipeline rank (Sec. 3.2: the
+// pf_simulate.cu -- simulator tier: a group of lanes per survivor, one lane per pipeline rank (Sec. 3.2: the
 // list-scheduling timeline refines the schedules the closed form only approximates).
 //
 // Each lane walks its rank's fixed op order (1F1B and interleaved orders are generated on the fly from
-// counters; the DualPipe-style order comes from a host-built table) and computes
+// cursors; the DualPipe-style order comes from a host-built table) and computes
 //   end(op) = max(end of the rank's previous op, end(dependency) + latency) + duration.
 // A forward of stage q needs the forward of stage q-1 of the same microbatch, a backward of stage q needs
-// the backward of stage q+1; the op's own forward is already behind the lane's clock.  Within one stage,
-// forwards (and backwards) finish in microbatch order, so "is the dependency done" is a per-stage counter
-// compare and the end-time arrays in shared memory never need clearing.  Lanes advance in lock step with
-// __syncwarp between rounds; a round in which no lane advances ends the candidate with PF_SIM_STALL, so
-// the loop is bounded by the op count.
+// the backward of stage q+1; the op's own forward is already behind the lane's clock.
+//
+// Launch structure: a counting-sort pre-pass (classify, offsets, scatter) bins the survivors by
+// (timeline size class, lane-group width 8/16/32, schedule kind), then ONE simulate_kernel launch serves all
+// bins, largest timelines first.  Every warp owns a slice of the block's shared memory and runs its own
+// candidates there; the timeline is one signed 32-bit word per (stage stream, microbatch) -- 0 nothing
+// finished, +t forward ended at t, -t backward ended at t -- written by its owner lane and polled by the
+// neighbour.  No block barrier is used, and a warp whose lanes make no progress for 64 rounds reports its
+// unfinished candidates as PF_SIM_STALL, so every loop is bounded by the op count.
 #include <cstdlib>
 #include <cstring>
 #include <vector>
