@@ -18,6 +18,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "planfront_oracle.c")
 _HDR = os.path.join(_HERE, "planfront_oracle.h")
 _LIB = os.path.join(_HERE, "liborc.so")
+_LIB_COUNT = os.path.join(_HERE, "liborc_count.so")
 
 MAX_SCHED, MAX_KERN, NBUCKET, MAX_AXES = 8, 16, 8, 10
 
@@ -28,16 +29,22 @@ REASON_NAMES = {0: "FEASIBLE", 1: "WORLD", 2: "TP", 3: "EP", 4: "BATCH", 5: "VST
 i64, f64 = C.c_int64, C.c_double
 
 
-def build(force: bool = False) -> str:
-    """Compile the oracle with gcc (OpenMP for the range/list helpers).  Returns the .so path."""
-    if not force and os.path.exists(_LIB):
+def build(force: bool = False, count_ops: bool = False) -> str:
+    """Compile the oracle with gcc (OpenMP for the range/list helpers).  Returns the .so path.
+
+    `count_ops=True` makes the operation-tallying build (-DORACLE_COUNT_OPS, liborc_count.so): same results,
+    plus per-candidate integer/floating operation counts for an ALU roofline."""
+    out = _LIB_COUNT if count_ops else _LIB
+    if not force and os.path.exists(out):
         newest = max(os.path.getmtime(_SRC), os.path.getmtime(_HDR))
-        if os.path.getmtime(_LIB) >= newest:
-            return _LIB
-    cmd = ["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-fopenmp", "-ffp-contract=off", "-Wall", "-Wextra",
-           "-o", _LIB, _SRC, "-lm"]
+        if os.path.getmtime(out) >= newest:
+            return out
+    cmd = ["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-fopenmp", "-ffp-contract=off", "-Wall", "-Wextra"]
+    if count_ops:
+        cmd.append("-DORACLE_COUNT_OPS")
+    cmd += ["-o", out, _SRC, "-lm"]
     subprocess.run(cmd, check=True, cwd=_HERE)
-    return _LIB
+    return out
 
 
 class Model(C.Structure):
@@ -148,6 +155,36 @@ def lib():
         L.orc_simulate_list.argtypes = [PP, C.c_void_p, u64, u32, C.c_void_p, C.c_void_p, C.c_int]
         del u8p
     return _lib
+
+
+_lib_count = None
+
+
+def count_ops(oracle: "Oracle", first: int = 0, count: int | None = None, threads: int = 1) -> dict:
+    """Run the operation-tallying build over [first, first+count) of `oracle`'s space.
+
+    Returns {"int_ops", "fp_ops", "candidates"} (totals); the reasons it computes are checked against nothing
+    here -- the tally build differs from the plain one only by its counters."""
+    global _lib_count
+    if _lib_count is None:
+        _lib_count = C.CDLL(build(count_ops=True))
+        _lib_count.orc_score_range.restype = C.c_int
+        _lib_count.orc_score_range.argtypes = [C.POINTER(Problem), C.c_uint64, C.c_uint64, C.c_void_p, C.c_void_p,
+                                               C.c_void_p, C.c_int]
+        _lib_count.orc_ops_enabled.restype = C.c_int
+        _lib_count.orc_ops_reset.restype = None
+        _lib_count.orc_ops_read.restype = None
+        _lib_count.orc_ops_read.argtypes = [C.POINTER(i64 * 3)]
+    L = _lib_count
+    if not L.orc_ops_enabled():
+        raise RuntimeError("liborc_count.so was not built with -DORACLE_COUNT_OPS")
+    if count is None:
+        count = oracle.size - first
+    L.orc_ops_reset()
+    L.orc_score_range(C.byref(oracle.pb), first, count, None, None, None, threads)
+    out = (i64 * 3)()
+    L.orc_ops_read(C.byref(out))
+    return {"int_ops": int(out[0]), "fp_ops": int(out[1]), "candidates": int(out[2])}
 
 
 def _ptr(a: np.ndarray):

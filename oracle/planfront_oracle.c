@@ -15,6 +15,47 @@
 #include <omp.h>
 #endif
 
+/* ------------------------------------------------------------------ op tally (-DORACLE_COUNT_OPS)
+ *
+ * The counting build charges, block by block, the arithmetic, comparison and logic operators that
+ * the definition writes out (loads, stores and assignments are free; a ceil-division is 3 integer
+ * ops, a highest-set-bit search 4).  A block's operators are charged when control reaches it, so a
+ * candidate rejected by rule r pays for decode and rules 1..r only.  The totals give the
+ * algorithmic operation count per candidate for an ALU roofline; they change no result. */
+#ifdef ORACLE_COUNT_OPS
+static _Thread_local int64_t tl_ops_i, tl_ops_f, tl_ops_n;
+static int64_t g_ops_i, g_ops_f, g_ops_n;
+#define OPS(i, f) (tl_ops_i += (i), tl_ops_f += (f))
+#else
+#define OPS(i, f) ((void)0)
+#endif
+
+int orc_ops_enabled(void)
+{
+#ifdef ORACLE_COUNT_OPS
+    return 1;
+#else
+    return 0;
+#endif
+}
+
+void orc_ops_reset(void)
+{
+#ifdef ORACLE_COUNT_OPS
+    g_ops_i = g_ops_f = g_ops_n = 0;
+#endif
+}
+
+/* out[0] integer ops, out[1] floating ops, out[2] candidates evaluated since the last reset */
+void orc_ops_read(int64_t out[3])
+{
+#ifdef ORACLE_COUNT_OPS
+    out[0] = g_ops_i; out[1] = g_ops_f; out[2] = g_ops_n;
+#else
+    out[0] = out[1] = out[2] = 0;
+#endif
+}
+
 /* ------------------------------------------------------------------ helpers */
 
 static int64_t cdiv(int64_t a, int64_t b) { return (a + b - 1) / b; }
@@ -108,6 +149,7 @@ uint64_t orc_space_size(const orc_problem_t *pb)
 static void decode(const orc_axes_t *ax, uint64_t idx, int64_t *value)
 {
     uint64_t rem = idx;
+    OPS(2 * ax->n_axes, 0); /* one mod and one div per axis */
     for (int a = 0; a < ax->n_axes; a++) {
         uint64_t n = (uint64_t)ax->len[a];
         uint64_t digit = rem % n;
@@ -164,6 +206,7 @@ static int eval_train(const orc_problem_t *pb, const orc_derived_t *dv, uint64_t
 
     /* rule 1 WORLD: data parallelism is derived from the world size (Sec. 3.1) unless both are
      * enumerated, in which case the product must match; whole nodes beyond one node */
+    OPS(dp == 0 ? 15 : 10, 0);
     if (dp == 0) {
         if (world % (tp * pp) != 0) return o->reason = ORC_R_WORLD;
         dp = world / (tp * pp);
@@ -175,11 +218,13 @@ static int eval_train(const orc_problem_t *pb, const orc_derived_t *dv, uint64_t
     if (world > C->G && world % C->G != 0) return o->reason = ORC_R_WORLD;
 
     /* rule 2 TP: tensor degrees over the head-divisible subset (Sec. 3.3) */
+    OPS(10, 0);
     if (tp > R->tp_max || tp > C->G || M->nh % tp != 0) return o->reason = ORC_R_TP;
     if (M->S > 0 && M->Fs % tp != 0) return o->reason = ORC_R_TP;
     if (R->ep_scope == 0 && M->F % tp != 0) return o->reason = ORC_R_TP;
 
     /* rule 3 EP: expert degrees over the admissible divisors; EP inside DP (Sec. 4) or inside DP*TP */
+    OPS(R->ep_scope ? 6 : 5, 0);
     if (M->E % ep != 0) return o->reason = ORC_R_EP;
     if (R->ep_scope == 0) {
         if (dp % ep != 0) return o->reason = ORC_R_EP;
@@ -188,8 +233,10 @@ static int eval_train(const orc_problem_t *pb, const orc_derived_t *dv, uint64_t
     }
 
     /* rule 4 BATCH */
+    OPS(3, 0);
     if (pb->workload.gbs % (dp * mb) != 0) return o->reason = ORC_R_BATCH;
 
+    OPS(6 + 3, 0); /* derived integers, then rule 5 */
     int64_t kind = pb->sched[s].kind, ov = pb->sched[s].overlap;
     int64_t v_eff = (v == 0) ? (kind == ORC_KIND_INTERLEAVED ? 2 : 1) : v;
     int64_t m = pb->workload.gbs / (dp * mb);
@@ -205,6 +252,7 @@ static int eval_train(const orc_problem_t *pb, const orc_derived_t *dv, uint64_t
     }
 
     /* rule 6 LAYERS: layer count vs pipeline depth (Fig. 2: 27 mod pp*v != 0) */
+    OPS(3 + 4, 0); /* the rule, then Lc and Ls */
     if (R->layer_mode == 0) {
         if (M->L % Q != 0) return o->reason = ORC_R_LAYERS;
     } else {
@@ -215,6 +263,7 @@ static int eval_train(const orc_problem_t *pb, const orc_derived_t *dv, uint64_t
     o->Lc = Lc; o->Ls = Ls;
 
     /* rule 7 MICROBATCH: what each static schedule order needs to be well formed */
+    OPS(kind == ORC_KIND_1F1B ? 2 : kind == ORC_KIND_INTERLEAVED ? 3 : 8, 0);
     if (kind == ORC_KIND_INTERLEAVED) {
         if (m % pp != 0) return o->reason = ORC_R_MICROBATCH;
     } else if (kind == ORC_KIND_DUALPIPE) {
@@ -224,6 +273,7 @@ static int eval_train(const orc_problem_t *pb, const orc_derived_t *dv, uint64_t
 
     /* rule 8 KERNEL_MISSING: variant needs a capability the cluster lacks, or the autotune
      * report has no entry at this expert shape (Sec. 3.3 kernel tier) */
+    OPS(5 + 4 + 4 + 6, 0); /* group sizes, m_e, its bucket, the two table tests */
     int64_t tps = R->ep_scope ? tp : 1;
     int64_t etp = R->ep_scope ? 1 : tp;
     int64_t edp = R->ep_scope ? dp * tp / ep : dp / ep;
@@ -235,6 +285,7 @@ static int eval_train(const orc_problem_t *pb, const orc_derived_t *dv, uint64_t
     if (((kn->avail_mask >> b) & 1) == 0) return o->reason = ORC_R_KERNEL_MISSING;
 
     /* rules 9, 10: the emit dry-run (Sec. 4 "Emitters"); skipped in unconstrained mode (Sec. 3.3) */
+    OPS(R->enforce_realizability ? 8 : 1, 0);
     if (R->enforce_realizability) {
         if (!pb->sched[s].mapped) return o->reason = ORC_R_UNMAPPED_SCHEDULE;
         if (ov && (rec == ORC_REC_FULL || (kind == ORC_KIND_1F1B && pp > 1)))
@@ -242,6 +293,10 @@ static int eval_train(const orc_problem_t *pb, const orc_derived_t *dv, uint64_t
     }
 
     /* ---- memory (bytes on rank 0, which holds the most in-flight activations) ---- */
+    OPS(3 + 6 + 7 + 7 + 4 + 9 + 2 + 4 + 6 + 1 + 5, 0); /* pm, emb, N_dense, N_exp, w+g, o, A_tok, A_layer, units,
+                                                          bytes_a, sum and gate */
+    if (rec == ORC_REC_FULL) OPS(6, 0);
+    if ((pp == 1 || kind == ORC_KIND_DUALPIPE) && M->count_embeddings) OPS(9, 0);
     int64_t pm = (kind == ORC_KIND_DUALPIPE && pp > 1) ? 2 : 1; /* two stage copies per rank */
     int64_t emb = cdiv(dv->P_emb, tp) * ((pp == 1 || kind == ORC_KIND_DUALPIPE) ? 2 : 1);
     int64_t N_dense = pm * Ls * (cdiv(dv->P_dl, tp) + dv->P_rt) + emb;
@@ -275,6 +330,10 @@ static int eval_train(const orc_problem_t *pb, const orc_derived_t *dv, uint64_t
     if (mem > C->budget_bytes) return o->reason = ORC_R_MEMORY;
 
     /* ---- analytic step time ---- */
+    /* compute 4+5+1+1, recompute <= 7, TP all-reduce 10 (+6 int), all-to-all 8 (+4 int), exposure 7,
+     * per-layer sums 8, head 4, stage sums 7, p2p <= 4 (+2 int), closed form <= 10 (+4 int),
+     * gradient all-reduces 20 (+12 int), optimizer 2, step 5, throughput and prices 7 (+3 int), flag 2 int */
+    OPS(6 + 4 + 2 + 4 + 12 + 3 + 2, 4 + 5 + 1 + 1 + 7 + 10 + 8 + 7 + 8 + 4 + 7 + 4 + 10 + 20 + 2 + 5 + 7);
     double td = (double)t, tpd = (double)tp;
     double peak = C->peak_flops;
     double cD = td * (double)dv->f_dense / (tpd * peak * K0->eff_dense);
@@ -349,6 +408,7 @@ static int eval_serve(const orc_problem_t *pb, const orc_derived_t *dv, uint64_t
 
     /* rule 1 WORLD: dp-attention needs dp == ep with the real world size (Sec. 2.1, boundary B5);
      * without it experts shard inside the tensor-parallel world, ep*moe_dp == tp (Sec. 4) */
+    OPS(2 + 4, 0);
     if (world % tp != 0) return o->reason = ORC_R_WORLD;
     if (dpa) {
         if (world / tp != ep || ep < 2) return o->reason = ORC_R_WORLD;
@@ -356,16 +416,20 @@ static int eval_serve(const orc_problem_t *pb, const orc_derived_t *dv, uint64_t
         if (tp % ep != 0) return o->reason = ORC_R_WORLD;
     }
     /* rule 2 TP */
+    OPS(4 + 3, 0); /* the rule, then engine sizes */
     if (tp > C->G || M->nh % tp != 0) return o->reason = ORC_R_TP;
     int64_t n_eng = dpa ? tp * ep : tp;
     int64_t moe_tp = n_eng / ep;
     /* rule 3 EP */
+    OPS(5, 0);
     if (M->E % ep != 0 || M->F % moe_tp != 0) return o->reason = ORC_R_EP;
     /* rule 4 BATCH */
+    OPS(3 + 1, 0);
     if (dpa && Bd % ep != 0) return o->reason = ORC_R_BATCH;
     int64_t b_loc = dpa ? Bd / ep : Bd;
 
     /* rule 8 KERNEL_MISSING: decode and prefill expert shapes both need an entry */
+    OPS(4 + 8 + 3 + 7, 0); /* two shapes, two buckets, capability test, two table tests */
     int64_t m_e = (Bd * M->K) / M->E;
     int64_t m_ep = (Cc * M->K) / M->E;
     int b = me_bucket(m_e), b_pre = me_bucket(m_ep);
@@ -376,6 +440,7 @@ static int eval_serve(const orc_problem_t *pb, const orc_derived_t *dv, uint64_t
         return o->reason = ORC_R_KERNEL_MISSING;
 
     /* ---- memory: weights + KV cache + prefill activation workspace ---- */
+    OPS(19 + 6 + 5 + 3 + 3 + 1, 0); /* weights, KV bytes per token, cache, workspace, sum, gate */
     int64_t w = M->L * (cdiv(dv->P_dl, tp) * M->wb + dv->P_rt * M->wb +
                         (M->E / ep) * cdiv(dv->P_e, moe_tp) * kn->wbytes) +
                 2 * cdiv(M->vocab * M->H, tp) * M->wb;
@@ -388,6 +453,10 @@ static int eval_serve(const orc_problem_t *pb, const orc_derived_t *dv, uint64_t
     if (mem > C->budget_bytes) return o->reason = ORC_R_MEMORY;
 
     /* ---- time: per-layer max(compute, HBM) + collectives; decode at mean context ---- */
+    /* decode step: context and weight terms 9, experts touched 5, attention 14, experts 8, collective <= 11,
+     * layer sum 4; prefill: chunking 2 (+3 int), experts touched 6, attention 13, experts 8, collective <= 11,
+     * sum 5; throughput and price 8, flag 2 int; plus ~10 int in operand products and collective shapes */
+    OPS(1 + 3 + 2 + 10, 9 + 5 + 14 + 8 + 11 + 4 + 2 + 6 + 13 + 8 + 11 + 5 + 8);
     link_t lk = link_of(C, n_eng);
     double peak = C->peak_flops, hbm = C->hbm_bw, effd = K0->eff_dense;
     double tpd = (double)tp, nen = (double)n_eng, bl = (double)b_loc, dk = (double)dv->dk;
@@ -427,7 +496,7 @@ static int eval_serve(const orc_problem_t *pb, const orc_derived_t *dv, uint64_t
     return o->reason = reason;
 }
 
-int orc_eval(const orc_problem_t *pb, uint64_t idx, orc_detail_t *detail)
+static int eval_one(const orc_problem_t *pb, uint64_t idx, orc_detail_t *detail)
 {
     orc_detail_t local;
     orc_derived_t dv;
@@ -436,6 +505,27 @@ int orc_eval(const orc_problem_t *pb, uint64_t idx, orc_detail_t *detail)
     orc_derive(&pb->model, &dv);
     int r = pb->workload.phase == 0 ? eval_train(pb, &dv, idx, detail) : eval_serve(pb, &dv, idx, detail);
     if ((r & 0x7f) != 0) detail->tput = 0.0;
+#ifdef ORACLE_COUNT_OPS
+    tl_ops_n++;
+#endif
+    return r;
+}
+
+/* add the calling thread's tally to the totals */
+static void ops_fold(void)
+{
+#ifdef ORACLE_COUNT_OPS
+    __atomic_fetch_add(&g_ops_i, tl_ops_i, __ATOMIC_RELAXED);
+    __atomic_fetch_add(&g_ops_f, tl_ops_f, __ATOMIC_RELAXED);
+    __atomic_fetch_add(&g_ops_n, tl_ops_n, __ATOMIC_RELAXED);
+    tl_ops_i = tl_ops_f = tl_ops_n = 0;
+#endif
+}
+
+int orc_eval(const orc_problem_t *pb, uint64_t idx, orc_detail_t *detail)
+{
+    int r = eval_one(pb, idx, detail);
+    ops_fold();
     return r;
 }
 
@@ -452,20 +542,22 @@ int orc_score_range(const orc_problem_t *pb, uint64_t first, uint64_t count, uin
 #pragma omp for schedule(static)
         for (int64_t i = 0; i < (int64_t)count; i++) {
             orc_detail_t d;
-            int r = orc_eval(pb, first + (uint64_t)i, &d);
+            int r = eval_one(pb, first + (uint64_t)i, &d);
             if (reason) reason[i] = (uint8_t)r;
             if (tput) tput[i] = d.tput;
             if (mem) mem[i] = d.mem;
         }
+        ops_fold();
     }
 #else
     for (uint64_t i = 0; i < count; i++) {
         orc_detail_t d;
-        int r = orc_eval(pb, first + i, &d);
+        int r = eval_one(pb, first + i, &d);
         if (reason) reason[i] = (uint8_t)r;
         if (tput) tput[i] = d.tput;
         if (mem) mem[i] = d.mem;
     }
+    ops_fold();
 #endif
     return used;
 }

@@ -164,6 +164,12 @@ int64_t orc_budget_bytes(int64_t hbm_bytes); /* floor(0.9 * capacity), in intege
 void orc_derive(const orc_model_t *m, orc_derived_t *d);
 uint64_t orc_space_size(const orc_problem_t *pb);
 
+/* Operation tally for the ALU roofline.  Only a build with -DORACLE_COUNT_OPS counts; the plain build
+ * returns zeros.  out[0] integer ops, out[1] floating ops, out[2] candidates, since the last reset. */
+int orc_ops_enabled(void);
+void orc_ops_reset(void);
+void orc_ops_read(int64_t out[3]);
+
 /* score one candidate: fills detail (may be NULL); returns the reason byte */
 int orc_eval(const orc_problem_t *pb, uint64_t idx, orc_detail_t *detail);
 

@@ -526,3 +526,30 @@ def test_serving_plan_is_infeasible_if_any_scenario_is():
     assert (any_bad & ~all_bad).sum() > 0                      # mixed plans exist in this space
     np.testing.assert_array_equal((pr & 0x7F) != 0, any_bad)
     assert np.all(pt[any_bad] == 0) and np.all(pt[~any_bad] > 0)
+
+
+# --------------------------------------------------------------------------- operation tally (counting build)
+
+def test_operation_tally_charges_by_how_far_a_candidate_gets():
+    """Hand counts: a candidate rejected by the first rule pays the decode (one mod and one div per axis) and
+    that rule's ten integer operators (fifteen when dp is derived from the world size), nothing else; a feasible candidate pays for every block, floating part
+    included; the tally build computes the same reasons as the plain build."""
+    cfg = make_config("tiny")
+    orc = Oracle(cfg)
+    reason, _, _, _ = orc.score_range(0, orc.size)
+    n_axes = len(cfg["axes"])
+    rule1 = 15 if list(dict(cfg["axes"])["dp"]) == [0] else 10
+    first_rule = [i for i in range(orc.size) if reason[i] == 1]
+    feasible = [i for i in range(orc.size) if (reason[i] & 0x7F) == 0]
+    assert first_rule and feasible
+    c = oracle.count_ops(orc, first_rule[0], 1)
+    assert c == {"int_ops": 2 * n_axes + rule1, "fp_ops": 0, "candidates": 1}
+    c = oracle.count_ops(orc, feasible[0], 1)
+    assert c["fp_ops"] == 110 and c["int_ops"] > 150 and c["candidates"] == 1
+    # totals add up candidate by candidate and do not depend on the thread count
+    whole = oracle.count_ops(orc, 0, orc.size, threads=1)
+    assert whole == oracle.count_ops(orc, 0, orc.size, threads=4)
+    assert whole["candidates"] == orc.size
+    assert whole["fp_ops"] == 110 * len(feasible)
+    parts = [oracle.count_ops(orc, i, 1)["int_ops"] for i in range(0, orc.size, 7)]
+    assert min(parts) >= 2 * n_axes + rule1
