@@ -169,6 +169,56 @@ def run_reference(args):
 
 # --------------------------------------------------------------------------------------------- CUDA side
 
+def _time_launches(torch, stream, fn, reps=5, warm=2):
+    """Average device time (ms) of fn() over `reps` launches on `stream`, after `warm` untimed ones."""
+    for _ in range(warm):
+        fn()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    a.record(stream)
+    for _ in range(reps):
+        fn()
+    b.record(stream)
+    torch.cuda.synchronize()
+    return a.elapsed_time(b) / reps
+
+
+def _probe_peaks(torch, binding, stream, big):
+    """Issue-rate peaks (thread-instructions/s) per instruction kind and the pure streaming-write rate (GB/s),
+    measured with the library's probe kernels; `big` is a device buffer far larger than L2."""
+    sink = torch.zeros(1, dtype=torch.int32, device=big.device)
+    out = {}
+    for kind in ("ffma", "imad", "logic"):
+        n = [0]
+
+        def go():
+            n[0] = binding.pf_probe_alu(kind, 8192, sink)
+        ms = _time_launches(torch, stream, go)
+        out[kind] = n[0] / (ms * 1e-3)
+    nbytes = big.numel() * big.element_size()
+    ms = _time_launches(torch, stream, lambda: binding.pf_probe_write(big))
+    return out, nbytes / (ms * 1e-3) / 1e9
+
+
+def _simulated_ops(plan, cfg, surv_host):
+    """Ops the schedule simulator evaluates for these survivors: 2 * (simulated microbatches) * (virtual
+    stages) each, with the 64-microbatch window (for an interleaved schedule, a multiple of pp)."""
+    gbs = int(cfg["workload"]["gbs"])
+    total = 0
+    for idx in surv_host:
+        t = plan.decode(int(idx))
+        kind = int(cfg["sched"][t["sched"]]["kind"])
+        dp = t["dp"] if t["dp"] else t["world"] // (t["tp"] * t["pp"])
+        m = gbs // (dp * t["mb"])
+        v_eff = t["v"] if t["v"] else (2 if kind == 1 else 1)
+        m_sim = min(m, 64)
+        if kind == 1:
+            m_sim = m if m <= 64 else (64 // t["pp"]) * t["pp"]
+        q = t["pp"] * (v_eff if kind == 1 else 1)
+        total += 2 * m_sim * q
+    return total
+
+
 def run_ours(args):
     import torch
     from paper_2607_18631_b200 import Plan, binding
@@ -281,6 +331,27 @@ def run_ours(args):
             dist.destroy_process_group()
         return
 
+    # ---- side measurements (single-GPU runs): top-k-only mode, the probes behind the two rooflines, the
+    # simulator's own rates
+    extra = {}
+    if world == 1 and not args.no_report:
+        ms_topk_only = _time_launches(
+            torch, stream, lambda: plan.score(0, N, K_TOP, topk_idx=tk_idx, topk_score=tk_sc, topk_count=tk_cnt,
+                                              workspace=ws_score, stream=stream, dense=False), reps=10, warm=3)
+        extra["topk_only"] = {"ms_per_launch": ms_topk_only, "value": N / (ms_topk_only * 1e-3), "unit": UNIT,
+                              "note": "dense outputs not written (NULL): rules + cost + top-1024 only"}
+        peaks, write_gbs = _probe_peaks(torch, binding, stream, mem)
+        step()                                   # the write probe overwrote `mem`: restore the step's outputs
+        torch.cuda.synchronize()
+        n_feas = int(((reason & 0x7F) == 0).sum().item())
+        sim_ms = per_class["simulate"][0] / args.steps
+        sim_ops = _simulated_ops(plan, cfg, surv[:n_surv].cpu().numpy())
+        extra["simulator"] = {"survivors": n_surv, "ms_per_launch": sim_ms,
+                              "survivors_per_s": n_surv / (sim_ms * 1e-3), "simulated_ops": sim_ops,
+                              "simulated_ops_per_s": sim_ops / (sim_ms * 1e-3)}
+        extra["probes"] = {"thread_inst_per_s": peaks, "stream_write_gbs": write_gbs, "feasible": n_feas,
+                           "feasible_fraction": n_feas / N}
+
     # ---- roofline of the dominant kernel class
     dom = max(per_class, key=lambda c: per_class[c][0])
     hbm, how = _measured_hbm()
@@ -303,9 +374,27 @@ def run_ours(args):
         t0 = time.perf_counter()
         scored = oracle_step(orc, threads, 1)
         dt = time.perf_counter() - t0
+        t1 = time.perf_counter()
+        orc.score_range(60_000_000, 2_457_600, threads=1)
+        single = 2_457_600 / (time.perf_counter() - t1)
         cpu_baseline = {"value": scored / dt, "unit": UNIT, "cores": used, "kind": "oracle",
                         "sample": f"one whole step (all {scored:,} candidates + {n_surv:,} simulated survivors), "
-                                  f"{dt:.1f} s"}
+                                  f"{dt:.1f} s",
+                        "single_thread_value": single,
+                        "single_thread_sample": "scoring only, candidates [60,000,000, 62,457,600)"}
+        if "probes" in extra:
+            # ALU-side roofline: the oracle's operation tally (its counting build) over the whole space against
+            # the measured issue rates; integer ops are charged at the slower of the two integer kinds
+            ops = oracle.count_ops(orc, 0, N, threads=threads)
+            pk = extra["probes"]["thread_inst_per_s"]
+            i_per, f_per = ops["int_ops"] / ops["candidates"], ops["fp_ops"] / ops["candidates"]
+            t_alu = N * (i_per / min(pk["imad"], pk["logic"]) + f_per / pk["ffma"])
+            t_hbm = N * BYTES_PER_CANDIDATE / (hbm * 1e9)
+            extra["alu_roofline"] = {"int_ops_per_candidate": i_per, "fp_ops_per_candidate": f_per,
+                                     "ops_source": "oracle operation tally, every candidate of the space",
+                                     "t_alu_ms": t_alu * 1e3, "t_hbm_ms": t_hbm * 1e3,
+                                     "bound": "hbm" if t_hbm >= t_alu else "alu",
+                                     "achieved_over_alu_peak": t_alu / (score_ms * 1e-3)}
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
@@ -318,6 +407,7 @@ def run_ours(args):
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "steps": e2e_steps},
             "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu_baseline}
+    line.update(extra)
     print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
@@ -330,6 +420,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", choices=("ours", "reference"), default="ours")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing leg")
+    ap.add_argument("--no-report", action="store_true", help="skip the side measurements (probes, top-k-only)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

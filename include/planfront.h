@@ -313,6 +313,23 @@ int pf_timing_read(pf_plan_t *plan, float *ms, uint32_t *kernels);
 /* Number of kernels this library has launched in this process (for launch accounting in benchmarks). */
 uint64_t pf_launch_count(void);
 
+/* Roofline probes (measurement utilities; the paper has no counterpart and no scoring call uses them).
+ * The caller times them with events on `stream`; neither call synchronises or allocates.
+ *
+ * pf_probe_alu: one launch at full occupancy (8 blocks of 256 threads per SM) in which every thread runs
+ * 8 independent dependency chains of one instruction kind for `iters` loop trips of 4 steps each:
+ * PF_PROBE_FFMA fp32 fused multiply-add, PF_PROBE_IMAD 32-bit integer multiply-add, PF_PROBE_LOGIC an
+ * alternation of 3-input logic ops and 32-bit adds.  *h_thread_instructions (host) receives the number of
+ * thread-level instructions of that kind the launch executes; dividing by the launch's duration gives the
+ * issue-rate peak for that kind.  d_sink: 4 device bytes, practically never written.  1 <= iters <= 2^24.
+ *
+ * pf_probe_write: fills `bytes` (a multiple of 16, 16-byte aligned device buffer) with 16-byte streaming
+ * stores, the store the scoring kernel uses for its dense outputs; bytes / duration is the write rate.
+ * Errors: PF_EINVAL for a null pointer, a bad kind, iters or size; PF_ECUDA if the launch fails. */
+enum { PF_PROBE_FFMA = 0, PF_PROBE_IMAD = 1, PF_PROBE_LOGIC = 2 };
+int pf_probe_alu(int kind, uint32_t iters, uint32_t *d_sink, uint64_t *h_thread_instructions, void *stream);
+int pf_probe_write(void *d_buf, size_t bytes, void *stream);
+
 #ifdef __cplusplus
 }
 #endif
