@@ -13,6 +13,9 @@ constexpr int kThreads = 256;        // threads per block of the scoring kernel
 constexpr int kTopkCap = 2048;       // shared-memory candidate buffer per block (2 * PF_K_MAX)
 constexpr uint32_t kSlabMax = 16384; // upper bound on candidates per slab (inner-axis product)
 constexpr int kInnerVals = 1024;     // inner-axis values the scoring kernel keeps in shared memory
+constexpr int kOrderMaxSlabs = 1 << 20;  // calls with more slabs visit them by a permutation instead of an order table
+constexpr int kTailFillsPerBlock = 4;    // constant-fill slabs per block kept for the end of the visiting order
+constexpr int kQueueCap = 4096;   // cost-model queue of the scoring kernel (entries), drained when it may fill up
 
 struct DevSched {
     int kind, overlap, mapped;

@@ -29,6 +29,7 @@ struct ScoreArgs {
     unsigned int *slab_counter;     // zeroed before launch
     const int32_t *vals;            // packed axis value lists
     const int32_t *scen;            // serve: P[n_scen], O[n_scen]
+    const uint32_t *order;          // ticket -> (pre_reason << 24) | slab, or NULL: visit by slab_mul, classify here
 };
 
 struct SlabInfo {
@@ -36,6 +37,99 @@ struct SlabInfo {
     int pre_reason;                 // != 0: every candidate of the slab fails this rule
     int outer[PF_MAX_AXES];         // values of the outer axes (entries [n_inner, n_axes))
 };
+
+// Values of a slab's outer axes and, on request, the first failing rule among those that depend on the outer
+// axes alone (0: the slab has to be evaluated candidate by candidate).
+template <typename RI>
+__device__ __forceinline__ int slab_outer_axes(const DevPlan &P, const int32_t *vals, uint64_t slab_abs,
+                                               int (&outer)[PF_MAX_AXES], bool classify)
+{
+    uint64_t o = slab_abs;
+    for (int a = P.n_inner; a < P.n_axes; a++) {
+        uint64_t r = P.radix[a];
+        uint64_t q = o / r;
+        outer[a] = __ldg(vals + P.val_off[a] + (int)(o - q * r));
+        o = q;
+    }
+    if (!classify || P.n_pre_rules <= 0) return 0;
+    if (P.phase == PF_PHASE_TRAIN) {
+        TrainTuple c;
+        c.mb = P.n_inner <= 3 ? outer[3] : 1;
+        c.ep = P.n_inner <= 5 ? outer[5] : 1;
+        c.pp = outer[6]; c.tp = outer[7]; c.dp = outer[8]; c.world = outer[9];
+        RI dp, world;
+        int r = train_layout_rules<RI>(P, c, 1, P.n_pre_rules < 3 ? P.n_pre_rules : 3, dp, world);
+        if (r == 0 && P.n_pre_rules >= 4) {
+            RI dpmb = dp * (RI)c.mb;
+            if (((RI)P.gbs) % dpmb != 0) r = PF_R_BATCH;
+        }
+        return r;
+    }
+    ServeTuple c;
+    c.batch = P.n_inner <= 2 ? outer[2] : 1;
+    c.dpa = outer[3]; c.ep = outer[4]; c.tp = outer[5];
+    return serve_layout_rules<RI>(P, c, 1, P.n_pre_rules >= 4);
+}
+
+// Visiting order of a call's slabs.  A slab that has to be evaluated takes several times as long as one that is
+// filled with a constant, so the evaluated ones go first, spread evenly between the filled ones (their
+// arithmetic then runs under the other blocks' store traffic), and the last tickets are all fills: the kernel's
+// tail is one short slab long.
+//
+// Step 1, one thread per slab: the slab's class (its pre_reason byte).
+template <typename RI>
+__global__ void __launch_bounds__(256) slab_class_kernel(const __grid_constant__ DevPlan P, const int32_t *vals,
+                                                         uint64_t slab_lo, uint32_t n_slabs, uint8_t *cls)
+{
+    const uint32_t s = blockIdx.x * blockDim.x + threadIdx.x;
+    if (s >= n_slabs) return;
+    int outer[PF_MAX_AXES];
+    cls[s] = (uint8_t)slab_outer_axes<RI>(P, vals, slab_lo + s, outer, true);
+}
+
+// Step 2, one block: ranks within each class by a block-wide scan over per-thread chunks, then every slab's
+// ticket in closed form.  With H evaluated and F filled slabs, the last min(F, tail) fills form the tail and
+// the other Fs fills are interleaved: evaluated slab i sits after floor(i * Fs / H) fills, fill j after
+// min(H, ceil((j + 1) * H / Fs)) evaluated slabs.
+__global__ void __launch_bounds__(1024) slab_order_kernel(const uint8_t *cls, uint32_t n_slabs, uint32_t tail,
+                                                          uint32_t *order)
+{
+    __shared__ uint32_t s_part[1024];
+    const uint32_t tid = threadIdx.x;
+    const uint32_t chunk = (n_slabs + 1023u) / 1024u;
+    const uint32_t lo = min(tid * chunk, n_slabs), hi = min(lo + chunk, n_slabs);
+    uint32_t h = 0;
+    for (uint32_t s = lo; s < hi; s++) h += cls[s] == 0;
+    s_part[tid] = h;
+    __syncthreads();
+    for (uint32_t d = 1; d < 1024u; d <<= 1) {  // inclusive scan
+        const uint32_t v = tid >= d ? s_part[tid - d] : 0u;
+        __syncthreads();
+        s_part[tid] += v;
+        __syncthreads();
+    }
+    const uint64_t H = s_part[1023], F = n_slabs - H;
+    const uint64_t Fs = F > tail ? F - tail : 0;
+    uint64_t hi_rank = s_part[tid] - h;        // evaluated slabs before this chunk
+    uint64_t fi_rank = lo - hi_rank;           // filled slabs before this chunk
+    for (uint32_t s = lo; s < hi; s++) {
+        const uint32_t c = cls[s];
+        uint64_t pos;
+        if (c == 0) {
+            pos = hi_rank + (H ? hi_rank * Fs / H : 0);
+            hi_rank++;
+        } else {
+            if (fi_rank < Fs) {
+                uint64_t before = ((fi_rank + 1) * H + Fs - 1) / Fs;
+                pos = fi_rank + (before < H ? before : H);
+            } else {
+                pos = H + fi_rank;
+            }
+            fi_rank++;
+        }
+        order[pos] = (c << 24) | s;
+    }
+}
 
 // Fill n bytes at p with byte b using 16-byte streaming stores where alignment allows.  Block-collective.
 __device__ __forceinline__ void block_fill(uint8_t *p, uint64_t n, uint32_t b)
@@ -53,6 +147,21 @@ __device__ __forceinline__ void block_fill(uint8_t *p, uint64_t n, uint32_t b)
     for (uint64_t i = done + tid; i < n; i += nt) p[i] = (uint8_t)b;
 }
 
+// Copy n bytes from shared memory to global memory, src and dst at the same offset modulo 16, with 16-byte
+// streaming stores for the aligned body.  Block-collective.
+__device__ __forceinline__ void block_copy_out(uint8_t *dst, const uint8_t *src, uint32_t n)
+{
+    const uint32_t tid = threadIdx.x, nt = blockDim.x;
+    uint32_t head = (16u - (uint32_t)(reinterpret_cast<uintptr_t>(dst) & 15u)) & 15u;
+    if (head > n) head = n;
+    for (uint32_t i = tid; i < head; i += nt) dst[i] = src[i];
+    const uint32_t nv = (n - head) >> 4;
+    const uint4 *s4 = reinterpret_cast<const uint4 *>(src + head);
+    uint4 *d4 = reinterpret_cast<uint4 *>(dst + head);
+    for (uint32_t i = tid; i < nv; i += nt) __stcs(d4 + i, s4[i]);
+    for (uint32_t i = head + (nv << 4) + tid; i < n; i += nt) dst[i] = src[i];
+}
+
 template <typename RI>
 __global__ void __launch_bounds__(kThreads, 4) score_kernel(const __grid_constant__ DevPlan P, const ScoreArgs A)
 {
@@ -67,7 +176,11 @@ __global__ void __launch_bounds__(kThreads, 4) score_kernel(const __grid_constan
     __shared__ uint16_t s_pass[2048];       // table entries of the current slab that pass rules 4-7
     __shared__ int s_np;
     __shared__ int s_qn;                    // candidates of the current slab queued for the cost model
-    extern __shared__ uint16_t s_queue[];   // their positions in the slab (P.slab entries, training plans)
+    // training plans: reason bytes of the current slab (P.slab + 16 bytes), then the queue of positions in the
+    // slab that go to the cost model (kQueueCap entries, drained whenever it may fill up)
+    extern __shared__ __align__(16) uint8_t s_dyn[];
+    uint8_t *const s_img = s_dyn;
+    uint16_t *const s_queue = reinterpret_cast<uint16_t *>(s_dyn + ((P.slab + 16 + 15) & ~15u));
 
     const int tid = threadIdx.x;
     const bool train = P.phase == PF_PHASE_TRAIN;
@@ -93,37 +206,20 @@ __global__ void __launch_bounds__(kThreads, 4) score_kernel(const __grid_constan
         uint32_t s = atomicAdd(A.slab_counter, 1u);
         s_gthr = want_topk ? *reinterpret_cast<volatile unsigned long long *>(A.g_thr) : 0ull;
         SlabInfo si;
-        // heavy (evaluated) and light (constant-fill) slabs cluster in index order; a multiplicative
-        // permutation interleaves them so that arithmetic and store traffic overlap on every SM
-        si.slab = s < A.n_slabs ? (uint32_t)(((uint64_t)s * A.slab_mul) % A.n_slabs) : 0xFFFFFFFFu;
+        si.slab = 0xFFFFFFFFu;
         si.pre_reason = 0;
         if (s < A.n_slabs) {
-            uint64_t o = A.slab_lo + si.slab;
-            for (int a = P.n_inner; a < P.n_axes; a++) {
-                uint64_t r = P.radix[a];
-                uint64_t q = o / r;
-                si.outer[a] = __ldg(A.vals + P.val_off[a] + (int)(o - q * r));
-                o = q;
-            }
-            if (P.n_pre_rules > 0) {
-                if (train) {
-                    TrainTuple c;
-                    c.mb = P.n_inner <= 3 ? si.outer[3] : 1;
-                    c.ep = P.n_inner <= 5 ? si.outer[5] : 1;
-                    c.pp = si.outer[6]; c.tp = si.outer[7]; c.dp = si.outer[8]; c.world = si.outer[9];
-                    RI dp, world;
-                    int r = train_layout_rules<RI>(P, c, 1, P.n_pre_rules < 3 ? P.n_pre_rules : 3, dp, world);
-                    if (r == 0 && P.n_pre_rules >= 4) {
-                        RI dpmb = dp * (RI)c.mb;
-                        if (((RI)P.gbs) % dpmb != 0) r = PF_R_BATCH;
-                    }
-                    si.pre_reason = r;
-                } else {
-                    ServeTuple c;
-                    c.batch = P.n_inner <= 2 ? si.outer[2] : 1;
-                    c.dpa = si.outer[3]; c.ep = si.outer[4]; c.tp = si.outer[5];
-                    si.pre_reason = serve_layout_rules<RI>(P, c, 1, P.n_pre_rules >= 4);
-                }
+            if (A.order) {
+                // the visiting order and every slab's class were prepared by the launches before this one
+                const uint32_t w = __ldcg(A.order + s);
+                si.slab = w & 0xFFFFFFu;
+                si.pre_reason = (int)(w >> 24);
+                if (si.pre_reason == 0) slab_outer_axes<RI>(P, A.vals, A.slab_lo + si.slab, si.outer, false);
+            } else {
+                // too many slabs for an order table: a multiplicative permutation interleaves evaluated and
+                // filled slabs, which cluster in index order
+                si.slab = (uint32_t)(((uint64_t)s * A.slab_mul) % A.n_slabs);
+                si.pre_reason = slab_outer_axes<RI>(P, A.vals, A.slab_lo + si.slab, si.outer, true);
             }
         }
         dst = si;
@@ -213,15 +309,78 @@ __global__ void __launch_bounds__(kThreads, 4) score_kernel(const __grid_constan
         };
 
         if (train) {
+            // Under the store stream of the fill slabs every store instruction of a warp waits a few hundred
+            // nanoseconds whatever its width, so an evaluated slab writes as few and as wide stores as a filled
+            // one: tput and mem are zeroed up front with 16-byte stores and only the candidates that reach the
+            // cost model are patched; reason bytes are collected in a shared-memory image of the slab (laid
+            // out at the same 16-byte phase as its destination) and copied out once at the end.
+            const uint32_t pad = A.reason ? (uint32_t)(reinterpret_cast<uintptr_t>(A.reason + rel0) & 15u) : 0u;
+            uint8_t *img = s_img + pad;
+            if (A.tput) block_fill(reinterpret_cast<uint8_t *>(A.tput + rel0), (uint64_t)n * 4, 0u);
+            if (A.mem) block_fill(reinterpret_cast<uint8_t *>(A.mem + rel0), (uint64_t)n * 8, 0u);
             if (tid == 0) {
                 s_qn = 0;
                 s_np = 0;
             }
             __syncthreads();
+            // Phase 2 (block-collective): memory model, gate, step time and pricing for the queued candidates,
+            // one per thread, every warp full; empties the queue.
+            auto drain = [&]() {
+                const uint32_t qn = (uint32_t)s_qn;
+                for (uint32_t it = 0; it < qn; it += kThreads) {
+                    const uint32_t qi = it + tid;
+                    const bool active = qi < qn;
+                    int reason = 0;
+                    float tput = 0.f;
+                    uint32_t i = 0;
+                    if (active) {
+                        i = s_queue[qi];
+                        int v[PF_MAX_AXES], dg[5] = {0, 0, 0, 0, 0};
+                        decode_inner(j0 + i, v, dg);
+                        TrainTuple c;
+                        c.kv = v[0]; c.rec = v[1]; c.s = v[2]; c.mb = v[3]; c.v = v[4];
+                        c.ep = v[5]; c.pp = v[6]; c.tp = v[7]; c.dp = v[8]; c.world = v[9];
+                        RI dp, world;
+                        TrainDerived<RI> D;
+                        train_layout_rules<RI>(P, c, 4, 3, dp, world);      // derives dp / world only
+                        train_plan_rules<RI>(P, c, dp, world, 4, D);        // passed in phase 1: fills D
+                        TrainMem M;
+                        train_memory<RI>(P, c, D, M);
+                        if (M.mem > P.budget_bytes) {
+                            reason = PF_R_MEMORY;
+                        } else {
+                            TrainTimes T;
+                            train_times<RI>(P, c, D, M, T);
+                            tput = train_price<RI>(P, c, D, T, train_pipe_analytic<RI>(P, c, D, T));
+                            if (D.m_e < (RI)64 || D.m_e > (RI)8192) reason = PF_FLAG_EXTRAPOLATED;
+                        }
+                        const uint64_t o = rel0 + i;
+                        img[i] = (uint8_t)reason;
+                        if (A.tput && tput != 0.f) A.tput[o] = tput;
+                        if (A.mem) A.mem[o] = M.mem;
+                    }
+                    offer(active && (reason & 0x7f) == 0, tput, (uint32_t)(rel0 + i));
+                }
+                __syncthreads();
+                if (tid == 0) s_qn = 0;
+                __syncthreads();
+            };
+            // append this thread's candidate (position i in the clipped slab) to the queue; warp-collective
+            auto enqueue = [&](bool queued, uint32_t i) {
+                const unsigned mask = __ballot_sync(0xFFFFFFFFu, queued);
+                if (mask) {
+                    const int lane2 = tid & 31, leader = __ffs(mask) - 1;
+                    int qb = 0;
+                    if (lane2 == leader) qb = atomicAdd(&s_qn, __popc(mask));
+                    qb = __shfl_sync(0xFFFFFFFFu, qb, leader);
+                    if (queued) s_queue[qb + __popc(mask & ((1u << lane2) - 1u))] = (uint16_t)i;
+                }
+            };
+            int since_drain = 0;  // iterations that appended (at most kThreads entries each) since the last drain
             if (use_tab) {
                 // Phase 1a.  Candidates that share (sched, mb, v) are contiguous: a run of R = |kv| x |rec|
-                // indices.  A warp takes 32 table entries at a time; runs whose entry holds a failing rule are
-                // written at once, cooperatively and coalesced; passing entries are only listed.
+                // indices.  A warp takes 32 table entries at a time; runs whose entry holds a failing rule get
+                // their reason bytes at once; passing entries are only listed.
                 const uint32_t n_combos = (uint32_t)(P.tab_n[0] * P.tab_n[1] * P.tab_n[2]);
                 const uint32_t R = P.slab / n_combos;
                 const int lane = tid & 31, warp = tid >> 5;
@@ -242,17 +401,12 @@ __global__ void __launch_bounds__(kThreads, 4) score_kernel(const __grid_constan
                         const uint32_t run = min(x / R, 31u);
                         const int r = __shfl_sync(0xFFFFFFFFu, t, (int)run);
                         const uint32_t j = cb * R + x;
-                        if (x < cnt && r != 0 && j >= j0 && j < j0 + n) {
-                            const uint64_t o = rel0 + (j - j0);
-                            if (A.reason) A.reason[o] = (uint8_t)r;
-                            if (A.tput) A.tput[o] = 0.f;
-                            if (A.mem) A.mem[o] = 0;
-                        }
+                        if (x < cnt && r != 0 && j >= j0 && j < j0 + n) img[j - j0] = (uint8_t)r;
                     }
                 }
                 __syncthreads();
                 // Phase 1b.  The candidates of the passing entries, densely: kernel availability and the
-                // emit dry-run rules (8-10).  Rejected ones are written, the rest queued for the cost model.
+                // emit dry-run rules (8-10).  Rejected ones get their reason byte, the rest are queued.
                 const uint32_t total = (uint32_t)s_np * R;
                 for (uint32_t it = 0; it < total; it += kThreads) {
                     const uint32_t x = it + tid;
@@ -272,101 +426,54 @@ __global__ void __launch_bounds__(kThreads, 4) score_kernel(const __grid_constan
                             TrainDerived<RI> D;
                             train_layout_rules<RI>(P, c, 4, 3, dp, world);   // derives dp / world only
                             const int reason = train_plan_rules<RI>(P, c, dp, world, 4, D);
-                            if (reason != 0) {
-                                const uint64_t o = rel0 + i;
-                                if (A.reason) A.reason[o] = (uint8_t)reason;
-                                if (A.tput) A.tput[o] = 0.f;
-                                if (A.mem) A.mem[o] = 0;
-                            } else {
+                            if (reason != 0)
+                                img[i] = (uint8_t)reason;
+                            else
                                 queued = true;
-                            }
                         }
                     }
-                    const unsigned mask = __ballot_sync(0xFFFFFFFFu, queued);
-                    if (mask) {
-                        const int lane2 = tid & 31, leader = __ffs(mask) - 1;
-                        int qb = 0;
-                        if (lane2 == leader) qb = atomicAdd(&s_qn, __popc(mask));
-                        qb = __shfl_sync(0xFFFFFFFFu, qb, leader);
-                        if (queued) s_queue[qb + __popc(mask & ((1u << lane2) - 1u))] = (uint16_t)i;
+                    enqueue(queued, i);
+                    if (++since_drain == kQueueCap / kThreads) {
+                        __syncthreads();
+                        drain();
+                        since_drain = 0;
                     }
                 }
             } else {
-            // Phase 1 without a rule table: integer rules for every candidate of the slab.  Rejected
-            // candidates are written at once; the ones that reach the memory gate are only queued, because
-            // they come in short runs and would leave most lanes of their warps idle.
-            for (uint32_t it = 0; it < n; it += kThreads) {
-                const uint32_t i = it + tid;
-                bool queued = false;
-                if (i < n) {
-                    int v[PF_MAX_AXES], dg[5] = {0, 0, 0, 0, 0};
-                    decode_inner(j0 + i, v, dg);
-                    TrainTuple c;
-                    c.kv = v[0]; c.rec = v[1]; c.s = v[2]; c.mb = v[3]; c.v = v[4];
-                    c.ep = v[5]; c.pp = v[6]; c.tp = v[7]; c.dp = v[8]; c.world = v[9];
-                    RI dp, world;
-                    int reason = train_layout_rules<RI>(P, c, first_rule, 3, dp, world);
-                    if (reason == 0) {
-                        TrainDerived<RI> D;
-                        reason = train_plan_rules<RI>(P, c, dp, world, first_rule, D);
+                // Phase 1 without a rule table: integer rules for every candidate of the slab.  Rejected
+                // candidates get their reason byte; the ones that reach the memory gate are only queued, because
+                // they come in short runs and would leave most lanes of their warps idle.
+                for (uint32_t it = 0; it < n; it += kThreads) {
+                    const uint32_t i = it + tid;
+                    bool queued = false;
+                    if (i < n) {
+                        int v[PF_MAX_AXES], dg[5] = {0, 0, 0, 0, 0};
+                        decode_inner(j0 + i, v, dg);
+                        TrainTuple c;
+                        c.kv = v[0]; c.rec = v[1]; c.s = v[2]; c.mb = v[3]; c.v = v[4];
+                        c.ep = v[5]; c.pp = v[6]; c.tp = v[7]; c.dp = v[8]; c.world = v[9];
+                        RI dp, world;
+                        int reason = train_layout_rules<RI>(P, c, first_rule, 3, dp, world);
+                        if (reason == 0) {
+                            TrainDerived<RI> D;
+                            reason = train_plan_rules<RI>(P, c, dp, world, first_rule, D);
+                        }
+                        if (reason != 0)
+                            img[i] = (uint8_t)reason;
+                        else
+                            queued = true;
                     }
-                    if (reason != 0) {
-                        const uint64_t o = rel0 + i;
-                        if (A.reason) A.reason[o] = (uint8_t)reason;
-                        if (A.tput) A.tput[o] = 0.f;
-                        if (A.mem) A.mem[o] = 0;
-                    } else {
-                        queued = true;
+                    enqueue(queued, i);
+                    if (++since_drain == kQueueCap / kThreads) {
+                        __syncthreads();
+                        drain();
+                        since_drain = 0;
                     }
                 }
-                const unsigned mask = __ballot_sync(0xFFFFFFFFu, queued);
-                if (mask) {
-                    const int lane = tid & 31, leader = __ffs(mask) - 1;
-                    int qb = 0;
-                    if (lane == leader) qb = atomicAdd(&s_qn, __popc(mask));
-                    qb = __shfl_sync(0xFFFFFFFFu, qb, leader);
-                    if (queued) s_queue[qb + __popc(mask & ((1u << lane) - 1u))] = (uint16_t)i;
-                }
-            }
             }
             __syncthreads();
-            // Phase 2: memory model, gate, step time and pricing for the queued candidates, one per thread,
-            // every warp full.
-            const uint32_t qn = (uint32_t)s_qn;
-            for (uint32_t it = 0; it < qn; it += kThreads) {
-                const uint32_t qi = it + tid;
-                const bool active = qi < qn;
-                int reason = 0;
-                float tput = 0.f;
-                uint32_t i = 0;
-                if (active) {
-                    i = s_queue[qi];
-                    int v[PF_MAX_AXES], dg[5] = {0, 0, 0, 0, 0};
-                    decode_inner(j0 + i, v, dg);
-                    TrainTuple c;
-                    c.kv = v[0]; c.rec = v[1]; c.s = v[2]; c.mb = v[3]; c.v = v[4];
-                    c.ep = v[5]; c.pp = v[6]; c.tp = v[7]; c.dp = v[8]; c.world = v[9];
-                    RI dp, world;
-                    TrainDerived<RI> D;
-                    train_layout_rules<RI>(P, c, 4, 3, dp, world);      // derives dp / world only
-                    train_plan_rules<RI>(P, c, dp, world, 4, D);        // passed in phase 1: fills D
-                    TrainMem M;
-                    train_memory<RI>(P, c, D, M);
-                    if (M.mem > P.budget_bytes) {
-                        reason = PF_R_MEMORY;
-                    } else {
-                        TrainTimes T;
-                        train_times<RI>(P, c, D, M, T);
-                        tput = train_price<RI>(P, c, D, T, train_pipe_analytic<RI>(P, c, D, T));
-                        if (D.m_e < (RI)64 || D.m_e > (RI)8192) reason = PF_FLAG_EXTRAPOLATED;
-                    }
-                    const uint64_t o = rel0 + i;
-                    if (A.reason) A.reason[o] = (uint8_t)reason;
-                    if (A.tput) A.tput[o] = tput;
-                    if (A.mem) A.mem[o] = M.mem;
-                }
-                offer(active && (reason & 0x7f) == 0, tput, (uint32_t)(rel0 + i));
-            }
+            drain();
+            if (A.reason) block_copy_out(A.reason + rel0, img, n);
         } else {
             for (uint32_t it = 0; it < n; it += kThreads) {
                 const uint32_t i = it + tid;
@@ -584,12 +691,20 @@ static void slab_span(const pf_plan_t *p, uint64_t first, uint64_t count, uint64
 
 using namespace pf;
 
+// bytes of the visiting-order table (uint32 per slab) and the class bytes behind it; 0 when the call has too
+// many slabs for a table
+static size_t order_bytes(uint64_t n_slabs)
+{
+    if (n_slabs > (uint64_t)kOrderMaxSlabs) return 0;
+    return (((size_t)n_slabs * 4 + 255) & ~(size_t)255) + (((size_t)n_slabs + 255) & ~(size_t)255);
+}
+
 extern "C" size_t pf_score_workspace(const pf_plan_t *p, uint64_t count, uint32_t k)
 {
     if (!p || count == 0) return 256;
     uint64_t slab_lo, n_slabs;
     slab_span(p, 0, count + p->dev.slab, slab_lo, n_slabs);  // any alignment of `first`
-    return topk_layout((uint64_t)grid_for(p, n_slabs) * k, k).total;
+    return topk_layout((uint64_t)grid_for(p, n_slabs) * k, k).total + order_bytes(n_slabs);
 }
 
 extern "C" int pf_score(pf_plan_t *p, uint64_t first, uint64_t count, uint8_t *d_reason, float *d_tput,
@@ -627,8 +742,29 @@ extern "C" int pf_score(pf_plan_t *p, uint64_t first, uint64_t count, uint8_t *d
     a.key_count = a.slab_counter + 1;
     a.g_thr = (unsigned long long *)(ws + lay.off_ctrl + 16);
     a.vals = p->d_vals; a.scen = p->d_scen;
+    a.order = nullptr;
     PF_CUDA_TRY(cudaMemsetAsync(a.slab_counter, 0, 256, st), "pf_score: counter reset");
-    const size_t queue_bytes = p->dev.phase == PF_PHASE_TRAIN ? (size_t)p->dev.slab * sizeof(uint16_t) : 0;
+    timing_begin(p, PF_T_SCORE, st);
+    int n_score_kernels = 1;
+    if (order_bytes(n_slabs) != 0 && n_slabs > (uint64_t)grid) {
+        uint32_t *order = (uint32_t *)(ws + lay.total);
+        uint8_t *cls = ws + lay.total + (((size_t)n_slabs * 4 + 255) & ~(size_t)255);
+        const unsigned cgrid = (unsigned)((n_slabs + 255) / 256);
+        if (p->dev.wide)
+            slab_class_kernel<unsigned long long><<<cgrid, 256, 0, st>>>(p->dev, p->d_vals, slab_lo,
+                                                                        (uint32_t)n_slabs, cls);
+        else
+            slab_class_kernel<uint32_t><<<cgrid, 256, 0, st>>>(p->dev, p->d_vals, slab_lo, (uint32_t)n_slabs, cls);
+        slab_order_kernel<<<1, 1024, 0, st>>>(cls, (uint32_t)n_slabs, (uint32_t)grid * kTailFillsPerBlock, order);
+        PF_CUDA_TRY(cudaGetLastError(), "slab order launch");
+        count_launch();
+        count_launch();
+        n_score_kernels = 3;
+        a.order = order;
+    }
+    const size_t queue_bytes = p->dev.phase == PF_PHASE_TRAIN
+                                   ? (((size_t)p->dev.slab + 16 + 15) & ~(size_t)15) + kQueueCap * sizeof(uint16_t)
+                                   : 0;
     // static + dynamic shared memory passes the 48 KB default for large slabs: opt in
     if (p->dev.wide)
         PF_CUDA_TRY(cudaFuncSetAttribute(score_kernel<unsigned long long>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -636,13 +772,12 @@ extern "C" int pf_score(pf_plan_t *p, uint64_t first, uint64_t count, uint8_t *d
     else
         PF_CUDA_TRY(cudaFuncSetAttribute(score_kernel<uint32_t>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)queue_bytes), "score_kernel smem");
-    timing_begin(p, PF_T_SCORE, st);
     if (p->dev.wide)
         score_kernel<unsigned long long><<<grid, kThreads, queue_bytes, st>>>(p->dev, a);
     else
         score_kernel<uint32_t><<<grid, kThreads, queue_bytes, st>>>(p->dev, a);
     count_launch();
-    timing_end(p, PF_T_SCORE, 1, st);
+    timing_end(p, PF_T_SCORE, n_score_kernels, st);
     PF_CUDA_TRY(cudaGetLastError(), "score_kernel launch");
     if (k > 0) {
         timing_begin(p, PF_T_TOPK, st);
