@@ -32,6 +32,15 @@ struct ScoreArgs {
     const uint32_t *order;          // ticket -> (pre_reason << 24) | slab, or NULL: visit by slab_mul, classify here
 };
 
+// Per passing (sched, mb, v) entry of a slab: what its candidates share across kernel variant and recompute mode.
+constexpr int kEntryBatch = kThreads / 4;
+struct EntryInfo {
+    long long mem[3];               // peak bytes per recompute mode
+    uint32_t kv_bad;                // bit q: kernel variant q has no kernel for this entry's expert shape
+    uint8_t unmapped;               // the schedule has no emitter mapping (and realizability is enforced)
+    uint8_t rec_bad;                // bit r: recompute mode r breaks the overlap preconditions
+};
+
 struct SlabInfo {
     uint32_t slab;                  // slab number relative to slab_lo, or 0xFFFFFFFF when the queue is empty
     int pre_reason;                 // != 0: every candidate of the slab fails this rule
@@ -175,6 +184,7 @@ __global__ void __launch_bounds__(kThreads, 4) score_kernel(const __grid_constan
     __shared__ int32_t s_vals[kInnerVals];  // value lists of the inner axes (the packed array's prefix)
     __shared__ uint16_t s_pass[2048];       // table entries of the current slab that pass rules 4-7
     __shared__ int s_np;
+    __shared__ EntryInfo s_info[kEntryBatch];  // what a batch of passing entries shares across kv and rec
     __shared__ int s_qn;                    // candidates of the current slab queued for the cost model
     // training plans: reason bytes of the current slab (P.slab + 16 bytes), then the queue of positions in the
     // slab that go to the cost model (kQueueCap entries, drained whenever it may fill up)
@@ -200,18 +210,17 @@ __global__ void __launch_bounds__(kThreads, 4) score_kernel(const __grid_constan
     if (vals_in_smem)
         for (int i = tid; i < n_inner_vals; i += kThreads) s_vals[i] = A.vals[i];
     const int32_t *inner_vals = vals_in_smem ? s_vals : A.vals;
-    // Slab tickets are double-buffered: while the block works on one slab, thread 0 already draws and decodes
-    // the next one, so the queue round trip and the outer-digit divisions stay off the critical path.
-    auto fetch_slab = [&](SlabInfo &dst) {
-        uint32_t s = atomicAdd(A.slab_counter, 1u);
-        s_gthr = want_topk ? *reinterpret_cast<volatile unsigned long long *>(A.g_thr) : 0ull;
+    // Slab tickets run two ahead.  Under the store stream an atomic or a load that goes to L2 takes microseconds,
+    // so thread 0 never waits for one where it was issued: the ticket drawn at the top of one slab is first
+    // used at the top of the next one (to load its order word), and that word is first used at the bottom of
+    // the same slab, after thread 0's share of the slab's stores, to set up the following slab.
+    auto resolve = [&](uint32_t s, uint32_t w, SlabInfo &dst) {
         SlabInfo si;
         si.slab = 0xFFFFFFFFu;
         si.pre_reason = 0;
         if (s < A.n_slabs) {
             if (A.order) {
                 // the visiting order and every slab's class were prepared by the launches before this one
-                const uint32_t w = __ldcg(A.order + s);
                 si.slab = w & 0xFFFFFFu;
                 si.pre_reason = (int)(w >> 24);
                 if (si.pre_reason == 0) slab_outer_axes<RI>(P, A.vals, A.slab_lo + si.slab, si.outer, false);
@@ -224,13 +233,33 @@ __global__ void __launch_bounds__(kThreads, 4) score_kernel(const __grid_constan
         }
         dst = si;
     };
-    if (tid == 0) fetch_slab(s_slabs[0]);
+    uint32_t tkt_next = 0, tkt_after = 0, word_next = 0;  // thread 0: tickets and order word in flight
+    unsigned long long gthr_next = 0ull;                   // thread 0: the grid-wide threshold, in flight
+    if (tid == 0) {
+        const uint32_t t0 = atomicAdd(A.slab_counter, 1u);
+        s_gthr = 0ull;
+        resolve(t0, (A.order && t0 < A.n_slabs) ? __ldcg(A.order + t0) : 0u, s_slabs[0]);
+        tkt_next = atomicAdd(A.slab_counter, 1u);
+    }
     __syncthreads();
 
     for (int cur = 0;; cur ^= 1) {
         const SlabInfo &s_slab = s_slabs[cur];
         if (s_slab.slab == 0xFFFFFFFFu) break;
-        if (tid == 0) fetch_slab(s_slabs[cur ^ 1]);
+        if (tid == 0) {
+            word_next = (A.order && tkt_next < A.n_slabs) ? __ldcg(A.order + tkt_next) : 0u;
+            tkt_after = atomicAdd(A.slab_counter, 1u);
+            if (want_topk) gthr_next = *reinterpret_cast<volatile unsigned long long *>(A.g_thr);
+        }
+        // end of a slab: set up the next one from what was requested at its top
+        auto finish_slab = [&]() {
+            if (tid == 0) {
+                resolve(tkt_next, word_next, s_slabs[cur ^ 1]);
+                tkt_next = tkt_after;
+                s_gthr = gthr_next;
+            }
+            __syncthreads();  // the next slab's record is complete and this one's no longer read
+        };
 
         // candidate range of this slab clipped to the call's range
         const uint64_t slab_no = A.slab_lo + s_slab.slab;
@@ -245,7 +274,7 @@ __global__ void __launch_bounds__(kThreads, 4) score_kernel(const __grid_constan
             if (A.reason) block_fill(A.reason + rel0, n, (uint32_t)s_slab.pre_reason);
             if (A.tput) block_fill(reinterpret_cast<uint8_t *>(A.tput + rel0), (uint64_t)n * 4, 0u);
             if (A.mem) block_fill(reinterpret_cast<uint8_t *>(A.mem + rel0), (uint64_t)n * 8, 0u);
-            __syncthreads();  // the next ticket is complete and this one no longer read
+            finish_slab();
             continue;
         }
 
@@ -383,9 +412,9 @@ __global__ void __launch_bounds__(kThreads, 4) score_kernel(const __grid_constan
                 // their reason bytes at once; passing entries are only listed.
                 const uint32_t n_combos = (uint32_t)(P.tab_n[0] * P.tab_n[1] * P.tab_n[2]);
                 const uint32_t R = P.slab / n_combos;
-                const int lane = tid & 31, warp = tid >> 5;
-                for (uint32_t cb = (uint32_t)warp * 32; cb < n_combos; cb += (kThreads / 32) * 32) {
-                    const uint32_t e = cb + lane;
+                const int lane = tid & 31;
+                for (uint32_t cb = 0; cb < n_combos; cb += kThreads) {
+                    const uint32_t e = cb + tid;
                     const int t = e < n_combos ? (int)s_tab[e] : 0xFF;
                     const unsigned pm = __ballot_sync(0xFFFFFFFFu, t == 0);
                     if (pm) {
@@ -395,49 +424,101 @@ __global__ void __launch_bounds__(kThreads, 4) score_kernel(const __grid_constan
                         pb = __shfl_sync(0xFFFFFFFFu, pb, leader);
                         if (t == 0) s_pass[pb + __popc(pm & ((1u << lane) - 1u))] = (uint16_t)e;
                     }
-                    const uint32_t cnt = min(32u, n_combos - cb) * R;
-                    for (uint32_t xb = 0; xb < cnt; xb += 32) {
-                        const uint32_t x = xb + lane;
-                        const uint32_t run = min(x / R, 31u);
-                        const int r = __shfl_sync(0xFFFFFFFFu, t, (int)run);
-                        const uint32_t j = cb * R + x;
-                        if (x < cnt && r != 0 && j >= j0 && j < j0 + n) img[j - j0] = (uint8_t)r;
+                    if (t != 0 && t != 0xFF) {
+                        // the run's candidates, clipped to the call's range
+                        const uint32_t ja = max(e * R, j0), jb = min(e * R + R, j0 + n);
+                        for (uint32_t j = ja; j < jb; j++) img[j - j0] = (uint8_t)t;
                     }
                 }
                 __syncthreads();
-                // Phase 1b.  The candidates of the passing entries, densely: kernel availability and the
-                // emit dry-run rules (8-10).  Rejected ones get their reason byte, the rest are queued.
-                const uint32_t total = (uint32_t)s_np * R;
-                for (uint32_t it = 0; it < total; it += kThreads) {
-                    const uint32_t x = it + tid;
-                    bool queued = false;
-                    uint32_t i = 0;
-                    if (x < total) {
-                        const uint32_t pe = x / R;
-                        const uint32_t j = (uint32_t)s_pass[pe] * R + (x - pe * R);
-                        if (j >= j0 && j < j0 + n) {
-                            i = j - j0;
-                            int v[PF_MAX_AXES], dg[5] = {0, 0, 0, 0, 0};
-                            decode_inner(j, v, dg);
-                            TrainTuple c;
-                            c.kv = v[0]; c.rec = v[1]; c.s = v[2]; c.mb = v[3]; c.v = v[4];
-                            c.ep = v[5]; c.pp = v[6]; c.tp = v[7]; c.dp = v[8]; c.world = v[9];
-                            RI dp, world;
-                            TrainDerived<RI> D;
-                            train_layout_rules<RI>(P, c, 4, 3, dp, world);   // derives dp / world only
-                            const int reason = train_plan_rules<RI>(P, c, dp, world, 4, D);
-                            if (reason != 0)
-                                img[i] = (uint8_t)reason;
-                            else
-                                queued = true;
+                // Phase 1b.  Inside a passing entry only the kernel variant and the recompute mode vary.  One
+                // thread per entry works out what depends on neither: which variants lack a kernel at this
+                // expert shape (rule 8), whether the schedule is unmapped (9), which recompute modes break the
+                // overlap preconditions (10), and the peak memory per recompute mode (the variant does not
+                // enter it).  The entry's candidates then only look these up; the few that pass the memory
+                // gate are queued for the cost model.
+                const uint32_t np = (uint32_t)s_np;
+                for (uint32_t b0 = 0; b0 < np; b0 += kEntryBatch) {
+                    const uint32_t nb = min((uint32_t)kEntryBatch, np - b0);
+                    if ((uint32_t)(tid >> 2) < nb) {
+                        // four lanes per entry: lanes 0-2 take one recompute mode's memory each, lane 3 the rules
+                        const int role = tid & 3, slot = tid >> 2;
+                        const int e = s_pass[b0 + slot];
+                        const int n2 = P.tab_n[0], n3 = P.tab_n[1];
+                        const int d2 = e % n2, d3 = (e / n2) % n3, d4 = e / (n2 * n3);
+                        TrainTuple c;
+                        c.kv = 0; c.rec = role < 3 ? role : 0;
+                        c.s = P.n_inner > 2 ? inner_vals[P.val_off[2] + d2] : s_slab.outer[2];
+                        c.mb = P.n_inner > 3 ? inner_vals[P.val_off[3] + d3] : s_slab.outer[3];
+                        c.v = P.n_inner > 4 ? inner_vals[P.val_off[4] + d4] : s_slab.outer[4];
+                        c.ep = s_slab.outer[5]; c.pp = s_slab.outer[6]; c.tp = s_slab.outer[7];
+                        c.dp = s_slab.outer[8]; c.world = s_slab.outer[9];
+                        RI dp, world;
+                        TrainDerived<RI> D;
+                        train_layout_rules<RI>(P, c, 4, 3, dp, world);   // derives dp / world only
+                        train_plan_rules<RI>(P, c, dp, world, 4, D);     // rules 4-7 hold: fills D
+                        if (role < 3) {
+                            TrainMem M;
+                            train_memory<RI>(P, c, D, M);
+                            s_info[slot].mem[role] = M.mem;
+                        } else {
+                            uint32_t kv_bad = 0u;
+                            for (int q = 0; q < P.n_kern; q++) {
+                                const DevKern &kn = P.kern[q];
+                                if ((kn.needs_caps & ~P.caps) != 0u || ((kn.avail_mask >> D.bucket) & 1u) == 0u)
+                                    kv_bad |= 1u << q;
+                            }
+                            const DevSched &sc = P.sched[c.s];
+                            uint32_t rec_bad = 0u;
+                            if (P.enforce && sc.overlap)
+                                rec_bad = (D.kind == PF_KIND_1F1B && c.pp > 1) ? 7u : (1u << PF_REC_FULL);
+                            s_info[slot].kv_bad = kv_bad;
+                            s_info[slot].unmapped = (P.enforce && !sc.mapped) ? 1 : 0;
+                            s_info[slot].rec_bad = (uint8_t)rec_bad;
                         }
                     }
-                    enqueue(queued, i);
-                    if (++since_drain == kQueueCap / kThreads) {
-                        __syncthreads();
-                        drain();
-                        since_drain = 0;
+                    __syncthreads();
+                    const uint32_t total = nb * R;
+                    for (uint32_t it = 0; it < total; it += kThreads) {
+                        const uint32_t x = it + tid;
+                        bool queued = false;
+                        uint32_t i = 0;
+                        if (x < total) {
+                            const uint32_t pe = x / R, ro = x - pe * R;
+                            const uint32_t j = (uint32_t)s_pass[b0 + pe] * R + ro;
+                            if (j >= j0 && j < j0 + n) {
+                                i = j - j0;
+                                const uint32_t r0 = P.radix[0];
+                                const uint32_t qd = r0 == 1u ? ro : __umulhi(ro, P.magic[0]);
+                                const int kvv = inner_vals[P.val_off[0] + (int)(ro - qd * r0)];
+                                const int recv = P.n_inner > 1 ? inner_vals[P.val_off[1] + (int)qd] : s_slab.outer[1];
+                                const EntryInfo &info = s_info[pe];
+                                int reason = 0;
+                                if ((info.kv_bad >> kvv) & 1u) {
+                                    reason = PF_R_KERNEL_MISSING;
+                                } else if (info.unmapped) {
+                                    reason = PF_R_UNMAPPED_SCHEDULE;
+                                } else if ((info.rec_bad >> recv) & 1) {
+                                    reason = PF_R_OVERLAP_PRECOND;
+                                } else {
+                                    const long long mem = info.mem[recv];
+                                    if (A.mem) A.mem[rel0 + i] = mem;
+                                    if (mem > P.budget_bytes)
+                                        reason = PF_R_MEMORY;
+                                    else
+                                        queued = true;
+                                }
+                                if (!queued) img[i] = (uint8_t)reason;
+                            }
+                        }
+                        enqueue(queued, i);
+                        if (++since_drain == kQueueCap / kThreads) {
+                            __syncthreads();
+                            drain();
+                            since_drain = 0;
+                        }
                     }
+                    __syncthreads();  // the batch's entry records are read no more
                 }
             } else {
                 // Phase 1 without a rule table: integer rules for every candidate of the slab.  Rejected
@@ -494,7 +575,7 @@ __global__ void __launch_bounds__(kThreads, 4) score_kernel(const __grid_constan
                 offer(active && (so.reason & 0x7f) == 0, so.tput, (uint32_t)(rel0 + i));
             }
         }
-        __syncthreads();  // the next ticket is complete and this one no longer read
+        finish_slab();
     }
 
     if (want_topk) {
