@@ -189,6 +189,12 @@ int pf_decode(const pf_plan_t *plan, uint64_t idx, pf_tuple_t *out);
  *   slots), d_topk_score[k] (float, 0 in unused slots), d_topk_count[1] (uint32) are required.
  *   d_workspace: at least pf_score_workspace(plan, count, k) bytes, 256-byte aligned, contents ignored.
  * count < PF_MAX_COUNT per call; larger spaces are scored in chunks and merged with pf_topk_merge.
+ * The plan keeps, in device memory it allocated at creation, the order in which the kernel visits the blocks
+ * of candidates of its latest range (evaluated blocks first, spread between constant ones); a call on another
+ * range rebuilds it on `stream` with two small launches, a call on the same range reuses it.  Device work of
+ * calls on one plan must therefore be ordered (one stream, or events between streams); a table that does not
+ * hold the call's range -- e.g. its rebuild was captured into a graph that has not run -- is detected on the
+ * device and ignored, at some cost in speed only.
  * Errors: PF_EINVAL, PF_ERANGE, PF_EWORKSPACE, PF_ECUDA (launch failure). */
 size_t pf_score_workspace(const pf_plan_t *plan, uint64_t count, uint32_t k);
 int pf_score(pf_plan_t *plan, uint64_t first, uint64_t count, uint8_t *d_reason, float *d_tput, int64_t *d_mem,

@@ -376,6 +376,17 @@ extern "C" int pf_plan_create(const pf_model_t *model, const pf_cluster_t *clust
         if (e == cudaSuccess)
             e = cudaMemcpy(p->d_scen + n, workload->scen_O, sizeof(int32_t) * n, cudaMemcpyHostToDevice);
     }
+    if (e == cudaSuccess) {
+        // room for the slab visiting order of one pf_score range (any alignment of its first candidate)
+        const uint64_t slabs = (p->size + d.slab - 1) / d.slab + 1;
+        p->order_cap = 0;
+        p->order_n_slabs = 0;
+        if (slabs <= (uint64_t)pf::kOrderMaxSlabs) {
+            e = cudaMalloc((void **)&p->d_order, 256 + (size_t)slabs * 5);
+            if (e == cudaSuccess) e = cudaMemset(p->d_order, 0, 256);
+            p->order_cap = (uint32_t)slabs;
+        }
+    }
     if (e != cudaSuccess) {
         pf::set_cuda_error(e, "pf_plan_create: upload");
         pf_plan_destroy(p);
@@ -434,6 +445,7 @@ extern "C" void pf_plan_destroy(pf_plan_t *p)
     pf::free_sim_tables(p);
     if (p->d_vals) cudaFree(p->d_vals);
     if (p->d_scen) cudaFree(p->d_scen);
+    if (p->d_order) cudaFree(p->d_order);
     free(p->h_vals);
     delete p;
 }

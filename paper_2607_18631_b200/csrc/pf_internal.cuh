@@ -81,6 +81,13 @@ struct pf_plan {
     // device buffers owned by the handle
     int32_t *d_vals;               // packed axis value lists
     int32_t *d_scen;               // serve: P[n_scen] then O[n_scen]
+    // Slab visiting order of the most recent pf_score range (device: 64 header words, order_cap order words,
+    // order_cap class bytes); NULL when the space has too many slabs.  The host key below says which range
+    // the table was last built for; the device header says which range it actually holds.
+    uint32_t *d_order;
+    uint32_t order_cap;
+    uint64_t order_slab_lo;
+    uint32_t order_n_slabs, order_tail;
     // simulator order tables (built at create for training plans)
     void *sim_tables;
     // optional per-kernel-class event timing (pf_timing_enable)

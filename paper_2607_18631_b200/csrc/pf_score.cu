@@ -30,6 +30,8 @@ struct ScoreArgs {
     const int32_t *vals;            // packed axis value lists
     const int32_t *scen;            // serve: P[n_scen], O[n_scen]
     const uint32_t *order;          // ticket -> (pre_reason << 24) | slab, or NULL: visit by slab_mul, classify here
+    const uint32_t *order_hdr;      // the range the order table holds: slab_lo (2 words), n_slabs, tail
+    uint32_t order_tail;            // the tail length this call wants
 };
 
 // Per passing (sched, mb, v) entry of a slab: what its candidates share across kernel variant and recompute mode.
@@ -100,8 +102,8 @@ __global__ void __launch_bounds__(256) slab_class_kernel(const __grid_constant__
 // ticket in closed form.  With H evaluated and F filled slabs, the last min(F, tail) fills form the tail and
 // the other Fs fills are interleaved: evaluated slab i sits after floor(i * Fs / H) fills, fill j after
 // min(H, ceil((j + 1) * H / Fs)) evaluated slabs.
-__global__ void __launch_bounds__(1024) slab_order_kernel(const uint8_t *cls, uint32_t n_slabs, uint32_t tail,
-                                                          uint32_t *order)
+__global__ void __launch_bounds__(1024) slab_order_kernel(const uint8_t *cls, uint64_t slab_lo, uint32_t n_slabs,
+                                                          uint32_t tail, uint32_t *order, uint32_t *hdr)
 {
     __shared__ uint32_t s_part[1024];
     const uint32_t tid = threadIdx.x;
@@ -137,6 +139,13 @@ __global__ void __launch_bounds__(1024) slab_order_kernel(const uint8_t *cls, ui
             fi_rank++;
         }
         order[pos] = (c << 24) | s;
+    }
+    // the header names the range this table now holds; a reader that wants another range ignores the table
+    if (tid == 0) {
+        hdr[0] = (uint32_t)slab_lo;
+        hdr[1] = (uint32_t)(slab_lo >> 32);
+        hdr[2] = n_slabs;
+        hdr[3] = tail;
     }
 }
 
@@ -214,12 +223,17 @@ __global__ void __launch_bounds__(kThreads, 4) score_kernel(const __grid_constan
     // so thread 0 never waits for one where it was issued: the ticket drawn at the top of one slab is first
     // used at the top of the next one (to load its order word), and that word is first used at the bottom of
     // the same slab, after thread 0's share of the slab's stores, to set up the following slab.
+    // The order table belongs to the plan and holds one range: use it only if that is this call's range.
+    const uint32_t *order = nullptr;
+    if (A.order && A.order_hdr[0] == (uint32_t)A.slab_lo && A.order_hdr[1] == (uint32_t)(A.slab_lo >> 32) &&
+        A.order_hdr[2] == A.n_slabs && A.order_hdr[3] == A.order_tail)
+        order = A.order;
     auto resolve = [&](uint32_t s, uint32_t w, SlabInfo &dst) {
         SlabInfo si;
         si.slab = 0xFFFFFFFFu;
         si.pre_reason = 0;
         if (s < A.n_slabs) {
-            if (A.order) {
+            if (order) {
                 // the visiting order and every slab's class were prepared by the launches before this one
                 si.slab = w & 0xFFFFFFu;
                 si.pre_reason = (int)(w >> 24);
@@ -238,7 +252,7 @@ __global__ void __launch_bounds__(kThreads, 4) score_kernel(const __grid_constan
     if (tid == 0) {
         const uint32_t t0 = atomicAdd(A.slab_counter, 1u);
         s_gthr = 0ull;
-        resolve(t0, (A.order && t0 < A.n_slabs) ? __ldcg(A.order + t0) : 0u, s_slabs[0]);
+        resolve(t0, (order && t0 < A.n_slabs) ? __ldcg(order + t0) : 0u, s_slabs[0]);
         tkt_next = atomicAdd(A.slab_counter, 1u);
     }
     __syncthreads();
@@ -247,7 +261,7 @@ __global__ void __launch_bounds__(kThreads, 4) score_kernel(const __grid_constan
         const SlabInfo &s_slab = s_slabs[cur];
         if (s_slab.slab == 0xFFFFFFFFu) break;
         if (tid == 0) {
-            word_next = (A.order && tkt_next < A.n_slabs) ? __ldcg(A.order + tkt_next) : 0u;
+            word_next = (order && tkt_next < A.n_slabs) ? __ldcg(order + tkt_next) : 0u;
             tkt_after = atomicAdd(A.slab_counter, 1u);
             if (want_topk) gthr_next = *reinterpret_cast<volatile unsigned long long *>(A.g_thr);
         }
@@ -772,20 +786,12 @@ static void slab_span(const pf_plan_t *p, uint64_t first, uint64_t count, uint64
 
 using namespace pf;
 
-// bytes of the visiting-order table (uint32 per slab) and the class bytes behind it; 0 when the call has too
-// many slabs for a table
-static size_t order_bytes(uint64_t n_slabs)
-{
-    if (n_slabs > (uint64_t)kOrderMaxSlabs) return 0;
-    return (((size_t)n_slabs * 4 + 255) & ~(size_t)255) + (((size_t)n_slabs + 255) & ~(size_t)255);
-}
-
 extern "C" size_t pf_score_workspace(const pf_plan_t *p, uint64_t count, uint32_t k)
 {
     if (!p || count == 0) return 256;
     uint64_t slab_lo, n_slabs;
     slab_span(p, 0, count + p->dev.slab, slab_lo, n_slabs);  // any alignment of `first`
-    return topk_layout((uint64_t)grid_for(p, n_slabs) * k, k).total + order_bytes(n_slabs);
+    return topk_layout((uint64_t)grid_for(p, n_slabs) * k, k).total;
 }
 
 extern "C" int pf_score(pf_plan_t *p, uint64_t first, uint64_t count, uint8_t *d_reason, float *d_tput,
@@ -827,21 +833,31 @@ extern "C" int pf_score(pf_plan_t *p, uint64_t first, uint64_t count, uint8_t *d
     PF_CUDA_TRY(cudaMemsetAsync(a.slab_counter, 0, 256, st), "pf_score: counter reset");
     timing_begin(p, PF_T_SCORE, st);
     int n_score_kernels = 1;
-    if (order_bytes(n_slabs) != 0 && n_slabs > (uint64_t)grid) {
-        uint32_t *order = (uint32_t *)(ws + lay.total);
-        uint8_t *cls = ws + lay.total + (((size_t)n_slabs * 4 + 255) & ~(size_t)255);
-        const unsigned cgrid = (unsigned)((n_slabs + 255) / 256);
-        if (p->dev.wide)
-            slab_class_kernel<unsigned long long><<<cgrid, 256, 0, st>>>(p->dev, p->d_vals, slab_lo,
-                                                                        (uint32_t)n_slabs, cls);
-        else
-            slab_class_kernel<uint32_t><<<cgrid, 256, 0, st>>>(p->dev, p->d_vals, slab_lo, (uint32_t)n_slabs, cls);
-        slab_order_kernel<<<1, 1024, 0, st>>>(cls, (uint32_t)n_slabs, (uint32_t)grid * kTailFillsPerBlock, order);
-        PF_CUDA_TRY(cudaGetLastError(), "slab order launch");
-        count_launch();
-        count_launch();
-        n_score_kernels = 3;
+    a.order_hdr = nullptr;
+    a.order_tail = (uint32_t)grid * kTailFillsPerBlock;
+    if (p->d_order && n_slabs <= p->order_cap && n_slabs > (uint64_t)grid) {
+        uint32_t *hdr = p->d_order, *order = p->d_order + 64;
+        if (p->order_slab_lo != slab_lo || p->order_n_slabs != (uint32_t)n_slabs || p->order_tail != a.order_tail) {
+            // another range than the table was last built for: rebuild it (two small launches)
+            uint8_t *cls = (uint8_t *)(order + p->order_cap);
+            const unsigned cgrid = (unsigned)((n_slabs + 255) / 256);
+            if (p->dev.wide)
+                slab_class_kernel<unsigned long long><<<cgrid, 256, 0, st>>>(p->dev, p->d_vals, slab_lo,
+                                                                            (uint32_t)n_slabs, cls);
+            else
+                slab_class_kernel<uint32_t><<<cgrid, 256, 0, st>>>(p->dev, p->d_vals, slab_lo, (uint32_t)n_slabs,
+                                                                   cls);
+            slab_order_kernel<<<1, 1024, 0, st>>>(cls, slab_lo, (uint32_t)n_slabs, a.order_tail, order, hdr);
+            PF_CUDA_TRY(cudaGetLastError(), "slab order launch");
+            count_launch();
+            count_launch();
+            n_score_kernels = 3;
+            p->order_slab_lo = slab_lo;
+            p->order_n_slabs = (uint32_t)n_slabs;
+            p->order_tail = a.order_tail;
+        }
         a.order = order;
+        a.order_hdr = hdr;
     }
     const size_t queue_bytes = p->dev.phase == PF_PHASE_TRAIN
                                    ? (((size_t)p->dev.slab + 16 + 15) & ~(size_t)15) + kQueueCap * sizeof(uint16_t)

@@ -176,6 +176,55 @@ def test_large_space_full_size():
     plan.close()
 
 
+def test_slab_order_table_follows_the_range_and_is_ignored_when_stale():
+    """The plan keeps the slab visiting order of its latest pf_score range.  Alternating ranges rebuild it; a
+    table that does not hold the call's range (here: its rebuild was only captured into a CUDA graph, not run)
+    is ignored on the device and the call still gives the oracle's results."""
+    import torch
+    cfg = make_config("large")
+    plan, orc = _plan(cfg), Oracle(cfg)
+    ranges = ((50_000_000, 30_000_000), (12_345, 40_000_000), (50_000_000, 30_000_000))
+    expect = {}
+    for first, count in ranges:
+        if (first, count) not in expect:
+            expect[(first, count)] = orc.score_range(first, count, threads=64)
+        reason, tput, mem, _ = expect[(first, count)]
+        res = gpu_score(plan, first=first, count=count, k=256)
+        compare_dense(res, reason, tput, mem)
+        compare_topk(res, orc, reason, tput, first, 256)
+    # capture a call on a new range: the table rebuild is recorded, not executed
+    first, count = 100_000_000, 20_000_000
+    reason, tput, mem, _ = orc.score_range(first, count, threads=64)
+    out = plan.score(first=ranges[0][0], count=count, k=256)          # allocates the buffers, old range
+    torch.cuda.synchronize()
+    kw = dict(first=first, count=count, k=256, reason=out["reason"], tput=out["tput"], mem=out["mem"],
+              topk_idx=out["topk_idx"], topk_score=out["topk_score"], topk_count=out["topk_count"],
+              workspace=out["workspace"])
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        plan.score(**kw)
+
+    def check():
+        torch.cuda.synchronize()
+        res = dict(reason=out["reason"].cpu().numpy(), tput=out["tput"].cpu().numpy(), mem=out["mem"].cpu().numpy())
+        n = int(out["topk_count"].item())
+        res["topk_idx"] = out["topk_idx"].cpu().numpy().view(np.uint64)[:n]
+        res["topk_score"] = out["topk_score"].cpu().numpy()[:n]
+        compare_dense(res, reason, tput, mem)
+        compare_topk(res, orc, reason, tput, first, 256)
+
+    out["reason"].fill_(99)
+    plan.score(**kw)                # eager: the host believes the table is current, the device sees it is not
+    check()
+    out["reason"].fill_(99)
+    graph.replay()                  # now the rebuild runs, followed by the scoring kernel
+    check()
+    out["reason"].fill_(99)
+    plan.score(**kw)                # and the eager call uses the rebuilt table
+    check()
+    plan.close()
+
+
 def test_large_unconstrained_topk():
     cfg = make_config("large_unconstrained")
     plan, orc = _plan(cfg), Oracle(cfg)
