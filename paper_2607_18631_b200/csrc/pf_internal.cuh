@@ -14,7 +14,8 @@ constexpr int kTopkCap = 2048;       // shared-memory candidate buffer per block
 constexpr uint32_t kSlabMax = 16384; // upper bound on candidates per slab (inner-axis product)
 constexpr int kInnerVals = 1024;     // inner-axis values the scoring kernel keeps in shared memory
 constexpr int kOrderMaxSlabs = 1 << 20;  // calls with more slabs visit them by a permutation instead of an order table
-constexpr int kTailFillsPerBlock = 4;    // constant-fill slabs per block kept for the end of the visiting order
+constexpr int kTailFillsPerBlock = 4;    // constant-fill slabs per block kept, at least, for the end of the visiting order
+constexpr int kFillsPerEvaluated = 2;    // fills interleaved per evaluated slab at the start of the visiting order
 constexpr int kQueueCap = 4096;   // cost-model queue of the scoring kernel (entries), drained when it may fill up
 
 struct DevSched {
