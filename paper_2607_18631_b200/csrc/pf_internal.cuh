@@ -274,6 +274,7 @@ __device__ __forceinline__ void tk_push(unsigned long long *buf, int *count, uns
 // uint64 at byte 16: the producers' shared admission threshold (largest k-th key any block has reached).
 constexpr int kReduceSeg = 2048;     // keys one block of the reduce kernel walks through
 constexpr int kReduceThreads = 1024;
+constexpr int kFastKeys = 16384;     // a key list up to this long is sorted whole by the final reduce block
 struct TopkLayout {
     size_t off_ctrl, off_keys_a, off_keys_b, total;
 };

@@ -610,6 +610,8 @@ __global__ void __launch_bounds__(kThreads, 4) score_kernel(const __grid_constan
 struct ReduceArgs {
     const unsigned long long *in;   // compact keys
     const unsigned int *in_count;
+    const unsigned long long *in0;  // the producers' list and its length: short lists skip the block pass
+    const unsigned int *in0_count;
     unsigned long long *out;        // compact keys of the next pass (when not final)
     unsigned int *out_count;
     uint32_t k;
@@ -625,6 +627,8 @@ struct ReduceArgs {
 // Block b walks keys [b*seg, (b+1)*seg) of the input one tile at a time, admitting only keys above its
 // running k-th best, and keeps the k best.  A tile's admissions are counted before they are appended, so the
 // buffer is pruned only when it would really overflow.
+// Pass 1: every block reduces one segment of kReduceSeg keys to its k best and appends them to the second list.
+// A producers' list of at most kFastKeys keys is left to the final kernel, which sorts it in one go.
 __global__ void __launch_bounds__(kReduceThreads) reduce_kernel(const ReduceArgs A)
 {
     __shared__ unsigned long long s_buf[kTopkCap];
@@ -633,9 +637,10 @@ __global__ void __launch_bounds__(kReduceThreads) reduce_kernel(const ReduceArgs
     __shared__ int s_base[2];
     const int tid = threadIdx.x, k = (int)A.k;
     const unsigned int n = *A.in_count;
+    if (n <= (unsigned int)kFastKeys) return;
     const unsigned int lo = blockIdx.x * A.seg;
     const unsigned int hi = min(lo + A.seg, n);
-    if (lo >= hi && !A.final) return;
+    if (lo >= hi) return;
     if (tid == 0) {
         s_count = 0;
         s_thr = 0ull;
@@ -654,23 +659,127 @@ __global__ void __launch_bounds__(kReduceThreads) reduce_kernel(const ReduceArgs
         __syncthreads();
     }
     tk_prune<kTopkCap / 2 / kReduceThreads>(s_buf, &s_count, &s_thr, k);
-    const int c = s_count;
-    if (!A.final) {
-        tk_flush(s_buf, c, 0ull, s_base, A.out, A.out_count);
-    } else {
-        for (int i = tid; i < k; i += kReduceThreads) {
-            if (i < c) {
-                unsigned long long key = s_buf[i];
-                uint32_t rel = key_rel(key);
-                A.topk_idx[i] = A.idx_map ? A.idx_map[rel] : A.first + rel;
-                A.topk_score[i] = key_score(key);
-            } else {
-                A.topk_idx[i] = UINT64_MAX;
-                A.topk_score[i] = 0.f;
+    tk_flush(s_buf, s_count, 0ull, s_base, A.out, A.out_count);
+}
+
+// Final pass, one block.  A short producers' list (at most kFastKeys keys) is loaded whole into shared memory;
+// the k-th largest key is found by a radix select over the eight key bytes, the keys from there up are gathered
+// and only those (at most k) are sorted.  Otherwise the list left by pass 1 is walked through with the usual
+// prune-on-overflow.
+__global__ void __launch_bounds__(kReduceThreads) reduce_final_kernel(const ReduceArgs A)
+{
+    extern __shared__ __align__(16) unsigned long long s_big[];  // kFastKeys keys, then kTopkCap keys to sort in
+    __shared__ int s_count;
+    __shared__ unsigned long long s_thr;
+    __shared__ unsigned int s_hist[256];
+    __shared__ unsigned long long s_prefix;
+    __shared__ unsigned int s_need;
+    const int tid = threadIdx.x, k = (int)A.k;
+    const unsigned int n0 = *A.in0_count;
+    unsigned long long *s_out = s_big;
+    int c;
+    if (n0 <= (unsigned int)kFastKeys) {
+        s_out = s_big + kFastKeys;
+        for (unsigned int i = tid; i < n0; i += kReduceThreads) s_big[i] = A.in0[i];
+        if (tid == 0) {
+            s_prefix = 0ull;
+            s_need = (unsigned int)k;
+            s_count = 0;
+        }
+        __syncthreads();
+        if (n0 > (unsigned int)k) {
+            for (int shift = 56; shift >= 0; shift -= 8) {
+                for (int i = tid; i < 256; i += kReduceThreads) s_hist[i] = 0u;
+                __syncthreads();
+                const unsigned long long hi_mask = shift == 56 ? 0ull : (~0ull << (shift + 8));
+                const unsigned long long prefix = s_prefix;
+                for (unsigned int i = tid; i < n0; i += kReduceThreads) {
+                    const unsigned long long key = s_big[i];
+                    if ((key & hi_mask) == prefix) atomicAdd(&s_hist[(unsigned int)(key >> shift) & 255u], 1u);
+                }
+                __syncthreads();
+                if (tid < 32) {
+                    // lane l owns digits 255 - 8l down to 248 - 8l; cumulative counts run from the top digit down
+                    unsigned int own = 0;
+                    for (int j = 0; j < 8; j++) own += s_hist[255 - 8 * tid - j];
+                    unsigned int incl = own;
+                    for (int off = 1; off < 32; off <<= 1) {
+                        const unsigned int y = __shfl_up_sync(0xFFFFFFFFu, incl, off);
+                        if (tid >= off) incl += y;
+                    }
+                    const unsigned int need = s_need;
+                    if (incl - own < need && incl >= need) {
+                        unsigned int run = incl - own;
+                        for (int j = 0; j < 8; j++) {
+                            const int d = 255 - 8 * tid - j;
+                            const unsigned int h = s_hist[d];
+                            if (run + h >= need) {
+                                s_prefix = prefix | ((unsigned long long)d << shift);
+                                s_need = need - run;
+                                break;
+                            }
+                            run += h;
+                        }
+                    }
+                }
+                __syncthreads();
             }
         }
-        if (tid == 0) *A.topk_count = (uint32_t)c;
+        const unsigned long long cut = n0 > (unsigned int)k ? s_prefix : 1ull;  // keys are distinct: exactly k pass
+        for (unsigned int base = 0; base < n0; base += kReduceThreads) {
+            const unsigned int i = base + tid;
+            const unsigned long long key = i < n0 ? s_big[i] : 0ull;
+            const bool take = key >= cut && key != 0ull;
+            const unsigned mask = __ballot_sync(0xFFFFFFFFu, take);
+            if (mask) {
+                const int lane = tid & 31, leader = __ffs(mask) - 1;
+                int pos = 0;
+                if (lane == leader) pos = atomicAdd(&s_count, __popc(mask));
+                pos = __shfl_sync(0xFFFFFFFFu, pos, leader);
+                pos += __popc(mask & ((1u << lane) - 1u));
+                if (take && pos < kTopkCap) s_out[pos] = key;
+            }
+        }
+        __syncthreads();
+        c = s_count < k ? s_count : k;
+        int n_sort = 64;
+        while (n_sort < c) n_sort <<= 1;
+        for (int i = c + tid; i < n_sort; i += kReduceThreads) s_out[i] = 0ull;
+        tk_sort_desc<kTopkCap / 2 / kReduceThreads>(s_out, n_sort);
+    } else {
+        const unsigned int n = *A.in_count;
+        if (tid == 0) {
+            s_count = 0;
+            s_thr = 0ull;
+        }
+        __syncthreads();
+        for (unsigned int pos = 0; pos < n; pos += kReduceThreads) {
+            const unsigned int i = pos + tid;
+            const unsigned long long key = i < n ? A.in[i] : 0ull;
+            unsigned long long thr = s_thr;
+            const int takers = __syncthreads_count(key > thr);
+            if (s_count + takers > kTopkCap) {
+                tk_prune<kTopkCap / 2 / kReduceThreads>(s_big, &s_count, &s_thr, k);
+                thr = s_thr;
+            }
+            tk_push(s_big, &s_count, thr, key != 0ull, key);
+            __syncthreads();
+        }
+        tk_prune<kTopkCap / 2 / kReduceThreads>(s_big, &s_count, &s_thr, k);
+        c = s_count;
     }
+    for (int i = tid; i < k; i += kReduceThreads) {
+        if (i < c) {
+            unsigned long long key = s_out[i];
+            uint32_t rel = key_rel(key);
+            A.topk_idx[i] = A.idx_map ? A.idx_map[rel] : A.first + rel;
+            A.topk_score[i] = key_score(key);
+        } else {
+            A.topk_idx[i] = UINT64_MAX;
+            A.topk_score[i] = 0.f;
+        }
+    }
+    if (tid == 0) *A.topk_count = (uint32_t)c;
 }
 
 int launch_topk_reduce(void *d_workspace, const TopkLayout &lay, uint64_t n_keys_max, uint32_t k, uint64_t first,
@@ -681,27 +790,30 @@ int launch_topk_reduce(void *d_workspace, const TopkLayout &lay, uint64_t n_keys
     unsigned int *ctrl = (unsigned int *)(ws + lay.off_ctrl);
     unsigned long long *in = (unsigned long long *)(ws + lay.off_keys_a);
     unsigned long long *out = (unsigned long long *)(ws + lay.off_keys_b);
-    int in_slot = 1, out_slot = 2;
     *n_kernels = 0;
-    // pass 1 spreads a long list over blocks of kReduceSeg keys; whatever it leaves (at most k keys per
-    // block) is finished by one block
-    for (int pass = 0; pass < 2; pass++) {
-        const uint64_t blocks = pass == 0 ? (n_keys_max + kReduceSeg - 1) / kReduceSeg : 1;
-        ReduceArgs r;
-        r.in = in; r.in_count = ctrl + in_slot; r.out = out; r.out_count = ctrl + out_slot;
-        r.k = k; r.final = blocks <= 1; r.first = first; r.idx_map = d_idx_map;
-        r.seg = blocks <= 1 ? 0xFFFFFFFFu : (unsigned int)kReduceSeg;
-        r.topk_idx = d_topk_idx; r.topk_score = d_topk_score; r.topk_count = d_topk_count;
-        reduce_kernel<<<(unsigned int)(blocks < 1 ? 1 : blocks), kReduceThreads, 0, st>>>(r);
+    // pass 1 spreads a long list over blocks of kReduceSeg keys; whatever it leaves (at most k keys per block) is
+    // finished by one block; a short list goes to that block directly
+    ReduceArgs r;
+    r.in = in; r.in_count = ctrl + 1; r.out = out; r.out_count = ctrl + 2;
+    r.in0 = in; r.in0_count = ctrl + 1;
+    r.k = k; r.final = 0; r.first = first; r.idx_map = d_idx_map;
+    r.seg = (unsigned int)kReduceSeg;
+    r.topk_idx = d_topk_idx; r.topk_score = d_topk_score; r.topk_count = d_topk_count;
+    const uint64_t blocks = (n_keys_max + kReduceSeg - 1) / kReduceSeg;
+    if (n_keys_max > (uint64_t)kFastKeys) {
+        reduce_kernel<<<(unsigned int)blocks, kReduceThreads, 0, st>>>(r);
         count_launch();
         (*n_kernels)++;
         PF_CUDA_TRY(cudaGetLastError(), "reduce_kernel launch");
-        if (r.final) return PF_OK;
-        unsigned long long *t = in; in = out; out = t;
-        in_slot = 2;
-        out_slot = 3;
     }
-    return PF_EINVAL;
+    r.in = out; r.in_count = ctrl + 2; r.final = 1;
+    PF_CUDA_TRY(cudaFuncSetAttribute(reduce_final_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (kFastKeys + kTopkCap) * 8), "reduce_final_kernel smem");
+    reduce_final_kernel<<<1, kReduceThreads, (kFastKeys + kTopkCap) * 8, st>>>(r);
+    count_launch();
+    (*n_kernels)++;
+    PF_CUDA_TRY(cudaGetLastError(), "reduce_final_kernel launch");
+    return PF_OK;
 }
 
 // ------------------------------------------------------------------ merge of two finished top-k lists

@@ -103,7 +103,7 @@ __device__ __forceinline__ void for_each_eligible16(const DevPlan &P, const int3
     }
 }
 
-constexpr int kSelTiles = 16;                              // tiles of 256 x 16 candidates per block
+constexpr int kSelTiles = 4;                               // tiles of 256 x 16 candidates per block
 constexpr uint64_t kSelTile = (uint64_t)kSelThreads * 16;  // candidates per tile
 
 // Load this thread's group of every tile of the block's chunk before any of them is looked at, so the
