@@ -35,9 +35,9 @@ K_TOP, S_MAX, K_SIM, JITTER_SEED = 1024, 1_000_000, 100, 4
 BYTES_PER_CANDIDATE = 13          # dense outputs: reason u8 + tput f32 + mem i64
 FALLBACK_HBM_GBS = 6650.0         # used only when MEASURED_PEAKS.json is absent
 # dram__bytes_read.sum + dram__bytes_write.sum of one score_kernel launch on this workload: captured with ncu
-# on a 50,000,000-candidate slice (599.0 MB) and scaled by candidates to the full space (the ncu summary is
+# on a 50,000,000-candidate slice (604.2 MB) and scaled by candidates to the full space (the ncu summary is
 # kept under profiles/).  Below the algorithmic bytes because dirty lines still sit in L2 when the kernel ends.
-SCORE_KERNEL_DRAM_BYTES = int(598.990336e6 * 179_908_608 / 50_000_000)
+SCORE_KERNEL_DRAM_BYTES = int(604.236800e6 * 179_908_608 / 50_000_000)
 
 
 def _measured_hbm():
