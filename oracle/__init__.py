@@ -20,7 +20,7 @@ _HDR = os.path.join(_HERE, "planfront_oracle.h")
 _LIB = os.path.join(_HERE, "liborc.so")
 _LIB_COUNT = os.path.join(_HERE, "liborc_count.so")
 
-MAX_SCHED, MAX_KERN, NBUCKET, MAX_AXES = 8, 16, 8, 10
+MAX_SCHED, MAX_KERN, NBUCKET, MAX_AXES = 8, 16, 8, 11
 
 REASON_NAMES = {0: "FEASIBLE", 1: "WORLD", 2: "TP", 3: "EP", 4: "BATCH", 5: "VSTAGE", 6: "LAYERS",
                 7: "MICROBATCH", 8: "KERNEL_MISSING", 9: "UNMAPPED_SCHEDULE", 10: "OVERLAP_PRECOND",
@@ -55,7 +55,8 @@ class Model(C.Structure):
 
 class Cluster(C.Structure):
     _fields_ = [(n, i64) for n in ("G", "budget_bytes", "reserved_bytes", "caps")] + \
-               [(n, f64) for n in ("peak_flops", "hbm_bw", "bw_intra", "bw_inter", "alpha_intra", "alpha_inter")]
+               [(n, f64) for n in ("peak_flops", "hbm_bw", "bw_intra", "bw_inter", "alpha_intra", "alpha_inter",
+                                   "bw_host")]
 
 
 class Workload(C.Structure):
@@ -65,7 +66,7 @@ class Workload(C.Structure):
 
 class Consts(C.Structure):
     _fields_ = [(n, f64) for n in ("eff_dense", "bwd_factor", "dp_overlap_frac", "dualpipe_startup_div",
-                                   "step_overhead")]
+                                   "step_overhead", "offload_overlap_penalty")]
 
 
 class Sched(C.Structure):
@@ -99,10 +100,11 @@ class Derived(C.Structure):
 
 
 class Detail(C.Structure):
-    _fields_ = [(n, i64) for n in ("kv", "rec", "sched", "mb", "v", "ep", "pp", "tp", "dp", "world", "chunk",
+    _fields_ = [(n, i64) for n in ("kv", "rec", "sched", "mb", "v", "ep", "pp", "tp", "dp", "world", "shard", "chunk",
                                    "batch", "dpa", "scen", "kind", "ov", "v_eff", "m", "t", "Q", "Lc", "Ls",
                                    "edp", "m_e", "bucket", "bucket_pre", "N_dense", "N_exp", "bytes_w",
-                                   "bytes_g", "bytes_o_dense", "bytes_o_expert", "bytes_o", "bytes_a", "mem")] + \
+                                   "bytes_g", "bytes_o_dense", "bytes_o_expert", "bytes_o", "bytes_a", "bytes_buf",
+                                   "mem")] + \
                [(n, f64) for n in ("cF", "cB", "rc", "tpc", "a2a", "xF", "xB", "F_l", "B_l", "headF", "F", "B",
                                    "p", "T_pipe", "T_dp", "T_opt", "T_step", "T_dec", "T_pre", "tput_unpriced",
                                    "tput")] + [("reason", i64)]

@@ -183,6 +183,12 @@ static double t_allreduce(int64_t n, double bytes, link_t lk)
     if (n <= 1) return 0.0;
     return 2.0 * (double)(n - 1) / (double)n * bytes / lk.bw + 2.0 * (double)clog2(n) * lk.alpha;
 }
+/* all-gather of `bytes` (the gathered size); a reduce-scatter has the same alpha-beta form */
+static double t_allgather(int64_t n, double bytes, link_t lk)
+{
+    if (n <= 1) return 0.0;
+    return (double)(n - 1) / (double)n * bytes / lk.bw + (double)clog2(n) * lk.alpha;
+}
 static double t_alltoall(int64_t n, double bytes, link_t lk)
 {
     if (n <= 1) return 0.0;
@@ -197,12 +203,14 @@ static int eval_train(const orc_problem_t *pb, const orc_derived_t *dv, uint64_t
     const orc_cluster_t *C = &pb->cluster;
     const orc_rules_t *R = &pb->rules;
     const orc_consts_t *K0 = &pb->consts;
-    int64_t val[ORC_MAX_AXES];
+    int64_t val[ORC_MAX_AXES] = {0};
     decode(&pb->axes, idx, val);
     int64_t kv = val[0], rec = val[1], s = val[2], mb = val[3], v = val[4];
     int64_t ep = val[5], pp = val[6], tp = val[7], dp = val[8], world = val[9];
+    /* the sharding dimension is orthogonal to the layout and defaults to zero1 (Sec. 3.1) */
+    int64_t shard = pb->axes.n_axes > 10 ? val[10] : ORC_SHARD_ZERO1;
     o->kv = kv; o->rec = rec; o->sched = s; o->mb = mb; o->v = v;
-    o->ep = ep; o->pp = pp; o->tp = tp;
+    o->ep = ep; o->pp = pp; o->tp = tp; o->shard = shard;
 
     /* rule 1 WORLD: data parallelism is derived from the world size (Sec. 3.1) unless both are
      * enumerated, in which case the product must match; whole nodes beyond one node */
@@ -296,6 +304,7 @@ static int eval_train(const orc_problem_t *pb, const orc_derived_t *dv, uint64_t
     OPS(3 + 6 + 7 + 7 + 4 + 9 + 2 + 4 + 6 + 1 + 5, 0); /* pm, emb, N_dense, N_exp, w+g, o, A_tok, A_layer, units,
                                                           bytes_a, sum and gate */
     if (rec == ORC_REC_FULL) OPS(6, 0);
+    if (pb->axes.n_axes > 10) OPS(val[10] == ORC_SHARD_FSDP ? 16 : 4, val[10] == ORC_SHARD_FSDP ? 22 : val[10] ? 4 : 0);
     if ((pp == 1 || kind == ORC_KIND_DUALPIPE) && M->count_embeddings) OPS(9, 0);
     int64_t pm = (kind == ORC_KIND_DUALPIPE && pp > 1) ? 2 : 1; /* two stage copies per rank */
     int64_t emb = cdiv(dv->P_emb, tp) * ((pp == 1 || kind == ORC_KIND_DUALPIPE) ? 2 : 1);
@@ -305,9 +314,23 @@ static int eval_train(const orc_problem_t *pb, const orc_derived_t *dv, uint64_t
     int64_t bytes_g = M->gb * (N_dense + N_exp);
     /* distributed optimizer: dense shard over dp, expert shard over the expert-DP group
      * (Sec. 5 RQ1: the expert optimizer state is ep-invariant) */
+    int64_t n_shard = cdiv(N_dense, dp) + cdiv(N_exp, edp); /* parameters whose state this rank owns */
     int64_t bytes_o_dense = M->ob * cdiv(N_dense, dp);
     int64_t bytes_o_expert = M->ob * cdiv(N_exp, edp);
     int64_t bytes_o = bytes_o_dense + bytes_o_expert;
+    int64_t bytes_buf = 0;
+    if (shard == ORC_SHARD_ZERO1_OFFLOAD) {
+        /* the optimizer state lives in host memory */
+        bytes_o_dense = bytes_o_expert = bytes_o = 0;
+    } else if (shard == ORC_SHARD_FSDP) {
+        /* parameters and gradients are sharded like the optimizer state; the all-gather working buffer
+         * (boundary B7 of the paper's catalogue) holds the unsharded parameters of the layer in use and of
+         * the one being prefetched */
+        bytes_w = M->wb * n_shard;
+        bytes_g = M->gb * n_shard;
+        int64_t P_layer = cdiv(dv->P_dl, tp) + dv->P_rt + (M->E / ep) * cdiv(dv->P_e, etp);
+        bytes_buf = imin(2, pm * Ls) * M->wb * P_layer;
+    }
     int64_t A_tok = rec == ORC_REC_NONE ? dv->a_full : rec == ORC_REC_SELECTIVE ? dv->a_sel : dv->a_ckpt;
     int64_t A_layer = cdiv(t * A_tok, tp);
     int64_t units;
@@ -321,10 +344,10 @@ static int eval_train(const orc_problem_t *pb, const orc_derived_t *dv, uint64_t
     if (rec == ORC_REC_FULL) bytes_a += cdiv(t * dv->a_full, tp); /* the layer being recomputed */
     if ((pp == 1 || kind == ORC_KIND_DUALPIPE) && M->count_embeddings)
         bytes_a += 4 * cdiv(t * M->vocab, tp); /* fp32 logits where the head lives */
-    int64_t mem = bytes_w + bytes_g + bytes_o + bytes_a + C->reserved_bytes;
+    int64_t mem = bytes_w + bytes_g + bytes_o + bytes_buf + bytes_a + C->reserved_bytes;
     o->N_dense = N_dense; o->N_exp = N_exp; o->bytes_w = bytes_w; o->bytes_g = bytes_g;
     o->bytes_o_dense = bytes_o_dense; o->bytes_o_expert = bytes_o_expert; o->bytes_o = bytes_o;
-    o->bytes_a = bytes_a; o->mem = mem;
+    o->bytes_a = bytes_a; o->bytes_buf = bytes_buf; o->mem = mem;
 
     /* rule 11 MEMORY: the gate rejects when the peak exceeds the budget (Sec. 5 RQ1: 79.39 > 72) */
     if (mem > C->budget_bytes) return o->reason = ORC_R_MEMORY;
@@ -349,7 +372,8 @@ static int eval_train(const orc_problem_t *pb, const orc_derived_t *dv, uint64_t
         rc = cF;
     double tpc = 2.0 * t_allreduce(tp, (double)(M->ab * t * M->H), link_of(C, tp));
     double a2a = 2.0 * t_alltoall(ep, (double)(M->ab * t * M->K * M->H) / tpd, link_of(C, tp * ep));
-    double h = ov ? pb->sched[s].hide_frac : 0.0;
+    /* the hiding benefit is conditioned out in the offload domain (Sec. 5 RQ2) */
+    double h = (ov && shard != ORC_SHARD_ZERO1_OFFLOAD) ? pb->sched[s].hide_frac : 0.0;
     double xF = a2a - fmin(h * a2a, cF);
     double xB = a2a - fmin(h * a2a, cB + rc);
     double F_l = cF + tpc + xF;
@@ -374,6 +398,16 @@ static int eval_train(const orc_problem_t *pb, const orc_derived_t *dv, uint64_t
     double T_dp = t_allreduce(dp, (double)((M->gb + M->wb) * N_dense), ldp) +
                   t_allreduce(edp, (double)((M->gb + M->wb) * N_exp), ldp);
     double T_opt = 2.0 * (double)bytes_o / C->hbm_bw;
+    if (shard == ORC_SHARD_ZERO1_OFFLOAD) {
+        /* the step runs on the host: the shard's gradients go down and its updated weights come back */
+        T_opt = (double)((M->gb + M->wb) * n_shard) / C->bw_host;
+    } else if (shard == ORC_SHARD_FSDP) {
+        /* per microbatch the parameters are gathered for the forward and again for the backward pass and the
+         * gradients are reduce-scattered; this replaces the gradient all-reduce of the replicated regimes */
+        double ag = t_allgather(dp, (double)(M->wb * N_dense), ldp) + t_allgather(edp, (double)(M->wb * N_exp), ldp);
+        double rs = t_allgather(dp, (double)(M->gb * N_dense), ldp) + t_allgather(edp, (double)(M->gb * N_exp), ldp);
+        T_dp = (double)m * (2.0 * ag + rs);
+    }
     double T_step = T_pipe + (1.0 - K0->dp_overlap_frac) * T_dp + T_opt + K0->step_overhead;
 
     /* ---- pricing: throughput / (1 + frac) on the plans that take the taxed path ---- */
@@ -381,6 +415,8 @@ static int eval_train(const orc_problem_t *pb, const orc_derived_t *dv, uint64_t
     o->tput_unpriced = tput;
     if (!kn->is_native) tput = tput / (1.0 + kn->patch_ovh);
     if (ov) tput = tput / (1.0 + pb->sched[s].sched_ovh);
+    /* the contention penalty prices exactly the offloaded-and-overlapped plans (Sec. 3.2) */
+    if (ov && shard == ORC_SHARD_ZERO1_OFFLOAD) tput = tput / (1.0 + K0->offload_overlap_penalty);
 
     o->cF = cF; o->cB = cB; o->rc = rc; o->tpc = tpc; o->a2a = a2a; o->xF = xF; o->xB = xB;
     o->F_l = F_l; o->B_l = B_l; o->headF = headF; o->F = F; o->B = B; o->p = p;
@@ -398,7 +434,7 @@ static int eval_serve(const orc_problem_t *pb, const orc_derived_t *dv, uint64_t
     const orc_model_t *M = &pb->model;
     const orc_cluster_t *C = &pb->cluster;
     const orc_consts_t *K0 = &pb->consts;
-    int64_t val[ORC_MAX_AXES];
+    int64_t val[ORC_MAX_AXES] = {0};
     decode(&pb->axes, idx, val);
     int64_t kv = val[0], Cc = val[1], Bd = val[2], dpa = val[3], ep = val[4], tp = val[5], sc = val[6];
     int64_t world = pb->workload.world;
@@ -630,7 +666,7 @@ uint64_t orc_topk_list(const uint64_t *idx, const double *score, uint64_t n, uin
 static int in_sim_domain(const orc_problem_t *pb, uint64_t idx)
 {
     if (pb->workload.phase != 0) return 0;
-    int64_t val[ORC_MAX_AXES];
+    int64_t val[ORC_MAX_AXES] = {0};
     decode(&pb->axes, idx, val);
     int64_t s = val[2], v = val[4], pp = val[6];
     int64_t kind = pb->sched[s].kind;
@@ -1010,6 +1046,7 @@ int orc_simulate(const orc_problem_t *pb, uint64_t idx, uint32_t seed, double *t
     double tput = (double)(pb->workload.gbs * M->seq) / (T_step * (double)d.world);
     if (!pb->kern[d.kv].is_native) tput = tput / (1.0 + pb->kern[d.kv].patch_ovh);
     if (d.ov) tput = tput / (1.0 + pb->sched[d.sched].sched_ovh);
+    if (d.ov && d.shard == ORC_SHARD_ZERO1_OFFLOAD) tput = tput / (1.0 + K0->offload_overlap_penalty);
     *tput_sim = tput;
     return ORC_SIM_OK;
 }

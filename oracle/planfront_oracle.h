@@ -40,7 +40,7 @@ extern "C" {
 #define ORC_MAX_SCHED 8
 #define ORC_MAX_KERN 16
 #define ORC_NBUCKET 8
-#define ORC_MAX_AXES 10
+#define ORC_MAX_AXES 11
 #define ORC_MAX_RANKS 32   /* simulator domain: pp <= 32 */
 #define ORC_MAX_V 8        /* simulator domain: virtual stages per rank <= 8 */
 #define ORC_SIM_WINDOW 64  /* simulated microbatches per step at most */
@@ -64,6 +64,9 @@ enum {
 
 enum { ORC_KIND_1F1B = 0, ORC_KIND_INTERLEAVED = 1, ORC_KIND_DUALPIPE = 2 };
 enum { ORC_REC_NONE = 0, ORC_REC_SELECTIVE = 1, ORC_REC_FULL = 2 };
+/* memory sharding (Sec. 3.1, memory plan): optimizer state sharded / and kept in host memory / parameters and
+ * gradients sharded as well */
+enum { ORC_SHARD_ZERO1 = 0, ORC_SHARD_ZERO1_OFFLOAD = 1, ORC_SHARD_FSDP = 2 };
 enum { ORC_SIM_OK = 0, ORC_SIM_UNSUPPORTED = 1, ORC_SIM_STALL = 2 };
 
 typedef struct {
@@ -83,6 +86,7 @@ typedef struct {
     int64_t reserved_bytes;
     int64_t caps; /* bit 0: fp8, bit 1: device-initiated communication */
     double peak_flops, hbm_bw, bw_intra, bw_inter, alpha_intra, alpha_inter;
+    double bw_host; /* host link of one GPU, bytes/s (offloaded optimizer) */
 } orc_cluster_t;
 
 typedef struct {
@@ -96,6 +100,7 @@ typedef struct {
 
 typedef struct {
     double eff_dense, bwd_factor, dp_overlap_frac, dualpipe_startup_div, step_overhead;
+    double offload_overlap_penalty; /* realization tax of an offloaded-and-overlapped plan (Sec. 3.2) */
 } orc_consts_t;
 
 typedef struct {
@@ -116,7 +121,7 @@ typedef struct {
 } orc_rules_t;
 
 /* axis value lists, least-significant digit first.
- * train: kv, rec, sched, mb, v, ep, pp, tp, dp, world   (10 axes)
+ * train: kv, rec, sched, mb, v, ep, pp, tp, dp, world [, shard]   (10 or 11 axes; no shard axis = zero1)
  * serve: kv, chunk, batch, dpa, ep, tp, scen             (7 axes) */
 typedef struct {
     int64_t n_axes;
@@ -147,12 +152,12 @@ typedef struct {
 /* everything computed for one candidate; unfilled parts stay 0 */
 typedef struct {
     /* decoded tuple (train names; serve: chunk->mb slot unused, see fields below) */
-    int64_t kv, rec, sched, mb, v, ep, pp, tp, dp, world;
+    int64_t kv, rec, sched, mb, v, ep, pp, tp, dp, world, shard;
     int64_t chunk, batch, dpa, scen; /* serve */
     /* derived integers */
     int64_t kind, ov, v_eff, m, t, Q, Lc, Ls, edp, m_e, bucket, bucket_pre;
     /* memory terms */
-    int64_t N_dense, N_exp, bytes_w, bytes_g, bytes_o_dense, bytes_o_expert, bytes_o, bytes_a, mem;
+    int64_t N_dense, N_exp, bytes_w, bytes_g, bytes_o_dense, bytes_o_expert, bytes_o, bytes_a, bytes_buf, mem;
     /* time terms */
     double cF, cB, rc, tpc, a2a, xF, xB, F_l, B_l, headF, F, B, p, T_pipe, T_dp, T_opt, T_step;
     double T_dec, T_pre; /* serve */

@@ -45,8 +45,9 @@ def table_draws(seed: int, n_kern: int, n_sched: int, p_avail: float):
 
 
 def _consts():
+    # offload_overlap_penalty: the measured contention penalty the paper reports (0.0271)
     return dict(eff_dense=f32(0.5), bwd_factor=f32(2.0), dp_overlap_frac=f32(0.5),
-                dualpipe_startup_div=f32(8.0), step_overhead=f32(0.0))
+                dualpipe_startup_div=f32(8.0), step_overhead=f32(0.0), offload_overlap_penalty=f32(0.0271))
 
 
 # hidden fraction of the expert all-to-all per schedule class when overlap is on
@@ -71,11 +72,11 @@ def _model(**kw):
     return m
 
 
-def _cluster(G, budget_bytes, peak, hbm_bw, bw_intra, bw_inter, a_intra, a_inter, caps=0):
+def _cluster(G, budget_bytes, peak, hbm_bw, bw_intra, bw_inter, a_intra, a_inter, caps=0, bw_host=55e9):
     # budget_bytes: usable HBM per modeled GPU (0.9 of a 24 GB / 80 GB part), given as integer bytes
     return dict(G=G, budget_bytes=budget_bytes, reserved_bytes=0, caps=caps,
                 peak_flops=f32(peak), hbm_bw=f32(hbm_bw), bw_intra=f32(bw_intra), bw_inter=f32(bw_inter),
-                alpha_intra=f32(a_intra), alpha_inter=f32(a_inter))
+                alpha_intra=f32(a_intra), alpha_inter=f32(a_inter), bw_host=f32(bw_host))
 
 
 def _tiny():
