@@ -37,7 +37,7 @@ extern "C" {
 #endif
 
 #define PF_VERSION 100
-#define PF_MAX_AXES 10
+#define PF_MAX_AXES 11
 #define PF_MAX_AXIS_LEN 4096
 #define PF_MAX_SCHED 8
 #define PF_MAX_KERN 16
@@ -81,6 +81,9 @@ enum {
 
 enum { PF_KIND_1F1B = 0, PF_KIND_INTERLEAVED = 1, PF_KIND_DUALPIPE = 2 };
 enum { PF_REC_NONE = 0, PF_REC_SELECTIVE = 1, PF_REC_FULL = 2 };
+/* memory sharding (Sec. 3.1, memory plan): optimizer state sharded over the data-parallel groups; the same with
+ * the state kept in host memory; parameters and gradients sharded as well (with an all-gather working buffer) */
+enum { PF_SHARD_ZERO1 = 0, PF_SHARD_ZERO1_OFFLOAD = 1, PF_SHARD_FSDP = 2 };
 enum { PF_PHASE_TRAIN = 0, PF_PHASE_SERVE = 1 };
 enum { PF_CAP_FP8 = 1, PF_CAP_DEVICE_COMM = 2 };
 /* per-survivor simulator status */
@@ -103,6 +106,7 @@ typedef struct {
     int64_t budget_bytes;         /* usable HBM per GPU: the memory gate rejects mem > budget (Sec. 5 RQ1) */
     int64_t reserved_bytes;       /* added to every candidate's memory */
     float peak_flops, hbm_bw, bw_intra, bw_inter, alpha_intra, alpha_inter;
+    float bw_host;                /* host link of one GPU, bytes/s: carries an offloaded optimizer step */
 } pf_cluster_t;
 
 typedef struct {
@@ -115,7 +119,7 @@ typedef struct {
 } pf_workload_t;
 
 typedef struct {
-    int32_t n_axes;               /* 10 (train) or 7 (serve) */
+    int32_t n_axes;               /* 10 or 11 (train: 11 with the sharding axis last) or 7 (serve) */
     int32_t len[PF_MAX_AXES];     /* 1 .. PF_MAX_AXIS_LEN */
     const int32_t *val[PF_MAX_AXES]; /* host value lists */
 } pf_axes_t;
@@ -140,6 +144,7 @@ typedef struct {
 
 typedef struct {
     float eff_dense, bwd_factor, dp_overlap_frac, dualpipe_startup_div, step_overhead;
+    float offload_overlap_penalty; /* realization tax of offloaded-and-overlapped plans, tput / (1 + frac) (Sec. 3.2) */
     int32_t n_sched;
     pf_sched_t sched[PF_MAX_SCHED];
     int32_t n_kern;
@@ -157,6 +162,7 @@ typedef struct {
 typedef struct {
     int32_t kv, rec, sched, mb, v, ep, pp, tp, dp, world; /* train (dp/world as listed, before derivation) */
     int32_t chunk, batch, dpa, scen;                      /* serve */
+    int32_t shard;                                        /* train: PF_SHARD_* (zero1 when the axis is absent) */
 } pf_tuple_t;
 
 typedef struct pf_plan pf_plan_t;
@@ -170,8 +176,11 @@ const char *pf_last_cuda_error(void);
 /* Build a plan space (Sec. 3.1: one normalized tuple carries every knob; Sec. 3.3: enumeration).
  * Validates the specs, derives the candidate-independent constants (parameter, activation and FLOP
  * counts per layer; radices; schedule-order tables for the simulator) and uploads them.
+ * A training space may carry the memory-sharding dimension (Sec. 3.1, memory plan) as an 11th, most significant
+ * axis with values PF_SHARD_*; without it every plan is zero1.  Such a space needs cluster->bw_host > 0.
  * Errors: PF_EINVAL (NULL pointer, phase/axis-count mismatch, table index out of range, both dp and
- * world derived), PF_ERANGE (axis length, value range, space size), PF_ECUDA. */
+ * world derived, a sharding value outside PF_SHARD_*), PF_ERANGE (axis length, value range, space size),
+ * PF_ECUDA. */
 int pf_plan_create(const pf_model_t *model, const pf_cluster_t *cluster, const pf_workload_t *workload,
                    const pf_axes_t *axes, const pf_tables_t *tables, const pf_rules_t *rules, pf_plan_t **out);
 void pf_plan_destroy(pf_plan_t *plan);

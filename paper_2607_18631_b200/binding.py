@@ -16,7 +16,7 @@ import numpy as np
 HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(HERE, "libplanfront.so")
 
-MAX_AXES, MAX_SCHED, MAX_KERN, NBUCKET, K_MAX = 10, 8, 16, 8, 1024
+MAX_AXES, MAX_SCHED, MAX_KERN, NBUCKET, K_MAX = 11, 8, 16, 8, 1024
 PF_OK, PF_EINVAL, PF_ERANGE, PF_EWORKSPACE, PF_ECUDA, PF_EUNSUPPORTED = 0, -1, -2, -3, -4, -5
 UINT64_MAX = 0xFFFFFFFFFFFFFFFF
 
@@ -38,7 +38,8 @@ class PfModel(C.Structure):
 
 class PfCluster(C.Structure):
     _fields_ = [("G", i32), ("caps", u32), ("budget_bytes", i64), ("reserved_bytes", i64)] + \
-               [(n, f32) for n in ("peak_flops", "hbm_bw", "bw_intra", "bw_inter", "alpha_intra", "alpha_inter")]
+               [(n, f32) for n in ("peak_flops", "hbm_bw", "bw_intra", "bw_inter", "alpha_intra", "alpha_inter",
+                                   "bw_host")]
 
 
 class PfWorkload(C.Structure):
@@ -61,7 +62,7 @@ class PfKern(C.Structure):
 
 class PfTables(C.Structure):
     _fields_ = [(n, f32) for n in ("eff_dense", "bwd_factor", "dp_overlap_frac", "dualpipe_startup_div",
-                                   "step_overhead")] + \
+                                   "step_overhead", "offload_overlap_penalty")] + \
                [("n_sched", i32), ("sched", PfSched * MAX_SCHED), ("n_kern", i32), ("kern", PfKern * MAX_KERN)]
 
 
@@ -72,7 +73,7 @@ class PfRules(C.Structure):
 
 class PfTuple(C.Structure):
     _fields_ = [(n, i32) for n in ("kv", "rec", "sched", "mb", "v", "ep", "pp", "tp", "dp", "world", "chunk",
-                                   "batch", "dpa", "scen")]
+                                   "batch", "dpa", "scen", "shard")]
 
 
 class PlanfrontError(RuntimeError):
@@ -238,7 +239,7 @@ class Plan:
         cl = PfCluster(G=int(c["G"]), caps=int(c["caps"]), budget_bytes=int(c["budget_bytes"]),
                        reserved_bytes=int(c["reserved_bytes"]),
                        **{n: float(c[n]) for n in ("peak_flops", "hbm_bw", "bw_intra", "bw_inter", "alpha_intra",
-                                                   "alpha_inter")})
+                                                   "alpha_inter")}, bw_host=float(c.get("bw_host", 0.0)))
         w = cfg["workload"]
         sp = np.asarray(w.get("scen_P", []), dtype=np.int32)
         so = np.asarray(w.get("scen_O", []), dtype=np.int32)
@@ -253,7 +254,8 @@ class Plan:
             ax.len[a] = len(arr)
             ax.val[a] = arr.ctypes.data_as(C.POINTER(i32))
         tb = PfTables(**{n: float(cfg["consts"][n]) for n in ("eff_dense", "bwd_factor", "dp_overlap_frac",
-                                                               "dualpipe_startup_div", "step_overhead")})
+                                                               "dualpipe_startup_div", "step_overhead")},
+                      offload_overlap_penalty=float(cfg["consts"].get("offload_overlap_penalty", 0.0)))
         tb.n_sched = len(cfg["sched"])
         for i, s in enumerate(cfg["sched"]):
             tb.sched[i] = PfSched(kind=int(s["kind"]), overlap=int(s["overlap"]), mapped=int(s["mapped"]),

@@ -159,7 +159,8 @@ extern "C" int pf_plan_create(const pf_model_t *model, const pf_cluster_t *clust
     *out = nullptr;
     const int phase = workload->phase;
     if (phase != PF_PHASE_TRAIN && phase != PF_PHASE_SERVE) return PF_EINVAL;
-    const int want_axes = phase == PF_PHASE_TRAIN ? 10 : 7;
+    // training spaces may carry the memory-sharding axis as an 11th, most significant one
+    const int want_axes = phase == PF_PHASE_TRAIN ? (axes->n_axes == 11 ? 11 : 10) : 7;
     if (axes->n_axes != want_axes) return PF_EINVAL;
     if (tables->n_sched < 1 || tables->n_sched > PF_MAX_SCHED || tables->n_kern < 1 || tables->n_kern > PF_MAX_KERN)
         return PF_EINVAL;
@@ -171,6 +172,7 @@ extern "C" int pf_plan_create(const pf_model_t *model, const pf_cluster_t *clust
     if (cluster->G <= 0 || cluster->budget_bytes < 0 || cluster->reserved_bytes < 0) return PF_EINVAL;
     if (!(cluster->peak_flops > 0) || !(cluster->hbm_bw > 0) || !(cluster->bw_intra > 0) || !(cluster->bw_inter > 0))
         return PF_EINVAL;
+    if (want_axes == 11 && (!(cluster->bw_host > 0) || !(tables->offload_overlap_penalty > -1.f))) return PF_EINVAL;
     if (!(tables->eff_dense > 0) || !(tables->dualpipe_startup_div > 0)) return PF_EINVAL;
     if (phase == PF_PHASE_TRAIN && workload->gbs <= 0) return PF_EINVAL;
     if (phase == PF_PHASE_SERVE) {
@@ -205,6 +207,7 @@ extern "C" int pf_plan_create(const pf_model_t *model, const pf_cluster_t *clust
         if (!in_range(3, 1, 1 << 16) || !in_range(4, 0, 255)) return PF_ERANGE;
         if (!in_range(5, 1, kDeg) || !in_range(6, 1, kDeg) || !in_range(7, 1, kDeg)) return PF_ERANGE;
         if (!in_range(8, 0, kDeg) || !in_range(9, 0, kDeg)) return PF_ERANGE;
+        if (want_axes == 11 && !in_range(10, PF_SHARD_ZERO1, PF_SHARD_FSDP)) return PF_EINVAL;
         // "derived" is a whole-axis statement: the list {0}
         for (int a = 8; a <= 9; a++) {
             bool has0 = false;
@@ -250,6 +253,12 @@ extern "C" int pf_plan_create(const pf_model_t *model, const pf_cluster_t *clust
         d.val_off[a] = off;
         memcpy(p->h_vals + off, axes->val[a], sizeof(int32_t) * (size_t)axes->len[a]);
         off += axes->len[a];
+    }
+    // axes the space does not have decode as a single digit 0 that reads the first packed value
+    for (int a = want_axes; a < PF_MAX_AXES; a++) {
+        p->axis_len[a] = 1;
+        d.radix[a] = 1;
+        d.val_off[a] = 0;
     }
 
     // slab = longest axis prefix whose product stays under a size that still leaves a few blocks per SM
@@ -309,6 +318,7 @@ extern "C" int pf_plan_create(const pf_model_t *model, const pf_cluster_t *clust
     d.peak_flops = cluster->peak_flops; d.hbm_bw = cluster->hbm_bw;
     d.bw_intra = cluster->bw_intra; d.bw_inter = cluster->bw_inter;
     d.alpha_intra = cluster->alpha_intra; d.alpha_inter = cluster->alpha_inter;
+    d.bw_host = cluster->bw_host; d.offload_overlap_penalty = tables->offload_overlap_penalty;
     d.gbs = workload->gbs; d.world = workload->world; d.n_scen = phase == PF_PHASE_SERVE ? workload->n_scen : 0;
     d.eff_dense = tables->eff_dense; d.bwd_factor = tables->bwd_factor; d.dp_overlap_frac = tables->dp_overlap_frac;
     d.dualpipe_startup_div = tables->dualpipe_startup_div; d.step_overhead = tables->step_overhead;
@@ -467,6 +477,7 @@ extern "C" int pf_decode(const pf_plan_t *p, uint64_t idx, pf_tuple_t *out)
     if (p->dev.phase == PF_PHASE_TRAIN) {
         out->kv = v[0]; out->rec = v[1]; out->sched = v[2]; out->mb = v[3]; out->v = v[4];
         out->ep = v[5]; out->pp = v[6]; out->tp = v[7]; out->dp = v[8]; out->world = v[9];
+        out->shard = p->dev.n_axes > 10 ? v[10] : PF_SHARD_ZERO1;
     } else {
         out->kv = v[0]; out->chunk = v[1]; out->batch = v[2]; out->dpa = v[3];
         out->ep = v[4]; out->tp = v[5]; out->scen = v[6];

@@ -51,6 +51,13 @@ __device__ __forceinline__ float t_allreduce(i64 n, float bytes, Link lk)
     float fn = (float)n;
     return fdiv(2.f * (fn - 1.f) * bytes, fn * lk.bw) + 2.f * ceil_log2f(n) * lk.alpha;
 }
+// all-gather of `bytes` (the gathered size); a reduce-scatter has the same form
+__device__ __forceinline__ float t_allgather(i64 n, float bytes, Link lk)
+{
+    if (n <= 1) return 0.f;
+    const float nf = (float)n;
+    return fdiv((nf - 1.f) * bytes, nf * lk.bw) + ceil_log2f(n) * lk.alpha;
+}
 __device__ __forceinline__ float t_alltoall(i64 n, float bytes, Link lk)
 {
     if (n <= 1) return 0.f;
@@ -62,6 +69,7 @@ __device__ __forceinline__ float t_alltoall(i64 n, float bytes, Link lk)
 
 struct TrainTuple {
     int kv, rec, s, mb, v, ep, pp, tp, dp, world;  // dp / world as listed (0 = derived)
+    int sh = PF_SHARD_ZERO1;                       // memory sharding (zero1 when the space has no such axis)
 };
 
 // Quantities the rules derive on the way, kept for the memory / time models and the simulator.
@@ -162,7 +170,7 @@ __device__ __forceinline__ int train_plan_rules(const DevPlan &P, const TrainTup
 }
 
 struct TrainMem {
-    i64 N_dense, N_exp, bytes_o, mem;
+    i64 N_dense, N_exp, n_shard, bytes_o, mem;
 };
 
 // Peak bytes on rank 0 (most in-flight activations): weights + gradients + sharded optimizer state
@@ -179,8 +187,17 @@ __device__ __forceinline__ void train_memory(const DevPlan &P, const TrainTuple 
     const i64 etp = P.ep_scope ? 1 : tp;
     M.N_dense = copies * Ls * (cdiv64(P.P_dl, tp) + P.P_rt) + emb;
     M.N_exp = copies * Ls * (i64)(P.E / c.ep) * cdiv64(P.P_e, etp);
-    const i64 n_all = M.N_dense + M.N_exp;
-    M.bytes_o = (i64)P.ob * (cdiv64(M.N_dense, (i64)D.dp) + cdiv64(M.N_exp, (i64)D.edp));
+    // parameters whose optimizer state this rank owns: dense over dp, experts over the expert-DP group
+    M.n_shard = cdiv64(M.N_dense, (i64)D.dp) + cdiv64(M.N_exp, (i64)D.edp);
+    // zero1: whole parameters and gradients, sharded state; offload: the state lives in host memory; fsdp:
+    // parameters and gradients sharded like the state, plus the all-gather buffer of two layers' parameters
+    i64 n_all = M.N_dense + M.N_exp, buf = 0;
+    M.bytes_o = c.sh == PF_SHARD_ZERO1_OFFLOAD ? 0 : (i64)P.ob * M.n_shard;
+    if (c.sh == PF_SHARD_FSDP) {
+        n_all = M.n_shard;
+        const i64 p_layer = cdiv64(P.P_dl, tp) + P.P_rt + (i64)(P.E / c.ep) * cdiv64(P.P_e, etp);
+        buf = min((i64)2, copies * Ls) * (i64)P.wb * p_layer;
+    }
     const i64 a_tok = c.rec == PF_REC_NONE ? P.a_full : (c.rec == PF_REC_SELECTIVE ? P.a_sel : P.a_ckpt);
     const i64 a_layer = cdiv64(t * a_tok, tp);
     i64 units;
@@ -193,7 +210,7 @@ __device__ __forceinline__ void train_memory(const DevPlan &P, const TrainTuple 
     i64 act = units * a_layer;
     if (c.rec == PF_REC_FULL) act += cdiv64(t * P.a_full, tp);
     if (owns_head && P.count_embeddings) act += 4 * cdiv64(t * (i64)P.vocab, tp);
-    M.mem = (i64)(P.wb + P.gb) * n_all + M.bytes_o + act + P.reserved_bytes;
+    M.mem = (i64)(P.wb + P.gb) * n_all + M.bytes_o + buf + act + P.reserved_bytes;
 }
 
 // Per-layer and per-step time terms shared by the analytic scorer and the simulator.
@@ -219,7 +236,8 @@ __device__ __forceinline__ void train_times(const DevPlan &P, const TrainTuple &
     const i64 act_bytes = (i64)P.ab * (i64)D.t * (i64)P.H;  // one activation tensor of the microbatch
     const float tpc = 2.f * t_allreduce(c.tp, (float)act_bytes, link_of(P, c.tp));
     const float a2a = 2.f * t_alltoall(c.ep, fdiv((float)(act_bytes * P.K), tp), link_of(P, (i64)c.tp * c.ep));
-    const float hid = D.ov ? P.sched[c.s].hide_frac * a2a : 0.f;
+    // the hiding benefit is conditioned out when the optimizer is offloaded (Sec. 5 RQ2)
+    const float hid = (D.ov && c.sh != PF_SHARD_ZERO1_OFFLOAD) ? P.sched[c.s].hide_frac * a2a : 0.f;
     const float xF = a2a - fminf(hid, cF);
     const float xB = a2a - fminf(hid, cB + rc);
     T.F_l = cF + tpc + xF;
@@ -234,6 +252,17 @@ __device__ __forceinline__ void train_times(const DevPlan &P, const TrainTuple &
     const float gw = (float)(P.gb + P.wb);
     T.T_dp = t_allreduce((i64)D.dp, gw * (float)M.N_dense, ldp) + t_allreduce((i64)D.edp, gw * (float)M.N_exp, ldp);
     T.T_opt = fdiv(2.f * (float)M.bytes_o, P.hbm_bw);
+    if (c.sh == PF_SHARD_ZERO1_OFFLOAD) {
+        // the step runs on the host: the shard's gradients go down, its updated weights come back
+        T.T_opt = fdiv(gw * (float)M.n_shard, P.bw_host);
+    } else if (c.sh == PF_SHARD_FSDP) {
+        // per microbatch: parameters gathered for forward and again for backward, gradients reduce-scattered
+        const float ag = t_allgather((i64)D.dp, (float)P.wb * (float)M.N_dense, ldp) +
+                         t_allgather((i64)D.edp, (float)P.wb * (float)M.N_exp, ldp);
+        const float rs = t_allgather((i64)D.dp, (float)P.gb * (float)M.N_dense, ldp) +
+                         t_allgather((i64)D.edp, (float)P.gb * (float)M.N_exp, ldp);
+        T.T_dp = (float)D.m * (2.f * ag + rs);
+    }
 }
 
 // tokens/s/GPU from a pipeline time, with the realization taxes of the plans that pay them
@@ -246,6 +275,8 @@ __device__ __forceinline__ float train_price(const DevPlan &P, const TrainTuple 
     const DevKern &kn = P.kern[c.kv];
     if (!kn.is_native) tput = fdiv(tput, 1.f + kn.patch_ovh);
     if (D.ov) tput = fdiv(tput, 1.f + P.sched[c.s].sched_ovh);
+    // the contention penalty prices exactly the offloaded-and-overlapped plans (Sec. 3.2)
+    if (D.ov && c.sh == PF_SHARD_ZERO1_OFFLOAD) tput = fdiv(tput, 1.f + P.offload_overlap_penalty);
     return tput;
 }
 

@@ -56,12 +56,12 @@ struct DevPlan {
     int G;
     uint32_t caps;
     long long budget_bytes, reserved_bytes;
-    float peak_flops, hbm_bw, bw_intra, bw_inter, alpha_intra, alpha_inter;
+    float peak_flops, hbm_bw, bw_intra, bw_inter, alpha_intra, alpha_inter, bw_host;
     // --- workload
     long long gbs, world;
     int n_scen;
     // --- cost constants, rules, tables
-    float eff_dense, bwd_factor, dp_overlap_frac, dualpipe_startup_div, step_overhead;
+    float eff_dense, bwd_factor, dp_overlap_frac, dualpipe_startup_div, step_overhead, offload_overlap_penalty;
     int ep_scope, layer_mode, tp_max, world_min, world_max, enforce;
     int n_sched, n_kern;
     DevSched sched[PF_MAX_SCHED];

@@ -308,6 +308,7 @@ __global__ void __launch_bounds__(kThreads, 4) score_kernel(const __grid_constan
                 c.v = P.n_inner > 4 ? inner_vals[P.val_off[4] + d4] : s_slab.outer[4];
                 c.ep = s_slab.outer[5]; c.pp = s_slab.outer[6]; c.tp = s_slab.outer[7];
                 c.dp = s_slab.outer[8]; c.world = s_slab.outer[9];
+                c.sh = P.n_axes > 10 ? s_slab.outer[10] : PF_SHARD_ZERO1;
                 RI dp, world;
                 int r = train_layout_rules<RI>(P, c, first_rule, 3, dp, world);
                 if (r == 0) {
@@ -385,6 +386,7 @@ __global__ void __launch_bounds__(kThreads, 4) score_kernel(const __grid_constan
                         TrainTuple c;
                         c.kv = v[0]; c.rec = v[1]; c.s = v[2]; c.mb = v[3]; c.v = v[4];
                         c.ep = v[5]; c.pp = v[6]; c.tp = v[7]; c.dp = v[8]; c.world = v[9];
+                        c.sh = P.n_axes > 10 ? v[10] : PF_SHARD_ZERO1;
                         RI dp, world;
                         TrainDerived<RI> D;
                         train_layout_rules<RI>(P, c, 4, 3, dp, world);      // derives dp / world only
@@ -469,6 +471,7 @@ __global__ void __launch_bounds__(kThreads, 4) score_kernel(const __grid_constan
                         c.v = P.n_inner > 4 ? inner_vals[P.val_off[4] + d4] : s_slab.outer[4];
                         c.ep = s_slab.outer[5]; c.pp = s_slab.outer[6]; c.tp = s_slab.outer[7];
                         c.dp = s_slab.outer[8]; c.world = s_slab.outer[9];
+                        c.sh = P.n_axes > 10 ? s_slab.outer[10] : PF_SHARD_ZERO1;
                         RI dp, world;
                         TrainDerived<RI> D;
                         train_layout_rules<RI>(P, c, 4, 3, dp, world);   // derives dp / world only
@@ -549,6 +552,7 @@ __global__ void __launch_bounds__(kThreads, 4) score_kernel(const __grid_constan
                         TrainTuple c;
                         c.kv = v[0]; c.rec = v[1]; c.s = v[2]; c.mb = v[3]; c.v = v[4];
                         c.ep = v[5]; c.pp = v[6]; c.tp = v[7]; c.dp = v[8]; c.world = v[9];
+                        c.sh = P.n_axes > 10 ? v[10] : PF_SHARD_ZERO1;
                         RI dp, world;
                         int reason = train_layout_rules<RI>(P, c, first_rule, 3, dp, world);
                         if (reason == 0) {

@@ -490,6 +490,7 @@ __global__ void __launch_bounds__(kSimThreads, 4) simulate_kernel(const __grid_c
                     }
                     c.kv = v[0]; c.rec = v[1]; c.s = v[2]; c.mb = v[3]; c.v = v[4];
                     c.ep = v[5]; c.pp = v[6]; c.tp = v[7]; c.dp = v[8]; c.world = v[9];
+                    c.sh = P.n_axes > 10 ? v[10] : PF_SHARD_ZERO1;
                 }
                 RI dp, world;
                 TrainDerived<RI> D;
