@@ -22,7 +22,7 @@
  *   - spec structs are copied by pf_plan_create; the caller may free them afterwards.
  *   - a handle may be used from one thread at a time, on the device that was current at create.
  *   - candidates are addressed by a linear index: idx = sum_a digit_a * prod_{b<a} len_b, axes listed
- *     least-significant first.  train axes: kv, rec, sched, mb, v, ep, pp, tp, dp, world;
+ *     least-significant first.  train axes: kv, rec, sched, mb, v, ep, pp, tp, dp, world [, shard];
  *     serve axes: kv, chunk, batch, dpa, ep, tp, scen.  An axis value list {0} for dp / world / v means
  *     "derived" (dp = world/(tp*pp); world = tp*pp*dp; v = 2 for interleaved schedules, else 1).
  */
