@@ -338,8 +338,9 @@ uint64_t pf_launch_count(void);
  * thread-level instructions of that kind the launch executes; dividing by the launch's duration gives the
  * issue-rate peak for that kind.  d_sink: 4 device bytes, practically never written.  1 <= iters <= 2^24.
  *
- * pf_probe_write: fills `bytes` (a multiple of 16, 16-byte aligned device buffer) with 16-byte streaming
- * stores, the store the scoring kernel uses for its dense outputs; bytes / duration is the write rate.
+ * pf_probe_write: fills `bytes` (a multiple of 16, below 2^35, 16-byte aligned device buffer) with 16-byte
+ * streaming stores, one per thread over a grid as large as the buffer -- the store the scoring kernel uses for
+ * its dense outputs, in the fastest pure-write pattern; bytes / duration is the write ceiling.
  * Errors: PF_EINVAL for a null pointer, a bad kind, iters or size; PF_ECUDA if the launch fails. */
 enum { PF_PROBE_FFMA = 0, PF_PROBE_IMAD = 1, PF_PROBE_LOGIC = 2 };
 int pf_probe_alu(int kind, uint32_t iters, uint32_t *d_sink, uint64_t *h_thread_instructions, void *stream);
