@@ -56,7 +56,7 @@ class Model(C.Structure):
 class Cluster(C.Structure):
     _fields_ = [(n, i64) for n in ("G", "budget_bytes", "reserved_bytes", "caps")] + \
                [(n, f64) for n in ("peak_flops", "hbm_bw", "bw_intra", "bw_inter", "alpha_intra", "alpha_inter",
-                                   "bw_host")]
+                                   "bw_host")] + [("gpu_id", i64)]
 
 
 class Workload(C.Structure):
@@ -75,12 +75,16 @@ class Sched(C.Structure):
 
 class Kern(C.Structure):
     _fields_ = [("needs_caps", i64), ("avail_mask", i64), ("is_native", i64), ("wbytes", i64),
-                ("dtype_mult", f64), ("eff", f64 * NBUCKET), ("patch_ovh", f64)]
+                ("dtype_mult", f64), ("eff", f64 * NBUCKET), ("patch_ovh", f64), ("dtype", i64)]
 
 
 class Rules(C.Structure):
     _fields_ = [(n, i64) for n in ("ep_scope", "layer_mode", "tp_max", "world_min", "world_max",
                                    "enforce_realizability")]
+
+
+class Domain(C.Structure):
+    _fields_ = [(n, i64) for n in ("attached", "gpu_id", "dtype_mask", "m_lo", "m_hi")]
 
 
 class Axes(C.Structure):
@@ -90,7 +94,7 @@ class Axes(C.Structure):
 class Problem(C.Structure):
     _fields_ = [("model", Model), ("cluster", Cluster), ("workload", Workload), ("consts", Consts),
                 ("n_sched", i64), ("sched", Sched * MAX_SCHED), ("n_kern", i64), ("kern", Kern * MAX_KERN),
-                ("rules", Rules), ("axes", Axes)]
+                ("rules", Rules), ("axes", Axes), ("domain", Domain)]
 
 
 class Derived(C.Structure):
@@ -107,7 +111,7 @@ class Detail(C.Structure):
                                    "mem")] + \
                [(n, f64) for n in ("cF", "cB", "rc", "tpc", "a2a", "xF", "xB", "F_l", "B_l", "headF", "F", "B",
                                    "p", "T_pipe", "T_dp", "T_opt", "T_step", "T_dec", "T_pre", "tput_unpriced",
-                                   "tput")] + [("reason", i64)]
+                                   "tput")] + [("reason", i64), ("why", i64)]
 
     def as_dict(self):
         return {n: getattr(self, n) for n, _ in self._fields_}
@@ -258,10 +262,13 @@ class Oracle:
                 setattr(pb.kern[i], n, int(k[n]))
             pb.kern[i].dtype_mult = float(k["dtype_mult"])
             pb.kern[i].patch_ovh = float(k["patch_ovh"])
+            pb.kern[i].dtype = int(k.get("dtype", 0))
             for b in range(NBUCKET):
                 pb.kern[i].eff[b] = float(k["eff"][b])
         for n, _ in Rules._fields_:
             setattr(pb.rules, n, int(cfg["rules"][n]))
+        for n, _ in Domain._fields_:
+            setattr(pb.domain, n, int(cfg["domain"][n]))
         pb.axes.n_axes = len(cfg["axes"])
         for a, (_, vals) in enumerate(cfg["axes"]):
             arr = np.asarray(vals, dtype=np.int64)

@@ -158,6 +158,19 @@ static void decode(const orc_axes_t *ax, uint64_t idx, int64_t *value)
     }
 }
 
+/* Which parts of the calibration domain a query falls outside of (principle P4): 0 = inside, or no domain */
+static int64_t domain_why(const orc_problem_t *pb, const orc_kern_t *kn, int64_t m_e)
+{
+    const orc_domain_t *dm = &pb->domain;
+    int64_t why = 0;
+    if (!dm->attached) return 0;
+    if (dm->gpu_id >= 0 && dm->gpu_id != pb->cluster.gpu_id) why |= ORC_WHY_GPU;
+    if (((dm->dtype_mask >> kn->dtype) & 1) == 0) why |= ORC_WHY_DTYPE;
+    if (m_e < dm->m_lo) why |= ORC_WHY_M_LOW;
+    if (m_e > dm->m_hi) why |= ORC_WHY_M_HIGH;
+    return why;
+}
+
 /* ------------------------------------------------------------------ alpha-beta collectives */
 
 typedef struct {
@@ -423,7 +436,8 @@ static int eval_train(const orc_problem_t *pb, const orc_derived_t *dv, uint64_t
     o->T_pipe = T_pipe; o->T_dp = T_dp; o->T_opt = T_opt; o->T_step = T_step; o->tput = tput;
 
     int reason = ORC_FEASIBLE;
-    if (m_e < 64 || m_e > 8192) reason |= ORC_FLAG_EXTRAPOLATED;
+    o->why = domain_why(pb, kn, m_e);
+    if (o->why) reason |= ORC_FLAG_EXTRAPOLATED;
     return o->reason = reason;
 }
 
@@ -528,7 +542,8 @@ static int eval_serve(const orc_problem_t *pb, const orc_derived_t *dv, uint64_t
     o->T_dec = T_dec; o->T_pre = T_pre; o->tput = tput;
 
     int reason = ORC_FEASIBLE;
-    if (m_e < 64 || m_e > 8192) reason |= ORC_FLAG_EXTRAPOLATED;
+    o->why = domain_why(pb, kn, m_e);
+    if (o->why) reason |= ORC_FLAG_EXTRAPOLATED;
     return o->reason = reason;
 }
 

@@ -87,6 +87,7 @@ typedef struct {
     int64_t caps; /* bit 0: fp8, bit 1: device-initiated communication */
     double peak_flops, hbm_bw, bw_intra, bw_inter, alpha_intra, alpha_inter;
     double bw_host; /* host link of one GPU, bytes/s (offloaded optimizer) */
+    int64_t gpu_id; /* which GPU model the modeled cluster has (an id the caller assigns) */
 } orc_cluster_t;
 
 typedef struct {
@@ -111,7 +112,20 @@ typedef struct {
 typedef struct {
     int64_t needs_caps, avail_mask, is_native, wbytes;
     double dtype_mult, eff[ORC_NBUCKET], patch_ovh;
+    int64_t dtype; /* id of the variant's compute dtype (0 bf16, 1 fp8, ...) for the calibration domain */
 } orc_kern_t;
+
+/* Calibration domain of the constants (principle P4, Appendix "Testbeds and calibration domains"): the GPU,
+ * the dtypes and the tokens-per-expert range they were fit over.  A query outside it is flagged extrapolated;
+ * with no domain attached the check is vacuously true and nothing is flagged. */
+typedef struct {
+    int64_t attached;
+    int64_t gpu_id;     /* -1: any GPU */
+    int64_t dtype_mask; /* bit d: dtype id d is covered */
+    int64_t m_lo, m_hi; /* tokens per expert, inclusive */
+} orc_domain_t;
+/* why a candidate is extrapolated (bits) */
+enum { ORC_WHY_GPU = 1, ORC_WHY_DTYPE = 2, ORC_WHY_M_LOW = 4, ORC_WHY_M_HIGH = 8 };
 
 typedef struct {
     int64_t ep_scope;   /* 0: ep | dp, 1: ep | dp*tp */
@@ -140,6 +154,7 @@ typedef struct {
     orc_kern_t kern[ORC_MAX_KERN];
     orc_rules_t rules;
     orc_axes_t axes;
+    orc_domain_t domain;
 } orc_problem_t;
 
 /* candidate-independent model constants (exact integers) */
@@ -163,6 +178,7 @@ typedef struct {
     double T_dec, T_pre; /* serve */
     double tput_unpriced, tput;
     int64_t reason;
+    int64_t why; /* ORC_WHY_* bits behind the extrapolated flag (feasible candidates only) */
 } orc_detail_t;
 
 int64_t orc_budget_bytes(int64_t hbm_bytes); /* floor(0.9 * capacity), in integers */

@@ -62,7 +62,7 @@ def _sched(kind, overlap, mapped, sched_ovh):
 def _kern(eff_row, patch, mask, is_native, fp8=False):
     return dict(needs_caps=CAP_FP8 if fp8 else 0, avail_mask=mask, is_native=is_native,
                 wbytes=1 if fp8 else 2, dtype_mult=f32(2.0 if fp8 else 1.0),
-                eff=[f32(e) for e in eff_row], patch_ovh=f32(patch))
+                eff=[f32(e) for e in eff_row], patch_ovh=f32(patch), dtype=1 if fp8 else 0)
 
 
 def _model(**kw):
@@ -76,7 +76,7 @@ def _cluster(G, budget_bytes, peak, hbm_bw, bw_intra, bw_inter, a_intra, a_inter
     # budget_bytes: usable HBM per modeled GPU (0.9 of a 24 GB / 80 GB part), given as integer bytes
     return dict(G=G, budget_bytes=budget_bytes, reserved_bytes=0, caps=caps,
                 peak_flops=f32(peak), hbm_bw=f32(hbm_bw), bw_intra=f32(bw_intra), bw_inter=f32(bw_inter),
-                alpha_intra=f32(a_intra), alpha_inter=f32(a_inter), bw_host=f32(bw_host))
+                alpha_intra=f32(a_intra), alpha_inter=f32(a_inter), bw_host=f32(bw_host), gpu_id=0)
 
 
 def _tiny():
@@ -158,22 +158,31 @@ def _large(enforce: int, seed: int = 0):
     )
 
 
+# The calibration domain the constants carry (paper, Appendix: tokens per expert in [64, 8192]); any GPU and any
+# dtype by default, so that attaching it flags exactly the plans outside the fitted tokens-per-expert range.
+def default_domain() -> dict:
+    return dict(attached=1, gpu_id=-1, dtype_mask=0xFFFF, m_lo=64, m_hi=8192)
+
+
 def make_config(name: str, seed: int = 0) -> dict:
     """Return a fresh config dict.  'large_unconstrained' is 'large' with the dry-run rules off
     (the paper's unconstrained search mode), used by the simulator tier.  `seed` re-draws the tables of
     the large spaces (independent problems of the same shape, one per GPU in a multi-GPU benchmark);
     the other spaces keep their fixed seeds."""
     if name == "tiny":
-        return _tiny()
-    if name == "mid":
-        return _mid()
-    if name == "serve":
-        return _serve()
-    if name == "large":
-        return _large(1, seed)
-    if name == "large_unconstrained":
-        return _large(0, seed)
-    raise KeyError(name)
+        cfg = _tiny()
+    elif name == "mid":
+        cfg = _mid()
+    elif name == "serve":
+        cfg = _serve()
+    elif name == "large":
+        cfg = _large(1, seed)
+    elif name == "large_unconstrained":
+        cfg = _large(0, seed)
+    else:
+        raise KeyError(name)
+    cfg["domain"] = default_domain()
+    return cfg
 
 
 def space_size(cfg: dict) -> int:
