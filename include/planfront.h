@@ -107,6 +107,7 @@ typedef struct {
     int64_t reserved_bytes;       /* added to every candidate's memory */
     float peak_flops, hbm_bw, bw_intra, bw_inter, alpha_intra, alpha_inter;
     float bw_host;                /* host link of one GPU, bytes/s: carries an offloaded optimizer step */
+    int32_t gpu_id;               /* which GPU model the cluster has (an id the caller assigns; see pf_domain_t) */
 } pf_cluster_t;
 
 typedef struct {
@@ -140,7 +141,20 @@ typedef struct {
     float dtype_mult;             /* peak multiplier of the variant's dtype (1 bf16, 2 fp8) */
     float eff[PF_NBUCKET];        /* efficiency per bucket: m_e <128, 128.., 256.., ... , >=8192 */
     float patch_ovh;              /* realization tax, applied as tput / (1 + ovh) when !is_native */
+    int32_t dtype;                /* id of the variant's compute dtype, 0..31 (0 bf16, 1 fp8, ...; see pf_domain_t) */
 } pf_kern_t;
+
+/* Calibration domain of the constants (principle P4; Appendix "Testbeds and calibration domains"): the GPU, the
+ * dtypes and the tokens-per-expert range they were fit over.  A feasible plan outside it gets PF_FLAG_EXTRAPOLATED;
+ * its score is not changed.  With no domain attached nothing is flagged. */
+typedef struct {
+    int32_t attached;             /* 0: no domain (the factory model) */
+    int32_t gpu_id;               /* -1: any GPU */
+    uint32_t dtype_mask;          /* bit d: dtype id d is covered */
+    int32_t m_lo, m_hi;           /* tokens per expert, inclusive (the paper's domains: [64, 8192]) */
+} pf_domain_t;
+/* why a plan is extrapolated (bits of pf_report_t.why) */
+enum { PF_WHY_GPU = 1, PF_WHY_DTYPE = 2, PF_WHY_M_LOW = 4, PF_WHY_M_HIGH = 8 };
 
 typedef struct {
     float eff_dense, bwd_factor, dp_overlap_frac, dualpipe_startup_div, step_overhead;
@@ -149,6 +163,7 @@ typedef struct {
     pf_sched_t sched[PF_MAX_SCHED];
     int32_t n_kern;
     pf_kern_t kern[PF_MAX_KERN];
+    pf_domain_t domain;
 } pf_tables_t;
 
 typedef struct {
@@ -327,6 +342,21 @@ int pf_timing_read(pf_plan_t *plan, float *ms, uint32_t *kernels);
 
 /* Number of kernels this library has launched in this process (for launch accounting in benchmarks). */
 uint64_t pf_launch_count(void);
+
+/* Extrapolation report for a list of plans, e.g. a top-k list (principle P4: a query outside the calibration
+ * domain is flagged, not silently trusted).  Entry i of d_out describes plan d_idx[i]: its reason byte as pf_score
+ * writes it, the PF_WHY_* bits behind an extrapolated flag, its tokens per expert and efficiency bucket (0 where
+ * the plan fails before they are derived).  An index of UINT64_MAX (an unused top-k slot) or >= N gives
+ * reason 0xFF.  d_n (device, may be NULL): only the first min(n, *d_n) entries are written.  One small launch on
+ * `stream`, no workspace.  Errors: PF_EINVAL (NULL pointer), PF_ECUDA. */
+typedef struct {
+    uint8_t reason, why;
+    uint16_t bucket;
+    uint32_t reserved;
+    int64_t m_e;
+} pf_report_t;
+int pf_report(pf_plan_t *plan, const uint64_t *d_idx, uint32_t n, const uint32_t *d_n, pf_report_t *d_out,
+              void *stream);
 
 /* Roofline probes (measurement utilities; the paper has no counterpart and no scoring call uses them).
  * The caller times them with events on `stream`; neither call synchronises or allocates.

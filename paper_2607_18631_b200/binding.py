@@ -24,7 +24,7 @@ EXPORTS = ("pf_version", "pf_strerror", "pf_reason_str", "pf_last_cuda_error", "
            "pf_plan_size", "pf_decode", "pf_score_workspace", "pf_score", "pf_topk_merge", "pf_select_workspace",
            "pf_select_survivors", "pf_simulate_workspace", "pf_simulate", "pf_search_workspace", "pf_search_host",
            "pf_launch_count", "pf_dualpipe_order", "pf_timing_enable", "pf_timing_read", "pf_score_static", "pf_serve_plan_count", "pf_aggregate_workspace", "pf_aggregate_serving",
-           "pf_probe_alu", "pf_probe_write")
+           "pf_probe_alu", "pf_probe_write", "pf_report")
 STATIC_SCRATCH_BYTES = 4 << 20
 T_CLASSES = ("score", "topk", "select", "simulate", "aggregate")
 
@@ -39,7 +39,7 @@ class PfModel(C.Structure):
 class PfCluster(C.Structure):
     _fields_ = [("G", i32), ("caps", u32), ("budget_bytes", i64), ("reserved_bytes", i64)] + \
                [(n, f32) for n in ("peak_flops", "hbm_bw", "bw_intra", "bw_inter", "alpha_intra", "alpha_inter",
-                                   "bw_host")]
+                                   "bw_host")] + [("gpu_id", i32)]
 
 
 class PfWorkload(C.Structure):
@@ -57,13 +57,26 @@ class PfSched(C.Structure):
 
 class PfKern(C.Structure):
     _fields_ = [("needs_caps", u32), ("avail_mask", u32), ("is_native", i32), ("wbytes", i32),
-                ("dtype_mult", f32), ("eff", f32 * NBUCKET), ("patch_ovh", f32)]
+                ("dtype_mult", f32), ("eff", f32 * NBUCKET), ("patch_ovh", f32), ("dtype", i32)]
+
+
+class PfDomain(C.Structure):
+    _fields_ = [("attached", i32), ("gpu_id", i32), ("dtype_mask", u32), ("m_lo", i32), ("m_hi", i32)]
+
+
+class PfReport(C.Structure):
+    _fields_ = [("reason", C.c_uint8), ("why", C.c_uint8), ("bucket", C.c_uint16), ("reserved", u32), ("m_e", i64)]
+
+
+REPORT_DTYPE = np.dtype([("reason", np.uint8), ("why", np.uint8), ("bucket", np.uint16), ("reserved", np.uint32),
+                         ("m_e", np.int64)])
 
 
 class PfTables(C.Structure):
     _fields_ = [(n, f32) for n in ("eff_dense", "bwd_factor", "dp_overlap_frac", "dualpipe_startup_div",
                                    "step_overhead", "offload_overlap_penalty")] + \
-               [("n_sched", i32), ("sched", PfSched * MAX_SCHED), ("n_kern", i32), ("kern", PfKern * MAX_KERN)]
+               [("n_sched", i32), ("sched", PfSched * MAX_SCHED), ("n_kern", i32), ("kern", PfKern * MAX_KERN),
+                ("domain", PfDomain)]
 
 
 class PfRules(C.Structure):
@@ -143,6 +156,8 @@ def load_library(path: str | None = None):
     L.pf_timing_read.argtypes = [vp, vp, vp]
     L.pf_dualpipe_order.restype = C.c_int
     L.pf_dualpipe_order.argtypes = [C.c_int, C.c_int, vp]
+    L.pf_report.restype = C.c_int
+    L.pf_report.argtypes = [vp, vp, u32, vp, vp, vp]
     L.pf_probe_alu.restype = C.c_int
     L.pf_probe_alu.argtypes = [C.c_int, u32, vp, C.POINTER(u64), vp]
     L.pf_probe_write.restype = C.c_int
@@ -239,7 +254,7 @@ class Plan:
         cl = PfCluster(G=int(c["G"]), caps=int(c["caps"]), budget_bytes=int(c["budget_bytes"]),
                        reserved_bytes=int(c["reserved_bytes"]),
                        **{n: float(c[n]) for n in ("peak_flops", "hbm_bw", "bw_intra", "bw_inter", "alpha_intra",
-                                                   "alpha_inter")}, bw_host=float(c.get("bw_host", 0.0)))
+                                                   "alpha_inter")}, bw_host=float(c.get("bw_host", 0.0)), gpu_id=int(c.get("gpu_id", 0)))
         w = cfg["workload"]
         sp = np.asarray(w.get("scen_P", []), dtype=np.int32)
         so = np.asarray(w.get("scen_O", []), dtype=np.int32)
@@ -263,10 +278,14 @@ class Plan:
         tb.n_kern = len(cfg["kern"])
         for i, k in enumerate(cfg["kern"]):
             kk = PfKern(needs_caps=int(k["needs_caps"]), avail_mask=int(k["avail_mask"]), is_native=int(k["is_native"]),
-                        wbytes=int(k["wbytes"]), dtype_mult=float(k["dtype_mult"]), patch_ovh=float(k["patch_ovh"]))
+                        wbytes=int(k["wbytes"]), dtype_mult=float(k["dtype_mult"]), patch_ovh=float(k["patch_ovh"]),
+                        dtype=int(k.get("dtype", 0)))
             for b in range(NBUCKET):
                 kk.eff[b] = float(k["eff"][b])
             tb.kern[i] = kk
+        dm = cfg.get("domain", dict(attached=0, gpu_id=-1, dtype_mask=0, m_lo=0, m_hi=0))
+        tb.domain = PfDomain(attached=int(dm["attached"]), gpu_id=int(dm["gpu_id"]), dtype_mask=int(dm["dtype_mask"]),
+                             m_lo=int(dm["m_lo"]), m_hi=int(dm["m_hi"]))
         ru = PfRules(**{n: int(cfg["rules"][n]) for n, _ in PfRules._fields_})
         h = C.c_void_p()
         _check(self._L.pf_plan_create(C.byref(m), C.byref(cl), C.byref(wl), C.byref(ax), C.byref(tb), C.byref(ru),
@@ -386,6 +405,21 @@ class Plan:
                     topk_count=topk_count, workspace=workspace)
 
     # ---- pf_aggregate_serving
+    # ---- pf_report
+    def report(self, idx, n: int | None = None, d_n=None, out=None, stream=None):
+        """Enqueue pf_report for the plan indices in `idx` (int64/uint64 device tensor).  Returns a uint8 device
+        tensor of n x 16 bytes; `report_to_numpy` views it as records (reason, why, bucket, m_e)."""
+        torch = _torch()
+        n = idx.numel() if n is None else n
+        out = torch.empty(max(n, 1) * C.sizeof(PfReport), dtype=torch.uint8, device=self.device) if out is None else out
+        _check(self._L.pf_report(self._h, _dptr(idx), n, _dptr(d_n), _dptr(out), _stream_ptr(torch, stream)),
+               "pf_report")
+        return out
+
+    @staticmethod
+    def report_to_numpy(out, n: int):
+        return out.cpu().numpy()[:n * REPORT_DTYPE.itemsize].view(REPORT_DTYPE)
+
     def serve_plan_count(self) -> int:
         return int(self._L.pf_serve_plan_count(self._h))
 

@@ -8,7 +8,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(HERE, "libplanfront.so")
-SOURCES = ["pf_api.cu", "pf_score.cu", "pf_select.cu", "pf_simulate.cu", "pf_search.cu", "pf_aggregate.cu", "pf_probe.cu"]
+SOURCES = ["pf_api.cu", "pf_score.cu", "pf_select.cu", "pf_simulate.cu", "pf_search.cu", "pf_aggregate.cu", "pf_probe.cu", "pf_report.cu"]
 
 
 def _newest_source() -> float:

@@ -231,7 +231,7 @@ extern "C" int pf_plan_create(const pf_model_t *model, const pf_cluster_t *clust
     }
     for (int i = 0; i < tables->n_kern; i++) {
         const pf_kern_t &k = tables->kern[i];
-        if (!(k.dtype_mult > 0) || k.wbytes < 1) return PF_EINVAL;
+        if (!(k.dtype_mult > 0) || k.wbytes < 1 || k.dtype < 0 || k.dtype > 31) return PF_EINVAL;
         for (int b = 0; b < PF_NBUCKET; b++)
             if (!(k.eff[b] > 0)) return PF_EINVAL;
     }
@@ -319,6 +319,9 @@ extern "C" int pf_plan_create(const pf_model_t *model, const pf_cluster_t *clust
     d.bw_intra = cluster->bw_intra; d.bw_inter = cluster->bw_inter;
     d.alpha_intra = cluster->alpha_intra; d.alpha_inter = cluster->alpha_inter;
     d.bw_host = cluster->bw_host; d.offload_overlap_penalty = tables->offload_overlap_penalty;
+    d.gpu_id = cluster->gpu_id;
+    d.dom_attached = tables->domain.attached ? 1 : 0; d.dom_gpu = tables->domain.gpu_id;
+    d.dom_dtypes = tables->domain.dtype_mask; d.dom_m_lo = tables->domain.m_lo; d.dom_m_hi = tables->domain.m_hi;
     d.gbs = workload->gbs; d.world = workload->world; d.n_scen = phase == PF_PHASE_SERVE ? workload->n_scen : 0;
     d.eff_dense = tables->eff_dense; d.bwd_factor = tables->bwd_factor; d.dp_overlap_frac = tables->dp_overlap_frac;
     d.dualpipe_startup_div = tables->dualpipe_startup_div; d.step_overhead = tables->step_overhead;
@@ -337,6 +340,7 @@ extern "C" int pf_plan_create(const pf_model_t *model, const pf_cluster_t *clust
         d.kern[i].is_native = k.is_native ? 1 : 0; d.kern[i].wbytes = k.wbytes;
         d.kern[i].dtype_mult = k.dtype_mult; d.kern[i].patch_ovh = k.patch_ovh;
         for (int b = 0; b < PF_NBUCKET; b++) d.kern[i].eff[b] = k.eff[b];
+        d.kern[i].dtype = k.dtype;
     }
 
     // can the rule arithmetic stay in 32 bits?  (largest products the rules form)

@@ -23,6 +23,19 @@ __device__ __forceinline__ i64 cdiv64(i64 a, i64 b)
 // quotients per candidate are otherwise the largest block of instructions in the cost model
 __device__ __forceinline__ float fdiv(float a, float b) { return __fdividef(a, b); }
 
+// Which parts of the calibration domain a query falls outside of (PF_WHY_* bits); 0 inside or with no domain.
+template <typename RI>
+__device__ __forceinline__ uint32_t domain_why(const DevPlan &P, const DevKern &kn, RI m_e)
+{
+    if (!P.dom_attached) return 0u;
+    uint32_t why = 0u;
+    if (P.dom_gpu >= 0 && P.dom_gpu != P.gpu_id) why |= PF_WHY_GPU;
+    if (((P.dom_dtypes >> kn.dtype) & 1u) == 0u) why |= PF_WHY_DTYPE;
+    if ((i64)m_e < (i64)P.dom_m_lo) why |= PF_WHY_M_LOW;
+    if ((i64)m_e > (i64)P.dom_m_hi) why |= PF_WHY_M_HIGH;
+    return why;
+}
+
 // tokens-per-expert bucket over the calibration domain [64, 8192]: <128, 128.., 256.., ..., >= 8192
 template <typename RI>
 __device__ __forceinline__ int me_bucket(RI m_e)
@@ -333,6 +346,9 @@ struct ServeOut {
     int reason;
     float tput;
     i64 mem;
+    i64 m_e = 0;       // decode-step tokens per expert and its bucket (set once rule 8 is reached)
+    int bucket = 0;
+    uint32_t why = 0;  // PF_WHY_* bits of a feasible plan
 };
 
 template <typename RI>
@@ -352,6 +368,8 @@ __device__ __forceinline__ void serve_eval(const DevPlan &P, const ServeTuple &c
     const RI m_e = ((RI)c.batch * (RI)P.K) / (RI)P.E;
     const RI m_ep = ((RI)c.chunk * (RI)P.K) / (RI)P.E;
     const int b = me_bucket<RI>(m_e), b_pre = me_bucket<RI>(m_ep);
+    out.m_e = (i64)m_e;
+    out.bucket = b;
     const DevKern &kn = P.kern[c.kv];
     if ((kn.needs_caps & ~P.caps) != 0u || ((kn.avail_mask >> b) & 1u) == 0u || ((kn.avail_mask >> b_pre) & 1u) == 0u) {
         out.reason = PF_R_KERNEL_MISSING;
@@ -402,7 +420,8 @@ __device__ __forceinline__ void serve_eval(const DevPlan &P, const ServeTuple &c
     float tput = fdiv((float)((i64)c.batch * On), (bl * T_pre + Of * T_dec) * nen);
     if (!kn.is_native) tput = fdiv(tput, 1.f + kn.patch_ovh);
     out.tput = tput;
-    out.reason = (m_e < (RI)64 || m_e > (RI)8192) ? PF_FLAG_EXTRAPOLATED : PF_FEASIBLE;
+    out.why = domain_why<RI>(P, kn, m_e);
+    out.reason = out.why ? PF_FLAG_EXTRAPOLATED : PF_FEASIBLE;
 }
 
 }  // namespace pf

@@ -28,6 +28,7 @@ struct DevKern {
     int is_native, wbytes;
     float dtype_mult, patch_ovh;
     float eff[PF_NBUCKET];
+    int dtype;
 };
 
 // Everything a kernel needs about the plan space except the axis value lists (global memory).
@@ -66,6 +67,9 @@ struct DevPlan {
     int n_sched, n_kern;
     DevSched sched[PF_MAX_SCHED];
     DevKern kern[PF_MAX_KERN];
+    // --- calibration domain of the constants
+    int dom_attached, dom_gpu, dom_m_lo, dom_m_hi, gpu_id;
+    uint32_t dom_dtypes;
 };
 
 }  // namespace pf

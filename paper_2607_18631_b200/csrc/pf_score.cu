@@ -399,7 +399,7 @@ __global__ void __launch_bounds__(kThreads, 4) score_kernel(const __grid_constan
                             TrainTimes T;
                             train_times<RI>(P, c, D, M, T);
                             tput = train_price<RI>(P, c, D, T, train_pipe_analytic<RI>(P, c, D, T));
-                            if (D.m_e < (RI)64 || D.m_e > (RI)8192) reason = PF_FLAG_EXTRAPOLATED;
+                            if (domain_why<RI>(P, P.kern[c.kv], D.m_e)) reason = PF_FLAG_EXTRAPOLATED;
                         }
                         const uint64_t o = rel0 + i;
                         img[i] = (uint8_t)reason;
