@@ -50,7 +50,7 @@ def build(force: bool = False, count_ops: bool = False) -> str:
 class Model(C.Structure):
     _fields_ = [(n, i64) for n in ("L", "H", "nh", "nkv", "hd", "attn_kind", "kv_latent", "rope_dim", "E", "K",
                                    "F", "S", "Fs", "seq", "vocab", "wb", "gb", "ob", "ab", "n_mats",
-                                   "count_embeddings")]
+                                   "count_embeddings", "L_dense", "F_dense", "hd_q")]
 
 
 class Cluster(C.Structure):
@@ -100,17 +100,18 @@ class Problem(C.Structure):
 class Derived(C.Structure):
     _fields_ = [(n, i64) for n in ("dk", "P_attn", "P_rt", "P_e", "P_sh", "P_dl", "P_emb", "a_attn", "a_fix",
                                    "a_ffn", "a_full", "a_sel", "a_ckpt", "f_attn", "f_rt", "f_sh", "f_dense",
-                                   "f_exp", "f_head")]
+                                   "f_exp", "f_head", "P_dld", "a_full_d", "a_sel_d", "f_mlp_d", "f_dense_d")]
 
 
 class Detail(C.Structure):
     _fields_ = [(n, i64) for n in ("kv", "rec", "sched", "mb", "v", "ep", "pp", "tp", "dp", "world", "shard", "chunk",
                                    "batch", "dpa", "scen", "kind", "ov", "v_eff", "m", "t", "Q", "Lc", "Ls",
-                                   "edp", "m_e", "bucket", "bucket_pre", "N_dense", "N_exp", "bytes_w",
+                                   "edp", "m_e", "bucket", "bucket_pre", "nd0", "nd_last", "N_dense", "N_exp", "bytes_w",
                                    "bytes_g", "bytes_o_dense", "bytes_o_expert", "bytes_o", "bytes_a", "bytes_buf",
                                    "mem")] + \
                [(n, f64) for n in ("cF", "cB", "rc", "tpc", "a2a", "xF", "xB", "F_l", "B_l", "headF", "F", "B",
-                                   "p", "T_pipe", "T_dp", "T_opt", "T_step", "T_dec", "T_pre", "tput_unpriced",
+                                   "p", "T_pipe", "T_dp", "T_opt", "T_step", "T_dec", "T_pre", "F_ld", "B_ld",
+                                   "tput_unpriced",
                                    "tput")] + [("reason", i64), ("why", i64)]
 
     def as_dict(self):
@@ -237,7 +238,7 @@ class Oracle:
         self._keep = []
         pb = Problem()
         for n, _ in Model._fields_:
-            setattr(pb.model, n, int(cfg["model"][n]))
+            setattr(pb.model, n, int(cfg["model"].get(n, 0)))
         for n, _ in Cluster._fields_:
             setattr(pb.cluster, n, cfg["cluster"][n])
         w = cfg["workload"]

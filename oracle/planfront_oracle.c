@@ -102,14 +102,15 @@ int64_t orc_budget_bytes(int64_t hbm_bytes)
 void orc_derive(const orc_model_t *m, orc_derived_t *d)
 {
     const int64_t H = m->H, nh = m->nh, nkv = m->nkv, hd = m->hd, ab = m->ab;
+    const int64_t hq = m->hd_q > 0 ? m->hd_q : hd;
     memset(d, 0, sizeof(*d));
     d->dk = m->attn_kind ? m->kv_latent + m->rope_dim : hd;
     if (m->attn_kind == 0) {
         /* q, k, v, o projections */
-        d->P_attn = H * nh * hd + 2 * H * nkv * hd + nh * hd * H;
+        d->P_attn = H * nh * hq + 2 * H * nkv * hd + nh * hd * H;
     } else {
         /* q proj, compressed kv (+ rope) down-proj, kv up-proj, o proj */
-        d->P_attn = H * nh * hd + H * (m->kv_latent + m->rope_dim) + m->kv_latent * nh * 2 * hd + nh * hd * H;
+        d->P_attn = H * nh * hq + H * (m->kv_latent + m->rope_dim) + m->kv_latent * nh * 2 * hd + nh * hd * H;
     }
     d->P_rt = H * m->E;                      /* router */
     d->P_e = m->n_mats * H * m->F;           /* one routed expert */
@@ -136,6 +137,13 @@ void orc_derive(const orc_model_t *m, orc_derived_t *d)
     d->f_dense = d->f_attn + d->f_rt + d->f_sh;
     d->f_exp = 2 * m->K * d->P_e;
     d->f_head = 2 * m->vocab * H;
+
+    /* a leading dense layer: attention + a plain FFN (gate, up, down of width F_dense), no router, no experts */
+    d->P_dld = d->P_attn + m->n_mats * H * m->F_dense;
+    d->a_sel_d = d->a_attn + ab * (2 * H);              /* ln2 input, FFN input */
+    d->a_full_d = d->a_sel_d + ab * 3 * m->F_dense;     /* gate, up, act*up */
+    d->f_mlp_d = 2 * m->n_mats * H * m->F_dense;
+    d->f_dense_d = d->f_attn + d->f_mlp_d;
 }
 
 uint64_t orc_space_size(const orc_problem_t *pb)
@@ -282,6 +290,14 @@ static int eval_train(const orc_problem_t *pb, const orc_derived_t *dv, uint64_t
     int64_t Lc = cdiv(M->L, Q);
     int64_t Ls = v_eff * Lc; /* layers on the bottleneck rank */
     o->Lc = Lc; o->Ls = Ls;
+    /* leading dense layers on the first rank (it holds virtual stages 0, pp, 2pp, ...) and on the last one:
+     * stage q covers layers [q*Lc, (q+1)*Lc) */
+    int64_t nd0 = 0, nd_last = 0;
+    for (int64_t c = 0; c < v_eff; c++) {
+        nd0 += imax(0, imin(Lc, M->L_dense - c * pp * Lc));
+        nd_last += imax(0, imin(Lc, M->L_dense - (c * pp + pp - 1) * Lc));
+    }
+    o->nd0 = nd0; o->nd_last = nd_last;
 
     /* rule 7 MICROBATCH: what each static schedule order needs to be well formed */
     OPS(kind == ORC_KIND_1F1B ? 2 : kind == ORC_KIND_INTERLEAVED ? 3 : 8, 0);
@@ -321,8 +337,11 @@ static int eval_train(const orc_problem_t *pb, const orc_derived_t *dv, uint64_t
     if ((pp == 1 || kind == ORC_KIND_DUALPIPE) && M->count_embeddings) OPS(9, 0);
     int64_t pm = (kind == ORC_KIND_DUALPIPE && pp > 1) ? 2 : 1; /* two stage copies per rank */
     int64_t emb = cdiv(dv->P_emb, tp) * ((pp == 1 || kind == ORC_KIND_DUALPIPE) ? 2 : 1);
-    int64_t N_dense = pm * Ls * (cdiv(dv->P_dl, tp) + dv->P_rt) + emb;
-    int64_t N_exp = pm * Ls * (M->E / ep) * cdiv(dv->P_e, etp);
+    /* the rank's MoE layers (both stage copies of a DualPipe-style rank; its second copy sits at the far end of
+     * the pipeline and has no leading dense layer) and its leading dense layers */
+    int64_t n_moe = pm * Ls - nd0;
+    int64_t N_dense = n_moe * (cdiv(dv->P_dl, tp) + dv->P_rt) + nd0 * cdiv(dv->P_dld, tp) + emb;
+    int64_t N_exp = n_moe * (M->E / ep) * cdiv(dv->P_e, etp);
     int64_t bytes_w = M->wb * (N_dense + N_exp);
     int64_t bytes_g = M->gb * (N_dense + N_exp);
     /* distributed optimizer: dense shard over dp, expert shard over the expert-DP group
@@ -345,15 +364,18 @@ static int eval_train(const orc_problem_t *pb, const orc_derived_t *dv, uint64_t
         bytes_buf = imin(2, pm * Ls) * M->wb * P_layer;
     }
     int64_t A_tok = rec == ORC_REC_NONE ? dv->a_full : rec == ORC_REC_SELECTIVE ? dv->a_sel : dv->a_ckpt;
+    int64_t A_tok_d = rec == ORC_REC_NONE ? dv->a_full_d : rec == ORC_REC_SELECTIVE ? dv->a_sel_d : dv->a_ckpt;
     int64_t A_layer = cdiv(t * A_tok, tp);
-    int64_t units;
+    int64_t A_layer_d = cdiv(t * A_tok_d, tp);
+    /* activation bytes of one microbatch across the rank's Ls layers */
+    int64_t A_rank = (Ls - nd0) * A_layer + nd0 * A_layer_d;
+    int64_t bytes_a;
     if (kind == ORC_KIND_1F1B)
-        units = imin(pp, m) * Ls;
-    else if (kind == ORC_KIND_INTERLEAVED)
-        units = imin(pp * v_eff + pp - 1, m * v_eff) * Lc;
+        bytes_a = imin(pp, m) * A_rank;
+    else if (kind == ORC_KIND_INTERLEAVED) /* chunks in flight, each a v-th of the rank's layers */
+        bytes_a = imin(pp * v_eff + pp - 1, m * v_eff) * A_rank / v_eff;
     else
-        units = imin(pp + 1, m) * Ls;
-    int64_t bytes_a = units * A_layer;
+        bytes_a = imin(pp + 1, m) * A_rank;
     if (rec == ORC_REC_FULL) bytes_a += cdiv(t * dv->a_full, tp); /* the layer being recomputed */
     if ((pp == 1 || kind == ORC_KIND_DUALPIPE) && M->count_embeddings)
         bytes_a += 4 * cdiv(t * M->vocab, tp); /* fp32 logits where the head lives */
@@ -392,8 +414,21 @@ static int eval_train(const orc_problem_t *pb, const orc_derived_t *dv, uint64_t
     double F_l = cF + tpc + xF;
     double B_l = cB + rc + tpc + xB + (rec == ORC_REC_FULL ? tpc + xF : 0.0);
     double headF = td * (double)dv->f_head / (tpd * peak * K0->eff_dense);
-    double F = (double)Ls * F_l + headF / (double)pp;
-    double B = (double)Ls * B_l + K0->bwd_factor * headF / (double)pp;
+    /* a leading dense layer: no experts, no all-to-all */
+    double cDd = td * (double)dv->f_dense_d / (tpd * peak * K0->eff_dense);
+    double rcd = rec == ORC_REC_NONE ? 0.0
+                 : rec == ORC_REC_SELECTIVE ? (2.0 / 3.0) * td * (double)dv->f_mlp_d / (tpd * peak * K0->eff_dense)
+                                            : cDd;
+    double F_ld = cDd + tpc;
+    double B_ld = K0->bwd_factor * cDd + rcd + tpc + (rec == ORC_REC_FULL ? tpc : 0.0);
+    /* the closed forms take the slower of the two extreme ranks: the first (most leading dense layers) and the
+     * last (fewest) */
+    double F0 = (double)(Ls - nd0) * F_l + (double)nd0 * F_ld, B0 = (double)(Ls - nd0) * B_l + (double)nd0 * B_ld;
+    double F1 = (double)(Ls - nd_last) * F_l + (double)nd_last * F_ld;
+    double B1 = (double)(Ls - nd_last) * B_l + (double)nd_last * B_ld;
+    int first_slower = F0 + B0 > F1 + B1;
+    double F = (first_slower ? F0 : F1) + headF / (double)pp;
+    double B = (first_slower ? B0 : B1) + K0->bwd_factor * headF / (double)pp;
     double p = 0.0;
     if (pp > 1) {
         link_t lw = link_of(C, world);
@@ -433,6 +468,7 @@ static int eval_train(const orc_problem_t *pb, const orc_derived_t *dv, uint64_t
 
     o->cF = cF; o->cB = cB; o->rc = rc; o->tpc = tpc; o->a2a = a2a; o->xF = xF; o->xB = xB;
     o->F_l = F_l; o->B_l = B_l; o->headF = headF; o->F = F; o->B = B; o->p = p;
+    o->F_ld = F_ld; o->B_ld = B_ld;
     o->T_pipe = T_pipe; o->T_dp = T_dp; o->T_opt = T_opt; o->T_step = T_step; o->tput = tput;
 
     int reason = ORC_FEASIBLE;
@@ -1040,8 +1076,10 @@ int orc_simulate(const orc_problem_t *pb, uint64_t idx, uint32_t seed, double *t
     for (int q = 0; q < Q; q++) {
         /* exact balanced layer split over virtual stages; the head sits on the last one */
         int64_t nq = M->L / Q + (q < M->L % Q ? 1 : 0);
-        double f = (double)nq * d.F_l + (q == Q - 1 ? d.headF : 0.0);
-        double b = (double)nq * d.B_l + (q == Q - 1 ? K0->bwd_factor * d.headF : 0.0);
+        int64_t start = q * (M->L / Q) + (q < M->L % Q ? q : M->L % Q); /* first layer of the stage */
+        int64_t ndq = imax(0, imin(nq, M->L_dense - start));               /* its leading dense layers */
+        double f = (double)(nq - ndq) * d.F_l + (double)ndq * d.F_ld + (q == Q - 1 ? d.headF : 0.0);
+        double b = (double)(nq - ndq) * d.B_l + (double)ndq * d.B_ld + (q == Q - 1 ? K0->bwd_factor * d.headF : 0.0);
         Fq[q] = f * orc_jitter(seed, idx, q, 0);
         Bq[q] = b * orc_jitter(seed, idx, q, 1);
     }

@@ -78,6 +78,9 @@ typedef struct {
     int64_t wb, gb, ob, ab; /* bytes: weight, gradient, optimizer state per parameter, activation */
     int64_t n_mats;         /* matrices per expert FFN (3 = gate, up, down) */
     int64_t count_embeddings;
+    /* DeepSeek-style stacks: the first L_dense layers have a plain FFN of width F_dense instead of experts
+     * (0 = every layer is MoE); hd_q: query head dimension where it differs from hd (MLA: nope + rope; 0 = hd) */
+    int64_t L_dense, F_dense, hd_q;
 } orc_model_t;
 
 typedef struct {
@@ -162,6 +165,8 @@ typedef struct {
     int64_t dk, P_attn, P_rt, P_e, P_sh, P_dl, P_emb;
     int64_t a_attn, a_fix, a_ffn, a_full, a_sel, a_ckpt;
     int64_t f_attn, f_rt, f_sh, f_dense, f_exp, f_head;
+    /* a leading dense layer: parameters that shard by tp, activation bytes per token, forward FLOPs per token */
+    int64_t P_dld, a_full_d, a_sel_d, f_mlp_d, f_dense_d;
 } orc_derived_t;
 
 /* everything computed for one candidate; unfilled parts stay 0 */
@@ -171,11 +176,13 @@ typedef struct {
     int64_t chunk, batch, dpa, scen; /* serve */
     /* derived integers */
     int64_t kind, ov, v_eff, m, t, Q, Lc, Ls, edp, m_e, bucket, bucket_pre;
+    int64_t nd0, nd_last; /* leading dense layers on the first and on the last rank */
     /* memory terms */
     int64_t N_dense, N_exp, bytes_w, bytes_g, bytes_o_dense, bytes_o_expert, bytes_o, bytes_a, bytes_buf, mem;
     /* time terms */
     double cF, cB, rc, tpc, a2a, xF, xB, F_l, B_l, headF, F, B, p, T_pipe, T_dp, T_opt, T_step;
     double T_dec, T_pre; /* serve */
+    double F_ld, B_ld;   /* a leading dense layer's forward and backward time */
     double tput_unpriced, tput;
     int64_t reason;
     int64_t why; /* ORC_WHY_* bits behind the extrapolated flag (feasible candidates only) */
