@@ -33,7 +33,8 @@ i32, u32, i64, u64, f32 = C.c_int32, C.c_uint32, C.c_int64, C.c_uint64, C.c_floa
 
 class PfModel(C.Structure):
     _fields_ = [(n, i32) for n in ("L", "H", "nh", "nkv", "hd", "attn_kind", "kv_latent", "rope_dim", "E", "K", "F",
-                                   "S", "Fs", "seq", "vocab", "wb", "gb", "ob", "ab", "n_mats", "count_embeddings")]
+                                   "S", "Fs", "seq", "vocab", "wb", "gb", "ob", "ab", "n_mats", "count_embeddings",
+                                   "L_dense", "F_dense", "hd_q")]
 
 
 class PfCluster(C.Structure):
@@ -249,7 +250,7 @@ class Plan:
         self._L = load_library()
         self.cfg = cfg
         self._keep = []
-        m = PfModel(**{n: int(cfg["model"][n]) for n, _ in PfModel._fields_})
+        m = PfModel(**{n: int(cfg["model"].get(n, 0)) for n, _ in PfModel._fields_})
         c = cfg["cluster"]
         cl = PfCluster(G=int(c["G"]), caps=int(c["caps"]), budget_bytes=int(c["budget_bytes"]),
                        reserved_bytes=int(c["reserved_bytes"]),

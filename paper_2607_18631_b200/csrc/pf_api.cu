@@ -116,7 +116,8 @@ static void derive_model(const pf_model_t &m, DevPlan &d)
     const long long lat = m.kv_latent, rope = m.rope_dim;
     const bool mla = m.attn_kind != 0;
     d.dk = mla ? (int)(lat + rope) : m.hd;
-    const long long q_proj = H * nh * hd, o_proj = nh * hd * H;
+    const long long hq = m.hd_q > 0 ? m.hd_q : hd;
+    const long long q_proj = H * nh * hq, o_proj = nh * hd * H;
     if (!mla)
         d.P_attn = q_proj + 2 * H * nkv * hd + o_proj;
     else
@@ -142,6 +143,15 @@ static void derive_model(const pf_model_t &m, DevPlan &d)
     d.f_exp = (float)(2ll * m.K * d.P_e);
     d.f_head = (float)(2ll * m.vocab * H);
     d.f_sh = (float)f_sh;
+
+    // a leading dense layer: attention + a plain FFN, no router, no experts
+    d.L_dense = m.L_dense;
+    d.P_dld = d.P_attn + (long long)m.n_mats * H * m.F_dense;
+    d.a_sel_d = a_attn + ab * 2 * H;
+    d.a_full_d = d.a_sel_d + ab * 3 * (long long)m.F_dense;
+    const long long f_mlp_d = 2ll * m.n_mats * H * m.F_dense;
+    d.f_mlp_d = (float)f_mlp_d;
+    d.f_dense_d = (float)(f_attn + f_mlp_d);
 }
 
 static bool positive(std::initializer_list<long long> xs)
@@ -168,6 +178,9 @@ extern "C" int pf_plan_create(const pf_model_t *model, const pf_cluster_t *clust
     if (!positive({M.L, M.H, M.nh, M.hd, M.E, M.K, M.F, M.seq, M.vocab, M.wb, M.gb, M.ob, M.ab, M.n_mats}))
         return PF_EINVAL;
     if (M.S < 0 || (M.S > 0 && M.Fs <= 0) || M.K > M.E) return PF_EINVAL;
+    if (M.L_dense < 0 || M.L_dense >= M.L || (M.L_dense > 0 && M.F_dense <= 0) || M.F_dense < 0 || M.hd_q < 0)
+        return PF_EINVAL;
+    if (M.L_dense > 0 && phase == PF_PHASE_SERVE) return PF_EUNSUPPORTED;  // leading dense layers: training plans only
     if (M.attn_kind == 0 ? M.nkv <= 0 : (M.kv_latent <= 0 || M.rope_dim < 0)) return PF_EINVAL;
     if (cluster->G <= 0 || cluster->budget_bytes < 0 || cluster->reserved_bytes < 0) return PF_EINVAL;
     if (!(cluster->peak_flops > 0) || !(cluster->hbm_bw > 0) || !(cluster->bw_intra > 0) || !(cluster->bw_inter > 0))

@@ -90,6 +90,7 @@ template <typename RI>
 struct TrainDerived {
     RI dp, world, m, t, edp, m_e;
     int kind, ov, v_eff, Q, Lc, Ls, bucket;
+    int nd0, nd_last;   // leading dense layers on the first rank and on the last one
 };
 
 // Rules first_rule..last_rule of the layout rules 1-3.  Returns 0 or the failing rule; fills dp / world.
@@ -161,6 +162,13 @@ __device__ __forceinline__ int train_plan_rules(const DevPlan &P, const TrainTup
     D.Q = Q;
     D.Lc = (P.L + Q - 1) / Q;
     D.Ls = v_eff * D.Lc;
+    // stage q covers layers [q Lc, (q+1) Lc); rank r holds stages r, r + pp, ...
+    D.nd0 = D.nd_last = 0;
+    if (P.L_dense > 0)
+        for (int cc = 0; cc < v_eff; cc++) {
+            D.nd0 += max(0, min(D.Lc, P.L_dense - cc * c.pp * D.Lc));
+            D.nd_last += max(0, min(D.Lc, P.L_dense - (cc * c.pp + c.pp - 1) * D.Lc));
+        }
     if (kind == PF_KIND_INTERLEAVED) {
         if (m % (RI)c.pp != 0) return PF_R_MICROBATCH;
     } else if (kind == PF_KIND_DUALPIPE) {
@@ -198,8 +206,12 @@ __device__ __forceinline__ void train_memory(const DevPlan &P, const TrainTuple 
     const bool owns_head = (pp == 1) || dual;
     const i64 emb = cdiv64(P.P_emb, tp) * (owns_head ? 2 : 1);
     const i64 etp = P.ep_scope ? 1 : tp;
-    M.N_dense = copies * Ls * (cdiv64(P.P_dl, tp) + P.P_rt) + emb;
-    M.N_exp = copies * Ls * (i64)(P.E / c.ep) * cdiv64(P.P_e, etp);
+    // the rank's MoE layers (both stage copies of a DualPipe-style rank; the second copy sits at the far end of
+    // the pipeline and has no leading dense layer) and its leading dense layers
+    const i64 nd0 = D.nd0, n_moe = copies * Ls - nd0;
+    M.N_dense = n_moe * (cdiv64(P.P_dl, tp) + P.P_rt) + emb;
+    if (nd0) M.N_dense += nd0 * cdiv64(P.P_dld, tp);
+    M.N_exp = n_moe * (i64)(P.E / c.ep) * cdiv64(P.P_e, etp);
     // parameters whose optimizer state this rank owns: dense over dp, experts over the expert-DP group
     M.n_shard = cdiv64(M.N_dense, (i64)D.dp) + cdiv64(M.N_exp, (i64)D.edp);
     // zero1: whole parameters and gradients, sharded state; offload: the state lives in host memory; fsdp:
@@ -213,14 +225,19 @@ __device__ __forceinline__ void train_memory(const DevPlan &P, const TrainTuple 
     }
     const i64 a_tok = c.rec == PF_REC_NONE ? P.a_full : (c.rec == PF_REC_SELECTIVE ? P.a_sel : P.a_ckpt);
     const i64 a_layer = cdiv64(t * a_tok, tp);
-    i64 units;
+    // activation bytes of one microbatch across the rank's Ls layers (leading dense layers hold less)
+    i64 a_rank = (Ls - nd0) * a_layer;
+    if (nd0) {
+        const i64 a_tok_d = c.rec == PF_REC_NONE ? P.a_full_d : (c.rec == PF_REC_SELECTIVE ? P.a_sel_d : P.a_ckpt);
+        a_rank += nd0 * cdiv64(t * a_tok_d, tp);
+    }
+    i64 act;
     if (D.kind == PF_KIND_1F1B)
-        units = min(pp, m) * Ls;
-    else if (D.kind == PF_KIND_INTERLEAVED)
-        units = min(pp * D.v_eff + pp - 1, m * D.v_eff) * (i64)D.Lc;
+        act = min(pp, m) * a_rank;
+    else if (D.kind == PF_KIND_INTERLEAVED)   // chunks in flight, each a v-th of the rank's layers
+        act = min(pp * D.v_eff + pp - 1, m * D.v_eff) * a_rank / (i64)D.v_eff;
     else
-        units = min(pp + 1, m) * Ls;
-    i64 act = units * a_layer;
+        act = min(pp + 1, m) * a_rank;
     if (c.rec == PF_REC_FULL) act += cdiv64(t * P.a_full, tp);
     if (owns_head && P.count_embeddings) act += 4 * cdiv64(t * (i64)P.vocab, tp);
     M.mem = (i64)(P.wb + P.gb) * n_all + M.bytes_o + buf + act + P.reserved_bytes;
@@ -229,6 +246,7 @@ __device__ __forceinline__ void train_memory(const DevPlan &P, const TrainTuple 
 // Per-layer and per-step time terms shared by the analytic scorer and the simulator.
 struct TrainTimes {
     float F_l, B_l, headF, p, T_dp, T_opt;
+    float F_ld, B_ld;   // a leading dense layer (0 when the model has none)
 };
 
 template <typename RI>
@@ -256,6 +274,15 @@ __device__ __forceinline__ void train_times(const DevPlan &P, const TrainTuple &
     T.F_l = cF + tpc + xF;
     T.B_l = cB + rc + tpc + xB + (c.rec == PF_REC_FULL ? tpc + xF : 0.f);
     T.headF = fdiv(t * P.f_head, dense_rate);
+    // a leading dense layer: no experts, no all-to-all
+    T.F_ld = T.B_ld = 0.f;
+    if (P.L_dense > 0) {
+        const float cDd = fdiv(t * P.f_dense_d, dense_rate);
+        const float rcd = c.rec == PF_REC_NONE ? 0.f
+                          : (c.rec == PF_REC_SELECTIVE ? (2.f / 3.f) * fdiv(t * P.f_mlp_d, dense_rate) : cDd);
+        T.F_ld = cDd + tpc;
+        T.B_ld = P.bwd_factor * cDd + rcd + tpc + (c.rec == PF_REC_FULL ? tpc : 0.f);
+    }
     T.p = 0.f;
     if (c.pp > 1) {
         Link lw = link_of(P, (i64)D.world);
@@ -299,8 +326,19 @@ __device__ __forceinline__ float train_pipe_analytic(const DevPlan &P, const Tra
                                                      const TrainTimes &T)
 {
     const float pp = (float)c.pp, m = (float)D.m;
-    const float F = (float)D.Ls * T.F_l + fdiv(T.headF, pp);
-    const float B = (float)D.Ls * T.B_l + P.bwd_factor * fdiv(T.headF, pp);
+    // the slower of the two extreme ranks: the first (most leading dense layers) and the last (fewest)
+    float Fr = (float)D.Ls * T.F_l, Br = (float)D.Ls * T.B_l;
+    if (P.L_dense > 0) {
+        const float F0 = (float)(D.Ls - D.nd0) * T.F_l + (float)D.nd0 * T.F_ld;
+        const float B0 = (float)(D.Ls - D.nd0) * T.B_l + (float)D.nd0 * T.B_ld;
+        const float F1 = (float)(D.Ls - D.nd_last) * T.F_l + (float)D.nd_last * T.F_ld;
+        const float B1 = (float)(D.Ls - D.nd_last) * T.B_l + (float)D.nd_last * T.B_ld;
+        const bool first_slower = F0 + B0 > F1 + B1;
+        Fr = first_slower ? F0 : F1;
+        Br = first_slower ? B0 : B1;
+    }
+    const float F = Fr + fdiv(T.headF, pp);
+    const float B = Br + P.bwd_factor * fdiv(T.headF, pp);
     if (D.kind == PF_KIND_1F1B) return (m + pp - 1.f) * (F + B) + 2.f * (pp - 1.f) * T.p;
     if (D.kind == PF_KIND_INTERLEAVED)
         return (m + fdiv(pp - 1.f, (float)D.v_eff)) * (F + B) + 2.f * (float)(D.Q - 1) * T.p;

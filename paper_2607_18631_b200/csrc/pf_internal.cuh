@@ -52,6 +52,9 @@ struct DevPlan {
     int dk;
     long long P_attn, P_rt, P_e, P_sh, P_dl, P_emb;
     long long a_full, a_sel, a_ckpt;
+    int L_dense;                       // leading layers with a plain FFN instead of experts
+    long long P_dld, a_full_d, a_sel_d;   // such a layer: parameters that shard by tp, activation bytes per token
+    float f_dense_d, f_mlp_d;          // its forward FLOPs per token, and its FFN's share
     float f_dense, f_exp, f_head, f_sh;   // forward FLOPs per token (per layer; head once), rounded to fp32 once
     // --- modeled cluster
     int G;

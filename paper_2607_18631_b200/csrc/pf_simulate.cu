@@ -532,10 +532,14 @@ __global__ void __launch_bounds__(kSimThreads, 4) simulate_kernel(const __grid_c
                 if (run) {
                     const int L_lo = P.L / Q, L_rem = P.L - L_lo * Q;
                     for (int q = glane; q < Q; q += g) {
-                        const float nq = (float)(L_lo + (q < L_rem ? 1 : 0));
+                        const int nq_i = L_lo + (q < L_rem ? 1 : 0);
+                        const int start = q * L_lo + min(q, L_rem);              // first layer of the stage
+                        const int ndq = max(0, min(nq_i, P.L_dense - start));    // its leading dense layers
+                        const float nq = (float)(nq_i - ndq), nd = (float)ndq;
                         const bool last = q == Q - 1;
-                        durF[q] = (nq * T.F_l + (last ? T.headF : 0.f)) * jitter(seed_mixed, idx, q, 0);
-                        durB[q] = (nq * T.B_l + (last ? P.bwd_factor * T.headF : 0.f)) * jitter(seed_mixed, idx, q, 1);
+                        durF[q] = (nq * T.F_l + nd * T.F_ld + (last ? T.headF : 0.f)) * jitter(seed_mixed, idx, q, 0);
+                        durB[q] = (nq * T.B_l + nd * T.B_ld + (last ? P.bwd_factor * T.headF : 0.f)) *
+                                  jitter(seed_mixed, idx, q, 1);
                     }
                     for (int i = glane; i < n_entries; i += g) tl[i] = 0.f;
                 }
