@@ -70,7 +70,8 @@ class Consts(C.Structure):
 
 
 class Sched(C.Structure):
-    _fields_ = [("kind", i64), ("overlap", i64), ("mapped", i64), ("hide_frac", f64), ("sched_ovh", f64)]
+    _fields_ = [("kind", i64), ("overlap", i64), ("mapped", i64), ("hide_frac", f64), ("sched_ovh", f64),
+                ("n_chunks", i64), ("sm_frac", f64)]
 
 
 class Kern(C.Structure):
@@ -110,7 +111,7 @@ class Detail(C.Structure):
                                    "bytes_g", "bytes_o_dense", "bytes_o_expert", "bytes_o", "bytes_a", "bytes_buf",
                                    "mem")] + \
                [(n, f64) for n in ("cF", "cB", "rc", "tpc", "a2a", "xF", "xB", "F_l", "B_l", "headF", "F", "B",
-                                   "p", "T_pipe", "T_dp", "T_opt", "T_step", "T_dec", "T_pre", "F_ld", "B_ld",
+                                   "p", "T_pipe", "T_dp", "T_opt", "T_step", "T_dec", "T_pre", "F_ld", "B_ld", "cD", "cE",
                                    "tput_unpriced",
                                    "tput")] + [("reason", i64), ("why", i64)]
 
@@ -152,6 +153,8 @@ def lib():
         L.orc_schedule_order.argtypes = [C.c_int, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_int]
         L.orc_makespan.restype = f64
         L.orc_makespan.argtypes = [C.c_int, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p, f64]
+        L.orc_two_stream_layer.restype = f64
+        L.orc_two_stream_layer.argtypes = [f64, f64, f64, f64, C.c_int]
         L.orc_mix32.restype = u32
         L.orc_mix32.argtypes = [u32]
         L.orc_jitter.restype = f64
@@ -222,6 +225,10 @@ def makespan(kind: int, pp: int, v: int, m: int, Fq, Bq, p: float) -> float:
     return float(lib().orc_makespan(kind, pp, v, m, _ptr(Fq), _ptr(Bq), float(p)))
 
 
+def two_stream_layer(A: float, e_tot: float, d_tot: float, c_tot: float, n: int) -> float:
+    return float(lib().orc_two_stream_layer(A, e_tot, d_tot, c_tot, n))
+
+
 def mix32(x: int) -> int:
     return int(lib().orc_mix32(x & 0xFFFFFFFF))
 
@@ -256,7 +263,7 @@ class Oracle:
         pb.n_sched = len(cfg["sched"])
         for i, s in enumerate(cfg["sched"]):
             for n, _ in Sched._fields_:
-                setattr(pb.sched[i], n, s[n])
+                setattr(pb.sched[i], n, s.get(n, 0))
         pb.n_kern = len(cfg["kern"])
         for i, k in enumerate(cfg["kern"]):
             for n in ("needs_caps", "avail_mask", "is_native", "wbytes"):

@@ -468,7 +468,7 @@ static int eval_train(const orc_problem_t *pb, const orc_derived_t *dv, uint64_t
 
     o->cF = cF; o->cB = cB; o->rc = rc; o->tpc = tpc; o->a2a = a2a; o->xF = xF; o->xB = xB;
     o->F_l = F_l; o->B_l = B_l; o->headF = headF; o->F = F; o->B = B; o->p = p;
-    o->F_ld = F_ld; o->B_ld = B_ld;
+    o->F_ld = F_ld; o->B_ld = B_ld; o->cD = cD; o->cE = cE;
     o->T_pipe = T_pipe; o->T_dp = T_dp; o->T_opt = T_opt; o->T_step = T_step; o->tput = tput;
 
     int reason = ORC_FEASIBLE;
@@ -1053,6 +1053,74 @@ double orc_jitter(uint32_t seed, uint64_t idx, int q, int is_backward)
     return 0.9 + 0.2 * u;
 }
 
+/* ------------------------------------------------------------------ two-stream layer timeline */
+
+/* Generic list scheduling over a small op DAG: every op has a stream, a duration and up to two predecessors;
+ * a stream that is free starts, among its ops whose predecessors are done, the one that became ready first
+ * (ties: lower op number).  Returns the time the last op ends. */
+typedef struct {
+    int stream, dep0, dep1; /* dep = -1: none */
+    double dur;
+} ts_op_t;
+
+static double list_schedule(const ts_op_t *op, int n_ops, int n_streams)
+{
+    double end[64], free_at[4] = {0.0, 0.0, 0.0, 0.0};
+    int done[64] = {0};
+    int left = n_ops;
+    double makespan = 0.0;
+    while (left > 0) {
+        /* the op that can start earliest over all streams; its start = max(stream free, ready) */
+        int best = -1;
+        double best_start = 0.0, best_ready = 0.0;
+        for (int s = 0; s < n_streams; s++) {
+            /* this stream's pick: earliest ready time, then lowest number */
+            int pick = -1;
+            double pick_ready = 0.0;
+            for (int i = 0; i < n_ops; i++) {
+                if (done[i] || op[i].stream != s) continue;
+                if ((op[i].dep0 >= 0 && !done[op[i].dep0]) || (op[i].dep1 >= 0 && !done[op[i].dep1])) continue;
+                double ready = 0.0;
+                if (op[i].dep0 >= 0) ready = end[op[i].dep0];
+                if (op[i].dep1 >= 0 && end[op[i].dep1] > ready) ready = end[op[i].dep1];
+                if (pick < 0 || ready < pick_ready) {
+                    pick = i;
+                    pick_ready = ready;
+                }
+            }
+            if (pick < 0) continue;
+            double start = free_at[s] > pick_ready ? free_at[s] : pick_ready;
+            if (best < 0 || start < best_start || (start == best_start && pick < best)) {
+                best = pick;
+                best_start = start;
+                best_ready = pick_ready;
+            }
+        }
+        (void)best_ready;
+        if (best < 0) return -1.0; /* cyclic input: cannot happen for the layer DAG */
+        end[best] = best_start + op[best].dur;
+        free_at[op[best].stream] = end[best];
+        done[best] = 1;
+        if (end[best] > makespan) makespan = end[best];
+        left--;
+    }
+    return makespan;
+}
+
+double orc_two_stream_layer(double A, double e_tot, double d_tot, double c_tot, int n)
+{
+    ts_op_t op[64];
+    if (n < 1) n = 1;
+    if (n > 16) n = 16;
+    int k = 0;
+    op[k++] = (ts_op_t){0, -1, -1, A};                                    /* op 0: the dense part */
+    for (int i = 0; i < n; i++) op[k++] = (ts_op_t){1, 0, -1, d_tot / n}; /* ops 1..n: dispatch chunks */
+    for (int i = 0; i < n; i++)                                           /* ops n+1..2n: expert chunks, in order */
+        op[k++] = (ts_op_t){0, 1 + i, i ? n + i : -1, e_tot / n};
+    for (int i = 0; i < n; i++) op[k++] = (ts_op_t){1, n + 1 + i, -1, c_tot / n}; /* combine chunks */
+    return list_schedule(op, k, 2);
+}
+
 /* ------------------------------------------------------------------ simulator tier */
 
 int orc_simulate(const orc_problem_t *pb, uint64_t idx, uint32_t seed, double *tput_sim, double *T_pipe_sim)
@@ -1073,13 +1141,30 @@ int orc_simulate(const orc_problem_t *pb, uint64_t idx, uint32_t seed, double *t
     int kind = (int)d.kind, pp = (int)d.pp, v = (int)d.v_eff;
     int Q = kind == ORC_KIND_DUALPIPE ? pp : pp * v;
     double Fq[ORC_MAX_RANKS * ORC_MAX_V], Bq[ORC_MAX_RANKS * ORC_MAX_V];
+    /* Per-layer times of a MoE layer.  Where the schedule overlaps and says how (comm chunking, SM budget), the
+     * exposed communication comes from the two-stream timeline of the layer instead of the alpha-table's hidden
+     * fraction: compute is slowed by the SMs the communication kernels hold, the all-to-all halves are the
+     * dispatch and the combine, backward splits its compute like forward. */
+    const orc_sched_t *sc = &pb->sched[d.sched];
+    double F_l = d.F_l, B_l = d.B_l;
+    if (d.ov && sc->n_chunks > 0 && d.shard != ORC_SHARD_ZERO1_OFFLOAD) {
+        int n = (int)sc->n_chunks;
+        double slow = 1.0 / (1.0 - sc->sm_frac);
+        double half = 0.5 * d.a2a;
+        double fwd = orc_two_stream_layer(d.cD * slow, d.cE * slow, half, half, n);
+        double cBt = d.cB + d.rc;                       /* backward compute incl. recompute */
+        double share = d.cE / d.cF;                     /* the experts' share of a layer's compute */
+        double bwd = orc_two_stream_layer(cBt * (1.0 - share) * slow, cBt * share * slow, half, half, n);
+        F_l = d.tpc + fwd;
+        B_l = d.tpc + bwd + (d.rec == ORC_REC_FULL ? d.tpc + (fwd - d.cF * slow) : 0.0);
+    }
     for (int q = 0; q < Q; q++) {
         /* exact balanced layer split over virtual stages; the head sits on the last one */
         int64_t nq = M->L / Q + (q < M->L % Q ? 1 : 0);
         int64_t start = q * (M->L / Q) + (q < M->L % Q ? q : M->L % Q); /* first layer of the stage */
         int64_t ndq = imax(0, imin(nq, M->L_dense - start));               /* its leading dense layers */
-        double f = (double)(nq - ndq) * d.F_l + (double)ndq * d.F_ld + (q == Q - 1 ? d.headF : 0.0);
-        double b = (double)(nq - ndq) * d.B_l + (double)ndq * d.B_ld + (q == Q - 1 ? K0->bwd_factor * d.headF : 0.0);
+        double f = (double)(nq - ndq) * F_l + (double)ndq * d.F_ld + (q == Q - 1 ? d.headF : 0.0);
+        double b = (double)(nq - ndq) * B_l + (double)ndq * d.B_ld + (q == Q - 1 ? K0->bwd_factor * d.headF : 0.0);
         Fq[q] = f * orc_jitter(seed, idx, q, 0);
         Bq[q] = b * orc_jitter(seed, idx, q, 1);
     }

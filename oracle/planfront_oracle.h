@@ -110,6 +110,11 @@ typedef struct {
 typedef struct {
     int64_t kind, overlap, mapped;
     double hide_frac, sched_ovh;
+    /* what the timeline simulator needs about the overlap (Sec. 3.1 "schedule"): the all-to-all is cut into
+     * n_chunks pieces (0: the simulator uses hide_frac like the analytic scorer), and while communication
+     * kernels run beside compute they hold sm_frac of the SMs */
+    int64_t n_chunks;
+    double sm_frac;
 } orc_sched_t;
 
 typedef struct {
@@ -183,6 +188,7 @@ typedef struct {
     double cF, cB, rc, tpc, a2a, xF, xB, F_l, B_l, headF, F, B, p, T_pipe, T_dp, T_opt, T_step;
     double T_dec, T_pre; /* serve */
     double F_ld, B_ld;   /* a leading dense layer's forward and backward time */
+    double cD, cE;       /* per-layer forward compute: dense part (attention, router, shared experts), experts */
     double tput_unpriced, tput;
     int64_t reason;
     int64_t why; /* ORC_WHY_* bits behind the extrapolated flag (feasible candidates only) */
@@ -197,6 +203,13 @@ uint64_t orc_space_size(const orc_problem_t *pb);
 int orc_ops_enabled(void);
 void orc_ops_reset(void);
 void orc_ops_read(int64_t out[3]);
+
+/* Makespan of one MoE layer pass on two streams (Sec. 3.2: the simulator models the overlap of compute and
+ * communication explicitly).  Compute stream: the dense part A, then n expert chunks of e_tot / n; communication
+ * stream: n dispatch chunks of d_tot / n (ready once A is done) and n combine chunks of c_tot / n (chunk i ready
+ * once expert chunk i is done); expert chunk i needs dispatch chunk i.  Each stream runs the ready op that became
+ * ready first (ties: lower op number; dispatches are numbered before combines). */
+double orc_two_stream_layer(double A, double e_tot, double d_tot, double c_tot, int n);
 
 /* score one candidate: fills detail (may be NULL); returns the reason byte */
 int orc_eval(const orc_problem_t *pb, uint64_t idx, orc_detail_t *detail);
