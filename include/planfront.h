@@ -135,6 +135,12 @@ typedef struct {
     int32_t mapped;               /* 0: the toolchain cannot emit this class (Sec. 2.1) */
     float hide_frac;              /* hidden fraction of the all-to-all when overlapped (alpha-table) */
     float sched_ovh;              /* realization overhead, applied as tput / (1 + ovh) when overlap = 1 */
+    /* What the timeline simulator needs about the overlap (Sec. 3.1, schedule): the all-to-all is cut into
+     * n_chunks pieces, 0..16 (0: pf_simulate uses hide_frac like the analytic scorer; >= 1: it runs the layer's
+     * two-stream timeline, Sec. 3.2), and communication kernels hold sm_frac of the SMs, 0 <= sm_frac <= 0.9,
+     * while they run beside compute.  pf_score ignores both. */
+    int32_t n_chunks;
+    float sm_frac;
 } pf_sched_t;
 
 typedef struct {

@@ -53,7 +53,8 @@ class PfAxes(C.Structure):
 
 
 class PfSched(C.Structure):
-    _fields_ = [("kind", i32), ("overlap", i32), ("mapped", i32), ("hide_frac", f32), ("sched_ovh", f32)]
+    _fields_ = [("kind", i32), ("overlap", i32), ("mapped", i32), ("hide_frac", f32), ("sched_ovh", f32),
+                ("n_chunks", i32), ("sm_frac", f32)]
 
 
 class PfKern(C.Structure):
@@ -275,7 +276,8 @@ class Plan:
         tb.n_sched = len(cfg["sched"])
         for i, s in enumerate(cfg["sched"]):
             tb.sched[i] = PfSched(kind=int(s["kind"]), overlap=int(s["overlap"]), mapped=int(s["mapped"]),
-                                  hide_frac=float(s["hide_frac"]), sched_ovh=float(s["sched_ovh"]))
+                                  hide_frac=float(s["hide_frac"]), sched_ovh=float(s["sched_ovh"]),
+                                  n_chunks=int(s.get("n_chunks", 0)), sm_frac=float(s.get("sm_frac", 0.0)))
         tb.n_kern = len(cfg["kern"])
         for i, k in enumerate(cfg["kern"]):
             kk = PfKern(needs_caps=int(k["needs_caps"]), avail_mask=int(k["avail_mask"]), is_native=int(k["is_native"]),

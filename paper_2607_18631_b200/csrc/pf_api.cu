@@ -235,7 +235,9 @@ extern "C" int pf_plan_create(const pf_model_t *model, const pf_cluster_t *clust
             if (has0 && axes->len[4] != 1) return PF_EINVAL;
         }
         for (int s = 0; s < tables->n_sched; s++)
-            if (tables->sched[s].kind < 0 || tables->sched[s].kind > 2) return PF_EINVAL;
+            if (tables->sched[s].kind < 0 || tables->sched[s].kind > 2 || tables->sched[s].n_chunks < 0 ||
+                tables->sched[s].n_chunks > 16 || !(tables->sched[s].sm_frac >= 0.f) || tables->sched[s].sm_frac > 0.9f)
+                return PF_EINVAL;
     } else {
         if (!in_range(0, 0, tables->n_kern - 1)) return PF_EINVAL;
         if (!in_range(1, 1, 1 << 20) || !in_range(2, 1, 1 << 20) || !in_range(3, 0, 1)) return PF_ERANGE;
@@ -346,6 +348,7 @@ extern "C" int pf_plan_create(const pf_model_t *model, const pf_cluster_t *clust
         d.sched[s].kind = tables->sched[s].kind; d.sched[s].overlap = tables->sched[s].overlap ? 1 : 0;
         d.sched[s].mapped = tables->sched[s].mapped ? 1 : 0;
         d.sched[s].hide_frac = tables->sched[s].hide_frac; d.sched[s].sched_ovh = tables->sched[s].sched_ovh;
+        d.sched[s].n_chunks = tables->sched[s].n_chunks; d.sched[s].sm_frac = tables->sched[s].sm_frac;
     }
     for (int i = 0; i < tables->n_kern; i++) {
         const pf_kern_t &k = tables->kern[i];

@@ -247,6 +247,7 @@ __device__ __forceinline__ void train_memory(const DevPlan &P, const TrainTuple 
 struct TrainTimes {
     float F_l, B_l, headF, p, T_dp, T_opt;
     float F_ld, B_ld;   // a leading dense layer (0 when the model has none)
+    float cD, cE, rc, tpc, a2a;   // a MoE layer's parts: dense and expert compute, recompute, TP and EP collectives
 };
 
 template <typename RI>
@@ -271,6 +272,7 @@ __device__ __forceinline__ void train_times(const DevPlan &P, const TrainTuple &
     const float hid = (D.ov && c.sh != PF_SHARD_ZERO1_OFFLOAD) ? P.sched[c.s].hide_frac * a2a : 0.f;
     const float xF = a2a - fminf(hid, cF);
     const float xB = a2a - fminf(hid, cB + rc);
+    T.cD = cD; T.cE = cE; T.rc = rc; T.tpc = tpc; T.a2a = a2a;
     T.F_l = cF + tpc + xF;
     T.B_l = cB + rc + tpc + xB + (c.rec == PF_REC_FULL ? tpc + xF : 0.f);
     T.headF = fdiv(t * P.f_head, dense_rate);
@@ -303,6 +305,25 @@ __device__ __forceinline__ void train_times(const DevPlan &P, const TrainTuple &
                          t_allgather((i64)D.edp, (float)P.gb * (float)M.N_exp, ldp);
         T.T_dp = (float)D.m * (2.f * ag + rs);
     }
+}
+
+// Makespan of one MoE layer pass on two streams (Sec. 3.2: the simulator models the overlap of compute and
+// communication explicitly).  Compute stream: the dense part A, then n expert chunks; communication stream: n
+// dispatch chunks (ready once A is done), then the combine chunks as their expert chunks finish -- the order a
+// first-ready-first-served stream produces, since every dispatch is ready before any combine.
+__device__ __forceinline__ float two_stream_layer(float A, float e_tot, float d_tot, float c_tot, int n)
+{
+    const float inv = fdiv(1.f, (float)n);
+    const float e = e_tot * inv, d = d_tot * inv, c = c_tot * inv;
+    float comm = A;
+    for (int i = 0; i < n; i++) comm += d;          // the stream is busy with dispatches until here
+    float dend = A, eend = A;
+    for (int i = 0; i < n; i++) {
+        dend += d;
+        eend = fmaxf(eend, dend) + e;               // expert chunk i: after chunk i-1 and its dispatch
+        comm = fmaxf(comm, eend) + c;               // combine chunk i
+    }
+    return comm;
 }
 
 // tokens/s/GPU from a pipeline time, with the realization taxes of the plans that pay them

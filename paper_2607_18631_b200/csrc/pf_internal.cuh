@@ -21,6 +21,8 @@ constexpr int kQueueCap = 4096;   // cost-model queue of the scoring kernel (ent
 struct DevSched {
     int kind, overlap, mapped;
     float hide_frac, sched_ovh;
+    int n_chunks;      // comm chunking for the simulator's two-stream layer timeline (0: use hide_frac)
+    float sm_frac;     // SMs held by communication kernels while overlapping
 };
 
 struct DevKern {

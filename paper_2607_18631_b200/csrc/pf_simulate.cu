@@ -509,6 +509,19 @@ __global__ void __launch_bounds__(kSimThreads, 4) simulate_kernel(const __grid_c
                 if (have && reason != 0) status = PF_SIM_UNSUPPORTED;
                 if (run) {
                     train_times<RI>(P, c, D, M, T);
+                    const DevSched &sc = P.sched[c.s];
+                    if (D.ov && sc.n_chunks > 0 && c.sh != PF_SHARD_ZERO1_OFFLOAD) {
+                        // the schedule says how it overlaps: the exposed communication of a MoE layer comes from
+                        // its two-stream timeline instead of the alpha-table's hidden fraction
+                        const float slow = fdiv(1.f, 1.f - sc.sm_frac), half = 0.5f * T.a2a;
+                        const float cF = T.cD + T.cE, cBt = P.bwd_factor * cF + T.rc;
+                        const float share = fdiv(T.cE, cF);
+                        const float fwd = two_stream_layer(T.cD * slow, T.cE * slow, half, half, sc.n_chunks);
+                        const float bwd = two_stream_layer(cBt * (1.f - share) * slow, cBt * share * slow, half, half,
+                                                           sc.n_chunks);
+                        T.F_l = T.tpc + fwd;
+                        T.B_l = T.tpc + bwd + (c.rec == PF_REC_FULL ? T.tpc + (fwd - cF * slow) : 0.f);
+                    }
                     if (c.pp > PF_SIM_MAX_RANKS || D.v_eff > PF_SIM_MAX_V) {
                         tput_out = train_price<RI>(P, c, D, T, train_pipe_analytic<RI>(P, c, D, T));
                         status = PF_SIM_UNSUPPORTED;
