@@ -678,6 +678,7 @@ __global__ void __launch_bounds__(kReduceThreads) reduce_final_kernel(const Redu
     __shared__ unsigned int s_hist[256];
     __shared__ unsigned long long s_prefix;
     __shared__ unsigned int s_need;
+    __shared__ int s_stop;
     const int tid = threadIdx.x, k = (int)A.k;
     const unsigned int n0 = *A.in0_count;
     unsigned long long *s_out = s_big;
@@ -689,6 +690,7 @@ __global__ void __launch_bounds__(kReduceThreads) reduce_final_kernel(const Redu
             s_prefix = 0ull;
             s_need = (unsigned int)k;
             s_count = 0;
+            s_stop = 0;
         }
         __syncthreads();
         if (n0 > (unsigned int)k) {
@@ -720,6 +722,8 @@ __global__ void __launch_bounds__(kReduceThreads) reduce_final_kernel(const Redu
                             if (run + h >= need) {
                                 s_prefix = prefix | ((unsigned long long)d << shift);
                                 s_need = need - run;
+                                // every key of this digit is needed: the cut is the digit's lowest key
+                                if (run + h == need) s_stop = 1;
                                 break;
                             }
                             run += h;
@@ -727,6 +731,7 @@ __global__ void __launch_bounds__(kReduceThreads) reduce_final_kernel(const Redu
                     }
                 }
                 __syncthreads();
+                if (s_stop) break;
             }
         }
         const unsigned long long cut = n0 > (unsigned int)k ? s_prefix : 1ull;  // keys are distinct: exactly k pass

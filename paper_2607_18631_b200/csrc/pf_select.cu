@@ -264,12 +264,19 @@ __global__ void __launch_bounds__(kSelThreads) sel_count_kernel(const __grid_con
         }
         return;
     }
+    const bool all = A.ctrl->take_all != 0;
+    if (all) {   // every eligible candidate is taken: the first pass has counted them already
+        if (threadIdx.x == 0) {
+            A.blk_gt[blockIdx.x] = A.blk_elig[blockIdx.x];
+            A.blk_eq[blockIdx.x] = 0;
+        }
+        return;
+    }
     if (threadIdx.x == 0) s_gt = s_eq = 0;
     __syncthreads();
     const uint64_t lo = (uint64_t)blockIdx.x * A.chunk;
     const uint64_t hi = min(lo + A.chunk, A.count);
     const uint32_t thr = A.ctrl->thr_bits;
-    const bool all = A.ctrl->take_all != 0;
     unsigned int gt = 0, eq = 0;
     uint4 r[kSelTiles];
     load_chunk(A, lo, hi, r);
@@ -294,25 +301,23 @@ __global__ void __launch_bounds__(kSelThreads) sel_count_kernel(const __grid_con
 __global__ void __launch_bounds__(1024) sel_blockscan_kernel(const SelArgs A, int nblocks)
 {
     __shared__ unsigned long long s_warp[32];
-    __shared__ unsigned long long s_carry_g, s_carry_e;
     const int tid = threadIdx.x;
-    if (tid == 0) s_carry_g = s_carry_e = 0;
-    __syncthreads();
-    for (int base = 0; base < nblocks; base += 1024) {
-        const int b = base + tid;
-        const unsigned long long cg = b < nblocks ? A.blk_gt[b] : 0, ce = b < nblocks ? A.blk_eq[b] : 0;
-        const unsigned long long ig = block_prefix_1024(cg, s_warp);
-        const unsigned long long ie = block_prefix_1024(ce, s_warp);
-        if (b < nblocks) {
-            A.blk_gt[b] = s_carry_g + ig - cg;
-            A.blk_eq[b] = s_carry_e + ie - ce;
-        }
-        __syncthreads();
-        if (tid == 1023) {
-            s_carry_g += ig;
-            s_carry_e += ie;
-        }
-        __syncthreads();
+    // every thread owns a run of consecutive blocks: serial sums inside the run, one block-wide scan across runs
+    const int per = (nblocks + 1023) / 1024;
+    const int lo = min(tid * per, nblocks), hi = min(lo + per, nblocks);
+    unsigned long long sg = 0, se = 0;
+    for (int b = lo; b < hi; b++) {
+        sg += A.blk_gt[b];
+        se += A.blk_eq[b];
+    }
+    unsigned long long run_g = block_prefix_1024(sg, s_warp) - sg;
+    unsigned long long run_e = block_prefix_1024(se, s_warp) - se;
+    for (int b = lo; b < hi; b++) {
+        const unsigned long long cg = A.blk_gt[b], ce = A.blk_eq[b];
+        A.blk_gt[b] = run_g;
+        A.blk_eq[b] = run_e;
+        run_g += cg;
+        run_e += ce;
     }
     if (tid == 0) {
         const SelCtrl *c = A.ctrl;
