@@ -20,6 +20,7 @@ struct SelCtrl {
     unsigned long long target;    // S
     uint32_t b1, thr_bits;
     int take_all;
+    unsigned int n_elig;          // chunks that hold eligible candidates (length of SelArgs::elig_list)
 };
 
 struct SelArgs {
@@ -28,7 +29,8 @@ struct SelArgs {
     const float *tput;
     unsigned int *hist1, *hist2;      // kBins each
     unsigned int *coarse1, *coarse2;  // 256 bins each: sums over groups of 256 fine bins
-    unsigned int *blk_elig;           // eligible candidates per block, written by the first pass
+    unsigned int *blk_elig;           // eligible candidates per chunk, written by the first pass
+    unsigned int *elig_list;          // the chunks with blk_elig > 0, in no particular order
     SelCtrl *ctrl;
     unsigned long long *blk_gt, *blk_eq;  // per block counts, then exclusive prefixes
     uint64_t *surv_idx, *surv_count;
@@ -117,15 +119,14 @@ __device__ __forceinline__ void load_chunk(const SelArgs &A, uint64_t lo, uint64
     }
 }
 
-__global__ void __launch_bounds__(kSelThreads) sel_hist_kernel(const __grid_constant__ DevPlan P, const SelArgs A,
-                                                                const int32_t *vals, int pass)
+// One chunk of the histogram passes.  pass 0: every chunk; pass 1: the chunks on the eligible list.
+__device__ __forceinline__ void sel_hist_chunk(const DevPlan &P, const SelArgs &A, const int32_t *vals, int pass,
+                                               unsigned int chunk, unsigned int *s_elig)
 {
-    __shared__ unsigned int s_elig;
-    const uint64_t lo = (uint64_t)blockIdx.x * A.chunk;
+    const uint64_t lo = (uint64_t)chunk * A.chunk;
     const uint64_t hi = min(lo + A.chunk, A.count);
-    if (pass == 1 && (A.ctrl->take_all || A.blk_elig[blockIdx.x] == 0)) return;   // nothing to refine here
     if (pass == 0) {
-        if (threadIdx.x == 0) s_elig = 0;
+        if (threadIdx.x == 0) *s_elig = 0;
         __syncthreads();
     }
     const uint32_t b1 = pass == 1 ? A.ctrl->b1 : 0;
@@ -147,10 +148,29 @@ __global__ void __launch_bounds__(kSelThreads) sel_hist_kernel(const __grid_cons
         });
     }
     if (pass == 0) {
-        if (mine) atomicAdd(&s_elig, mine);
+        if (mine) atomicAdd(s_elig, mine);
         __syncthreads();
-        if (threadIdx.x == 0) A.blk_elig[blockIdx.x] = s_elig;
+        if (threadIdx.x == 0) {
+            const unsigned int n = *s_elig;
+            A.blk_elig[chunk] = n;
+            // later passes only visit the chunks on this list
+            if (n) A.elig_list[atomicAdd(&A.ctrl->n_elig, 1u)] = chunk;
+        }
     }
+}
+
+__global__ void __launch_bounds__(kSelThreads) sel_hist_kernel(const __grid_constant__ DevPlan P, const SelArgs A,
+                                                                const int32_t *vals, int pass)
+{
+    __shared__ unsigned int s_elig;
+    if (pass == 0) {
+        sel_hist_chunk(P, A, vals, 0, blockIdx.x, &s_elig);
+        return;
+    }
+    if (A.ctrl->take_all) return;   // nothing to refine
+    const unsigned int n_list = A.ctrl->n_elig;
+    for (unsigned int li = blockIdx.x; li < n_list; li += gridDim.x)
+        sel_hist_chunk(P, A, vals, 1, A.elig_list[li], &s_elig);
 }
 
 // Block-wide inclusive prefix sum over 1024 threads (warp shuffles, then the warp totals).
@@ -253,71 +273,71 @@ __global__ void __launch_bounds__(256) sel_scan_kernel(const SelArgs A, int pass
     }
 }
 
+// Per-chunk counts of admitted candidates, for the chunks on the eligible list (the others keep their zeros).
 __global__ void __launch_bounds__(kSelThreads) sel_count_kernel(const __grid_constant__ DevPlan P, const SelArgs A,
                                                                  const int32_t *vals)
 {
     __shared__ unsigned int s_gt, s_eq;
-    if (A.blk_elig[blockIdx.x] == 0) {   // nothing eligible in this chunk: its counts are zero
-        if (threadIdx.x == 0) {
-            A.blk_gt[blockIdx.x] = 0;
-            A.blk_eq[blockIdx.x] = 0;
-        }
-        return;
-    }
+    const unsigned int n_list = A.ctrl->n_elig;
     const bool all = A.ctrl->take_all != 0;
-    if (all) {   // every eligible candidate is taken: the first pass has counted them already
-        if (threadIdx.x == 0) {
-            A.blk_gt[blockIdx.x] = A.blk_elig[blockIdx.x];
-            A.blk_eq[blockIdx.x] = 0;
-        }
-        return;
-    }
-    if (threadIdx.x == 0) s_gt = s_eq = 0;
-    __syncthreads();
-    const uint64_t lo = (uint64_t)blockIdx.x * A.chunk;
-    const uint64_t hi = min(lo + A.chunk, A.count);
     const uint32_t thr = A.ctrl->thr_bits;
-    unsigned int gt = 0, eq = 0;
-    uint4 r[kSelTiles];
-    load_chunk(A, lo, hi, r);
+    for (unsigned int li = blockIdx.x; li < n_list; li += gridDim.x) {
+        const unsigned int chunk = A.elig_list[li];
+        if (all) {   // every eligible candidate is taken: the first pass has counted them already
+            if (threadIdx.x == 0) {
+                A.blk_gt[chunk] = A.blk_elig[chunk];
+                A.blk_eq[chunk] = 0;
+            }
+            continue;
+        }
+        if (threadIdx.x == 0) s_gt = s_eq = 0;
+        __syncthreads();
+        const uint64_t lo = (uint64_t)chunk * A.chunk;
+        const uint64_t hi = min(lo + A.chunk, A.count);
+        unsigned int gt = 0, eq = 0;
+        uint4 r[kSelTiles];
+        load_chunk(A, lo, hi, r);
 #pragma unroll
-    for (int t = 0; t < kSelTiles; t++) {
-        const uint64_t e = lo + (uint64_t)t * kSelTile + (uint64_t)threadIdx.x * 16;
-        for_each_eligible16(P, vals, A, e, r[t], [&](uint64_t, uint32_t bits) {
-            if (all || bits > thr) gt++;
-            else if (bits == thr) eq++;
-        });
-    }
-    if (gt) atomicAdd(&s_gt, gt);
-    if (eq) atomicAdd(&s_eq, eq);
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        A.blk_gt[blockIdx.x] = s_gt;
-        A.blk_eq[blockIdx.x] = s_eq;
+        for (int t = 0; t < kSelTiles; t++) {
+            const uint64_t e = lo + (uint64_t)t * kSelTile + (uint64_t)threadIdx.x * 16;
+            for_each_eligible16(P, vals, A, e, r[t], [&](uint64_t, uint32_t bits) {
+                if (bits > thr) gt++;
+                else if (bits == thr) eq++;
+            });
+        }
+        if (gt) atomicAdd(&s_gt, gt);
+        if (eq) atomicAdd(&s_eq, eq);
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            A.blk_gt[chunk] = s_gt;
+            A.blk_eq[chunk] = s_eq;
+        }
+        __syncthreads();
     }
 }
 
-// exclusive prefix over the per-block counts (tiles of 1024 blocks with a carry) + the survivor count
+// Exclusive prefix over the per-chunk counts + the survivor count.  One block walks the chunks in tiles of 1024;
+// both counts travel through one scan as (greater << 32 | equal) -- their totals stay below 2^32 -- and the next
+// tile's counts are loaded before the current tile is scanned.
 __global__ void __launch_bounds__(1024) sel_blockscan_kernel(const SelArgs A, int nblocks)
 {
     __shared__ unsigned long long s_warp[32];
     const int tid = threadIdx.x;
-    // every thread owns a run of consecutive blocks: serial sums inside the run, one block-wide scan across runs
-    const int per = (nblocks + 1023) / 1024;
-    const int lo = min(tid * per, nblocks), hi = min(lo + per, nblocks);
-    unsigned long long sg = 0, se = 0;
-    for (int b = lo; b < hi; b++) {
-        sg += A.blk_gt[b];
-        se += A.blk_eq[b];
-    }
-    unsigned long long run_g = block_prefix_1024(sg, s_warp) - sg;
-    unsigned long long run_e = block_prefix_1024(se, s_warp) - se;
-    for (int b = lo; b < hi; b++) {
-        const unsigned long long cg = A.blk_gt[b], ce = A.blk_eq[b];
-        A.blk_gt[b] = run_g;
-        A.blk_eq[b] = run_e;
-        run_g += cg;
-        run_e += ce;
+    unsigned long long carry = 0ull;
+    unsigned long long nxt = tid < nblocks ? ((A.blk_gt[tid] << 32) | A.blk_eq[tid]) : 0ull;
+    for (int base = 0; base < nblocks; base += 1024) {
+        const int b = base + tid, bn = b + 1024;
+        const unsigned long long cur = nxt;
+        nxt = bn < nblocks ? ((A.blk_gt[bn] << 32) | A.blk_eq[bn]) : 0ull;
+        const unsigned long long incl = block_prefix_1024(cur, s_warp);
+        const unsigned long long total = s_warp[31];
+        const unsigned long long excl = carry + incl - cur;
+        if (b < nblocks) {
+            A.blk_gt[b] = excl >> 32;
+            A.blk_eq[b] = excl & 0xFFFFFFFFull;
+        }
+        carry += total;
+        __syncthreads();   // s_warp is rewritten by the next tile's scan
     }
     if (tid == 0) {
         const SelCtrl *c = A.ctrl;
@@ -326,21 +346,19 @@ __global__ void __launch_bounds__(1024) sel_blockscan_kernel(const SelArgs A, in
 }
 
 // Ordered write: position of an admitted candidate = (# taken "greater" before it) + min(# "equal" before it, need_eq)
-__global__ void __launch_bounds__(kSelThreads) sel_write_kernel(const __grid_constant__ DevPlan P, const SelArgs A,
-                                                                 const int32_t *vals)
+__device__ __forceinline__ void sel_write_chunk(const DevPlan &P, const SelArgs &A, const int32_t *vals,
+                                                unsigned int chunk, unsigned int *s_gt, unsigned int *s_eq,
+                                                unsigned long long &s_run_gt, unsigned long long &s_run_eq)
 {
-    __shared__ unsigned int s_gt[kSelThreads], s_eq[kSelThreads];
-    __shared__ unsigned long long s_run_gt, s_run_eq;
     const int tid = threadIdx.x;
-    if (A.blk_elig[blockIdx.x] == 0) return;   // nothing to write from this chunk
-    const uint64_t lo = (uint64_t)blockIdx.x * A.chunk;
+    const uint64_t lo = (uint64_t)chunk * A.chunk;
     const uint64_t hi = min(lo + A.chunk, A.count);
     const uint32_t thr = A.ctrl->thr_bits;
     const bool all = A.ctrl->take_all != 0;
     const unsigned long long need_eq = all ? 0ull : A.ctrl->need_eq;
     if (tid == 0) {
-        s_run_gt = A.blk_gt[blockIdx.x];
-        s_run_eq = A.blk_eq[blockIdx.x];
+        s_run_gt = A.blk_gt[chunk];
+        s_run_eq = A.blk_eq[chunk];
     }
     uint4 r[kSelTiles];
     load_chunk(A, lo, hi, r);
@@ -387,8 +405,20 @@ __global__ void __launch_bounds__(kSelThreads) sel_write_kernel(const __grid_con
     }
 }
 
+__global__ void __launch_bounds__(kSelThreads) sel_write_kernel(const __grid_constant__ DevPlan P, const SelArgs A,
+                                                                 const int32_t *vals)
+{
+    __shared__ unsigned int s_gt[kSelThreads], s_eq[kSelThreads];
+    __shared__ unsigned long long s_run_gt, s_run_eq;
+    const unsigned int n_list = A.ctrl->n_elig;
+    for (unsigned int li = blockIdx.x; li < n_list; li += gridDim.x) {
+        sel_write_chunk(P, A, vals, A.elig_list[li], s_gt, s_eq, s_run_gt, s_run_eq);
+        __syncthreads();   // the running offsets are reset by the next chunk
+    }
+}
+
 struct SelLayout {
-    size_t off_ctrl, off_hist1, off_hist2, off_coarse, off_gt, off_eq, off_elig, total;
+    size_t off_ctrl, off_hist1, off_hist2, off_coarse, off_gt, off_eq, off_elig, off_list, total;
     int nblocks;
     uint64_t chunk;
 };
@@ -410,7 +440,8 @@ static SelLayout sel_layout(const pf_plan_t *p, uint64_t count)
     size_t per = (((size_t)l.nblocks + 1) * 8 + 255) & ~(size_t)255;
     l.off_eq = l.off_gt + per;
     l.off_elig = l.off_eq + per;
-    l.total = l.off_elig + per;
+    l.off_list = l.off_elig + per;
+    l.total = l.off_list + per;
     return l;
 }
 
@@ -445,18 +476,23 @@ extern "C" int pf_select_survivors(pf_plan_t *p, uint64_t first, uint64_t count,
     a.coarse1 = (unsigned int *)(ws + lay.off_coarse);
     a.coarse2 = a.coarse1 + 256;
     a.blk_elig = (unsigned int *)(ws + lay.off_elig);
+    a.elig_list = (unsigned int *)(ws + lay.off_list);
     a.blk_gt = (unsigned long long *)(ws + lay.off_gt);
     a.blk_eq = (unsigned long long *)(ws + lay.off_eq);
     a.surv_idx = d_surv_idx; a.surv_count = d_surv_count; a.chunk = lay.chunk;
-    PF_CUDA_TRY(cudaMemsetAsync(ws, 0, lay.off_gt, st), "pf_select_survivors: clear");
+    // control words, histograms and the per-chunk counts start at zero (chunks that are not on the eligible list
+    // are never written again)
+    PF_CUDA_TRY(cudaMemsetAsync(ws, 0, lay.off_elig, st), "pf_select_survivors: clear");
+    // the passes after the first visit the eligible chunks only: a grid that fills the GPU walks the list
+    const int list_grid = lay.nblocks < p->sm_count * 8 ? lay.nblocks : p->sm_count * 8;
     timing_begin(p, PF_T_SELECT, st);
     sel_hist_kernel<<<lay.nblocks, kSelThreads, 0, st>>>(p->dev, a, p->d_vals, 0);
     sel_scan_kernel<<<1, 256, 0, st>>>(a, 0);
-    sel_hist_kernel<<<lay.nblocks, kSelThreads, 0, st>>>(p->dev, a, p->d_vals, 1);
+    sel_hist_kernel<<<list_grid, kSelThreads, 0, st>>>(p->dev, a, p->d_vals, 1);
     sel_scan_kernel<<<1, 256, 0, st>>>(a, 1);
-    sel_count_kernel<<<lay.nblocks, kSelThreads, 0, st>>>(p->dev, a, p->d_vals);
+    sel_count_kernel<<<list_grid, kSelThreads, 0, st>>>(p->dev, a, p->d_vals);
     sel_blockscan_kernel<<<1, 1024, 0, st>>>(a, lay.nblocks);
-    sel_write_kernel<<<lay.nblocks, kSelThreads, 0, st>>>(p->dev, a, p->d_vals);
+    sel_write_kernel<<<list_grid, kSelThreads, 0, st>>>(p->dev, a, p->d_vals);
     timing_end(p, PF_T_SELECT, 7, st);
     for (int i = 0; i < 7; i++) count_launch();
     PF_CUDA_TRY(cudaGetLastError(), "pf_select_survivors launch");
