@@ -435,7 +435,7 @@ __device__ __forceinline__ void sim_rounds_dual(volatile float *tl, const float 
 template <typename RI>
 __global__ void __launch_bounds__(kSimThreads, 4) simulate_kernel(const __grid_constant__ DevPlan P, const SimArgs A)
 {
-    extern __shared__ float s_mem[];
+    extern __shared__ __align__(16) float s_mem[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint32_t seed_mixed = mix32(A.seed + 0x9e3779b9u);
     const int E_hi = sim_class_entries(A.cls_hi);
@@ -554,7 +554,12 @@ __global__ void __launch_bounds__(kSimThreads, 4) simulate_kernel(const __grid_c
                         durB[q] = (nq * T.B_l + nd * T.B_ld + (last ? P.bwd_factor * T.headF : 0.f)) *
                                   jitter(seed_mixed, idx, q, 1);
                     }
-                    for (int i = glane; i < n_entries; i += g) tl[i] = 0.f;
+                    // clear the timeline with 16-byte stores (the slot is a multiple of four words, 16-byte aligned)
+                    {
+                        float4 *tl4 = reinterpret_cast<float4 *>(const_cast<float *>(tl));
+                        const int n4 = (n_entries + 3) >> 2;
+                        for (int i = glane; i < n4; i += g) tl4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    }
                 }
                 __syncwarp();
 
