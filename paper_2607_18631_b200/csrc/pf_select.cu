@@ -163,7 +163,7 @@ __global__ void __launch_bounds__(kSelThreads) sel_hist_kernel(const __grid_cons
                                                                 const int32_t *vals, int pass)
 {
     __shared__ unsigned int s_elig;
-    if (pass == 0) {
+    if (pass == 0) {   // one block per chunk: the whole array is read, the more loads in flight the better
         sel_hist_chunk(P, A, vals, 0, blockIdx.x, &s_elig);
         return;
     }
@@ -316,28 +316,79 @@ __global__ void __launch_bounds__(kSelThreads) sel_count_kernel(const __grid_con
     }
 }
 
-// Exclusive prefix over the per-chunk counts + the survivor count.  One block walks the chunks in tiles of 1024;
-// both counts travel through one scan as (greater << 32 | equal) -- their totals stay below 2^32 -- and the next
-// tile's counts are loaded before the current tile is scanned.
+// Exclusive prefix over the per-chunk counts + the survivor count.  One block; both counts travel through one
+// scan as (greater << 32 | equal) -- their totals stay below 2^32.  Up to kScanTiles * 1024 chunks are scanned
+// in one go: every thread holds one entry of every tile, the tiles' warp-level scans run side by side, and one
+// round through shared memory turns the warp totals into offsets.  Longer lists are walked tile by tile.
+constexpr int kScanTiles = 16;
 __global__ void __launch_bounds__(1024) sel_blockscan_kernel(const SelArgs A, int nblocks)
 {
     __shared__ unsigned long long s_warp[32];
-    const int tid = threadIdx.x;
-    unsigned long long carry = 0ull;
-    unsigned long long nxt = tid < nblocks ? ((A.blk_gt[tid] << 32) | A.blk_eq[tid]) : 0ull;
-    for (int base = 0; base < nblocks; base += 1024) {
-        const int b = base + tid, bn = b + 1024;
-        const unsigned long long cur = nxt;
-        nxt = bn < nblocks ? ((A.blk_gt[bn] << 32) | A.blk_eq[bn]) : 0ull;
-        const unsigned long long incl = block_prefix_1024(cur, s_warp);
-        const unsigned long long total = s_warp[31];
-        const unsigned long long excl = carry + incl - cur;
-        if (b < nblocks) {
-            A.blk_gt[b] = excl >> 32;
-            A.blk_eq[b] = excl & 0xFFFFFFFFull;
+    __shared__ unsigned long long s_tot[kScanTiles][33];   // warp totals per tile, then their exclusive prefixes
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (nblocks <= kScanTiles * 1024) {
+        const int tiles = (nblocks + 1023) / 1024;
+        unsigned long long v[kScanTiles], x[kScanTiles];
+#pragma unroll
+        for (int k = 0; k < kScanTiles; k++) {
+            const int b = k * 1024 + tid;
+            v[k] = (k < tiles && b < nblocks) ? ((A.blk_gt[b] << 32) | A.blk_eq[b]) : 0ull;
+            x[k] = v[k];
         }
-        carry += total;
-        __syncthreads();   // s_warp is rewritten by the next tile's scan
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+#pragma unroll
+            for (int k = 0; k < kScanTiles; k++) {
+                const unsigned long long y = __shfl_up_sync(0xFFFFFFFFu, x[k], off);
+                if (lane >= off) x[k] += y;
+            }
+        }
+        if (lane == 31) {
+#pragma unroll
+            for (int k = 0; k < kScanTiles; k++) s_tot[k][warp] = x[k];
+        }
+        __syncthreads();
+        // warp k turns tile k's 32 warp totals into exclusive prefixes and leaves the tile total in slot 32
+        if (warp < kScanTiles) {
+            const unsigned long long t = s_tot[warp][lane];
+            unsigned long long incl = t;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const unsigned long long y = __shfl_up_sync(0xFFFFFFFFu, incl, off);
+                if (lane >= off) incl += y;
+            }
+            s_tot[warp][lane] = incl - t;
+            if (lane == 31) s_tot[warp][32] = incl;
+        }
+        __syncthreads();
+        unsigned long long carry = 0ull;
+#pragma unroll
+        for (int k = 0; k < kScanTiles; k++) {
+            const int b = k * 1024 + tid;
+            if (k < tiles && b < nblocks) {
+                const unsigned long long excl = carry + s_tot[k][warp] + x[k] - v[k];
+                A.blk_gt[b] = excl >> 32;
+                A.blk_eq[b] = excl & 0xFFFFFFFFull;
+            }
+            carry += s_tot[k][32];
+        }
+    } else {
+        unsigned long long carry = 0ull;
+        unsigned long long nxt = tid < nblocks ? ((A.blk_gt[tid] << 32) | A.blk_eq[tid]) : 0ull;
+        for (int base = 0; base < nblocks; base += 1024) {
+            const int b = base + tid, bn = b + 1024;
+            const unsigned long long cur = nxt;
+            nxt = bn < nblocks ? ((A.blk_gt[bn] << 32) | A.blk_eq[bn]) : 0ull;
+            const unsigned long long incl = block_prefix_1024(cur, s_warp);
+            const unsigned long long total = s_warp[31];
+            const unsigned long long excl = carry + incl - cur;
+            if (b < nblocks) {
+                A.blk_gt[b] = excl >> 32;
+                A.blk_eq[b] = excl & 0xFFFFFFFFull;
+            }
+            carry += total;
+            __syncthreads();   // s_warp is rewritten by the next tile's scan
+        }
     }
     if (tid == 0) {
         const SelCtrl *c = A.ctrl;
@@ -372,19 +423,27 @@ __device__ __forceinline__ void sel_write_chunk(const DevPlan &P, const SelArgs 
             else if (bits == thr) eq++;
         });
         if (!__syncthreads_or((int)(gt | eq))) continue;   // nothing eligible in this tile (the common case)
-        s_gt[tid] = gt;
-        s_eq[tid] = eq;
-        __syncthreads();
-        // inclusive Hillis-Steele scan of the per-thread counts
-        for (int off = 1; off < kSelThreads; off <<= 1) {
-            unsigned int ag = tid >= off ? s_gt[tid - off] : 0, ae = tid >= off ? s_eq[tid - off] : 0;
-            __syncthreads();
-            s_gt[tid] += ag;
-            s_eq[tid] += ae;
-            __syncthreads();
+        // inclusive scan of the per-thread counts: both travel as (gt << 16 | eq) -- a thread holds at most 16 of
+        // each, a tile at most 4096 -- through warp shuffles, then across the eight warp totals
+        const int lane = tid & 31, warp = tid >> 5;
+        unsigned int x = (gt << 16) | eq;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const unsigned int y = __shfl_up_sync(0xFFFFFFFFu, x, off);
+            if (lane >= off) x += y;
         }
-        unsigned long long my_gt = s_run_gt + (s_gt[tid] - gt);
-        unsigned long long my_eq = s_run_eq + (s_eq[tid] - eq);
+        if (lane == 31) s_gt[warp] = x;
+        __syncthreads();
+        unsigned int before = 0, total = 0;
+#pragma unroll
+        for (int w = 0; w < kSelThreads / 32; w++) {
+            const unsigned int wt = s_gt[w];
+            if (w < warp) before += wt;
+            total += wt;
+        }
+        x += before;
+        unsigned long long my_gt = s_run_gt + ((x >> 16) - gt);
+        unsigned long long my_eq = s_run_eq + ((x & 0xFFFFu) - eq);
         if (gt | eq)
             for_each_eligible16(P, vals, A, e, r[t], [&](uint64_t rel, uint32_t bits) {
                 if (all || bits > thr) {
@@ -397,9 +456,9 @@ __device__ __forceinline__ void sel_write_chunk(const DevPlan &P, const SelArgs 
                 }
             });
         __syncthreads();
-        if (tid == kSelThreads - 1) {
-            s_run_gt += s_gt[tid];
-            s_run_eq += s_eq[tid];
+        if (tid == 0) {
+            s_run_gt += total >> 16;
+            s_run_eq += total & 0xFFFFu;
         }
         __syncthreads();
     }
