@@ -3,13 +3,18 @@
 //
 // Work decomposition.  The index space is cut into slabs: one slab = all combinations of the `n_inner`
 // fastest-varying axes (<= 16384 candidates) for one combination of the remaining (outer) axes.  A
-// persistent grid (a few blocks per SM) pulls slab numbers from an atomic counter.  For each slab one
-// thread decodes the outer digits and evaluates the leading rules that depend on outer axes only; when one
-// of them fails the whole slab has the same reason and the block just streams constant bytes into the
-// dense outputs with 16-byte stores.  Otherwise each thread takes candidates slab_base + j, decodes the
-// inner digits with multiply-high divisions and runs the remaining rules, the memory model and the cost
-// model in registers.  Feasible candidates are offered to a shared-memory top-k buffer; each block writes
-// its k best keys at the end and a small merge kernel reduces the per-block lists.
+// persistent grid (four blocks per SM) draws tickets from an atomic counter; a table built by two small
+// launches (and kept in the plan per range) maps tickets to slabs so that the slabs that must be evaluated
+// come first, interleaved with a few constant ones, and the rest of the constant ones come last.
+//   - Constant slab: a rule that depends on the outer axes alone fails, every candidate has the same reason;
+//     the block streams that byte and zeros into the dense outputs with 16-byte stores.
+//   - Evaluated slab: rules 4-7 go into a per-slab table over (sched, mb, v); inside a passing entry only the
+//     kernel variant and the recompute mode vary, so rules 8-10 and the memory model are worked out once per
+//     entry and looked up per candidate; the few candidates that pass the memory gate are queued and costed
+//     one per thread.  The slab's outputs are written like a constant slab's: zeros up front, a reason image
+//     collected in shared memory and copied out once, scattered patches only for gate-reaching candidates.
+// Feasible candidates are offered to a shared-memory top-k buffer; each block appends its best keys to a
+// compact list and the reduce kernels below finish the top-k.
 #include "pf_eval.cuh"
 
 namespace pf {
@@ -265,7 +270,8 @@ __global__ void __launch_bounds__(kThreads, 4) score_kernel(const __grid_constan
         if (tid == 0) {
             word_next = (order && tkt_next < A.n_slabs) ? __ldcg(order + tkt_next) : 0u;
             tkt_after = atomicAdd(A.slab_counter, 1u);
-            if (want_topk) gthr_next = *reinterpret_cast<volatile unsigned long long *>(A.g_thr);
+            // the grid-wide threshold only matters to evaluated slabs: refresh it on those
+            if (want_topk && s_slab.pre_reason == 0) gthr_next = *reinterpret_cast<volatile unsigned long long *>(A.g_thr);
         }
         // end of a slab: set up the next one from what was requested at its top
         auto finish_slab = [&]() {

@@ -3,8 +3,8 @@
 // index order, as a two-level radix select on the fp32 score bits followed by an ordered compaction:
 //   hist(hi 16 bits) -> scan -> hist(lo 16 bits inside the threshold bin) -> scan -> per-block counts ->
 //   block-offset scan -> ordered write.
-// Every pass reads the reason bytes with 16-byte loads and touches a score only where the candidate is
-// feasible, so a sparse space costs little more than one byte per candidate per pass.
+// The first pass reads every reason byte with 16-byte loads (a score is touched only where the candidate is
+// feasible) and lists the chunks that hold eligible candidates; the later passes visit only those.
 #include "pf_internal.cuh"
 
 namespace pf {
@@ -398,7 +398,7 @@ __global__ void __launch_bounds__(1024) sel_blockscan_kernel(const SelArgs A, in
 
 // Ordered write: position of an admitted candidate = (# taken "greater" before it) + min(# "equal" before it, need_eq)
 __device__ __forceinline__ void sel_write_chunk(const DevPlan &P, const SelArgs &A, const int32_t *vals,
-                                                unsigned int chunk, unsigned int *s_gt, unsigned int *s_eq,
+                                                unsigned int chunk, unsigned int *s_gt,
                                                 unsigned long long &s_run_gt, unsigned long long &s_run_eq)
 {
     const int tid = threadIdx.x;
@@ -467,11 +467,11 @@ __device__ __forceinline__ void sel_write_chunk(const DevPlan &P, const SelArgs 
 __global__ void __launch_bounds__(kSelThreads) sel_write_kernel(const __grid_constant__ DevPlan P, const SelArgs A,
                                                                  const int32_t *vals)
 {
-    __shared__ unsigned int s_gt[kSelThreads], s_eq[kSelThreads];
+    __shared__ unsigned int s_gt[kSelThreads / 32];   // warp totals of a tile's scan
     __shared__ unsigned long long s_run_gt, s_run_eq;
     const unsigned int n_list = A.ctrl->n_elig;
     for (unsigned int li = blockIdx.x; li < n_list; li += gridDim.x) {
-        sel_write_chunk(P, A, vals, A.elig_list[li], s_gt, s_eq, s_run_gt, s_run_eq);
+        sel_write_chunk(P, A, vals, A.elig_list[li], s_gt, s_run_gt, s_run_eq);
         __syncthreads();   // the running offsets are reset by the next chunk
     }
 }
@@ -485,7 +485,7 @@ struct SelLayout {
 static SelLayout sel_layout(const pf_plan_t *p, uint64_t count)
 {
     SelLayout l;
-    // contiguous chunks of 16 tiles (256 threads x 16 candidates each): many more blocks than SMs, so a
+    // contiguous chunks of kSelTiles tiles (256 threads x 16 candidates each): many more blocks than SMs, so a
     // chunk that happens to hold most of the feasible candidates does not hold up the rest
     uint64_t chunk = (uint64_t)kSelTiles * kSelTile;
     l.chunk = chunk;
