@@ -25,8 +25,16 @@
  * ep8 -> ep4 -> ep2 increments), the tax rule, rule outcomes the paper states (27 layers vs
  * pp*v, serving dp != ep, DualPipe unmapped), the 1F1B bubble closed form, the interleaved
  * closed form, brute-force enumeration of the tiny space, and monotonicity invariants.
+ * Later additions and their pins: the operation tally (hand counts); the sharding dimension (zero1
+ * bit-identity, the printed optimizer sizes, one-rank special cases, the tax rule); the calibration
+ * domain (inclusive range, unattached = factory model); leading dense layers (a reconstructed
+ * reference model reproduces the printed 0.892e9 dense parameters and 1.34 / 22.93 GB optimizer
+ * state); the two-stream layer timeline (an independent event-driven simulation, closed forms).
  * PARITY UNPINNED: absolute throughputs (the paper's cost constants are not published), the
- * DualPipe analytic closed form and its startup divisor, and the serving time model.
+ * DualPipe analytic closed form and its startup divisor, the serving time model, the absolute
+ * times of the offloaded and fully sharded regimes, the activation and time formulas of a leading
+ * dense layer beyond its FLOP count, and the choice of the two-stream timeline's op graph (the
+ * paper names the ingredients, not the graph).
  */
 #ifndef PLANFRONT_ORACLE_H
 #define PLANFRONT_ORACLE_H
