@@ -304,39 +304,63 @@ __global__ void __launch_bounds__(256) sim_scatter_kernel(const SimArgs A)
         moved = false;                                                   \
     }
 
-// 1F1B: rank = stage = lane; `warm` forwards, then one forward / one backward, then the remaining backwards
+// The static 1F1B and interleaved orders have one shape per rank: `warm` forward units, then forward / backward
+// pairs, then the remaining backward units.  With nF forwards and nB backwards done, the next op is a forward
+// iff nF < U and nF - nB <= warm, otherwise a backward.  One loop iteration therefore offers every lane a forward
+// step and then a backward step, each straight-line code for its one kind of op; in the steady state a lane does
+// both, so an iteration retires two ops for about the instructions one generic step would take.  A value written
+// in a step is seen by the neighbour's next step of the same kind, one iteration later.
+#define PF_SIM_ITER_END()                                                \
+    if (!__any_sync(0xFFFFFFFFu, nF + nB < total_ops)) break;            \
+    if ((++rounds & 63) == 0) {                                          \
+        if (!__any_sync(0xFFFFFFFFu, moved)) break;                      \
+        moved = false;                                                   \
+    }
+
+// 1F1B: rank = stage = lane
 __device__ __forceinline__ void sim_rounds_1f1b(volatile float *tl, const float *durF, const float *durB, int glane,
                                                 int pp, int nj, int warm, int total_ops, float lat, float &clock_out,
                                                 int &done_out)
 {
-    const bool depF = glane > 0, depB = glane < pp - 1;
-    volatile float *inF = tl + (depF ? glane - 1 : glane) * nj, *inB = tl + (depB ? glane + 1 : glane) * nj;
-    volatile float *out = tl + glane * nj;
-    const float dF = total_ops ? durF[glane] : 0.f, dB = total_ops ? durB[glane] : 0.f;
-    int nF = 0, nB = 0, done = 0, rounds = 0;
+    // lanes beyond the pipeline depth take no part: they poll row 0 and never act
+    const bool active = total_ops > 0;
+    const int row = active ? glane : 0;
+    const bool depF = active && row > 0, depB = active && row < pp - 1;
+    volatile float *inF = tl + (depF ? row - 1 : row) * nj, *inB = tl + (depB ? row + 1 : row) * nj;
+    volatile float *out = tl + row * nj;
+    const float dF = active ? durF[row] : 0.f, dB = active ? durB[row] : 0.f;
+    const float latF = depF ? lat : 0.f, latB = depB ? lat : 0.f;
+    int nF = 0, nB = 0, rounds = 0;
     bool moved = false;
     float clock = 0.f;
     for (;;) {
 #pragma unroll
-        for (int rep = 0; rep < 4; rep++)
-        if (done < total_ops) {
-            const bool isb = !(nF < warm || (nF < nj && nF - warm == nB));
-            const int j = isb ? nB : nF;
-            const bool dep = isb ? depB : depF;
-            const float e = (isb ? inB : inF)[j];
-            if (!dep || (isb ? e < 0.f : e > 0.f)) {
-                clock = fmaxf(clock, dep ? fabsf(e) + lat : 0.f) + (isb ? dB : dF);
-                out[j] = isb ? -clock : clock;
-                nF += isb ? 0 : 1;
-                nB += isb ? 1 : 0;
-                done++;
-                moved = true;
+        for (int rep = 0; rep < 2; rep++) {
+            {   // forward step
+                const bool want = active && nF < nj && nF - nB <= warm;
+                const float e = inF[min(nF, nj - 1)];
+                if (want && (!depF || e > 0.f)) {
+                    clock = fmaxf(clock, depF ? e + latF : 0.f) + dF;
+                    out[nF] = clock;
+                    nF++;
+                    moved = true;
+                }
+            }
+            {   // backward step
+                const bool want = active && nB < nj && (nF - nB > warm || nF == nj);
+                const float e = inB[min(nB, nj - 1)];
+                if (want && (!depB || e < 0.f)) {
+                    clock = fmaxf(clock, depB ? latB - e : 0.f) + dB;
+                    out[nB] = -clock;
+                    nB++;
+                    moved = true;
+                }
             }
         }
-        PF_SIM_ROUND_END()
+        PF_SIM_ITER_END()
     }
     clock_out = clock;
-    done_out = done;
+    done_out = nF + nB;
 }
 
 // Interleaved: v chunks per rank; unit k of a rank is microbatch (k / (pp v)) pp + k mod pp of chunk
@@ -346,41 +370,56 @@ __device__ __forceinline__ void sim_rounds_interleaved(volatile float *tl, const
                                                        int total_ops, float lat, float &clock_out, int &done_out)
 {
     const int Q = pp * v;
-    int nF = 0, nB = 0, done = 0, rounds = 0;
-    int fw = 0, fc = 0, fg = 0, bw = 0, bc = 0, bg = 0;
+    const bool active = total_ops > 0;
+    const int row = active ? glane : 0;                    // lanes beyond the pipeline depth poll rank 0's rows
+    int nF = 0, nB = 0, rounds = 0;
+    int fw = 0, fc = 0, fg = 0, bw = 0, bc = 0, bg = 0;   // position in the pp-wide window, chunk, window number
     bool moved = false;
     float clock = 0.f;
     for (;;) {
 #pragma unroll
-        for (int rep = 0; rep < 4; rep++)
-        if (done < total_ops) {
-            const bool isb = !(nF < warm || (nF < U && nF - warm == nB));
-            const int cw = isb ? bw : fw, cc = isb ? bc : fc, cg = isb ? bg : fg;
-            const int j = cg * pp + cw;
-            const int q = (isb ? v - 1 - cc : cc) * pp + glane;
-            const bool dep = isb ? (q < Q - 1) : (q > 0);
-            const int nb = dep ? (isb ? q + 1 : q - 1) : q;
-            const float e = tl[nb * nj + j];
-            const float dur = (isb ? durB : durF)[q];
-            if (!dep || (isb ? e < 0.f : e > 0.f)) {
-                clock = fmaxf(clock, dep ? fabsf(e) + lat : 0.f) + dur;
-                tl[q * nj + j] = isb ? -clock : clock;
-                int w_ = cw + 1, c_ = cc, g_ = cg;
-                if (w_ == pp) {
-                    w_ = 0;
-                    if (++c_ == v) c_ = 0, g_++;
+        for (int rep = 0; rep < 2; rep++) {
+            {   // forward step: unit (fg, fc, fw) = microbatch fg pp + fw of chunk fc
+                const bool want = active && nF < U && nF - nB <= warm;
+                const int j = min(fg * pp + fw, nj - 1);
+                const int q = fc * pp + row;
+                const bool dep = q > 0;
+                const float e = tl[(dep ? q - 1 : q) * nj + j];
+                if (want && (!dep || e > 0.f)) {
+                    clock = fmaxf(clock, dep ? e + lat : 0.f) + durF[q];
+                    tl[q * nj + j] = clock;
+                    if (++fw == pp) {
+                        fw = 0;
+                        if (++fc == v) fc = 0, fg++;
+                    }
+                    nF++;
+                    moved = true;
                 }
-                if (isb) bw = w_, bc = c_, bg = g_, nB++;
-                else fw = w_, fc = c_, fg = g_, nF++;
-                done++;
-                moved = true;
+            }
+            {   // backward step: chunks walk downward
+                const bool want = active && nB < U && (nF - nB > warm || nF == U);
+                const int j = min(bg * pp + bw, nj - 1);
+                const int q = (v - 1 - bc) * pp + row;
+                const bool dep = q < Q - 1;
+                const float e = tl[(dep ? q + 1 : q) * nj + j];
+                if (want && (!dep || e < 0.f)) {
+                    clock = fmaxf(clock, dep ? lat - e : 0.f) + durB[q];
+                    tl[q * nj + j] = -clock;
+                    if (++bw == pp) {
+                        bw = 0;
+                        if (++bc == v) bc = 0, bg++;
+                    }
+                    nB++;
+                    moved = true;
+                }
             }
         }
-        PF_SIM_ROUND_END()
+        PF_SIM_ITER_END()
     }
     clock_out = clock;
-    done_out = done;
+    done_out = nF + nB;
 }
+#undef PF_SIM_ITER_END
 
 // DualPipe-style: two directions; the per-rank order comes from the host-built table
 __device__ __forceinline__ void sim_rounds_dual(volatile float *tl, const float *durF, const float *durB, int glane,
