@@ -257,10 +257,11 @@ __global__ void __launch_bounds__(kThreads, 4) score_kernel(const __grid_constan
     uint32_t tkt_next = 0, tkt_after = 0, word_next = 0;  // thread 0: tickets and order word in flight
     unsigned long long gthr_next = 0ull;                   // thread 0: the grid-wide threshold, in flight
     if (tid == 0) {
-        const uint32_t t0 = atomicAdd(A.slab_counter, 1u);
+        // the first gridDim.x tickets are handed out by block number, the counter serves the ones after them
+        const uint32_t t0 = blockIdx.x;
         s_gthr = 0ull;
+        tkt_next = gridDim.x + atomicAdd(A.slab_counter, 1u);
         resolve(t0, (order && t0 < A.n_slabs) ? __ldcg(order + t0) : 0u, s_slabs[0]);
-        tkt_next = atomicAdd(A.slab_counter, 1u);
     }
     __syncthreads();
 
@@ -269,7 +270,7 @@ __global__ void __launch_bounds__(kThreads, 4) score_kernel(const __grid_constan
         if (s_slab.slab == 0xFFFFFFFFu) break;
         if (tid == 0) {
             word_next = (order && tkt_next < A.n_slabs) ? __ldcg(order + tkt_next) : 0u;
-            tkt_after = atomicAdd(A.slab_counter, 1u);
+            tkt_after = gridDim.x + atomicAdd(A.slab_counter, 1u);
             // the grid-wide threshold only matters to evaluated slabs: refresh it on those
             if (want_topk && s_slab.pre_reason == 0) gthr_next = *reinterpret_cast<volatile unsigned long long *>(A.g_thr);
         }
