@@ -313,8 +313,8 @@ __global__ void __launch_bounds__(256) sim_scatter_kernel(const SimArgs A)
 #define PF_SIM_ITER_END()                                                \
     if (!__any_sync(0xFFFFFFFFu, nF + nB < total_ops)) break;            \
     if ((++rounds & 63) == 0) {                                          \
-        if (!__any_sync(0xFFFFFFFFu, moved)) break;                      \
-        moved = false;                                                   \
+        if (!__any_sync(0xFFFFFFFFu, nF + nB != seen)) break;            \
+        seen = nF + nB;                                                  \
     }
 
 // 1F1B: rank = stage = lane
@@ -330,30 +330,29 @@ __device__ __forceinline__ void sim_rounds_1f1b(volatile float *tl, const float 
     volatile float *out = tl + row * nj;
     const float dF = active ? durF[row] : 0.f, dB = active ? durB[row] : 0.f;
     const float latF = depF ? lat : 0.f, latB = depB ? lat : 0.f;
-    int nF = 0, nB = 0, rounds = 0;
-    bool moved = false;
+    const int njl = active ? nj : 0;   // a lane beyond the pipeline depth has nothing to do
+    int nF = 0, nB = 0, rounds = 0, seen = 0;
     float clock = 0.f;
     for (;;) {
 #pragma unroll
         for (int rep = 0; rep < 2; rep++) {
             {   // forward step
-                const bool want = active && nF < nj && nF - nB <= warm;
-                const float e = inF[min(nF, nj - 1)];
+                // (index nF may be nj once all forwards are done: that word lies inside the warp's slice)
+                const bool want = nF < njl && nF - nB <= warm;
+                const float e = inF[nF];
                 if (want && (!depF || e > 0.f)) {
                     clock = fmaxf(clock, depF ? e + latF : 0.f) + dF;
                     out[nF] = clock;
                     nF++;
-                    moved = true;
                 }
             }
             {   // backward step
-                const bool want = active && nB < nj && (nF - nB > warm || nF == nj);
-                const float e = inB[min(nB, nj - 1)];
+                const bool want = nB < njl && (nF - nB > warm || nF == njl);
+                const float e = inB[nB];
                 if (want && (!depB || e < 0.f)) {
                     clock = fmaxf(clock, depB ? latB - e : 0.f) + dB;
                     out[nB] = -clock;
                     nB++;
-                    moved = true;
                 }
             }
         }
@@ -372,16 +371,17 @@ __device__ __forceinline__ void sim_rounds_interleaved(volatile float *tl, const
     const int Q = pp * v;
     const bool active = total_ops > 0;
     const int row = active ? glane : 0;                    // lanes beyond the pipeline depth poll rank 0's rows
-    int nF = 0, nB = 0, rounds = 0;
+    const int Ul = active ? U : 0;                         // a lane beyond the pipeline depth has nothing to do
+    int nF = 0, nB = 0, rounds = 0, seen = 0;
     int fw = 0, fc = 0, fg = 0, bw = 0, bc = 0, bg = 0;   // position in the pp-wide window, chunk, window number
-    bool moved = false;
     float clock = 0.f;
     for (;;) {
 #pragma unroll
         for (int rep = 0; rep < 2; rep++) {
             {   // forward step: unit (fg, fc, fw) = microbatch fg pp + fw of chunk fc
-                const bool want = active && nF < U && nF - nB <= warm;
-                const int j = min(fg * pp + fw, nj - 1);
+                // (j may be nj once all forwards are done: that word lies inside the warp's slice)
+                const bool want = nF < Ul && nF - nB <= warm;
+                const int j = fg * pp + fw;
                 const int q = fc * pp + row;
                 const bool dep = q > 0;
                 const float e = tl[(dep ? q - 1 : q) * nj + j];
@@ -393,12 +393,11 @@ __device__ __forceinline__ void sim_rounds_interleaved(volatile float *tl, const
                         if (++fc == v) fc = 0, fg++;
                     }
                     nF++;
-                    moved = true;
                 }
             }
             {   // backward step: chunks walk downward
-                const bool want = active && nB < U && (nF - nB > warm || nF == U);
-                const int j = min(bg * pp + bw, nj - 1);
+                const bool want = nB < Ul && (nF - nB > warm || nF == Ul);
+                const int j = bg * pp + bw;
                 const int q = (v - 1 - bc) * pp + row;
                 const bool dep = q < Q - 1;
                 const float e = tl[(dep ? q + 1 : q) * nj + j];
@@ -410,7 +409,6 @@ __device__ __forceinline__ void sim_rounds_interleaved(volatile float *tl, const
                         if (++bc == v) bc = 0, bg++;
                     }
                     nB++;
-                    moved = true;
                 }
             }
         }
