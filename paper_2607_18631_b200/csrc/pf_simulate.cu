@@ -319,8 +319,8 @@ __global__ void __launch_bounds__(256) sim_scatter_kernel(const SimArgs A)
 
 // 1F1B: rank = stage = lane
 __device__ __forceinline__ void sim_rounds_1f1b(volatile float *tl, const float *durF, const float *durB, int glane,
-                                                int pp, int nj, int warm, int total_ops, float lat, float &clock_out,
-                                                int &done_out)
+                                                int pp, int nj, int warm, int total_ops, float lat, int fonly,
+                                                float &clock_out, int &done_out)
 {
     // lanes beyond the pipeline depth take no part: they poll row 0 and never act
     const bool active = total_ops > 0;
@@ -333,6 +333,17 @@ __device__ __forceinline__ void sim_rounds_1f1b(volatile float *tl, const float 
     const int njl = active ? nj : 0;   // a lane beyond the pipeline depth has nothing to do
     int nF = 0, nB = 0, rounds = 0, seen = 0;
     float clock = 0.f;
+    // No backward can run before the first microbatch has crossed the shallowest pipeline of the warp: the first
+    // `fonly` steps are forward steps only (the same step as in the loop below).
+    for (int i = 0; i < fonly; i++) {
+        const bool want = nF < njl && nF - nB <= warm;
+        const float e = inF[nF];
+        if (want && (!depF || e > 0.f)) {
+            clock = fmaxf(clock, depF ? e + latF : 0.f) + dF;
+            out[nF] = clock;
+            nF++;
+        }
+    }
     for (;;) {
 #pragma unroll
         for (int rep = 0; rep < 2; rep++) {
@@ -366,7 +377,8 @@ __device__ __forceinline__ void sim_rounds_1f1b(volatile float *tl, const float 
 // (k mod (pp v)) / pp, backward units walk the chunks downward; cursors advance without divisions
 __device__ __forceinline__ void sim_rounds_interleaved(volatile float *tl, const float *durF, const float *durB,
                                                        int glane, int pp, int v, int nj, int U, int warm,
-                                                       int total_ops, float lat, float &clock_out, int &done_out)
+                                                       int total_ops, float lat, int fonly, float &clock_out,
+                                                       int &done_out)
 {
     const int Q = pp * v;
     const bool active = total_ops > 0;
@@ -375,6 +387,23 @@ __device__ __forceinline__ void sim_rounds_interleaved(volatile float *tl, const
     int nF = 0, nB = 0, rounds = 0, seen = 0;
     int fw = 0, fc = 0, fg = 0, bw = 0, bc = 0, bg = 0;   // position in the pp-wide window, chunk, window number
     float clock = 0.f;
+    // forward steps only until the first microbatch can have crossed the shallowest pipeline of the warp
+    for (int i = 0; i < fonly; i++) {
+        const bool want = nF < Ul && nF - nB <= warm;
+        const int j = fg * pp + fw;
+        const int q = fc * pp + row;
+        const bool dep = q > 0;
+        const float e = tl[(dep ? q - 1 : q) * nj + j];
+        if (want && (!dep || e > 0.f)) {
+            clock = fmaxf(clock, dep ? e + lat : 0.f) + durF[q];
+            tl[q * nj + j] = clock;
+            if (++fw == pp) {
+                fw = 0;
+                if (++fc == v) fc = 0, fg++;
+            }
+            nF++;
+        }
+    }
     for (;;) {
 #pragma unroll
         for (int rep = 0; rep < 2; rep++) {
@@ -616,10 +645,15 @@ __global__ void __launch_bounds__(kSimThreads, 4) simulate_kernel(const __grid_c
                 // a batch's candidates share the schedule class of their bin: one specialised loop per class
                 int done = 0;
                 float clock = 0.f;
+                // forward-only steps at the start: one fewer than the stages of the shallowest pipeline in the warp
+                int fonly = (run && !dual) ? Q - 1 : 0x7FFFFFFF;
+                fonly = __reduce_min_sync(0xFFFFFFFFu, fonly);
+                if (fonly == 0x7FFFFFFF) fonly = 0;
                 if (bin_kind == PF_KIND_1F1B)
-                    sim_rounds_1f1b(tl, durF, durB, glane, pp, nj, warm, total_ops, lat, clock, done);
+                    sim_rounds_1f1b(tl, durF, durB, glane, pp, nj, warm, total_ops, lat, fonly, clock, done);
                 else if (bin_kind == PF_KIND_INTERLEAVED)
-                    sim_rounds_interleaved(tl, durF, durB, glane, pp, v, nj, U, warm, total_ops, lat, clock, done);
+                    sim_rounds_interleaved(tl, durF, durB, glane, pp, v, nj, U, warm, total_ops, lat, fonly, clock,
+                                           done);
                 else
                     sim_rounds_dual(tl, durF, durB, glane, pp, nj, dops, total_ops, lat, clock, done);
                 if (done < total_ops) stalled = true;
