@@ -310,8 +310,9 @@ __global__ void __launch_bounds__(256) sim_scatter_kernel(const SimArgs A)
 // step and then a backward step, each straight-line code for its one kind of op; in the steady state a lane does
 // both, so an iteration retires two ops for about the instructions one generic step would take.  A value written
 // in a step is seen by the neighbour's next step of the same kind, one iteration later.
-#define PF_SIM_ITER_END()                                                \
-    if (!__any_sync(0xFFFFFFFFu, nF + nB < total_ops)) break;            \
+// (UL: the lane's unit count; once no lane of the warp has a forward left the loop is left for a backward-only one)
+#define PF_SIM_ITER_END(UL)                                              \
+    if (!__any_sync(0xFFFFFFFFu, nF < (UL))) break;                      \
     if ((++rounds & 63) == 0) {                                          \
         if (!__any_sync(0xFFFFFFFFu, nF + nB != seen)) break;            \
         seen = nF + nB;                                                  \
@@ -367,7 +368,23 @@ __device__ __forceinline__ void sim_rounds_1f1b(volatile float *tl, const float 
                 }
             }
         }
-        PF_SIM_ITER_END()
+        PF_SIM_ITER_END(njl)
+    }
+    // cool-down: every forward of the warp is done, only backward steps are left
+    while (__any_sync(0xFFFFFFFFu, nB < njl)) {
+#pragma unroll
+        for (int rep = 0; rep < 4; rep++) {
+            const float e = inB[nB];
+            if (nB < njl && (!depB || e < 0.f)) {
+                clock = fmaxf(clock, depB ? latB - e : 0.f) + dB;
+                out[nB] = -clock;
+                nB++;
+            }
+        }
+        if ((++rounds & 15) == 0) {
+            if (!__any_sync(0xFFFFFFFFu, nF + nB != seen)) break;
+            seen = nF + nB;
+        }
     }
     clock_out = clock;
     done_out = nF + nB;
@@ -441,7 +458,30 @@ __device__ __forceinline__ void sim_rounds_interleaved(volatile float *tl, const
                 }
             }
         }
-        PF_SIM_ITER_END()
+        PF_SIM_ITER_END(Ul)
+    }
+    // cool-down: every forward of the warp is done, only backward steps are left
+    while (__any_sync(0xFFFFFFFFu, nB < Ul)) {
+#pragma unroll
+        for (int rep = 0; rep < 4; rep++) {
+            const int j = bg * pp + bw;
+            const int q = (v - 1 - bc) * pp + row;
+            const bool dep = q < Q - 1;
+            const float e = tl[(dep ? q + 1 : q) * nj + j];
+            if (nB < Ul && (!dep || e < 0.f)) {
+                clock = fmaxf(clock, dep ? lat - e : 0.f) + durB[q];
+                tl[q * nj + j] = -clock;
+                if (++bw == pp) {
+                    bw = 0;
+                    if (++bc == v) bc = 0, bg++;
+                }
+                nB++;
+            }
+        }
+        if ((++rounds & 15) == 0) {
+            if (!__any_sync(0xFFFFFFFFu, nF + nB != seen)) break;
+            seen = nF + nB;
+        }
     }
     clock_out = clock;
     done_out = nF + nB;
