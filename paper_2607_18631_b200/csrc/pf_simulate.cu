@@ -497,6 +497,8 @@ __device__ __forceinline__ void sim_rounds_dual(volatile float *tl, const float 
     bool moved = false;
     float clock = 0.f;
     for (;;) {
+#pragma unroll
+        for (int rep = 0; rep < 4; rep++)
         if (done < total_ops) {
             const uint32_t op = __ldg(ops + done);
             const bool isb = op & 1;
