@@ -256,16 +256,15 @@ def run_ours(args):
     sim_sc = torch.empty(K_SIM, dtype=torch.float32, device=dev)
     sim_cnt = torch.empty(1, dtype=torch.int32, device=dev)
     ws_score = torch.empty(plan.score_workspace(N, K_TOP), dtype=torch.uint8, device=dev)
-    ws_sel = torch.empty(plan.select_workspace(N, S_MAX), dtype=torch.uint8, device=dev)
-    ws_sim = torch.empty(plan.simulate_workspace(S_MAX, K_SIM), dtype=torch.uint8, device=dev)
+    bufs = dict(reason=reason, tput=tput, mem=mem, topk_idx=tk_idx, topk_score=tk_sc, topk_count=tk_cnt,
+                surv_idx=surv, surv_count=surv_cnt, sim_topk_idx=sim_idx, sim_topk_score=sim_sc,
+                sim_topk_count=sim_cnt,
+                workspace=torch.empty(plan.search_device_workspace(K_TOP, S_MAX, K_SIM), dtype=torch.uint8,
+                                      device=dev))
 
     def step():
-        plan.score(0, N, K_TOP, reason=reason, tput=tput, mem=mem, topk_idx=tk_idx, topk_score=tk_sc,
-                   topk_count=tk_cnt, workspace=ws_score, stream=stream)
-        plan.select_survivors(reason, tput, S_MAX, surv_idx=surv, surv_count=surv_cnt, workspace=ws_sel,
-                              stream=stream)
-        plan.simulate(surv, S_MAX, JITTER_SEED, k=K_SIM, d_n=surv_cnt, topk_idx=sim_idx, topk_score=sim_sc,
-                      topk_count=sim_cnt, workspace=ws_sim, stream=stream, dense=False)
+        # one call: score (dense outputs + top-1024) -> select survivors -> simulate + top-100, all on the device
+        plan.search(K_TOP, S_MAX, K_SIM, JITTER_SEED, bufs=bufs, stream=stream)
 
     sampler = ClockSampler(local)
     for _ in range(max(args.warmup, 3)):

@@ -326,6 +326,20 @@ int pf_aggregate_serving(pf_plan_t *plan, const uint8_t *d_reason, const float *
  * Errors: PF_EINVAL (shape outside the domain, NULL). */
 int pf_dualpipe_order(int pp, int m, uint8_t *out_ops);
 
+/* Whole search on DEVICE buffers in one call: pf_score over the full space (dense outputs + analytic top-k), then,
+ * for training plans with s_max > 0, pf_select_survivors and pf_simulate (top-k_sim of the simulated survivors;
+ * their dense simulator outputs are not kept).  Results are what the three calls give one after the other; inside
+ * one call the scoring kernel also gathers what the selection's first pass would re-read the dense outputs for,
+ * so the selection starts at its second pass.  d_reason, d_tput and the top-k buffers are required, d_mem may be
+ * NULL; the survivor and simulator buffers are required when the simulator tier runs (d_surv_idx: s_max entries).
+ * d_workspace: pf_search_device_workspace() bytes, 256-byte aligned.  Enqueues on `stream`, does not synchronize.
+ * Errors as the calls above. */
+size_t pf_search_device_workspace(const pf_plan_t *plan, uint32_t k, uint64_t s_max, uint32_t k_sim);
+int pf_search(pf_plan_t *plan, uint32_t k, uint64_t s_max, uint32_t k_sim, uint32_t jitter_seed, uint8_t *d_reason,
+              float *d_tput, int64_t *d_mem, uint64_t *d_topk_idx, float *d_topk_score, uint32_t *d_topk_count,
+              uint64_t *d_surv_idx, uint64_t *d_surv_count, uint64_t *d_sim_topk_idx, float *d_sim_topk_score,
+              uint32_t *d_sim_topk_count, void *d_workspace, size_t workspace_bytes, void *stream);
+
 /* Whole search with HOST result buffers (the call a user without device code makes): scores the full
  * space, returns the analytic top-k and -- for training plans with s_max > 0 -- the simulator-refined
  * top-k_sim over the s_max best survivors.  Dense per-candidate outputs are copied back only for the

@@ -24,7 +24,7 @@ EXPORTS = ("pf_version", "pf_strerror", "pf_reason_str", "pf_last_cuda_error", "
            "pf_plan_size", "pf_decode", "pf_score_workspace", "pf_score", "pf_topk_merge", "pf_select_workspace",
            "pf_select_survivors", "pf_simulate_workspace", "pf_simulate", "pf_search_workspace", "pf_search_host",
            "pf_launch_count", "pf_dualpipe_order", "pf_timing_enable", "pf_timing_read", "pf_score_static", "pf_serve_plan_count", "pf_aggregate_workspace", "pf_aggregate_serving",
-           "pf_probe_alu", "pf_probe_write", "pf_report")
+           "pf_probe_alu", "pf_probe_write", "pf_report", "pf_search", "pf_search_device_workspace")
 STATIC_SCRATCH_BYTES = 4 << 20
 T_CLASSES = ("score", "topk", "select", "simulate", "aggregate")
 
@@ -158,6 +158,10 @@ def load_library(path: str | None = None):
     L.pf_timing_read.argtypes = [vp, vp, vp]
     L.pf_dualpipe_order.restype = C.c_int
     L.pf_dualpipe_order.argtypes = [C.c_int, C.c_int, vp]
+    L.pf_search_device_workspace.restype = sz
+    L.pf_search_device_workspace.argtypes = [vp, u32, u64, u32]
+    L.pf_search.restype = C.c_int
+    L.pf_search.argtypes = [vp, u32, u64, u32, u32] + [vp] * 12 + [sz, vp]
     L.pf_report.restype = C.c_int
     L.pf_report.argtypes = [vp, vp, u32, vp, vp, vp]
     L.pf_probe_alu.restype = C.c_int
@@ -408,6 +412,35 @@ class Plan:
                     topk_count=topk_count, workspace=workspace)
 
     # ---- pf_aggregate_serving
+    # ---- pf_search (device buffers)
+    def search_device_workspace(self, k: int, s_max: int, k_sim: int) -> int:
+        return int(self._L.pf_search_device_workspace(self._h, k, s_max, k_sim))
+
+    def search(self, k: int, s_max: int, k_sim: int, jitter_seed: int, bufs: dict | None = None, stream=None,
+               want_mem: bool = True):
+        """Enqueue pf_search: score + select + simulate in one call, everything on the device.  `bufs` (as returned
+        by an earlier call) is reused; missing buffers are allocated here.  Does not synchronize."""
+        torch = _torch()
+        dev, N = self.device, self.size
+        b = dict(bufs) if bufs else {}
+
+        def get(name, n, dtype):
+            if name not in b:
+                b[name] = torch.empty(max(n, 1), dtype=dtype, device=dev)
+            return b[name]
+        reason, tput = get("reason", N, torch.uint8), get("tput", N, torch.float32)
+        mem = get("mem", N, torch.int64) if want_mem else None
+        tk_i, tk_s, tk_c = get("topk_idx", k, torch.int64), get("topk_score", k, torch.float32), get("topk_count", 1, torch.int32)
+        sv, sv_c = get("surv_idx", s_max, torch.int64), get("surv_count", 1, torch.int64)
+        si_i, si_s, si_c = (get("sim_topk_idx", k_sim, torch.int64), get("sim_topk_score", k_sim, torch.float32),
+                            get("sim_topk_count", 1, torch.int32))
+        ws = get("workspace", self.search_device_workspace(k, s_max, k_sim), torch.uint8)
+        _check(self._L.pf_search(self._h, k, s_max, k_sim, jitter_seed, _dptr(reason), _dptr(tput), _dptr(mem),
+                                 _dptr(tk_i), _dptr(tk_s), _dptr(tk_c), _dptr(sv), _dptr(sv_c), _dptr(si_i),
+                                 _dptr(si_s), _dptr(si_c), _dptr(ws), ws.numel(), _stream_ptr(torch, stream)),
+               "pf_search")
+        return b
+
     # ---- pf_report
     def report(self, idx, n: int | None = None, d_n=None, out=None, stream=None):
         """Enqueue pf_report for the plan indices in `idx` (int64/uint64 device tensor).  Returns a uint8 device

@@ -278,6 +278,24 @@ __device__ __forceinline__ void tk_push(unsigned long long *buf, int *count, uns
     }
 }
 
+// What the first pass of the survivor selection would collect, gathered by the scoring kernel instead when the
+// two run inside one search call: the coarse / fine histograms of the eligible candidates' score bits, the
+// eligible count of every selection chunk, the list of chunks with any, and its length.  All zeroed by the caller.
+struct ScoreDigest {
+    unsigned int *hist1, *coarse1, *elig, *list, *n_list;
+    uint32_t chunk;   // candidates per selection chunk
+};
+
+// internal entry points behind pf_score / pf_select_survivors (dg / have_digest: the fused search call)
+int score_run(pf_plan_t *p, uint64_t first, uint64_t count, uint8_t *d_reason, float *d_tput, int64_t *d_mem,
+              uint32_t k, uint64_t *d_topk_idx, float *d_topk_score, uint32_t *d_topk_count, void *d_workspace,
+              size_t workspace_bytes, cudaStream_t st, const ScoreDigest *dg);
+int select_clear(pf_plan_t *p, uint64_t count, void *d_workspace, size_t workspace_bytes, cudaStream_t st,
+                 ScoreDigest *dg_out);
+int select_run(pf_plan_t *p, uint64_t first, uint64_t count, const uint8_t *d_reason, const float *d_tput,
+               uint64_t s_max, uint64_t *d_surv_idx, uint64_t *d_surv_count, void *d_workspace,
+               size_t workspace_bytes, cudaStream_t st, bool have_digest);
+
 // host: workspace layout of one top-k reduction whose producers append at most n_keys_max keys in total.
 // ctrl is 256 bytes: uint32 [0] producer work counter, [1] keys in list A, [2] keys in list B, [3] spare;
 // uint64 at byte 16: the producers' shared admission threshold (largest k-th key any block has reached).

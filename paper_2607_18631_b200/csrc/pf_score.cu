@@ -37,6 +37,7 @@ struct ScoreArgs {
     const uint32_t *order;          // ticket -> (pre_reason << 24) | slab, or NULL: visit by slab_mul, classify here
     const uint32_t *order_hdr;      // the range the order table holds: slab_lo (2 words), n_slabs, tail
     uint32_t order_tail;            // the tail length this call wants
+    ScoreDigest dg;                 // hist1 == NULL: not collected
 };
 
 // Per passing (sched, mb, v) entry of a slab: what its candidates share across kernel variant and recompute mode.
@@ -412,6 +413,15 @@ __global__ void __launch_bounds__(kThreads, 4) score_kernel(const __grid_constan
                         img[i] = (uint8_t)reason;
                         if (A.tput && tput != 0.f) A.tput[o] = tput;
                         if (A.mem) A.mem[o] = M.mem;
+                        // the selection's first pass, done here for the few feasible plans inside the simulator's
+                        // domain: score-bit histograms, the chunk's eligible count, the list of non-empty chunks
+                        if (A.dg.hist1 && tput != 0.f && c.pp <= PF_SIM_MAX_RANKS && D.v_eff <= PF_SIM_MAX_V) {
+                            const uint32_t bits = __float_as_uint(tput);
+                            atomicAdd(A.dg.hist1 + (bits >> 16), 1u);
+                            atomicAdd(A.dg.coarse1 + (bits >> 24), 1u);
+                            const uint32_t chunk = (uint32_t)(o / A.dg.chunk);
+                            if (atomicAdd(A.dg.elig + chunk, 1u) == 0u) A.dg.list[atomicAdd(A.dg.n_list, 1u)] = chunk;
+                        }
                     }
                     offer(active && (reason & 0x7f) == 0, tput, (uint32_t)(rel0 + i));
                 }
@@ -928,6 +938,14 @@ extern "C" int pf_score(pf_plan_t *p, uint64_t first, uint64_t count, uint8_t *d
                         int64_t *d_mem, uint32_t k, uint64_t *d_topk_idx, float *d_topk_score,
                         uint32_t *d_topk_count, void *d_workspace, size_t workspace_bytes, void *stream)
 {
+    return pf::score_run(p, first, count, d_reason, d_tput, d_mem, k, d_topk_idx, d_topk_score, d_topk_count,
+                         d_workspace, workspace_bytes, (cudaStream_t)stream, nullptr);
+}
+
+int pf::score_run(pf_plan_t *p, uint64_t first, uint64_t count, uint8_t *d_reason, float *d_tput, int64_t *d_mem,
+                  uint32_t k, uint64_t *d_topk_idx, float *d_topk_score, uint32_t *d_topk_count, void *d_workspace,
+                  size_t workspace_bytes, cudaStream_t st, const ScoreDigest *dg)
+{
     if (!p) return PF_EINVAL;
     if (k > PF_K_MAX) return PF_EINVAL;
     if (k > 0 && (!d_topk_idx || !d_topk_score || !d_topk_count)) return PF_EINVAL;
@@ -935,7 +953,6 @@ extern "C" int pf_score(pf_plan_t *p, uint64_t first, uint64_t count, uint8_t *d
     if (first >= p->size || count > p->size - first) return PF_ERANGE;
     if (!d_workspace || ((uintptr_t)d_workspace & 255) != 0) return PF_EWORKSPACE;
     if (workspace_bytes < pf_score_workspace(p, count, k)) return PF_EWORKSPACE;
-    cudaStream_t st = (cudaStream_t)stream;
 
     uint64_t slab_lo, n_slabs;
     slab_span(p, first, count, slab_lo, n_slabs);
@@ -960,6 +977,8 @@ extern "C" int pf_score(pf_plan_t *p, uint64_t first, uint64_t count, uint8_t *d
     a.g_thr = (unsigned long long *)(ws + lay.off_ctrl + 16);
     a.vals = p->d_vals; a.scen = p->d_scen;
     a.order = nullptr;
+    a.dg.hist1 = nullptr;
+    if (dg && p->dev.phase == PF_PHASE_TRAIN && d_tput) a.dg = *dg;
     PF_CUDA_TRY(cudaMemsetAsync(a.slab_counter, 0, 256, st), "pf_score: counter reset");
     timing_begin(p, PF_T_SCORE, st);
     int n_score_kernels = 1;

@@ -1,15 +1,37 @@
-// pf_search.cu -- pf_search_host: the whole search for callers that hold only host memory.
-// score (dense + top-k) -> survivor selection -> simulation + re-rank -> copies to the host buffers.
+// pf_search.cu -- the whole search in one call: score (dense + top-k) -> survivor selection -> simulation +
+// re-rank.  pf_search leaves everything on the device; pf_search_host is for callers that hold only host memory
+// and adds the copies.  Inside one call the scoring kernel also collects what the selection's first pass would
+// read the dense outputs for (score-bit histograms and per-chunk counts of the eligible plans), so the selection
+// starts at its second pass.
 #include "pf_internal.cuh"
 
 namespace pf {
 
 struct SearchLayout {
     size_t off_reason, off_tput, off_mem, off_topk_idx, off_topk_score, off_topk_count, off_surv, off_surv_count,
-        off_sim_idx, off_sim_score, off_sim_count, off_ws, ws_bytes, total;
+        off_sim_idx, off_sim_score, off_sim_count, off_ws, ws_bytes, off_ws_sel, ws_sel_bytes, total;
 };
 
 static size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
+
+// scratch of one search: the scoring / simulator part and the selection's part
+struct WorkLayout {
+    size_t ws_bytes, ws_sel_bytes, total;
+};
+static WorkLayout work_layout(const pf_plan_t *p, uint32_t k, uint64_t s_max, uint32_t k_sim)
+{
+    WorkLayout w;
+    size_t a = pf_score_workspace(p, p->size, k);
+    w.ws_sel_bytes = 0;
+    if (s_max > 0 && p->dev.phase == PF_PHASE_TRAIN) {
+        const size_t b = pf_simulate_workspace(p, s_max, k_sim);
+        a = b > a ? b : a;
+        w.ws_sel_bytes = align256(pf_select_workspace(p, p->size, s_max));
+    }
+    w.ws_bytes = align256(a);
+    w.total = w.ws_bytes + w.ws_sel_bytes;
+    return w;
+}
 
 static SearchLayout search_layout(const pf_plan_t *p, uint32_t k, uint64_t s_max, uint32_t k_sim)
 {
@@ -27,16 +49,39 @@ static SearchLayout search_layout(const pf_plan_t *p, uint32_t k, uint64_t s_max
     l.off_sim_idx = o; o += align256((size_t)(k_sim ? k_sim : 1) * 8);
     l.off_sim_score = o; o += align256((size_t)(k_sim ? k_sim : 1) * 4);
     l.off_sim_count = o; o += 256;
-    size_t w = pf_score_workspace(p, p->size, k);
-    if (s_max > 0 && p->dev.phase == PF_PHASE_TRAIN) {
-        size_t a = pf_select_workspace(p, p->size, s_max), b = pf_simulate_workspace(p, s_max, k_sim);
-        w = a > w ? a : w;
-        w = b > w ? b : w;
-    }
+    const WorkLayout w = work_layout(p, k, s_max, k_sim);
     l.off_ws = o;
-    l.ws_bytes = align256(w);
-    l.total = o + l.ws_bytes;
+    l.ws_bytes = w.ws_bytes;
+    l.off_ws_sel = o + w.ws_bytes;
+    l.ws_sel_bytes = w.ws_sel_bytes;
+    l.total = o + w.total;
     return l;
+}
+
+// The stages of one search on device buffers.  ws: scratch of the scoring call, reused by the simulator; ws_sel:
+// the selection's scratch, alive from before the scoring kernel (which fills the first pass's part) to the end
+// of the selection.
+static int search_device(pf_plan_t *p, uint32_t k, uint64_t s_max, uint32_t k_sim, uint32_t jitter_seed,
+                         uint8_t *d_reason, float *d_tput, int64_t *d_mem, uint64_t *d_tk_idx, float *d_tk_sc,
+                         uint32_t *d_tk_cnt, uint64_t *d_surv, uint64_t *d_surv_cnt, uint64_t *d_sim_idx,
+                         float *d_sim_sc, uint32_t *d_sim_cnt, uint8_t *ws, size_t ws_bytes, uint8_t *ws_sel,
+                         size_t ws_sel_bytes, cudaStream_t st)
+{
+    const bool sim = s_max > 0 && p->dev.phase == PF_PHASE_TRAIN;
+    ScoreDigest dg;
+    const ScoreDigest *pdg = nullptr;
+    int rc;
+    if (sim) {
+        rc = select_clear(p, p->size, ws_sel, ws_sel_bytes, st, &dg);
+        if (rc != PF_OK) return rc;
+        pdg = &dg;
+    }
+    rc = score_run(p, 0, p->size, d_reason, d_tput, d_mem, k, d_tk_idx, d_tk_sc, d_tk_cnt, ws, ws_bytes, st, pdg);
+    if (rc != PF_OK || !sim) return rc;
+    rc = select_run(p, 0, p->size, d_reason, d_tput, s_max, d_surv, d_surv_cnt, ws_sel, ws_sel_bytes, st, true);
+    if (rc != PF_OK) return rc;
+    return pf_simulate(p, d_surv, s_max, d_surv_cnt, jitter_seed, nullptr, nullptr, k_sim, d_sim_idx, d_sim_sc,
+                       d_sim_cnt, ws, ws_bytes, (void *)st);
 }
 
 }  // namespace pf
@@ -47,6 +92,33 @@ extern "C" size_t pf_search_workspace(const pf_plan_t *p, uint32_t k, uint64_t s
 {
     if (!p) return 0;
     return search_layout(p, k, s_max, k_sim).total;
+}
+
+extern "C" size_t pf_search_device_workspace(const pf_plan_t *p, uint32_t k, uint64_t s_max, uint32_t k_sim)
+{
+    if (!p) return 0;
+    return work_layout(p, k, s_max, k_sim).total;
+}
+
+extern "C" int pf_search(pf_plan_t *p, uint32_t k, uint64_t s_max, uint32_t k_sim, uint32_t jitter_seed,
+                         uint8_t *d_reason, float *d_tput, int64_t *d_mem, uint64_t *d_topk_idx, float *d_topk_score,
+                         uint32_t *d_topk_count, uint64_t *d_surv_idx, uint64_t *d_surv_count,
+                         uint64_t *d_sim_topk_idx, float *d_sim_topk_score, uint32_t *d_sim_topk_count,
+                         void *d_workspace, size_t workspace_bytes, void *stream)
+{
+    if (!p) return PF_EINVAL;
+    if (k < 1 || k > PF_K_MAX || k_sim > PF_K_MAX) return PF_EINVAL;
+    if (!d_reason || !d_tput || !d_topk_idx || !d_topk_score || !d_topk_count) return PF_EINVAL;
+    if (p->size >= PF_MAX_COUNT) return PF_ERANGE;
+    const bool sim = s_max > 0 && p->dev.phase == PF_PHASE_TRAIN;
+    if (sim && (k_sim < 1 || !d_surv_idx || !d_surv_count || !d_sim_topk_idx || !d_sim_topk_score || !d_sim_topk_count))
+        return PF_EINVAL;
+    const WorkLayout w = work_layout(p, k, s_max, k_sim);
+    if (!d_workspace || ((uintptr_t)d_workspace & 255) != 0 || workspace_bytes < w.total) return PF_EWORKSPACE;
+    uint8_t *ws = (uint8_t *)d_workspace;
+    return search_device(p, k, s_max, k_sim, jitter_seed, d_reason, d_tput, d_mem, d_topk_idx, d_topk_score,
+                         d_topk_count, d_surv_idx, d_surv_count, d_sim_topk_idx, d_sim_topk_score, d_sim_topk_count,
+                         ws, w.ws_bytes, ws + w.ws_bytes, w.ws_sel_bytes, (cudaStream_t)stream);
 }
 
 extern "C" int pf_search_host(pf_plan_t *p, uint32_t k, uint64_t s_max, uint32_t k_sim, uint32_t jitter_seed,
@@ -73,22 +145,15 @@ extern "C" int pf_search_host(pf_plan_t *p, uint32_t k, uint64_t s_max, uint32_t
     uint64_t *d_tk_idx = (uint64_t *)(ws + l.off_topk_idx);
     float *d_tk_sc = (float *)(ws + l.off_topk_score);
     uint32_t *d_tk_cnt = (uint32_t *)(ws + l.off_topk_count);
-    int rc = pf_score(p, 0, p->size, d_reason, d_tput, d_mem, k, d_tk_idx, d_tk_sc, d_tk_cnt, ws + l.off_ws,
-                      l.ws_bytes, stream);
-    if (rc != PF_OK) return rc;
     uint64_t *d_surv = (uint64_t *)(ws + l.off_surv);
     uint64_t *d_surv_cnt = (uint64_t *)(ws + l.off_surv_count);
     uint64_t *d_sim_idx = (uint64_t *)(ws + l.off_sim_idx);
     float *d_sim_sc = (float *)(ws + l.off_sim_score);
     uint32_t *d_sim_cnt = (uint32_t *)(ws + l.off_sim_count);
-    if (sim) {
-        rc = pf_select_survivors(p, 0, p->size, d_reason, d_tput, s_max, d_surv, d_surv_cnt, ws + l.off_ws,
-                                 l.ws_bytes, stream);
-        if (rc != PF_OK) return rc;
-        rc = pf_simulate(p, d_surv, s_max, d_surv_cnt, jitter_seed, nullptr, nullptr, k_sim, d_sim_idx, d_sim_sc,
-                         d_sim_cnt, ws + l.off_ws, l.ws_bytes, stream);
-        if (rc != PF_OK) return rc;
-    }
+    int rc = search_device(p, k, s_max, k_sim, jitter_seed, d_reason, d_tput, d_mem, d_tk_idx, d_tk_sc, d_tk_cnt,
+                           d_surv, d_surv_cnt, d_sim_idx, d_sim_sc, d_sim_cnt, ws + l.off_ws, l.ws_bytes,
+                           ws + l.off_ws_sel, l.ws_sel_bytes, st);
+    if (rc != PF_OK) return rc;
     if (h_reason) PF_CUDA_TRY(cudaMemcpyAsync(h_reason, d_reason, N, cudaMemcpyDeviceToHost, st), "copy reason");
     if (h_tput) PF_CUDA_TRY(cudaMemcpyAsync(h_tput, d_tput, N * 4, cudaMemcpyDeviceToHost, st), "copy tput");
     if (h_mem) PF_CUDA_TRY(cudaMemcpyAsync(h_mem, d_mem, N * 8, cudaMemcpyDeviceToHost, st), "copy mem");

@@ -519,13 +519,41 @@ extern "C" int pf_select_survivors(pf_plan_t *p, uint64_t first, uint64_t count,
                                    const float *d_tput, uint64_t s_max, uint64_t *d_surv_idx, uint64_t *d_surv_count,
                                    void *d_workspace, size_t workspace_bytes, void *stream)
 {
+    return select_run(p, first, count, d_reason, d_tput, s_max, d_surv_idx, d_surv_count, d_workspace,
+                      workspace_bytes, (cudaStream_t)stream, false);
+}
+
+// Zero the selection's control words, histograms and per-chunk counts and say where the scoring kernel may collect
+// the first pass's results (the fused search call: clear -> score with digest -> select_run(have_digest)).
+int pf::select_clear(pf_plan_t *p, uint64_t count, void *d_workspace, size_t workspace_bytes, cudaStream_t st,
+                     ScoreDigest *dg_out)
+{
+    if (!p || count == 0 || count >= PF_MAX_COUNT) return PF_ERANGE;
+    const SelLayout lay = sel_layout(p, count);
+    if (!d_workspace || ((uintptr_t)d_workspace & 255) != 0 || workspace_bytes < lay.total) return PF_EWORKSPACE;
+    uint8_t *ws = (uint8_t *)d_workspace;
+    PF_CUDA_TRY(cudaMemsetAsync(ws, 0, lay.off_list, st), "selection workspace: clear");
+    if (dg_out) {
+        dg_out->hist1 = (unsigned int *)(ws + lay.off_hist1);
+        dg_out->coarse1 = (unsigned int *)(ws + lay.off_coarse);
+        dg_out->elig = (unsigned int *)(ws + lay.off_elig);
+        dg_out->list = (unsigned int *)(ws + lay.off_list);
+        dg_out->n_list = &((SelCtrl *)(ws + lay.off_ctrl))->n_elig;
+        dg_out->chunk = (uint32_t)lay.chunk;
+    }
+    return PF_OK;
+}
+
+int pf::select_run(pf_plan_t *p, uint64_t first, uint64_t count, const uint8_t *d_reason, const float *d_tput,
+                   uint64_t s_max, uint64_t *d_surv_idx, uint64_t *d_surv_count, void *d_workspace,
+                   size_t workspace_bytes, cudaStream_t st, bool have_digest)
+{
     if (!p || !d_reason || !d_tput || !d_surv_idx || !d_surv_count) return PF_EINVAL;
     if (p->dev.phase != PF_PHASE_TRAIN) return PF_EUNSUPPORTED;
     if (count == 0 || count >= PF_MAX_COUNT || s_max == 0) return PF_ERANGE;
     if (first >= p->size || count > p->size - first) return PF_ERANGE;
     const SelLayout lay = sel_layout(p, count);
     if (!d_workspace || ((uintptr_t)d_workspace & 255) != 0 || workspace_bytes < lay.total) return PF_EWORKSPACE;
-    cudaStream_t st = (cudaStream_t)stream;
     uint8_t *ws = (uint8_t *)d_workspace;
     SelArgs a;
     a.first = first; a.count = count; a.s_max = s_max; a.reason = d_reason; a.tput = d_tput;
@@ -540,20 +568,24 @@ extern "C" int pf_select_survivors(pf_plan_t *p, uint64_t first, uint64_t count,
     a.blk_eq = (unsigned long long *)(ws + lay.off_eq);
     a.surv_idx = d_surv_idx; a.surv_count = d_surv_count; a.chunk = lay.chunk;
     // control words, histograms and the per-chunk counts start at zero (chunks that are not on the eligible list
-    // are never written again)
-    PF_CUDA_TRY(cudaMemsetAsync(ws, 0, lay.off_elig, st), "pf_select_survivors: clear");
+    // are never written again); with a digest the scoring kernel has filled the first pass's part already
+    if (!have_digest) PF_CUDA_TRY(cudaMemsetAsync(ws, 0, lay.off_elig, st), "pf_select_survivors: clear");
     // the passes after the first visit the eligible chunks only: a grid that fills the GPU walks the list
     const int list_grid = lay.nblocks < p->sm_count * 8 ? lay.nblocks : p->sm_count * 8;
     timing_begin(p, PF_T_SELECT, st);
-    sel_hist_kernel<<<lay.nblocks, kSelThreads, 0, st>>>(p->dev, a, p->d_vals, 0);
+    int launches = 6;
+    if (!have_digest) {
+        sel_hist_kernel<<<lay.nblocks, kSelThreads, 0, st>>>(p->dev, a, p->d_vals, 0);
+        launches++;
+    }
     sel_scan_kernel<<<1, 256, 0, st>>>(a, 0);
     sel_hist_kernel<<<list_grid, kSelThreads, 0, st>>>(p->dev, a, p->d_vals, 1);
     sel_scan_kernel<<<1, 256, 0, st>>>(a, 1);
     sel_count_kernel<<<list_grid, kSelThreads, 0, st>>>(p->dev, a, p->d_vals);
     sel_blockscan_kernel<<<1, 1024, 0, st>>>(a, lay.nblocks);
     sel_write_kernel<<<list_grid, kSelThreads, 0, st>>>(p->dev, a, p->d_vals);
-    timing_end(p, PF_T_SELECT, 7, st);
-    for (int i = 0; i < 7; i++) count_launch();
+    timing_end(p, PF_T_SELECT, launches, st);
+    for (int i = 0; i < launches; i++) count_launch();
     PF_CUDA_TRY(cudaGetLastError(), "pf_select_survivors launch");
     return PF_OK;
 }

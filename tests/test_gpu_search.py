@@ -1,0 +1,85 @@
+"""The one-call search on device buffers (pf_search): same results as pf_score -> pf_select_survivors -> pf_simulate
+called one after the other, on spaces where the selection keeps everything and where it has to cut."""
+from __future__ import annotations
+
+import numpy as np
+import pytest
+
+from workloads import make_config
+
+from helpers import variant
+
+pytestmark = pytest.mark.gpu
+
+
+def _plan(cfg):
+    from paper_2607_18631_b200 import Plan
+    return Plan(cfg)
+
+
+def _separate(plan, k, s_max, k_sim, seed):
+    import torch
+    out = plan.score(k=k)
+    sel = plan.select_survivors(out["reason"], out["tput"], s_max)
+    sim = plan.simulate(sel["surv_idx"], s_max, seed, k=k_sim, d_n=sel["surv_count"], dense=False)
+    torch.cuda.synchronize()
+    return out, sel, sim
+
+
+def _same(plan, k, s_max, k_sim, seed=4):
+    import torch
+    out, sel, sim = _separate(plan, k, s_max, k_sim, seed)
+    b = plan.search(k, s_max, k_sim, seed)
+    torch.cuda.synchronize()
+    for key in ("reason", "tput", "mem", "topk_idx", "topk_score", "topk_count"):
+        assert torch.equal(out[key], b[key]), key
+    n = int(sel["surv_count"].item())
+    assert int(b["surv_count"].item()) == n
+    assert torch.equal(sel["surv_idx"][:n], b["surv_idx"][:n])
+    assert torch.equal(sim["topk_count"], b["sim_topk_count"])
+    c = int(sim["topk_count"].item())
+    assert torch.equal(sim["topk_idx"][:c], b["sim_topk_idx"][:c])
+    assert torch.equal(sim["topk_score"][:c], b["sim_topk_score"][:c])
+    # a second call on the same buffers gives the same again (the scratch is re-initialised by the call)
+    b2 = plan.search(k, s_max, k_sim, seed, bufs=b)
+    torch.cuda.synchronize()
+    assert int(b2["surv_count"].item()) == n and torch.equal(sel["surv_idx"][:n], b2["surv_idx"][:n])
+    return n
+
+
+@pytest.mark.parametrize("s_max", [10 ** 6, 700, 1])
+def test_search_equals_the_three_calls_mid(s_max):
+    cfg = variant("mid", cluster=dict(budget_bytes=10 ** 15), rules=dict(enforce_realizability=0))
+    plan = _plan(cfg)
+    n = _same(plan, 128, s_max, 100)
+    assert n == min(s_max, n) and n > 0
+    plan.close()
+
+
+def test_search_equals_the_three_calls_large_and_out_of_domain_plans():
+    plan = _plan(make_config("large"))
+    assert _same(plan, 1024, 10 ** 6, 100) == 12_905
+    plan.close()
+    # feasible plans outside the simulator's domain must not reach the digest
+    cfg = variant("large_unconstrained", cluster=dict(budget_bytes=10 ** 15))
+    cfg["model"]["L"] = 128
+    cfg["axes"][4] = ("v", [1, 2, 9])
+    cfg["axes"][5] = ("ep", [8, 64])
+    cfg["axes"][6] = ("pp", [1, 4, 32, 64])
+    cfg["axes"][7] = ("tp", [1, 2])
+    cfg["axes"][8] = ("dp", [8, 16, 64])
+    plan = _plan(cfg)
+    _same(plan, 256, 5000, 64)
+    _same(plan, 256, 10 ** 6, 64)
+    plan.close()
+
+
+def test_search_on_a_serving_space_scores_only():
+    import torch
+    plan = _plan(make_config("serve"))
+    out = plan.score(k=128)
+    b = plan.search(128, 1000, 10, 4)
+    torch.cuda.synchronize()
+    for key in ("reason", "tput", "mem", "topk_idx", "topk_score", "topk_count"):
+        assert torch.equal(out[key], b[key]), key
+    plan.close()
