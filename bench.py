@@ -5,7 +5,8 @@
 
 One step = one pass of the whole path over the large training space (179,908,608 candidates): score every
 candidate (reason byte, tokens/s/GPU, peak bytes, top-1024), select the best feasible survivors (up to 1e6),
-simulate each survivor's pipeline schedule and re-rank the top-100.  Rank 0 prints ONE JSON line.
+simulate each survivor's pipeline schedule and re-rank the top-100 -- one pf_search call.  Rank 0 prints ONE JSON
+line.
 
 N > 1 (launched under torch.distributed.run): every rank scores an independent space of the same shape
 (tables re-drawn from seed = rank); no data-path collective; value = all ranks' candidates / max time.
