@@ -83,3 +83,28 @@ def test_search_on_a_serving_space_scores_only():
     for key in ("reason", "tput", "mem", "topk_idx", "topk_score", "topk_count"):
         assert torch.equal(out[key], b[key]), key
     plan.close()
+
+
+def test_search_replays_from_a_cuda_graph():
+    """The whole search enqueues on one stream without synchronizing or allocating, so it can be captured once and
+    replayed; each replay re-initialises its scratch and gives the same results."""
+    import torch
+    cfg = variant("mid", cluster=dict(budget_bytes=10 ** 15), rules=dict(enforce_realizability=0))
+    plan = _plan(cfg)
+    b = plan.search(128, 2000, 100, 4)                 # allocates the buffers, builds the plan's order table
+    torch.cuda.synchronize()
+    want = {k: v.clone() for k, v in b.items() if k != "workspace"}
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        plan.search(128, 2000, 100, 4, bufs=b)
+    for _ in range(3):
+        for k in ("reason", "surv_idx", "sim_topk_score"):
+            b[k].zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        n = int(b["surv_count"].item())
+        assert n == int(want["surv_count"].item()) == 2000
+        for k in ("reason", "tput", "mem", "topk_idx", "topk_score", "sim_topk_idx", "sim_topk_score"):
+            assert torch.equal(b[k], want[k]), k
+        assert torch.equal(b["surv_idx"][:n], want["surv_idx"][:n])
+    plan.close()
