@@ -102,3 +102,48 @@ def test_random_space_full_pipeline(seed):
         np.testing.assert_array_equal(sim["sim_status"][:n].cpu().numpy(), ref_st)
         np.testing.assert_allclose(sim["tput_sim"][:n].cpu().numpy(), ref, rtol=TPUT_RTOL, atol=0)
     plan.close()
+
+
+def random_serving_space(seed: int) -> dict:
+    rng = np.random.default_rng(seed)
+    cfg = copy.deepcopy(make_config("serve"))
+    pick = lambda pool, lo, hi: sorted(rng.choice(pool, size=int(rng.integers(lo, hi + 1)), replace=False).tolist())
+    m = cfg["model"]
+    m["L"] = int(rng.choice([24, 48, 61]))
+    m["nh"] = int(rng.choice([24, 40, 64]))
+    m["nkv"] = m["nh"]
+    m["E"] = int(rng.choice([48, 128, 160]))
+    m["K"] = int(rng.choice([4, 6, 8]))
+    m["attn_kind"] = int(rng.integers(0, 2))
+    world = int(rng.choice([4, 8, 16]))
+    cfg["workload"]["world"] = world
+    cfg["cluster"]["budget_bytes"] = int(rng.choice([40e9, 72e9, 1e15]))
+    n_scen = int(rng.choice([1, 7, 32]))
+    cfg["workload"]["scen_P"] = [int(x) for x in rng.integers(16, 20000, size=n_scen)]
+    cfg["workload"]["scen_O"] = [int(x) for x in rng.integers(1, 4000, size=n_scen)]
+    cfg["axes"] = [("kv", pick(list(range(6)), 1, 6)), ("chunk", pick([512, 1000, 2048, 4096, 8192], 1, 4)),
+                   ("batch", pick([1, 2, 3, 8, 16, 48, 128, 512], 2, 6)), ("dpa", pick([0, 1], 1, 2)),
+                   ("ep", pick([1, 2, 4, 8, 16], 1, 4)), ("tp", pick([1, 2, 4, 8], 1, 4)), ("scen", list(range(n_scen)))]
+    for k in cfg["kern"]:
+        k["avail_mask"] = int(rng.integers(1, 256))
+    cfg["domain"].update(m_lo=int(rng.choice([1, 64])), m_hi=int(rng.choice([16, 8192])))
+    return cfg
+
+
+@pytest.mark.parametrize("seed", range(10))
+def test_random_serving_space(seed):
+    import torch
+    from paper_2607_18631_b200 import Plan
+    cfg = random_serving_space(2000 + seed)
+    plan, orc = Plan(cfg), Oracle(cfg)
+    reason, tput, mem, _ = orc.score_range(threads=8)
+    res = gpu_score(plan, k=32)
+    compare_dense(res, reason, tput, mem)
+    compare_topk(res, orc, reason, tput, 0, 32)
+    out = plan.score(k=0)
+    agg = plan.aggregate_serving(out["reason"], out["tput"], k=8)
+    torch.cuda.synchronize()
+    pr, pt = orc.aggregate_serving(out["reason"].cpu().numpy(), out["tput"].cpu().numpy().astype(np.float64))
+    np.testing.assert_array_equal(agg["plan_reason"].cpu().numpy(), pr)
+    np.testing.assert_allclose(agg["plan_tput"].cpu().numpy(), pt, rtol=TPUT_RTOL, atol=0)
+    plan.close()
