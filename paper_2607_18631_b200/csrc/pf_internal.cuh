@@ -15,7 +15,7 @@ constexpr uint32_t kSlabMax = 16384; // upper bound on candidates per slab (inne
 constexpr int kInnerVals = 1024;     // inner-axis values the scoring kernel keeps in shared memory
 constexpr int kOrderMaxSlabs = 1 << 20;  // calls with more slabs visit them by a permutation instead of an order table
 constexpr int kTailFillsPerBlock = 4;    // constant-fill slabs per block kept, at least, for the end of the visiting order
-constexpr int kFillsPerEvaluated = 2;    // fills interleaved per evaluated slab at the start of the visiting order
+constexpr int kFillsPerEvaluated = 3;    // fills interleaved per evaluated slab at the start of the visiting order (measured: 1: 0.392 ms, 2: 0.384, 3: 0.380, 4: 0.379, 6: 0.382, 8: 0.385, 12: 0.396)
 constexpr int kQueueCap = 4096;   // cost-model queue of the scoring kernel (entries), drained when it may fill up
 
 struct DevSched {

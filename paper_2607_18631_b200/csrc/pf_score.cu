@@ -106,8 +106,8 @@ __global__ void __launch_bounds__(256) slab_class_kernel(const __grid_constant__
 
 // Step 2, one block: ranks within each class by a block-wide scan over per-thread chunks, then every slab's
 // ticket in closed form.  With H evaluated and F filled slabs, Fs = min(kFillsPerEvaluated * H, F - tail) fills
-// are interleaved with the evaluated slabs (measured best: about two thirds of the blocks evaluate while the
-// rest keep the store stream going) and the other fills follow: evaluated slab i sits after floor(i * Fs / H)
+// are interleaved with the evaluated slabs (measured best: three or four fills per evaluated slab, i.e. about
+// half of the blocks evaluating while the rest keep the store stream going) and the other fills follow: evaluated slab i sits after floor(i * Fs / H)
 // fills, fill j < Fs after min(H, ceil((j + 1) * H / Fs)) evaluated slabs.
 __global__ void __launch_bounds__(1024) slab_order_kernel(const uint8_t *cls, uint64_t slab_lo, uint32_t n_slabs,
                                                           uint32_t tail, uint32_t *order, uint32_t *hdr)
