@@ -423,6 +423,14 @@ extern "C" int pf_plan_create(const pf_model_t *model, const pf_cluster_t *clust
         return PF_ECUDA;
     }
     if (phase == PF_PHASE_TRAIN) {
+        e = cudaStreamCreateWithFlags(&p->side_stream, cudaStreamNonBlocking);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->ev_fork, cudaEventDisableTiming);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->ev_join, cudaEventDisableTiming);
+        if (e != cudaSuccess) {
+            pf::set_cuda_error(e, "pf_plan_create: side stream");
+            pf_plan_destroy(p);
+            return PF_ECUDA;
+        }
         int rc = pf::build_sim_tables(p);
         if (rc != PF_OK) {
             pf_plan_destroy(p);
@@ -476,6 +484,9 @@ extern "C" void pf_plan_destroy(pf_plan_t *p)
     if (p->d_vals) cudaFree(p->d_vals);
     if (p->d_scen) cudaFree(p->d_scen);
     if (p->d_order) cudaFree(p->d_order);
+    if (p->ev_fork) cudaEventDestroy(p->ev_fork);
+    if (p->ev_join) cudaEventDestroy(p->ev_join);
+    if (p->side_stream) cudaStreamDestroy(p->side_stream);
     free(p->h_vals);
     delete p;
 }

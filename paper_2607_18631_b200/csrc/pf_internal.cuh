@@ -98,6 +98,10 @@ struct pf_plan {
     uint32_t order_cap;
     uint64_t order_slab_lo;
     uint32_t order_n_slabs, order_tail;
+    // pf_search runs the scoring call's top-k reduction beside the survivor selection: a second stream and the
+    // two events of the fork and the join (training plans; created with the plan)
+    cudaStream_t side_stream;
+    cudaEvent_t ev_fork, ev_join;
     // simulator order tables (built at create for training plans)
     void *sim_tables;
     // optional per-kernel-class event timing (pf_timing_enable)
@@ -289,7 +293,7 @@ struct ScoreDigest {
 // internal entry points behind pf_score / pf_select_survivors (dg / have_digest: the fused search call)
 int score_run(pf_plan_t *p, uint64_t first, uint64_t count, uint8_t *d_reason, float *d_tput, int64_t *d_mem,
               uint32_t k, uint64_t *d_topk_idx, float *d_topk_score, uint32_t *d_topk_count, void *d_workspace,
-              size_t workspace_bytes, cudaStream_t st, const ScoreDigest *dg);
+              size_t workspace_bytes, cudaStream_t st, const ScoreDigest *dg, bool topk_on_side_stream);
 int select_clear(pf_plan_t *p, uint64_t count, void *d_workspace, size_t workspace_bytes, cudaStream_t st,
                  ScoreDigest *dg_out);
 int select_run(pf_plan_t *p, uint64_t first, uint64_t count, const uint8_t *d_reason, const float *d_tput,

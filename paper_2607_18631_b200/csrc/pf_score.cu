@@ -939,12 +939,12 @@ extern "C" int pf_score(pf_plan_t *p, uint64_t first, uint64_t count, uint8_t *d
                         uint32_t *d_topk_count, void *d_workspace, size_t workspace_bytes, void *stream)
 {
     return pf::score_run(p, first, count, d_reason, d_tput, d_mem, k, d_topk_idx, d_topk_score, d_topk_count,
-                         d_workspace, workspace_bytes, (cudaStream_t)stream, nullptr);
+                         d_workspace, workspace_bytes, (cudaStream_t)stream, nullptr, false);
 }
 
 int pf::score_run(pf_plan_t *p, uint64_t first, uint64_t count, uint8_t *d_reason, float *d_tput, int64_t *d_mem,
                   uint32_t k, uint64_t *d_topk_idx, float *d_topk_score, uint32_t *d_topk_count, void *d_workspace,
-                  size_t workspace_bytes, cudaStream_t st, const ScoreDigest *dg)
+                  size_t workspace_bytes, cudaStream_t st, const ScoreDigest *dg, bool topk_on_side_stream)
 {
     if (!p) return PF_EINVAL;
     if (k > PF_K_MAX) return PF_EINVAL;
@@ -1026,11 +1026,21 @@ int pf::score_run(pf_plan_t *p, uint64_t first, uint64_t count, uint8_t *d_reaso
     timing_end(p, PF_T_SCORE, n_score_kernels, st);
     PF_CUDA_TRY(cudaGetLastError(), "score_kernel launch");
     if (k > 0) {
-        timing_begin(p, PF_T_TOPK, st);
+        // The reduction of the key list depends on the scoring kernel only.  Inside a search call it runs on the
+        // plan's second stream, beside the survivor selection; the caller joins (ev_join) before it reuses the
+        // workspace.
+        cudaStream_t rs = st;
+        if (topk_on_side_stream && p->side_stream) {
+            rs = p->side_stream;
+            PF_CUDA_TRY(cudaEventRecord(p->ev_fork, st), "top-k fork");
+            PF_CUDA_TRY(cudaStreamWaitEvent(rs, p->ev_fork, 0), "top-k fork");
+        }
+        timing_begin(p, PF_T_TOPK, rs);
         int nk = 0;
         int rc = launch_topk_reduce(ws, lay, (uint64_t)grid * k, k, first, nullptr, d_topk_idx, d_topk_score,
-                                    d_topk_count, st, &nk);
-        timing_end(p, PF_T_TOPK, nk, st);
+                                    d_topk_count, rs, &nk);
+        timing_end(p, PF_T_TOPK, nk, rs);
+        if (rs != st) PF_CUDA_TRY(cudaEventRecord(p->ev_join, rs), "top-k join");
         return rc;
     }
     return PF_OK;

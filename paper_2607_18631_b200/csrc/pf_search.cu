@@ -76,9 +76,14 @@ static int search_device(pf_plan_t *p, uint32_t k, uint64_t s_max, uint32_t k_si
         if (rc != PF_OK) return rc;
         pdg = &dg;
     }
-    rc = score_run(p, 0, p->size, d_reason, d_tput, d_mem, k, d_tk_idx, d_tk_sc, d_tk_cnt, ws, ws_bytes, st, pdg);
+    // with a simulator tier to follow, the analytic top-k is reduced on the plan's second stream while this one
+    // goes on with the selection; the simulator reuses the scoring scratch, so the two join before it
+    const bool side = sim && p->side_stream != nullptr;
+    rc = score_run(p, 0, p->size, d_reason, d_tput, d_mem, k, d_tk_idx, d_tk_sc, d_tk_cnt, ws, ws_bytes, st, pdg,
+                   side);
     if (rc != PF_OK || !sim) return rc;
     rc = select_run(p, 0, p->size, d_reason, d_tput, s_max, d_surv, d_surv_cnt, ws_sel, ws_sel_bytes, st, true);
+    if (side) PF_CUDA_TRY(cudaStreamWaitEvent(st, p->ev_join, 0), "top-k join");
     if (rc != PF_OK) return rc;
     return pf_simulate(p, d_surv, s_max, d_surv_cnt, jitter_seed, nullptr, nullptr, k_sim, d_sim_idx, d_sim_sc,
                        d_sim_cnt, ws, ws_bytes, (void *)st);
