@@ -333,6 +333,8 @@ int pf_dualpipe_order(int pp, int m, uint8_t *out_ops);
  * so the selection starts at its second pass.  d_reason, d_tput and the top-k buffers are required, d_mem may be
  * NULL; the survivor and simulator buffers are required when the simulator tier runs (d_surv_idx: s_max entries).
  * d_workspace: pf_search_device_workspace() bytes, 256-byte aligned.  Enqueues on `stream`, does not synchronize.
+ * (With a simulator tier, the reduction of the analytic top-k runs on a second stream that belongs to the plan,
+ * forked from and joined back into `stream` by events inside the call; the call can be captured into a graph.)
  * Errors as the calls above. */
 size_t pf_search_device_workspace(const pf_plan_t *plan, uint32_t k, uint64_t s_max, uint32_t k_sim);
 int pf_search(pf_plan_t *plan, uint32_t k, uint64_t s_max, uint32_t k_sim, uint32_t jitter_seed, uint8_t *d_reason,
