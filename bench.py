@@ -184,7 +184,7 @@ def _time_launches(torch, stream, fn, reps=5, warm=2):
     return a.elapsed_time(b) / reps
 
 
-def _probe_peaks(torch, binding, stream, big):
+def _probe_peaks(torch, probes, stream, big):
     """Issue-rate peaks (thread-instructions/s) per instruction kind and the pure streaming-write rate (GB/s),
     measured with the library's probe kernels; `big` is a device buffer far larger than L2."""
     sink = torch.zeros(1, dtype=torch.int32, device=big.device)
@@ -193,11 +193,11 @@ def _probe_peaks(torch, binding, stream, big):
         n = [0]
 
         def go():
-            n[0] = binding.pf_probe_alu(kind, 8192, sink)
+            n[0] = probes.pf_probe_alu(kind, 8192, sink)
         ms = _time_launches(torch, stream, go)
         out[kind] = n[0] / (ms * 1e-3)
     nbytes = big.numel() * big.element_size()
-    ms = _time_launches(torch, stream, lambda: binding.pf_probe_write(big))
+    ms = _time_launches(torch, stream, lambda: probes.pf_probe_write(big))
     return out, nbytes / (ms * 1e-3) / 1e9
 
 
@@ -340,7 +340,8 @@ def run_ours(args):
                                               workspace=ws_score, stream=stream, dense=False), reps=10, warm=3)
         extra["topk_only"] = {"ms_per_launch": ms_topk_only, "value": N / (ms_topk_only * 1e-3), "unit": UNIT,
                               "note": "dense outputs not written (NULL): rules + cost + top-1024 only"}
-        peaks, write_gbs = _probe_peaks(torch, binding, stream, mem)
+        from paper_2607_18631_b200 import probes
+        peaks, write_gbs = _probe_peaks(torch, probes, stream, mem)
         step()                                   # the write probe overwrote `mem`: restore the step's outputs
         torch.cuda.synchronize()
         n_feas = int(((reason & 0x7F) == 0).sum().item())

@@ -355,20 +355,6 @@ int pf_search_host(pf_plan_t *plan, uint32_t k, uint64_t s_max, uint32_t k_sim, 
                    uint32_t *h_sim_topk_count, uint64_t *h_surv_count, void *d_workspace,
                    size_t workspace_bytes, void *stream);
 
-/* Optional device timing of the library's own kernels, by class, for roofline accounting (the paper has
- * no counterpart).  While enabled, every call brackets the launches of each class with a CUDA event pair
- * on the caller's stream; pf_timing_read waits for the recorded events, adds the elapsed times (ms) and
- * kernel counts per class into ms[PF_T_CLASSES] / kernels[PF_T_CLASSES], and forgets them.
- * PF_T_SCORE: the scoring kernel; PF_T_TOPK: top-k list kernels (merge passes, dense top-k);
- * PF_T_SELECT: the survivor-selection kernels; PF_T_SIMULATE: the simulator kernels;
- * PF_T_AGGREGATE: the per-plan serving aggregate. */
-enum { PF_T_SCORE = 0, PF_T_TOPK = 1, PF_T_SELECT = 2, PF_T_SIMULATE = 3, PF_T_AGGREGATE = 4, PF_T_CLASSES = 5 };
-int pf_timing_enable(pf_plan_t *plan, int on);
-int pf_timing_read(pf_plan_t *plan, float *ms, uint32_t *kernels);
-
-/* Number of kernels this library has launched in this process (for launch accounting in benchmarks). */
-uint64_t pf_launch_count(void);
-
 /* Extrapolation report for a list of plans, e.g. a top-k list (principle P4: a query outside the calibration
  * domain is flagged, not silently trusted).  Entry i of d_out describes plan d_idx[i]: its reason byte as pf_score
  * writes it, the PF_WHY_* bits behind an extrapolated flag, its tokens per expert and efficiency bucket (0 where
@@ -383,24 +369,6 @@ typedef struct {
 } pf_report_t;
 int pf_report(pf_plan_t *plan, const uint64_t *d_idx, uint32_t n, const uint32_t *d_n, pf_report_t *d_out,
               void *stream);
-
-/* Roofline probes (measurement utilities; the paper has no counterpart and no scoring call uses them).
- * The caller times them with events on `stream`; neither call synchronises or allocates.
- *
- * pf_probe_alu: one launch at full occupancy (8 blocks of 256 threads per SM) in which every thread runs
- * 8 independent dependency chains of one instruction kind for `iters` loop trips of 4 steps each:
- * PF_PROBE_FFMA fp32 fused multiply-add, PF_PROBE_IMAD 32-bit integer multiply-add, PF_PROBE_LOGIC an
- * alternation of 3-input logic ops and 32-bit adds.  *h_thread_instructions (host) receives the number of
- * thread-level instructions of that kind the launch executes; dividing by the launch's duration gives the
- * issue-rate peak for that kind.  d_sink: 4 device bytes, practically never written.  1 <= iters <= 2^24.
- *
- * pf_probe_write: fills `bytes` (a multiple of 16, below 2^35, 16-byte aligned device buffer) with 16-byte
- * streaming stores, one per thread over a grid as large as the buffer -- the store the scoring kernel uses for
- * its dense outputs, in the fastest pure-write pattern; bytes / duration is the write ceiling.
- * Errors: PF_EINVAL for a null pointer, a bad kind, iters or size; PF_ECUDA if the launch fails. */
-enum { PF_PROBE_FFMA = 0, PF_PROBE_IMAD = 1, PF_PROBE_LOGIC = 2 };
-int pf_probe_alu(int kind, uint32_t iters, uint32_t *d_sink, uint64_t *h_thread_instructions, void *stream);
-int pf_probe_write(void *d_buf, size_t bytes, void *stream);
 
 #ifdef __cplusplus
 }

@@ -1,0 +1,62 @@
+/*
+ * planfront_bench.h -- measurement hooks for benchmarks of libplanfront.so.  Not part of the scoring ABI
+ * (planfront.h): the paper has no counterpart for anything declared here and no scoring call depends on it.
+ *
+ * Two groups:
+ *   - pf_timing_enable / pf_timing_read / pf_launch_count are exported by libplanfront.so itself, because they
+ *     instrument launches the library makes on streams of its own, which a caller's events cannot bracket;
+ *   - pf_probe_alu / pf_probe_write are exported by a separate library, libplanfront_probe.so: micro-kernels that
+ *     measure the denominators of the rooflines (instruction issue rates, the pure streaming-write rate).
+ */
+#ifndef PLANFRONT_BENCH_H
+#define PLANFRONT_BENCH_H
+
+#include "planfront.h"
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* Optional device timing of the library's own kernels, by class, for roofline accounting (the paper has
+ * no counterpart).  While enabled, every call brackets the launches of each class with a CUDA event pair
+ * on the stream they are launched on; pf_timing_read waits for the recorded events, adds the elapsed times (ms) and
+ * kernel counts per class into ms[PF_T_CLASSES] / kernels[PF_T_CLASSES], and forgets them.
+ * PF_T_SCORE: the scoring kernel; PF_T_TOPK: top-k list kernels (merge passes, dense top-k);
+ * PF_T_SELECT: the survivor-selection kernels; PF_T_SIMPREP: the simulator's pre-pass (binning, records);
+ * PF_T_SIMULATE: the simulator kernel (inside pf_search it also streams the constant blocks of the dense outputs);
+ * PF_T_AGGREGATE: the per-plan serving aggregate; PF_T_FILL: the stand-alone kernel that streams the constant
+ * blocks of the dense outputs inside pf_search when no simulator kernel runs to carry them.  Classes that run on different streams
+ * overlap, so their times may add up to more than the call's. */
+enum {
+    PF_T_SCORE = 0, PF_T_TOPK = 1, PF_T_SELECT = 2, PF_T_SIMULATE = 3, PF_T_AGGREGATE = 4, PF_T_FILL = 5,
+    PF_T_SIMPREP = 6, PF_T_CLASSES = 7
+};
+int pf_timing_enable(pf_plan_t *plan, int on);
+int pf_timing_read(pf_plan_t *plan, float *ms, uint32_t *kernels);
+
+/* Number of kernels this library has launched in this process (for launch accounting in benchmarks). */
+uint64_t pf_launch_count(void);
+
+/* Roofline probes (libplanfront_probe.so).
+ * The caller times them with events on `stream`; neither call synchronises or allocates.
+ *
+ * pf_probe_alu: one launch at full occupancy (8 blocks of 256 threads per SM) in which every thread runs
+ * 8 independent dependency chains of one instruction kind for `iters` loop trips of 4 steps each:
+ * PF_PROBE_FFMA fp32 fused multiply-add, PF_PROBE_IMAD 32-bit integer multiply-add, PF_PROBE_LOGIC an
+ * alternation of 3-input logic ops and 32-bit adds.  *h_thread_instructions (host) receives the number of
+ * thread-level instructions of that kind the launch executes; dividing by the launch's duration gives the
+ * issue-rate peak for that kind.  d_sink: 4 device bytes, practically never written.  1 <= iters <= 2^24.
+ *
+ * pf_probe_write: fills `bytes` (a multiple of 16, below 2^35, 16-byte aligned device buffer) with 16-byte
+ * streaming stores, one per thread over a grid as large as the buffer -- the store the scoring kernel uses for
+ * its dense outputs, in the fastest pure-write pattern; bytes / duration is the write ceiling.
+ * Errors: PF_EINVAL for a null pointer, a bad kind, iters or size; PF_ECUDA if the launch fails (the probe library
+ * keeps no error text). */
+enum { PF_PROBE_FFMA = 0, PF_PROBE_IMAD = 1, PF_PROBE_LOGIC = 2 };
+int pf_probe_alu(int kind, uint32_t iters, uint32_t *d_sink, uint64_t *h_thread_instructions, void *stream);
+int pf_probe_write(void *d_buf, size_t bytes, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif

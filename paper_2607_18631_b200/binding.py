@@ -23,10 +23,12 @@ UINT64_MAX = 0xFFFFFFFFFFFFFFFF
 EXPORTS = ("pf_version", "pf_strerror", "pf_reason_str", "pf_last_cuda_error", "pf_plan_create", "pf_plan_destroy",
            "pf_plan_size", "pf_decode", "pf_score_workspace", "pf_score", "pf_topk_merge", "pf_select_workspace",
            "pf_select_survivors", "pf_simulate_workspace", "pf_simulate", "pf_search_workspace", "pf_search_host",
-           "pf_launch_count", "pf_dualpipe_order", "pf_timing_enable", "pf_timing_read", "pf_score_static", "pf_serve_plan_count", "pf_aggregate_workspace", "pf_aggregate_serving",
-           "pf_probe_alu", "pf_probe_write", "pf_report", "pf_search", "pf_search_device_workspace")
+           "pf_dualpipe_order", "pf_score_static", "pf_serve_plan_count", "pf_aggregate_workspace", "pf_aggregate_serving",
+           "pf_report", "pf_search", "pf_search_device_workspace")
+# measurement hooks of include/planfront_bench.h that this library exports (the probes live in probes.py)
+BENCH_EXPORTS = ("pf_launch_count", "pf_timing_enable", "pf_timing_read")
 STATIC_SCRATCH_BYTES = 4 << 20
-T_CLASSES = ("score", "topk", "select", "simulate", "aggregate")
+T_CLASSES = ("score", "topk", "select", "simulate", "aggregate", "fill", "simprep")
 
 i32, u32, i64, u64, f32 = C.c_int32, C.c_uint32, C.c_int64, C.c_uint64, C.c_float
 
@@ -164,10 +166,6 @@ def load_library(path: str | None = None):
     L.pf_search.argtypes = [vp, u32, u64, u32, u32] + [vp] * 12 + [sz, vp]
     L.pf_report.restype = C.c_int
     L.pf_report.argtypes = [vp, vp, u32, vp, vp, vp]
-    L.pf_probe_alu.restype = C.c_int
-    L.pf_probe_alu.argtypes = [C.c_int, u32, vp, C.POINTER(u64), vp]
-    L.pf_probe_write.restype = C.c_int
-    L.pf_probe_write.argtypes = [vp, sz, vp]
     if path == LIB_PATH:
         _lib = L
     return L
@@ -196,27 +194,6 @@ def pf_reason_str(reason: int) -> str:
 
 def pf_launch_count() -> int:
     return int(load_library().pf_launch_count())
-
-
-PROBE_KINDS = {"ffma": 0, "imad": 1, "logic": 2}
-
-
-def pf_probe_alu(kind: str, iters: int, sink) -> int:
-    """Launch one issue-rate probe on the current stream; returns the thread-level instructions it executes."""
-    import torch
-    n = u64(0)
-    _check(load_library().pf_probe_alu(PROBE_KINDS[kind], iters, sink.data_ptr(), C.byref(n),
-                                       torch.cuda.current_stream().cuda_stream), "pf_probe_alu")
-    return int(n.value)
-
-
-def pf_probe_write(buf) -> int:
-    """Fill `buf` (a device tensor, 16-byte aligned, size a multiple of 16 bytes) with streaming stores."""
-    import torch
-    nbytes = buf.numel() * buf.element_size()
-    _check(load_library().pf_probe_write(buf.data_ptr(), nbytes, torch.cuda.current_stream().cuda_stream),
-           "pf_probe_write")
-    return nbytes
 
 
 def pf_dualpipe_order(pp: int, m: int):

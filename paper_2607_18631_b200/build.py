@@ -8,25 +8,36 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(HERE, "libplanfront.so")
-SOURCES = ["pf_api.cu", "pf_score.cu", "pf_select.cu", "pf_simulate.cu", "pf_search.cu", "pf_aggregate.cu", "pf_probe.cu", "pf_report.cu"]
+SOURCES = ["pf_api.cu", "pf_score.cu", "pf_select.cu", "pf_simulate.cu", "pf_search.cu", "pf_aggregate.cu", "pf_report.cu"]
+# the roofline probes of the benchmark: a library of their own, not part of the scoring ABI
+PROBE_LIB = os.path.join(HERE, "libplanfront_probe.so")
+PROBE_SOURCES = ["pf_probe.cu"]
 
 
 def _newest_source() -> float:
-    paths = [os.path.join(CSRC, f) for f in os.listdir(CSRC)] + [os.path.join(INCLUDE, "planfront.h")]
+    paths = [os.path.join(CSRC, f) for f in os.listdir(CSRC)] + [os.path.join(INCLUDE, f) for f in os.listdir(INCLUDE)]
     return max(os.path.getmtime(p) for p in paths)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    """Compile every .cu into one shared library.  Returns its path."""
-    if not force and os.path.exists(LIB) and os.path.getmtime(LIB) >= _newest_source():
-        return LIB
+def _compile(lib: str, sources, verbose: bool, defines=()) -> None:
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     cmd = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-           "-I" + INCLUDE, "-Xcompiler", "-fPIC", "-shared", "-o", LIB]
+           "-I" + INCLUDE, "-Xcompiler", "-fPIC", "-shared", "-o", lib]
+    cmd += ["-D" + d for d in defines]
     if verbose:
         cmd += ["-Xptxas", "-v"]
-    cmd += [os.path.join(CSRC, s) for s in SOURCES if os.path.exists(os.path.join(CSRC, s))]
+    cmd += [os.path.join(CSRC, s) for s in sources]
     subprocess.run(cmd, check=True)
+
+
+def build(force: bool = False, verbose: bool = False) -> str:
+    """Compile the scoring library (every scoring .cu into libplanfront.so) and the benchmark's probe library.
+    Returns the scoring library's path."""
+    newest = _newest_source()
+    if force or not os.path.exists(LIB) or os.path.getmtime(LIB) < newest:
+        _compile(LIB, SOURCES, verbose)
+    if force or not os.path.exists(PROBE_LIB) or os.path.getmtime(PROBE_LIB) < newest:
+        _compile(PROBE_LIB, PROBE_SOURCES, verbose)
     return LIB
 
 

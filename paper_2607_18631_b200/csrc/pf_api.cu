@@ -22,6 +22,7 @@ void count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
 
 struct TimingRec {
     int cls, n_kernels;
+    bool open;
     cudaEvent_t a, b;
 };
 struct Timing {
@@ -48,6 +49,7 @@ void timing_begin(pf_plan_t *p, int cls, cudaStream_t st)
     TimingRec r;
     r.cls = cls;
     r.n_kernels = 0;
+    r.open = true;
     r.a = t->get();
     r.b = t->get();
     cudaEventRecord(r.a, st);
@@ -57,9 +59,16 @@ void timing_begin(pf_plan_t *p, int cls, cudaStream_t st)
 void timing_end(pf_plan_t *p, int cls, int n_kernels, cudaStream_t st)
 {
     Timing *t = (Timing *)p->timing;
-    if (!t || !t->on || t->recs.empty() || t->recs.back().cls != cls) return;
-    t->recs.back().n_kernels = n_kernels;
-    cudaEventRecord(t->recs.back().b, st);
+    if (!t || !t->on) return;
+    // the latest open record of this class (records of classes launched on other streams may lie in between)
+    for (size_t i = t->recs.size(); i-- > 0;) {
+        TimingRec &r = t->recs[i];
+        if (r.cls != cls || !r.open) continue;
+        r.open = false;
+        r.n_kernels = n_kernels;
+        cudaEventRecord(r.b, st);
+        return;
+    }
 }
 
 }  // namespace pf
@@ -423,9 +432,15 @@ extern "C" int pf_plan_create(const pf_model_t *model, const pf_cluster_t *clust
         return PF_ECUDA;
     }
     if (phase == PF_PHASE_TRAIN) {
-        e = cudaStreamCreateWithFlags(&p->side_stream, cudaStreamNonBlocking);
+        // the fill stream carries long streaming-store kernels that should yield to everything else: lowest priority
+        int prio_lo = 0, prio_hi = 0;
+        e = cudaDeviceGetStreamPriorityRange(&prio_lo, &prio_hi);
+        if (e == cudaSuccess) e = cudaStreamCreateWithPriority(&p->side_stream, cudaStreamNonBlocking, prio_hi);
+        if (e == cudaSuccess) e = cudaStreamCreateWithPriority(&p->fill_stream, cudaStreamNonBlocking, prio_lo);
         if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->ev_fork, cudaEventDisableTiming);
         if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->ev_join, cudaEventDisableTiming);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->ev_fill, cudaEventDisableTiming);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->ev_fork2, cudaEventDisableTiming);
         if (e != cudaSuccess) {
             pf::set_cuda_error(e, "pf_plan_create: side stream");
             pf_plan_destroy(p);
@@ -457,6 +472,11 @@ extern "C" int pf_timing_read(pf_plan_t *p, float *ms, uint32_t *kernels)
     if (!t) return PF_OK;
     for (auto &r : t->recs) {
         float x = 0.f;
+        if (r.open) {   // never closed (an error return in between): no interval to report
+            t->pool.push_back(r.a);
+            t->pool.push_back(r.b);
+            continue;
+        }
         PF_CUDA_TRY(cudaEventSynchronize(r.b), "pf_timing_read");
         PF_CUDA_TRY(cudaEventElapsedTime(&x, r.a, r.b), "pf_timing_read");
         ms[r.cls] += x;
@@ -486,7 +506,10 @@ extern "C" void pf_plan_destroy(pf_plan_t *p)
     if (p->d_order) cudaFree(p->d_order);
     if (p->ev_fork) cudaEventDestroy(p->ev_fork);
     if (p->ev_join) cudaEventDestroy(p->ev_join);
+    if (p->ev_fill) cudaEventDestroy(p->ev_fill);
+    if (p->ev_fork2) cudaEventDestroy(p->ev_fork2);
     if (p->side_stream) cudaStreamDestroy(p->side_stream);
+    if (p->fill_stream) cudaStreamDestroy(p->fill_stream);
     free(p->h_vals);
     delete p;
 }

@@ -6,6 +6,7 @@
 #include <stdint.h>
 
 #include "planfront.h"
+#include "planfront_bench.h"   // timing classes of the measurement hooks
 
 namespace pf {
 
@@ -16,6 +17,15 @@ constexpr int kInnerVals = 1024;     // inner-axis values the scoring kernel kee
 constexpr int kOrderMaxSlabs = 1 << 20;  // calls with more slabs visit them by a permutation instead of an order table
 constexpr int kTailFillsPerBlock = 4;    // constant-fill slabs per block kept, at least, for the end of the visiting order
 constexpr int kFillsPerEvaluated = 3;    // fills interleaved per evaluated slab at the start of the visiting order (measured: 1: 0.392 ms, 2: 0.384, 3: 0.380, 4: 0.379, 6: 0.382, 8: 0.385, 12: 0.396)
+// Inside a search call a kernel of its own streams the constant slabs beside the simulator kernel.  Measured on
+// the benchmark's space (step time; simulator kernel / fill kernel durations while they overlap): 256 threads per
+// SM 0.651 ms (0.38 / 0.31), 128: 0.583 (0.32 / 0.29), 96: 0.578 (0.26 / 0.33), 64: 0.630 (0.25 / 0.35), 32: 0.88
+// (0.24 / 0.60) -- more store warps crowd the simulator's shared-memory polling out of the load/store pipe, fewer
+// cannot keep HBM busy.  Fills interleaved with the evaluated slabs of the scoring kernel only move time from
+// one kernel to the other (0, 2, 3, 4 per evaluated slab: 0.578, 0.582, 0.587, 0.590 ms).
+constexpr int kFillsPerEvaluatedSplit = 0;
+constexpr int kFillBlocksPerSm = 1;
+constexpr int kFillThreads = 96;
 constexpr int kQueueCap = 4096;   // cost-model queue of the scoring kernel (entries), drained when it may fill up
 
 struct DevSched {
@@ -97,11 +107,13 @@ struct pf_plan {
     uint32_t *d_order;
     uint32_t order_cap;
     uint64_t order_slab_lo;
-    uint32_t order_n_slabs, order_tail;
-    // pf_search runs the scoring call's top-k reduction beside the survivor selection: a second stream and the
-    // two events of the fork and the join (training plans; created with the plan)
-    cudaStream_t side_stream;
-    cudaEvent_t ev_fork, ev_join;
+    uint32_t order_n_slabs, order_tail, order_fpe;
+    // pf_search overlaps three things once the evaluated part of the space has been scored: the reduction of the
+    // analytic top-k (side_stream), the streaming of the constant slabs (fill_stream) and, on the caller's stream,
+    // the survivor selection and the simulator.  Streams and fork / join events belong to the plan (training
+    // plans; created with the plan).
+    cudaStream_t side_stream, fill_stream;
+    cudaEvent_t ev_fork, ev_join, ev_fork2, ev_fill;
     // simulator order tables (built at create for training plans)
     void *sim_tables;
     // optional per-kernel-class event timing (pf_timing_enable)
@@ -290,15 +302,66 @@ struct ScoreDigest {
     uint32_t chunk;   // candidates per selection chunk
 };
 
+// does the plan's order table hold this range and shape?  (hdr: slab_lo (2 words), n_slabs, tail, head length,
+// fills per evaluated slab)
+__device__ __forceinline__ bool order_table_valid(const uint32_t *hdr, uint64_t slab_lo, uint32_t n_slabs, uint32_t tail,
+                                                  uint32_t fpe)
+{
+    return hdr[0] == (uint32_t)slab_lo && hdr[1] == (uint32_t)(slab_lo >> 32) && hdr[2] == n_slabs && hdr[3] == tail &&
+           hdr[5] == fpe;
+}
+
+// While the constant slabs of a scoring call are still being streamed out, a reader of the dense outputs may
+// only trust the slabs the scoring kernel itself has written: the evaluated ones (class byte 0).  cls == NULL: no
+// fill is in flight, everything may be read.  The class bytes count only while the order table they were made
+// with is the one the scoring call used (otherwise that call's scoring kernel wrote every slab itself).
+struct FillGuard {
+    const uint8_t *cls = nullptr;
+    const uint32_t *hdr = nullptr;
+    uint64_t slab_lo = 0;
+    uint32_t n_slabs = 0, slab = 1, tail = 0, fpe = 0;
+};
+
+// What the kernel that streams the constant slabs behind the head of the visiting order needs (pf_score.cu).
+struct FillArgs {
+    uint64_t first, count, slab_lo;
+    uint32_t n_slabs, slab, order_tail, order_fpe;
+    uint8_t *reason;
+    float *tput;
+    long long *mem;
+    const uint32_t *order, *order_hdr;
+};
+
+// How a scoring call may spread over the plan's streams (all off: one stream, one scoring kernel).
+//   topk_aside: the key-list reduction runs on side_stream; ev_join is recorded when it is done.
+//   fill_aside: the scoring kernel visits the evaluated slabs only (plus `fills_per_evaluated` constant ones each);
+//               the remaining constant slabs are left to a second, lean kernel that the caller starts on
+//               fill_stream when it sees fit (fill_launch); ev_fill is recorded when that is done.
+// The caller makes its stream wait for the events it was told were recorded (*joined bits) before it touches
+// the workspace (ev_join) or lets the call's results count as complete (ev_fill).
+struct ScoreSpread {
+    bool topk_aside = false, fill_aside = false;
+    int fills_per_evaluated = kFillsPerEvaluated;
+    bool join_pending = false, fill_pending = false;   // out: events the caller still has to wait for
+    bool fill_deferred = false;                        // out: constant slabs are still to be streamed (fill_launch)
+    FillArgs fill;                                     // out: what fill_launch launches
+    FillGuard guard;                                   // out: set when fill_deferred
+};
+int fill_launch(pf_plan_t *p, ScoreSpread &sp, cudaStream_t st);
+int simulate_run(pf_plan_t *p, const uint64_t *d_surv_idx, uint64_t n, const uint64_t *d_n, uint32_t jitter_seed,
+                 float *d_tput_sim, uint8_t *d_sim_status, uint32_t k, uint64_t *d_topk_idx, float *d_topk_score,
+                 uint32_t *d_topk_count, void *d_workspace, size_t workspace_bytes, cudaStream_t st,
+                 ScoreSpread *spread);
+
 // internal entry points behind pf_score / pf_select_survivors (dg / have_digest: the fused search call)
 int score_run(pf_plan_t *p, uint64_t first, uint64_t count, uint8_t *d_reason, float *d_tput, int64_t *d_mem,
               uint32_t k, uint64_t *d_topk_idx, float *d_topk_score, uint32_t *d_topk_count, void *d_workspace,
-              size_t workspace_bytes, cudaStream_t st, const ScoreDigest *dg, bool topk_on_side_stream);
+              size_t workspace_bytes, cudaStream_t st, const ScoreDigest *dg, ScoreSpread *spread);
 int select_clear(pf_plan_t *p, uint64_t count, void *d_workspace, size_t workspace_bytes, cudaStream_t st,
                  ScoreDigest *dg_out);
 int select_run(pf_plan_t *p, uint64_t first, uint64_t count, const uint8_t *d_reason, const float *d_tput,
                uint64_t s_max, uint64_t *d_surv_idx, uint64_t *d_surv_count, void *d_workspace,
-               size_t workspace_bytes, cudaStream_t st, bool have_digest);
+               size_t workspace_bytes, cudaStream_t st, bool have_digest, const FillGuard *guard);
 
 // host: workspace layout of one top-k reduction whose producers append at most n_keys_max keys in total.
 // ctrl is 256 bytes: uint32 [0] producer work counter, [1] keys in list A, [2] keys in list B, [3] spare;

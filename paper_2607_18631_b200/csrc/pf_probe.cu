@@ -2,7 +2,17 @@
 // against: thread-instruction issue rate (independent FFMA, IMAD and LOP3/IADD chains at full occupancy)
 // and the rate of a pure streaming write.  Measurement utilities only: the paper has no counterpart and no
 // scoring call depends on them.  The caller times the launches with events on the stream it passes.
-#include "pf_internal.cuh"
+// Built into a library of its own (libplanfront_probe.so) and self-contained: nothing of the scoring library is
+// linked in.
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "planfront_bench.h"
+
+#define PF_PROBE_TRY(expr)                       \
+    do {                                         \
+        if ((expr) != cudaSuccess) return PF_ECUDA; \
+    } while (0)
 
 namespace pf {
 
@@ -70,8 +80,8 @@ __global__ void __launch_bounds__(kProbeThreads) probe_write_kernel(uint4 *dst, 
 static int sm_count(int *out)
 {
     int dev = 0;
-    PF_CUDA_TRY(cudaGetDevice(&dev), "cudaGetDevice");
-    PF_CUDA_TRY(cudaDeviceGetAttribute(out, cudaDevAttrMultiProcessorCount, dev), "cudaDeviceGetAttribute");
+    PF_PROBE_TRY(cudaGetDevice(&dev));
+    PF_PROBE_TRY(cudaDeviceGetAttribute(out, cudaDevAttrMultiProcessorCount, dev));
     return PF_OK;
 }
 
@@ -94,8 +104,7 @@ extern "C" int pf_probe_alu(int kind, uint32_t iters, uint32_t *d_sink, uint64_t
         probe_alu_kernel<PF_PROBE_IMAD><<<grid, kProbeThreads, 0, st>>>(iters, 3u, d_sink);
     else
         probe_alu_kernel<PF_PROBE_LOGIC><<<grid, kProbeThreads, 0, st>>>(iters, 3u, d_sink);
-    PF_CUDA_TRY(cudaGetLastError(), "probe_alu_kernel launch");
-    count_launch();
+    PF_PROBE_TRY(cudaGetLastError());
     *h_thread_instructions = (uint64_t)grid * kProbeThreads * (uint64_t)iters * kProbeChains * kProbeUnroll;
     return PF_OK;
 }
@@ -109,7 +118,6 @@ extern "C" int pf_probe_write(void *d_buf, size_t bytes, void *stream)
     if (blocks > 0x7FFFFFFFull) return PF_EINVAL;
     probe_write_kernel<<<(unsigned int)blocks, kProbeThreads, 0, (cudaStream_t)stream>>>((uint4 *)d_buf, n16,
                                                                                         0x5a5a5a5au);
-    PF_CUDA_TRY(cudaGetLastError(), "probe_write_kernel launch");
-    count_launch();
+    PF_PROBE_TRY(cudaGetLastError());
     return PF_OK;
 }

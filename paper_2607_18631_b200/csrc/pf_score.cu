@@ -35,8 +35,12 @@ struct ScoreArgs {
     const int32_t *vals;            // packed axis value lists
     const int32_t *scen;            // serve: P[n_scen], O[n_scen]
     const uint32_t *order;          // ticket -> (pre_reason << 24) | slab, or NULL: visit by slab_mul, classify here
-    const uint32_t *order_hdr;      // the range the order table holds: slab_lo (2 words), n_slabs, tail
+    const uint32_t *order_hdr;      // what the order table holds: slab_lo (2 words), n_slabs, tail, head length,
+                                    // fills per evaluated slab
     uint32_t order_tail;            // the tail length this call wants
+    uint32_t order_fpe;             // the fills per evaluated slab this call wants
+    uint32_t head_only;             // 1: visit the head of the order only (tickets below hdr[4]); a second kernel
+                                    // streams the constant slabs behind it
     ScoreDigest dg;                 // hist1 == NULL: not collected
 };
 
@@ -110,7 +114,7 @@ __global__ void __launch_bounds__(256) slab_class_kernel(const __grid_constant__
 // half of the blocks evaluating while the rest keep the store stream going) and the other fills follow: evaluated slab i sits after floor(i * Fs / H)
 // fills, fill j < Fs after min(H, ceil((j + 1) * H / Fs)) evaluated slabs.
 __global__ void __launch_bounds__(1024) slab_order_kernel(const uint8_t *cls, uint64_t slab_lo, uint32_t n_slabs,
-                                                          uint32_t tail, uint32_t *order, uint32_t *hdr)
+                                                          uint32_t tail, uint32_t fpe, uint32_t *order, uint32_t *hdr)
 {
     __shared__ uint32_t s_part[1024];
     const uint32_t tid = threadIdx.x;
@@ -128,7 +132,7 @@ __global__ void __launch_bounds__(1024) slab_order_kernel(const uint8_t *cls, ui
     }
     const uint64_t H = s_part[1023], F = n_slabs - H;
     uint64_t Fs = F > tail ? F - tail : 0;
-    if (Fs > H * kFillsPerEvaluated) Fs = H * kFillsPerEvaluated;
+    if (Fs > H * fpe) Fs = H * fpe;
     uint64_t hi_rank = s_part[tid] - h;        // evaluated slabs before this chunk
     uint64_t fi_rank = lo - hi_rank;           // filled slabs before this chunk
     for (uint32_t s = lo; s < hi; s++) {
@@ -154,6 +158,8 @@ __global__ void __launch_bounds__(1024) slab_order_kernel(const uint8_t *cls, ui
         hdr[1] = (uint32_t)(slab_lo >> 32);
         hdr[2] = n_slabs;
         hdr[3] = tail;
+        hdr[4] = (uint32_t)(H + Fs);   // the head: every evaluated slab and the fills interleaved with them
+        hdr[5] = fpe;
     }
 }
 
@@ -233,14 +239,15 @@ __global__ void __launch_bounds__(kThreads, 4) score_kernel(const __grid_constan
     // the same slab, after thread 0's share of the slab's stores, to set up the following slab.
     // The order table belongs to the plan and holds one range: use it only if that is this call's range.
     const uint32_t *order = nullptr;
-    if (A.order && A.order_hdr[0] == (uint32_t)A.slab_lo && A.order_hdr[1] == (uint32_t)(A.slab_lo >> 32) &&
-        A.order_hdr[2] == A.n_slabs && A.order_hdr[3] == A.order_tail)
-        order = A.order;
+    if (A.order && order_table_valid(A.order_hdr, A.slab_lo, A.n_slabs, A.order_tail, A.order_fpe)) order = A.order;
+    // tickets this launch serves: the whole order, or its head when a fill kernel follows (without a valid table
+    // this launch does everything and the fill kernel, which makes the same test, nothing)
+    const uint32_t n_tickets = (order && A.head_only) ? A.order_hdr[4] : A.n_slabs;
     auto resolve = [&](uint32_t s, uint32_t w, SlabInfo &dst) {
         SlabInfo si;
         si.slab = 0xFFFFFFFFu;
         si.pre_reason = 0;
-        if (s < A.n_slabs) {
+        if (s < n_tickets) {
             if (order) {
                 // the visiting order and every slab's class were prepared by the launches before this one
                 si.slab = w & 0xFFFFFFu;
@@ -262,7 +269,7 @@ __global__ void __launch_bounds__(kThreads, 4) score_kernel(const __grid_constan
         const uint32_t t0 = blockIdx.x;
         s_gthr = 0ull;
         tkt_next = gridDim.x + atomicAdd(A.slab_counter, 1u);
-        resolve(t0, (order && t0 < A.n_slabs) ? __ldcg(order + t0) : 0u, s_slabs[0]);
+        resolve(t0, (order && t0 < n_tickets) ? __ldcg(order + t0) : 0u, s_slabs[0]);
     }
     __syncthreads();
 
@@ -270,7 +277,7 @@ __global__ void __launch_bounds__(kThreads, 4) score_kernel(const __grid_constan
         const SlabInfo &s_slab = s_slabs[cur];
         if (s_slab.slab == 0xFFFFFFFFu) break;
         if (tid == 0) {
-            word_next = (order && tkt_next < A.n_slabs) ? __ldcg(order + tkt_next) : 0u;
+            word_next = (order && tkt_next < n_tickets) ? __ldcg(order + tkt_next) : 0u;
             tkt_after = gridDim.x + atomicAdd(A.slab_counter, 1u);
             // the grid-wide threshold only matters to evaluated slabs: refresh it on those
             if (want_topk && s_slab.pre_reason == 0) gthr_next = *reinterpret_cast<volatile unsigned long long *>(A.g_thr);
@@ -626,6 +633,27 @@ __global__ void __launch_bounds__(kThreads, 4) score_kernel(const __grid_constan
     }
 }
 
+// The constant slabs behind the head of the visiting order, streamed by a kernel of their own: no shared memory,
+// few registers, so that it shares the SMs with whatever else runs meanwhile (the survivor selection and the
+// simulator inside a search call).  Tickets [hdr[4], n_slabs) are all constant slabs by construction of the order;
+// blocks take them round robin (they are all the same size but for a clipped first or last one).
+__global__ void __launch_bounds__(kThreads) fill_tail_kernel(const FillArgs A)
+{
+    if (!order_table_valid(A.order_hdr, A.slab_lo, A.n_slabs, A.order_tail, A.order_fpe)) return;
+    const uint32_t head_n = A.order_hdr[4];
+    for (uint32_t t = head_n + blockIdx.x; t < A.n_slabs; t += gridDim.x) {
+        const uint32_t w = __ldg(A.order + t);
+        const uint64_t base = (A.slab_lo + (w & 0xFFFFFFu)) * (uint64_t)A.slab;
+        const uint64_t lo = base > A.first ? base : A.first;
+        const uint64_t end_slab = base + A.slab, end_call = A.first + A.count;
+        const uint64_t hi = end_slab < end_call ? end_slab : end_call;
+        const uint64_t rel0 = lo - A.first, n = hi - lo;
+        if (A.reason) block_fill(A.reason + rel0, n, w >> 24);
+        if (A.tput) block_fill(reinterpret_cast<uint8_t *>(A.tput + rel0), n * 4, 0u);
+        if (A.mem) block_fill(reinterpret_cast<uint8_t *>(A.mem + rel0), n * 8, 0u);
+    }
+}
+
 // ------------------------------------------------------------------ reducing a compact key list
 
 struct ReduceArgs {
@@ -907,6 +935,30 @@ __global__ void __launch_bounds__(kThreads) merge2_kernel(const Merge2Args A)
     if (tid == 0) *A.cnt_out = (uint32_t)n;
 }
 
+// Start streaming the constant slabs a split scoring call left behind: on the plan's fill stream, after everything
+// `st` holds so far.  Records ev_fill behind the kernel; the caller makes `st` wait for it before the call's
+// results count as complete.
+int fill_launch(pf_plan_t *p, ScoreSpread &sp, cudaStream_t st)
+{
+    if (!sp.fill_deferred) return PF_OK;
+    sp.fill_deferred = false;
+    cudaStream_t fs = p->fill_stream;
+    PF_CUDA_TRY(cudaEventRecord(p->ev_fork2, st), "fill fork");
+    PF_CUDA_TRY(cudaStreamWaitEvent(fs, p->ev_fork2, 0), "fill fork");
+    // from here on the fill stream is forked: record the join event whatever happens
+    timing_begin(p, PF_T_FILL, fs);
+    fill_tail_kernel<<<p->sm_count * kFillBlocksPerSm, kFillThreads, 0, fs>>>(sp.fill);
+    count_launch();
+    timing_end(p, PF_T_FILL, 1, fs);
+    const cudaError_t e = cudaGetLastError();
+    if (cudaEventRecord(p->ev_fill, fs) == cudaSuccess) sp.fill_pending = true;
+    if (e != cudaSuccess) {
+        set_cuda_error(e, "fill_tail_kernel launch");
+        return PF_ECUDA;
+    }
+    return PF_OK;
+}
+
 static int grid_for(const pf_plan_t *p, uint64_t n_slabs)
 {
     uint64_t g = (uint64_t)p->sm_count * 4;
@@ -939,13 +991,16 @@ extern "C" int pf_score(pf_plan_t *p, uint64_t first, uint64_t count, uint8_t *d
                         uint32_t *d_topk_count, void *d_workspace, size_t workspace_bytes, void *stream)
 {
     return pf::score_run(p, first, count, d_reason, d_tput, d_mem, k, d_topk_idx, d_topk_score, d_topk_count,
-                         d_workspace, workspace_bytes, (cudaStream_t)stream, nullptr, false);
+                         d_workspace, workspace_bytes, (cudaStream_t)stream, nullptr, nullptr);
 }
 
 int pf::score_run(pf_plan_t *p, uint64_t first, uint64_t count, uint8_t *d_reason, float *d_tput, int64_t *d_mem,
                   uint32_t k, uint64_t *d_topk_idx, float *d_topk_score, uint32_t *d_topk_count, void *d_workspace,
-                  size_t workspace_bytes, cudaStream_t st, const ScoreDigest *dg, bool topk_on_side_stream)
+                  size_t workspace_bytes, cudaStream_t st, const ScoreDigest *dg, ScoreSpread *spread)
 {
+    ScoreSpread plain;
+    ScoreSpread &sp = spread ? *spread : plain;
+    sp.join_pending = sp.fill_pending = sp.fill_deferred = false;
     if (!p) return PF_EINVAL;
     if (k > PF_K_MAX) return PF_EINVAL;
     if (k > 0 && (!d_topk_idx || !d_topk_score || !d_topk_count)) return PF_EINVAL;
@@ -984,9 +1039,16 @@ int pf::score_run(pf_plan_t *p, uint64_t first, uint64_t count, uint8_t *d_reaso
     int n_score_kernels = 1;
     a.order_hdr = nullptr;
     a.order_tail = (uint32_t)grid * kTailFillsPerBlock;
+    a.order_fpe = (uint32_t)(sp.fills_per_evaluated < 0 ? 0 : sp.fills_per_evaluated);
+    a.head_only = 0;
+    bool split = false;
     if (p->d_order && n_slabs <= p->order_cap && n_slabs > (uint64_t)grid) {
         uint32_t *hdr = p->d_order, *order = p->d_order + 64;
-        if (p->order_slab_lo != slab_lo || p->order_n_slabs != (uint32_t)n_slabs || p->order_tail != a.order_tail) {
+        split = sp.fill_aside && p->fill_stream && (d_reason || d_tput || d_mem);
+        // with a fill kernel behind it the scoring kernel ends on evaluated slabs anyway: no fills are held back
+        if (split) a.order_tail = 0;
+        if (p->order_slab_lo != slab_lo || p->order_n_slabs != (uint32_t)n_slabs || p->order_tail != a.order_tail ||
+            p->order_fpe != a.order_fpe) {
             // another range than the table was last built for: rebuild it (two small launches)
             uint8_t *cls = (uint8_t *)(order + p->order_cap);
             const unsigned cgrid = (unsigned)((n_slabs + 255) / 256);
@@ -996,7 +1058,8 @@ int pf::score_run(pf_plan_t *p, uint64_t first, uint64_t count, uint8_t *d_reaso
             else
                 slab_class_kernel<uint32_t><<<cgrid, 256, 0, st>>>(p->dev, p->d_vals, slab_lo, (uint32_t)n_slabs,
                                                                    cls);
-            slab_order_kernel<<<1, 1024, 0, st>>>(cls, slab_lo, (uint32_t)n_slabs, a.order_tail, order, hdr);
+            slab_order_kernel<<<1, 1024, 0, st>>>(cls, slab_lo, (uint32_t)n_slabs, a.order_tail, a.order_fpe, order,
+                                                  hdr);
             PF_CUDA_TRY(cudaGetLastError(), "slab order launch");
             count_launch();
             count_launch();
@@ -1004,9 +1067,11 @@ int pf::score_run(pf_plan_t *p, uint64_t first, uint64_t count, uint8_t *d_reaso
             p->order_slab_lo = slab_lo;
             p->order_n_slabs = (uint32_t)n_slabs;
             p->order_tail = a.order_tail;
+            p->order_fpe = a.order_fpe;
         }
         a.order = order;
         a.order_hdr = hdr;
+        a.head_only = split ? 1u : 0u;
     }
     const size_t queue_bytes = p->dev.phase == PF_PHASE_TRAIN
                                    ? (((size_t)p->dev.slab + 16 + 15) & ~(size_t)15) + kQueueCap * sizeof(uint16_t)
@@ -1025,25 +1090,45 @@ int pf::score_run(pf_plan_t *p, uint64_t first, uint64_t count, uint8_t *d_reaso
     count_launch();
     timing_end(p, PF_T_SCORE, n_score_kernels, st);
     PF_CUDA_TRY(cudaGetLastError(), "score_kernel launch");
+    const bool topk_aside = k > 0 && sp.topk_aside && p->side_stream;
+    int rc = PF_OK;
+    if (topk_aside) PF_CUDA_TRY(cudaEventRecord(p->ev_fork, st), "score fork");
+    if (split) {
+        // the caller decides when the constant slabs start to stream (fill_launch): until then, and while they do,
+        // only the evaluated slabs of the dense outputs hold results (guard)
+        FillArgs &f = sp.fill;
+        f.first = first; f.count = count; f.slab_lo = slab_lo; f.n_slabs = (uint32_t)n_slabs;
+        f.slab = p->dev.slab; f.order_tail = a.order_tail; f.order_fpe = a.order_fpe;
+        f.reason = d_reason; f.tput = d_tput; f.mem = (long long *)d_mem;
+        f.order = a.order; f.order_hdr = a.order_hdr;
+        sp.fill_deferred = true;
+        sp.guard.cls = (const uint8_t *)(a.order + p->order_cap);
+        sp.guard.hdr = a.order_hdr;
+        sp.guard.slab_lo = slab_lo; sp.guard.n_slabs = (uint32_t)n_slabs; sp.guard.slab = p->dev.slab;
+        sp.guard.tail = a.order_tail; sp.guard.fpe = a.order_fpe;
+    }
     if (k > 0) {
         // The reduction of the key list depends on the scoring kernel only.  Inside a search call it runs on the
         // plan's second stream, beside the survivor selection; the caller joins (ev_join) before it reuses the
         // workspace.
         cudaStream_t rs = st;
-        if (topk_on_side_stream && p->side_stream) {
+        if (topk_aside) {
             rs = p->side_stream;
-            PF_CUDA_TRY(cudaEventRecord(p->ev_fork, st), "top-k fork");
-            PF_CUDA_TRY(cudaStreamWaitEvent(rs, p->ev_fork, 0), "top-k fork");
+            cudaError_t e = cudaStreamWaitEvent(rs, p->ev_fork, 0);
+            if (e != cudaSuccess) {
+                set_cuda_error(e, "top-k fork");
+                return PF_ECUDA;   // nothing was forked onto the side stream
+            }
         }
         timing_begin(p, PF_T_TOPK, rs);
         int nk = 0;
-        int rc = launch_topk_reduce(ws, lay, (uint64_t)grid * k, k, first, nullptr, d_topk_idx, d_topk_score,
-                                    d_topk_count, rs, &nk);
+        const int rc2 = launch_topk_reduce(ws, lay, (uint64_t)grid * k, k, first, nullptr, d_topk_idx, d_topk_score,
+                                           d_topk_count, rs, &nk);
         timing_end(p, PF_T_TOPK, nk, rs);
-        if (rs != st) PF_CUDA_TRY(cudaEventRecord(p->ev_join, rs), "top-k join");
-        return rc;
+        if (rs != st && cudaEventRecord(p->ev_join, rs) == cudaSuccess) sp.join_pending = true;
+        if (rc == PF_OK) rc = rc2;
     }
-    return PF_OK;
+    return rc;
 }
 
 // ------------------------------------------------------------------ pf_score without a caller workspace

@@ -76,17 +76,29 @@ static int search_device(pf_plan_t *p, uint32_t k, uint64_t s_max, uint32_t k_si
         if (rc != PF_OK) return rc;
         pdg = &dg;
     }
-    // with a simulator tier to follow, the analytic top-k is reduced on the plan's second stream while this one
-    // goes on with the selection; the simulator reuses the scoring scratch, so the two join before it
-    const bool side = sim && p->side_stream != nullptr;
-    rc = score_run(p, 0, p->size, d_reason, d_tput, d_mem, k, d_tk_idx, d_tk_sc, d_tk_cnt, ws, ws_bytes, st, pdg,
-                   side);
-    if (rc != PF_OK || !sim) return rc;
-    rc = select_run(p, 0, p->size, d_reason, d_tput, s_max, d_surv, d_surv_cnt, ws_sel, ws_sel_bytes, st, true);
-    if (side) PF_CUDA_TRY(cudaStreamWaitEvent(st, p->ev_join, 0), "top-k join");
-    if (rc != PF_OK) return rc;
-    return pf_simulate(p, d_surv, s_max, d_surv_cnt, jitter_seed, nullptr, nullptr, k_sim, d_sim_idx, d_sim_sc,
-                       d_sim_cnt, ws, ws_bytes, (void *)st);
+    // With a simulator tier to follow, the call spreads over the plan's streams.  The scoring kernel deals with the
+    // evaluated slabs (every feasible plan, the digest and the top-k keys come from those) and a share of the
+    // constant ones; then the analytic top-k is reduced on the second stream beside the selection -- chains of
+    // short launches that crawl under a saturated store stream, so nothing streams meanwhile; then the remaining
+    // constant slabs (most of the dense outputs' bytes, which nothing downstream reads) are streamed by a lean
+    // kernel on the fill stream beside the simulator kernel, which works in shared memory; the two join before
+    // the re-ranking.  The simulator reuses the scoring scratch, so the top-k joins before it.
+    ScoreSpread sp;
+    sp.topk_aside = sim && p->side_stream != nullptr;
+    sp.fill_aside = sim && p->fill_stream != nullptr;
+    sp.fills_per_evaluated = sp.fill_aside ? kFillsPerEvaluatedSplit : kFillsPerEvaluated;
+    rc = score_run(p, 0, p->size, d_reason, d_tput, d_mem, k, d_tk_idx, d_tk_sc, d_tk_cnt, ws, ws_bytes, st, pdg, &sp);
+    if (rc == PF_OK && sim)
+        rc = select_run(p, 0, p->size, d_reason, d_tput, s_max, d_surv, d_surv_cnt, ws_sel, ws_sel_bytes, st, true,
+                        (sp.fill_deferred || sp.fill_pending) ? &sp.guard : nullptr);
+    // joins are unconditional once a fork has happened, error returns included
+    if (sp.join_pending && cudaStreamWaitEvent(st, p->ev_join, 0) != cudaSuccess && rc == PF_OK) rc = PF_ECUDA;
+    if (rc == PF_OK && sim)
+        rc = simulate_run(p, d_surv, s_max, d_surv_cnt, jitter_seed, nullptr, nullptr, k_sim, d_sim_idx, d_sim_sc,
+                          d_sim_cnt, ws, ws_bytes, st, &sp);
+    if (rc == PF_OK && sp.fill_deferred) rc = fill_launch(p, sp, st);
+    if (sp.fill_pending && cudaStreamWaitEvent(st, p->ev_fill, 0) != cudaSuccess && rc == PF_OK) rc = PF_ECUDA;
+    return rc;
 }
 
 }  // namespace pf

@@ -35,7 +35,16 @@ struct SelArgs {
     unsigned long long *blk_gt, *blk_eq;  // per block counts, then exclusive prefixes
     uint64_t *surv_idx, *surv_count;
     uint64_t chunk;                   // candidates per block (multiple of 16)
+    FillGuard guard;                  // slabs still being filled by another stream must not be read
 };
+
+// class bytes to consult, or NULL when every slab may be read
+__device__ __forceinline__ const uint8_t *sel_guard_cls(const SelArgs &A)
+{
+    const FillGuard &g = A.guard;
+    if (!g.cls || !order_table_valid(g.hdr, g.slab_lo, g.n_slabs, g.tail, g.fpe)) return nullptr;
+    return g.cls;
+}
 
 // eligibility beyond feasibility: the simulator's domain (pp <= 32 ranks, <= 8 virtual stages per rank)
 __device__ __forceinline__ bool in_sim_domain(const DevPlan &P, const int32_t *vals, uint64_t idx)
@@ -97,10 +106,13 @@ __device__ __forceinline__ void for_each_eligible16(const DevPlan &P, const int3
                        ((x3 - 0x01010101u) & ~x3);
     if ((z & 0x80808080u) == 0) return;
     uint32_t m = feasible_mask16(r);
+    const uint8_t *cls = sel_guard_cls(A);
     while (m) {
         int i = __ffs(m) - 1;
         m &= m - 1;
         uint64_t rel = e + i;
+        // a byte of a slab that is still being filled is not a result yet
+        if (cls && cls[(A.first + rel) / A.guard.slab - A.guard.slab_lo] != 0) continue;
         if (in_sim_domain(P, vals, A.first + rel)) f(rel, __float_as_uint(__ldg(A.tput + rel)));
     }
 }
@@ -520,7 +532,7 @@ extern "C" int pf_select_survivors(pf_plan_t *p, uint64_t first, uint64_t count,
                                    void *d_workspace, size_t workspace_bytes, void *stream)
 {
     return select_run(p, first, count, d_reason, d_tput, s_max, d_surv_idx, d_surv_count, d_workspace,
-                      workspace_bytes, (cudaStream_t)stream, false);
+                      workspace_bytes, (cudaStream_t)stream, false, nullptr);
 }
 
 // Zero the selection's control words, histograms and per-chunk counts and say where the scoring kernel may collect
@@ -546,7 +558,7 @@ int pf::select_clear(pf_plan_t *p, uint64_t count, void *d_workspace, size_t wor
 
 int pf::select_run(pf_plan_t *p, uint64_t first, uint64_t count, const uint8_t *d_reason, const float *d_tput,
                    uint64_t s_max, uint64_t *d_surv_idx, uint64_t *d_surv_count, void *d_workspace,
-                   size_t workspace_bytes, cudaStream_t st, bool have_digest)
+                   size_t workspace_bytes, cudaStream_t st, bool have_digest, const FillGuard *guard)
 {
     if (!p || !d_reason || !d_tput || !d_surv_idx || !d_surv_count) return PF_EINVAL;
     if (p->dev.phase != PF_PHASE_TRAIN) return PF_EUNSUPPORTED;
@@ -567,6 +579,7 @@ int pf::select_run(pf_plan_t *p, uint64_t first, uint64_t count, const uint8_t *
     a.blk_gt = (unsigned long long *)(ws + lay.off_gt);
     a.blk_eq = (unsigned long long *)(ws + lay.off_eq);
     a.surv_idx = d_surv_idx; a.surv_count = d_surv_count; a.chunk = lay.chunk;
+    if (guard) a.guard = *guard;
     // control words, histograms and the per-chunk counts start at zero (chunks that are not on the eligible list
     // are never written again); with a digest the scoring kernel has filled the first pass's part already
     if (!have_digest) PF_CUDA_TRY(cudaMemsetAsync(ws, 0, lay.off_elig, st), "pf_select_survivors: clear");

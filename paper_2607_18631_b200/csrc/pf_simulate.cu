@@ -172,12 +172,11 @@ __device__ __forceinline__ uint32_t mix32(uint32_t x)
     return x;
 }
 
-// multiplicative jitter in [0.9, 1.1): counter hash of (seed, candidate, stage, F/B)
-__device__ __forceinline__ float jitter(uint32_t seed_mixed, uint64_t idx, int q, int is_b)
+// multiplicative jitter in [0.9, 1.1): counter hash of (seed, candidate, stage, F/B); `cand_hash` is the part of
+// the chain that depends on the seed and the candidate only
+__device__ __forceinline__ float jitter(uint32_t cand_hash, int q, int is_b)
 {
-    uint32_t h = mix32(seed_mixed ^ (uint32_t)idx);
-    h = mix32(h ^ (uint32_t)(idx >> 32));
-    h = mix32(h ^ (uint32_t)(2 * q + is_b));
+    const uint32_t h = mix32(cand_hash ^ (uint32_t)(2 * q + is_b));
     float u = (float)(h >> 8) * (1.0f / 16777216.0f);
     return 0.9f + 0.2f * u;
 }
@@ -190,6 +189,22 @@ constexpr int kSimThreads = 128;        // 4 warps per block, each with its own 
 __host__ __device__ inline int sim_class_entries(int c) { return 256 << c; }
 __host__ __device__ inline int sim_group_lanes(int g) { return 8 << g; }
 
+// What the simulator kernel needs about one survivor, worked out once by the pre-pass (one thread per survivor)
+// instead of by every lane of the group that simulates it: the per-layer times, the hand-over latency, the rest of
+// the step, the pricing, the shape.  64 bytes, read with four 16-byte loads.
+struct __align__(16) SimRec {
+    float F_l, B_l, F_ld, B_ld;     // forward / backward time of a MoE layer and of a leading dense layer
+    float headF, p, rest, denom;    // head forward, stage hand-over, step time beyond the pipeline, world x taxes
+    uint32_t hash, w, meta, m;      // jitter hash of (seed, candidate); position in the caller's list; shape; microbatches
+    uint32_t pad[4];
+};
+static_assert(sizeof(SimRec) == 64, "SimRec is read as four 16-byte words");
+// meta: pp - 1 (5 bits) | v - 1 (3 bits) << 5 | kind (2 bits) << 8 | m_sim (7 bits) << 10
+__device__ __forceinline__ uint32_t sim_meta(int pp, int v, int kind, int m_sim)
+{
+    return (uint32_t)(pp - 1) | ((uint32_t)(v - 1) << 5) | ((uint32_t)kind << 8) | ((uint32_t)m_sim << 10);
+}
+
 struct SimArgs {
     const uint64_t *surv;
     uint64_t n;
@@ -197,12 +212,14 @@ struct SimArgs {
     uint32_t seed;
     float *tput_sim;
     uint8_t *status;
-    unsigned int *work;             // [kSimBins] work-queue heads
+    unsigned int *work;             // [1] the batch queue's head
     unsigned int *bin_count;        // [kSimBins] survivors per bin
-    unsigned int *bin_off;          // [kSimBins + 1] start of each bin in the list
+    unsigned int *bin_off;          // [kSimBins + 1] start of each bin in the record array
     unsigned int *bin_fill;         // [kSimBins] scatter cursors
-    uint8_t *bin_of;                // [n] bin of each survivor
-    uint32_t *list;                 // [n] positions in surv, grouped by bin
+    unsigned int *bin_seq;          // [64] bins in the order the batch queue serves them
+    unsigned int *batch_pre;        // [65] batches before each position of that order; [64] = all batches
+    uint8_t *bin_of;                // [n] bin of each survivor (0xFF: not simulated)
+    SimRec *recs;                   // [n] records, grouped by bin
     const int32_t *vals;
     const uint8_t *dual_ops;
     const int32_t *dual_off;
@@ -211,11 +228,69 @@ struct SimArgs {
     int warp_floats;                // shared-memory slice of one warp, in floats
 };
 
-// Pre-pass 1: one thread per survivor decides its bin -- the smallest timeline class that holds its
-// stage-streams x microbatches, and the lane-group width that holds its pipeline depth -- so that timelines of
-// similar size are scheduled together and several shallow pipelines share a warp.  Entries that cannot be
-// simulated (outside the domain, malformed) go to bin 0, where the simulator rejects them before touching a
-// timeline.
+// candidates a warp simulates side by side in one batch of a bin: as many lane groups as fit the warp, as many
+// timelines as fit its slice
+__host__ __device__ inline int sim_bin_batch(int bin, int cls_hi)
+{
+    const int cls = bin / (kSimGroups * kSimKinds), gi = (bin / kSimKinds) % kSimGroups;
+    const int by_lanes = 32 / sim_group_lanes(gi), by_room = sim_class_entries(cls_hi) / sim_class_entries(cls);
+    return by_lanes < by_room ? by_lanes : by_room;
+}
+
+// A survivor as the pre-pass sees it: decoded, checked, timed.
+template <typename RI>
+struct SimCand {
+    TrainTuple c;
+    TrainDerived<RI> D;
+    TrainMem M;
+    TrainTimes T;
+    int reason;
+};
+
+template <typename RI>
+__device__ __forceinline__ void sim_decode(const DevPlan &P, const int32_t *vals, uint64_t idx, SimCand<RI> &S,
+                                           bool with_times)
+{
+    int v[PF_MAX_AXES];
+    uint64_t rem = idx;
+#pragma unroll
+    for (int a = 0; a < PF_MAX_AXES; a++) {
+        uint64_t r = P.radix[a];
+        uint64_t q = rem / r;
+        v[a] = __ldg(vals + P.val_off[a] + (int)(rem - q * r));
+        rem = q;
+    }
+    TrainTuple &c = S.c;
+    c.kv = v[0]; c.rec = v[1]; c.s = v[2]; c.mb = v[3]; c.v = v[4];
+    c.ep = v[5]; c.pp = v[6]; c.tp = v[7]; c.dp = v[8]; c.world = v[9];
+    c.sh = P.n_axes > 10 ? v[10] : PF_SHARD_ZERO1;
+    RI dp, world;
+    S.reason = train_layout_rules<RI>(P, c, 1, 3, dp, world);
+    if (S.reason == 0) S.reason = train_plan_rules<RI>(P, c, dp, world, 1, S.D);
+    if (S.reason == 0) {
+        train_memory<RI>(P, c, S.D, S.M);
+        if (S.M.mem > P.budget_bytes) S.reason = PF_R_MEMORY;
+    }
+    if (S.reason == 0 && with_times) train_times<RI>(P, c, S.D, S.M, S.T);
+}
+
+// timeline shape of a feasible candidate inside the simulator's domain
+template <typename RI>
+__device__ __forceinline__ void sim_shape(const SimCand<RI> &S, int &m_sim, int &streams)
+{
+    const int pp = S.c.pp, kind = S.D.kind;
+    m_sim = S.D.m < (RI)PF_SIM_WINDOW ? (int)S.D.m : PF_SIM_WINDOW;
+    if (kind == PF_KIND_INTERLEAVED) m_sim = (m_sim / pp) * pp;
+    streams = kind == PF_KIND_DUALPIPE ? pp : pp * S.D.v_eff;   // DualPipe-style: 2 directions x m/2
+}
+
+// Pre-pass 1, one thread per survivor: decode it, run the predicate again (the list may hold anything), and
+//   - infeasible: score 0, status UNSUPPORTED, written here;
+//   - feasible but outside the simulator's domain (or a shape no bin holds): the analytic score, status
+//     UNSUPPORTED, written here;
+//   - otherwise its bin: the smallest timeline class that holds its stage streams x microbatches, the lane-group
+//     width that holds its pipeline depth, its schedule class -- so that timelines of similar size are scheduled
+//     together, several shallow pipelines share a warp and a batch runs one specialised loop.
 template <typename RI>
 __global__ void __launch_bounds__(256) sim_classify_kernel(const __grid_constant__ DevPlan P, const SimArgs A)
 {
@@ -227,55 +302,96 @@ __global__ void __launch_bounds__(256) sim_classify_kernel(const __grid_constant
     const uint64_t w = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
     int bin = -1;
     if (w < n) {
-        uint64_t rem = A.surv[w];
-        int v[PF_MAX_AXES];
-#pragma unroll
-        for (int a = 0; a < PF_MAX_AXES; a++) {
-            uint64_t r = P.radix[a];
-            uint64_t q = rem / r;
-            v[a] = __ldg(A.vals + P.val_off[a] + (int)(rem - q * r));
-            rem = q;
-        }
-        const int s = v[2], mb = v[3], vv = v[4], pp = v[6], tp = v[7];
-        RI dp = (RI)v[8];
-        if (v[8] == 0) dp = (RI)v[9] / ((RI)tp * (RI)pp);
-        const int kind = P.sched[s].kind;
-        const int v_eff = vv == 0 ? (kind == PF_KIND_INTERLEAVED ? 2 : 1) : vv;
-        bin = 0;
-        const RI dpmb = dp * (RI)mb;
-        if (dpmb != 0 && pp <= PF_SIM_MAX_RANKS && v_eff <= PF_SIM_MAX_V) {
-            RI m = (RI)P.gbs / dpmb;
-            int m_sim = m < (RI)PF_SIM_WINDOW ? (int)m : PF_SIM_WINDOW;
-            if (kind == PF_KIND_INTERLEAVED) m_sim = (m_sim / pp) * pp;
-            const int streams = kind == PF_KIND_DUALPIPE ? pp : pp * v_eff;  // DualPipe: 2 directions x m/2
-            const int entries = streams * m_sim;
+        SimCand<RI> S;
+        sim_decode<RI>(P, A.vals, A.surv[w], S, false);
+        float out = 0.f;
+        bool direct = true;
+        if (S.reason == 0) {
+            int m_sim, streams;
+            sim_shape<RI>(S, m_sim, streams);
+            const int pp = S.c.pp, entries = streams * m_sim;
             int cls = 0;
             while (cls < kSimClasses - 1 && sim_class_entries(cls) < entries) cls++;
-            if (sim_class_entries(cls) >= entries && streams <= A.q_max)
-                bin = (cls * kSimGroups + (pp <= 8 ? 0 : (pp <= 16 ? 1 : 2))) * kSimKinds + kind;
+            const bool table_ok = S.D.kind != PF_KIND_DUALPIPE || __ldg(A.dual_off + pp * 33 + m_sim / 2) >= 0;
+            if (pp <= PF_SIM_MAX_RANKS && S.D.v_eff <= PF_SIM_MAX_V && cls <= A.cls_hi &&
+                sim_class_entries(cls) >= entries && streams <= A.q_max && table_ok) {
+                bin = (cls * kSimGroups + (pp <= 8 ? 0 : (pp <= 16 ? 1 : 2))) * kSimKinds + S.D.kind;
+                direct = false;
+            } else {
+                train_times<RI>(P, S.c, S.D, S.M, S.T);
+                out = train_price<RI>(P, S.c, S.D, S.T, train_pipe_analytic<RI>(P, S.c, S.D, S.T));
+                // inside the domain but without a bin (a shape the plan's bounds do not cover): reported, not run
+                if (pp <= PF_SIM_MAX_RANKS && S.D.v_eff <= PF_SIM_MAX_V) out = 0.f;
+            }
         }
-        A.bin_of[w] = (uint8_t)bin;
+        if (direct) {
+            const bool in_domain = S.reason == 0 && S.c.pp <= PF_SIM_MAX_RANKS && S.D.v_eff <= PF_SIM_MAX_V;
+            if (A.tput_sim) A.tput_sim[w] = out;
+            if (A.status) A.status[w] = (uint8_t)(in_domain ? PF_SIM_STALL : PF_SIM_UNSUPPORTED);
+        }
+        A.bin_of[w] = (uint8_t)(bin < 0 ? 0xFF : bin);
     }
     // warp-aggregated count per bin
     const unsigned peers = __match_any_sync(0xFFFFFFFFu, bin);
     if (bin >= 0 && (int)(threadIdx.x & 31) == __ffs(peers) - 1) atomicAdd(A.bin_count + bin, (unsigned int)__popc(peers));
 }
 
-// Pre-pass 2 (one thread): bin offsets.
-__global__ void sim_offsets_kernel(const SimArgs A)
+// Pre-pass 2 (one warp): where each bin's records start, and the batch queue: bins are served interleaved
+// schedules first, then DualPipe-style, then 1F1B (the per-rank op chains of an interleaved schedule are v times
+// longer, so the longest simulations start first and the kernel's tail is short), larger timelines first within a
+// class; batches are numbered through in that order.  Lane l owns bins / queue positions l and l + 32, so every
+// global word is read once, all loads in flight together.
+__device__ __forceinline__ unsigned int warp_incl_scan(unsigned int x, int lane)
 {
-    if (threadIdx.x == 0) {
-        unsigned int run = 0;
-        for (int b = 0; b < kSimBins; b++) {
-            A.bin_off[b] = run;
-            run += A.bin_count[b];
-        }
-        A.bin_off[kSimBins] = run;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const unsigned int y = __shfl_up_sync(0xFFFFFFFFu, x, off);
+        if (lane >= off) x += y;
     }
+    return x;
+}
+__global__ void __launch_bounds__(32) sim_offsets_kernel(const SimArgs A)
+{
+    const int lane = threadIdx.x;
+    const unsigned int c_lo = A.bin_count[lane];
+    const unsigned int c_hi = lane + 32 < kSimBins ? A.bin_count[lane + 32] : 0u;
+    const unsigned int i_lo = warp_incl_scan(c_lo, lane), i_hi = warp_incl_scan(c_hi, lane);
+    const unsigned int t_lo = __shfl_sync(0xFFFFFFFFu, i_lo, 31);
+    A.bin_off[lane] = i_lo - c_lo;
+    A.bin_off[lane + 32] = t_lo + i_hi - c_hi;        // entry kSimBins (lane 31) = all records
+    unsigned int nb[2];
+    int bin_at[2];
+#pragma unroll
+    for (int h = 0; h < 2; h++) {
+        const int pos = lane + 32 * h;
+        const bool valid = pos < kSimBins;
+        const int ko = pos / (kSimClasses * kSimGroups), rem = pos - ko * (kSimClasses * kSimGroups);
+        const int cls = kSimClasses - 1 - rem / kSimGroups, gi = rem % kSimGroups;
+        const int kind = (ko + 1) % kSimKinds;        // 0 -> interleaved, 1 -> DualPipe-style, 2 -> 1F1B
+        const int bin = valid ? (cls * kSimGroups + gi) * kSimKinds + kind : 0;
+        const unsigned int from_lo = __shfl_sync(0xFFFFFFFFu, c_lo, bin & 31);
+        const unsigned int from_hi = __shfl_sync(0xFFFFFFFFu, c_hi, bin & 31);
+        const unsigned int cnt = bin < 32 ? from_lo : from_hi;
+        bin_at[h] = bin;
+        nb[h] = 0u;
+        if (valid && cls <= A.cls_hi) {
+            const unsigned int per = (unsigned int)sim_bin_batch(bin, A.cls_hi);
+            nb[h] = (cnt + per - 1) / per;
+        }
+    }
+    const unsigned int b_lo = warp_incl_scan(nb[0], lane), b_hi = warp_incl_scan(nb[1], lane);
+    const unsigned int bt_lo = __shfl_sync(0xFFFFFFFFu, b_lo, 31);
+    A.bin_seq[lane] = (unsigned int)bin_at[0];
+    A.bin_seq[lane + 32] = (unsigned int)bin_at[1];
+    A.batch_pre[lane] = b_lo - nb[0];
+    A.batch_pre[lane + 32] = bt_lo + b_hi - nb[1];
+    if (lane == 31) A.batch_pre[64] = bt_lo + b_hi;   // all batches
 }
 
-// Pre-pass 3: scatter survivor positions into their bins.
-__global__ void __launch_bounds__(256) sim_scatter_kernel(const SimArgs A)
+// Pre-pass 3, one thread per survivor again: the binned ones get their record -- every term the simulator kernel
+// needs -- written at their place in the bin.
+template <typename RI>
+__global__ void __launch_bounds__(256) sim_records_kernel(const __grid_constant__ DevPlan P, const SimArgs A)
 {
     uint64_t n = A.n;
     if (A.d_n) {
@@ -283,13 +399,51 @@ __global__ void __launch_bounds__(256) sim_scatter_kernel(const SimArgs A)
         n = dn < n ? dn : n;
     }
     const uint64_t w = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    const int bin = w < n ? (int)A.bin_of[w] : -1;
+    const int bin = (w < n && A.bin_of[w] != 0xFF) ? (int)A.bin_of[w] : -1;
     const unsigned peers = __match_any_sync(0xFFFFFFFFu, bin);
     const int lane = threadIdx.x & 31, leader = __ffs(peers) - 1;
     unsigned int base = 0;
     if (bin >= 0 && lane == leader) base = atomicAdd(A.bin_fill + bin, (unsigned int)__popc(peers));
     base = __shfl_sync(0xFFFFFFFFu, base, leader);
-    if (bin >= 0) A.list[A.bin_off[bin] + base + __popc(peers & ((1u << lane) - 1u))] = (uint32_t)w;
+    if (bin < 0) return;
+    const uint64_t idx = A.surv[w];
+    SimCand<RI> S;
+    sim_decode<RI>(P, A.vals, idx, S, true);
+    const TrainTuple &c = S.c;
+    TrainTimes &T = S.T;
+    const DevSched &sc = P.sched[c.s];
+    if (S.D.ov && sc.n_chunks > 0 && c.sh != PF_SHARD_ZERO1_OFFLOAD) {
+        // the schedule says how it overlaps: the exposed communication of a MoE layer comes from its two-stream
+        // timeline instead of the alpha-table's hidden fraction
+        const float slow = fdiv(1.f, 1.f - sc.sm_frac), half = 0.5f * T.a2a;
+        const float cF = T.cD + T.cE, cBt = P.bwd_factor * cF + T.rc;
+        const float share = fdiv(T.cE, cF);
+        const float fwd = two_stream_layer(T.cD * slow, T.cE * slow, half, half, sc.n_chunks);
+        const float bwd = two_stream_layer(cBt * (1.f - share) * slow, cBt * share * slow, half, half, sc.n_chunks);
+        T.F_l = T.tpc + fwd;
+        T.B_l = T.tpc + bwd + (c.rec == PF_REC_FULL ? T.tpc + (fwd - cF * slow) : 0.f);
+    }
+    int m_sim, streams;
+    sim_shape<RI>(S, m_sim, streams);
+    SimRec r;
+    r.F_l = T.F_l; r.B_l = T.B_l; r.F_ld = T.F_ld; r.B_ld = T.B_ld;
+    r.headF = T.headF; r.p = T.p;
+    r.rest = (1.f - P.dp_overlap_frac) * T.T_dp + T.T_opt + P.step_overhead;
+    // what the pipeline time is priced with: tokens/s/GPU = tokens / ((T_pipe + rest) * world * taxes)
+    float denom = (float)S.D.world;
+    if (!P.kern[c.kv].is_native) denom *= 1.f + P.kern[c.kv].patch_ovh;
+    if (S.D.ov) denom *= 1.f + sc.sched_ovh;
+    if (S.D.ov && c.sh == PF_SHARD_ZERO1_OFFLOAD) denom *= 1.f + P.offload_overlap_penalty;
+    r.denom = denom;
+    r.hash = mix32(mix32(mix32(A.seed + 0x9e3779b9u) ^ (uint32_t)idx) ^ (uint32_t)(idx >> 32));
+    r.w = (uint32_t)w;
+    r.meta = sim_meta(c.pp, S.D.v_eff, S.D.kind, m_sim);
+    r.m = (uint32_t)(S.D.m > (RI)0xFFFFFFFFu ? (RI)0xFFFFFFFFu : S.D.m);
+    r.pad[0] = r.pad[1] = r.pad[2] = r.pad[3] = 0u;
+    const uint4 *src = reinterpret_cast<const uint4 *>(&r);
+    uint4 *dst = reinterpret_cast<uint4 *>(A.recs + A.bin_off[bin] + base + __popc(peers & ((1u << lane) - 1u)));
+#pragma unroll
+    for (int i = 0; i < 4; i++) dst[i] = src[i];
 }
 
 // The round loops, one per schedule class (all candidates of a batch share the class).  The timeline has one
@@ -524,9 +678,14 @@ __device__ __forceinline__ void sim_rounds_dual(volatile float *tl, const float 
 #undef PF_SIM_ROUND_END
 
 // One launch serves every bin.  Every warp owns a fixed slice of the block's shared memory, large enough for
-// one timeline of the largest class (or several of a smaller one), and works through the bins on its own --
-// largest timelines first, so the longest simulations start earliest and the tail is one candidate long.  No
-// block-level barrier is involved.
+// one timeline of the largest class (or several of a smaller one), and draws batches from one queue that runs
+// through the bins -- longest simulations first, so the tail is one candidate long.  No block-level barrier is
+// involved after the queue's tables have been staged.
+//
+// Global memory is touched three times per batch and hardly on the critical path: the next batch's queue ticket
+// is drawn while the current batch is simulated, its records are requested before the current results are reduced,
+// and the results are stored without waiting.  That matters inside a search call, where this kernel shares the GPU with a
+// saturated store stream under which every round trip to L2 takes microseconds.
 //
 // Inside a warp a candidate is run by a group of 8, 16 or 32 lanes, lane = pipeline rank; a warp takes as many
 // candidates per batch as it has groups and its slice has room.  Each lane walks its rank's fixed op order and
@@ -540,204 +699,179 @@ __device__ __forceinline__ void sim_rounds_dual(volatile float *tl, const float 
 // (and the groups of a warp) stay converged and a round costs one shared-memory poll plus one vote.  Every 64
 // rounds some lane of the warp must have advanced, otherwise its unfinished candidates are reported as
 // PF_SIM_STALL: the loop is bounded by the op count.
-template <typename RI>
 __global__ void __launch_bounds__(kSimThreads, 4) simulate_kernel(const __grid_constant__ DevPlan P, const SimArgs A)
 {
     extern __shared__ __align__(16) float s_mem[];
+    __shared__ unsigned int s_seq[64], s_pre[65], s_off[kSimBins + 1], s_cnt[kSimBins];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const uint32_t seed_mixed = mix32(A.seed + 0x9e3779b9u);
     const int E_hi = sim_class_entries(A.cls_hi);
+    for (int i = threadIdx.x; i < 65; i += kSimThreads) {
+        if (i < 64) s_seq[i] = A.bin_seq[i];
+        s_pre[i] = A.batch_pre[i];
+        if (i <= kSimBins) s_off[i] = A.bin_off[i];
+        if (i < kSimBins) s_cnt[i] = A.bin_count[i];
+    }
+    __syncthreads();
     float *slice = s_mem + (size_t)warp * A.warp_floats;   // [E_hi] timelines, then 4 x (durF, durB)[q_max]
+    const unsigned int n_batches = s_pre[64];
 
-    for (int cls = A.cls_hi; cls >= 0; cls--) {
-        for (int gk = 0; gk < kSimGroups * kSimKinds; gk++) {
-            const int gi = gk / kSimKinds, bin_kind = gk - gi * kSimKinds;
-            const int bin = (cls * kSimGroups + gi) * kSimKinds + bin_kind;
-            const unsigned int n_bin = A.bin_count[bin];
-            if (n_bin == 0) continue;
-            const int g = sim_group_lanes(gi);
-            const int E = sim_class_entries(cls);
-            const int batch = min(32 / g, E_hi / E);               // candidates this warp runs side by side
-            const int gidx = lane / g, glane = lane - gidx * g;
-            const bool group_on = gidx < batch;
-            volatile float *tl = slice + (size_t)(group_on ? gidx : 0) * E;   // the timeline
-            float *durF = slice + E_hi + (size_t)(group_on ? gidx : 0) * 2 * A.q_max, *durB = durF + A.q_max;
-            const uint32_t *list = A.list + A.bin_off[bin];
-
-            for (;;) {
-                unsigned int wi = 0;
-                if (lane == 0) wi = atomicAdd(A.work + bin, (unsigned int)batch);
-                wi = __shfl_sync(0xFFFFFFFFu, wi, 0);
-                if (wi >= n_bin) break;
-                const bool have = group_on && wi + gidx < n_bin;   // this group's candidate exists
-                const uint32_t w = have ? list[wi + gidx] : 0u;
-                const uint64_t idx = have ? A.surv[w] : 0ull;
-
-                // ---- every lane of the group derives the group's candidate
-                TrainTuple c;
-                {
-                    int v[PF_MAX_AXES];
-                    if ((idx >> 32) == 0) {
-                        uint32_t rem = (uint32_t)idx;
+    // a batch number -> its bin, its place in the bin, this lane's record
+    struct Fetch {
+        int bin;
+        bool have;
+        uint4 r[4];
+    };
+    auto locate = [&](unsigned int t, Fetch &f) {
+        f.bin = -1;
+        f.have = false;
+        if (t >= n_batches) return;
+        // position in the queue's bin order: how many positions end at or before t
+        const unsigned c0 = __ballot_sync(0xFFFFFFFFu, s_pre[lane + 1] <= t);
+        const unsigned c1 = __ballot_sync(0xFFFFFFFFu, s_pre[lane + 33] <= t);
+        const int pos = __popc(c0) + __popc(c1);
+        f.bin = (int)s_seq[pos];
+        const int gi = (f.bin / kSimKinds) % kSimGroups;
+        const int g = sim_group_lanes(gi), batch = sim_bin_batch(f.bin, A.cls_hi);
+        const unsigned int first = (t - s_pre[pos]) * (unsigned int)batch;
+        const int gidx = lane / g;
+        f.have = gidx < batch && first + gidx < s_cnt[f.bin];
+        if (f.have) {
+            const uint4 *src = reinterpret_cast<const uint4 *>(A.recs + s_off[f.bin] + first + gidx);
 #pragma unroll
-                        for (int a = 0; a < PF_MAX_AXES; a++) {
-                            uint32_t r = P.radix[a];
-                            uint32_t q = rem / r;
-                            v[a] = __ldg(A.vals + P.val_off[a] + (int)(rem - q * r));
-                            rem = q;
-                        }
-                    } else {
-                        uint64_t rem = idx;
-#pragma unroll
-                        for (int a = 0; a < PF_MAX_AXES; a++) {
-                            uint64_t r = P.radix[a];
-                            uint64_t q = rem / r;
-                            v[a] = __ldg(A.vals + P.val_off[a] + (int)(rem - q * r));
-                            rem = q;
-                        }
-                    }
-                    c.kv = v[0]; c.rec = v[1]; c.s = v[2]; c.mb = v[3]; c.v = v[4];
-                    c.ep = v[5]; c.pp = v[6]; c.tp = v[7]; c.dp = v[8]; c.world = v[9];
-                    c.sh = P.n_axes > 10 ? v[10] : PF_SHARD_ZERO1;
-                }
-                RI dp, world;
-                TrainDerived<RI> D;
-                TrainMem M;
-                TrainTimes T;
-                int reason = train_layout_rules<RI>(P, c, 1, 3, dp, world);
-                if (reason == 0) reason = train_plan_rules<RI>(P, c, dp, world, 1, D);
-                if (reason == 0) {
-                    train_memory<RI>(P, c, D, M);
-                    if (M.mem > P.budget_bytes) reason = PF_R_MEMORY;
-                }
-                // outcome without a simulation: infeasible -> 0, outside the domain -> analytic score
-                int status = PF_SIM_OK;
-                float tput_out = 0.f;
-                bool run = have && reason == 0;
-                if (have && reason != 0) status = PF_SIM_UNSUPPORTED;
-                if (run) {
-                    train_times<RI>(P, c, D, M, T);
-                    const DevSched &sc = P.sched[c.s];
-                    if (D.ov && sc.n_chunks > 0 && c.sh != PF_SHARD_ZERO1_OFFLOAD) {
-                        // the schedule says how it overlaps: the exposed communication of a MoE layer comes from
-                        // its two-stream timeline instead of the alpha-table's hidden fraction
-                        const float slow = fdiv(1.f, 1.f - sc.sm_frac), half = 0.5f * T.a2a;
-                        const float cF = T.cD + T.cE, cBt = P.bwd_factor * cF + T.rc;
-                        const float share = fdiv(T.cE, cF);
-                        const float fwd = two_stream_layer(T.cD * slow, T.cE * slow, half, half, sc.n_chunks);
-                        const float bwd = two_stream_layer(cBt * (1.f - share) * slow, cBt * share * slow, half, half,
-                                                           sc.n_chunks);
-                        T.F_l = T.tpc + fwd;
-                        T.B_l = T.tpc + bwd + (c.rec == PF_REC_FULL ? T.tpc + (fwd - cF * slow) : 0.f);
-                    }
-                    if (c.pp > PF_SIM_MAX_RANKS || D.v_eff > PF_SIM_MAX_V) {
-                        tput_out = train_price<RI>(P, c, D, T, train_pipe_analytic<RI>(P, c, D, T));
-                        status = PF_SIM_UNSUPPORTED;
-                        run = false;
-                    }
-                }
-                const int pp = run ? c.pp : 1, v = run ? D.v_eff : 1, kind = run ? D.kind : PF_KIND_1F1B;
-                const bool dual = kind == PF_KIND_DUALPIPE;
-                const int Q = dual ? pp : pp * v;
-                const long long m = run ? (long long)D.m : 1;
-                int m_sim = m < PF_SIM_WINDOW ? (int)m : PF_SIM_WINDOW;
-                if (kind == PF_KIND_INTERLEAVED) m_sim = (m_sim / pp) * pp;
-                const int nj = dual ? m_sim / 2 : m_sim;      // microbatches per stage stream
-                const int n_entries = (dual ? 2 * Q : Q) * nj;
-                // filed under a bin that cannot hold it: never for a feasible plan; reported, not overrun
-                bool stalled = run && (n_entries > E || Q > A.q_max || pp > g || kind != bin_kind);
-                if (stalled) run = false;
+            for (int i = 0; i < 4; i++) f.r[i] = __ldcg(src + i);
+        }
+    };
+    // lane 0 draws the tickets; a ticket is drawn when the batch before it starts, so that a warp commits to no
+    // more than one batch ahead (the queue's last, short batches go to whoever is free)
+    unsigned int tkt = 0;
+    if (lane == 0) tkt = atomicAdd(A.work, 1u);
+    Fetch cur, nxt;
+    locate(__shfl_sync(0xFFFFFFFFu, tkt, 0), cur);
 
-                // ---- stage durations (balanced layer split, head on the last stage, jitter), cleared timeline
-                __syncwarp();
-                if (run) {
-                    const int L_lo = P.L / Q, L_rem = P.L - L_lo * Q;
-                    for (int q = glane; q < Q; q += g) {
-                        const int nq_i = L_lo + (q < L_rem ? 1 : 0);
-                        const int start = q * L_lo + min(q, L_rem);              // first layer of the stage
-                        const int ndq = max(0, min(nq_i, P.L_dense - start));    // its leading dense layers
-                        const float nq = (float)(nq_i - ndq), nd = (float)ndq;
-                        const bool last = q == Q - 1;
-                        durF[q] = (nq * T.F_l + nd * T.F_ld + (last ? T.headF : 0.f)) * jitter(seed_mixed, idx, q, 0);
-                        durB[q] = (nq * T.B_l + nd * T.B_ld + (last ? P.bwd_factor * T.headF : 0.f)) *
-                                  jitter(seed_mixed, idx, q, 1);
-                    }
-                    // clear the timeline with 16-byte stores (the slot is a multiple of four words, 16-byte aligned)
-                    {
-                        float4 *tl4 = reinterpret_cast<float4 *>(const_cast<float *>(tl));
-                        const int n4 = (n_entries + 3) >> 2;
-                        for (int i = glane; i < n4; i += g) tl4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-                    }
-                }
-                __syncwarp();
+    while (cur.bin >= 0) {
+        if (lane == 0) tkt = atomicAdd(A.work, 1u);   // the next ticket: in flight while this batch is simulated
 
-                // ---- per-lane order state (1F1B is the one-chunk case of the unit cursors)
-                const bool rank_active = run && glane < pp;
-                const int U = dual ? 2 * nj : nj * v;          // forward units of this rank
-                const int warm = kind == PF_KIND_INTERLEAVED ? min(2 * (pp - glane - 1) + (v - 1) * pp, U)
-                                                             : min(pp - glane - 1, U);
-                const uint8_t *dops = A.dual_ops;              // any valid address for lanes that do not use it
-                if (dual && run) {
-                    const int off = __ldg(A.dual_off + pp * 33 + nj);
-                    if (off < 0) stalled = true, run = false;  // no table for this shape
-                    else dops = A.dual_ops + off + (size_t)glane * 2 * m_sim;
-                }
-                const int total_ops = (rank_active && run) ? 2 * U : 0;
-                const float lat = run ? T.p : 0.f;
-                // a batch's candidates share the schedule class of their bin: one specialised loop per class
-                int done = 0;
-                float clock = 0.f;
-                // forward-only steps at the start: one fewer than the stages of the shallowest pipeline in the warp
-                int fonly = (run && !dual) ? Q - 1 : 0x7FFFFFFF;
-                fonly = __reduce_min_sync(0xFFFFFFFFu, fonly);
-                if (fonly == 0x7FFFFFFF) fonly = 0;
-                if (bin_kind == PF_KIND_1F1B)
-                    sim_rounds_1f1b(tl, durF, durB, glane, pp, nj, warm, total_ops, lat, fonly, clock, done);
-                else if (bin_kind == PF_KIND_INTERLEAVED)
-                    sim_rounds_interleaved(tl, durF, durB, glane, pp, v, nj, U, warm, total_ops, lat, fonly, clock,
-                                           done);
-                else
-                    sim_rounds_dual(tl, durF, durB, glane, pp, nj, dops, total_ops, lat, clock, done);
-                if (done < total_ops) stalled = true;
+        const int bin = cur.bin;
+        const int cls = bin / (kSimGroups * kSimKinds), gi = (bin / kSimKinds) % kSimGroups;
+        const int bin_kind = bin % kSimKinds;
+        const int g = sim_group_lanes(gi);
+        const int E = sim_class_entries(cls);
+        const int batch = sim_bin_batch(bin, A.cls_hi);       // candidates this warp runs side by side
+        const int gidx = lane / g, glane = lane - gidx * g;
+        const bool group_on = gidx < batch;
+        volatile float *tl = slice + (size_t)(group_on ? gidx : 0) * E;   // the timeline
+        float *durF = slice + E_hi + (size_t)(group_on ? gidx : 0) * 2 * A.q_max, *durB = durF + A.q_max;
+        const bool have = cur.have;                            // this group's candidate exists
 
-                // ---- makespan, steady-state extension beyond the window, pricing (reductions inside the group)
-                float work = 0.f;
-                if (rank_active && run) {
-                    if (dual) {
-                        work = 0.5f * (durF[glane] + durB[glane] + durF[pp - 1 - glane] + durB[pp - 1 - glane]);
-                    } else {
-                        for (int cc = 0; cc < v; cc++) work += durF[cc * pp + glane] + durB[cc * pp + glane];
-                    }
-                }
-                float span = rank_active ? clock : 0.f;
-                int any_stall = stalled ? 1 : 0;
-#pragma unroll
-                for (int off = 16; off > 0; off >>= 1) {
-                    const float s2 = __shfl_xor_sync(0xFFFFFFFFu, span, off);
-                    const float w2 = __shfl_xor_sync(0xFFFFFFFFu, work, off);
-                    const int a2 = __shfl_xor_sync(0xFFFFFFFFu, any_stall, off);
-                    if (off < g) {
-                        span = fmaxf(span, s2);
-                        work = fmaxf(work, w2);
-                        any_stall |= a2;
-                    }
-                }
-                if (glane == 0 && have) {
-                    if (any_stall) {
-                        status = PF_SIM_STALL;
-                        tput_out = 0.f;
-                    } else if (run) {
-                        float T_pipe = span;
-                        if (m > m_sim) T_pipe += (float)(m - m_sim) * work;
-                        tput_out = train_price<RI>(P, c, D, T, T_pipe);
-                    }
-                    if (A.tput_sim) A.tput_sim[w] = tput_out;
-                    if (A.status) A.status[w] = (uint8_t)status;
-                }
-                __syncwarp();
+        // ---- the group's candidate, from its record
+        const float F_l = __uint_as_float(cur.r[0].x), B_l = __uint_as_float(cur.r[0].y);
+        const float F_ld = __uint_as_float(cur.r[0].z), B_ld = __uint_as_float(cur.r[0].w);
+        const float headF = __uint_as_float(cur.r[1].x), lat_p = __uint_as_float(cur.r[1].y);
+        const float rest = __uint_as_float(cur.r[1].z), denom = __uint_as_float(cur.r[1].w);
+        const uint32_t cand_hash = cur.r[2].x, w = cur.r[2].y, meta = cur.r[2].z, m_all = cur.r[2].w;
+        bool run = have;
+        const int pp = run ? (int)(meta & 31u) + 1 : 1, v = run ? (int)((meta >> 5) & 7u) + 1 : 1;
+        const int kind = run ? (int)((meta >> 8) & 3u) : PF_KIND_1F1B;
+        const int m_sim = run ? (int)((meta >> 10) & 127u) : 1;
+        const bool dual = kind == PF_KIND_DUALPIPE;
+        const int Q = dual ? pp : pp * v;
+        const int nj = dual ? m_sim / 2 : m_sim;      // microbatches per stage stream
+        const int n_entries = (dual ? 2 * Q : Q) * nj;
+        // filed under a bin that cannot hold it: never happens for the pre-pass's records; reported, not overrun
+        bool stalled = run && (n_entries > E || Q > A.q_max || pp > g || kind != bin_kind);
+        if (stalled) run = false;
+
+        // ---- stage durations (balanced layer split, head on the last stage, jitter), cleared timeline
+        __syncwarp();
+        if (run) {
+            const int L_lo = P.L / Q, L_rem = P.L - L_lo * Q;
+            for (int q = glane; q < Q; q += g) {
+                const int nq_i = L_lo + (q < L_rem ? 1 : 0);
+                const int start = q * L_lo + min(q, L_rem);              // first layer of the stage
+                const int ndq = max(0, min(nq_i, P.L_dense - start));    // its leading dense layers
+                const float nq = (float)(nq_i - ndq), nd = (float)ndq;
+                const bool last = q == Q - 1;
+                durF[q] = (nq * F_l + nd * F_ld + (last ? headF : 0.f)) * jitter(cand_hash, q, 0);
+                durB[q] = (nq * B_l + nd * B_ld + (last ? P.bwd_factor * headF : 0.f)) * jitter(cand_hash, q, 1);
             }
-        }  // lane-group widths
-    }  // classes
+            // clear the timeline with 16-byte stores (the slot is a multiple of four words, 16-byte aligned)
+            {
+                float4 *tl4 = reinterpret_cast<float4 *>(const_cast<float *>(tl));
+                const int n4 = (n_entries + 3) >> 2;
+                for (int i = glane; i < n4; i += g) tl4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+        }
+        __syncwarp();
+
+        // ---- per-lane order state (1F1B is the one-chunk case of the unit cursors)
+        const bool rank_active = run && glane < pp;
+        const int U = dual ? 2 * nj : nj * v;          // forward units of this rank
+        const int warm = kind == PF_KIND_INTERLEAVED ? min(2 * (pp - glane - 1) + (v - 1) * pp, U)
+                                                     : min(pp - glane - 1, U);
+        const uint8_t *dops = A.dual_ops;              // any valid address for lanes that do not use it
+        if (dual && run) {
+            const int off = __ldg(A.dual_off + pp * 33 + nj);
+            if (off < 0) stalled = true, run = false;  // no table for this shape
+            else dops = A.dual_ops + off + (size_t)glane * 2 * m_sim;
+        }
+        const int total_ops = (rank_active && run) ? 2 * U : 0;
+        const float lat = run ? lat_p : 0.f;
+        // a batch's candidates share the schedule class of their bin: one specialised loop per class
+        int done = 0;
+        float clock = 0.f;
+        // forward-only steps at the start: one fewer than the stages of the shallowest pipeline in the warp
+        int fonly = (run && !dual) ? Q - 1 : 0x7FFFFFFF;
+        fonly = __reduce_min_sync(0xFFFFFFFFu, fonly);
+        if (fonly == 0x7FFFFFFF) fonly = 0;
+        if (bin_kind == PF_KIND_1F1B)
+            sim_rounds_1f1b(tl, durF, durB, glane, pp, nj, warm, total_ops, lat, fonly, clock, done);
+        else if (bin_kind == PF_KIND_INTERLEAVED)
+            sim_rounds_interleaved(tl, durF, durB, glane, pp, v, nj, U, warm, total_ops, lat, fonly, clock, done);
+        else
+            sim_rounds_dual(tl, durF, durB, glane, pp, nj, dops, total_ops, lat, clock, done);
+        if (done < total_ops) stalled = true;
+
+        // the next batch's records are requested before this batch's results are reduced and stored
+        locate(__shfl_sync(0xFFFFFFFFu, tkt, 0), nxt);
+
+        // ---- makespan, steady-state extension beyond the window, pricing (reductions inside the group)
+        float work = 0.f;
+        if (rank_active && run) {
+            if (dual) {
+                work = 0.5f * (durF[glane] + durB[glane] + durF[pp - 1 - glane] + durB[pp - 1 - glane]);
+            } else {
+                for (int cc = 0; cc < v; cc++) work += durF[cc * pp + glane] + durB[cc * pp + glane];
+            }
+        }
+        float span = rank_active ? clock : 0.f;
+        int any_stall = stalled ? 1 : 0;
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+            const float s2 = __shfl_xor_sync(0xFFFFFFFFu, span, off);
+            const float w2 = __shfl_xor_sync(0xFFFFFFFFu, work, off);
+            const int a2 = __shfl_xor_sync(0xFFFFFFFFu, any_stall, off);
+            if (off < g) {
+                span = fmaxf(span, s2);
+                work = fmaxf(work, w2);
+                any_stall |= a2;
+            }
+        }
+        if (glane == 0 && have) {
+            int status = PF_SIM_OK;
+            float tput_out = 0.f;
+            if (any_stall) {
+                status = PF_SIM_STALL;
+            } else {
+                float T_pipe = span;
+                if (m_all > (uint32_t)m_sim) T_pipe += (float)(m_all - (uint32_t)m_sim) * work;
+                tput_out = fdiv((float)(P.gbs * (i64)P.seq), (T_pipe + rest) * denom);
+            }
+            if (A.tput_sim) A.tput_sim[w] = tput_out;
+            if (A.status) A.status[w] = (uint8_t)status;
+        }
+        __syncwarp();
+        cur = nxt;
+    }
 }
 
 // ------------------------------------------------------------------ top-k over a dense score array
@@ -822,18 +956,19 @@ int launch_dense_topk(const float *d_score, uint64_t n, const uint64_t *d_n, uin
 }
 
 struct SimLayout {
-    size_t off_ctrl, off_bin_of, off_list, off_scores, off_topk, total;
+    size_t off_ctrl, off_bin_of, off_recs, off_scores, off_topk, total;
     DenseTopkLayout dt;
 };
+constexpr size_t kSimCtrlBytes = 4096;   // work, bin_count, bin_off, bin_fill, bin_seq, batch_pre
 
 static SimLayout sim_layout(const pf_plan_t *p, uint64_t n, uint32_t k)
 {
     SimLayout l;
     const size_t nn = (size_t)(n ? n : 1);
-    l.off_ctrl = 0;                       // 2 KB: work, bin_count, bin_off, bin_fill (kSimBins words each)
-    l.off_bin_of = 2048;
-    l.off_list = l.off_bin_of + ((nn + 255) & ~(size_t)255);
-    l.off_scores = l.off_list + ((nn * 4 + 255) & ~(size_t)255);
+    l.off_ctrl = 0;
+    l.off_bin_of = kSimCtrlBytes;
+    l.off_recs = l.off_bin_of + ((nn + 255) & ~(size_t)255);
+    l.off_scores = l.off_recs + ((nn * sizeof(SimRec) + 255) & ~(size_t)255);
     l.off_topk = l.off_scores + ((nn * 4 + 255) & ~(size_t)255);
     l.dt = dense_topk_layout(p->sm_count, n, k);
     l.total = l.off_topk + (k ? l.dt.tk.total : 0);
@@ -858,36 +993,59 @@ static int plan_q_max(const pf_plan_t *p)
     return (int)q;
 }
 
+// geometry of the simulator kernel for a plan: largest timeline class, a warp's slice, the pool of a block
+struct SimGeom {
+    int cls_hi, warp_floats, per_sm;
+    size_t pool;
+};
+static SimGeom sim_geom(int q_max)
+{
+    SimGeom g;
+    // largest class the plan can produce; a warp's slice holds one such timeline plus four duration tables
+    const int entries_max = q_max * PF_SIM_WINDOW;
+    g.cls_hi = 0;
+    while (g.cls_hi < kSimClasses - 1 && sim_class_entries(g.cls_hi) < entries_max) g.cls_hi++;
+    g.warp_floats = sim_class_entries(g.cls_hi) + 4 * 2 * q_max;
+    g.pool = (size_t)(kSimThreads / 32) * g.warp_floats * sizeof(float);
+    g.per_sm = (int)((size_t)(227 * 1024) / (g.pool + 1024 + 1280));
+    g.per_sm = g.per_sm < 1 ? 1 : (g.per_sm > 12 ? 12 : g.per_sm);
+    return g;
+}
+
 template <typename RI>
-static int launch_simulate(pf_plan_t *p, SimArgs a, uint64_t n, cudaStream_t st, int *n_kernels)
+static int launch_simulate(pf_plan_t *p, SimArgs a, uint64_t n, cudaStream_t st, int *n_kernels, ScoreSpread *spread)
 {
     *n_kernels = 0;
+    const SimGeom geo = sim_geom(a.q_max);
+    if (geo.pool > 224 * 1024) return PF_EUNSUPPORTED;
+    a.cls_hi = geo.cls_hi;
+    a.warp_floats = geo.warp_floats;
     const unsigned int nb = (unsigned int)((n + 255) / 256);
+    timing_begin(p, PF_T_SIMPREP, st);
     sim_classify_kernel<RI><<<nb, 256, 0, st>>>(p->dev, a);
     sim_offsets_kernel<<<1, 32, 0, st>>>(a);
-    sim_scatter_kernel<<<nb, 256, 0, st>>>(a);
+    sim_records_kernel<RI><<<nb, 256, 0, st>>>(p->dev, a);
     for (int i = 0; i < 3; i++) count_launch();
-    *n_kernels += 3;
+    timing_end(p, PF_T_SIMPREP, 3, st);
     PF_CUDA_TRY(cudaGetLastError(), "simulator pre-pass launch");
-    // largest class the plan can produce; a warp's slice holds one such timeline plus four duration tables
-    const int entries_max = a.q_max * PF_SIM_WINDOW;
-    int cls_hi = 0;
-    while (cls_hi < kSimClasses - 1 && sim_class_entries(cls_hi) < entries_max) cls_hi++;
-    const int warp_floats = sim_class_entries(cls_hi) + 4 * 2 * a.q_max;
-    const size_t pool = (size_t)(kSimThreads / 32) * warp_floats * sizeof(float);
-    if (pool > 226 * 1024) return PF_EUNSUPPORTED;
-    int per_sm = (int)((size_t)(227 * 1024) / (pool + 1024));
-    per_sm = per_sm < 1 ? 1 : (per_sm > 12 ? 12 : per_sm);
-    a.cls_hi = cls_hi;
-    a.warp_floats = warp_floats;
-    const uint64_t cap = (uint64_t)p->sm_count * per_sm;
+    // Inside a search call the constant slabs of the dense outputs start to stream here, on the plan's fill
+    // stream: the kernel below works in shared memory and fetches ahead, whereas the short latency-bound launches
+    // before this point would crawl under a saturated store stream.
+    if (spread && spread->fill_deferred) {
+        const int rc = fill_launch(p, *spread, st);
+        if (rc != PF_OK) return rc;
+    }
+    const uint64_t cap = (uint64_t)p->sm_count * geo.per_sm;
     const uint64_t want = (n + kSimThreads / 32 - 1) / (kSimThreads / 32);
     const int grid = (int)(want < cap ? want : cap);
-    PF_CUDA_TRY(cudaFuncSetAttribute(simulate_kernel<RI>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pool),
+    const int threads = kSimThreads;
+    PF_CUDA_TRY(cudaFuncSetAttribute(simulate_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)geo.pool),
                 "simulate_kernel smem");
-    simulate_kernel<RI><<<grid, kSimThreads, pool, st>>>(p->dev, a);
+    timing_begin(p, PF_T_SIMULATE, st);
+    simulate_kernel<<<grid, threads, geo.pool, st>>>(p->dev, a);
     count_launch();
-    (*n_kernels)++;
+    timing_end(p, PF_T_SIMULATE, 1, st);
+    *n_kernels = 4;
     PF_CUDA_TRY(cudaGetLastError(), "simulate_kernel launch");
     return PF_OK;
 }
@@ -914,6 +1072,17 @@ extern "C" int pf_simulate(pf_plan_t *p, const uint64_t *d_surv_idx, uint64_t n,
                            uint64_t *d_topk_idx, float *d_topk_score, uint32_t *d_topk_count, void *d_workspace,
                            size_t workspace_bytes, void *stream)
 {
+    return pf::simulate_run(p, d_surv_idx, n, d_n, jitter_seed, d_tput_sim, d_sim_status, k, d_topk_idx, d_topk_score,
+                            d_topk_count, d_workspace, workspace_bytes, (cudaStream_t)stream, nullptr);
+}
+
+// spread (the search call): a split scoring call's constant slabs are started beside the simulator kernel and
+// joined before the re-ranking, which is a chain of short launches again.
+int pf::simulate_run(pf_plan_t *p, const uint64_t *d_surv_idx, uint64_t n, const uint64_t *d_n, uint32_t jitter_seed,
+                     float *d_tput_sim, uint8_t *d_sim_status, uint32_t k, uint64_t *d_topk_idx, float *d_topk_score,
+                     uint32_t *d_topk_count, void *d_workspace, size_t workspace_bytes, cudaStream_t st,
+                     ScoreSpread *spread)
+{
     if (!p || !d_surv_idx) return PF_EINVAL;
     if (p->dev.phase != PF_PHASE_TRAIN) return PF_EUNSUPPORTED;
     if (k > PF_K_MAX) return PF_EINVAL;
@@ -924,7 +1093,6 @@ extern "C" int pf_simulate(pf_plan_t *p, const uint64_t *d_surv_idx, uint64_t n,
     if (!p->sim_tables) return PF_EINVAL;
     int rc = PF_OK;
     const SimTables *tab = (const SimTables *)p->sim_tables;
-    cudaStream_t st = (cudaStream_t)stream;
     uint8_t *ws = (uint8_t *)d_workspace;
     float *scores = d_tput_sim ? d_tput_sim : (float *)(ws + lay.off_scores);
 
@@ -932,23 +1100,33 @@ extern "C" int pf_simulate(pf_plan_t *p, const uint64_t *d_surv_idx, uint64_t n,
     a.surv = d_surv_idx; a.n = n; a.d_n = d_n; a.seed = jitter_seed;
     a.tput_sim = scores; a.status = d_sim_status;
     a.work = (unsigned int *)(ws + lay.off_ctrl);
-    a.bin_count = a.work + kSimBins;
-    a.bin_off = a.bin_count + kSimBins;
-    a.bin_fill = a.bin_off + kSimBins + 1;
+    a.bin_count = a.work + 64;
+    a.bin_off = a.bin_count + 64;
+    a.bin_fill = a.bin_off + 64;
+    a.bin_seq = a.bin_fill + 64;
+    a.batch_pre = a.bin_seq + 64;
     a.bin_of = ws + lay.off_bin_of;
-    a.list = (uint32_t *)(ws + lay.off_list);
+    a.recs = (SimRec *)(ws + lay.off_recs);
     a.vals = p->d_vals; a.dual_ops = tab->d_ops; a.dual_off = tab->d_offset;
     a.q_max = plan_q_max(p);
     a.cls_hi = 0;
     a.warp_floats = 0;
-    PF_CUDA_TRY(cudaMemsetAsync(ws + lay.off_ctrl, 0, 2048, st), "pf_simulate: counter reset");
+    PF_CUDA_TRY(cudaMemsetAsync(ws + lay.off_ctrl, 0, kSimCtrlBytes, st), "pf_simulate: counter reset");
     if (n > 0) {
         int nk = 0;
-        timing_begin(p, PF_T_SIMULATE, st);
-        rc = p->dev.wide ? launch_simulate<unsigned long long>(p, a, n, st, &nk)
-                         : launch_simulate<uint32_t>(p, a, n, st, &nk);
-        timing_end(p, PF_T_SIMULATE, nk, st);
+        rc = p->dev.wide ? launch_simulate<unsigned long long>(p, a, n, st, &nk, spread)
+                         : launch_simulate<uint32_t>(p, a, n, st, &nk, spread);
         if (rc != PF_OK) return rc;
+    }
+    if (spread) {
+        if (spread->fill_deferred) {   // nothing was simulated: the fills still have to go out
+            rc = fill_launch(p, *spread, st);
+            if (rc != PF_OK) return rc;
+        }
+        if (spread->fill_pending) {
+            PF_CUDA_TRY(cudaStreamWaitEvent(st, p->ev_fill, 0), "fill join");
+            spread->fill_pending = false;
+        }
     }
     if (k > 0) {
         int nk = 0;

@@ -20,8 +20,8 @@ def lib():
     return B.load_library()
 
 
-def _declared_functions():
-    text = open(os.path.join(ROOT, "include", "planfront.h")).read()
+def _declared_functions(header="planfront.h"):
+    text = open(os.path.join(ROOT, "include", header)).read()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
     return sorted(set(re.findall(r"\b(pf_[a-z0-9_]+)\s*\(", text)))
 
@@ -32,6 +32,22 @@ def test_library_exports_every_declared_symbol(lib):
     for n in names:
         assert hasattr(lib, n), f"{n} declared in planfront.h but not exported"
     assert set(names) == set(B.EXPORTS)
+
+
+def test_measurement_hooks_are_declared_apart_and_exported_by_their_libraries(lib):
+    """The scoring header declares no measurement utility; the benchmark header's hooks are exported by the scoring
+    library (timing, launch count) and by the probe library (the roofline probes)."""
+    from paper_2607_18631_b200 import probes
+    product = set(_declared_functions())
+    assert not {n for n in product if "probe" in n or "timing" in n or "launch_count" in n}
+    bench = set(_declared_functions("planfront_bench.h"))
+    assert bench == set(B.BENCH_EXPORTS) | set(probes.EXPORTS)
+    for n in B.BENCH_EXPORTS:
+        assert hasattr(lib, n)
+    plib = probes.load_library()
+    for n in probes.EXPORTS:
+        assert hasattr(plib, n)
+        assert not hasattr(lib, n), f"{n} must not be part of the scoring library"
 
 
 def test_version_and_strings(lib):

@@ -8,7 +8,8 @@ pytestmark = pytest.mark.gpu
 
 def test_probes_report_counts_and_plausible_rates():
     import torch
-    from paper_2607_18631_b200 import binding
+    from paper_2607_18631_b200 import build as pf_build, probes as binding
+    pf_build.build()
 
     dev = torch.device("cuda", 0)
     sms = torch.cuda.get_device_properties(dev).multi_processor_count
@@ -42,16 +43,17 @@ def test_probes_report_counts_and_plausible_rates():
 
 def test_probes_reject_bad_arguments():
     import torch
-    from paper_2607_18631_b200 import binding
+    from paper_2607_18631_b200 import build as pf_build, probes as binding
+    pf_build.build()
 
     dev = torch.device("cuda", 0)
     sink = torch.zeros(1, dtype=torch.int32, device=dev)
-    with pytest.raises(binding.PlanfrontError):
+    with pytest.raises(binding.ProbeError):
         binding.pf_probe_alu("ffma", 0, sink)
-    with pytest.raises(binding.PlanfrontError):
+    with pytest.raises(binding.ProbeError):
         binding.pf_probe_alu("ffma", (1 << 24) + 1, sink)
     buf = torch.empty(64, dtype=torch.uint8, device=dev)
-    with pytest.raises(binding.PlanfrontError):
+    with pytest.raises(binding.ProbeError):
         binding.pf_probe_write(buf[:24])                         # not a multiple of 16 bytes
-    with pytest.raises(binding.PlanfrontError):
+    with pytest.raises(binding.ProbeError):
         binding.pf_probe_write(buf[8:40])                        # not 16-byte aligned

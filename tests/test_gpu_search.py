@@ -108,3 +108,37 @@ def test_search_replays_from_a_cuda_graph():
             assert torch.equal(b[k], want[k]), k
         assert torch.equal(b["surv_idx"][:n], want["surv_idx"][:n])
     plan.close()
+
+
+def test_search_ignores_what_the_output_buffers_held_before():
+    """Inside one search the constant blocks of the dense outputs are streamed out while the selection already
+    reads the evaluated ones.  Whatever the buffers held before the call -- here: every reason byte 0 ("feasible")
+    and huge scores -- must not leak into the survivor list, and the dense outputs are complete when the call's
+    stream work is done."""
+    import torch
+    import oracle
+    plan = _plan(make_config("large"))
+    orc = oracle.Oracle(make_config("large"))
+    b = plan.search(1024, 10 ** 6, 100, 4)
+    torch.cuda.synchronize()
+    want = {k: v.clone() for k, v in b.items() if k != "workspace"}
+    for s_max in (10 ** 6, 3000):
+        b["reason"].zero_()
+        b["tput"].fill_(3.0e38)
+        b["mem"].fill_(-1)
+        b["surv_idx"].fill_(-1)
+        b = plan.search(1024, s_max, 100, 4, bufs=b)
+        torch.cuda.synchronize()
+        for key in ("reason", "tput", "mem", "topk_idx", "topk_score", "topk_count"):
+            assert torch.equal(b[key], want[key]), key
+        n = int(b["surv_count"].item())
+        assert n == min(s_max, 12_905)
+        if s_max >= 12_905:
+            assert torch.equal(b["surv_idx"][:n], want["surv_idx"][:n])
+        else:
+            feas = torch.nonzero((want["reason"] & 0x7F) == 0).flatten()
+            ref = orc.select_survivors(want["reason"].cpu().numpy(), want["tput"].cpu().numpy().astype(np.float64),
+                                       0, s_max)
+            assert np.array_equal(b["surv_idx"][:n].cpu().numpy().view(np.uint64), ref)
+            assert n < feas.numel()
+    plan.close()
