@@ -20,7 +20,8 @@
  *     synchronized by the caller.  pf_search_host is the exception: it takes host buffers and returns
  *     after its copies have completed.
  *   - spec structs are copied by pf_plan_create; the caller may free them afterwards.
- *   - a handle may be used from one thread at a time, on the device that was current at create.
+ *   - a handle may be used from one thread at a time, on the device that was current at create: every call
+ *     that enqueues device work returns PF_EINVAL (nothing launched) when another device is current.
  *   - candidates are addressed by a linear index: idx = sum_a digit_a * prod_{b<a} len_b, axes listed
  *     least-significant first.  train axes: kv, rec, sched, mb, v, ep, pp, tp, dp, world [, shard];
  *     serve axes: kv, chunk, batch, dpa, ep, tp, scen.  An axis value list {0} for dp / world / v means
@@ -255,7 +256,10 @@ int pf_score(pf_plan_t *plan, uint64_t first, uint64_t count, uint8_t *d_reason,
  *     threads) race on it: issue them on one stream, or order them yourself.
  *   - A request whose workspace need (pf_score_workspace) exceeds PF_STATIC_SCRATCH_BYTES is refused with
  *     PF_EWORKSPACE before anything is launched; use pf_score with your own workspace for it.
- * Errors: as pf_score; PF_ECUDA also if the address look-up fails. */
+ *   - Only the first call on a device may make the CUDA runtime load the library's device image there (the
+ *     image holds the array); no later call changes the device's free memory.
+ * Errors: as pf_score; PF_ECUDA also if the address look-up fails; PF_EUNSUPPORTED on a device whose ordinal is
+ * 64 or more (the per-device address table is that long). */
 #define PF_STATIC_SCRATCH_BYTES (4u << 20)
 int pf_score_static(pf_plan_t *plan, uint64_t first, uint64_t count, uint8_t *d_reason, float *d_tput,
                     int64_t *d_mem, uint32_t k, uint64_t *d_topk_idx, float *d_topk_score, uint32_t *d_topk_count,

@@ -84,6 +84,7 @@ extern "C" int pf_aggregate_serving(pf_plan_t *p, const uint8_t *d_reason, const
     if (n_plans >= PF_MAX_COUNT) return PF_ERANGE;
     const AggLayout lay = agg_layout(p, n_plans, k);
     if (!d_workspace || ((uintptr_t)d_workspace & 255) != 0 || workspace_bytes < lay.total) return PF_EWORKSPACE;
+    if (int rc_dev = check_device(p)) return rc_dev;
     cudaStream_t st = (cudaStream_t)stream;
     uint8_t *ws = (uint8_t *)d_workspace;
     const int scen_axis = p->dev.n_axes - 1;

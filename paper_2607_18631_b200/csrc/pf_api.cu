@@ -20,6 +20,17 @@ void set_cuda_error(cudaError_t e, const char *where)
 }
 void count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
 
+int check_device(const pf_plan_t *p)
+{
+    int dev = -1;
+    PF_CUDA_TRY(cudaGetDevice(&dev), "current device");
+    if (dev != p->device) {
+        snprintf(g_cuda_msg, sizeof(g_cuda_msg), "the plan belongs to device %d, the current device is %d", p->device, dev);
+        return PF_EINVAL;
+    }
+    return PF_OK;
+}
+
 struct TimingRec {
     int cls, n_kernels;
     bool open;

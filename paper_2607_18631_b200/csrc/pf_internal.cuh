@@ -124,6 +124,9 @@ namespace pf {
 
 // ------------------------------------------------------------------ error plumbing (host)
 void set_cuda_error(cudaError_t e, const char *where);
+// PF_OK when the plan's device is the calling thread's current device, PF_EINVAL otherwise (a launch on another
+// device would hand its kernels pointers of the plan's device: a fault on the GPU instead of an error code)
+int check_device(const pf_plan_t *p);
 void count_launch();
 // event pair around the launches of one kernel class; no-ops unless pf_timing_enable(plan, 1)
 void timing_begin(pf_plan_t *p, int cls, cudaStream_t st);

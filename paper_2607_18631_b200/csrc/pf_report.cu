@@ -87,6 +87,7 @@ extern "C" int pf_report(pf_plan_t *p, const uint64_t *d_idx, uint32_t n, const 
 {
     if (!p || !d_idx || !d_out) return PF_EINVAL;
     if (n == 0) return PF_OK;
+    if (int rc_dev = check_device(p)) return rc_dev;
     ReportArgs a;
     a.idx = d_idx; a.n = n; a.d_n = d_n; a.out = d_out; a.size = p->size; a.vals = p->d_vals; a.scen = p->d_scen;
     const unsigned grid = (n + 127) / 128;

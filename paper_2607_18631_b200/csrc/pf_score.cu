@@ -1008,6 +1008,7 @@ int pf::score_run(pf_plan_t *p, uint64_t first, uint64_t count, uint8_t *d_reaso
     if (first >= p->size || count > p->size - first) return PF_ERANGE;
     if (!d_workspace || ((uintptr_t)d_workspace & 255) != 0) return PF_EWORKSPACE;
     if (workspace_bytes < pf_score_workspace(p, count, k)) return PF_EWORKSPACE;
+    if (int rc_dev = check_device(p)) return rc_dev;
 
     uint64_t slab_lo, n_slabs;
     slab_span(p, first, count, slab_lo, n_slabs);
@@ -1152,8 +1153,9 @@ extern "C" int pf_score_static(pf_plan_t *p, uint64_t first, uint64_t count, uin
     if (count == 0 || count >= PF_MAX_COUNT) return PF_ERANGE;
     // refuse what the fixed array cannot hold before touching the device
     if (pf_score_workspace(p, count, k) > (size_t)PF_STATIC_SCRATCH_BYTES) return PF_EWORKSPACE;
-    int dev = -1;
-    PF_CUDA_TRY(cudaGetDevice(&dev), "pf_score_static: current device");
+    // the scratch that counts is the one on the plan's device, which must be the current one
+    if (int rc_dev = check_device(p)) return rc_dev;
+    const int dev = p->device;
     if (dev < 0 || dev >= kMaxDevices) return PF_EUNSUPPORTED;
     void *scratch = nullptr;
     {

@@ -132,6 +132,7 @@ extern "C" int pf_search(pf_plan_t *p, uint32_t k, uint64_t s_max, uint32_t k_si
         return PF_EINVAL;
     const WorkLayout w = work_layout(p, k, s_max, k_sim);
     if (!d_workspace || ((uintptr_t)d_workspace & 255) != 0 || workspace_bytes < w.total) return PF_EWORKSPACE;
+    if (int rc_dev = check_device(p)) return rc_dev;
     uint8_t *ws = (uint8_t *)d_workspace;
     return search_device(p, k, s_max, k_sim, jitter_seed, d_reason, d_tput, d_mem, d_topk_idx, d_topk_score,
                          d_topk_count, d_surv_idx, d_surv_count, d_sim_topk_idx, d_sim_topk_score, d_sim_topk_count,
@@ -152,6 +153,7 @@ extern "C" int pf_search_host(pf_plan_t *p, uint32_t k, uint64_t s_max, uint32_t
     if (sim && (k_sim < 1 || !h_sim_topk_idx || !h_sim_topk_score || !h_sim_topk_count)) return PF_EINVAL;
     const SearchLayout l = search_layout(p, k, s_max, k_sim);
     if (!d_workspace || ((uintptr_t)d_workspace & 255) != 0 || workspace_bytes < l.total) return PF_EWORKSPACE;
+    if (int rc_dev = check_device(p)) return rc_dev;
     cudaStream_t st = (cudaStream_t)stream;
     uint8_t *ws = (uint8_t *)d_workspace;
     const size_t N = (size_t)p->size;

@@ -566,6 +566,7 @@ int pf::select_run(pf_plan_t *p, uint64_t first, uint64_t count, const uint8_t *
     if (first >= p->size || count > p->size - first) return PF_ERANGE;
     const SelLayout lay = sel_layout(p, count);
     if (!d_workspace || ((uintptr_t)d_workspace & 255) != 0 || workspace_bytes < lay.total) return PF_EWORKSPACE;
+    if (int rc_dev = check_device(p)) return rc_dev;
     uint8_t *ws = (uint8_t *)d_workspace;
     SelArgs a;
     a.first = first; a.count = count; a.s_max = s_max; a.reason = d_reason; a.tput = d_tput;

@@ -1091,6 +1091,7 @@ int pf::simulate_run(pf_plan_t *p, const uint64_t *d_surv_idx, uint64_t n, const
     const SimLayout lay = sim_layout(p, n, k);
     if (!d_workspace || ((uintptr_t)d_workspace & 255) != 0 || workspace_bytes < lay.total) return PF_EWORKSPACE;
     if (!p->sim_tables) return PF_EINVAL;
+    if (int rc_dev = check_device(p)) return rc_dev;
     int rc = PF_OK;
     const SimTables *tab = (const SimTables *)p->sim_tables;
     uint8_t *ws = (uint8_t *)d_workspace;
