@@ -359,6 +359,43 @@ int pf_search_host(pf_plan_t *plan, uint32_t k, uint64_t s_max, uint32_t k_sim, 
                    uint32_t *h_sim_topk_count, uint64_t *h_surv_count, void *d_workspace,
                    size_t workspace_bytes, void *stream);
 
+/* A compact view of dense scoring outputs (the paper's search reports which plans pass and why the others fail,
+ * Sec. 3.3: "the pruned set is attributable"; in its spaces, as in this library's, a few candidates in ten thousand
+ * pass).  From d_reason / d_tput / d_mem of candidates [first, first+count), as pf_score wrote them:
+ *   d_hist[PF_REASON_BINS] uint64: candidates per reason code (entry 0: feasible, flagged ones included);
+ *   d_mask (may be NULL): ceil(count / 8) bytes, bit (i mod 8) of byte i / 8 set iff candidate first + i is feasible;
+ *   d_records[record_cap] (record_cap may be 0): the feasible candidates in ascending index order -- index,
+ *     peak bytes (0 when d_mem is NULL), tokens/s/GPU, reason byte (0 or PF_FLAG_EXTRAPOLATED); when more than
+ *     record_cap are feasible the first record_cap are written;
+ *   d_n_feasible[1] uint64: how many are feasible (compare with record_cap to detect a truncated list).
+ * d_workspace: pf_compact_workspace(count) bytes, 256-byte aligned.  Enqueues on `stream`, does not synchronize.
+ * Errors: PF_EINVAL, PF_ERANGE, PF_EWORKSPACE, PF_ECUDA. */
+#define PF_REASON_BINS 16
+typedef struct {
+    uint64_t idx;
+    int64_t mem;
+    float tput;
+    uint8_t reason, pad[3];
+} pf_record_t;
+size_t pf_compact_workspace(uint64_t count);
+int pf_compact(pf_plan_t *plan, uint64_t first, uint64_t count, const uint8_t *d_reason, const float *d_tput,
+               const int64_t *d_mem, uint64_t *d_hist, uint8_t *d_mask, pf_record_t *d_records, uint64_t record_cap,
+               uint64_t *d_n_feasible, void *d_workspace, size_t workspace_bytes, void *stream);
+
+/* pf_search_host with the compact view in place of the dense per-candidate arrays: what crosses the host link is
+ * the reason histogram (h_hist[PF_REASON_BINS]), the feasibility bits (h_mask, N / 8 bytes, may be NULL), the
+ * feasible plans' records (h_records[record_cap], may be NULL with record_cap 0) and their number (h_n_feasible),
+ * besides the two top-k lists -- on the 1.8e8-candidate space about 23 MB instead of 2.3 GB.
+ * d_workspace: pf_search_compact_workspace() bytes of DEVICE memory.  Returns after all copies have completed.
+ * Errors as pf_search_host. */
+size_t pf_search_compact_workspace(const pf_plan_t *plan, uint32_t k, uint64_t s_max, uint32_t k_sim,
+                                   uint64_t record_cap);
+int pf_search_host_compact(pf_plan_t *plan, uint32_t k, uint64_t s_max, uint32_t k_sim, uint32_t jitter_seed,
+                           uint64_t *h_hist, uint8_t *h_mask, pf_record_t *h_records, uint64_t record_cap,
+                           uint64_t *h_n_feasible, uint64_t *h_topk_idx, float *h_topk_score, uint32_t *h_topk_count,
+                           uint64_t *h_sim_topk_idx, float *h_sim_topk_score, uint32_t *h_sim_topk_count,
+                           uint64_t *h_surv_count, void *d_workspace, size_t workspace_bytes, void *stream);
+
 /* Extrapolation report for a list of plans, e.g. a top-k list (principle P4: a query outside the calibration
  * domain is flagged, not silently trusted).  Entry i of d_out describes plan d_idx[i]: its reason byte as pf_score
  * writes it, the PF_WHY_* bits behind an extrapolated flag, its tokens per expert and efficiency bucket (0 where

@@ -24,12 +24,12 @@ extern "C" {
  * PF_T_SCORE: the scoring kernel; PF_T_TOPK: top-k list kernels (merge passes, dense top-k);
  * PF_T_SELECT: the survivor-selection kernels; PF_T_SIMPREP: the simulator's pre-pass (binning, records);
  * PF_T_SIMULATE: the simulator kernel (inside pf_search it also streams the constant blocks of the dense outputs);
- * PF_T_AGGREGATE: the per-plan serving aggregate; PF_T_FILL: the stand-alone kernel that streams the constant
+ * PF_T_COMPACT: the kernels of pf_compact; PF_T_AGGREGATE: the per-plan serving aggregate; PF_T_FILL: the stand-alone kernel that streams the constant
  * blocks of the dense outputs inside pf_search when no simulator kernel runs to carry them.  Classes that run on different streams
  * overlap, so their times may add up to more than the call's. */
 enum {
     PF_T_SCORE = 0, PF_T_TOPK = 1, PF_T_SELECT = 2, PF_T_SIMULATE = 3, PF_T_AGGREGATE = 4, PF_T_FILL = 5,
-    PF_T_SIMPREP = 6, PF_T_CLASSES = 7
+    PF_T_SIMPREP = 6, PF_T_COMPACT = 7, PF_T_CLASSES = 8
 };
 int pf_timing_enable(pf_plan_t *plan, int on);
 int pf_timing_read(pf_plan_t *plan, float *ms, uint32_t *kernels);

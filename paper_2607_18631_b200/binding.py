@@ -24,11 +24,14 @@ EXPORTS = ("pf_version", "pf_strerror", "pf_reason_str", "pf_last_cuda_error", "
            "pf_plan_size", "pf_decode", "pf_score_workspace", "pf_score", "pf_topk_merge", "pf_select_workspace",
            "pf_select_survivors", "pf_simulate_workspace", "pf_simulate", "pf_search_workspace", "pf_search_host",
            "pf_dualpipe_order", "pf_score_static", "pf_serve_plan_count", "pf_aggregate_workspace", "pf_aggregate_serving",
-           "pf_report", "pf_search", "pf_search_device_workspace")
+           "pf_report", "pf_search", "pf_search_device_workspace", "pf_compact_workspace", "pf_compact",
+           "pf_search_compact_workspace", "pf_search_host_compact")
 # measurement hooks of include/planfront_bench.h that this library exports (the probes live in probes.py)
 BENCH_EXPORTS = ("pf_launch_count", "pf_timing_enable", "pf_timing_read")
 STATIC_SCRATCH_BYTES = 4 << 20
-T_CLASSES = ("score", "topk", "select", "simulate", "aggregate", "fill", "simprep")
+T_CLASSES = ("score", "topk", "select", "simulate", "aggregate", "fill", "simprep", "compact")
+REASON_BINS = 16
+RECORD_DTYPE = np.dtype([("idx", "<u8"), ("mem", "<i8"), ("tput", "<f4"), ("reason", "u1"), ("pad", "u1", (3,))])
 
 i32, u32, i64, u64, f32 = C.c_int32, C.c_uint32, C.c_int64, C.c_uint64, C.c_float
 
@@ -160,6 +163,14 @@ def load_library(path: str | None = None):
     L.pf_timing_read.argtypes = [vp, vp, vp]
     L.pf_dualpipe_order.restype = C.c_int
     L.pf_dualpipe_order.argtypes = [C.c_int, C.c_int, vp]
+    L.pf_compact_workspace.restype = sz
+    L.pf_compact_workspace.argtypes = [u64]
+    L.pf_compact.restype = C.c_int
+    L.pf_compact.argtypes = [vp, u64, u64, vp, vp, vp, vp, vp, vp, u64, vp, vp, sz, vp]
+    L.pf_search_compact_workspace.restype = sz
+    L.pf_search_compact_workspace.argtypes = [vp, u32, u64, u32, u64]
+    L.pf_search_host_compact.restype = C.c_int
+    L.pf_search_host_compact.argtypes = [vp, u32, u64, u32, u32, vp, vp, vp, u64] + [vp] * 8 + [vp, sz, vp]
     L.pf_search_device_workspace.restype = sz
     L.pf_search_device_workspace.argtypes = [vp, u32, u64, u32]
     L.pf_search.restype = C.c_int
@@ -456,6 +467,63 @@ class Plan:
                "pf_aggregate_serving")
         return dict(plan_reason=plan_reason, plan_tput=plan_tput, topk_idx=topk_idx, topk_score=topk_score,
                     topk_count=topk_count, workspace=workspace)
+
+    # ---- pf_compact
+    def compact(self, reason, tput, mem, record_cap: int, first: int = 0, want_mask: bool = True, stream=None):
+        """Enqueue pf_compact on dense outputs of candidates [first, first + len(reason)).  Returns device tensors:
+        hist (int64[16]), mask (uint8[ceil(count / 8)] or None), records (uint8 view of record_cap records),
+        n_feasible (int64[1]).  Does not synchronize."""
+        torch = _torch()
+        dev, count = self.device, reason.numel()
+        hist = torch.empty(REASON_BINS, dtype=torch.int64, device=dev)
+        mask = torch.empty((count + 7) // 8, dtype=torch.uint8, device=dev) if want_mask else None
+        records = torch.empty(max(record_cap, 1) * RECORD_DTYPE.itemsize, dtype=torch.uint8, device=dev)
+        n_feas = torch.empty(1, dtype=torch.int64, device=dev)
+        ws = torch.empty(int(self._L.pf_compact_workspace(count)), dtype=torch.uint8, device=dev)
+        _check(self._L.pf_compact(self._h, first, count, _dptr(reason), _dptr(tput), _dptr(mem), _dptr(hist),
+                                  _dptr(mask), _dptr(records), record_cap, _dptr(n_feas), _dptr(ws), ws.numel(),
+                                  _stream_ptr(torch, stream)), "pf_compact")
+        return dict(hist=hist, mask=mask, records=records, n_feasible=n_feas, workspace=ws)
+
+    @staticmethod
+    def records_to_numpy(records, n: int):
+        return records.cpu().numpy()[:n * RECORD_DTYPE.itemsize].view(RECORD_DTYPE)
+
+    # ---- pf_search_host_compact
+    def search_compact_workspace(self, k: int, s_max: int, k_sim: int, record_cap: int) -> int:
+        return int(self._L.pf_search_compact_workspace(self._h, k, s_max, k_sim, record_cap))
+
+    def search_host_compact(self, k: int, s_max: int, k_sim: int, jitter_seed: int, workspace, record_cap: int,
+                            h_mask=None, h_records=None, stream=None):
+        """pf_search_host_compact: the whole search with the compact view as the per-candidate result.  h_mask
+        (uint8[N / 8]) and h_records (RECORD_DTYPE[record_cap]) may be numpy arrays or pinned torch tensors (bytes);
+        both optional.  Returns a dict of numpy results; synchronous."""
+        torch = _torch()
+
+        def hptr(x):
+            if x is None:
+                return None
+            return C.c_void_p(x.data_ptr()) if hasattr(x, "data_ptr") else x.ctypes.data_as(C.c_void_p)
+        if record_cap > 0 and h_records is None:
+            h_records = np.empty(record_cap, dtype=RECORD_DTYPE)
+        hist = np.zeros(REASON_BINS, dtype=np.uint64)
+        nfeas = np.zeros(1, dtype=np.uint64)
+        ti = np.empty(max(k, 1), dtype=np.uint64)
+        ts = np.empty(max(k, 1), dtype=np.float32)
+        tc = np.zeros(1, dtype=np.uint32)
+        si = np.empty(max(k_sim, 1), dtype=np.uint64)
+        ss = np.empty(max(k_sim, 1), dtype=np.float32)
+        sc = np.zeros(1, dtype=np.uint32)
+        nsurv = np.zeros(1, dtype=np.uint64)
+        _check(self._L.pf_search_host_compact(self._h, k, s_max, k_sim, jitter_seed, hptr(hist), hptr(h_mask),
+                                              hptr(h_records), record_cap, hptr(nfeas), hptr(ti), hptr(ts), hptr(tc),
+                                              hptr(si), hptr(ss), hptr(sc), hptr(nsurv), _dptr(workspace),
+                                              workspace.numel(), _stream_ptr(torch, stream)),
+               "pf_search_host_compact")
+        n_rec = int(min(int(nfeas[0]), record_cap))
+        return dict(hist=hist, n_feasible=int(nfeas[0]), n_records=n_rec, mask=h_mask, records=h_records,
+                    topk_idx=ti[:tc[0]], topk_score=ts[:tc[0]], sim_topk_idx=si[:sc[0]], sim_topk_score=ss[:sc[0]],
+                    n_survivors=int(nsurv[0]))
 
     # ---- pf_search_host
     def search_workspace(self, k: int, s_max: int, k_sim: int) -> int:

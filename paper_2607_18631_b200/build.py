@@ -8,7 +8,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(HERE, "libplanfront.so")
-SOURCES = ["pf_api.cu", "pf_score.cu", "pf_select.cu", "pf_simulate.cu", "pf_search.cu", "pf_aggregate.cu", "pf_report.cu"]
+SOURCES = ["pf_api.cu", "pf_score.cu", "pf_select.cu", "pf_simulate.cu", "pf_search.cu", "pf_aggregate.cu", "pf_report.cu", "pf_compact.cu"]
 # the roofline probes of the benchmark: a library of their own, not part of the scoring ABI
 PROBE_LIB = os.path.join(HERE, "libplanfront_probe.so")
 PROBE_SOURCES = ["pf_probe.cu"]

@@ -192,3 +192,105 @@ extern "C" int pf_search_host(pf_plan_t *p, uint32_t k, uint64_t s_max, uint32_t
     PF_CUDA_TRY(cudaStreamSynchronize(st), "pf_search_host: synchronize");
     return PF_OK;
 }
+
+// ------------------------------------------------------------------ host buffers, compact results
+
+namespace pf {
+struct CompactSearchLayout {
+    SearchLayout base;
+    size_t off_hist, off_nfeas, off_mask, off_records, off_cws, cws_bytes, total;
+};
+static CompactSearchLayout compact_search_layout(const pf_plan_t *p, uint32_t k, uint64_t s_max, uint32_t k_sim,
+                                                 uint64_t record_cap)
+{
+    CompactSearchLayout l;
+    l.base = search_layout(p, k, s_max, k_sim);
+    size_t o = l.base.total;
+    l.off_hist = o; o += 256;
+    l.off_nfeas = o; o += 256;
+    l.off_mask = o; o += align256(((size_t)p->size + 7) / 8);
+    l.off_records = o; o += align256((size_t)(record_cap ? record_cap : 1) * sizeof(pf_record_t));
+    l.off_cws = o;
+    l.cws_bytes = align256(pf_compact_workspace(p->size));
+    l.total = o + l.cws_bytes;
+    return l;
+}
+}  // namespace pf
+
+extern "C" size_t pf_search_compact_workspace(const pf_plan_t *p, uint32_t k, uint64_t s_max, uint32_t k_sim,
+                                              uint64_t record_cap)
+{
+    if (!p) return 0;
+    return compact_search_layout(p, k, s_max, k_sim, record_cap).total;
+}
+
+extern "C" int pf_search_host_compact(pf_plan_t *p, uint32_t k, uint64_t s_max, uint32_t k_sim, uint32_t jitter_seed,
+                                      uint64_t *h_hist, uint8_t *h_mask, pf_record_t *h_records, uint64_t record_cap,
+                                      uint64_t *h_n_feasible, uint64_t *h_topk_idx, float *h_topk_score,
+                                      uint32_t *h_topk_count, uint64_t *h_sim_topk_idx, float *h_sim_topk_score,
+                                      uint32_t *h_sim_topk_count, uint64_t *h_surv_count, void *d_workspace,
+                                      size_t workspace_bytes, void *stream)
+{
+    if (!p) return PF_EINVAL;
+    if (k < 1 || k > PF_K_MAX || k_sim > PF_K_MAX) return PF_EINVAL;
+    if (!h_hist || !h_n_feasible || !h_topk_idx || !h_topk_score || !h_topk_count) return PF_EINVAL;
+    if (record_cap > 0 && !h_records) return PF_EINVAL;
+    if (p->size >= PF_MAX_COUNT) return PF_ERANGE;
+    const bool sim = s_max > 0 && p->dev.phase == PF_PHASE_TRAIN;
+    if (sim && (k_sim < 1 || !h_sim_topk_idx || !h_sim_topk_score || !h_sim_topk_count)) return PF_EINVAL;
+    const CompactSearchLayout cl = compact_search_layout(p, k, s_max, k_sim, record_cap);
+    const SearchLayout &l = cl.base;
+    if (!d_workspace || ((uintptr_t)d_workspace & 255) != 0 || workspace_bytes < cl.total) return PF_EWORKSPACE;
+    if (int rc_dev = check_device(p)) return rc_dev;
+    cudaStream_t st = (cudaStream_t)stream;
+    uint8_t *ws = (uint8_t *)d_workspace;
+    const size_t N = (size_t)p->size;
+    uint8_t *d_reason = ws + l.off_reason;
+    float *d_tput = (float *)(ws + l.off_tput);
+    int64_t *d_mem = record_cap ? (int64_t *)(ws + l.off_mem) : nullptr;   // only the records carry it
+    uint64_t *d_tk_idx = (uint64_t *)(ws + l.off_topk_idx);
+    float *d_tk_sc = (float *)(ws + l.off_topk_score);
+    uint32_t *d_tk_cnt = (uint32_t *)(ws + l.off_topk_count);
+    uint64_t *d_surv = (uint64_t *)(ws + l.off_surv);
+    uint64_t *d_surv_cnt = (uint64_t *)(ws + l.off_surv_count);
+    uint64_t *d_sim_idx = (uint64_t *)(ws + l.off_sim_idx);
+    float *d_sim_sc = (float *)(ws + l.off_sim_score);
+    uint32_t *d_sim_cnt = (uint32_t *)(ws + l.off_sim_count);
+    uint64_t *d_hist = (uint64_t *)(ws + cl.off_hist), *d_nfeas = (uint64_t *)(ws + cl.off_nfeas);
+    uint8_t *d_mask = h_mask ? ws + cl.off_mask : nullptr;
+    pf_record_t *d_records = (pf_record_t *)(ws + cl.off_records);
+    int rc = search_device(p, k, s_max, k_sim, jitter_seed, d_reason, d_tput, d_mem, d_tk_idx, d_tk_sc, d_tk_cnt,
+                           d_surv, d_surv_cnt, d_sim_idx, d_sim_sc, d_sim_cnt, ws + l.off_ws, l.ws_bytes,
+                           ws + l.off_ws_sel, l.ws_sel_bytes, st);
+    if (rc != PF_OK) return rc;
+    rc = pf_compact(p, 0, N, d_reason, d_tput, d_mem, d_hist, d_mask, d_records, record_cap, d_nfeas, ws + cl.off_cws,
+                    cl.cws_bytes, stream);
+    if (rc != PF_OK) return rc;
+    PF_CUDA_TRY(cudaMemcpyAsync(h_hist, d_hist, PF_REASON_BINS * 8, cudaMemcpyDeviceToHost, st), "copy histogram");
+    PF_CUDA_TRY(cudaMemcpyAsync(h_n_feasible, d_nfeas, 8, cudaMemcpyDeviceToHost, st), "copy count");
+    if (h_mask) PF_CUDA_TRY(cudaMemcpyAsync(h_mask, d_mask, (N + 7) / 8, cudaMemcpyDeviceToHost, st), "copy mask");
+    PF_CUDA_TRY(cudaMemcpyAsync(h_topk_idx, d_tk_idx, (size_t)k * 8, cudaMemcpyDeviceToHost, st), "copy top-k");
+    PF_CUDA_TRY(cudaMemcpyAsync(h_topk_score, d_tk_sc, (size_t)k * 4, cudaMemcpyDeviceToHost, st), "copy top-k");
+    PF_CUDA_TRY(cudaMemcpyAsync(h_topk_count, d_tk_cnt, 4, cudaMemcpyDeviceToHost, st), "copy top-k");
+    if (sim) {
+        PF_CUDA_TRY(cudaMemcpyAsync(h_sim_topk_idx, d_sim_idx, (size_t)k_sim * 8, cudaMemcpyDeviceToHost, st), "copy sim");
+        PF_CUDA_TRY(cudaMemcpyAsync(h_sim_topk_score, d_sim_sc, (size_t)k_sim * 4, cudaMemcpyDeviceToHost, st), "copy sim");
+        PF_CUDA_TRY(cudaMemcpyAsync(h_sim_topk_count, d_sim_cnt, 4, cudaMemcpyDeviceToHost, st), "copy sim");
+        if (h_surv_count)
+            PF_CUDA_TRY(cudaMemcpyAsync(h_surv_count, d_surv_cnt, 8, cudaMemcpyDeviceToHost, st), "copy count");
+    } else {
+        if (h_sim_topk_count) *h_sim_topk_count = 0;
+        if (h_surv_count) *h_surv_count = 0;
+    }
+    // the record count decides how many records travel: wait for it, then copy exactly those
+    PF_CUDA_TRY(cudaStreamSynchronize(st), "pf_search_host_compact: synchronize");
+    if (record_cap > 0) {
+        const uint64_t n = *h_n_feasible < record_cap ? *h_n_feasible : record_cap;
+        if (n > 0) {
+            PF_CUDA_TRY(cudaMemcpyAsync(h_records, d_records, (size_t)n * sizeof(pf_record_t), cudaMemcpyDeviceToHost, st),
+                        "copy records");
+            PF_CUDA_TRY(cudaStreamSynchronize(st), "pf_search_host_compact: synchronize");
+        }
+    }
+    return PF_OK;
+}

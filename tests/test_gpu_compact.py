@@ -1,0 +1,93 @@
+"""The compact view of dense scoring outputs (pf_compact, pf_search_host_compact) against the oracle: the reason
+histogram is the bincount of the oracle's reason codes, the mask its feasibility bits, the records its feasible set
+in ascending index order with its scores and byte counts."""
+from __future__ import annotations
+
+import numpy as np
+import pytest
+
+from oracle import Oracle
+from workloads import make_config
+
+from helpers import TPUT_RTOL, check_topk, variant
+
+pytestmark = pytest.mark.gpu
+
+
+def _plan(cfg):
+    from paper_2607_18631_b200 import Plan
+    return Plan(cfg)
+
+
+def _check_view(hist, mask, recs, n_feasible, o_reason, o_tput, o_mem, first):
+    count = len(o_reason)
+    np.testing.assert_array_equal(hist[:12].astype(np.int64), np.bincount(o_reason & 0x7F, minlength=12)[:12])
+    assert np.all(hist[12:] == 0)
+    feas = (o_reason & 0x7F) == 0
+    assert n_feasible == int(feas.sum())
+    if mask is not None:
+        bits = np.unpackbits(np.asarray(mask, dtype=np.uint8), bitorder="little")[:count].astype(bool)
+        np.testing.assert_array_equal(bits, feas)
+        assert not np.unpackbits(np.asarray(mask, dtype=np.uint8), bitorder="little")[count:].any()
+    if recs is not None:
+        want = np.flatnonzero(feas)[:len(recs)]
+        np.testing.assert_array_equal(recs["idx"].astype(np.int64), want + first)
+        np.testing.assert_array_equal(recs["mem"], o_mem[want])
+        np.testing.assert_array_equal(recs["reason"], o_reason[want])
+        np.testing.assert_allclose(recs["tput"], o_tput[want], rtol=TPUT_RTOL, atol=0)
+
+
+@pytest.mark.parametrize("name,first,count", [("tiny", 0, None), ("mid", 0, None), ("mid", 1003, 70_001),
+                                              ("serve", 16, 500_000)])
+def test_compact_view_matches_the_oracle(name, first, count):
+    import torch
+    cfg = variant(name, cluster=dict(budget_bytes=10 ** 15)) if name == "mid" else make_config(name)
+    plan, orc = _plan(cfg), Oracle(cfg)
+    count = plan.size - first if count is None else count
+    out = plan.score(first=first, count=count, k=0)
+    o_reason, o_tput, o_mem, _ = orc.score_range(first, count, threads=8)
+    n_feas = int(((o_reason & 0x7F) == 0).sum())
+    for cap in (n_feas + 5, max(n_feas // 3, 1), 0):
+        c = plan.compact(out["reason"], out["tput"], out["mem"], cap, first=first)
+        torch.cuda.synchronize()
+        n = int(c["n_feasible"].item())
+        recs = plan.records_to_numpy(c["records"], min(n, cap)) if cap else None
+        _check_view(c["hist"].cpu().numpy().astype(np.uint64), c["mask"].cpu().numpy(), recs, n, o_reason, o_tput,
+                    o_mem, first)
+    # without the mask and without the memory array
+    c = plan.compact(out["reason"], out["tput"], None, n_feas, first=first, want_mask=False)
+    torch.cuda.synchronize()
+    recs = plan.records_to_numpy(c["records"], n_feas)
+    assert np.all(recs["mem"] == 0)
+    plan.close()
+
+
+def test_search_host_compact_on_the_large_space():
+    """The whole search through host buffers with the compact view: the 1.8e8-candidate space comes back as a
+    histogram, 22.5 MB of feasibility bits and 12,905 records instead of 2.3 GB of dense arrays."""
+    import torch
+    cfg = make_config("large")
+    plan, orc = _plan(cfg), Oracle(cfg)
+    N = plan.size
+    cap = 100_000
+    ws = torch.empty(plan.search_compact_workspace(1024, 10 ** 6, 100, cap), dtype=torch.uint8, device="cuda")
+    h_mask = np.empty((N + 7) // 8, dtype=np.uint8)
+    r = plan.search_host_compact(1024, 10 ** 6, 100, 4, ws, cap, h_mask=h_mask)
+    o_reason, o_tput, o_mem, _ = orc.score_range(threads=64)
+    assert r["n_records"] == r["n_feasible"] == 12_905
+    _check_view(r["hist"], r["mask"], r["records"][:r["n_records"]], r["n_feasible"], o_reason, o_tput, o_mem, 0)
+    idx, sc = orc.topk(o_reason, o_tput, 0, 1024)
+    check_topk(r["topk_idx"], r["topk_score"], idx, sc)
+    surv = orc.select_survivors(o_reason, o_tput, 0, 10 ** 6)
+    assert r["n_survivors"] == len(surv)
+    ref, _, _ = orc.simulate_list(surv, 4, threads=64)
+    ref_idx, ref_sc = Oracle.topk_list(surv, ref, 100)
+    check_topk(r["sim_topk_idx"], r["sim_topk_score"], ref_idx, ref_sc)
+    # records and mask are optional, and a short record buffer is filled from the front
+    r2 = plan.search_host_compact(1024, 10 ** 6, 100, 4, ws, 1000)
+    assert r2["n_feasible"] == 12_905 and r2["n_records"] == 1000
+    np.testing.assert_array_equal(r2["records"][:1000]["idx"], r["records"][:1000]["idx"])
+    np.testing.assert_array_equal(r2["hist"], r["hist"])
+    r3 = plan.search_host_compact(1024, 10 ** 6, 100, 4, ws, 0)
+    assert r3["n_feasible"] == 12_905 and r3["records"] is None
+    plan.close()
