@@ -37,6 +37,13 @@ int pf_timing_read(pf_plan_t *plan, float *ms, uint32_t *kernels);
 /* Number of kernels this library has launched in this process (for launch accounting in benchmarks). */
 uint64_t pf_launch_count(void);
 
+/* How the plan's latest scoring call inside pf_search was divided between the scoring kernel and the kernel that
+ * streams constant blocks: the number of blocks of candidates the call's range was cut into, candidates per block,
+ * and how many blocks the scoring kernel took itself (the evaluated ones and the constant ones interleaved with
+ * them); the rest went to the fill kernel.  Reads a few words back from the device (synchronizes the device).
+ * Errors: PF_EINVAL (NULL pointer, or the plan has no such record), PF_ECUDA. */
+int pf_bench_fill_span(pf_plan_t *plan, uint64_t *n_blocks, uint64_t *block_candidates, uint64_t *scored_blocks);
+
 /* Roofline probes (libplanfront_probe.so).
  * The caller times them with events on `stream`; neither call synchronises or allocates.
  *

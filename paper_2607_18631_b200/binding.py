@@ -27,7 +27,7 @@ EXPORTS = ("pf_version", "pf_strerror", "pf_reason_str", "pf_last_cuda_error", "
            "pf_report", "pf_search", "pf_search_device_workspace", "pf_compact_workspace", "pf_compact",
            "pf_search_compact_workspace", "pf_search_host_compact")
 # measurement hooks of include/planfront_bench.h that this library exports (the probes live in probes.py)
-BENCH_EXPORTS = ("pf_launch_count", "pf_timing_enable", "pf_timing_read")
+BENCH_EXPORTS = ("pf_launch_count", "pf_timing_enable", "pf_timing_read", "pf_bench_fill_span")
 STATIC_SCRATCH_BYTES = 4 << 20
 T_CLASSES = ("score", "topk", "select", "simulate", "aggregate", "fill", "simprep", "compact")
 REASON_BINS = 16
@@ -161,6 +161,8 @@ def load_library(path: str | None = None):
     L.pf_timing_enable.argtypes = [vp, C.c_int]
     L.pf_timing_read.restype = C.c_int
     L.pf_timing_read.argtypes = [vp, vp, vp]
+    L.pf_bench_fill_span.restype = C.c_int
+    L.pf_bench_fill_span.argtypes = [vp, C.POINTER(u64), C.POINTER(u64), C.POINTER(u64)]
     L.pf_dualpipe_order.restype = C.c_int
     L.pf_dualpipe_order.argtypes = [C.c_int, C.c_int, vp]
     L.pf_compact_workspace.restype = sz
@@ -303,6 +305,12 @@ class Plan:
     # ---- pf_timing_enable / pf_timing_read
     def timing_enable(self, on: bool = True):
         _check(self._L.pf_timing_enable(self._h, 1 if on else 0), "pf_timing_enable")
+
+    def fill_span(self) -> dict:
+        """pf_bench_fill_span: how the latest pf_search split the space between the scoring and the fill kernel."""
+        a, b, c = u64(0), u64(0), u64(0)
+        _check(self._L.pf_bench_fill_span(self._h, C.byref(a), C.byref(b), C.byref(c)), "pf_bench_fill_span")
+        return dict(n_blocks=int(a.value), block_candidates=int(b.value), scored_blocks=int(c.value))
 
     def timing_read(self) -> dict:
         """{class: (milliseconds, kernels)} accumulated since the last read; waits for the recorded events."""

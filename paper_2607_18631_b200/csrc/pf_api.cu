@@ -499,6 +499,19 @@ extern "C" int pf_timing_read(pf_plan_t *p, float *ms, uint32_t *kernels)
     return PF_OK;
 }
 
+extern "C" int pf_bench_fill_span(pf_plan_t *p, uint64_t *n_blocks, uint64_t *block_candidates, uint64_t *scored_blocks)
+{
+    if (!p || !n_blocks || !block_candidates || !scored_blocks || !p->d_order) return PF_EINVAL;
+    if (int rc_dev = pf::check_device(p)) return rc_dev;
+    uint32_t hdr[8] = {0};
+    PF_CUDA_TRY(cudaDeviceSynchronize(), "pf_bench_fill_span");
+    PF_CUDA_TRY(cudaMemcpy(hdr, p->d_order, sizeof(hdr), cudaMemcpyDeviceToHost), "pf_bench_fill_span");
+    *n_blocks = hdr[2];
+    *block_candidates = p->dev.slab;
+    *scored_blocks = hdr[4];
+    return PF_OK;
+}
+
 extern "C" void pf_plan_destroy(pf_plan_t *p)
 {
     if (!p) return;

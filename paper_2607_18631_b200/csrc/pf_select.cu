@@ -98,7 +98,7 @@ __device__ __forceinline__ uint32_t feasible_mask16(uint4 r)
 // f(rel, score_bits).
 template <typename F>
 __device__ __forceinline__ void for_each_eligible16(const DevPlan &P, const int32_t *vals, const SelArgs &A,
-                                                    uint64_t e, const uint4 r, F f)
+                                                    const uint8_t *cls, uint64_t e, const uint4 r, F f)
 {
     // any byte with its low 7 bits clear?  (zero-byte test on the masked words; most groups have none)
     const uint32_t x0 = r.x & 0x7F7F7F7Fu, x1 = r.y & 0x7F7F7F7Fu, x2 = r.z & 0x7F7F7F7Fu, x3 = r.w & 0x7F7F7F7Fu;
@@ -106,13 +106,19 @@ __device__ __forceinline__ void for_each_eligible16(const DevPlan &P, const int3
                        ((x3 - 0x01010101u) & ~x3);
     if ((z & 0x80808080u) == 0) return;
     uint32_t m = feasible_mask16(r);
-    const uint8_t *cls = sel_guard_cls(A);
+    if (cls) {
+        // bytes of a slab that is still being filled are not results yet: keep the candidates of evaluated slabs
+        // (class byte 0) only.  The sixteen candidates lie in one slab or straddle one boundary.
+        const uint64_t abs0 = A.first + e, s0 = abs0 / A.guard.slab;
+        const uint32_t in0 = (uint32_t)min((uint64_t)16, (s0 + 1) * A.guard.slab - abs0);   // candidates in slab s0
+        const uint64_t rel_s = s0 - A.guard.slab_lo;
+        if (cls[rel_s] != 0) m &= ~((1u << in0) - 1u);
+        if (in0 < 16u && (m >> in0) != 0u && rel_s + 1 < A.guard.n_slabs && cls[rel_s + 1] != 0) m &= (1u << in0) - 1u;
+    }
     while (m) {
         int i = __ffs(m) - 1;
         m &= m - 1;
         uint64_t rel = e + i;
-        // a byte of a slab that is still being filled is not a result yet
-        if (cls && cls[(A.first + rel) / A.guard.slab - A.guard.slab_lo] != 0) continue;
         if (in_sim_domain(P, vals, A.first + rel)) f(rel, __float_as_uint(__ldg(A.tput + rel)));
     }
 }
@@ -137,6 +143,7 @@ __device__ __forceinline__ void sel_hist_chunk(const DevPlan &P, const SelArgs &
 {
     const uint64_t lo = (uint64_t)chunk * A.chunk;
     const uint64_t hi = min(lo + A.chunk, A.count);
+    const uint8_t *cls = sel_guard_cls(A);
     if (pass == 0) {
         if (threadIdx.x == 0) *s_elig = 0;
         __syncthreads();
@@ -148,7 +155,7 @@ __device__ __forceinline__ void sel_hist_chunk(const DevPlan &P, const SelArgs &
 #pragma unroll
     for (int t = 0; t < kSelTiles; t++) {
         const uint64_t e = lo + (uint64_t)t * kSelTile + (uint64_t)threadIdx.x * 16;
-        for_each_eligible16(P, vals, A, e, r[t], [&](uint64_t, uint32_t bits) {
+        for_each_eligible16(P, vals, A, cls, e, r[t], [&](uint64_t, uint32_t bits) {
             if (pass == 0) {
                 atomicAdd(A.hist1 + (bits >> 16), 1u);
                 atomicAdd(A.coarse1 + (bits >> 24), 1u);
@@ -293,6 +300,7 @@ __global__ void __launch_bounds__(kSelThreads) sel_count_kernel(const __grid_con
     const unsigned int n_list = A.ctrl->n_elig;
     const bool all = A.ctrl->take_all != 0;
     const uint32_t thr = A.ctrl->thr_bits;
+    const uint8_t *cls = sel_guard_cls(A);
     for (unsigned int li = blockIdx.x; li < n_list; li += gridDim.x) {
         const unsigned int chunk = A.elig_list[li];
         if (all) {   // every eligible candidate is taken: the first pass has counted them already
@@ -312,7 +320,7 @@ __global__ void __launch_bounds__(kSelThreads) sel_count_kernel(const __grid_con
 #pragma unroll
         for (int t = 0; t < kSelTiles; t++) {
             const uint64_t e = lo + (uint64_t)t * kSelTile + (uint64_t)threadIdx.x * 16;
-            for_each_eligible16(P, vals, A, e, r[t], [&](uint64_t, uint32_t bits) {
+            for_each_eligible16(P, vals, A, cls, e, r[t], [&](uint64_t, uint32_t bits) {
                 if (bits > thr) gt++;
                 else if (bits == thr) eq++;
             });
@@ -419,6 +427,7 @@ __device__ __forceinline__ void sel_write_chunk(const DevPlan &P, const SelArgs 
     const uint32_t thr = A.ctrl->thr_bits;
     const bool all = A.ctrl->take_all != 0;
     const unsigned long long need_eq = all ? 0ull : A.ctrl->need_eq;
+    const uint8_t *cls = sel_guard_cls(A);
     if (tid == 0) {
         s_run_gt = A.blk_gt[chunk];
         s_run_eq = A.blk_eq[chunk];
@@ -430,7 +439,7 @@ __device__ __forceinline__ void sel_write_chunk(const DevPlan &P, const SelArgs 
     for (int t = 0; t < kSelTiles; t++) {
         const uint64_t e = lo + (uint64_t)t * kSelTile + (uint64_t)tid * 16;
         unsigned int gt = 0, eq = 0;
-        for_each_eligible16(P, vals, A, e, r[t], [&](uint64_t, uint32_t bits) {
+        for_each_eligible16(P, vals, A, cls, e, r[t], [&](uint64_t, uint32_t bits) {
             if (all || bits > thr) gt++;
             else if (bits == thr) eq++;
         });
@@ -457,7 +466,7 @@ __device__ __forceinline__ void sel_write_chunk(const DevPlan &P, const SelArgs 
         unsigned long long my_gt = s_run_gt + ((x >> 16) - gt);
         unsigned long long my_eq = s_run_eq + ((x & 0xFFFFu) - eq);
         if (gt | eq)
-            for_each_eligible16(P, vals, A, e, r[t], [&](uint64_t rel, uint32_t bits) {
+            for_each_eligible16(P, vals, A, cls, e, r[t], [&](uint64_t rel, uint32_t bits) {
                 if (all || bits > thr) {
                     unsigned long long pos = my_gt + (my_eq < need_eq ? my_eq : need_eq);
                     A.surv_idx[pos] = A.first + rel;
