@@ -10,6 +10,8 @@ line.
 
 N > 1 (launched under torch.distributed.run): every rank scores an independent space of the same shape
 (tables re-drawn from seed = rank); no data-path collective; value = all ranks' candidates / max time.
+With --split the ranks share ONE space instead (contiguous index slices, strong scaling): the selection's
+histograms are all-reduced and the top-k lists all-gathered over NCCL (paper_2607_18631_b200/sharding.py).
 
 --impl reference times the CPU oracle (fp64, OpenMP over the host cores) on the same workload.
 """
@@ -371,6 +373,60 @@ def _config_lines(torch, stream, hbm, peaks):
     return out
 
 
+def run_split(args, torch, dist, world, rank, local):
+    """--split: ONE space cut into contiguous slices over the ranks (strong scaling).  A step is sharded_search:
+    every rank scores and selects inside its slice, the selection's histograms are all-reduced so that the cut to the
+    s_max best is exact across ranks, each rank simulates its own survivors, the top-k lists are all-gathered and
+    folded.  The collectives are NCCL's through torch.distributed; one small device-to-host read per step (the cut)
+    sits inside the timed region."""
+    from paper_2607_18631_b200 import Plan, binding
+    from paper_2607_18631_b200.sharding import CudaOps, sharded_search, shard_range
+    cfg = make_config("large")
+    plan = Plan(cfg)
+    ops = CudaOps(plan)
+    N = plan.size
+    stream = torch.cuda.current_stream()
+
+    def step():
+        return sharded_search(ops, K_TOP, S_MAX, K_SIM, JITTER_SEED)
+
+    for _ in range(max(args.warmup, 3)):
+        r = step()
+    dist.barrier()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local)
+    launches0 = binding.pf_launch_count()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler.start()
+    dist.barrier()
+    torch.cuda.synchronize()
+    ev0.record(stream)
+    for _ in range(args.steps):
+        r = step()
+    ev1.record(stream)
+    torch.cuda.synchronize()
+    dist.barrier()
+    clocks = sampler.stop()
+    t = torch.tensor([ev0.elapsed_time(ev1)], dtype=torch.float64, device=plan.device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_step = float(t.item()) / args.steps
+    launches = binding.pf_launch_count() - launches0
+    if rank == 0:
+        first, count = shard_range(N, 0, world)
+        cfgd = workload_config(world, count)
+        cfgd["parallelism"] = f"one space split over {world} rank(s): contiguous index slices"
+        line = {"metric": METRIC, "value": N / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True,
+                "scaling": "strong", "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": cfgd,
+                "survivors": r["n_survivors_total"], "clocks": clocks, "gpu_launches": int(launches),
+                "collectives_per_step": {"all_reduce": 2, "all_reduce_bytes": 2 * 65536 * 8, "all_gather": 8,
+                                         "all_gather_bytes_per_rank": (K_TOP + K_SIM) * 12 + 8 + 16},
+                "note": "host-driven: per step one device-to-host read of the cut (48 bytes) sits between the "
+                        "selection's passes; dense outputs and survivor lists stay on their ranks"}
+        print(json.dumps(line))
+    dist.destroy_process_group()
+
+
 def run_ours(args):
     import torch
     from paper_2607_18631_b200 import Plan, binding
@@ -380,9 +436,13 @@ def run_ours(args):
         raise SystemExit("bench.py: no CUDA device (the scoring path has no CPU fallback)")
     torch.cuda.set_device(local)
     dist = None
-    if world > 1:
+    if world > 1 or args.split:
         import torch.distributed as dist
+        if "MASTER_ADDR" not in os.environ:          # a single process asked for the split path
+            os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT="29531", RANK="0", WORLD_SIZE="1")
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    if args.split:
+        return run_split(args, torch, dist, world, rank, local)
 
     def barrier():
         if dist is not None:
@@ -644,6 +704,8 @@ def main():
     ap.add_argument("--no-configs", action="store_true", help="skip the per-config lines")
     ap.add_argument("--no-sustained", action="store_true", help="skip the two-second sustained region")
     ap.add_argument("--no-dense-e2e", action="store_true", help="skip the dense-output end-to-end leg")
+    ap.add_argument("--split", action="store_true",
+                    help="one space split over the ranks (strong scaling) instead of one space per rank")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

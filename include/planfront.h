@@ -285,6 +285,41 @@ int pf_select_survivors(pf_plan_t *plan, uint64_t first, uint64_t count, const u
                         const float *d_tput, uint64_t s_max, uint64_t *d_surv_idx, uint64_t *d_surv_count,
                         void *d_workspace, size_t workspace_bytes, void *stream);
 
+/* The same selection in steps, for one space split over several GPUs (candidates are independent, so a rank scores
+ * and selects inside a contiguous slice of the index range; only histograms and counts travel).  With ranks
+ * r = 0..G-1 holding slices in ascending index order:
+ *   1. every rank: pf_select_hist(..., d_cut = NULL, d_hist): 65,536-bin histogram of the HIGH 16 bits of the fp32
+ *      score of its eligible candidates; the caller sums the ranks' histograms (as 64-bit counts);
+ *   2. pf_select_cut(sum, level 0, s_max, d_cut): the bin in which the running count from the top reaches s_max
+ *      (or take_all when no more than s_max are eligible in all);
+ *   3. every rank: pf_select_hist(..., d_cut, d_hist): histogram of the LOW 16 bits inside that bin; summed again;
+ *   4. pf_select_cut(sum, level 1, 0, d_cut): the threshold score bits, how many candidates lie above it and how
+ *      many of those exactly AT it are still needed (need_eq) -- taken in ascending index order, i.e. rank by rank;
+ *   5. every rank: pf_select_write(..., d_cut, eq_before, ...) with eq_before = the number of candidates at the
+ *      threshold on lower ranks (each rank's count is entry thr_bits & 0xFFFF of its own step-3 histogram): its
+ *      survivors in ascending index order.  The ranks' lists, concatenated in rank order, are what
+ *      pf_select_survivors returns for the whole space.  d_surv_idx holds surv_cap entries (a slice yields at most
+ *      min(count, s_max)); *d_surv_count is the slice's full count even when it exceeds surv_cap.
+ * Every call is self-contained (d_workspace: pf_select_workspace bytes, contents ignored).  d_hist: uint32[65536];
+ * the sums passed to pf_select_cut: uint64[65536].  Errors as pf_select_survivors. */
+typedef struct {
+    uint64_t total;      /* eligible candidates in all */
+    uint64_t above_hi;   /* eligible with high score bits above bin_hi */
+    uint64_t n_gt;       /* eligible with score bits above the threshold */
+    uint64_t need_eq;    /* candidates exactly at the threshold that are taken (smallest indices first) */
+    uint64_t target;     /* min(s_max, total) once both levels are done: s_max */
+    uint32_t bin_hi, thr_bits;
+    int32_t take_all;    /* 1: no more than s_max are eligible: everything is taken, no threshold */
+    uint32_t reserved;
+} pf_select_cut_t;
+int pf_select_hist(pf_plan_t *plan, uint64_t first, uint64_t count, const uint8_t *d_reason, const float *d_tput,
+                   const pf_select_cut_t *d_cut, uint32_t *d_hist, void *d_workspace, size_t workspace_bytes,
+                   void *stream);
+int pf_select_cut(const uint64_t *d_hist, int level, uint64_t s_max, pf_select_cut_t *d_cut, void *stream);
+int pf_select_write(pf_plan_t *plan, uint64_t first, uint64_t count, const uint8_t *d_reason, const float *d_tput,
+                    const pf_select_cut_t *d_cut, uint64_t eq_before, uint64_t *d_surv_idx, uint64_t surv_cap,
+                    uint64_t *d_surv_count, void *d_workspace, size_t workspace_bytes, void *stream);
+
 /* Simulator tier (Sec. 3.2: the list-scheduling timeline is the higher-fidelity scorer used to refine
  * schedules).  For each of the n candidates listed in d_surv_idx (n may also be given on the device:
  * if d_n is not NULL the kernel uses min(n, *d_n)): per-stage forward/backward durations from the

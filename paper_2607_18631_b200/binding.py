@@ -25,7 +25,8 @@ EXPORTS = ("pf_version", "pf_strerror", "pf_reason_str", "pf_last_cuda_error", "
            "pf_select_survivors", "pf_simulate_workspace", "pf_simulate", "pf_search_workspace", "pf_search_host",
            "pf_dualpipe_order", "pf_score_static", "pf_serve_plan_count", "pf_aggregate_workspace", "pf_aggregate_serving",
            "pf_report", "pf_search", "pf_search_device_workspace", "pf_compact_workspace", "pf_compact",
-           "pf_search_compact_workspace", "pf_search_host_compact")
+           "pf_search_compact_workspace", "pf_search_host_compact", "pf_select_hist", "pf_select_cut",
+           "pf_select_write")
 # measurement hooks of include/planfront_bench.h that this library exports (the probes live in probes.py)
 BENCH_EXPORTS = ("pf_launch_count", "pf_timing_enable", "pf_timing_read", "pf_bench_fill_span")
 STATIC_SCRATCH_BYTES = 4 << 20
@@ -165,6 +166,12 @@ def load_library(path: str | None = None):
     L.pf_bench_fill_span.argtypes = [vp, C.POINTER(u64), C.POINTER(u64), C.POINTER(u64)]
     L.pf_dualpipe_order.restype = C.c_int
     L.pf_dualpipe_order.argtypes = [C.c_int, C.c_int, vp]
+    L.pf_select_hist.restype = C.c_int
+    L.pf_select_hist.argtypes = [vp, u64, u64, vp, vp, vp, vp, vp, sz, vp]
+    L.pf_select_cut.restype = C.c_int
+    L.pf_select_cut.argtypes = [vp, C.c_int, u64, vp, vp]
+    L.pf_select_write.restype = C.c_int
+    L.pf_select_write.argtypes = [vp, u64, u64, vp, vp, vp, u64, vp, u64, vp, vp, sz, vp]
     L.pf_compact_workspace.restype = sz
     L.pf_compact_workspace.argtypes = [u64]
     L.pf_compact.restype = C.c_int
@@ -384,6 +391,33 @@ class Plan:
                                            _stream_ptr(torch, stream)), "pf_select_survivors")
         return dict(surv_idx=surv_idx, surv_count=surv_count, workspace=workspace)
 
+    # ---- the selection in steps (one space split over several GPUs)
+    def select_hist(self, reason, tput, first: int = 0, cut=None, workspace=None, stream=None):
+        """pf_select_hist: int32[65536] histogram of the high (cut None) or low (inside the cut's bin) 16 score bits
+        of this slice's eligible candidates.  Does not synchronize."""
+        torch = _torch()
+        count = reason.numel()
+        hist = torch.empty(65536, dtype=torch.int32, device=self.device)
+        if workspace is None:
+            workspace = torch.empty(self.select_workspace(count, 1), dtype=torch.uint8, device=self.device)
+        _check(self._L.pf_select_hist(self._h, first, count, _dptr(reason), _dptr(tput), _dptr(cut), _dptr(hist),
+                                      _dptr(workspace), workspace.numel(), _stream_ptr(torch, stream)),
+               "pf_select_hist")
+        return hist
+
+    def select_write(self, reason, tput, cut, eq_before: int, cap: int, first: int = 0, workspace=None, stream=None):
+        """pf_select_write: this slice's survivors under a cut.  Returns (surv_idx int64[cap], surv_count int64[1])."""
+        torch = _torch()
+        count = reason.numel()
+        surv = torch.empty(max(cap, 1), dtype=torch.int64, device=self.device)
+        n = torch.empty(1, dtype=torch.int64, device=self.device)
+        if workspace is None:
+            workspace = torch.empty(self.select_workspace(count, 1), dtype=torch.uint8, device=self.device)
+        _check(self._L.pf_select_write(self._h, first, count, _dptr(reason), _dptr(tput), _dptr(cut), int(eq_before),
+                                       _dptr(surv), max(cap, 1), _dptr(n), _dptr(workspace), workspace.numel(),
+                                       _stream_ptr(torch, stream)), "pf_select_write")
+        return surv, n
+
     # ---- pf_simulate
     def simulate_workspace(self, n: int, k: int) -> int:
         return int(self._L.pf_simulate_workspace(self._h, n, k))
@@ -560,6 +594,25 @@ class Plan:
                "pf_search_host")
         return dict(topk_idx=ti[:tc[0]], topk_score=ts[:tc[0]], sim_topk_idx=si[:sc[0]], sim_topk_score=ss[:sc[0]],
                     n_survivors=int(nsurv[0]))
+
+
+CUT_DTYPE = np.dtype([("total", "<u8"), ("above_hi", "<u8"), ("n_gt", "<u8"), ("need_eq", "<u8"), ("target", "<u8"),
+                      ("bin_hi", "<u4"), ("thr_bits", "<u4"), ("take_all", "<i4"), ("reserved", "<u4")])
+
+
+def pf_select_cut(hist_sum, level: int, s_max: int, cut=None, stream=None):
+    """pf_select_cut on a summed histogram (int64[65536] device tensor).  `cut`: the uint8[48] device tensor of the
+    level-0 call when level is 1.  Returns the cut tensor.  Does not synchronize."""
+    torch = _torch()
+    if cut is None:
+        cut = torch.zeros(CUT_DTYPE.itemsize, dtype=torch.uint8, device=hist_sum.device)
+    _check(load_library().pf_select_cut(_dptr(hist_sum), level, s_max, _dptr(cut), _stream_ptr(torch, stream)),
+           "pf_select_cut")
+    return cut
+
+
+def cut_to_numpy(cut):
+    return cut.cpu().numpy().view(CUT_DTYPE)[0]
 
 
 def pf_topk_merge(k: int, idx_a, score_a, count_a, idx_b, score_b, count_b, stream=None):

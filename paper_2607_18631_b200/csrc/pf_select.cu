@@ -12,6 +12,7 @@ namespace pf {
 constexpr int kSelThreads = 256;
 constexpr int kBins = 65536;
 
+// The first eight fields are the public pf_select_cut_t (same order, same widths).
 struct SelCtrl {
     unsigned long long total;     // eligible candidates
     unsigned long long above1;    // eligible with hi16 > b1
@@ -22,6 +23,7 @@ struct SelCtrl {
     int take_all;
     unsigned int n_elig;          // chunks that hold eligible candidates (length of SelArgs::elig_list)
 };
+static_assert(sizeof(SelCtrl) == sizeof(pf_select_cut_t), "the cut record is the selection's control block");
 
 struct SelArgs {
     uint64_t first, count, s_max;
@@ -35,6 +37,7 @@ struct SelArgs {
     unsigned long long *blk_gt, *blk_eq;  // per block counts, then exclusive prefixes
     uint64_t *surv_idx, *surv_count;
     uint64_t chunk;                   // candidates per block (multiple of 16)
+    unsigned long long eq_before;     // candidates AT the threshold that lower-ranked shards of the space hold
     FillGuard guard;                  // slabs still being filled by another stream must not be read
 };
 
@@ -346,6 +349,7 @@ __global__ void __launch_bounds__(1024) sel_blockscan_kernel(const SelArgs A, in
     __shared__ unsigned long long s_warp[32];
     __shared__ unsigned long long s_tot[kScanTiles][33];   // warp totals per tile, then their exclusive prefixes
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    unsigned long long grand = 0ull;   // totals over all chunks: greater << 32 | equal
     if (nblocks <= kScanTiles * 1024) {
         const int tiles = (nblocks + 1023) / 1024;
         unsigned long long v[kScanTiles], x[kScanTiles];
@@ -392,6 +396,7 @@ __global__ void __launch_bounds__(1024) sel_blockscan_kernel(const SelArgs A, in
             }
             carry += s_tot[k][32];
         }
+        grand = carry;
     } else {
         unsigned long long carry = 0ull;
         unsigned long long nxt = tid < nblocks ? ((A.blk_gt[tid] << 32) | A.blk_eq[tid]) : 0ull;
@@ -409,10 +414,14 @@ __global__ void __launch_bounds__(1024) sel_blockscan_kernel(const SelArgs A, in
             carry += total;
             __syncthreads();   // s_warp is rewritten by the next tile's scan
         }
+        grand = carry;
     }
     if (tid == 0) {
+        // taken here: everything above the threshold, and of those at it what the cut leaves for this range
         const SelCtrl *c = A.ctrl;
-        *A.surv_count = c->take_all ? c->total : c->target;
+        const unsigned long long need = (c->take_all || c->need_eq <= A.eq_before) ? 0ull : c->need_eq - A.eq_before;
+        const unsigned long long n_eq = grand & 0xFFFFFFFFull;
+        *A.surv_count = (grand >> 32) + (n_eq < need ? n_eq : need);
     }
 }
 
@@ -426,7 +435,8 @@ __device__ __forceinline__ void sel_write_chunk(const DevPlan &P, const SelArgs 
     const uint64_t hi = min(lo + A.chunk, A.count);
     const uint32_t thr = A.ctrl->thr_bits;
     const bool all = A.ctrl->take_all != 0;
-    const unsigned long long need_eq = all ? 0ull : A.ctrl->need_eq;
+    const unsigned long long need_eq =
+        (all || A.ctrl->need_eq <= A.eq_before) ? 0ull : A.ctrl->need_eq - A.eq_before;
     const uint8_t *cls = sel_guard_cls(A);
     if (tid == 0) {
         s_run_gt = A.blk_gt[chunk];
@@ -469,10 +479,10 @@ __device__ __forceinline__ void sel_write_chunk(const DevPlan &P, const SelArgs 
             for_each_eligible16(P, vals, A, cls, e, r[t], [&](uint64_t rel, uint32_t bits) {
                 if (all || bits > thr) {
                     unsigned long long pos = my_gt + (my_eq < need_eq ? my_eq : need_eq);
-                    A.surv_idx[pos] = A.first + rel;
+                    if (pos < A.s_max) A.surv_idx[pos] = A.first + rel;   // s_max: the list's capacity
                     my_gt++;
                 } else if (bits == thr) {
-                    if (my_eq < need_eq) A.surv_idx[my_gt + my_eq] = A.first + rel;
+                    if (my_eq < need_eq && my_gt + my_eq < A.s_max) A.surv_idx[my_gt + my_eq] = A.first + rel;
                     my_eq++;
                 }
             });
@@ -589,6 +599,7 @@ int pf::select_run(pf_plan_t *p, uint64_t first, uint64_t count, const uint8_t *
     a.blk_gt = (unsigned long long *)(ws + lay.off_gt);
     a.blk_eq = (unsigned long long *)(ws + lay.off_eq);
     a.surv_idx = d_surv_idx; a.surv_count = d_surv_count; a.chunk = lay.chunk;
+    a.eq_before = 0ull;
     if (guard) a.guard = *guard;
     // control words, histograms and the per-chunk counts start at zero (chunks that are not on the eligible list
     // are never written again); with a digest the scoring kernel has filled the first pass's part already
@@ -610,5 +621,174 @@ int pf::select_run(pf_plan_t *p, uint64_t first, uint64_t count, const uint8_t *
     timing_end(p, PF_T_SELECT, launches, st);
     for (int i = 0; i < launches; i++) count_launch();
     PF_CUDA_TRY(cudaGetLastError(), "pf_select_survivors launch");
+    return PF_OK;
+}
+
+// ------------------------------------------------------------------ the selection in steps, for one space split
+// over several GPUs: every rank histograms its own slice, the histograms are summed by the caller, the cut is
+// found on the sums, every rank compacts its slice against the same cut.
+
+namespace pf {
+
+// One block: scanning a 65,536-bin histogram of 64-bit counts from the top bin down, find the bin in which the
+// running count reaches `target`.  Thread t owns the 64 bins just below 65536 - 64 t.
+__global__ void __launch_bounds__(1024) sel_cut_kernel(const unsigned long long *hist, int level, uint64_t s_max,
+                                                       SelCtrl *c)
+{
+    __shared__ unsigned long long s_warp[32];
+    const int tid = threadIdx.x;
+    if (level == 1 && c->take_all) return;
+    const int top = kBins - 1 - 64 * tid;   // this thread's highest bin
+    unsigned long long mine = 0ull;
+    for (int j = 0; j < 64; j++) mine += hist[top - j];
+    const unsigned long long incl = block_prefix_1024(mine, s_warp);
+    __shared__ unsigned long long s_total;
+    if (tid == 1023) s_total = incl;
+    __syncthreads();
+    unsigned long long target;
+    if (level == 0) {
+        const unsigned long long total = s_total;
+        target = s_max;
+        if (tid == 0) {
+            c->total = total;
+            c->target = target;
+            c->take_all = total <= target ? 1 : 0;
+            c->n_elig = 0;
+            if (total <= target) {
+                c->b1 = 0;
+                c->above1 = 0;
+                c->thr_bits = 0;
+                c->n_gt = total;
+                c->need_eq = 0;
+            }
+        }
+        if (total <= target) return;
+    } else {
+        target = c->target - c->above1;
+    }
+    if (incl - mine < target && incl >= target) {
+        unsigned long long run = incl - mine;   // count strictly above the bin under test
+        for (int j = 0; j < 64; j++) {
+            const unsigned long long h = hist[top - j];
+            if (run + h >= target) {
+                const uint32_t bin = (uint32_t)(top - j);
+                if (level == 0) {
+                    c->b1 = bin;
+                    c->above1 = run;
+                } else {
+                    c->thr_bits = (c->b1 << 16) | bin;
+                    c->n_gt = c->above1 + run;
+                    c->need_eq = c->target - (c->above1 + run);
+                }
+                break;
+            }
+            run += h;
+        }
+    }
+}
+
+static int sel_args(pf_plan_t *p, uint64_t first, uint64_t count, const uint8_t *d_reason, const float *d_tput,
+                    void *d_workspace, size_t workspace_bytes, SelArgs &a, SelLayout &lay)
+{
+    if (!p || !d_reason || !d_tput) return PF_EINVAL;
+    if (p->dev.phase != PF_PHASE_TRAIN) return PF_EUNSUPPORTED;
+    if (count == 0 || count >= PF_MAX_COUNT) return PF_ERANGE;
+    if (first >= p->size || count > p->size - first) return PF_ERANGE;
+    lay = sel_layout(p, count);
+    if (!d_workspace || ((uintptr_t)d_workspace & 255) != 0 || workspace_bytes < lay.total) return PF_EWORKSPACE;
+    if (int rc_dev = check_device(p)) return rc_dev;
+    uint8_t *ws = (uint8_t *)d_workspace;
+    a.first = first; a.count = count; a.s_max = 0; a.reason = d_reason; a.tput = d_tput;
+    a.ctrl = (SelCtrl *)(ws + lay.off_ctrl);
+    a.hist1 = (unsigned int *)(ws + lay.off_hist1);
+    a.hist2 = (unsigned int *)(ws + lay.off_hist2);
+    a.coarse1 = (unsigned int *)(ws + lay.off_coarse);
+    a.coarse2 = a.coarse1 + 256;
+    a.blk_elig = (unsigned int *)(ws + lay.off_elig);
+    a.elig_list = (unsigned int *)(ws + lay.off_list);
+    a.blk_gt = (unsigned long long *)(ws + lay.off_gt);
+    a.blk_eq = (unsigned long long *)(ws + lay.off_eq);
+    a.surv_idx = nullptr; a.surv_count = nullptr; a.chunk = lay.chunk;
+    a.eq_before = 0ull;
+    return PF_OK;
+}
+
+}  // namespace pf
+
+extern "C" int pf_select_hist(pf_plan_t *p, uint64_t first, uint64_t count, const uint8_t *d_reason,
+                              const float *d_tput, const pf_select_cut_t *d_cut, uint32_t *d_hist, void *d_workspace,
+                              size_t workspace_bytes, void *stream)
+{
+    if (!d_hist) return PF_EINVAL;
+    SelArgs a;
+    SelLayout lay;
+    int rc = sel_args(p, first, count, d_reason, d_tput, d_workspace, workspace_bytes, a, lay);
+    if (rc != PF_OK) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    uint8_t *ws = (uint8_t *)d_workspace;
+    PF_CUDA_TRY(cudaMemsetAsync(ws, 0, lay.off_list, st), "pf_select_hist: clear");
+    PF_CUDA_TRY(cudaMemsetAsync(d_hist, 0, kBins * sizeof(uint32_t), st), "pf_select_hist: clear");
+    timing_begin(p, PF_T_SELECT, st);
+    int launches = 1;
+    if (!d_cut) {
+        a.hist1 = d_hist;                     // level 0: the high 16 score bits of every eligible candidate
+        sel_hist_kernel<<<lay.nblocks, kSelThreads, 0, st>>>(p->dev, a, p->d_vals, 0);
+    } else {
+        // level 1: the low 16 bits of those whose high bits are the cut's bin.  The chunk list comes from a
+        // level-0 pass into scratch; the cut's fields are copied behind it (the list length survives).
+        sel_hist_kernel<<<lay.nblocks, kSelThreads, 0, st>>>(p->dev, a, p->d_vals, 0);
+        PF_CUDA_TRY(cudaMemcpyAsync(a.ctrl, d_cut, offsetof(SelCtrl, n_elig), cudaMemcpyDeviceToDevice, st),
+                    "pf_select_hist: cut");
+        a.hist2 = d_hist;
+        const int list_grid = lay.nblocks < p->sm_count * 8 ? lay.nblocks : p->sm_count * 8;
+        sel_hist_kernel<<<list_grid, kSelThreads, 0, st>>>(p->dev, a, p->d_vals, 1);
+        launches = 2;
+    }
+    timing_end(p, PF_T_SELECT, launches, st);
+    for (int i = 0; i < launches; i++) count_launch();
+    PF_CUDA_TRY(cudaGetLastError(), "pf_select_hist launch");
+    return PF_OK;
+}
+
+extern "C" int pf_select_cut(const uint64_t *d_hist, int level, uint64_t s_max, pf_select_cut_t *d_cut, void *stream)
+{
+    if (!d_hist || !d_cut || (level != 0 && level != 1)) return PF_EINVAL;
+    if (level == 0 && s_max == 0) return PF_ERANGE;
+    sel_cut_kernel<<<1, 1024, 0, (cudaStream_t)stream>>>((const unsigned long long *)d_hist, level, s_max,
+                                                         (SelCtrl *)d_cut);
+    count_launch();
+    PF_CUDA_TRY(cudaGetLastError(), "pf_select_cut launch");
+    return PF_OK;
+}
+
+extern "C" int pf_select_write(pf_plan_t *p, uint64_t first, uint64_t count, const uint8_t *d_reason,
+                               const float *d_tput, const pf_select_cut_t *d_cut, uint64_t eq_before,
+                               uint64_t *d_surv_idx, uint64_t surv_cap, uint64_t *d_surv_count, void *d_workspace,
+                               size_t workspace_bytes, void *stream)
+{
+    if (!d_cut || !d_surv_idx || !d_surv_count) return PF_EINVAL;
+    SelArgs a;
+    SelLayout lay;
+    int rc = sel_args(p, first, count, d_reason, d_tput, d_workspace, workspace_bytes, a, lay);
+    if (rc != PF_OK) return rc;
+    if (surv_cap == 0) return PF_ERANGE;
+    cudaStream_t st = (cudaStream_t)stream;
+    uint8_t *ws = (uint8_t *)d_workspace;
+    a.surv_idx = d_surv_idx; a.surv_count = d_surv_count; a.eq_before = eq_before;
+    a.s_max = surv_cap;   // entries past the capacity are counted but not written
+    PF_CUDA_TRY(cudaMemsetAsync(ws, 0, lay.off_list, st), "pf_select_write: clear");
+    timing_begin(p, PF_T_SELECT, st);
+    // the chunk list and per-chunk eligible counts (a level-0 pass into scratch), then the cut, then the usual
+    // count / prefix / ordered write
+    sel_hist_kernel<<<lay.nblocks, kSelThreads, 0, st>>>(p->dev, a, p->d_vals, 0);
+    PF_CUDA_TRY(cudaMemcpyAsync(a.ctrl, d_cut, offsetof(SelCtrl, n_elig), cudaMemcpyDeviceToDevice, st),
+                "pf_select_write: cut");
+    const int list_grid = lay.nblocks < p->sm_count * 8 ? lay.nblocks : p->sm_count * 8;
+    sel_count_kernel<<<list_grid, kSelThreads, 0, st>>>(p->dev, a, p->d_vals);
+    sel_blockscan_kernel<<<1, 1024, 0, st>>>(a, lay.nblocks);
+    sel_write_kernel<<<list_grid, kSelThreads, 0, st>>>(p->dev, a, p->d_vals);
+    timing_end(p, PF_T_SELECT, 4, st);
+    for (int i = 0; i < 4; i++) count_launch();
+    PF_CUDA_TRY(cudaGetLastError(), "pf_select_write launch");
     return PF_OK;
 }

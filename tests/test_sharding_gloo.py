@@ -89,3 +89,68 @@ def test_two_rank_gather_and_merge_equals_global_topk():
         assert gc == len(want_idx)
         np.testing.assert_array_equal(gi[:gc].astype(np.uint64), want_idx)
         np.testing.assert_allclose(gs[:gc], want_sc, rtol=1e-6)
+
+
+# ----------------------------------------------------------------------------- the whole search, split
+
+def _search_cfg(ties: bool):
+    from helpers import variant
+    cfg = variant("mid", cluster=dict(budget_bytes=10 ** 15), rules=dict(enforce_realizability=0))
+    if ties:
+        for kv in (1, 2, 3):          # four identical kernel variants: every score appears four times
+            cfg["kern"][kv] = dict(cfg["kern"][0])
+    return cfg
+
+
+def _search_worker(rank, world, port, k, s_max, k_sim, ties, ret):
+    import torch.distributed as dist
+    from oracle import Oracle
+    from paper_2607_18631_b200.sharding import sharded_search
+    from sharded_common import OracleOps
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        r = sharded_search(OracleOps(Oracle(_search_cfg(ties))), k, s_max, k_sim, 4)
+        n = int(r["surv"][1].item())
+        ret[rank] = dict(first=r["local"]["first"], count=r["local"]["count"],
+                         topk=tuple(t.numpy().copy() for t in r["topk"]),
+                         surv=r["surv"][0][:n].numpy().copy(), total=r["n_survivors_total"],
+                         sim_topk=tuple(t.numpy().copy() for t in r["sim_topk"]))
+    finally:
+        dist.destroy_process_group()
+
+
+@pytest.mark.parametrize("s_max,ties", [(10 ** 6, False), (700, False), (501, True), (1, True)])
+def test_two_rank_sharded_search_equals_the_unsplit_search(s_max, ties):
+    """sharded_search itself on two gloo ranks (the oracle doing each rank's share of the work): the folded top-k,
+    the concatenated survivor lists and the folded simulator top-k are those of the unsplit space -- with a cut that
+    falls inside a run of equal scores spread over both ranks."""
+    import torch.multiprocessing as mp
+    from oracle import Oracle
+    world, k, k_sim = 2, 64, 50
+    port = _free_port()
+    ret = mp.Manager().dict()
+    mp.spawn(_search_worker, args=(world, port, k, s_max, k_sim, ties, ret), nprocs=world, join=True)
+    orc = Oracle(_search_cfg(ties))
+    reason, tput, _, _ = orc.score_range(threads=4)
+    tput32 = tput.astype(np.float32).astype(np.float64)       # the ranks rank fp32 scores, like the device
+    want_idx, want_sc = orc.topk(reason, tput32, 0, k)
+    want_surv = orc.select_survivors(reason, tput32, 0, s_max)
+    sim, _, _ = orc.simulate_list(want_surv, 4, threads=4)
+    want_sim_idx, want_sim_sc = Oracle.topk_list(want_surv, sim, k_sim)
+    got_surv = np.concatenate([ret[r]["surv"] for r in range(world)]).astype(np.uint64)
+    np.testing.assert_array_equal(got_surv, want_surv)
+    for r in range(world):
+        assert ret[r]["total"] == len(want_surv)
+        gi, gs, gc = ret[r]["topk"]
+        np.testing.assert_array_equal(gi[:int(gc[0])].astype(np.uint64), want_idx)
+        si, ss, sc = ret[r]["sim_topk"]
+        n = int(sc[0])
+        assert n == len(want_sim_idx)
+        np.testing.assert_array_equal(si[:n].astype(np.uint64), want_sim_idx)
+        np.testing.assert_allclose(ss[:n], want_sim_sc, rtol=1e-6)
+    if ties and s_max > 1:
+        # the cut did fall inside a run of equal scores
+        cut_score = tput32[want_surv.astype(np.int64)].min()
+        assert (tput32[(reason & 0x7F) == 0] == cut_score).sum() > (tput32[want_surv.astype(np.int64)] == cut_score).sum()
