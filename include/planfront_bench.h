@@ -37,6 +37,18 @@ int pf_timing_read(pf_plan_t *plan, float *ms, uint32_t *kernels);
 /* Number of kernels this library has launched in this process (for launch accounting in benchmarks). */
 uint64_t pf_launch_count(void);
 
+/* The checked build (the library compiled with -DPF_BOUNDS_CHECK: every index into a shared-memory image, queue,
+ * table, timeline, order table, key list or output array is range-checked on the device; a violation is recorded
+ * and the access redirected to element 0 -- nothing traps).  pf_check_read waits for the device, copies the plan's
+ * record to out[6] and clears it: out[0] = one bit per kind of array that saw a bad index (0 = clean), out[1] = the
+ * last such kind, out[2..3] = the offending index, out[4..5] = the array's length.  The ordinary build returns
+ * PF_EUNSUPPORTED and zeros. */
+int pf_check_read(pf_plan_t *plan, uint32_t *out);
+/* The checks' own check (checked build only, else PF_EUNSUPPORTED): one device thread asks for element 7 of a
+ * 4-element array through the checking macro; the store is redirected inside the array and the next pf_check_read
+ * must show bit 17, index 7, length 4. */
+int pf_check_selftest(pf_plan_t *plan);
+
 /* How the plan's latest scoring call inside pf_search was divided between the scoring kernel and the kernel that
  * streams constant blocks: the number of blocks of candidates the call's range was cut into, candidates per block,
  * and how many blocks the scoring kernel took itself (the evaluated ones and the constant ones interleaved with

@@ -14,7 +14,8 @@ import os
 import numpy as np
 
 HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(HERE, "libplanfront.so")
+# PLANFRONT_LIB: another build of the same library (the checked build, build.build(bounds_check=True))
+LIB_PATH = os.environ.get("PLANFRONT_LIB") or os.path.join(HERE, "libplanfront.so")
 
 MAX_AXES, MAX_SCHED, MAX_KERN, NBUCKET, K_MAX = 11, 8, 16, 8, 1024
 PF_OK, PF_EINVAL, PF_ERANGE, PF_EWORKSPACE, PF_ECUDA, PF_EUNSUPPORTED = 0, -1, -2, -3, -4, -5
@@ -28,7 +29,7 @@ EXPORTS = ("pf_version", "pf_strerror", "pf_reason_str", "pf_last_cuda_error", "
            "pf_search_compact_workspace", "pf_search_host_compact", "pf_select_hist", "pf_select_cut",
            "pf_select_write")
 # measurement hooks of include/planfront_bench.h that this library exports (the probes live in probes.py)
-BENCH_EXPORTS = ("pf_launch_count", "pf_timing_enable", "pf_timing_read", "pf_bench_fill_span")
+BENCH_EXPORTS = ("pf_launch_count", "pf_timing_enable", "pf_timing_read", "pf_bench_fill_span", "pf_check_read", "pf_check_selftest")
 STATIC_SCRATCH_BYTES = 4 << 20
 T_CLASSES = ("score", "topk", "select", "simulate", "aggregate", "fill", "simprep", "compact")
 REASON_BINS = 16
@@ -162,6 +163,10 @@ def load_library(path: str | None = None):
     L.pf_timing_enable.argtypes = [vp, C.c_int]
     L.pf_timing_read.restype = C.c_int
     L.pf_timing_read.argtypes = [vp, vp, vp]
+    L.pf_check_selftest.restype = C.c_int
+    L.pf_check_selftest.argtypes = [vp]
+    L.pf_check_read.restype = C.c_int
+    L.pf_check_read.argtypes = [vp, vp]
     L.pf_bench_fill_span.restype = C.c_int
     L.pf_bench_fill_span.argtypes = [vp, C.POINTER(u64), C.POINTER(u64), C.POINTER(u64)]
     L.pf_dualpipe_order.restype = C.c_int
@@ -312,6 +317,15 @@ class Plan:
     # ---- pf_timing_enable / pf_timing_read
     def timing_enable(self, on: bool = True):
         _check(self._L.pf_timing_enable(self._h, 1 if on else 0), "pf_timing_enable")
+
+    def check_selftest(self) -> int:
+        return int(self._L.pf_check_selftest(self._h))
+
+    def check_read(self):
+        """pf_check_read: (status, record of six words) of the checked build; status PF_EUNSUPPORTED otherwise."""
+        out = np.zeros(6, dtype=np.uint32)
+        st = self._L.pf_check_read(self._h, out.ctypes.data_as(C.c_void_p))
+        return int(st), out
 
     def fill_span(self) -> dict:
         """pf_bench_fill_span: how the latest pf_search split the space between the scoring and the fill kernel."""

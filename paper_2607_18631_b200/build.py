@@ -11,6 +11,8 @@ LIB = os.path.join(HERE, "libplanfront.so")
 SOURCES = ["pf_api.cu", "pf_score.cu", "pf_select.cu", "pf_simulate.cu", "pf_search.cu", "pf_aggregate.cu", "pf_report.cu", "pf_compact.cu"]
 # the roofline probes of the benchmark: a library of their own, not part of the scoring ABI
 PROBE_LIB = os.path.join(HERE, "libplanfront_probe.so")
+# the same library with every device-side index range-checked (-DPF_BOUNDS_CHECK): for the checked test run
+CHECK_LIB = os.path.join(HERE, "libplanfront_check.so")
 PROBE_SOURCES = ["pf_probe.cu"]
 
 
@@ -30,10 +32,15 @@ def _compile(lib: str, sources, verbose: bool, defines=()) -> None:
     subprocess.run(cmd, check=True)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
+def build(force: bool = False, verbose: bool = False, bounds_check: bool = False) -> str:
     """Compile the scoring library (every scoring .cu into libplanfront.so) and the benchmark's probe library.
-    Returns the scoring library's path."""
+    Returns the scoring library's path.  bounds_check=True builds (only) the checked variant,
+    libplanfront_check.so, and returns its path; PLANFRONT_LIB=<that path> makes the binding load it."""
     newest = _newest_source()
+    if bounds_check:
+        if force or not os.path.exists(CHECK_LIB) or os.path.getmtime(CHECK_LIB) < newest:
+            _compile(CHECK_LIB, SOURCES, verbose, defines=("PF_BOUNDS_CHECK",))
+        return CHECK_LIB
     if force or not os.path.exists(LIB) or os.path.getmtime(LIB) < newest:
         _compile(LIB, SOURCES, verbose)
     if force or not os.path.exists(PROBE_LIB) or os.path.getmtime(PROBE_LIB) < newest:

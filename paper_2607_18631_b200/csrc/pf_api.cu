@@ -426,6 +426,9 @@ extern "C" int pf_plan_create(const pf_model_t *model, const pf_cluster_t *clust
         if (e == cudaSuccess)
             e = cudaMemcpy(p->d_scen + n, workload->scen_O, sizeof(int32_t) * n, cudaMemcpyHostToDevice);
     }
+    if (e == cudaSuccess) e = cudaMalloc((void **)&p->d_check, 64);
+    if (e == cudaSuccess) e = cudaMemset(p->d_check, 0, 64);
+    d.chk = p->d_check;
     if (e == cudaSuccess) {
         // room for the slab visiting order of one pf_score range (any alignment of its first candidate)
         const uint64_t slabs = (p->size + d.slab - 1) / d.slab + 1;
@@ -499,6 +502,41 @@ extern "C" int pf_timing_read(pf_plan_t *p, float *ms, uint32_t *kernels)
     return PF_OK;
 }
 
+// The checks' own check: one thread asks for element 7 of a 4-element array through PF_AT.  In the checked build the
+// index comes back as 0 (the store lands inside the array) and the record names the site, index and length.
+__global__ void check_selftest_kernel(unsigned int *chk, unsigned int *four_words)
+{
+    four_words[PF_AT(chk, 3 + 4 * (int)(threadIdx.x + 1), 4, pf::PF_SITE_TOPK_BUF) & 3] = 1u;
+}
+
+extern "C" int pf_check_selftest(pf_plan_t *p)
+{
+    if (!p) return PF_EINVAL;
+#ifndef PF_BOUNDS_CHECK
+    return PF_EUNSUPPORTED;
+#else
+    if (int rc_dev = pf::check_device(p)) return rc_dev;
+    check_selftest_kernel<<<1, 1>>>(p->d_check, p->d_check + 8);   // words 8..11 of the record's block: scratch
+    PF_CUDA_TRY(cudaGetLastError(), "pf_check_selftest");
+    return PF_OK;
+#endif
+}
+
+extern "C" int pf_check_read(pf_plan_t *p, uint32_t *out)
+{
+    if (!p || !out) return PF_EINVAL;
+#ifndef PF_BOUNDS_CHECK
+    for (int i = 0; i < 6; i++) out[i] = 0;
+    return PF_EUNSUPPORTED;   // this build carries no index checks
+#else
+    if (int rc_dev = pf::check_device(p)) return rc_dev;
+    PF_CUDA_TRY(cudaDeviceSynchronize(), "pf_check_read");
+    PF_CUDA_TRY(cudaMemcpy(out, p->d_check, 6 * sizeof(uint32_t), cudaMemcpyDeviceToHost), "pf_check_read");
+    PF_CUDA_TRY(cudaMemset(p->d_check, 0, 64), "pf_check_read");
+    return PF_OK;
+#endif
+}
+
 extern "C" int pf_bench_fill_span(pf_plan_t *p, uint64_t *n_blocks, uint64_t *block_candidates, uint64_t *scored_blocks)
 {
     if (!p || !n_blocks || !block_candidates || !scored_blocks || !p->d_order) return PF_EINVAL;
@@ -528,6 +566,7 @@ extern "C" void pf_plan_destroy(pf_plan_t *p)
     if (p->d_vals) cudaFree(p->d_vals);
     if (p->d_scen) cudaFree(p->d_scen);
     if (p->d_order) cudaFree(p->d_order);
+    if (p->d_check) cudaFree(p->d_check);
     if (p->ev_fork) cudaEventDestroy(p->ev_fork);
     if (p->ev_join) cudaEventDestroy(p->ev_join);
     if (p->ev_fill) cudaEventDestroy(p->ev_fill);

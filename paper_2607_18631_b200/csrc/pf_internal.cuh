@@ -85,7 +85,38 @@ struct DevPlan {
     // --- calibration domain of the constants
     int dom_attached, dom_gpu, dom_m_lo, dom_m_hi, gpu_id;
     uint32_t dom_dtypes;
+    // --- the checked build's record (PF_BOUNDS_CHECK): word 0 = bits of the sites that saw an index outside its
+    // array, word 1 = the last such site, words 2-3 = the offending index, words 4-5 = the array's length
+    unsigned int *chk;
 };
+
+// Index checks of the checked build (-DPF_BOUNDS_CHECK; the ordinary build compiles them away).  PF_AT(i, n, site)
+// is the index to use for an array of n elements: i itself when 0 <= i < n; otherwise the violation is recorded in
+// the plan's check record and 0 is used instead, so the access stays inside the array and nothing traps.
+enum {
+    PF_SITE_ORDER = 0, PF_SITE_IMAGE = 1, PF_SITE_QUEUE = 2, PF_SITE_TABLE = 3, PF_SITE_PASS = 4, PF_SITE_INFO = 5,
+    PF_SITE_DENSE = 6, PF_SITE_KEYS = 7, PF_SITE_DIGEST = 8, PF_SITE_VALS = 9, PF_SITE_TIMELINE = 10,
+    PF_SITE_DURATION = 11, PF_SITE_RECORD = 12, PF_SITE_SIM_OUT = 13, PF_SITE_DUAL_OPS = 14, PF_SITE_CHUNK = 15,
+    PF_SITE_SURVIVOR = 16, PF_SITE_TOPK_BUF = 17, PF_SITE_SCEN = 18
+};
+#ifdef PF_BOUNDS_CHECK
+__device__ __forceinline__ long long check_at(unsigned int *chk, long long i, long long n, int site)
+{
+    if (i >= 0 && i < n) return i;
+    if (chk) {
+        atomicOr(chk, 1u << site);
+        chk[1] = (unsigned int)site;
+        chk[2] = (unsigned int)i;
+        chk[3] = (unsigned int)((unsigned long long)i >> 32);
+        chk[4] = (unsigned int)n;
+        chk[5] = (unsigned int)((unsigned long long)n >> 32);
+    }
+    return 0;
+}
+#define PF_AT(chk, i, n, site) pf::check_at((chk), (long long)(i), (long long)(n), (site))
+#else
+#define PF_AT(chk, i, n, site) (i)
+#endif
 
 }  // namespace pf
 
@@ -116,6 +147,7 @@ struct pf_plan {
     cudaEvent_t ev_fork, ev_join, ev_fork2, ev_fill;
     // simulator order tables (built at create for training plans)
     void *sim_tables;
+    unsigned int *d_check;         // the checked build's record (dev.chk); 64 bytes, zero unless a check fired
     // optional per-kernel-class event timing (pf_timing_enable)
     void *timing;
 };

@@ -269,7 +269,7 @@ __global__ void __launch_bounds__(kThreads, 4) score_kernel(const __grid_constan
         const uint32_t t0 = blockIdx.x;
         s_gthr = 0ull;
         tkt_next = gridDim.x + atomicAdd(A.slab_counter, 1u);
-        resolve(t0, (order && t0 < n_tickets) ? __ldcg(order + t0) : 0u, s_slabs[0]);
+        resolve(t0, (order && t0 < n_tickets) ? __ldcg(order + PF_AT(P.chk, t0, A.n_slabs, PF_SITE_ORDER)) : 0u, s_slabs[0]);
     }
     __syncthreads();
 
@@ -277,7 +277,7 @@ __global__ void __launch_bounds__(kThreads, 4) score_kernel(const __grid_constan
         const SlabInfo &s_slab = s_slabs[cur];
         if (s_slab.slab == 0xFFFFFFFFu) break;
         if (tid == 0) {
-            word_next = (order && tkt_next < n_tickets) ? __ldcg(order + tkt_next) : 0u;
+            word_next = (order && tkt_next < n_tickets) ? __ldcg(order + PF_AT(P.chk, tkt_next, A.n_slabs, PF_SITE_ORDER)) : 0u;
             tkt_after = gridDim.x + atomicAdd(A.slab_counter, 1u);
             // the grid-wide threshold only matters to evaluated slabs: refresh it on those
             if (want_topk && s_slab.pre_reason == 0) gthr_next = *reinterpret_cast<volatile unsigned long long *>(A.g_thr);
@@ -300,6 +300,7 @@ __global__ void __launch_bounds__(kThreads, 4) score_kernel(const __grid_constan
         const uint64_t hi = end_slab < end_call ? end_slab : end_call;
         const uint64_t rel0 = lo - A.first;  // offset of the first candidate in the dense outputs
         const uint32_t n = (uint32_t)(hi - lo);
+        (void)PF_AT(P.chk, rel0 + n - 1, A.count, PF_SITE_DENSE);   // the slab's whole span lies inside the outputs
 
         if (s_slab.pre_reason != 0) {
             if (A.reason) block_fill(A.reason + rel0, n, (uint32_t)s_slab.pre_reason);
@@ -330,7 +331,7 @@ __global__ void __launch_bounds__(kThreads, 4) score_kernel(const __grid_constan
                     TrainDerived<RI> D;
                     r = train_plan_rules<RI>(P, c, dp, world, first_rule, D, 7);
                 }
-                s_tab[e] = (uint8_t)r;
+                s_tab[PF_AT(P.chk, e, 2048, PF_SITE_TABLE)] = (uint8_t)r;
             }
             __syncthreads();
         }
@@ -344,7 +345,7 @@ __global__ void __launch_bounds__(kThreads, 4) score_kernel(const __grid_constan
                     uint32_t q = r == 1u ? rem : __umulhi(rem, P.magic[a]);
                     const int digit = (int)(rem - q * r);
                     if (a < 5) dg[a] = digit;
-                    v[a] = inner_vals[P.val_off[a] + digit];
+                    v[a] = inner_vals[PF_AT(P.chk, P.val_off[a] + digit, n_inner_vals, PF_SITE_VALS)];
                     rem = q;
                 } else {
                     v[a] = a < P.n_axes ? s_slab.outer[a] : 0;
@@ -395,7 +396,7 @@ __global__ void __launch_bounds__(kThreads, 4) score_kernel(const __grid_constan
                     float tput = 0.f;
                     uint32_t i = 0;
                     if (active) {
-                        i = s_queue[qi];
+                        i = s_queue[PF_AT(P.chk, qi, kQueueCap, PF_SITE_QUEUE)];
                         int v[PF_MAX_AXES], dg[5] = {0, 0, 0, 0, 0};
                         decode_inner(j0 + i, v, dg);
                         TrainTuple c;
@@ -416,18 +417,21 @@ __global__ void __launch_bounds__(kThreads, 4) score_kernel(const __grid_constan
                             tput = train_price<RI>(P, c, D, T, train_pipe_analytic<RI>(P, c, D, T));
                             if (domain_why<RI>(P, P.kern[c.kv], D.m_e)) reason = PF_FLAG_EXTRAPOLATED;
                         }
-                        const uint64_t o = rel0 + i;
-                        img[i] = (uint8_t)reason;
+                        const uint64_t o = PF_AT(P.chk, rel0 + i, A.count, PF_SITE_DENSE);
+                        img[PF_AT(P.chk, pad + i, P.slab + 16, PF_SITE_IMAGE) - pad] = (uint8_t)reason;
                         if (A.tput && tput != 0.f) A.tput[o] = tput;
                         if (A.mem) A.mem[o] = M.mem;
                         // the selection's first pass, done here for the few feasible plans inside the simulator's
                         // domain: score-bit histograms, the chunk's eligible count, the list of non-empty chunks
                         if (A.dg.hist1 && tput != 0.f && c.pp <= PF_SIM_MAX_RANKS && D.v_eff <= PF_SIM_MAX_V) {
                             const uint32_t bits = __float_as_uint(tput);
-                            atomicAdd(A.dg.hist1 + (bits >> 16), 1u);
-                            atomicAdd(A.dg.coarse1 + (bits >> 24), 1u);
-                            const uint32_t chunk = (uint32_t)(o / A.dg.chunk);
-                            if (atomicAdd(A.dg.elig + chunk, 1u) == 0u) A.dg.list[atomicAdd(A.dg.n_list, 1u)] = chunk;
+                            atomicAdd(A.dg.hist1 + PF_AT(P.chk, bits >> 16, 65536, PF_SITE_DIGEST), 1u);
+                            atomicAdd(A.dg.coarse1 + PF_AT(P.chk, bits >> 24, 256, PF_SITE_DIGEST), 1u);
+                            const uint32_t n_chunks = (uint32_t)((A.count + A.dg.chunk - 1) / A.dg.chunk);
+                            (void)n_chunks;
+                            const uint32_t chunk = (uint32_t)PF_AT(P.chk, o / A.dg.chunk, n_chunks, PF_SITE_CHUNK);
+                            if (atomicAdd(A.dg.elig + chunk, 1u) == 0u)
+                                A.dg.list[PF_AT(P.chk, atomicAdd(A.dg.n_list, 1u), n_chunks, PF_SITE_CHUNK)] = chunk;
                         }
                     }
                     offer(active && (reason & 0x7f) == 0, tput, (uint32_t)(rel0 + i));
@@ -444,7 +448,8 @@ __global__ void __launch_bounds__(kThreads, 4) score_kernel(const __grid_constan
                     int qb = 0;
                     if (lane2 == leader) qb = atomicAdd(&s_qn, __popc(mask));
                     qb = __shfl_sync(0xFFFFFFFFu, qb, leader);
-                    if (queued) s_queue[qb + __popc(mask & ((1u << lane2) - 1u))] = (uint16_t)i;
+                    if (queued)
+                        s_queue[PF_AT(P.chk, qb + __popc(mask & ((1u << lane2) - 1u)), kQueueCap, PF_SITE_QUEUE)] = (uint16_t)i;
                 }
             };
             int since_drain = 0;  // iterations that appended (at most kThreads entries each) since the last drain
@@ -457,19 +462,20 @@ __global__ void __launch_bounds__(kThreads, 4) score_kernel(const __grid_constan
                 const int lane = tid & 31;
                 for (uint32_t cb = 0; cb < n_combos; cb += kThreads) {
                     const uint32_t e = cb + tid;
-                    const int t = e < n_combos ? (int)s_tab[e] : 0xFF;
+                    const int t = e < n_combos ? (int)s_tab[PF_AT(P.chk, e, 2048, PF_SITE_TABLE)] : 0xFF;
                     const unsigned pm = __ballot_sync(0xFFFFFFFFu, t == 0);
                     if (pm) {
                         const int leader = __ffs(pm) - 1;
                         int pb = 0;
                         if (lane == leader) pb = atomicAdd(&s_np, __popc(pm));
                         pb = __shfl_sync(0xFFFFFFFFu, pb, leader);
-                        if (t == 0) s_pass[pb + __popc(pm & ((1u << lane) - 1u))] = (uint16_t)e;
+                        if (t == 0) s_pass[PF_AT(P.chk, pb + __popc(pm & ((1u << lane) - 1u)), 2048, PF_SITE_PASS)] = (uint16_t)e;
                     }
                     if (t != 0 && t != 0xFF) {
                         // the run's candidates, clipped to the call's range
                         const uint32_t ja = max(e * R, j0), jb = min(e * R + R, j0 + n);
-                        for (uint32_t j = ja; j < jb; j++) img[j - j0] = (uint8_t)t;
+                        for (uint32_t j = ja; j < jb; j++)
+                            img[PF_AT(P.chk, pad + j - j0, P.slab + 16, PF_SITE_IMAGE) - pad] = (uint8_t)t;
                     }
                 }
                 __syncthreads();
@@ -485,7 +491,7 @@ __global__ void __launch_bounds__(kThreads, 4) score_kernel(const __grid_constan
                     if ((uint32_t)(tid >> 2) < nb) {
                         // four lanes per entry: lanes 0-2 take one recompute mode's memory each, lane 3 the rules
                         const int role = tid & 3, slot = tid >> 2;
-                        const int e = s_pass[b0 + slot];
+                        const int e = s_pass[PF_AT(P.chk, b0 + slot, 2048, PF_SITE_PASS)];
                         const int n2 = P.tab_n[0], n3 = P.tab_n[1];
                         const int d2 = e % n2, d3 = (e / n2) % n3, d4 = e / (n2 * n3);
                         TrainTuple c;
@@ -528,14 +534,14 @@ __global__ void __launch_bounds__(kThreads, 4) score_kernel(const __grid_constan
                         uint32_t i = 0;
                         if (x < total) {
                             const uint32_t pe = x / R, ro = x - pe * R;
-                            const uint32_t j = (uint32_t)s_pass[b0 + pe] * R + ro;
+                            const uint32_t j = (uint32_t)s_pass[PF_AT(P.chk, b0 + pe, 2048, PF_SITE_PASS)] * R + ro;
                             if (j >= j0 && j < j0 + n) {
                                 i = j - j0;
                                 const uint32_t r0 = P.radix[0];
                                 const uint32_t qd = r0 == 1u ? ro : __umulhi(ro, P.magic[0]);
                                 const int kvv = inner_vals[P.val_off[0] + (int)(ro - qd * r0)];
                                 const int recv = P.n_inner > 1 ? inner_vals[P.val_off[1] + (int)qd] : s_slab.outer[1];
-                                const EntryInfo &info = s_info[pe];
+                                const EntryInfo &info = s_info[PF_AT(P.chk, pe, kEntryBatch, PF_SITE_INFO)];
                                 int reason = 0;
                                 if ((info.kv_bad >> kvv) & 1u) {
                                     reason = PF_R_KERNEL_MISSING;
@@ -545,13 +551,13 @@ __global__ void __launch_bounds__(kThreads, 4) score_kernel(const __grid_constan
                                     reason = PF_R_OVERLAP_PRECOND;
                                 } else {
                                     const long long mem = info.mem[recv];
-                                    if (A.mem) A.mem[rel0 + i] = mem;
+                                    if (A.mem) A.mem[PF_AT(P.chk, rel0 + i, A.count, PF_SITE_DENSE)] = mem;
                                     if (mem > P.budget_bytes)
                                         reason = PF_R_MEMORY;
                                     else
                                         queued = true;
                                 }
-                                if (!queued) img[i] = (uint8_t)reason;
+                                if (!queued) img[PF_AT(P.chk, pad + i, P.slab + 16, PF_SITE_IMAGE) - pad] = (uint8_t)reason;
                             }
                         }
                         enqueue(queued, i);
@@ -584,7 +590,7 @@ __global__ void __launch_bounds__(kThreads, 4) score_kernel(const __grid_constan
                             reason = train_plan_rules<RI>(P, c, dp, world, first_rule, D);
                         }
                         if (reason != 0)
-                            img[i] = (uint8_t)reason;
+                            img[PF_AT(P.chk, pad + i, P.slab + 16, PF_SITE_IMAGE) - pad] = (uint8_t)reason;
                         else
                             queued = true;
                     }
@@ -610,8 +616,9 @@ __global__ void __launch_bounds__(kThreads, 4) score_kernel(const __grid_constan
                     decode_inner(j0 + i, v, dg);
                     ServeTuple c;
                     c.kv = v[0]; c.chunk = v[1]; c.batch = v[2]; c.dpa = v[3]; c.ep = v[4]; c.tp = v[5]; c.scen = v[6];
-                    serve_eval<RI>(P, c, first_rule, __ldg(A.scen + c.scen), __ldg(A.scen + P.n_scen + c.scen), so);
-                    const uint64_t o = rel0 + i;
+                    const int sc_i = (int)PF_AT(P.chk, c.scen, P.n_scen, PF_SITE_SCEN);
+                    serve_eval<RI>(P, c, first_rule, __ldg(A.scen + sc_i), __ldg(A.scen + P.n_scen + sc_i), so);
+                    const uint64_t o = PF_AT(P.chk, rel0 + i, A.count, PF_SITE_DENSE);
                     if (A.reason) A.reason[o] = (uint8_t)so.reason;
                     if (A.tput) A.tput[o] = so.tput;
                     if (A.mem) A.mem[o] = so.mem;

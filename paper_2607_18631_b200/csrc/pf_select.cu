@@ -191,8 +191,10 @@ __global__ void __launch_bounds__(kSelThreads) sel_hist_kernel(const __grid_cons
     }
     if (A.ctrl->take_all) return;   // nothing to refine
     const unsigned int n_list = A.ctrl->n_elig;
+    const unsigned int n_chunks = (unsigned int)((A.count + A.chunk - 1) / A.chunk);
+    (void)n_chunks;
     for (unsigned int li = blockIdx.x; li < n_list; li += gridDim.x)
-        sel_hist_chunk(P, A, vals, 1, A.elig_list[li], &s_elig);
+        sel_hist_chunk(P, A, vals, 1, (unsigned int)PF_AT(P.chk, A.elig_list[li], n_chunks, PF_SITE_CHUNK), &s_elig);
 }
 
 // Block-wide inclusive prefix sum over 1024 threads (warp shuffles, then the warp totals).
@@ -305,7 +307,7 @@ __global__ void __launch_bounds__(kSelThreads) sel_count_kernel(const __grid_con
     const uint32_t thr = A.ctrl->thr_bits;
     const uint8_t *cls = sel_guard_cls(A);
     for (unsigned int li = blockIdx.x; li < n_list; li += gridDim.x) {
-        const unsigned int chunk = A.elig_list[li];
+        const unsigned int chunk = (unsigned int)PF_AT(P.chk, A.elig_list[li], (A.count + A.chunk - 1) / A.chunk, PF_SITE_CHUNK);
         if (all) {   // every eligible candidate is taken: the first pass has counted them already
             if (threadIdx.x == 0) {
                 A.blk_gt[chunk] = A.blk_elig[chunk];
@@ -479,6 +481,7 @@ __device__ __forceinline__ void sel_write_chunk(const DevPlan &P, const SelArgs 
             for_each_eligible16(P, vals, A, cls, e, r[t], [&](uint64_t rel, uint32_t bits) {
                 if (all || bits > thr) {
                     unsigned long long pos = my_gt + (my_eq < need_eq ? my_eq : need_eq);
+                    (void)PF_AT(P.chk, pos, A.s_max, PF_SITE_SURVIVOR);
                     if (pos < A.s_max) A.surv_idx[pos] = A.first + rel;   // s_max: the list's capacity
                     my_gt++;
                 } else if (bits == thr) {
@@ -502,7 +505,8 @@ __global__ void __launch_bounds__(kSelThreads) sel_write_kernel(const __grid_con
     __shared__ unsigned long long s_run_gt, s_run_eq;
     const unsigned int n_list = A.ctrl->n_elig;
     for (unsigned int li = blockIdx.x; li < n_list; li += gridDim.x) {
-        sel_write_chunk(P, A, vals, A.elig_list[li], s_gt, s_run_gt, s_run_eq);
+        sel_write_chunk(P, A, vals, (unsigned int)PF_AT(P.chk, A.elig_list[li], (A.count + A.chunk - 1) / A.chunk, PF_SITE_CHUNK),
+                        s_gt, s_run_gt, s_run_eq);
         __syncthreads();   // the running offsets are reset by the next chunk
     }
 }

@@ -441,7 +441,8 @@ __global__ void __launch_bounds__(256) sim_records_kernel(const __grid_constant_
     r.m = (uint32_t)(S.D.m > (RI)0xFFFFFFFFu ? (RI)0xFFFFFFFFu : S.D.m);
     r.pad[0] = r.pad[1] = r.pad[2] = r.pad[3] = 0u;
     const uint4 *src = reinterpret_cast<const uint4 *>(&r);
-    uint4 *dst = reinterpret_cast<uint4 *>(A.recs + A.bin_off[bin] + base + __popc(peers & ((1u << lane) - 1u)));
+    uint4 *dst = reinterpret_cast<uint4 *>(
+        A.recs + PF_AT(P.chk, A.bin_off[bin] + base + __popc(peers & ((1u << lane) - 1u)), A.n, PF_SITE_RECORD));
 #pragma unroll
     for (int i = 0; i < 4; i++) dst[i] = src[i];
 }
@@ -473,16 +474,19 @@ __global__ void __launch_bounds__(256) sim_records_kernel(const __grid_constant_
     }
 
 // 1F1B: rank = stage = lane
+// (chk, w_lim, r_lim: the checked build's record, the timeline's length for writes, the words from the timeline's
+// start to the end of the warp's slice for reads)
 __device__ __forceinline__ void sim_rounds_1f1b(volatile float *tl, const float *durF, const float *durB, int glane,
                                                 int pp, int nj, int warm, int total_ops, float lat, int fonly,
-                                                float &clock_out, int &done_out)
+                                                float &clock_out, int &done_out, unsigned int *chk, int w_lim,
+                                                int r_lim)
 {
     // lanes beyond the pipeline depth take no part: they poll row 0 and never act
     const bool active = total_ops > 0;
     const int row = active ? glane : 0;
     const bool depF = active && row > 0, depB = active && row < pp - 1;
-    volatile float *inF = tl + (depF ? row - 1 : row) * nj, *inB = tl + (depB ? row + 1 : row) * nj;
-    volatile float *out = tl + row * nj;
+    const int offF = (depF ? row - 1 : row) * nj, offB = (depB ? row + 1 : row) * nj, offO = row * nj;
+    (void)offF; (void)offB; (void)offO; (void)chk; (void)w_lim; (void)r_lim;
     const float dF = active ? durF[row] : 0.f, dB = active ? durB[row] : 0.f;
     const float latF = depF ? lat : 0.f, latB = depB ? lat : 0.f;
     const int njl = active ? nj : 0;   // a lane beyond the pipeline depth has nothing to do
@@ -492,10 +496,10 @@ __device__ __forceinline__ void sim_rounds_1f1b(volatile float *tl, const float 
     // `fonly` steps are forward steps only (the same step as in the loop below).
     for (int i = 0; i < fonly; i++) {
         const bool want = nF < njl && nF - nB <= warm;
-        const float e = inF[nF];
+        const float e = tl[PF_AT(chk, offF + nF, r_lim, PF_SITE_TIMELINE)];
         if (want && (!depF || e > 0.f)) {
             clock = fmaxf(clock, depF ? e + latF : 0.f) + dF;
-            out[nF] = clock;
+            tl[PF_AT(chk, offO + nF, w_lim, PF_SITE_TIMELINE)] = clock;
             nF++;
         }
     }
@@ -505,19 +509,19 @@ __device__ __forceinline__ void sim_rounds_1f1b(volatile float *tl, const float 
             {   // forward step
                 // (index nF may be nj once all forwards are done: that word lies inside the warp's slice)
                 const bool want = nF < njl && nF - nB <= warm;
-                const float e = inF[nF];
+                const float e = tl[PF_AT(chk, offF + nF, r_lim, PF_SITE_TIMELINE)];
                 if (want && (!depF || e > 0.f)) {
                     clock = fmaxf(clock, depF ? e + latF : 0.f) + dF;
-                    out[nF] = clock;
+                    tl[PF_AT(chk, offO + nF, w_lim, PF_SITE_TIMELINE)] = clock;
                     nF++;
                 }
             }
             {   // backward step
                 const bool want = nB < njl && (nF - nB > warm || nF == njl);
-                const float e = inB[nB];
+                const float e = tl[PF_AT(chk, offB + nB, r_lim, PF_SITE_TIMELINE)];
                 if (want && (!depB || e < 0.f)) {
                     clock = fmaxf(clock, depB ? latB - e : 0.f) + dB;
-                    out[nB] = -clock;
+                    tl[PF_AT(chk, offO + nB, w_lim, PF_SITE_TIMELINE)] = -clock;
                     nB++;
                 }
             }
@@ -528,10 +532,10 @@ __device__ __forceinline__ void sim_rounds_1f1b(volatile float *tl, const float 
     while (__any_sync(0xFFFFFFFFu, nB < njl)) {
 #pragma unroll
         for (int rep = 0; rep < 4; rep++) {
-            const float e = inB[nB];
+            const float e = tl[PF_AT(chk, offB + nB, r_lim, PF_SITE_TIMELINE)];
             if (nB < njl && (!depB || e < 0.f)) {
                 clock = fmaxf(clock, depB ? latB - e : 0.f) + dB;
-                out[nB] = -clock;
+                tl[PF_AT(chk, offO + nB, w_lim, PF_SITE_TIMELINE)] = -clock;
                 nB++;
             }
         }
@@ -549,8 +553,10 @@ __device__ __forceinline__ void sim_rounds_1f1b(volatile float *tl, const float 
 __device__ __forceinline__ void sim_rounds_interleaved(volatile float *tl, const float *durF, const float *durB,
                                                        int glane, int pp, int v, int nj, int U, int warm,
                                                        int total_ops, float lat, int fonly, float &clock_out,
-                                                       int &done_out)
+                                                       int &done_out, unsigned int *chk, int w_lim, int r_lim,
+                                                       int q_lim)
 {
+    (void)chk; (void)w_lim; (void)r_lim; (void)q_lim;
     const int Q = pp * v;
     const bool active = total_ops > 0;
     const int row = active ? glane : 0;                    // lanes beyond the pipeline depth poll rank 0's rows
@@ -564,10 +570,10 @@ __device__ __forceinline__ void sim_rounds_interleaved(volatile float *tl, const
         const int j = fg * pp + fw;
         const int q = fc * pp + row;
         const bool dep = q > 0;
-        const float e = tl[(dep ? q - 1 : q) * nj + j];
+        const float e = tl[PF_AT(chk, (dep ? q - 1 : q) * nj + j, r_lim, PF_SITE_TIMELINE)];
         if (want && (!dep || e > 0.f)) {
-            clock = fmaxf(clock, dep ? e + lat : 0.f) + durF[q];
-            tl[q * nj + j] = clock;
+            clock = fmaxf(clock, dep ? e + lat : 0.f) + durF[PF_AT(chk, q, q_lim, PF_SITE_DURATION)];
+            tl[PF_AT(chk, q * nj + j, w_lim, PF_SITE_TIMELINE)] = clock;
             if (++fw == pp) {
                 fw = 0;
                 if (++fc == v) fc = 0, fg++;
@@ -584,10 +590,10 @@ __device__ __forceinline__ void sim_rounds_interleaved(volatile float *tl, const
                 const int j = fg * pp + fw;
                 const int q = fc * pp + row;
                 const bool dep = q > 0;
-                const float e = tl[(dep ? q - 1 : q) * nj + j];
+                const float e = tl[PF_AT(chk, (dep ? q - 1 : q) * nj + j, r_lim, PF_SITE_TIMELINE)];
                 if (want && (!dep || e > 0.f)) {
-                    clock = fmaxf(clock, dep ? e + lat : 0.f) + durF[q];
-                    tl[q * nj + j] = clock;
+                    clock = fmaxf(clock, dep ? e + lat : 0.f) + durF[PF_AT(chk, q, q_lim, PF_SITE_DURATION)];
+                    tl[PF_AT(chk, q * nj + j, w_lim, PF_SITE_TIMELINE)] = clock;
                     if (++fw == pp) {
                         fw = 0;
                         if (++fc == v) fc = 0, fg++;
@@ -600,10 +606,10 @@ __device__ __forceinline__ void sim_rounds_interleaved(volatile float *tl, const
                 const int j = bg * pp + bw;
                 const int q = (v - 1 - bc) * pp + row;
                 const bool dep = q < Q - 1;
-                const float e = tl[(dep ? q + 1 : q) * nj + j];
+                const float e = tl[PF_AT(chk, (dep ? q + 1 : q) * nj + j, r_lim, PF_SITE_TIMELINE)];
                 if (want && (!dep || e < 0.f)) {
-                    clock = fmaxf(clock, dep ? lat - e : 0.f) + durB[q];
-                    tl[q * nj + j] = -clock;
+                    clock = fmaxf(clock, dep ? lat - e : 0.f) + durB[PF_AT(chk, q, q_lim, PF_SITE_DURATION)];
+                    tl[PF_AT(chk, q * nj + j, w_lim, PF_SITE_TIMELINE)] = -clock;
                     if (++bw == pp) {
                         bw = 0;
                         if (++bc == v) bc = 0, bg++;
@@ -621,10 +627,10 @@ __device__ __forceinline__ void sim_rounds_interleaved(volatile float *tl, const
             const int j = bg * pp + bw;
             const int q = (v - 1 - bc) * pp + row;
             const bool dep = q < Q - 1;
-            const float e = tl[(dep ? q + 1 : q) * nj + j];
+            const float e = tl[PF_AT(chk, (dep ? q + 1 : q) * nj + j, r_lim, PF_SITE_TIMELINE)];
             if (nB < Ul && (!dep || e < 0.f)) {
-                clock = fmaxf(clock, dep ? lat - e : 0.f) + durB[q];
-                tl[q * nj + j] = -clock;
+                clock = fmaxf(clock, dep ? lat - e : 0.f) + durB[PF_AT(chk, q, q_lim, PF_SITE_DURATION)];
+                tl[PF_AT(chk, q * nj + j, w_lim, PF_SITE_TIMELINE)] = -clock;
                 if (++bw == pp) {
                     bw = 0;
                     if (++bc == v) bc = 0, bg++;
@@ -645,8 +651,10 @@ __device__ __forceinline__ void sim_rounds_interleaved(volatile float *tl, const
 // DualPipe-style: two directions; the per-rank order comes from the host-built table
 __device__ __forceinline__ void sim_rounds_dual(volatile float *tl, const float *durF, const float *durB, int glane,
                                                 int pp, int nj, const uint8_t *ops, int total_ops, float lat,
-                                                float &clock_out, int &done_out)
+                                                float &clock_out, int &done_out, unsigned int *chk, int w_lim,
+                                                int r_lim, int q_lim)
 {
+    (void)chk; (void)w_lim; (void)r_lim; (void)q_lim;
     int done = 0, rounds = 0;
     bool moved = false;
     float clock = 0.f;
@@ -654,18 +662,18 @@ __device__ __forceinline__ void sim_rounds_dual(volatile float *tl, const float 
 #pragma unroll
         for (int rep = 0; rep < 4; rep++)
         if (done < total_ops) {
-            const uint32_t op = __ldg(ops + done);
+            const uint32_t op = __ldg(ops + PF_AT(chk, done, total_ops, PF_SITE_DUAL_OPS));
             const bool isb = op & 1;
             const int d = (op >> 1) & 1, j = op >> 2;
             const int q = d ? pp - 1 - glane : glane;
             const int sidx = d * pp + q;
             const bool dep = isb ? (q < pp - 1) : (q > 0);
             const int nb = dep ? (isb ? sidx + 1 : sidx - 1) : sidx;
-            const float e = tl[nb * nj + j];
-            const float dur = (isb ? durB : durF)[q];
+            const float e = tl[PF_AT(chk, nb * nj + j, r_lim, PF_SITE_TIMELINE)];
+            const float dur = (isb ? durB : durF)[PF_AT(chk, q, q_lim, PF_SITE_DURATION)];
             if (!dep || (isb ? e < 0.f : e > 0.f)) {
                 clock = fmaxf(clock, dep ? fabsf(e) + lat : 0.f) + dur;
-                tl[sidx * nj + j] = isb ? -clock : clock;
+                tl[PF_AT(chk, sidx * nj + j, w_lim, PF_SITE_TIMELINE)] = isb ? -clock : clock;
                 done++;
                 moved = true;
             }
@@ -736,7 +744,8 @@ __global__ void __launch_bounds__(kSimThreads, 4) simulate_kernel(const __grid_c
         const int gidx = lane / g;
         f.have = gidx < batch && first + gidx < s_cnt[f.bin];
         if (f.have) {
-            const uint4 *src = reinterpret_cast<const uint4 *>(A.recs + s_off[f.bin] + first + gidx);
+            const uint4 *src = reinterpret_cast<const uint4 *>(
+                A.recs + PF_AT(P.chk, s_off[f.bin] + first + gidx, s_off[kSimBins], PF_SITE_RECORD));
 #pragma unroll
             for (int i = 0; i < 4; i++) f.r[i] = __ldcg(src + i);
         }
@@ -791,8 +800,9 @@ __global__ void __launch_bounds__(kSimThreads, 4) simulate_kernel(const __grid_c
                 const int ndq = max(0, min(nq_i, P.L_dense - start));    // its leading dense layers
                 const float nq = (float)(nq_i - ndq), nd = (float)ndq;
                 const bool last = q == Q - 1;
-                durF[q] = (nq * F_l + nd * F_ld + (last ? headF : 0.f)) * jitter(cand_hash, q, 0);
-                durB[q] = (nq * B_l + nd * B_ld + (last ? P.bwd_factor * headF : 0.f)) * jitter(cand_hash, q, 1);
+                const int qd = (int)PF_AT(P.chk, q, A.q_max, PF_SITE_DURATION);
+                durF[qd] = (nq * F_l + nd * F_ld + (last ? headF : 0.f)) * jitter(cand_hash, q, 0);
+                durB[qd] = (nq * B_l + nd * B_ld + (last ? P.bwd_factor * headF : 0.f)) * jitter(cand_hash, q, 1);
             }
             // clear the timeline with 16-byte stores (the slot is a multiple of four words, 16-byte aligned)
             {
@@ -816,6 +826,10 @@ __global__ void __launch_bounds__(kSimThreads, 4) simulate_kernel(const __grid_c
         }
         const int total_ops = (rank_active && run) ? 2 * U : 0;
         const float lat = run ? lat_p : 0.f;
+        // limits for the checked build: writes stay inside the candidate's own timeline, reads inside the warp's slice
+        // (a lane that has run out of ops still polls one word past its row)
+        const int w_lim = run ? n_entries : 1;
+        const int r_lim = A.warp_floats - (group_on ? gidx : 0) * E;
         // a batch's candidates share the schedule class of their bin: one specialised loop per class
         int done = 0;
         float clock = 0.f;
@@ -824,11 +838,12 @@ __global__ void __launch_bounds__(kSimThreads, 4) simulate_kernel(const __grid_c
         fonly = __reduce_min_sync(0xFFFFFFFFu, fonly);
         if (fonly == 0x7FFFFFFF) fonly = 0;
         if (bin_kind == PF_KIND_1F1B)
-            sim_rounds_1f1b(tl, durF, durB, glane, pp, nj, warm, total_ops, lat, fonly, clock, done);
+            sim_rounds_1f1b(tl, durF, durB, glane, pp, nj, warm, total_ops, lat, fonly, clock, done, P.chk, w_lim, r_lim);
         else if (bin_kind == PF_KIND_INTERLEAVED)
-            sim_rounds_interleaved(tl, durF, durB, glane, pp, v, nj, U, warm, total_ops, lat, fonly, clock, done);
+            sim_rounds_interleaved(tl, durF, durB, glane, pp, v, nj, U, warm, total_ops, lat, fonly, clock, done, P.chk,
+                                   w_lim, r_lim, A.q_max);
         else
-            sim_rounds_dual(tl, durF, durB, glane, pp, nj, dops, total_ops, lat, clock, done);
+            sim_rounds_dual(tl, durF, durB, glane, pp, nj, dops, total_ops, lat, clock, done, P.chk, w_lim, r_lim, A.q_max);
         if (done < total_ops) stalled = true;
 
         // the next batch's records are requested before this batch's results are reduced and stored
@@ -866,8 +881,9 @@ __global__ void __launch_bounds__(kSimThreads, 4) simulate_kernel(const __grid_c
                 if (m_all > (uint32_t)m_sim) T_pipe += (float)(m_all - (uint32_t)m_sim) * work;
                 tput_out = fdiv((float)(P.gbs * (i64)P.seq), (T_pipe + rest) * denom);
             }
-            if (A.tput_sim) A.tput_sim[w] = tput_out;
-            if (A.status) A.status[w] = (uint8_t)status;
+            const uint32_t wo = (uint32_t)PF_AT(P.chk, w, A.n, PF_SITE_SIM_OUT);
+            if (A.tput_sim) A.tput_sim[wo] = tput_out;
+            if (A.status) A.status[wo] = (uint8_t)status;
         }
         __syncwarp();
         cur = nxt;
