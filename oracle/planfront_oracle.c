@@ -527,9 +527,12 @@ static int eval_serve(const orc_problem_t *pb, const orc_derived_t *dv, uint64_t
 
     /* ---- memory: weights + KV cache + prefill activation workspace ---- */
     OPS(19 + 6 + 5 + 3 + 3 + 1, 0); /* weights, KV bytes per token, cache, workspace, sum, gate */
-    int64_t w = M->L * (cdiv(dv->P_dl, tp) * M->wb + dv->P_rt * M->wb +
-                        (M->E / ep) * cdiv(dv->P_e, moe_tp) * kn->wbytes) +
-                2 * cdiv(M->vocab * M->H, tp) * M->wb;
+    /* leading dense layers (DeepSeek-style stacks): attention + a plain FFN sharded by tp, no router, no experts */
+    int64_t Ld = M->L_dense, Lm = M->L - M->L_dense;
+    if (Ld > 0) OPS(6, 30);
+    int64_t w = Lm * (cdiv(dv->P_dl, tp) * M->wb + dv->P_rt * M->wb +
+                      (M->E / ep) * cdiv(dv->P_e, moe_tp) * kn->wbytes) +
+                Ld * cdiv(dv->P_dld, tp) * M->wb + 2 * cdiv(M->vocab * M->H, tp) * M->wb;
     /* the MLA latent is replicated across tensor-parallel ranks */
     int64_t kv_tok = M->attn_kind ? (M->kv_latent + M->rope_dim) * M->ab : cdiv(2 * M->nkv * M->hd, tp) * M->ab;
     int64_t kvc = b_loc * (P + O) * M->L * kv_tok;
@@ -546,7 +549,7 @@ static int eval_serve(const orc_problem_t *pb, const orc_derived_t *dv, uint64_t
     link_t lk = link_of(C, n_eng);
     double peak = C->peak_flops, hbm = C->hbm_bw, effd = K0->eff_dense;
     double tpd = (double)tp, nen = (double)n_eng, bl = (double)b_loc, dk = (double)dv->dk;
-    double nh = (double)M->nh, L = (double)M->L;
+    double nh = (double)M->nh;
     double ctx = (double)P + (double)O / 2.0;
     double attn_w = (double)(dv->P_dl * M->wb) / tpd;
     double e_per = (double)(M->E / ep);
@@ -560,7 +563,17 @@ static int eval_serve(const orc_problem_t *pb, const orc_derived_t *dv, uint64_t
                           exp_w_d / hbm);
     double t_com_d = dpa ? 2.0 * t_alltoall(n_eng, (double)M->ab * bl * (double)(M->K * M->H), lk)
                          : 2.0 * t_allreduce(tp, (double)(M->ab * Bd * M->H), lk);
-    double T_dec = L * (t_attn_d + t_moe_d + t_com_d) + K0->step_overhead;
+    /* a leading dense layer: its weights (attention + FFN) stream once per step, its FLOPs are 2 per parameter and
+     * token plus the attention core, and its two tensor-parallel all-reduces carry the tokens of this attention
+     * group; no all-to-all */
+    double t_dl_d = 0.0, t_dl_p = 0.0;
+    double w_dl = (double)(dv->P_dld * M->wb) / tpd;
+    link_t ltp = link_of(C, tp);
+    if (Ld > 0)
+        t_dl_d = fmax(bl * (2.0 * (double)dv->P_dld + 4.0 * ctx * nh * dk) / (tpd * peak * effd),
+                      (w_dl + bl * ctx * (double)kv_tok) / hbm) +
+                 2.0 * t_allreduce(tp, (double)M->ab * bl * (double)M->H, ltp);
+    double T_dec = (double)Lm * (t_attn_d + t_moe_d + t_com_d) + (double)Ld * t_dl_d + K0->step_overhead;
     int64_t nc = cdiv(P, Cc);
     double c = (double)P / (double)nc;
     double xp = c * (double)M->K / (double)ep;
@@ -571,7 +584,10 @@ static int eval_serve(const orc_problem_t *pb, const orc_derived_t *dv, uint64_t
                           exp_w_p / hbm);
     double t_com_p = dpa ? 2.0 * t_alltoall(n_eng, (double)M->ab * c * (double)(M->K * M->H), lk)
                          : 2.0 * t_allreduce(tp, (double)M->ab * c * (double)M->H, lk);
-    double T_pre = (double)nc * L * (t_attn_p + t_moe_p + t_com_p);
+    if (Ld > 0)
+        t_dl_p = fmax(c * (2.0 * (double)dv->P_dld + 4.0 * ((double)P / 2.0) * nh * dk) / (tpd * peak * effd), w_dl / hbm) +
+                 2.0 * t_allreduce(tp, (double)M->ab * c * (double)M->H, ltp);
+    double T_pre = (double)nc * ((double)Lm * (t_attn_p + t_moe_p + t_com_p) + (double)Ld * t_dl_p);
     double tput = (double)(Bd * O) / (bl * T_pre + (double)O * T_dec) / nen;
     o->tput_unpriced = tput;
     if (!kn->is_native) tput = tput / (1.0 + kn->patch_ovh);

@@ -365,3 +365,56 @@ def test_golden_files_regenerate_from_their_committed_script():
     r = subprocess.run([sys.executable, os.path.join(GOLDEN, "make_goldens.py"), "--check"], capture_output=True,
                        text=True)
     assert r.returncode == 0, r.stdout + r.stderr
+
+
+# ----------------------------------------------------------------------------- serving with leading dense layers
+
+def hand_serve_dense() -> dict:
+    """hand_serve() with three layers of which the first carries a plain FFN of width 2048 instead of experts:
+    attention 4,194,304 + FFN 3 x 1024 x 2048 = 10,485,760 parameters, 20 x 2^20 bytes in bf16."""
+    cfg = hand_serve()
+    cfg["model"].update(L=3, L_dense=1, F_dense=2048)
+    return cfg
+
+
+def test_serving_leading_dense_layer_hand_computed():
+    """tp = ep = 1, one request, prompt 4096, output 512, chunk 4096 (u = 2^-20 s).
+    Memory: two MoE layers 2 x 33,570,816 B + the dense layer 20,971,520 B + embedding and head 4,096,000 B =
+    92,209,152 B of weights; KV cache 4608 tokens x 3 layers x 4,096 B = 56,623,104; workspace 67,108,864;
+    total 215,941,120 B.
+    Decode: a MoE layer streams 31 u as before; the dense layer streams its 20 x 2^20 B of weights and the 17 x 2^20 B
+    of KV cache: 37 u.  T_dec = 2 x 31 + 37 = 99 u.
+    Prefill: a MoE layer 176 u as before; the dense layer 4096 x (2 x 10,485,760 + 4 x 2048 x 8 x 128) = 28 x 2^32
+    FLOPs at 2^49 = 224 u (its weights stream in 20 u: compute-bound).  T_pre = 2 x 176 + 224 = 576 u.
+    Throughput 512 x 2^20 / (576 + 512 x 99) = 512 x 2^20 / 51,264."""
+    cfg = hand_serve_dense()
+    d = Oracle(cfg).eval(axis_index(cfg, kv=0, chunk=4096, batch=1, dpa=0, ep=1, tp=1, scen=0))
+    assert d["reason"] & 0x7F == 0
+    assert d["bytes_w"] == 92_209_152 and d["mem"] == 215_941_120
+    assert d["T_dec"] == pytest.approx(99 * U, rel=1e-13)
+    assert d["T_pre"] == pytest.approx(576 * U, rel=1e-13)
+    assert d["tput"] == pytest.approx(512 * 2 ** 20 / 51264, rel=1e-13)
+
+
+def test_serving_leading_dense_layer_is_sharded_and_all_reduced_over_tp():
+    """tp = 2 without dp-attention, two requests, prompt 1024, output 512, chunk 1024.  The dense layer's weights
+    halve (10 u), its KV reads are those of the MoE layers (2 x 1280 x 2,048 B = 5 u), and its two all-reduces of
+    the two requests' activations cost 2 x (4 u + 2 u) = 12 u like a MoE layer's: 27 u.  T_dec = 2 x 27 + 27 = 81 u.
+    Weights per GPU: 2 x (4,194,304 + 16,384 + 8 x 1,572,864) + 10,485,760 + 2,048,000 = 33,587,200 + 12,533,760 =
+    46,120,960 B."""
+    cfg = hand_serve_dense()
+    d = Oracle(cfg).eval(axis_index(cfg, kv=0, chunk=1024, batch=2, dpa=0, ep=1, tp=2, scen=1))
+    assert d["reason"] & 0x7F == 0
+    assert d["bytes_w"] == 46_120_960
+    assert d["T_dec"] == pytest.approx(81 * U, rel=1e-13)
+
+
+def test_serving_without_dense_layers_is_unchanged_by_the_dense_fields():
+    """L_dense = 0: the width of a dense FFN that no layer has changes nothing, to the bit."""
+    a, b = hand_serve(), hand_serve()
+    b["model"].update(F_dense=4096)
+    ra, ta, ma, _ = Oracle(a).score_range()
+    rb, tb, mb, _ = Oracle(b).score_range()
+    np.testing.assert_array_equal(ra, rb)
+    np.testing.assert_array_equal(ta, tb)
+    np.testing.assert_array_equal(ma, mb)
