@@ -99,9 +99,8 @@ typedef struct {
     int32_t wb, gb, ob, ab;       /* bytes per weight / gradient / optimizer state per param / activation */
     int32_t n_mats;               /* matrices per expert FFN (3 = gate, up, down) */
     int32_t count_embeddings;     /* 0/1: embedding + head counted in memory */
-    /* DeepSeek-style stacks (training plans only; 0 = not used): the first L_dense layers carry a plain FFN of
-     * width F_dense instead of experts; hd_q: query head dimension where it differs from hd (latent attention:
-     * nope + rope dims) */
+    /* DeepSeek-style stacks (0 = not used): the first L_dense layers carry a plain FFN of width F_dense instead
+     * of experts; hd_q: query head dimension where it differs from hd (latent attention: nope + rope dims) */
     int32_t L_dense, F_dense, hd_q;
 } pf_model_t;
 

@@ -200,7 +200,6 @@ extern "C" int pf_plan_create(const pf_model_t *model, const pf_cluster_t *clust
     if (M.S < 0 || (M.S > 0 && M.Fs <= 0) || M.K > M.E) return PF_EINVAL;
     if (M.L_dense < 0 || M.L_dense >= M.L || (M.L_dense > 0 && M.F_dense <= 0) || M.F_dense < 0 || M.hd_q < 0)
         return PF_EINVAL;
-    if (M.L_dense > 0 && phase == PF_PHASE_SERVE) return PF_EUNSUPPORTED;  // leading dense layers: training plans only
     if (M.attn_kind == 0 ? M.nkv <= 0 : (M.kv_latent <= 0 || M.rope_dim < 0)) return PF_EINVAL;
     if (cluster->G <= 0 || cluster->budget_bytes < 0 || cluster->reserved_bytes < 0) return PF_EINVAL;
     if (!(cluster->peak_flops > 0) || !(cluster->hbm_bw > 0) || !(cluster->bw_intra > 0) || !(cluster->bw_inter > 0))

@@ -436,9 +436,11 @@ __device__ __forceinline__ void serve_eval(const DevPlan &P, const ServeTuple &c
     }
     // memory: weights + KV cache + prefill workspace
     const i64 tp = c.tp;
-    const i64 w = (i64)P.L * (cdiv64(P.P_dl, tp) * P.wb + P.P_rt * P.wb +
-                              (i64)(P.E / c.ep) * cdiv64(P.P_e, moe_tp) * kn.wbytes) +
-                  2 * cdiv64((i64)P.vocab * P.H, tp) * P.wb;
+    // leading dense layers carry attention + a plain FFN sharded by tp: no router, no experts
+    const i64 Ld = P.L_dense, Lm = P.L - P.L_dense;
+    i64 w = Lm * (cdiv64(P.P_dl, tp) * P.wb + P.P_rt * P.wb + (i64)(P.E / c.ep) * cdiv64(P.P_e, moe_tp) * kn.wbytes) +
+            2 * cdiv64((i64)P.vocab * P.H, tp) * P.wb;
+    if (Ld > 0) w += Ld * cdiv64(P.P_dld, tp) * P.wb;
     const i64 kv_tok = P.attn_kind ? (i64)(P.kv_latent + P.rope_dim) * P.ab : cdiv64(2ll * P.nkv * P.hd, tp) * P.ab;
     const i64 kvc = (i64)b_loc * (i64)(Pn + On) * P.L * kv_tok;
     const i64 act = 8ll * P.ab * c.chunk * P.H;
@@ -451,7 +453,7 @@ __device__ __forceinline__ void serve_eval(const DevPlan &P, const ServeTuple &c
     const Link lk = link_of(P, n_eng);
     const float peak = P.peak_flops, hbm = P.hbm_bw;
     const float ftp = (float)c.tp, nen = (float)n_eng, bl = (float)b_loc, dk = (float)P.dk, nh = (float)P.nh;
-    const float Lf = (float)P.L, Pf = (float)Pn, Of = (float)On;
+    const float Lf = (float)Lm, Pf = (float)Pn, Of = (float)On;
     const float P_dl = (float)P.P_dl;
     const float dense_rate = ftp * peak * P.eff_dense;
     const float ctx = Pf + Of * 0.5f;
@@ -466,7 +468,14 @@ __device__ __forceinline__ void serve_eval(const DevPlan &P, const ServeTuple &c
     const float t_moe_d = fmaxf(fdiv((float)c.batch * P.f_exp, moe_rate * kn.eff[b]), fdiv(touched_d * exp_unit, hbm));
     const float t_com_d = c.dpa ? 2.f * t_alltoall(n_eng, (float)P.ab * bl * KH, lk)
                                 : 2.f * t_allreduce(c.tp, (float)((i64)P.ab * c.batch * P.H), lk);
-    const float T_dec = Lf * (t_attn_d + t_moe_d + t_com_d) + P.step_overhead;
+    // a leading dense layer: its weights stream once per step, two all-reduces over tp, no all-to-all
+    float t_dl_d = 0.f, t_dl_p = 0.f;
+    const float P_dld = (float)P.P_dld, w_dl = fdiv((float)(P.P_dld * P.wb), ftp);
+    const Link ltp = link_of(P, c.tp);
+    if (Ld > 0)
+        t_dl_d = fmaxf(fdiv(bl * (2.f * P_dld + 4.f * ctx * nh * dk), dense_rate), fdiv(w_dl + bl * ctx * (float)kv_tok, hbm)) +
+                 2.f * t_allreduce(c.tp, (float)P.ab * bl * (float)P.H, ltp);
+    const float T_dec = Lf * (t_attn_d + t_moe_d + t_com_d) + (float)Ld * t_dl_d + P.step_overhead;
     // chunked prefill
     const int nc = (Pn + c.chunk - 1) / c.chunk;
     const float cl = fdiv(Pf, (float)nc);
@@ -475,7 +484,10 @@ __device__ __forceinline__ void serve_eval(const DevPlan &P, const ServeTuple &c
     const float t_moe_p = fmaxf(fdiv(cl * P.f_exp, moe_rate * kn.eff[b_pre]), fdiv(touched_p * exp_unit, hbm));
     const float t_com_p = c.dpa ? 2.f * t_alltoall(n_eng, (float)P.ab * cl * KH, lk)
                                 : 2.f * t_allreduce(c.tp, (float)P.ab * cl * (float)P.H, lk);
-    const float T_pre = (float)nc * Lf * (t_attn_p + t_moe_p + t_com_p);
+    if (Ld > 0)
+        t_dl_p = fmaxf(fdiv(cl * (2.f * P_dld + 4.f * (Pf * 0.5f) * nh * dk), dense_rate), fdiv(w_dl, hbm)) +
+                 2.f * t_allreduce(c.tp, (float)P.ab * cl * (float)P.H, ltp);
+    const float T_pre = (float)nc * (Lf * (t_attn_p + t_moe_p + t_com_p) + (float)Ld * t_dl_p);
     float tput = fdiv((float)((i64)c.batch * On), (bl * T_pre + Of * T_dec) * nen);
     if (!kn.is_native) tput = fdiv(tput, 1.f + kn.patch_ovh);
     out.tput = tput;

@@ -96,7 +96,21 @@ def test_invalid_dense_layer_inputs():
     cfg["model"].update(L_dense=1, F_dense=0)
     with pytest.raises(PlanfrontError):
         _plan(cfg)
+
+
+@pytest.mark.parametrize("l_dense,f_dense,hd_q", [(1, 12288, 0), (3, 18432, 192), (47, 1024, 0)])
+def test_serving_space_with_leading_dense_layers(l_dense, f_dense, hd_q):
+    """The serving space with the first layers dense (and a separate query width): every candidate and the per-plan
+    aggregate against the oracle."""
+    import torch
     cfg = make_config("serve")
-    cfg["model"].update(L_dense=1, F_dense=1024)
-    with pytest.raises(PlanfrontError):
-        _plan(cfg)
+    cfg["model"].update(L_dense=l_dense, F_dense=f_dense, hd_q=hd_q)
+    plan, orc = _plan(cfg), Oracle(cfg)
+    res = gpu_score(plan, k=128)
+    reason, tput, mem, _ = orc.score_range(threads=16)
+    compare_dense(res, reason, tput, mem)
+    compare_topk(res, orc, reason, tput, 0, 128)
+    assert ((reason & 0x7F) == 0).sum() > 10_000
+    base = Oracle(make_config("serve")).score_range(threads=16)
+    assert not np.array_equal(base[2], mem)                  # the dense layers do change the byte counts
+    plan.close()

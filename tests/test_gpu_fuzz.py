@@ -127,6 +127,11 @@ def random_serving_space(seed: int) -> dict:
     for k in cfg["kern"]:
         k["avail_mask"] = int(rng.integers(1, 256))
     cfg["domain"].update(m_lo=int(rng.choice([1, 64])), m_hi=int(rng.choice([16, 8192])))
+    # drawn last, so that the spaces above keep their earlier draws: leading dense layers and a query head width
+    if rng.random() < 0.5:
+        m["L_dense"] = int(rng.choice([1, 3]))
+        m["F_dense"] = int(rng.choice([4096, 12288]))
+        m["hd_q"] = int(rng.choice([0, 192]))
     return cfg
 
 
