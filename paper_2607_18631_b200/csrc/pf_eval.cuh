@@ -162,13 +162,21 @@ __device__ __forceinline__ int train_plan_rules(const DevPlan &P, const TrainTup
     D.Q = Q;
     D.Lc = (P.L + Q - 1) / Q;
     D.Ls = v_eff * D.Lc;
-    // stage q covers layers [q Lc, (q+1) Lc); rank r holds stages r, r + pp, ...
+    // Stage q covers layers [q Lc, (q+1) Lc) and rank r holds stages r, r + pp, ...: its chunks start every
+    // pp Lc layers from layer r Lc.  Of the L_dense leading layers the rank's chunks before the last one reached are
+    // dense throughout, that one as far as the dense layers go.
     D.nd0 = D.nd_last = 0;
-    if (P.L_dense > 0)
-        for (int cc = 0; cc < v_eff; cc++) {
-            D.nd0 += max(0, min(D.Lc, P.L_dense - cc * c.pp * D.Lc));
-            D.nd_last += max(0, min(D.Lc, P.L_dense - (cc * c.pp + c.pp - 1) * D.Lc));
-        }
+    if (P.L_dense > 0) {
+        const int stride = c.pp * D.Lc;
+        auto dense_on_rank = [&](int first_layer) {
+            const int left = P.L_dense - first_layer;          // dense layers from the rank's first chunk on
+            if (left <= 0) return 0;
+            const int whole = left / stride, rest = left - whole * stride;
+            return whole >= v_eff ? v_eff * D.Lc : whole * D.Lc + min(rest, D.Lc);
+        };
+        D.nd0 = dense_on_rank(0);
+        D.nd_last = dense_on_rank((c.pp - 1) * D.Lc);
+    }
     if (kind == PF_KIND_INTERLEAVED) {
         if (m % (RI)c.pp != 0) return PF_R_MICROBATCH;
     } else if (kind == PF_KIND_DUALPIPE) {
