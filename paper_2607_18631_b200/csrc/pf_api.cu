@@ -425,6 +425,7 @@ extern "C" int pf_plan_create(const pf_model_t *model, const pf_cluster_t *clust
         if (e == cudaSuccess)
             e = cudaMemcpy(p->d_scen + n, workload->scen_O, sizeof(int32_t) * n, cudaMemcpyHostToDevice);
     }
+    if (e == cudaSuccess) e = cudaMalloc((void **)&p->d_fill_ctl, 2048);
     if (e == cudaSuccess) e = cudaMalloc((void **)&p->d_check, 64);
     if (e == cudaSuccess) e = cudaMemset(p->d_check, 0, 64);
     d.chk = p->d_check;
@@ -454,6 +455,7 @@ extern "C" int pf_plan_create(const pf_model_t *model, const pf_cluster_t *clust
         if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->ev_join, cudaEventDisableTiming);
         if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->ev_fill, cudaEventDisableTiming);
         if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->ev_fork2, cudaEventDisableTiming);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->ev_fork3, cudaEventDisableTiming);
         if (e != cudaSuccess) {
             pf::set_cuda_error(e, "pf_plan_create: side stream");
             pf_plan_destroy(p);
@@ -536,9 +538,10 @@ extern "C" int pf_check_read(pf_plan_t *p, uint32_t *out)
 #endif
 }
 
-extern "C" int pf_bench_fill_span(pf_plan_t *p, uint64_t *n_blocks, uint64_t *block_candidates, uint64_t *scored_blocks)
+extern "C" int pf_bench_fill_span(pf_plan_t *p, uint64_t *n_blocks, uint64_t *block_candidates, uint64_t *scored_blocks,
+                                  uint64_t *early_fill_blocks)
 {
-    if (!p || !n_blocks || !block_candidates || !scored_blocks || !p->d_order) return PF_EINVAL;
+    if (!p || !n_blocks || !block_candidates || !scored_blocks || !early_fill_blocks || !p->d_order) return PF_EINVAL;
     if (int rc_dev = pf::check_device(p)) return rc_dev;
     uint32_t hdr[8] = {0};
     PF_CUDA_TRY(cudaDeviceSynchronize(), "pf_bench_fill_span");
@@ -546,6 +549,9 @@ extern "C" int pf_bench_fill_span(pf_plan_t *p, uint64_t *n_blocks, uint64_t *bl
     *n_blocks = hdr[2];
     *block_candidates = p->dev.slab;
     *scored_blocks = hdr[4];
+    uint32_t ctl[4] = {0};
+    PF_CUDA_TRY(cudaMemcpy(ctl, p->d_fill_ctl, sizeof(ctl), cudaMemcpyDeviceToHost), "pf_bench_fill_span");
+    *early_fill_blocks = ctl[2];
     return PF_OK;
 }
 
@@ -566,10 +572,12 @@ extern "C" void pf_plan_destroy(pf_plan_t *p)
     if (p->d_scen) cudaFree(p->d_scen);
     if (p->d_order) cudaFree(p->d_order);
     if (p->d_check) cudaFree(p->d_check);
+    if (p->d_fill_ctl) cudaFree(p->d_fill_ctl);
     if (p->ev_fork) cudaEventDestroy(p->ev_fork);
     if (p->ev_join) cudaEventDestroy(p->ev_join);
     if (p->ev_fill) cudaEventDestroy(p->ev_fill);
     if (p->ev_fork2) cudaEventDestroy(p->ev_fork2);
+    if (p->ev_fork3) cudaEventDestroy(p->ev_fork3);
     if (p->side_stream) cudaStreamDestroy(p->side_stream);
     if (p->fill_stream) cudaStreamDestroy(p->fill_stream);
     free(p->h_vals);

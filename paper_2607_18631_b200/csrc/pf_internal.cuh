@@ -17,15 +17,21 @@ constexpr int kInnerVals = 1024;     // inner-axis values the scoring kernel kee
 constexpr int kOrderMaxSlabs = 1 << 20;  // calls with more slabs visit them by a permutation instead of an order table
 constexpr int kTailFillsPerBlock = 4;    // constant-fill slabs per block kept, at least, for the end of the visiting order
 constexpr int kFillsPerEvaluated = 3;    // fills interleaved per evaluated slab at the start of the visiting order (measured: 1: 0.392 ms, 2: 0.384, 3: 0.380, 4: 0.379, 6: 0.382, 8: 0.385, 12: 0.396)
-// Inside a search call a kernel of its own streams the constant slabs beside the simulator kernel.  Measured on
-// the benchmark's space (step time; simulator kernel / fill kernel durations while they overlap): 256 threads per
-// SM 0.651 ms (0.38 / 0.31), 128: 0.583 (0.32 / 0.29), 96: 0.578 (0.26 / 0.33), 64: 0.630 (0.25 / 0.35), 32: 0.88
-// (0.24 / 0.60) -- more store warps crowd the simulator's shared-memory polling out of the load/store pipe, fewer
-// cannot keep HBM busy.  Fills interleaved with the evaluated slabs of the scoring kernel only move time from
-// one kernel to the other (0, 2, 3, 4 per evaluated slab: 0.578, 0.582, 0.587, 0.590 ms).
+// Inside a search call a kernel of its own streams the constant slabs on the plan's fill stream, in two launches
+// that share one queue: a narrow one from the start of the call (beside the scoring kernel, the selection and the
+// simulator's pre-pass, which are latency-bound and stall under a saturated store stream), and a wide one beside the
+// simulator kernel, which works in shared memory.  Measured on the benchmark's space, step time with the wide launch
+// alone at 256 / 128 / 96 / 64 / 32 threads per SM: 0.651 / 0.583 / 0.578 / 0.630 / 0.88 ms (more store warps crowd
+// the simulator's shared-memory polling out of the load/store pipe, fewer cannot keep HBM busy); with the narrow
+// launch added at 64 / 96 / 128 / 160 / 192 / 256 threads per SM: 0.547 / 0.531 / 0.523 / 0.521 / 0.525 / 0.529 ms.
+// Fills interleaved with the evaluated slabs inside the scoring kernel only move time from one kernel to the other
+// (0, 2, 3, 4 per evaluated slab: 0.578, 0.582, 0.587, 0.590 ms without the narrow launch).
 constexpr int kFillsPerEvaluatedSplit = 0;
 constexpr int kFillBlocksPerSm = 1;
-constexpr int kFillThreads = 96;
+constexpr int kFillThreads = 96;         // the wide launch
+constexpr int kFillEarlyThreads = 160;   // the narrow launch: one block per SM, its stores paced by the other work
+constexpr int kFillGridPerSm = 32;       // blocks launched per SM: the grid covers every SM however the hardware
+                                         // places it; a block works only if it is among the first on its SM
 constexpr int kQueueCap = 4096;   // cost-model queue of the scoring kernel (entries), drained when it may fill up
 
 struct DevSched {
@@ -144,9 +150,10 @@ struct pf_plan {
     // the survivor selection and the simulator.  Streams and fork / join events belong to the plan (training
     // plans; created with the plan).
     cudaStream_t side_stream, fill_stream;
-    cudaEvent_t ev_fork, ev_join, ev_fork2, ev_fill;
+    cudaEvent_t ev_fork, ev_join, ev_fork2, ev_fork3, ev_fill;
     // simulator order tables (built at create for training plans)
     void *sim_tables;
+    unsigned int *d_fill_ctl;      // queue head and per-SM block counts of the fill kernels (2 KB)
     unsigned int *d_check;         // the checked build's record (dev.chk); 64 bytes, zero unless a check fired
     // optional per-kernel-class event timing (pf_timing_enable)
     void *timing;
@@ -365,6 +372,11 @@ struct FillArgs {
     float *tput;
     long long *mem;
     const uint32_t *order, *order_hdr;
+    // the queue of constant slabs and the per-SM registration of the kernel's blocks (plan-owned, zeroed per call)
+    unsigned int *ticket, *sm_slots;
+    const unsigned int *stop;      // may be NULL; once the word is non-zero the launch draws no further slab
+    unsigned int *done;            // counts the slabs the launch has filled
+    uint32_t per_sm;               // working blocks per SM
 };
 
 // How a scoring call may spread over the plan's streams (all off: one stream, one scoring kernel).

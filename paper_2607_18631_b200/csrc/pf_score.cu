@@ -646,10 +646,44 @@ __global__ void __launch_bounds__(kThreads, 4) score_kernel(const __grid_constan
 // blocks take them round robin (they are all the same size but for a clipped first or last one).
 __global__ void __launch_bounds__(kThreads) fill_tail_kernel(const FillArgs A)
 {
+    // Where the hardware puts the blocks of a small grid that starts beside other kernels is not even: launched
+    // early, most of a one-block-per-SM grid was seen to land on a few SMs, whose store rate then bounded the whole
+    // kernel.  So the grid is oversubscribed and a block works only if it is among the first `per_sm` to register
+    // on its SM; the others leave at once, and the scheduler keeps placing blocks until every SM has its share.
+    __shared__ unsigned int s_go, s_t;
+    const uint32_t tid = threadIdx.x;
+    if (tid == 0) {
+        unsigned int smid;
+        asm("mov.u32 %0, %%smid;" : "=r"(smid));
+        s_go = atomicAdd(A.sm_slots + (smid & 255u), 1u) < A.per_sm ? 1u : 0u;
+        if (s_go) s_t = atomicAdd(A.ticket, 1u);
+    }
+    __syncthreads();
+    if (!s_go) return;
     if (!order_table_valid(A.order_hdr, A.slab_lo, A.n_slabs, A.order_tail, A.order_fpe)) return;
     const uint32_t head_n = A.order_hdr[4];
-    for (uint32_t t = head_n + blockIdx.x; t < A.n_slabs; t += gridDim.x) {
-        const uint32_t w = __ldg(A.order + t);
+    for (;;) {
+        const uint32_t tk = s_t;
+        __syncthreads();
+        if (head_n + tk >= A.n_slabs) break;
+        if (A.stop && *reinterpret_cast<const volatile unsigned int *>(A.stop) != 0u) {
+            // the slab this block had drawn goes back to whoever takes over: it is filled here, then the block leaves
+            // (one slab per block at most: cheaper than handing tickets back)
+            const uint32_t w = __ldg(A.order + head_n + tk);
+            const uint64_t base = (A.slab_lo + (w & 0xFFFFFFu)) * (uint64_t)A.slab;
+            const uint64_t lo = base > A.first ? base : A.first;
+            const uint64_t end_slab = base + A.slab, end_call = A.first + A.count;
+            const uint64_t hi = end_slab < end_call ? end_slab : end_call;
+            const uint64_t rel0 = lo - A.first, n = hi - lo;
+            if (A.reason) block_fill(A.reason + rel0, n, w >> 24);
+            if (A.tput) block_fill(reinterpret_cast<uint8_t *>(A.tput + rel0), n * 4, 0u);
+            if (A.mem) block_fill(reinterpret_cast<uint8_t *>(A.mem + rel0), n * 8, 0u);
+            if (tid == 0) atomicAdd(A.done, 1u);
+            break;
+        }
+        uint32_t tk_next = 0;
+        if (tid == 0) tk_next = atomicAdd(A.ticket, 1u);   // in flight while this slab is stored
+        const uint32_t w = __ldg(A.order + head_n + tk);
         const uint64_t base = (A.slab_lo + (w & 0xFFFFFFu)) * (uint64_t)A.slab;
         const uint64_t lo = base > A.first ? base : A.first;
         const uint64_t end_slab = base + A.slab, end_call = A.first + A.count;
@@ -658,6 +692,11 @@ __global__ void __launch_bounds__(kThreads) fill_tail_kernel(const FillArgs A)
         if (A.reason) block_fill(A.reason + rel0, n, w >> 24);
         if (A.tput) block_fill(reinterpret_cast<uint8_t *>(A.tput + rel0), n * 4, 0u);
         if (A.mem) block_fill(reinterpret_cast<uint8_t *>(A.mem + rel0), n * 8, 0u);
+        if (tid == 0) {
+            s_t = tk_next;
+            atomicAdd(A.done, 1u);   // slabs this launch has filled (accounting only)
+        }
+        __syncthreads();
     }
 }
 
@@ -950,11 +989,20 @@ int fill_launch(pf_plan_t *p, ScoreSpread &sp, cudaStream_t st)
     if (!sp.fill_deferred) return PF_OK;
     sp.fill_deferred = false;
     cudaStream_t fs = p->fill_stream;
+    // tell an early, narrow fill launch to draw no further slab: the wide one takes the queue over
+    PF_CUDA_TRY(cudaMemsetAsync(p->d_fill_ctl + 1, 0xFF, 4, st), "fill hand-over");
     PF_CUDA_TRY(cudaEventRecord(p->ev_fork2, st), "fill fork");
     PF_CUDA_TRY(cudaStreamWaitEvent(fs, p->ev_fork2, 0), "fill fork");
     // from here on the fill stream is forked: record the join event whatever happens
     timing_begin(p, PF_T_FILL, fs);
-    fill_tail_kernel<<<p->sm_count * kFillBlocksPerSm, kFillThreads, 0, fs>>>(sp.fill);
+    {
+        FillArgs f = sp.fill;
+        f.stop = nullptr;                      // this launch empties the queue
+        f.done = p->d_fill_ctl + 3;
+        f.sm_slots = p->d_fill_ctl + 256 + 16;
+        f.per_sm = kFillBlocksPerSm;
+        fill_tail_kernel<<<p->sm_count * kFillGridPerSm, kFillThreads, 0, fs>>>(f);
+    }
     count_launch();
     timing_end(p, PF_T_FILL, 1, fs);
     const cudaError_t e = cudaGetLastError();
@@ -1081,6 +1129,33 @@ int pf::score_run(pf_plan_t *p, uint64_t first, uint64_t count, uint8_t *d_reaso
         a.order_hdr = hdr;
         a.head_only = split ? 1u : 0u;
     }
+    if (split) {
+        // The constant slabs start to stream at once, by a narrow launch of the fill kernel on the plan's fill
+        // stream that runs beside the scoring kernel, the selection and the simulator's pre-pass -- slowly, because
+        // those are latency-bound and a saturated store stream would stall them -- until the wide launch takes the
+        // queue over (fill_launch).  Queue head, hand-over word and block registrations start at zero.
+        PF_CUDA_TRY(cudaMemsetAsync(p->d_fill_ctl, 0, 2048, st), "fill control reset");
+        FillArgs &f = sp.fill;
+        f.first = first; f.count = count; f.slab_lo = slab_lo; f.n_slabs = (uint32_t)n_slabs;
+        f.slab = p->dev.slab; f.order_tail = a.order_tail; f.order_fpe = a.order_fpe;
+        f.reason = d_reason; f.tput = d_tput; f.mem = (long long *)d_mem;
+        f.order = a.order; f.order_hdr = a.order_hdr;
+        f.ticket = p->d_fill_ctl; f.stop = p->d_fill_ctl + 1; f.done = p->d_fill_ctl + 2;
+        f.sm_slots = p->d_fill_ctl + 16; f.per_sm = 1;
+        PF_CUDA_TRY(cudaEventRecord(p->ev_fork3, st), "early fill fork");
+        PF_CUDA_TRY(cudaStreamWaitEvent(p->fill_stream, p->ev_fork3, 0), "early fill fork");
+        timing_begin(p, PF_T_FILL_EARLY, p->fill_stream);
+        fill_tail_kernel<<<p->sm_count * kFillGridPerSm, kFillEarlyThreads, 0, p->fill_stream>>>(f);
+        count_launch();
+        timing_end(p, PF_T_FILL_EARLY, 1, p->fill_stream);
+        const cudaError_t e_early = cudaGetLastError();
+        // the fill stream is forked from here on: the join event is recorded whatever happens next
+        if (cudaEventRecord(p->ev_fill, p->fill_stream) == cudaSuccess) sp.fill_pending = true;
+        if (e_early != cudaSuccess) {
+            set_cuda_error(e_early, "fill_tail_kernel launch");
+            return PF_ECUDA;
+        }
+    }
     const size_t queue_bytes = p->dev.phase == PF_PHASE_TRAIN
                                    ? (((size_t)p->dev.slab + 16 + 15) & ~(size_t)15) + kQueueCap * sizeof(uint16_t)
                                    : 0;
@@ -1102,13 +1177,8 @@ int pf::score_run(pf_plan_t *p, uint64_t first, uint64_t count, uint8_t *d_reaso
     int rc = PF_OK;
     if (topk_aside) PF_CUDA_TRY(cudaEventRecord(p->ev_fork, st), "score fork");
     if (split) {
-        // the caller decides when the constant slabs start to stream (fill_launch): until then, and while they do,
-        // only the evaluated slabs of the dense outputs hold results (guard)
-        FillArgs &f = sp.fill;
-        f.first = first; f.count = count; f.slab_lo = slab_lo; f.n_slabs = (uint32_t)n_slabs;
-        f.slab = p->dev.slab; f.order_tail = a.order_tail; f.order_fpe = a.order_fpe;
-        f.reason = d_reason; f.tput = d_tput; f.mem = (long long *)d_mem;
-        f.order = a.order; f.order_hdr = a.order_hdr;
+        // the caller decides when the wide fill launch takes over (fill_launch); until the fills have joined, only
+        // the evaluated slabs of the dense outputs hold results (guard)
         sp.fill_deferred = true;
         sp.guard.cls = (const uint8_t *)(a.order + p->order_cap);
         sp.guard.hdr = a.order_hdr;

@@ -55,7 +55,8 @@ def main():
         span = plan.fill_span()
         fill = (span["n_blocks"] - span["scored_blocks"]) * span["block_candidates"]
         print(f"searched {plan.size} candidates; {int(bufs['surv_count'].item())} survivors; the fill kernel covers "
-              f"{fill} candidates ({span['n_blocks'] - span['scored_blocks']} of {span['n_blocks']} blocks)")
+              f"{fill} candidates ({span['n_blocks'] - span['scored_blocks']} of {span['n_blocks']} blocks, "
+              f"{span['early_fill_blocks']} of them in its first launch)")
     else:
         print(f"scored {plan.size} candidates; top-k holds {int(out['topk_count'].item())}"
               + (f"; {int(sel['surv_count'].item())} survivors" if sel is not None else ""))
