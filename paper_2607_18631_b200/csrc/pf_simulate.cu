@@ -506,10 +506,15 @@ __device__ __forceinline__ void sim_rounds_1f1b(volatile float *tl, const float 
     for (;;) {
 #pragma unroll
         for (int rep = 0; rep < 2; rep++) {
+            // both polls are issued before either step runs, so that their shared-memory latencies overlap (the
+            // backward step's dependency is another lane's word: reading it a few instructions early only means a
+            // value that arrives in between is seen one iteration later)
+            // (index nF may be nj once all forwards are done: that word lies inside the warp's slice)
+            const float eF = tl[PF_AT(chk, offF + nF, r_lim, PF_SITE_TIMELINE)];
+            const float eB = tl[PF_AT(chk, offB + nB, r_lim, PF_SITE_TIMELINE)];
             {   // forward step
-                // (index nF may be nj once all forwards are done: that word lies inside the warp's slice)
                 const bool want = nF < njl && nF - nB <= warm;
-                const float e = tl[PF_AT(chk, offF + nF, r_lim, PF_SITE_TIMELINE)];
+                const float e = eF;
                 if (want && (!depF || e > 0.f)) {
                     clock = fmaxf(clock, depF ? e + latF : 0.f) + dF;
                     tl[PF_AT(chk, offO + nF, w_lim, PF_SITE_TIMELINE)] = clock;
@@ -518,7 +523,7 @@ __device__ __forceinline__ void sim_rounds_1f1b(volatile float *tl, const float 
             }
             {   // backward step
                 const bool want = nB < njl && (nF - nB > warm || nF == njl);
-                const float e = tl[PF_AT(chk, offB + nB, r_lim, PF_SITE_TIMELINE)];
+                const float e = eB;
                 if (want && (!depB || e < 0.f)) {
                     clock = fmaxf(clock, depB ? latB - e : 0.f) + dB;
                     tl[PF_AT(chk, offO + nB, w_lim, PF_SITE_TIMELINE)] = -clock;
@@ -584,6 +589,9 @@ __device__ __forceinline__ void sim_rounds_interleaved(volatile float *tl, const
     for (;;) {
 #pragma unroll
         for (int rep = 0; rep < 2; rep++) {
+            // both polls first (see the 1F1B loop), then the two steps
+            const int jB0 = bg * pp + bw, qB0 = (v - 1 - bc) * pp + row;
+            const float eB0 = tl[PF_AT(chk, (qB0 < Q - 1 ? qB0 + 1 : qB0) * nj + jB0, r_lim, PF_SITE_TIMELINE)];
             {   // forward step: unit (fg, fc, fw) = microbatch fg pp + fw of chunk fc
                 // (j may be nj once all forwards are done: that word lies inside the warp's slice)
                 const bool want = nF < Ul && nF - nB <= warm;
@@ -603,10 +611,10 @@ __device__ __forceinline__ void sim_rounds_interleaved(volatile float *tl, const
             }
             {   // backward step: chunks walk downward
                 const bool want = nB < Ul && (nF - nB > warm || nF == Ul);
-                const int j = bg * pp + bw;
-                const int q = (v - 1 - bc) * pp + row;
+                const int j = jB0;
+                const int q = qB0;
                 const bool dep = q < Q - 1;
-                const float e = tl[PF_AT(chk, (dep ? q + 1 : q) * nj + j, r_lim, PF_SITE_TIMELINE)];
+                const float e = eB0;
                 if (want && (!dep || e < 0.f)) {
                     clock = fmaxf(clock, dep ? lat - e : 0.f) + durB[PF_AT(chk, q, q_lim, PF_SITE_DURATION)];
                     tl[PF_AT(chk, q * nj + j, w_lim, PF_SITE_TIMELINE)] = -clock;
