@@ -296,16 +296,16 @@ extern "C" int pf_plan_create(const pf_model_t *model, const pf_cluster_t *clust
     }
 
     // slab = longest axis prefix whose product stays under a size that still leaves a few blocks per SM
-    cudaDeviceProp prop;
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess) {
-        pf::set_cuda_error(cudaGetLastError(), "pf_plan_create: device query");
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {   // (the full property
+        pf::set_cuda_error(cudaGetLastError(), "pf_plan_create: device query");           // query takes a millisecond)
         free(p->h_vals);
         delete p;
         return PF_ECUDA;
     }
     p->device = dev;
-    p->sm_count = prop.multiProcessorCount;
+    p->sm_count = sms;
     uint64_t target = N / (uint64_t)(4 * p->sm_count);
     if (target < 256) target = 256;
     if (target > pf::kSlabMax) target = pf::kSlabMax;

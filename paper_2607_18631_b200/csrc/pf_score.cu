@@ -194,6 +194,37 @@ __device__ __forceinline__ void block_copy_out(uint8_t *dst, const uint8_t *src,
     for (uint32_t i = head + (nv << 4) + tid; i < n; i += nt) dst[i] = src[i];
 }
 
+// One queued candidate through the memory model, the gate, the step-time model and the price.
+struct CostOut {
+    long long mem;
+    float tput;
+    int reason, v_eff;
+};
+template <typename RI>
+__device__ __noinline__ CostOut train_cost(const DevPlan &P, const TrainTuple c)
+{
+    CostOut o;
+    o.reason = 0;
+    o.tput = 0.f;
+    RI dp, world;
+    TrainDerived<RI> D;
+    train_layout_rules<RI>(P, c, 4, 3, dp, world);      // derives dp / world only
+    train_plan_rules<RI>(P, c, dp, world, 4, D);        // the rules passed in phase 1: fills D
+    TrainMem M;
+    train_memory<RI>(P, c, D, M);
+    o.mem = M.mem;
+    o.v_eff = D.v_eff;
+    if (M.mem > P.budget_bytes) {
+        o.reason = PF_R_MEMORY;
+    } else {
+        TrainTimes T;
+        train_times<RI>(P, c, D, M, T);
+        o.tput = train_price<RI>(P, c, D, T, train_pipe_analytic<RI>(P, c, D, T));
+        if (domain_why<RI>(P, P.kern[c.kv], D.m_e)) o.reason = PF_FLAG_EXTRAPOLATED;
+    }
+    return o;
+}
+
 template <typename RI>
 __global__ void __launch_bounds__(kThreads, 4) score_kernel(const __grid_constant__ DevPlan P, const ScoreArgs A)
 {
@@ -403,20 +434,13 @@ __global__ void __launch_bounds__(kThreads, 4) score_kernel(const __grid_constan
                         c.kv = v[0]; c.rec = v[1]; c.s = v[2]; c.mb = v[3]; c.v = v[4];
                         c.ep = v[5]; c.pp = v[6]; c.tp = v[7]; c.dp = v[8]; c.world = v[9];
                         c.sh = P.n_axes > 10 ? v[10] : PF_SHARD_ZERO1;
-                        RI dp, world;
-                        TrainDerived<RI> D;
-                        train_layout_rules<RI>(P, c, 4, 3, dp, world);      // derives dp / world only
-                        train_plan_rules<RI>(P, c, dp, world, 4, D);        // passed in phase 1: fills D
-                        TrainMem M;
-                        train_memory<RI>(P, c, D, M);
-                        if (M.mem > P.budget_bytes) {
-                            reason = PF_R_MEMORY;
-                        } else {
-                            TrainTimes T;
-                            train_times<RI>(P, c, D, M, T);
-                            tput = train_price<RI>(P, c, D, T, train_pipe_analytic<RI>(P, c, D, T));
-                            if (domain_why<RI>(P, P.kern[c.kv], D.m_e)) reason = PF_FLAG_EXTRAPOLATED;
-                        }
+                        // memory model, gate, step time and price in a function of its own (its registers are
+                        // then allocated apart from this kernel's many live values)
+                        const CostOut co = train_cost<RI>(P, c);
+                        reason = co.reason;
+                        tput = co.tput;
+                        struct { long long mem; } M = {co.mem};
+                        struct { int v_eff; } D = {co.v_eff};
                         const uint64_t o = PF_AT(P.chk, rel0 + i, A.count, PF_SITE_DENSE);
                         img[PF_AT(P.chk, pad + i, P.slab + 16, PF_SITE_IMAGE) - pad] = (uint8_t)reason;
                         if (A.tput && tput != 0.f) A.tput[o] = tput;
