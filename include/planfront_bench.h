@@ -23,9 +23,10 @@ extern "C" {
  * kernel counts per class into ms[PF_T_CLASSES] / kernels[PF_T_CLASSES], and forgets them.
  * PF_T_SCORE: the scoring kernel; PF_T_TOPK: top-k list kernels (merge passes, dense top-k);
  * PF_T_SELECT: the survivor-selection kernels; PF_T_SIMPREP: the simulator's pre-pass (binning, records);
- * PF_T_SIMULATE: the simulator kernel (inside pf_search it also streams the constant blocks of the dense outputs);
- * PF_T_COMPACT: the kernels of pf_compact; PF_T_AGGREGATE: the per-plan serving aggregate; PF_T_FILL: the stand-alone kernel that streams the constant
- * blocks of the dense outputs inside pf_search when no simulator kernel runs to carry them.  Classes that run on different streams
+ * PF_T_SIMULATE: the simulator kernel; PF_T_COMPACT: the kernels of pf_compact; PF_T_AGGREGATE: the per-plan
+ * serving aggregate; PF_T_FILL_EARLY / PF_T_FILL: inside pf_search, the two launches of the kernel that streams
+ * the constant blocks of the dense outputs on a stream of its own (the narrow launch that starts with the call,
+ * and the wide one beside the simulator kernel that takes over its queue).  Classes that run on different streams
  * overlap, so their times may add up to more than the call's. */
 enum {
     PF_T_SCORE = 0, PF_T_TOPK = 1, PF_T_SELECT = 2, PF_T_SIMULATE = 3, PF_T_AGGREGATE = 4, PF_T_FILL = 5,
