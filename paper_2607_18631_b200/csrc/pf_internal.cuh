@@ -18,20 +18,24 @@ constexpr int kOrderMaxSlabs = 1 << 20;  // calls with more slabs visit them by 
 constexpr int kTailFillsPerBlock = 4;    // constant-fill slabs per block kept, at least, for the end of the visiting order
 constexpr int kFillsPerEvaluated = 3;    // fills interleaved per evaluated slab at the start of the visiting order (measured: 1: 0.392 ms, 2: 0.384, 3: 0.380, 4: 0.379, 6: 0.382, 8: 0.385, 12: 0.396)
 // Inside a search call a kernel of its own streams the constant slabs on the plan's fill stream, in two launches
-// that share one queue: a narrow one from the start of the call (beside the scoring kernel, the selection and the
-// simulator's pre-pass, which are latency-bound and stall under a saturated store stream), and a wide one beside the
-// simulator kernel, which works in shared memory.  Measured on the benchmark's space, step time with the wide launch
-// alone at 256 / 128 / 96 / 64 / 32 threads per SM: 0.651 / 0.583 / 0.578 / 0.630 / 0.88 ms (more store warps crowd
-// the simulator's shared-memory polling out of the load/store pipe, fewer cannot keep HBM busy); with the narrow
-// launch added at 64 / 96 / 128 / 160 / 192 / 256 threads per SM: 0.547 / 0.531 / 0.523 / 0.521 / 0.525 / 0.529 ms.
-// Fills interleaved with the evaluated slabs inside the scoring kernel only move time from one kernel to the other
-// (0, 2, 3, 4 per evaluated slab: 0.578, 0.582, 0.587, 0.590 ms without the narrow launch).
+// that share one queue: one from the start of the call (beside the scoring kernel, the selection and the
+// simulator's pre-pass) and one beside the simulator kernel.  The bytes travel as bulk copies issued by one block of
+// kFillThreads threads per SM.  Measured on the benchmark's space (ms per step): plain 16-byte stores instead of bulk
+// copies, 160 threads per SM early and 96 beside the simulator (more crowd the simulator's shared-memory polling out
+// of the load/store pipe, fewer cannot keep HBM busy): 0.529; bulk copies: 0.485, whatever the block size (32 .. 256
+// threads), the number of issuing threads (16 .. 128) or the piece size (2 .. 4 KB) -- but only with a working block
+// on every SM, which the early launch gets from a grid of 256 blocks per SM (32 per SM: 42 - 82 SMs covered, 0.55 -
+// 0.58 ms; 128: ~100 SMs, 0.535; 256: 144 - 148 SMs; 512: 148 SMs, no faster), whereas the launch beside the
+// simulator kernel is spread by that kernel's shared-memory footprint (a second fill block does not fit on an SM)
+// and covers all 148 SMs from 8 blocks per SM on.
+// Fills interleaved with the evaluated slabs inside the scoring kernel only move time from one kernel to the other.
 constexpr int kFillsPerEvaluatedSplit = 0;
 constexpr int kFillBlocksPerSm = 1;
-constexpr int kFillThreads = 96;         // the wide launch
-constexpr int kFillEarlyThreads = 160;   // the narrow launch: one block per SM, its stores paced by the other work
-constexpr int kFillGridPerSm = 32;       // blocks launched per SM: the grid covers every SM however the hardware
-                                         // places it; a block works only if it is among the first on its SM
+constexpr int kFillThreads = 128;          // block size of the fill kernel (both launches)
+constexpr int kFillEarlyIssuers = 32;      // threads that issue bulk copies in the early launch (all do in the late one)
+constexpr int kFillGridPerSm = 32;         // blocks launched per SM beside the simulator kernel ...
+constexpr int kFillEarlyGridPerSm = 256;   // ... and from the start of the call; a block works only if it is among
+                                           // the first on its SM
 constexpr int kQueueCap = 4096;   // cost-model queue of the scoring kernel (entries), drained when it may fill up
 
 struct DevSched {
@@ -377,6 +381,7 @@ struct FillArgs {
     const unsigned int *stop;      // may be NULL; once the word is non-zero the launch draws no further slab
     unsigned int *done;            // counts the slabs the launch has filled
     uint32_t per_sm;               // working blocks per SM
+    uint32_t piece, issuers;       // zeros travel as bulk copies of `piece` bytes, issued by the first `issuers` threads
 };
 
 // How a scoring call may spread over the plan's streams (all off: one stream, one scoring kernel).

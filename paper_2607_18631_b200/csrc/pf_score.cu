@@ -664,17 +664,53 @@ __global__ void __launch_bounds__(kThreads, 4) score_kernel(const __grid_constan
     }
 }
 
-// The constant slabs behind the head of the visiting order, streamed by a kernel of their own: no shared memory,
-// few registers, so that it shares the SMs with whatever else runs meanwhile (the survivor selection and the
-// simulator inside a search call).  Tickets [hdr[4], n_slabs) are all constant slabs by construction of the order;
-// blocks take them round robin (they are all the same size but for a clipped first or last one).
+constexpr uint32_t kFillZeroBytes = 3072;     // the fill kernel's shared-memory source of zeros ...
+constexpr uint32_t kFillReasonBytes = 1024;   // ... and of the reason byte of the slab in hand
+
+// n bytes of value b at p: the 16-byte aligned body as asynchronous bulk copies from shared memory (`src` holds at
+// least `piece` bytes of b; the block's first `issuers` threads issue the copies, `piece` bytes each: the copy engine
+// moves them, the load/store pipe is not involved), the ragged ends with plain stores.  A bulk copy needs a 16-byte
+// aligned destination and a size that is a multiple of 16: both hold by construction, and a piece that broke either
+// would be stored the plain way instead.
+__device__ __forceinline__ void block_fill_bulk(uint8_t *p, uint64_t n, uint32_t b, uint32_t src, uint32_t piece,
+                                                uint32_t issuers)
+{
+    const uint32_t tid = threadIdx.x, nt = blockDim.x;
+    uint64_t head = (16 - ((uintptr_t)p & 15)) & 15;
+    if (head > n) head = n;
+    for (uint64_t i = tid; i < head; i += nt) p[i] = (uint8_t)b;
+    const uint64_t body = (n - head) & ~(uint64_t)15;
+    uint8_t *q = p + head;
+    if (tid < issuers) {
+        for (uint64_t off = (uint64_t)tid * piece; off < body; off += (uint64_t)issuers * piece) {
+            const uint32_t len = (uint32_t)(body - off < piece ? body - off : piece);
+            uint8_t *d = q + off;
+            if ((((uintptr_t)d | len) & 15) == 0 && len != 0) {
+                asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(d), "r"(src), "r"(len)
+                             : "memory");
+            } else {
+                for (uint32_t i = 0; i < len; i++) d[i] = (uint8_t)b;
+            }
+        }
+    }
+    for (uint64_t i = head + body + tid; i < n; i += nt) p[i] = (uint8_t)b;
+}
+
+// The constant slabs behind the head of the visiting order, streamed by a kernel of their own.  Its bytes leave as
+// asynchronous bulk copies from a 4 KB shared-memory pattern buffer, i.e. through the copy engine: a handful of
+// instructions per 160 KB slab instead of ten thousand 16-byte stores, so the kernel neither queues in the SM's
+// load/store pipe in front of the kernels it runs beside (the survivor selection and the simulator inside a search
+// call, which polls shared memory) nor needs more than one small block per SM.  Tickets [hdr[4], n_slabs) are all
+// constant slabs by construction of the order; blocks take them round robin (they are all the same size but for a
+// clipped first or last one).
 __global__ void __launch_bounds__(kThreads) fill_tail_kernel(const FillArgs A)
 {
-    // Where the hardware puts the blocks of a small grid that starts beside other kernels is not even: launched
-    // early, most of a one-block-per-SM grid was seen to land on a few SMs, whose store rate then bounded the whole
-    // kernel.  So the grid is oversubscribed and a block works only if it is among the first `per_sm` to register
-    // on its SM; the others leave at once, and the scheduler keeps placing blocks until every SM has its share.
-    __shared__ unsigned int s_go, s_t;
+    // Where the hardware puts the blocks of a small grid is not even: of a grid of 32 blocks per SM, launched beside
+    // the scoring kernel, all blocks were seen to arrive on about half of the SMs.  So the grid is oversubscribed and
+    // a block works only if it is among the first `per_sm` to register on its SM; the others leave at once, and the
+    // scheduler keeps placing blocks until (nearly) every SM has its share.
+    __shared__ __align__(128) uint8_t s_src[kFillZeroBytes + kFillReasonBytes];
+    __shared__ unsigned int s_go, s_t, s_more;
     const uint32_t tid = threadIdx.x;
     if (tid == 0) {
         unsigned int smid;
@@ -685,43 +721,68 @@ __global__ void __launch_bounds__(kThreads) fill_tail_kernel(const FillArgs A)
     __syncthreads();
     if (!s_go) return;
     if (!order_table_valid(A.order_hdr, A.slab_lo, A.n_slabs, A.order_tail, A.order_fpe)) return;
+    // The dense outputs of a constant slab leave as bulk copies from this buffer: zeros (tput and mem, twelve of a
+    // candidate's thirteen bytes) from its first part, the slab's reason byte from the rest, which is rewritten
+    // when the byte changes (slabs of one kind come in runs).
+    for (uint32_t i = tid; i < kFillZeroBytes / 16; i += blockDim.x)
+        reinterpret_cast<uint4 *>(s_src)[i] = make_uint4(0u, 0u, 0u, 0u);
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    __syncthreads();
+    const uint32_t zsrc = (uint32_t)__cvta_generic_to_shared(s_src), rsrc = zsrc + kFillZeroBytes;
+    const uint32_t piece = A.piece < 16u ? 16u : (A.piece > kFillZeroBytes ? kFillZeroBytes : (A.piece & ~15u));
+    const uint32_t rpiece = piece < kFillReasonBytes ? piece : kFillReasonBytes;
+    uint32_t cur_b = 0xFFFFFFFFu;   // the byte the reason part holds
     const uint32_t head_n = A.order_hdr[4];
     for (;;) {
         const uint32_t tk = s_t;
         __syncthreads();
         if (head_n + tk >= A.n_slabs) break;
-        if (A.stop && *reinterpret_cast<const volatile unsigned int *>(A.stop) != 0u) {
-            // the slab this block had drawn goes back to whoever takes over: it is filled here, then the block leaves
-            // (one slab per block at most: cheaper than handing tickets back)
-            const uint32_t w = __ldg(A.order + head_n + tk);
-            const uint64_t base = (A.slab_lo + (w & 0xFFFFFFu)) * (uint64_t)A.slab;
-            const uint64_t lo = base > A.first ? base : A.first;
-            const uint64_t end_slab = base + A.slab, end_call = A.first + A.count;
-            const uint64_t hi = end_slab < end_call ? end_slab : end_call;
-            const uint64_t rel0 = lo - A.first, n = hi - lo;
-            if (A.reason) block_fill(A.reason + rel0, n, w >> 24);
-            if (A.tput) block_fill(reinterpret_cast<uint8_t *>(A.tput + rel0), n * 4, 0u);
-            if (A.mem) block_fill(reinterpret_cast<uint8_t *>(A.mem + rel0), n * 8, 0u);
-            if (tid == 0) atomicAdd(A.done, 1u);
-            break;
-        }
+        // Thread 0 decides for the block whether another slab follows.  Once the hand-over word is set the slab the
+        // block has already drawn is still filled here, then the block leaves (one slab per block at most: cheaper
+        // than handing tickets back).
         uint32_t tk_next = 0;
-        if (tid == 0) tk_next = atomicAdd(A.ticket, 1u);   // in flight while this slab is stored
+        bool more = true;
+        if (tid == 0) {
+            more = !(A.stop && *reinterpret_cast<const volatile unsigned int *>(A.stop) != 0u);
+            if (more) tk_next = atomicAdd(A.ticket, 1u);   // in flight while this slab is stored
+        }
         const uint32_t w = __ldg(A.order + head_n + tk);
         const uint64_t base = (A.slab_lo + (w & 0xFFFFFFu)) * (uint64_t)A.slab;
         const uint64_t lo = base > A.first ? base : A.first;
         const uint64_t end_slab = base + A.slab, end_call = A.first + A.count;
         const uint64_t hi = end_slab < end_call ? end_slab : end_call;
         const uint64_t rel0 = lo - A.first, n = hi - lo;
-        if (A.reason) block_fill(A.reason + rel0, n, w >> 24);
-        if (A.tput) block_fill(reinterpret_cast<uint8_t *>(A.tput + rel0), n * 4, 0u);
-        if (A.mem) block_fill(reinterpret_cast<uint8_t *>(A.mem + rel0), n * 8, 0u);
+        const uint32_t b = w >> 24;
+        if (A.reason && b != cur_b) {
+            // copies issued earlier may still be reading the old byte pattern
+            if (tid < A.issuers) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+            __syncthreads();
+            const uint32_t bw = b * 0x01010101u;
+            for (uint32_t i = tid; i < kFillReasonBytes / 16; i += blockDim.x)
+                reinterpret_cast<uint4 *>(s_src + kFillZeroBytes)[i] = make_uint4(bw, bw, bw, bw);
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncthreads();
+            cur_b = b;
+        }
+        if (A.reason) block_fill_bulk(A.reason + rel0, n, b, rsrc, rpiece, A.issuers);
+        if (A.tput) block_fill_bulk(reinterpret_cast<uint8_t *>(A.tput + rel0), n * 4, 0u, zsrc, piece, A.issuers);
+        if (A.mem) block_fill_bulk(reinterpret_cast<uint8_t *>(A.mem + rel0), n * 8, 0u, zsrc, piece, A.issuers);
+        if (tid < A.issuers) {
+            // a bound on the copies in flight per issuing thread: at most four slabs' worth
+            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+            asm volatile("cp.async.bulk.wait_group.read 3;" ::: "memory");
+        }
         if (tid == 0) {
             s_t = tk_next;
-            atomicAdd(A.done, 1u);   // slabs this launch has filled (accounting only)
+            s_more = more ? 1u : 0u;
+            atomicAdd(A.done, 1u);   // slabs this launch has taken (accounting only)
         }
         __syncthreads();
+        if (!s_more) break;
     }
+    // the block's copies must have been written before it ends (the zero buffer goes away with the block, and the
+    // end of the kernel is what the rest of the call waits for)
+    asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
 }
 
 // ------------------------------------------------------------------ reducing a compact key list
@@ -1025,6 +1086,8 @@ int fill_launch(pf_plan_t *p, ScoreSpread &sp, cudaStream_t st)
         f.done = p->d_fill_ctl + 3;
         f.sm_slots = p->d_fill_ctl + 256 + 16;
         f.per_sm = kFillBlocksPerSm;
+        f.piece = kFillZeroBytes;
+        f.issuers = kFillThreads;
         fill_tail_kernel<<<p->sm_count * kFillGridPerSm, kFillThreads, 0, fs>>>(f);
     }
     count_launch();
@@ -1169,7 +1232,9 @@ int pf::score_run(pf_plan_t *p, uint64_t first, uint64_t count, uint8_t *d_reaso
         PF_CUDA_TRY(cudaEventRecord(p->ev_fork3, st), "early fill fork");
         PF_CUDA_TRY(cudaStreamWaitEvent(p->fill_stream, p->ev_fork3, 0), "early fill fork");
         timing_begin(p, PF_T_FILL_EARLY, p->fill_stream);
-        fill_tail_kernel<<<p->sm_count * kFillGridPerSm, kFillEarlyThreads, 0, p->fill_stream>>>(f);
+        f.piece = kFillZeroBytes;
+        f.issuers = kFillEarlyIssuers;
+        fill_tail_kernel<<<p->sm_count * kFillEarlyGridPerSm, kFillThreads, 0, p->fill_stream>>>(f);
         count_launch();
         timing_end(p, PF_T_FILL_EARLY, 1, p->fill_stream);
         const cudaError_t e_early = cudaGetLastError();
