@@ -41,11 +41,11 @@ NOMINAL_HBM_GBS = 7700.0          # HGX B200 data-sheet figure, for context
 # DRAM traffic of the fill kernel (the dominant kernel of a step), from one ncu capture on the profiling slice
 # (profile_case.py: a 49 M-candidate cut of the same space; summary under profiles/): dram__bytes_read.sum +
 # dram__bytes_write.sum of one fill_tail_kernel launch there, and the candidates that launch covers.  The kernel
-# writes every byte once and reads nothing (23.8 KB read): the capture shows 542.1 MB of DRAM traffic for 602.1 MB
-# of dense outputs -- the difference, 59.9 MB, is what still sat dirty in the 126 MB L2 when the kernel ended, a
+# writes every byte once and reads nothing (0.1 MB read): the capture shows 543.1 MB of DRAM traffic for 602.1 MB
+# of dense outputs -- the difference, 59.0 MB, is what still sat dirty in the 126 MB L2 when the kernel ended, a
 # constant of the cache, not of the workload.  A full-space launch is therefore reported as its algorithmic bytes
 # minus that residue.
-FILL_KERNEL_SLICE_DRAM_BYTES = 542_133_760
+FILL_KERNEL_SLICE_DRAM_BYTES = 543_096_576
 FILL_KERNEL_SLICE_CANDIDATES = 46_313_472
 # thread-level instructions one simulated op needs at least: load the dependency's end, add the hand-over latency,
 # max with the rank's clock, add the duration, store the result, advance the cursor
@@ -582,8 +582,8 @@ def run_ours(args):
     dom = max(cls_ms, key=lambda c: cls_ms[c])
     span = plan.fill_span()
     fill_cands = (span["n_blocks"] - span["scored_blocks"]) * span["block_candidates"]
-    # the fill kernel is launched twice per step (a narrow launch from the start of the call, a wide one beside the
-    # simulator kernel, one queue): its bytes over the sum of the two launches' durations
+    # the fill kernel is launched twice per step (one launch from the start of the call, one beside the simulator
+    # kernel, one queue): its bytes over the sum of the two launches' durations
     fill_ms = cls_ms.get("fill", 0.0) + cls_ms.get("fill_early", 0.0)
     if fill_ms > 0:
         kernel, k_ms, k_bytes = "fill_tail_kernel", fill_ms, BYTES_PER_CANDIDATE * fill_cands
@@ -602,18 +602,18 @@ def run_ours(args):
                 "launch_split": {"blocks": span["n_blocks"], "candidates_per_block": span["block_candidates"],
                                  "scoring_kernel_blocks": span["scored_blocks"], "fill_kernel_candidates": fill_cands,
                                  "fill_launches": {
-                                     "early_narrow": {"blocks": span["early_fill_blocks"],
-                                                      "ms": cls_ms.get("fill_early", 0.0)},
-                                     "wide": {"blocks": span["n_blocks"] - span["scored_blocks"] - span["early_fill_blocks"],
+                                     "early": {"blocks": span["early_fill_blocks"],
+                                               "ms": cls_ms.get("fill_early", 0.0)},
+                                     "beside_simulator": {"blocks": span["n_blocks"] - span["scored_blocks"] - span["early_fill_blocks"],
                                               "ms": cls_ms.get("fill", 0.0)}}},
                 "whole_step": {"bytes": BYTES_PER_CANDIDATE * N, "ms": ms_step,
                                "achieved": BYTES_PER_CANDIDATE * N / (ms_step * 1e-3) / 1e9,
                                "frac": BYTES_PER_CANDIDATE * N / (ms_step * 1e-3) / 1e9 / hbm},
-                "note": "the fill kernel runs on a stream of its own in two launches that share one queue: 160 threads "
-                        "per SM from the start of the call (paced by the latency-bound kernels it runs beside), then "
-                        "96 threads per SM beside the simulator kernel (so as not to crowd it out of the load/store "
-                        "pipe); ms_per_launch is the sum of the two; classes on different streams overlap, so class "
-                        "times add up to more than the step"}
+                "note": "the fill kernel (bulk copies from shared memory, one 128-thread block per SM) runs on a stream "
+                        "of its own in two launches that share one queue: from the start of the call until the "
+                        "simulator's pre-pass is done (its rate is shared with the latency-bound kernels it runs "
+                        "beside), then beside the simulator kernel; ms_per_launch is the sum of the two; classes on "
+                        "different streams overlap, so class times add up to more than the step"}
 
     # ---- side measurements (single-GPU runs): probes, top-k-only mode, simulator figures, the other configs
     extra = {}
