@@ -1074,7 +1074,7 @@ int fill_launch(pf_plan_t *p, ScoreSpread &sp, cudaStream_t st)
     if (!sp.fill_deferred) return PF_OK;
     sp.fill_deferred = false;
     cudaStream_t fs = p->fill_stream;
-    // tell an early, narrow fill launch to draw no further slab: the wide one takes the queue over
+    // tell the fill launch that started with the call to draw no further slab: this one takes the queue over
     PF_CUDA_TRY(cudaMemsetAsync(p->d_fill_ctl + 1, 0xFF, 4, st), "fill hand-over");
     PF_CUDA_TRY(cudaEventRecord(p->ev_fork2, st), "fill fork");
     PF_CUDA_TRY(cudaStreamWaitEvent(fs, p->ev_fork2, 0), "fill fork");
@@ -1217,10 +1217,10 @@ int pf::score_run(pf_plan_t *p, uint64_t first, uint64_t count, uint8_t *d_reaso
         a.head_only = split ? 1u : 0u;
     }
     if (split) {
-        // The constant slabs start to stream at once, by a narrow launch of the fill kernel on the plan's fill
-        // stream that runs beside the scoring kernel, the selection and the simulator's pre-pass -- slowly, because
-        // those are latency-bound and a saturated store stream would stall them -- until the wide launch takes the
-        // queue over (fill_launch).  Queue head, hand-over word and block registrations start at zero.
+        // The constant slabs start to stream at once, by a first launch of the fill kernel on the plan's fill
+        // stream that runs beside the scoring kernel, the selection and the simulator's pre-pass, until the launch
+        // beside the simulator kernel takes the queue over (fill_launch).  Queue head, hand-over word and block
+        // registrations start at zero.
         PF_CUDA_TRY(cudaMemsetAsync(p->d_fill_ctl, 0, 2048, st), "fill control reset");
         FillArgs &f = sp.fill;
         f.first = first; f.count = count; f.slab_lo = slab_lo; f.n_slabs = (uint32_t)n_slabs;
@@ -1266,7 +1266,7 @@ int pf::score_run(pf_plan_t *p, uint64_t first, uint64_t count, uint8_t *d_reaso
     int rc = PF_OK;
     if (topk_aside) PF_CUDA_TRY(cudaEventRecord(p->ev_fork, st), "score fork");
     if (split) {
-        // the caller decides when the wide fill launch takes over (fill_launch); until the fills have joined, only
+        // the caller decides when the second fill launch takes over (fill_launch); until the fills have joined, only
         // the evaluated slabs of the dense outputs hold results (guard)
         sp.fill_deferred = true;
         sp.guard.cls = (const uint8_t *)(a.order + p->order_cap);
