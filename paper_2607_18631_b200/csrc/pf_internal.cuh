@@ -382,6 +382,7 @@ struct FillArgs {
     unsigned int *done;            // counts the slabs the launch has filled
     uint32_t per_sm;               // working blocks per SM
     uint32_t piece, issuers;       // zeros travel as bulk copies of `piece` bytes, issued by the first `issuers` threads
+    unsigned int *chk;             // the checked build's record (unused otherwise)
 };
 
 // How a scoring call may spread over the plan's streams (all off: one stream, one scoring kernel).

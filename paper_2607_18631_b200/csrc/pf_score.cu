@@ -752,6 +752,8 @@ __global__ void __launch_bounds__(kThreads) fill_tail_kernel(const FillArgs A)
         const uint64_t end_slab = base + A.slab, end_call = A.first + A.count;
         const uint64_t hi = end_slab < end_call ? end_slab : end_call;
         const uint64_t rel0 = lo - A.first, n = hi - lo;
+        (void)PF_AT(A.chk, head_n + tk, A.n_slabs, PF_SITE_ORDER);
+        (void)PF_AT(A.chk, rel0 + n - 1, A.count, PF_SITE_DENSE);   // the slab's whole span lies inside the outputs
         const uint32_t b = w >> 24;
         if (A.reason && b != cur_b) {
             // copies issued earlier may still be reading the old byte pattern
@@ -1225,6 +1227,7 @@ int pf::score_run(pf_plan_t *p, uint64_t first, uint64_t count, uint8_t *d_reaso
         FillArgs &f = sp.fill;
         f.first = first; f.count = count; f.slab_lo = slab_lo; f.n_slabs = (uint32_t)n_slabs;
         f.slab = p->dev.slab; f.order_tail = a.order_tail; f.order_fpe = a.order_fpe;
+        f.chk = p->dev.chk;
         f.reason = d_reason; f.tput = d_tput; f.mem = (long long *)d_mem;
         f.order = a.order; f.order_hdr = a.order_hdr;
         f.ticket = p->d_fill_ctl; f.stop = p->d_fill_ctl + 1; f.done = p->d_fill_ctl + 2;

@@ -69,6 +69,15 @@ def main():
     plan.simulate(idx, idx.numel(), 4, k=64)
     report("deep_pipelines", plan)
     plan.close()
+    # many blocks of odd size: the one-call search with the streaming kernel at work on the fill stream
+    cfg = make_config("large")
+    cut = {"kv": 7, "sched": 3, "mb": 15, "v": 7}
+    cfg["axes"] = [(n, (list(v)[:cut[n]] if n in cut else v)) for n, v in cfg["axes"]]
+    plan = Plan(cfg)
+    b = plan.search(256, 10 ** 6, 50, 4)
+    b = plan.search(256, 3000, 50, 4, bufs=b)
+    report("odd_blocks_search", plan)
+    plan.close()
 
 
 if __name__ == "__main__":

@@ -1,8 +1,8 @@
 """The checked build of the library (compiled with -DPF_BOUNDS_CHECK: every index into a shared-memory image, queue,
 table, timeline, order table, key list or output array is range-checked on the device; a violation sets a bit in the
 plan's check record and the access is redirected, nothing traps).  It stands in for a memory checker: the small
-spaces, eight randomized spaces, sub-ranges, the one-call search, the selection, the compact view and the
-deep-pipeline simulator cases must all leave the record empty.  Runs in a process of its own so that the checked
+spaces, eight randomized spaces, sub-ranges, the one-call search, the selection, the compact view, the
+deep-pipeline simulator cases and a 9.7e7-candidate search that splits its work over the plan's streams must all leave the record empty.  Runs in a process of its own so that the checked
 library never mixes with the ordinary one."""
 from __future__ import annotations
 
@@ -25,7 +25,7 @@ def test_checked_build_reports_no_bad_index():
                        text=True, timeout=900)
     assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-4000:]
     lines = [ln for ln in r.stdout.splitlines() if " status=" in ln]
-    assert len(lines) == 2 + 4 + 8 + 1, r.stdout
+    assert len(lines) == 2 + 4 + 8 + 1 + 1, r.stdout
     # the macro does record a bad index: site 17 (bit 131072), index 7, length 4 -- and reading clears the record
     assert lines[0] == "selftest status=0 record=131072 17 7 0 4 0", lines[0]
     assert lines[1] == "selftest_cleared status=0 record=0 0 0 0 0 0", lines[1]

@@ -142,3 +142,39 @@ def test_search_ignores_what_the_output_buffers_held_before():
             assert np.array_equal(b["surv_idx"][:n].cpu().numpy().view(np.uint64), ref)
             assert n < feas.numel()
     plan.close()
+
+
+def test_search_streams_constant_blocks_of_odd_size_exactly():
+    """Blocks of 6,615 candidates: the constant blocks' reason / tput / mem spans start at every 16-byte phase, so the
+    streaming kernel's bulk copies are preceded and followed by ragged ends.  The one-call search must give, byte
+    for byte, what pf_score gives (which writes every block with plain stores), whatever the buffers held before;
+    three ranges are also compared with the oracle."""
+    import torch
+    import oracle
+    from helpers import TPUT_RTOL
+    cfg = make_config("large")
+    cut = {"kv": 7, "sched": 3, "mb": 15, "v": 7}
+    cfg["axes"] = [(n, (list(v)[:cut[n]] if n in cut else v)) for n, v in cfg["axes"]]
+    plan = _plan(cfg)
+    assert plan.size == 6615 * 11 ** 4
+    out = plan.score(k=256)
+    b = plan.search(256, 10 ** 6, 50, 4)
+    for fill in (0xFF, 0x00):
+        b["reason"].fill_(fill)
+        b["tput"].fill_(1.5e30)
+        b["mem"].fill_(-7)
+        b = plan.search(256, 10 ** 6, 50, 4, bufs=b)
+        torch.cuda.synchronize()
+        for key in ("reason", "tput", "mem", "topk_idx", "topk_score", "topk_count"):
+            assert torch.equal(out[key], b[key]), key
+    span = plan.fill_span()
+    assert span["block_candidates"] == 6615 and span["n_blocks"] == 11 ** 4
+    assert 0 < span["scored_blocks"] < span["n_blocks"]          # the streaming kernel had work to do
+    orc = oracle.Oracle(cfg)
+    for first in (0, 6615 * 5000 + 17, plan.size - 300_001):
+        r, t, m, _ = orc.score_range(first, 300_001, threads=4)
+        sl = slice(first, first + 300_001)
+        assert np.array_equal(b["reason"][sl].cpu().numpy(), r)
+        assert np.array_equal(b["mem"][sl].cpu().numpy(), m)
+        assert np.allclose(b["tput"][sl].cpu().numpy(), t, rtol=TPUT_RTOL, atol=0)
+    plan.close()
