@@ -80,8 +80,9 @@ static int search_device(pf_plan_t *p, uint32_t k, uint64_t s_max, uint32_t k_si
     // evaluated slabs only (every feasible plan, the digest and the top-k keys come from those); the analytic top-k
     // is reduced on the second stream beside the selection; the constant slabs (most of the dense outputs' bytes,
     // which nothing downstream reads) are streamed by the fill kernel on the fill stream, from the start of the call
-    // and, in a second launch that takes the first one's queue over, beside the simulator kernel; everything joins
-    // before the re-ranking.  The simulator reuses the scoring scratch, so the top-k joins before it.
+    // and, in a second launch that takes the first one's queue over, beside the simulator kernel and the re-ranking (which
+    // reads simulator scores only); the fill stream joins last.  The simulator reuses the scoring scratch, so the
+    // analytic top-k joins before it.
     ScoreSpread sp;
     sp.topk_aside = sim && p->side_stream != nullptr;
     sp.fill_aside = sim && p->fill_stream != nullptr;

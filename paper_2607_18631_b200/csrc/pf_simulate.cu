@@ -554,7 +554,10 @@ __device__ __forceinline__ void sim_rounds_1f1b(volatile float *tl, const float 
 }
 
 // Interleaved: v chunks per rank; unit k of a rank is microbatch (k / (pp v)) pp + k mod pp of chunk
-// (k mod (pp v)) / pp, backward units walk the chunks downward; cursors advance without divisions
+// (k mod (pp v)) / pp, backward units walk the chunks downward.  Per direction a lane carries the timeline index of
+// its next unit's own word and that unit's stage, and advances both by one of three precomputed steps (next
+// microbatch of the window, next chunk, next window), chosen by two countdowns: no multiplications and no
+// divisions in the loop, and a step is straight-line code whose results are selected by its go / no-go predicate.
 __device__ __forceinline__ void sim_rounds_interleaved(volatile float *tl, const float *durF, const float *durB,
                                                        int glane, int pp, int v, int nj, int U, int warm,
                                                        int total_ops, float lat, int fonly, float &clock_out,
@@ -567,64 +570,60 @@ __device__ __forceinline__ void sim_rounds_interleaved(volatile float *tl, const
     const int row = active ? glane : 0;                    // lanes beyond the pipeline depth poll rank 0's rows
     const int Ul = active ? U : 0;                         // a lane beyond the pipeline depth has nothing to do
     int nF = 0, nB = 0, rounds = 0, seen = 0;
-    int fw = 0, fc = 0, fg = 0, bw = 0, bc = 0, bg = 0;   // position in the pp-wide window, chunk, window number
     float clock = 0.f;
+    // forward cursor: chunk 0, window 0, microbatch 0; backward cursor: the last chunk first
+    const int chunk_words = pp * nj;                       // timeline words between a rank's consecutive chunks
+    const int stepF_chunk = chunk_words - (pp - 1), stepF_window = 1 - (v - 1) * chunk_words;
+    const int stepB_chunk = -chunk_words - (pp - 1), stepB_window = 1 + (v - 1) * chunk_words;
+    int aF = row * nj, qF = row, fw = pp - 1, fc = v - 1;  // fw / fc: units left in the window / chunks left in the round
+    int aB = ((v - 1) * pp + row) * nj, qB = (v - 1) * pp + row, bw = pp - 1, bc = v - 1;
+    // one forward step: the unit's dependency is the same microbatch one stage earlier (e: that word, read by the caller)
+#define PF_SIM_FWD(e)                                                                                   \
+    {                                                                                                   \
+        const bool dep = qF > 0;                                                                        \
+        const bool go = nF < Ul && nF - nB <= warm && (!dep || (e) > 0.f);                              \
+        const float t = fmaxf(clock, dep ? (e) + lat : 0.f) + durF[PF_AT(chk, qF, q_lim, PF_SITE_DURATION)]; \
+        if (go) tl[PF_AT(chk, aF, w_lim, PF_SITE_TIMELINE)] = t;                                        \
+        clock = go ? t : clock;                                                                         \
+        const bool ww = fw == 0, wc = fc == 0;                                                          \
+        aF += go ? (ww ? (wc ? stepF_window : stepF_chunk) : 1) : 0;                                    \
+        qF += (go && ww) ? (wc ? -(v - 1) * pp : pp) : 0;                                               \
+        fc = (go && ww) ? (wc ? v - 1 : fc - 1) : fc;                                                   \
+        fw = go ? (ww ? pp - 1 : fw - 1) : fw;                                                          \
+        nF += go ? 1 : 0;                                                                               \
+    }
+    // one backward step: the dependency is the same microbatch one stage later
+#define PF_SIM_BWD(e)                                                                                   \
+    {                                                                                                   \
+        const bool dep = qB < Q - 1;                                                                    \
+        const bool go = nB < Ul && (nF - nB > warm || nF == Ul) && (!dep || (e) < 0.f);                 \
+        const float t = fmaxf(clock, dep ? lat - (e) : 0.f) + durB[PF_AT(chk, qB, q_lim, PF_SITE_DURATION)]; \
+        if (go) tl[PF_AT(chk, aB, w_lim, PF_SITE_TIMELINE)] = -t;                                       \
+        clock = go ? t : clock;                                                                         \
+        const bool ww = bw == 0, wc = bc == 0;                                                          \
+        aB += go ? (ww ? (wc ? stepB_window : stepB_chunk) : 1) : 0;                                    \
+        qB += (go && ww) ? (wc ? (v - 1) * pp : -pp) : 0;                                               \
+        bc = (go && ww) ? (wc ? v - 1 : bc - 1) : bc;                                                   \
+        bw = go ? (ww ? pp - 1 : bw - 1) : bw;                                                          \
+        nB += go ? 1 : 0;                                                                               \
+    }
+    // the words polled: one stage down / up from the own word (the own word when there is no dependency; once a
+    // direction has run out of units its cursor rests one word past the rank's row, inside the warp's slice)
+#define PF_SIM_POLL_F() tl[PF_AT(chk, aF - (qF > 0 ? nj : 0), r_lim, PF_SITE_TIMELINE)]
+#define PF_SIM_POLL_B() tl[PF_AT(chk, aB + (qB < Q - 1 ? nj : 0), r_lim, PF_SITE_TIMELINE)]
     // forward steps only until the first microbatch can have crossed the shallowest pipeline of the warp
     for (int i = 0; i < fonly; i++) {
-        const bool want = nF < Ul && nF - nB <= warm;
-        const int j = fg * pp + fw;
-        const int q = fc * pp + row;
-        const bool dep = q > 0;
-        const float e = tl[PF_AT(chk, (dep ? q - 1 : q) * nj + j, r_lim, PF_SITE_TIMELINE)];
-        if (want && (!dep || e > 0.f)) {
-            clock = fmaxf(clock, dep ? e + lat : 0.f) + durF[PF_AT(chk, q, q_lim, PF_SITE_DURATION)];
-            tl[PF_AT(chk, q * nj + j, w_lim, PF_SITE_TIMELINE)] = clock;
-            if (++fw == pp) {
-                fw = 0;
-                if (++fc == v) fc = 0, fg++;
-            }
-            nF++;
-        }
+        const float eF = PF_SIM_POLL_F();
+        PF_SIM_FWD(eF)
     }
     for (;;) {
 #pragma unroll
         for (int rep = 0; rep < 2; rep++) {
             // both polls first (see the 1F1B loop), then the two steps
-            const int jB0 = bg * pp + bw, qB0 = (v - 1 - bc) * pp + row;
-            const float eB0 = tl[PF_AT(chk, (qB0 < Q - 1 ? qB0 + 1 : qB0) * nj + jB0, r_lim, PF_SITE_TIMELINE)];
-            {   // forward step: unit (fg, fc, fw) = microbatch fg pp + fw of chunk fc
-                // (j may be nj once all forwards are done: that word lies inside the warp's slice)
-                const bool want = nF < Ul && nF - nB <= warm;
-                const int j = fg * pp + fw;
-                const int q = fc * pp + row;
-                const bool dep = q > 0;
-                const float e = tl[PF_AT(chk, (dep ? q - 1 : q) * nj + j, r_lim, PF_SITE_TIMELINE)];
-                if (want && (!dep || e > 0.f)) {
-                    clock = fmaxf(clock, dep ? e + lat : 0.f) + durF[PF_AT(chk, q, q_lim, PF_SITE_DURATION)];
-                    tl[PF_AT(chk, q * nj + j, w_lim, PF_SITE_TIMELINE)] = clock;
-                    if (++fw == pp) {
-                        fw = 0;
-                        if (++fc == v) fc = 0, fg++;
-                    }
-                    nF++;
-                }
-            }
-            {   // backward step: chunks walk downward
-                const bool want = nB < Ul && (nF - nB > warm || nF == Ul);
-                const int j = jB0;
-                const int q = qB0;
-                const bool dep = q < Q - 1;
-                const float e = eB0;
-                if (want && (!dep || e < 0.f)) {
-                    clock = fmaxf(clock, dep ? lat - e : 0.f) + durB[PF_AT(chk, q, q_lim, PF_SITE_DURATION)];
-                    tl[PF_AT(chk, q * nj + j, w_lim, PF_SITE_TIMELINE)] = -clock;
-                    if (++bw == pp) {
-                        bw = 0;
-                        if (++bc == v) bc = 0, bg++;
-                    }
-                    nB++;
-                }
-            }
+            const float eF = PF_SIM_POLL_F();
+            const float eB = PF_SIM_POLL_B();
+            PF_SIM_FWD(eF)
+            PF_SIM_BWD(eB)
         }
         PF_SIM_ITER_END(Ul)
     }
@@ -632,25 +631,18 @@ __device__ __forceinline__ void sim_rounds_interleaved(volatile float *tl, const
     while (__any_sync(0xFFFFFFFFu, nB < Ul)) {
 #pragma unroll
         for (int rep = 0; rep < 4; rep++) {
-            const int j = bg * pp + bw;
-            const int q = (v - 1 - bc) * pp + row;
-            const bool dep = q < Q - 1;
-            const float e = tl[PF_AT(chk, (dep ? q + 1 : q) * nj + j, r_lim, PF_SITE_TIMELINE)];
-            if (nB < Ul && (!dep || e < 0.f)) {
-                clock = fmaxf(clock, dep ? lat - e : 0.f) + durB[PF_AT(chk, q, q_lim, PF_SITE_DURATION)];
-                tl[PF_AT(chk, q * nj + j, w_lim, PF_SITE_TIMELINE)] = -clock;
-                if (++bw == pp) {
-                    bw = 0;
-                    if (++bc == v) bc = 0, bg++;
-                }
-                nB++;
-            }
+            const float eB = PF_SIM_POLL_B();
+            PF_SIM_BWD(eB)
         }
         if ((++rounds & 15) == 0) {
             if (!__any_sync(0xFFFFFFFFu, nF + nB != seen)) break;
             seen = nF + nB;
         }
     }
+#undef PF_SIM_FWD
+#undef PF_SIM_BWD
+#undef PF_SIM_POLL_F
+#undef PF_SIM_POLL_B
     clock_out = clock;
     done_out = nF + nB;
 }
@@ -1148,10 +1140,7 @@ int pf::simulate_run(pf_plan_t *p, const uint64_t *d_surv_idx, uint64_t n, const
             rc = fill_launch(p, *spread, st);
             if (rc != PF_OK) return rc;
         }
-        if (spread->fill_pending) {
-            PF_CUDA_TRY(cudaStreamWaitEvent(st, p->ev_fill, 0), "fill join");
-            spread->fill_pending = false;
-        }
+        // the fill stream is joined by the caller, after the re-ranking below (which does not read the dense outputs)
     }
     if (k > 0) {
         int nk = 0;
