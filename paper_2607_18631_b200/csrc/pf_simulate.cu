@@ -481,27 +481,45 @@ __device__ __forceinline__ void sim_rounds_1f1b(volatile float *tl, const float 
                                                 float &clock_out, int &done_out, unsigned int *chk, int w_lim,
                                                 int r_lim)
 {
+    (void)chk; (void)w_lim; (void)r_lim;
     // lanes beyond the pipeline depth take no part: they poll row 0 and never act
     const bool active = total_ops > 0;
     const int row = active ? glane : 0;
     const bool depF = active && row > 0, depB = active && row < pp - 1;
-    const int offF = (depF ? row - 1 : row) * nj, offB = (depB ? row + 1 : row) * nj, offO = row * nj;
-    (void)offF; (void)offB; (void)offO; (void)chk; (void)w_lim; (void)r_lim;
     const float dF = active ? durF[row] : 0.f, dB = active ? durB[row] : 0.f;
     const float latF = depF ? lat : 0.f, latB = depB ? lat : 0.f;
     const int njl = active ? nj : 0;   // a lane beyond the pipeline depth has nothing to do
     int nF = 0, nB = 0, rounds = 0, seen = 0;
     float clock = 0.f;
+    // microbatch-major timeline: word j * pp + stage.  aF / aB: the own word of the next forward / backward unit;
+    // the word polled is its neighbour one stage down / up (the own word when there is no dependency)
+    int aF = row, aB = row;
+    const int pF = depF ? -1 : 0, pB = depB ? 1 : 0;
+    // a step is straight-line code whose results are selected by its go / no-go predicate
+    // (index nF may be nj once all forwards are done: that word lies inside the warp's slice)
+#define PF_SIM_FWD(e)                                                                        \
+    {                                                                                        \
+        const bool go = nF < njl && nF - nB <= warm && (!depF || (e) > 0.f);                 \
+        const float t = fmaxf(clock, depF ? (e) + latF : 0.f) + dF;                          \
+        if (go) tl[PF_AT(chk, aF, w_lim, PF_SITE_TIMELINE)] = t;                             \
+        clock = go ? t : clock;                                                              \
+        aF += go ? pp : 0;                                                                   \
+        nF += go ? 1 : 0;                                                                    \
+    }
+#define PF_SIM_BWD(e)                                                                        \
+    {                                                                                        \
+        const bool go = nB < njl && (nF - nB > warm || nF == njl) && (!depB || (e) < 0.f);   \
+        const float t = fmaxf(clock, depB ? latB - (e) : 0.f) + dB;                          \
+        if (go) tl[PF_AT(chk, aB, w_lim, PF_SITE_TIMELINE)] = -t;                            \
+        clock = go ? t : clock;                                                              \
+        aB += go ? pp : 0;                                                                   \
+        nB += go ? 1 : 0;                                                                    \
+    }
     // No backward can run before the first microbatch has crossed the shallowest pipeline of the warp: the first
-    // `fonly` steps are forward steps only (the same step as in the loop below).
+    // `fonly` steps are forward steps only.
     for (int i = 0; i < fonly; i++) {
-        const bool want = nF < njl && nF - nB <= warm;
-        const float e = tl[PF_AT(chk, offF + nF, r_lim, PF_SITE_TIMELINE)];
-        if (want && (!depF || e > 0.f)) {
-            clock = fmaxf(clock, depF ? e + latF : 0.f) + dF;
-            tl[PF_AT(chk, offO + nF, w_lim, PF_SITE_TIMELINE)] = clock;
-            nF++;
-        }
+        const float eF = tl[PF_AT(chk, aF + pF, r_lim, PF_SITE_TIMELINE)];
+        PF_SIM_FWD(eF)
     }
     for (;;) {
 #pragma unroll
@@ -509,27 +527,10 @@ __device__ __forceinline__ void sim_rounds_1f1b(volatile float *tl, const float 
             // both polls are issued before either step runs, so that their shared-memory latencies overlap (the
             // backward step's dependency is another lane's word: reading it a few instructions early only means a
             // value that arrives in between is seen one iteration later)
-            // (index nF may be nj once all forwards are done: that word lies inside the warp's slice)
-            const float eF = tl[PF_AT(chk, offF + nF, r_lim, PF_SITE_TIMELINE)];
-            const float eB = tl[PF_AT(chk, offB + nB, r_lim, PF_SITE_TIMELINE)];
-            {   // forward step
-                const bool want = nF < njl && nF - nB <= warm;
-                const float e = eF;
-                if (want && (!depF || e > 0.f)) {
-                    clock = fmaxf(clock, depF ? e + latF : 0.f) + dF;
-                    tl[PF_AT(chk, offO + nF, w_lim, PF_SITE_TIMELINE)] = clock;
-                    nF++;
-                }
-            }
-            {   // backward step
-                const bool want = nB < njl && (nF - nB > warm || nF == njl);
-                const float e = eB;
-                if (want && (!depB || e < 0.f)) {
-                    clock = fmaxf(clock, depB ? latB - e : 0.f) + dB;
-                    tl[PF_AT(chk, offO + nB, w_lim, PF_SITE_TIMELINE)] = -clock;
-                    nB++;
-                }
-            }
+            const float eF = tl[PF_AT(chk, aF + pF, r_lim, PF_SITE_TIMELINE)];
+            const float eB = tl[PF_AT(chk, aB + pB, r_lim, PF_SITE_TIMELINE)];
+            PF_SIM_FWD(eF)
+            PF_SIM_BWD(eB)
         }
         PF_SIM_ITER_END(njl)
     }
@@ -537,18 +538,16 @@ __device__ __forceinline__ void sim_rounds_1f1b(volatile float *tl, const float 
     while (__any_sync(0xFFFFFFFFu, nB < njl)) {
 #pragma unroll
         for (int rep = 0; rep < 4; rep++) {
-            const float e = tl[PF_AT(chk, offB + nB, r_lim, PF_SITE_TIMELINE)];
-            if (nB < njl && (!depB || e < 0.f)) {
-                clock = fmaxf(clock, depB ? latB - e : 0.f) + dB;
-                tl[PF_AT(chk, offO + nB, w_lim, PF_SITE_TIMELINE)] = -clock;
-                nB++;
-            }
+            const float eB = tl[PF_AT(chk, aB + pB, r_lim, PF_SITE_TIMELINE)];
+            PF_SIM_BWD(eB)
         }
         if ((++rounds & 15) == 0) {
             if (!__any_sync(0xFFFFFFFFu, nF + nB != seen)) break;
             seen = nF + nB;
         }
     }
+#undef PF_SIM_FWD
+#undef PF_SIM_BWD
     clock_out = clock;
     done_out = nF + nB;
 }
@@ -572,11 +571,11 @@ __device__ __forceinline__ void sim_rounds_interleaved(volatile float *tl, const
     int nF = 0, nB = 0, rounds = 0, seen = 0;
     float clock = 0.f;
     // forward cursor: chunk 0, window 0, microbatch 0; backward cursor: the last chunk first
-    const int chunk_words = pp * nj;                       // timeline words between a rank's consecutive chunks
-    const int stepF_chunk = chunk_words - (pp - 1), stepF_window = 1 - (v - 1) * chunk_words;
-    const int stepB_chunk = -chunk_words - (pp - 1), stepB_window = 1 + (v - 1) * chunk_words;
-    int aF = row * nj, qF = row, fw = pp - 1, fc = v - 1;  // fw / fc: units left in the window / chunks left in the round
-    int aB = ((v - 1) * pp + row) * nj, qB = (v - 1) * pp + row, bw = pp - 1, bc = v - 1;
+    // microbatch-major timeline: word j * Q + stage (the lanes of a group touch neighbouring words: no bank conflicts)
+    const int stepF_chunk = pp - (pp - 1) * Q, stepF_window = Q - (v - 1) * pp;   // next chunk: stage + pp, back to the window's first microbatch
+    const int stepB_chunk = -pp - (pp - 1) * Q, stepB_window = Q + (v - 1) * pp;
+    int aF = row, qF = row, fw = pp - 1, fc = v - 1;       // fw / fc: units left in the window / chunks left in the round
+    int aB = (v - 1) * pp + row, qB = (v - 1) * pp + row, bw = pp - 1, bc = v - 1;
     // one forward step: the unit's dependency is the same microbatch one stage earlier (e: that word, read by the caller)
 #define PF_SIM_FWD(e)                                                                                   \
     {                                                                                                   \
@@ -586,7 +585,7 @@ __device__ __forceinline__ void sim_rounds_interleaved(volatile float *tl, const
         if (go) tl[PF_AT(chk, aF, w_lim, PF_SITE_TIMELINE)] = t;                                        \
         clock = go ? t : clock;                                                                         \
         const bool ww = fw == 0, wc = fc == 0;                                                          \
-        aF += go ? (ww ? (wc ? stepF_window : stepF_chunk) : 1) : 0;                                    \
+        aF += go ? (ww ? (wc ? stepF_window : stepF_chunk) : Q) : 0;                                    \
         qF += (go && ww) ? (wc ? -(v - 1) * pp : pp) : 0;                                               \
         fc = (go && ww) ? (wc ? v - 1 : fc - 1) : fc;                                                   \
         fw = go ? (ww ? pp - 1 : fw - 1) : fw;                                                          \
@@ -601,16 +600,16 @@ __device__ __forceinline__ void sim_rounds_interleaved(volatile float *tl, const
         if (go) tl[PF_AT(chk, aB, w_lim, PF_SITE_TIMELINE)] = -t;                                       \
         clock = go ? t : clock;                                                                         \
         const bool ww = bw == 0, wc = bc == 0;                                                          \
-        aB += go ? (ww ? (wc ? stepB_window : stepB_chunk) : 1) : 0;                                    \
+        aB += go ? (ww ? (wc ? stepB_window : stepB_chunk) : Q) : 0;                                    \
         qB += (go && ww) ? (wc ? (v - 1) * pp : -pp) : 0;                                               \
         bc = (go && ww) ? (wc ? v - 1 : bc - 1) : bc;                                                   \
         bw = go ? (ww ? pp - 1 : bw - 1) : bw;                                                          \
         nB += go ? 1 : 0;                                                                               \
     }
     // the words polled: one stage down / up from the own word (the own word when there is no dependency; once a
-    // direction has run out of units its cursor rests one word past the rank's row, inside the warp's slice)
-#define PF_SIM_POLL_F() tl[PF_AT(chk, aF - (qF > 0 ? nj : 0), r_lim, PF_SITE_TIMELINE)]
-#define PF_SIM_POLL_B() tl[PF_AT(chk, aB + (qB < Q - 1 ? nj : 0), r_lim, PF_SITE_TIMELINE)]
+    // direction has run out of units its cursor rests up to Q words past the timeline, inside the warp's slice)
+#define PF_SIM_POLL_F() tl[PF_AT(chk, aF - (qF > 0 ? 1 : 0), r_lim, PF_SITE_TIMELINE)]
+#define PF_SIM_POLL_B() tl[PF_AT(chk, aB + (qB < Q - 1 ? 1 : 0), r_lim, PF_SITE_TIMELINE)]
     // forward steps only until the first microbatch can have crossed the shallowest pipeline of the warp
     for (int i = 0; i < fonly; i++) {
         const float eF = PF_SIM_POLL_F();
@@ -669,11 +668,11 @@ __device__ __forceinline__ void sim_rounds_dual(volatile float *tl, const float 
             const int sidx = d * pp + q;
             const bool dep = isb ? (q < pp - 1) : (q > 0);
             const int nb = dep ? (isb ? sidx + 1 : sidx - 1) : sidx;
-            const float e = tl[PF_AT(chk, nb * nj + j, r_lim, PF_SITE_TIMELINE)];
+            const float e = tl[PF_AT(chk, j * 2 * pp + nb, r_lim, PF_SITE_TIMELINE)];
             const float dur = (isb ? durB : durF)[PF_AT(chk, q, q_lim, PF_SITE_DURATION)];
             if (!dep || (isb ? e < 0.f : e > 0.f)) {
                 clock = fmaxf(clock, dep ? fabsf(e) + lat : 0.f) + dur;
-                tl[PF_AT(chk, sidx * nj + j, w_lim, PF_SITE_TIMELINE)] = isb ? -clock : clock;
+                tl[PF_AT(chk, j * 2 * pp + sidx, w_lim, PF_SITE_TIMELINE)] = isb ? -clock : clock;
                 done++;
                 moved = true;
             }
