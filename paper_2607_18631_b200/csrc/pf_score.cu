@@ -1234,19 +1234,6 @@ int pf::score_run(pf_plan_t *p, uint64_t first, uint64_t count, uint8_t *d_reaso
         f.sm_slots = p->d_fill_ctl + 16; f.per_sm = 1;
         PF_CUDA_TRY(cudaEventRecord(p->ev_fork3, st), "early fill fork");
         PF_CUDA_TRY(cudaStreamWaitEvent(p->fill_stream, p->ev_fork3, 0), "early fill fork");
-        timing_begin(p, PF_T_FILL_EARLY, p->fill_stream);
-        f.piece = kFillZeroBytes;
-        f.issuers = kFillEarlyIssuers;
-        fill_tail_kernel<<<p->sm_count * kFillEarlyGridPerSm, kFillThreads, 0, p->fill_stream>>>(f);
-        count_launch();
-        timing_end(p, PF_T_FILL_EARLY, 1, p->fill_stream);
-        const cudaError_t e_early = cudaGetLastError();
-        // the fill stream is forked from here on: the join event is recorded whatever happens next
-        if (cudaEventRecord(p->ev_fill, p->fill_stream) == cudaSuccess) sp.fill_pending = true;
-        if (e_early != cudaSuccess) {
-            set_cuda_error(e_early, "fill_tail_kernel launch");
-            return PF_ECUDA;
-        }
     }
     const size_t queue_bytes = p->dev.phase == PF_PHASE_TRAIN
                                    ? (((size_t)p->dev.slab + 16 + 15) & ~(size_t)15) + kQueueCap * sizeof(uint16_t)
@@ -1265,6 +1252,26 @@ int pf::score_run(pf_plan_t *p, uint64_t first, uint64_t count, uint8_t *d_reaso
     count_launch();
     timing_end(p, PF_T_SCORE, n_score_kernels, st);
     PF_CUDA_TRY(cudaGetLastError(), "score_kernel launch");
+    if (split) {
+        // The fill kernel's first launch is issued after the scoring kernel (on the fill stream it waits only for
+        // what preceded that kernel), so that the two reach the device in the same order whether or not the host
+        // runs ahead of it: a grid that arrives first is handed out to the end before the next one starts, and this
+        // one is deliberately long.
+        FillArgs &f = sp.fill;
+        timing_begin(p, PF_T_FILL_EARLY, p->fill_stream);
+        f.piece = kFillZeroBytes;
+        f.issuers = kFillEarlyIssuers;
+        fill_tail_kernel<<<p->sm_count * kFillEarlyGridPerSm, kFillThreads, 0, p->fill_stream>>>(f);
+        count_launch();
+        timing_end(p, PF_T_FILL_EARLY, 1, p->fill_stream);
+        const cudaError_t e_early = cudaGetLastError();
+        // the fill stream is forked from here on: the join event is recorded whatever happens next
+        if (cudaEventRecord(p->ev_fill, p->fill_stream) == cudaSuccess) sp.fill_pending = true;
+        if (e_early != cudaSuccess) {
+            set_cuda_error(e_early, "fill_tail_kernel launch");
+            return PF_ECUDA;
+        }
+    }
     const bool topk_aside = k > 0 && sp.topk_aside && p->side_stream;
     int rc = PF_OK;
     if (topk_aside) PF_CUDA_TRY(cudaEventRecord(p->ev_fork, st), "score fork");
