@@ -456,6 +456,8 @@ extern "C" int pf_plan_create(const pf_model_t *model, const pf_cluster_t *clust
         if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->ev_fill, cudaEventDisableTiming);
         if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->ev_fork2, cudaEventDisableTiming);
         if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->ev_fork3, cudaEventDisableTiming);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->ev_count, cudaEventDisableTiming);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->ev_compact, cudaEventDisableTiming);
         if (e != cudaSuccess) {
             pf::set_cuda_error(e, "pf_plan_create: side stream");
             pf_plan_destroy(p);
@@ -578,6 +580,8 @@ extern "C" void pf_plan_destroy(pf_plan_t *p)
     if (p->ev_fill) cudaEventDestroy(p->ev_fill);
     if (p->ev_fork2) cudaEventDestroy(p->ev_fork2);
     if (p->ev_fork3) cudaEventDestroy(p->ev_fork3);
+    if (p->ev_count) cudaEventDestroy(p->ev_count);
+    if (p->ev_compact) cudaEventDestroy(p->ev_compact);
     if (p->side_stream) cudaStreamDestroy(p->side_stream);
     if (p->fill_stream) cudaStreamDestroy(p->fill_stream);
     free(p->h_vals);

@@ -30,7 +30,16 @@ struct CompactArgs {
     unsigned int *chunk_count;       // [n_chunks] feasible per chunk, then exclusive prefixes (as 64-bit pairs below)
     unsigned long long *chunk_pre;   // [n_chunks]
     unsigned int n_chunks;
+    FillGuard guard;                 // cls != NULL: constant blocks may still be in flight; take their bytes from the classes
 };
+
+// class bytes to consult, or NULL when every block of the dense outputs may be read
+__device__ __forceinline__ const uint8_t *cmp_guard_cls(const CompactArgs &A)
+{
+    const FillGuard &g = A.guard;
+    if (!g.cls || !order_table_valid(g.hdr, g.slab_lo, g.n_slabs, g.tail, g.fpe)) return nullptr;
+    return g.cls;
+}
 
 // 16 reason bytes starting at candidate e of the range (bytes past the end read as 0xFF = not a candidate)
 __device__ __forceinline__ uint4 cmp_load16(const uint8_t *reason, uint64_t e, uint64_t count)
@@ -42,6 +51,34 @@ __device__ __forceinline__ uint4 cmp_load16(const uint8_t *reason, uint64_t e, u
             const uint32_t b = reason[e + i];
             w[i >> 2] = (w[i >> 2] & ~(0xFFu << (8 * (i & 3)))) | (b << (8 * (i & 3)));
         }
+    return make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+// The 16 reason bytes of candidates [e, e + 16) of the range.  With class bytes (cls), the bytes of candidates in a
+// constant block are the block's class -- what the streaming kernel writes there, sooner or later -- and memory is
+// read only where an evaluated block is involved.
+__device__ __forceinline__ uint4 cmp_reason16(const CompactArgs &A, const uint8_t *cls, uint64_t e)
+{
+    if (!cls) return cmp_load16(A.reason, e, A.count);
+    const FillGuard &g = A.guard;
+    const uint64_t a0 = A.first + e;
+    const uint64_t last = (e + 15 < A.count ? e + 15 : A.count - 1) + A.first;
+    const uint64_t s0 = a0 / g.slab - g.slab_lo, s1 = last / g.slab - g.slab_lo;
+    const uint32_t c0 = s0 < g.n_slabs ? cls[s0] : 0u;
+    if (s0 == s1) {
+        if (c0 == 0u) return cmp_load16(A.reason, e, A.count);
+        const uint32_t w = c0 * 0x01010101u;
+        return make_uint4(w, w, w, w);
+    }
+    // the group straddles blocks (at most two when a block holds 16 candidates or more; any number otherwise)
+    uint4 r = cmp_load16(A.reason, e, A.count);
+    uint32_t w[4] = {r.x, r.y, r.z, r.w};
+    for (int i = 0; i < 16; i++) {
+        if (e + i >= A.count) break;
+        const uint64_t si = (a0 + i) / g.slab - g.slab_lo;
+        const uint32_t c = si < g.n_slabs ? cls[si] : 0u;
+        if (c != 0u) w[i >> 2] = (w[i >> 2] & ~(0xFFu << (8 * (i & 3)))) | (c << (8 * (i & 3)));
+    }
     return make_uint4(w[0], w[1], w[2], w[3]);
 }
 
@@ -72,11 +109,35 @@ __global__ void __launch_bounds__(kCmpThreads) compact_count_kernel(const Compac
     if (tid == 0) s_feas = 0u;
     __syncthreads();
     const uint64_t lo = (uint64_t)blockIdx.x * kCmpChunk;
+    const uint8_t *cls = cmp_guard_cls(A);
+    if (cls) {
+        // A chunk that lies in constant blocks only (most do) needs no look at its candidates: each block adds its
+        // overlap with the chunk to its class's bin, the chunk's bits are zero and it holds no feasible plan.
+        const FillGuard &g = A.guard;
+        const uint64_t hi = lo + kCmpChunk < A.count ? lo + kCmpChunk : A.count;
+        const uint64_t s_first = (A.first + lo) / g.slab - g.slab_lo, s_last = (A.first + hi - 1) / g.slab - g.slab_lo;
+        bool constant = true;
+        for (uint64_t sl = s_first + tid; sl <= s_last; sl += kCmpThreads) constant &= sl < g.n_slabs && cls[sl] != 0;
+        if (__syncthreads_and(constant)) {
+            for (uint64_t sl = s_first + tid; sl <= s_last; sl += kCmpThreads) {
+                const uint64_t b0 = (g.slab_lo + sl) * (uint64_t)g.slab, b1 = b0 + g.slab;
+                const uint64_t a0 = b0 > A.first + lo ? b0 : A.first + lo, a1 = b1 < A.first + hi ? b1 : A.first + hi;
+                atomicAdd(A.hist + (cls[sl] & 0x7Fu & (kCmpBins - 1)), (unsigned long long)(a1 - a0));
+            }
+            if (A.mask) {
+                // the chunk starts at a multiple of 8 candidates; its last byte may be partial (end of the range)
+                const uint64_t m0 = lo >> 3, m1 = (hi + 7) >> 3;
+                for (uint64_t i = m0 + tid; i < m1; i += kCmpThreads) A.mask[i] = 0;
+            }
+            if (tid == 0) A.chunk_count[blockIdx.x] = 0u;
+            return;
+        }
+    }
     uint4 r[kCmpTiles];
 #pragma unroll
     for (int t = 0; t < kCmpTiles; t++) {
         const uint64_t e = lo + (uint64_t)t * kCmpTile + (uint64_t)tid * 16;
-        r[t] = e < A.count ? cmp_load16(A.reason, e, A.count) : make_uint4(~0u, ~0u, ~0u, ~0u);
+        r[t] = e < A.count ? cmp_reason16(A, cls, e) : make_uint4(~0u, ~0u, ~0u, ~0u);
     }
     unsigned int feas = 0;
 #pragma unroll
@@ -160,6 +221,7 @@ __global__ void __launch_bounds__(kCmpThreads) compact_write_kernel(const Compac
     __shared__ unsigned int s_warp[kCmpThreads / 32];
     __shared__ unsigned long long s_run;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const uint8_t *cls = cmp_guard_cls(A);
     for (unsigned int chunk = blockIdx.x; chunk < A.n_chunks; chunk += gridDim.x) {
         if (A.chunk_count[chunk] == 0u) continue;   // uniform across the block
         const uint64_t lo = (uint64_t)chunk * kCmpChunk;
@@ -168,7 +230,7 @@ __global__ void __launch_bounds__(kCmpThreads) compact_write_kernel(const Compac
 #pragma unroll
         for (int t = 0; t < kCmpTiles; t++) {
             const uint64_t e = lo + (uint64_t)t * kCmpTile + (uint64_t)tid * 16;
-            r[t] = e < A.count ? cmp_load16(A.reason, e, A.count) : make_uint4(~0u, ~0u, ~0u, ~0u);
+            r[t] = e < A.count ? cmp_reason16(A, cls, e) : make_uint4(~0u, ~0u, ~0u, ~0u);
         }
         __syncthreads();
 #pragma unroll
@@ -232,6 +294,38 @@ static CompactLayout compact_layout(uint64_t count)
     return l;
 }
 
+// The three launches on `st`.  guard: the class bytes of a scoring call whose constant blocks may still be in flight
+// (NULL: the dense outputs are complete).  Arguments are the caller's to check.
+int compact_run(pf_plan_t *p, uint64_t first, uint64_t count, const uint8_t *d_reason, const float *d_tput,
+                const int64_t *d_mem, uint64_t *d_hist, uint8_t *d_mask, pf_record_t *d_records, uint64_t record_cap,
+                uint64_t *d_n_feasible, void *d_workspace, cudaStream_t st, const FillGuard *guard)
+{
+    const CompactLayout lay = compact_layout(count);
+    uint8_t *ws = (uint8_t *)d_workspace;
+    CompactArgs a;
+    a.first = first; a.count = count; a.reason = d_reason; a.tput = d_tput; a.mem = (const long long *)d_mem;
+    a.hist = (unsigned long long *)d_hist; a.mask = d_mask; a.records = record_cap ? d_records : nullptr;
+    a.record_cap = record_cap; a.n_feasible = (unsigned long long *)d_n_feasible;
+    a.chunk_count = (unsigned int *)(ws + lay.off_count);
+    a.chunk_pre = (unsigned long long *)(ws + lay.off_pre);
+    a.n_chunks = lay.n_chunks;
+    if (guard) a.guard = *guard;
+    PF_CUDA_TRY(cudaMemsetAsync(d_hist, 0, PF_REASON_BINS * sizeof(uint64_t), st), "pf_compact: histogram reset");
+    timing_begin(p, PF_T_COMPACT, st);
+    compact_count_kernel<<<lay.n_chunks, kCmpThreads, 0, st>>>(a);
+    compact_scan_kernel<<<1, 1024, 0, st>>>(a);
+    int launches = 2;
+    if (record_cap > 0) {
+        const unsigned int grid = lay.n_chunks < (unsigned int)p->sm_count * 8 ? lay.n_chunks : (unsigned int)p->sm_count * 8;
+        compact_write_kernel<<<grid, kCmpThreads, 0, st>>>(a);
+        launches++;
+    }
+    timing_end(p, PF_T_COMPACT, launches, st);
+    for (int i = 0; i < launches; i++) count_launch();
+    PF_CUDA_TRY(cudaGetLastError(), "pf_compact launch");
+    return PF_OK;
+}
+
 }  // namespace pf
 
 using namespace pf;
@@ -253,27 +347,6 @@ extern "C" int pf_compact(pf_plan_t *p, uint64_t first, uint64_t count, const ui
     const CompactLayout lay = compact_layout(count);
     if (!d_workspace || ((uintptr_t)d_workspace & 255) != 0 || workspace_bytes < lay.total) return PF_EWORKSPACE;
     if (int rc_dev = check_device(p)) return rc_dev;
-    cudaStream_t st = (cudaStream_t)stream;
-    uint8_t *ws = (uint8_t *)d_workspace;
-    CompactArgs a;
-    a.first = first; a.count = count; a.reason = d_reason; a.tput = d_tput; a.mem = (const long long *)d_mem;
-    a.hist = (unsigned long long *)d_hist; a.mask = d_mask; a.records = record_cap ? d_records : nullptr;
-    a.record_cap = record_cap; a.n_feasible = (unsigned long long *)d_n_feasible;
-    a.chunk_count = (unsigned int *)(ws + lay.off_count);
-    a.chunk_pre = (unsigned long long *)(ws + lay.off_pre);
-    a.n_chunks = lay.n_chunks;
-    PF_CUDA_TRY(cudaMemsetAsync(d_hist, 0, PF_REASON_BINS * sizeof(uint64_t), st), "pf_compact: histogram reset");
-    timing_begin(p, PF_T_COMPACT, st);
-    compact_count_kernel<<<lay.n_chunks, kCmpThreads, 0, st>>>(a);
-    compact_scan_kernel<<<1, 1024, 0, st>>>(a);
-    int launches = 2;
-    if (record_cap > 0) {
-        const unsigned int grid = lay.n_chunks < (unsigned int)p->sm_count * 8 ? lay.n_chunks : (unsigned int)p->sm_count * 8;
-        compact_write_kernel<<<grid, kCmpThreads, 0, st>>>(a);
-        launches++;
-    }
-    timing_end(p, PF_T_COMPACT, launches, st);
-    for (int i = 0; i < launches; i++) count_launch();
-    PF_CUDA_TRY(cudaGetLastError(), "pf_compact launch");
-    return PF_OK;
+    return compact_run(p, first, count, d_reason, d_tput, d_mem, d_hist, d_mask, d_records, record_cap, d_n_feasible,
+                       d_workspace, (cudaStream_t)stream, nullptr);
 }

@@ -154,7 +154,7 @@ struct pf_plan {
     // the survivor selection and the simulator.  Streams and fork / join events belong to the plan (training
     // plans; created with the plan).
     cudaStream_t side_stream, fill_stream;
-    cudaEvent_t ev_fork, ev_join, ev_fork2, ev_fork3, ev_fill;
+    cudaEvent_t ev_fork, ev_join, ev_fork2, ev_fork3, ev_fill, ev_count, ev_compact;
     // simulator order tables (built at create for training plans)
     void *sim_tables;
     unsigned int *d_fill_ctl;      // queue head and per-SM block counts of the fill kernels (2 KB)
@@ -401,6 +401,10 @@ struct ScoreSpread {
     FillGuard guard;                                   // out: set when fill_deferred
 };
 int fill_launch(pf_plan_t *p, ScoreSpread &sp, cudaStream_t st);
+// pf_compact's launches on `st`; guard: class bytes to trust instead of constant blocks still in flight (or NULL)
+int compact_run(pf_plan_t *p, uint64_t first, uint64_t count, const uint8_t *d_reason, const float *d_tput,
+                const int64_t *d_mem, uint64_t *d_hist, uint8_t *d_mask, pf_record_t *d_records, uint64_t record_cap,
+                uint64_t *d_n_feasible, void *d_workspace, cudaStream_t st, const FillGuard *guard);
 int simulate_run(pf_plan_t *p, const uint64_t *d_surv_idx, uint64_t n, const uint64_t *d_n, uint32_t jitter_seed,
                  float *d_tput_sim, uint8_t *d_sim_status, uint32_t k, uint64_t *d_topk_idx, float *d_topk_score,
                  uint32_t *d_topk_count, void *d_workspace, size_t workspace_bytes, cudaStream_t st,

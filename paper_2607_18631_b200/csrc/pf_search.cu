@@ -58,6 +58,21 @@ static SearchLayout search_layout(const pf_plan_t *p, uint32_t k, uint64_t s_max
     return l;
 }
 
+// The compact view of a search's dense outputs (pf_compact's results) and where they go on the host: produced on the
+// plan's second stream as soon as the scoring kernel is done -- every feasible plan comes from an evaluated block,
+// and what the constant blocks will hold is known from their classes -- so that its copies to the host overlap with
+// the selection and the simulator.
+struct CompactJob {
+    uint64_t *d_hist, *d_nfeas;
+    uint8_t *d_mask;
+    pf_record_t *d_records;
+    uint64_t record_cap;
+    void *cws;
+    uint64_t *h_hist, *h_nfeas;
+    uint8_t *h_mask;
+    bool launched = false;   // out: enqueued; ev_count follows the copy of the count, ev_compact the copy of the bits
+};
+
 // The stages of one search on device buffers.  ws: scratch of the scoring call, reused by the simulator; ws_sel:
 // the selection's scratch, alive from before the scoring kernel (which fills the first pass's part) to the end
 // of the selection.
@@ -65,7 +80,7 @@ static int search_device(pf_plan_t *p, uint32_t k, uint64_t s_max, uint32_t k_si
                          uint8_t *d_reason, float *d_tput, int64_t *d_mem, uint64_t *d_tk_idx, float *d_tk_sc,
                          uint32_t *d_tk_cnt, uint64_t *d_surv, uint64_t *d_surv_cnt, uint64_t *d_sim_idx,
                          float *d_sim_sc, uint32_t *d_sim_cnt, uint8_t *ws, size_t ws_bytes, uint8_t *ws_sel,
-                         size_t ws_sel_bytes, cudaStream_t st)
+                         size_t ws_sel_bytes, cudaStream_t st, CompactJob *cj = nullptr)
 {
     const bool sim = s_max > 0 && p->dev.phase == PF_PHASE_TRAIN;
     ScoreDigest dg;
@@ -88,6 +103,33 @@ static int search_device(pf_plan_t *p, uint32_t k, uint64_t s_max, uint32_t k_si
     sp.fill_aside = sim && p->fill_stream != nullptr;
     sp.fills_per_evaluated = sp.fill_aside ? kFillsPerEvaluatedSplit : kFillsPerEvaluated;
     rc = score_run(p, 0, p->size, d_reason, d_tput, d_mem, k, d_tk_idx, d_tk_sc, d_tk_cnt, ws, ws_bytes, st, pdg, &sp);
+    bool compact_forked = false;
+    if (rc == PF_OK && cj && sp.join_pending) {
+        // the second stream is forked behind the scoring kernel and has the analytic top-k's reduction queued: the
+        // compact view follows it there, reading evaluated blocks only while the constant ones are in flight
+        cudaStream_t cs = p->side_stream;
+        const FillGuard *guard = (sp.fill_deferred || sp.fill_pending) ? &sp.guard : nullptr;
+        int rc2 = compact_run(p, 0, p->size, d_reason, d_tput, d_mem, cj->d_hist, cj->d_mask, cj->d_records,
+                              cj->record_cap, cj->d_nfeas, cj->cws, cs, guard);
+        cudaError_t e = cudaSuccess;
+        if (rc2 == PF_OK) {
+            e = cudaMemcpyAsync(cj->h_hist, cj->d_hist, PF_REASON_BINS * 8, cudaMemcpyDeviceToHost, cs);
+            if (e == cudaSuccess) e = cudaMemcpyAsync(cj->h_nfeas, cj->d_nfeas, 8, cudaMemcpyDeviceToHost, cs);
+            if (e == cudaSuccess) e = cudaEventRecord(p->ev_count, cs);
+            if (e == cudaSuccess && cj->h_mask)
+                e = cudaMemcpyAsync(cj->h_mask, cj->d_mask, ((size_t)p->size + 7) / 8, cudaMemcpyDeviceToHost, cs);
+            if (e == cudaSuccess) e = cudaEventRecord(p->ev_compact, cs);
+            if (e == cudaSuccess) cj->launched = true;
+        }
+        if (e != cudaSuccess) {
+            set_cuda_error(e, "compact view beside the search");
+            rc2 = PF_ECUDA;
+        }
+        // whatever was enqueued on the second stream is joined at the end of the call (below)
+        if (!cj->launched && cudaEventRecord(p->ev_compact, cs) != cudaSuccess && rc2 == PF_OK) rc2 = PF_ECUDA;
+        compact_forked = true;
+        if (rc2 != PF_OK) rc = rc2;
+    }
     if (rc == PF_OK && sim)
         rc = select_run(p, 0, p->size, d_reason, d_tput, s_max, d_surv, d_surv_cnt, ws_sel, ws_sel_bytes, st, true,
                         (sp.fill_deferred || sp.fill_pending) ? &sp.guard : nullptr);
@@ -98,6 +140,7 @@ static int search_device(pf_plan_t *p, uint32_t k, uint64_t s_max, uint32_t k_si
                           d_sim_cnt, ws, ws_bytes, st, &sp);
     if (rc == PF_OK && sp.fill_deferred) rc = fill_launch(p, sp, st);
     if (sp.fill_pending && cudaStreamWaitEvent(st, p->ev_fill, 0) != cudaSuccess && rc == PF_OK) rc = PF_ECUDA;
+    if (compact_forked && cudaStreamWaitEvent(st, p->ev_compact, 0) != cudaSuccess && rc == PF_OK) rc = PF_ECUDA;
     return rc;
 }
 
@@ -259,16 +302,23 @@ extern "C" int pf_search_host_compact(pf_plan_t *p, uint32_t k, uint64_t s_max, 
     uint64_t *d_hist = (uint64_t *)(ws + cl.off_hist), *d_nfeas = (uint64_t *)(ws + cl.off_nfeas);
     uint8_t *d_mask = h_mask ? ws + cl.off_mask : nullptr;
     pf_record_t *d_records = (pf_record_t *)(ws + cl.off_records);
+    CompactJob cj;
+    cj.d_hist = d_hist; cj.d_nfeas = d_nfeas; cj.d_mask = d_mask; cj.d_records = d_records; cj.record_cap = record_cap;
+    cj.cws = ws + cl.off_cws;
+    cj.h_hist = h_hist; cj.h_nfeas = h_n_feasible; cj.h_mask = h_mask;
     int rc = search_device(p, k, s_max, k_sim, jitter_seed, d_reason, d_tput, d_mem, d_tk_idx, d_tk_sc, d_tk_cnt,
                            d_surv, d_surv_cnt, d_sim_idx, d_sim_sc, d_sim_cnt, ws + l.off_ws, l.ws_bytes,
-                           ws + l.off_ws_sel, l.ws_sel_bytes, st);
+                           ws + l.off_ws_sel, l.ws_sel_bytes, st, &cj);
     if (rc != PF_OK) return rc;
-    rc = pf_compact(p, 0, N, d_reason, d_tput, d_mem, d_hist, d_mask, d_records, record_cap, d_nfeas, ws + cl.off_cws,
-                    cl.cws_bytes, stream);
-    if (rc != PF_OK) return rc;
-    PF_CUDA_TRY(cudaMemcpyAsync(h_hist, d_hist, PF_REASON_BINS * 8, cudaMemcpyDeviceToHost, st), "copy histogram");
-    PF_CUDA_TRY(cudaMemcpyAsync(h_n_feasible, d_nfeas, 8, cudaMemcpyDeviceToHost, st), "copy count");
-    if (h_mask) PF_CUDA_TRY(cudaMemcpyAsync(h_mask, d_mask, (N + 7) / 8, cudaMemcpyDeviceToHost, st), "copy mask");
+    if (!cj.launched) {
+        // no second stream took the compact view (a serving space, or no simulator tier): after the search
+        rc = pf_compact(p, 0, N, d_reason, d_tput, d_mem, d_hist, d_mask, d_records, record_cap, d_nfeas, ws + cl.off_cws,
+                        cl.cws_bytes, stream);
+        if (rc != PF_OK) return rc;
+        PF_CUDA_TRY(cudaMemcpyAsync(h_hist, d_hist, PF_REASON_BINS * 8, cudaMemcpyDeviceToHost, st), "copy histogram");
+        PF_CUDA_TRY(cudaMemcpyAsync(h_n_feasible, d_nfeas, 8, cudaMemcpyDeviceToHost, st), "copy count");
+        if (h_mask) PF_CUDA_TRY(cudaMemcpyAsync(h_mask, d_mask, (N + 7) / 8, cudaMemcpyDeviceToHost, st), "copy mask");
+    }
     PF_CUDA_TRY(cudaMemcpyAsync(h_topk_idx, d_tk_idx, (size_t)k * 8, cudaMemcpyDeviceToHost, st), "copy top-k");
     PF_CUDA_TRY(cudaMemcpyAsync(h_topk_score, d_tk_sc, (size_t)k * 4, cudaMemcpyDeviceToHost, st), "copy top-k");
     PF_CUDA_TRY(cudaMemcpyAsync(h_topk_count, d_tk_cnt, 4, cudaMemcpyDeviceToHost, st), "copy top-k");
@@ -282,15 +332,18 @@ extern "C" int pf_search_host_compact(pf_plan_t *p, uint32_t k, uint64_t s_max, 
         if (h_sim_topk_count) *h_sim_topk_count = 0;
         if (h_surv_count) *h_surv_count = 0;
     }
-    // the record count decides how many records travel: wait for it, then copy exactly those
-    PF_CUDA_TRY(cudaStreamSynchronize(st), "pf_search_host_compact: synchronize");
+    // the record count decides how many records travel: wait for it (with a second stream at work it has been on
+    // the host since shortly after the scoring kernel ended), then copy exactly those
+    if (cj.launched)
+        PF_CUDA_TRY(cudaEventSynchronize(p->ev_count), "pf_search_host_compact: count");
+    else
+        PF_CUDA_TRY(cudaStreamSynchronize(st), "pf_search_host_compact: synchronize");
     if (record_cap > 0) {
         const uint64_t n = *h_n_feasible < record_cap ? *h_n_feasible : record_cap;
-        if (n > 0) {
+        if (n > 0)
             PF_CUDA_TRY(cudaMemcpyAsync(h_records, d_records, (size_t)n * sizeof(pf_record_t), cudaMemcpyDeviceToHost, st),
                         "copy records");
-            PF_CUDA_TRY(cudaStreamSynchronize(st), "pf_search_host_compact: synchronize");
-        }
     }
+    PF_CUDA_TRY(cudaStreamSynchronize(st), "pf_search_host_compact: synchronize");
     return PF_OK;
 }
