@@ -83,6 +83,17 @@ def test_search_host_compact_on_the_large_space():
     ref, _, _ = orc.simulate_list(surv, 4, threads=64)
     ref_idx, ref_sc = Oracle.topk_list(surv, ref, 100)
     check_topk(r["sim_topk_idx"], r["sim_topk_score"], ref_idx, ref_sc)
+    # the view is taken while the constant blocks of the dense arrays are still being streamed out: whatever the
+    # workspace held before (all zero bytes read as "feasible everywhere") must not show in it
+    for poison in (0, 0x85):
+        ws.fill_(poison)
+        h_mask2 = np.full((N + 7) // 8, 0xFF, dtype=np.uint8)
+        rp = plan.search_host_compact(1024, 10 ** 6, 100, 4, ws, cap, h_mask=h_mask2)
+        np.testing.assert_array_equal(rp["hist"], r["hist"])
+        np.testing.assert_array_equal(h_mask2, h_mask)
+        assert rp["n_records"] == r["n_records"]
+        np.testing.assert_array_equal(rp["records"][:rp["n_records"]], r["records"][:r["n_records"]])
+        np.testing.assert_array_equal(rp["sim_topk_idx"], r["sim_topk_idx"])
     # records and mask are optional, and a short record buffer is filled from the front
     r2 = plan.search_host_compact(1024, 10 ** 6, 100, 4, ws, 1000)
     assert r2["n_feasible"] == 12_905 and r2["n_records"] == 1000
