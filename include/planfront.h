@@ -371,8 +371,10 @@ int pf_dualpipe_order(int pp, int m, uint8_t *out_ops);
  * so the selection starts at its second pass.  d_reason, d_tput and the top-k buffers are required, d_mem may be
  * NULL; the survivor and simulator buffers are required when the simulator tier runs (d_surv_idx: s_max entries).
  * d_workspace: pf_search_device_workspace() bytes, 256-byte aligned.  Enqueues on `stream`, does not synchronize.
- * (With a simulator tier, the reduction of the analytic top-k runs on a second stream that belongs to the plan,
- * forked from and joined back into `stream` by events inside the call; the call can be captured into a graph.)
+ * (With a simulator tier, parts of the call run on two more streams that belong to the plan -- the reduction of
+ * the analytic top-k on one, the kernel that streams the constant blocks of the dense outputs on the other --
+ * forked from and joined back into `stream` by events inside the call: all outputs are complete when the work the
+ * call put on `stream` is done, and the call can be captured into a graph.)
  * Errors as the calls above. */
 size_t pf_search_device_workspace(const pf_plan_t *plan, uint32_t k, uint64_t s_max, uint32_t k_sim);
 int pf_search(pf_plan_t *plan, uint32_t k, uint64_t s_max, uint32_t k_sim, uint32_t jitter_seed, uint8_t *d_reason,
@@ -420,8 +422,9 @@ int pf_compact(pf_plan_t *plan, uint64_t first, uint64_t count, const uint8_t *d
  * the reason histogram (h_hist[PF_REASON_BINS]), the feasibility bits (h_mask, N / 8 bytes, may be NULL), the
  * feasible plans' records (h_records[record_cap], may be NULL with record_cap 0) and their number (h_n_feasible),
  * besides the two top-k lists -- on the 1.8e8-candidate space about 23 MB instead of 2.3 GB.
- * d_workspace: pf_search_compact_workspace() bytes of DEVICE memory.  Returns after all copies have completed.
- * Errors as pf_search_host. */
+ * d_workspace: pf_search_compact_workspace() bytes of DEVICE memory.  Returns after all copies have completed
+ * (the view is taken, and its copies start, as soon as the candidates are scored, beside the selection and the
+ * simulator; host buffers should be pinned for the copies to overlap).  Errors as pf_search_host. */
 size_t pf_search_compact_workspace(const pf_plan_t *plan, uint32_t k, uint64_t s_max, uint32_t k_sim,
                                    uint64_t record_cap);
 int pf_search_host_compact(pf_plan_t *plan, uint32_t k, uint64_t s_max, uint32_t k_sim, uint32_t jitter_seed,
