@@ -418,3 +418,122 @@ def test_serving_without_dense_layers_is_unchanged_by_the_dense_fields():
     np.testing.assert_array_equal(ra, rb)
     np.testing.assert_array_equal(ta, tb)
     np.testing.assert_array_equal(ma, mb)
+
+
+# ----------------------------------------------------------------------------- the sharding regimes, by hand
+
+def hand_train_sharded() -> dict:
+    """hand_train() with the sharding axis (0 zero1, 1 zero1 with the optimizer offloaded, 2 fully sharded), a host
+    link of 2^26 B/s and a contention penalty of 25 %."""
+    cfg = hand_train()
+    cfg["axes"] = list(cfg["axes"]) + [("shard", [0, 1, 2])]
+    cfg["cluster"]["bw_host"] = float(2 ** 26)
+    cfg["consts"]["offload_overlap_penalty"] = 0.25
+    return cfg
+
+
+def test_offloaded_optimizer_step_time_hand_computed():
+    """The plan of test_training_step_time_hand_computed_tp2_pp2_ep2_dp2 with the optimizer state in host memory.
+    The rank owns the state of half its dense parameters (dp = 2) and of all its expert parameters (expert-DP group
+    of one): 2,101,248 + 3,145,728 = 5,246,976 parameters.  Per step their fp32 gradients go down and their bf16
+    weights come back over the host link: 6 B x 5,246,976 = 31,481,856 B at 2^26 B/s = 491,904 u, instead of
+    120.09375 u of HBM sweeps.  Pipeline and gradient exchange are unchanged:
+      T_step = 1,136,266 + 24,626 / 2 + 491,904 = 1,640,483 u;  throughput 2048 x 2^20 / 1,640,483.
+    Memory: the 62,963,712 B of optimizer state leave the device, nothing else changes."""
+    cfg = hand_train_sharded()
+    o = Oracle(cfg)
+    z = o.eval(axis_index(cfg, kv=0, rec=0, sched=0, ep=2, pp=2, tp=2, dp=2, shard=0))
+    d = o.eval(axis_index(cfg, kv=0, rec=0, sched=0, ep=2, pp=2, tp=2, dp=2, shard=1))
+    assert d["reason"] == 0 and z["reason"] == 0
+    assert z["T_step"] == pytest.approx(1148699.09375 * U, rel=1e-13)          # zero1 = the plan without the axis
+    assert d["T_opt"] == pytest.approx(491904 * U, rel=1e-13)
+    assert d["T_dp"] == pytest.approx(24626 * U, rel=1e-13) and d["T_pipe"] == pytest.approx(1136266 * U, rel=1e-13)
+    assert d["T_step"] == pytest.approx(1640483 * U, rel=1e-13)
+    assert d["tput"] == pytest.approx(2048 * 2 ** 20 / 1640483, rel=1e-13)
+    assert d["bytes_o"] == 0 and z["mem"] - d["mem"] == 62_963_712
+
+
+def test_offload_switches_the_hiding_off_and_pays_the_contention_penalty_when_overlapped():
+    """The interleaved + overlap plan of test_training_overlap_hides_part_of_the_all_to_all_and_is_priced (half of
+    the 2,050 u all-to-all hidden under zero1, 25 % schedule overhead).  With the optimizer offloaded nothing is
+    hidden (2,050 u exposed in both passes, so the layer times are those of the plan without overlap: 22,542 and
+    38,934 u) and the plan pays the 25 % contention penalty on top of the schedule overhead:
+      F = 2 x 22,542 + 1,024 = 46,108 u;  B = 2 x 38,934 + 2,048 = 79,916 u
+      T_pipe = (8 + 1/2) x 126,024 + 6 x 1,025 = 1,071,204 + 6,150 = 1,077,354 u
+      T_step = 1,077,354 + 12,313 + 491,904 = 1,581,571 u;  priced throughput = unpriced / (1.25 x 1.25)."""
+    cfg = hand_train_sharded()
+    o = Oracle(cfg)
+    z = o.eval(axis_index(cfg, kv=0, rec=0, sched=1, ep=2, pp=2, tp=2, dp=2, shard=0))
+    d = o.eval(axis_index(cfg, kv=0, rec=0, sched=1, ep=2, pp=2, tp=2, dp=2, shard=1))
+    assert z["reason"] == 0 and d["reason"] == 0
+    assert z["xF"] == pytest.approx(1025 * U, rel=1e-13) and z["xB"] == pytest.approx(1025 * U, rel=1e-13)
+    assert z["tput"] == pytest.approx(2048 * 2 ** 20 / 1054937.09375 / 1.25, rel=1e-13)
+    for name, units in dict(a2a=2050, xF=2050, xB=2050, F_l=22542, B_l=38934, F=46108, B=79916, T_pipe=1077354,
+                            T_opt=491904, T_step=1581571).items():
+        assert d[name] == pytest.approx(units * U, rel=1e-13), name
+    assert d["tput_unpriced"] == pytest.approx(2048 * 2 ** 20 / 1581571, rel=1e-13)
+    assert d["tput"] == pytest.approx(d["tput_unpriced"] / (1.25 * 1.25), rel=1e-13)
+    # without overlap (1F1B) the offloaded plan pays neither overhead
+    d0 = o.eval(axis_index(cfg, kv=0, rec=0, sched=0, ep=2, pp=2, tp=2, dp=2, shard=1))
+    assert d0["tput"] == pytest.approx(d0["tput_unpriced"], rel=1e-13)
+
+
+def test_fully_sharded_memory_and_exchange_hand_computed():
+    """The same tp2 / pp2 / ep2 / dp2 plan, fully sharded.
+    Memory: weights and gradients are held for the 5,246,976 parameters the rank owns: 2 B x 5,246,976 = 10,493,952
+    and 4 B x 5,246,976 = 20,987,904 (replicated: 2 B and 4 B x 7,348,224 = 14,696,448 and 29,392,896); the
+    optimizer state is unchanged (62,963,712); the all-gather buffer holds two layers of unsharded bf16 parameters:
+    a layer is 2,097,152 (attention / tp) + 4,096 (router) + 2 local experts x 786,432 = 3,674,112 parameters ->
+    2 x 2 B x 3,674,112 = 14,696,448 B.
+    Exchange, per microbatch, over the dense data-parallel group of 2 (the expert group has one member and moves
+    nothing): gather the bf16 dense weights for the forward and again for the backward, 1/2 x 2 B x 4,202,496 /
+    2^30 s = 4,104 u + 1 u each; reduce-scatter the fp32 gradients, 1/2 x 4 B x 4,202,496 / 2^30 s = 8,208 u + 1 u:
+    2 x 4,105 + 8,209 = 16,419 u, times 8 microbatches = 131,352 u (the replicated regimes exchange 24,626 u once).
+      T_step = 1,136,266 + 131,352 / 2 + 120.09375 = 1,202,062.09375 u."""
+    cfg = hand_train_sharded()
+    o = Oracle(cfg)
+    z = o.eval(axis_index(cfg, kv=0, rec=0, sched=0, ep=2, pp=2, tp=2, dp=2, shard=0))
+    d = o.eval(axis_index(cfg, kv=0, rec=0, sched=0, ep=2, pp=2, tp=2, dp=2, shard=2))
+    assert d["reason"] == 0
+    assert (z["bytes_w"], z["bytes_g"], z["bytes_buf"]) == (14_696_448, 29_392_896, 0)
+    assert (d["bytes_w"], d["bytes_g"], d["bytes_o"], d["bytes_buf"]) == (10_493_952, 20_987_904, 62_963_712, 14_696_448)
+    assert d["mem"] - z["mem"] == (10_493_952 + 20_987_904 + 14_696_448) - (14_696_448 + 29_392_896)
+    assert d["bytes_a"] == z["bytes_a"]
+    assert d["T_dp"] == pytest.approx(131352 * U, rel=1e-13)
+    assert d["T_opt"] == pytest.approx(120.09375 * U, rel=1e-13)
+    assert d["T_step"] == pytest.approx(1202062.09375 * U, rel=1e-13)
+    assert d["tput"] == pytest.approx(2048 * 2 ** 20 / 1202062.09375, rel=1e-13)
+
+
+def test_activation_bytes_hand_computed_with_and_without_a_leading_dense_layer():
+    """Activations kept per token and layer, bf16 (2 B) unless stated; hidden 1024, 8 + 8 + 8 heads of 128:
+      attention: layer-norm input 1024 + projection input 1024 + q, k, v 3 x 1024 + output-projection input 1024
+        = 6,144 values = 12,288 B
+      MoE part kept under selective recompute: layer-norm input + router input 2 x 1024 values (4,096 B), fp32 router
+        logits 4 x 4 B (16 B), two dispatched copies 2 x 1024 values (4,096 B), combine output 1024 values (2,048 B)
+        = 10,256 B;  dropped by selective recompute: gate, up, act x up for two routed copies of width 512 =
+        3 x 1,024 values = 6,144 B                          -> MoE layer: 28,688 B (none), 22,544 B (selective)
+      leading dense layer of width 2048: layer-norm input + FFN input 4,096 B kept; gate, up, act x up 3 x 2048 values
+        = 12,288 B dropped by selective recompute           -> dense layer: 28,672 B (none), 16,384 B (selective)
+      full recompute keeps the layer input only: 2,048 B, and one layer is live while it is recomputed.
+    Plan tp2 / pp2 / ep2 / dp2, 1F1B: 1024 tokens per microbatch, sharded over tp = 2 (sequence parallel), two layers
+    per stage, min(pp, m) = 2 microbatches in flight on rank 0, whose first layer is the dense one:
+      none       2 x (14,688,256 + 14,680,064) = 58,736,640    (two MoE layers: 2 x 2 x 14,688,256 = 58,753,024)
+      selective  2 x (11,542,528 +  8,388,608) = 39,862,272
+      full       2 x ( 1,048,576 +  1,048,576) + 14,688,256 = 18,882,560."""
+    cfg = hand_train()
+    plain = Oracle(cfg)
+    cfg_d = hand_train()
+    cfg_d["model"].update(L_dense=1, F_dense=2048)
+    dense = Oracle(cfg_d)
+    want = {0: (58_753_024, 58_736_640), 1: (2 * 2 * 11_542_528, 39_862_272),
+            2: (2 * 2 * 1_048_576 + 14_688_256, 18_882_560)}
+    for rec, (w_plain, w_dense) in want.items():
+        i = axis_index(cfg, kv=0, rec=rec, sched=0, ep=2, pp=2, tp=2, dp=2)
+        a, b = plain.eval(i), dense.eval(i)
+        assert a["reason"] == 0 and b["reason"] == 0
+        assert a["bytes_a"] == w_plain, rec
+        assert b["bytes_a"] == w_dense, rec
+    dv = dense.derived()
+    assert (dv["a_attn"], dv["a_full"], dv["a_sel"], dv["a_ckpt"]) == (12_288, 28_688, 22_544, 2_048)
+    assert (dv["a_full_d"], dv["a_sel_d"]) == (28_672, 16_384)
