@@ -582,9 +582,8 @@ def run_ours(args):
     dom = max(cls_ms, key=lambda c: cls_ms[c])
     span = plan.fill_span()
     fill_cands = (span["n_blocks"] - span["scored_blocks"]) * span["block_candidates"]
-    # the fill kernel is launched twice per step (one launch from the start of the call, one beside the simulator
-    # kernel, one queue): its bytes over the sum of the two launches' durations
-    fill_ms = cls_ms.get("fill", 0.0) + cls_ms.get("fill_early", 0.0)
+    # the fill kernel runs once per step, from right behind the scoring kernel to the end of the call
+    fill_ms = cls_ms.get("fill", 0.0)
     if fill_ms > 0:
         kernel, k_ms, k_bytes = "fill_tail_kernel", fill_ms, BYTES_PER_CANDIDATE * fill_cands
     else:                                    # no separate fill kernel ran: the scoring kernel wrote everything
@@ -601,19 +600,14 @@ def run_ours(args):
                 "dominant_class": dom, "class_ms_per_step": cls_ms,
                 "launch_split": {"blocks": span["n_blocks"], "candidates_per_block": span["block_candidates"],
                                  "scoring_kernel_blocks": span["scored_blocks"], "fill_kernel_candidates": fill_cands,
-                                 "fill_launches": {
-                                     "early": {"blocks": span["early_fill_blocks"],
-                                               "ms": cls_ms.get("fill_early", 0.0)},
-                                     "beside_simulator": {"blocks": span["n_blocks"] - span["scored_blocks"] - span["early_fill_blocks"],
-                                              "ms": cls_ms.get("fill", 0.0)}}},
+                                 "fill_kernel_blocks": span["filled_blocks"]},
                 "whole_step": {"bytes": BYTES_PER_CANDIDATE * N, "ms": ms_step,
                                "achieved": BYTES_PER_CANDIDATE * N / (ms_step * 1e-3) / 1e9,
                                "frac": BYTES_PER_CANDIDATE * N / (ms_step * 1e-3) / 1e9 / hbm},
                 "note": "the fill kernel (bulk copies from shared memory, one 128-thread block per SM) runs on a stream "
-                        "of its own in two launches that share one queue: from the start of the call until the "
-                        "simulator's pre-pass is done (its rate is shared with the latency-bound kernels it runs "
-                        "beside), then beside the simulator kernel; ms_per_launch is the sum of the two; classes on "
-                        "different streams overlap, so class times add up to more than the step"}
+                        "of its own beside everything else in the call, from right behind the scoring kernel to the "
+                        "end: it shares the memory system with the kernels it runs beside and is what the step waits "
+                        "for last; classes on different streams overlap, so class times add up to more than the step"}
 
     # ---- side measurements (single-GPU runs): probes, top-k-only mode, simulator figures, the other configs
     extra = {}

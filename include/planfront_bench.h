@@ -24,13 +24,12 @@ extern "C" {
  * PF_T_SCORE: the scoring kernel; PF_T_TOPK: top-k list kernels (merge passes, dense top-k);
  * PF_T_SELECT: the survivor-selection kernels; PF_T_SIMPREP: the simulator's pre-pass (binning, records);
  * PF_T_SIMULATE: the simulator kernel; PF_T_COMPACT: the kernels of pf_compact; PF_T_AGGREGATE: the per-plan
- * serving aggregate; PF_T_FILL_EARLY / PF_T_FILL: inside pf_search, the two launches of the kernel that streams
- * the constant blocks of the dense outputs on a stream of its own (the narrow launch that starts with the call,
- * and the wide one beside the simulator kernel that takes over its queue).  Classes that run on different streams
- * overlap, so their times may add up to more than the call's. */
+ * serving aggregate; PF_T_FILL: inside pf_search, the kernel that streams the constant blocks of the dense outputs
+ * on a stream of its own, from right behind the scoring kernel to the end of the call.  Classes that run on
+ * different streams overlap, so their times may add up to more than the call's. */
 enum {
     PF_T_SCORE = 0, PF_T_TOPK = 1, PF_T_SELECT = 2, PF_T_SIMULATE = 3, PF_T_AGGREGATE = 4, PF_T_FILL = 5,
-    PF_T_SIMPREP = 6, PF_T_COMPACT = 7, PF_T_FILL_EARLY = 8, PF_T_CLASSES = 9
+    PF_T_SIMPREP = 6, PF_T_COMPACT = 7, PF_T_CLASSES = 8
 };
 int pf_timing_enable(pf_plan_t *plan, int on);
 int pf_timing_read(pf_plan_t *plan, float *ms, uint32_t *kernels);
@@ -52,12 +51,12 @@ int pf_check_selftest(pf_plan_t *plan);
 
 /* How the plan's latest scoring call inside pf_search was divided between the scoring kernel and the kernel that
  * streams constant blocks: the number of blocks of candidates the call's range was cut into, candidates per block,
- * and how many blocks the scoring kernel took itself (the evaluated ones and the constant ones interleaved with
- * them); the rest went to the fill kernel, *early_fill_blocks of them to its narrow first launch.  Reads a few words
- * back from the device (synchronizes the device).
+ * how many blocks the scoring kernel took itself (the evaluated ones), and how many the fill kernel counted as
+ * streamed (the rest, when the call has completed).  Reads a few words back from the device (synchronizes the
+ * device).
  * Errors: PF_EINVAL (NULL pointer, or the plan has no such record), PF_ECUDA. */
 int pf_bench_fill_span(pf_plan_t *plan, uint64_t *n_blocks, uint64_t *block_candidates, uint64_t *scored_blocks,
-                       uint64_t *early_fill_blocks);
+                       uint64_t *filled_blocks);
 
 /* Roofline probes (libplanfront_probe.so).
  * The caller times them with events on `stream`; neither call synchronises or allocates.

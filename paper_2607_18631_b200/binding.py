@@ -31,7 +31,7 @@ EXPORTS = ("pf_version", "pf_strerror", "pf_reason_str", "pf_last_cuda_error", "
 # measurement hooks of include/planfront_bench.h that this library exports (the probes live in probes.py)
 BENCH_EXPORTS = ("pf_launch_count", "pf_timing_enable", "pf_timing_read", "pf_bench_fill_span", "pf_check_read", "pf_check_selftest")
 STATIC_SCRATCH_BYTES = 4 << 20
-T_CLASSES = ("score", "topk", "select", "simulate", "aggregate", "fill", "simprep", "compact", "fill_early")
+T_CLASSES = ("score", "topk", "select", "simulate", "aggregate", "fill", "simprep", "compact")
 REASON_BINS = 16
 RECORD_DTYPE = np.dtype([("idx", "<u8"), ("mem", "<i8"), ("tput", "<f4"), ("reason", "u1"), ("pad", "u1", (3,))])
 
@@ -333,7 +333,7 @@ class Plan:
         _check(self._L.pf_bench_fill_span(self._h, C.byref(a), C.byref(b), C.byref(c), C.byref(d)),
                "pf_bench_fill_span")
         return dict(n_blocks=int(a.value), block_candidates=int(b.value), scored_blocks=int(c.value),
-                    early_fill_blocks=int(d.value))
+                    filled_blocks=int(d.value))
 
     def timing_read(self) -> dict:
         """{class: (milliseconds, kernels)} accumulated since the last read; waits for the recorded events."""

@@ -454,7 +454,6 @@ extern "C" int pf_plan_create(const pf_model_t *model, const pf_cluster_t *clust
         if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->ev_fork, cudaEventDisableTiming);
         if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->ev_join, cudaEventDisableTiming);
         if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->ev_fill, cudaEventDisableTiming);
-        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->ev_fork2, cudaEventDisableTiming);
         if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->ev_fork3, cudaEventDisableTiming);
         if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->ev_count, cudaEventDisableTiming);
         if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->ev_compact, cudaEventDisableTiming);
@@ -541,9 +540,9 @@ extern "C" int pf_check_read(pf_plan_t *p, uint32_t *out)
 }
 
 extern "C" int pf_bench_fill_span(pf_plan_t *p, uint64_t *n_blocks, uint64_t *block_candidates, uint64_t *scored_blocks,
-                                  uint64_t *early_fill_blocks)
+                                  uint64_t *filled_blocks)
 {
-    if (!p || !n_blocks || !block_candidates || !scored_blocks || !early_fill_blocks || !p->d_order) return PF_EINVAL;
+    if (!p || !n_blocks || !block_candidates || !scored_blocks || !filled_blocks || !p->d_order) return PF_EINVAL;
     if (int rc_dev = pf::check_device(p)) return rc_dev;
     uint32_t hdr[8] = {0};
     PF_CUDA_TRY(cudaDeviceSynchronize(), "pf_bench_fill_span");
@@ -553,7 +552,7 @@ extern "C" int pf_bench_fill_span(pf_plan_t *p, uint64_t *n_blocks, uint64_t *bl
     *scored_blocks = hdr[4];
     uint32_t ctl[4] = {0};
     PF_CUDA_TRY(cudaMemcpy(ctl, p->d_fill_ctl, sizeof(ctl), cudaMemcpyDeviceToHost), "pf_bench_fill_span");
-    *early_fill_blocks = ctl[2];
+    *filled_blocks = ctl[2];
     return PF_OK;
 }
 
@@ -578,7 +577,6 @@ extern "C" void pf_plan_destroy(pf_plan_t *p)
     if (p->ev_fork) cudaEventDestroy(p->ev_fork);
     if (p->ev_join) cudaEventDestroy(p->ev_join);
     if (p->ev_fill) cudaEventDestroy(p->ev_fill);
-    if (p->ev_fork2) cudaEventDestroy(p->ev_fork2);
     if (p->ev_fork3) cudaEventDestroy(p->ev_fork3);
     if (p->ev_count) cudaEventDestroy(p->ev_count);
     if (p->ev_compact) cudaEventDestroy(p->ev_compact);

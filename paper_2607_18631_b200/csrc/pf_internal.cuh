@@ -17,25 +17,21 @@ constexpr int kInnerVals = 1024;     // inner-axis values the scoring kernel kee
 constexpr int kOrderMaxSlabs = 1 << 20;  // calls with more slabs visit them by a permutation instead of an order table
 constexpr int kTailFillsPerBlock = 4;    // constant-fill slabs per block kept, at least, for the end of the visiting order
 constexpr int kFillsPerEvaluated = 3;    // fills interleaved per evaluated slab at the start of the visiting order (measured: 1: 0.392 ms, 2: 0.384, 3: 0.380, 4: 0.379, 6: 0.382, 8: 0.385, 12: 0.396)
-// Inside a search call a kernel of its own streams the constant slabs on the plan's fill stream, in two launches
-// that share one queue: one from the start of the call (beside the scoring kernel, the selection and the
-// simulator's pre-pass) and one beside the simulator kernel.  The bytes travel as bulk copies issued by one block of
-// kFillThreads threads per SM.  Measured on the benchmark's space (ms per step): plain 16-byte stores instead of bulk
-// copies, 160 threads per SM early and 96 beside the simulator (more crowd the simulator's shared-memory polling out
-// of the load/store pipe, fewer cannot keep HBM busy): 0.529; bulk copies: 0.485, whatever the block size (32 .. 256
-// threads), the number of issuing threads (16 .. 128) or the piece size (2 .. 4 KB) -- but only with a working block
-// on every SM, which the early launch gets from a grid of 256 blocks per SM (32 per SM: 42 - 82 SMs covered, 0.55 -
-// 0.58 ms; 128: ~100 SMs, 0.535; 256: 144 - 148 SMs; 512: 148 SMs, no faster), whereas the launch beside the
-// simulator kernel is spread by that kernel's shared-memory footprint (a second fill block does not fit on an SM)
-// and covers all 148 SMs from 8 blocks per SM on.
+// Inside a search call a kernel of its own streams the constant slabs on the plan's fill stream, from right behind
+// the scoring kernel to the end of the call: ONE launch beside the scoring kernel, the selection, the simulator and
+// the re-ranking.  The bytes travel as bulk copies issued by one block of kFillThreads threads per SM.  Measured on
+// the benchmark's space (ms per step): plain 16-byte stores instead of bulk copies, in two launches of 160 and 96
+// threads per SM (more crowd the simulator's shared-memory polling out of the load/store pipe, fewer cannot keep
+// HBM busy): 0.529; bulk copies in two launches (one until the simulator's pre-pass is done, one beside the
+// simulator kernel): 0.466; in one launch: 0.437 -- whatever the block size (32 .. 256 threads), the number of
+// issuing threads (16 .. 128) or the piece size (2 .. 4 KB), but only with a working block on (nearly) every SM,
+// which takes a grid of 256 blocks per SM (32 per SM: 42 - 82 SMs covered, 0.55 - 0.58 ms with two launches; 128:
+// ~100 SMs, 0.535; 256: 144 - 148 SMs; 512: 148 SMs, no faster).
 // Fills interleaved with the evaluated slabs inside the scoring kernel only move time from one kernel to the other.
 constexpr int kFillsPerEvaluatedSplit = 0;
 constexpr int kFillBlocksPerSm = 1;
-constexpr int kFillThreads = 128;          // block size of the fill kernel (both launches)
-constexpr int kFillEarlyIssuers = 32;      // threads that issue bulk copies in the early launch (all do in the late one)
-constexpr int kFillGridPerSm = 32;         // blocks launched per SM beside the simulator kernel ...
-constexpr int kFillEarlyGridPerSm = 256;   // ... and from the start of the call; a block works only if it is among
-                                           // the first on its SM
+constexpr int kFillThreads = 128;      // block size of the fill kernel; every thread issues copies
+constexpr int kFillGridPerSm = 256;    // blocks launched per SM; a block works only if it is among the first on its SM
 constexpr int kQueueCap = 4096;   // cost-model queue of the scoring kernel (entries), drained when it may fill up
 
 struct DevSched {
@@ -154,7 +150,7 @@ struct pf_plan {
     // the survivor selection and the simulator.  Streams and fork / join events belong to the plan (training
     // plans; created with the plan).
     cudaStream_t side_stream, fill_stream;
-    cudaEvent_t ev_fork, ev_join, ev_fork2, ev_fork3, ev_fill, ev_count, ev_compact;
+    cudaEvent_t ev_fork, ev_join, ev_fork3, ev_fill, ev_count, ev_compact;
     // simulator order tables (built at create for training plans)
     void *sim_tables;
     unsigned int *d_fill_ctl;      // queue head and per-SM block counts of the fill kernels (2 KB)
@@ -378,7 +374,6 @@ struct FillArgs {
     const uint32_t *order, *order_hdr;
     // the queue of constant slabs and the per-SM registration of the kernel's blocks (plan-owned, zeroed per call)
     unsigned int *ticket, *sm_slots;
-    const unsigned int *stop;      // may be NULL; once the word is non-zero the launch draws no further slab
     unsigned int *done;            // counts the slabs the launch has filled
     uint32_t per_sm;               // working blocks per SM
     uint32_t piece, issuers;       // zeros travel as bulk copies of `piece` bytes, issued by the first `issuers` threads
@@ -388,27 +383,23 @@ struct FillArgs {
 // How a scoring call may spread over the plan's streams (all off: one stream, one scoring kernel).
 //   topk_aside: the key-list reduction runs on side_stream; ev_join is recorded when it is done.
 //   fill_aside: the scoring kernel visits the evaluated slabs only (plus `fills_per_evaluated` constant ones each);
-//               the remaining constant slabs are left to a second, lean kernel that the caller starts on
-//               fill_stream when it sees fit (fill_launch); ev_fill is recorded when that is done.
+//               the remaining constant slabs are left to a second, lean kernel that is started on fill_stream
+//               right behind the scoring kernel; ev_fill is recorded when that is done.
 // The caller makes its stream wait for the events it was told were recorded (*joined bits) before it touches
 // the workspace (ev_join) or lets the call's results count as complete (ev_fill).
 struct ScoreSpread {
     bool topk_aside = false, fill_aside = false;
     int fills_per_evaluated = kFillsPerEvaluated;
     bool join_pending = false, fill_pending = false;   // out: events the caller still has to wait for
-    bool fill_deferred = false;                        // out: constant slabs are still to be streamed (fill_launch)
-    FillArgs fill;                                     // out: what fill_launch launches
-    FillGuard guard;                                   // out: set when fill_deferred
+    FillGuard guard;                                   // out: set when fill_pending
 };
-int fill_launch(pf_plan_t *p, ScoreSpread &sp, cudaStream_t st);
 // pf_compact's launches on `st`; guard: class bytes to trust instead of constant blocks still in flight (or NULL)
 int compact_run(pf_plan_t *p, uint64_t first, uint64_t count, const uint8_t *d_reason, const float *d_tput,
                 const int64_t *d_mem, uint64_t *d_hist, uint8_t *d_mask, pf_record_t *d_records, uint64_t record_cap,
                 uint64_t *d_n_feasible, void *d_workspace, cudaStream_t st, const FillGuard *guard);
 int simulate_run(pf_plan_t *p, const uint64_t *d_surv_idx, uint64_t n, const uint64_t *d_n, uint32_t jitter_seed,
                  float *d_tput_sim, uint8_t *d_sim_status, uint32_t k, uint64_t *d_topk_idx, float *d_topk_score,
-                 uint32_t *d_topk_count, void *d_workspace, size_t workspace_bytes, cudaStream_t st,
-                 ScoreSpread *spread);
+                 uint32_t *d_topk_count, void *d_workspace, size_t workspace_bytes, cudaStream_t st);
 
 // internal entry points behind pf_score / pf_select_survivors (dg / have_digest: the fused search call)
 int score_run(pf_plan_t *p, uint64_t first, uint64_t count, uint8_t *d_reason, float *d_tput, int64_t *d_mem,

@@ -710,7 +710,7 @@ __global__ void __launch_bounds__(kThreads) fill_tail_kernel(const FillArgs A)
     // a block works only if it is among the first `per_sm` to register on its SM; the others leave at once, and the
     // scheduler keeps placing blocks until (nearly) every SM has its share.
     __shared__ __align__(128) uint8_t s_src[kFillZeroBytes + kFillReasonBytes];
-    __shared__ unsigned int s_go, s_t, s_more;
+    __shared__ unsigned int s_go, s_t;
     const uint32_t tid = threadIdx.x;
     if (tid == 0) {
         unsigned int smid;
@@ -737,15 +737,8 @@ __global__ void __launch_bounds__(kThreads) fill_tail_kernel(const FillArgs A)
         const uint32_t tk = s_t;
         __syncthreads();
         if (head_n + tk >= A.n_slabs) break;
-        // Thread 0 decides for the block whether another slab follows.  Once the hand-over word is set the slab the
-        // block has already drawn is still filled here, then the block leaves (one slab per block at most: cheaper
-        // than handing tickets back).
         uint32_t tk_next = 0;
-        bool more = true;
-        if (tid == 0) {
-            more = !(A.stop && *reinterpret_cast<const volatile unsigned int *>(A.stop) != 0u);
-            if (more) tk_next = atomicAdd(A.ticket, 1u);   // in flight while this slab is stored
-        }
+        if (tid == 0) tk_next = atomicAdd(A.ticket, 1u);   // in flight while this slab is stored
         const uint32_t w = __ldg(A.order + head_n + tk);
         const uint64_t base = (A.slab_lo + (w & 0xFFFFFFu)) * (uint64_t)A.slab;
         const uint64_t lo = base > A.first ? base : A.first;
@@ -776,11 +769,9 @@ __global__ void __launch_bounds__(kThreads) fill_tail_kernel(const FillArgs A)
         }
         if (tid == 0) {
             s_t = tk_next;
-            s_more = more ? 1u : 0u;
             atomicAdd(A.done, 1u);   // slabs this launch has taken (accounting only)
         }
         __syncthreads();
-        if (!s_more) break;
     }
     // the block's copies must have been written before it ends (the zero buffer goes away with the block, and the
     // end of the kernel is what the rest of the call waits for)
@@ -1068,41 +1059,6 @@ __global__ void __launch_bounds__(kThreads) merge2_kernel(const Merge2Args A)
     if (tid == 0) *A.cnt_out = (uint32_t)n;
 }
 
-// Start streaming the constant slabs a split scoring call left behind: on the plan's fill stream, after everything
-// `st` holds so far.  Records ev_fill behind the kernel; the caller makes `st` wait for it before the call's
-// results count as complete.
-int fill_launch(pf_plan_t *p, ScoreSpread &sp, cudaStream_t st)
-{
-    if (!sp.fill_deferred) return PF_OK;
-    sp.fill_deferred = false;
-    cudaStream_t fs = p->fill_stream;
-    // tell the fill launch that started with the call to draw no further slab: this one takes the queue over
-    PF_CUDA_TRY(cudaMemsetAsync(p->d_fill_ctl + 1, 0xFF, 4, st), "fill hand-over");
-    PF_CUDA_TRY(cudaEventRecord(p->ev_fork2, st), "fill fork");
-    PF_CUDA_TRY(cudaStreamWaitEvent(fs, p->ev_fork2, 0), "fill fork");
-    // from here on the fill stream is forked: record the join event whatever happens
-    timing_begin(p, PF_T_FILL, fs);
-    {
-        FillArgs f = sp.fill;
-        f.stop = nullptr;                      // this launch empties the queue
-        f.done = p->d_fill_ctl + 3;
-        f.sm_slots = p->d_fill_ctl + 256 + 16;
-        f.per_sm = kFillBlocksPerSm;
-        f.piece = kFillZeroBytes;
-        f.issuers = kFillThreads;
-        fill_tail_kernel<<<p->sm_count * kFillGridPerSm, kFillThreads, 0, fs>>>(f);
-    }
-    count_launch();
-    timing_end(p, PF_T_FILL, 1, fs);
-    const cudaError_t e = cudaGetLastError();
-    if (cudaEventRecord(p->ev_fill, fs) == cudaSuccess) sp.fill_pending = true;
-    if (e != cudaSuccess) {
-        set_cuda_error(e, "fill_tail_kernel launch");
-        return PF_ECUDA;
-    }
-    return PF_OK;
-}
-
 static int grid_for(const pf_plan_t *p, uint64_t n_slabs)
 {
     uint64_t g = (uint64_t)p->sm_count * 4;
@@ -1144,7 +1100,7 @@ int pf::score_run(pf_plan_t *p, uint64_t first, uint64_t count, uint8_t *d_reaso
 {
     ScoreSpread plain;
     ScoreSpread &sp = spread ? *spread : plain;
-    sp.join_pending = sp.fill_pending = sp.fill_deferred = false;
+    sp.join_pending = sp.fill_pending = false;
     if (!p) return PF_EINVAL;
     if (k > PF_K_MAX) return PF_EINVAL;
     if (k > 0 && (!d_topk_idx || !d_topk_score || !d_topk_count)) return PF_EINVAL;
@@ -1218,19 +1174,17 @@ int pf::score_run(pf_plan_t *p, uint64_t first, uint64_t count, uint8_t *d_reaso
         a.order_hdr = hdr;
         a.head_only = split ? 1u : 0u;
     }
+    FillArgs f;
     if (split) {
-        // The constant slabs start to stream at once, by a first launch of the fill kernel on the plan's fill
-        // stream that runs beside the scoring kernel, the selection and the simulator's pre-pass, until the launch
-        // beside the simulator kernel takes the queue over (fill_launch).  Queue head, hand-over word and block
-        // registrations start at zero.
+        // The constant slabs are streamed by the fill kernel on the plan's fill stream, beside this kernel and
+        // everything that follows it in the call.  Queue head and block registrations start at zero.
         PF_CUDA_TRY(cudaMemsetAsync(p->d_fill_ctl, 0, 2048, st), "fill control reset");
-        FillArgs &f = sp.fill;
         f.first = first; f.count = count; f.slab_lo = slab_lo; f.n_slabs = (uint32_t)n_slabs;
         f.slab = p->dev.slab; f.order_tail = a.order_tail; f.order_fpe = a.order_fpe;
         f.chk = p->dev.chk;
         f.reason = d_reason; f.tput = d_tput; f.mem = (long long *)d_mem;
         f.order = a.order; f.order_hdr = a.order_hdr;
-        f.ticket = p->d_fill_ctl; f.stop = p->d_fill_ctl + 1; f.done = p->d_fill_ctl + 2;
+        f.ticket = p->d_fill_ctl; f.done = p->d_fill_ctl + 2;
         f.sm_slots = p->d_fill_ctl + 16; f.per_sm = 1;
         PF_CUDA_TRY(cudaEventRecord(p->ev_fork3, st), "early fill fork");
         PF_CUDA_TRY(cudaStreamWaitEvent(p->fill_stream, p->ev_fork3, 0), "early fill fork");
@@ -1253,17 +1207,16 @@ int pf::score_run(pf_plan_t *p, uint64_t first, uint64_t count, uint8_t *d_reaso
     timing_end(p, PF_T_SCORE, n_score_kernels, st);
     PF_CUDA_TRY(cudaGetLastError(), "score_kernel launch");
     if (split) {
-        // The fill kernel's first launch is issued after the scoring kernel (on the fill stream it waits only for
+        // The fill kernel is issued after the scoring kernel (on the fill stream it waits only for
         // what preceded that kernel), so that the two reach the device in the same order whether or not the host
         // runs ahead of it: a grid that arrives first is handed out to the end before the next one starts, and this
         // one is deliberately long.
-        FillArgs &f = sp.fill;
-        timing_begin(p, PF_T_FILL_EARLY, p->fill_stream);
+        timing_begin(p, PF_T_FILL, p->fill_stream);
         f.piece = kFillZeroBytes;
-        f.issuers = kFillEarlyIssuers;
-        fill_tail_kernel<<<p->sm_count * kFillEarlyGridPerSm, kFillThreads, 0, p->fill_stream>>>(f);
+        f.issuers = kFillThreads;
+        fill_tail_kernel<<<p->sm_count * kFillGridPerSm, kFillThreads, 0, p->fill_stream>>>(f);
         count_launch();
-        timing_end(p, PF_T_FILL_EARLY, 1, p->fill_stream);
+        timing_end(p, PF_T_FILL, 1, p->fill_stream);
         const cudaError_t e_early = cudaGetLastError();
         // the fill stream is forked from here on: the join event is recorded whatever happens next
         if (cudaEventRecord(p->ev_fill, p->fill_stream) == cudaSuccess) sp.fill_pending = true;
@@ -1276,9 +1229,7 @@ int pf::score_run(pf_plan_t *p, uint64_t first, uint64_t count, uint8_t *d_reaso
     int rc = PF_OK;
     if (topk_aside) PF_CUDA_TRY(cudaEventRecord(p->ev_fork, st), "score fork");
     if (split) {
-        // the caller decides when the second fill launch takes over (fill_launch); until the fills have joined, only
-        // the evaluated slabs of the dense outputs hold results (guard)
-        sp.fill_deferred = true;
+        // until the fill stream has joined, only the evaluated slabs of the dense outputs hold results (guard)
         sp.guard.cls = (const uint8_t *)(a.order + p->order_cap);
         sp.guard.hdr = a.order_hdr;
         sp.guard.slab_lo = slab_lo; sp.guard.n_slabs = (uint32_t)n_slabs; sp.guard.slab = p->dev.slab;

@@ -94,9 +94,8 @@ static int search_device(pf_plan_t *p, uint32_t k, uint64_t s_max, uint32_t k_si
     // With a simulator tier to follow, the call spreads over the plan's streams.  The scoring kernel deals with the
     // evaluated slabs only (every feasible plan, the digest and the top-k keys come from those); the analytic top-k
     // is reduced on the second stream beside the selection; the constant slabs (most of the dense outputs' bytes,
-    // which nothing downstream reads) are streamed by the fill kernel on the fill stream, from the start of the call
-    // and, in a second launch that takes the first one's queue over, beside the simulator kernel and the re-ranking (which
-    // reads simulator scores only); the fill stream joins last.  The simulator reuses the scoring scratch, so the
+    // which nothing downstream reads) are streamed by the fill kernel on the fill stream, from right behind the
+    // scoring kernel to the end of the call; the fill stream joins last.  The simulator reuses the scoring scratch, so the
     // analytic top-k joins before it.
     ScoreSpread sp;
     sp.topk_aside = sim && p->side_stream != nullptr;
@@ -108,7 +107,7 @@ static int search_device(pf_plan_t *p, uint32_t k, uint64_t s_max, uint32_t k_si
         // the second stream is forked behind the scoring kernel and has the analytic top-k's reduction queued: the
         // compact view follows it there, reading evaluated blocks only while the constant ones are in flight
         cudaStream_t cs = p->side_stream;
-        const FillGuard *guard = (sp.fill_deferred || sp.fill_pending) ? &sp.guard : nullptr;
+        const FillGuard *guard = sp.fill_pending ? &sp.guard : nullptr;
         int rc2 = compact_run(p, 0, p->size, d_reason, d_tput, d_mem, cj->d_hist, cj->d_mask, cj->d_records,
                               cj->record_cap, cj->d_nfeas, cj->cws, cs, guard);
         cudaError_t e = cudaSuccess;
@@ -132,13 +131,12 @@ static int search_device(pf_plan_t *p, uint32_t k, uint64_t s_max, uint32_t k_si
     }
     if (rc == PF_OK && sim)
         rc = select_run(p, 0, p->size, d_reason, d_tput, s_max, d_surv, d_surv_cnt, ws_sel, ws_sel_bytes, st, true,
-                        (sp.fill_deferred || sp.fill_pending) ? &sp.guard : nullptr);
+                        sp.fill_pending ? &sp.guard : nullptr);
     // joins are unconditional once a fork has happened, error returns included
     if (sp.join_pending && cudaStreamWaitEvent(st, p->ev_join, 0) != cudaSuccess && rc == PF_OK) rc = PF_ECUDA;
     if (rc == PF_OK && sim)
         rc = simulate_run(p, d_surv, s_max, d_surv_cnt, jitter_seed, nullptr, nullptr, k_sim, d_sim_idx, d_sim_sc,
-                          d_sim_cnt, ws, ws_bytes, st, &sp);
-    if (rc == PF_OK && sp.fill_deferred) rc = fill_launch(p, sp, st);
+                          d_sim_cnt, ws, ws_bytes, st);
     if (sp.fill_pending && cudaStreamWaitEvent(st, p->ev_fill, 0) != cudaSuccess && rc == PF_OK) rc = PF_ECUDA;
     if (compact_forked && cudaStreamWaitEvent(st, p->ev_compact, 0) != cudaSuccess && rc == PF_OK) rc = PF_ECUDA;
     return rc;

@@ -1028,7 +1028,7 @@ static SimGeom sim_geom(int q_max)
 }
 
 template <typename RI>
-static int launch_simulate(pf_plan_t *p, SimArgs a, uint64_t n, cudaStream_t st, int *n_kernels, ScoreSpread *spread)
+static int launch_simulate(pf_plan_t *p, SimArgs a, uint64_t n, cudaStream_t st, int *n_kernels)
 {
     *n_kernels = 0;
     const SimGeom geo = sim_geom(a.q_max);
@@ -1043,13 +1043,6 @@ static int launch_simulate(pf_plan_t *p, SimArgs a, uint64_t n, cudaStream_t st,
     for (int i = 0; i < 3; i++) count_launch();
     timing_end(p, PF_T_SIMPREP, 3, st);
     PF_CUDA_TRY(cudaGetLastError(), "simulator pre-pass launch");
-    // Inside a search call the constant slabs of the dense outputs start to stream here, on the plan's fill
-    // stream: the kernel below works in shared memory and fetches ahead, whereas the short latency-bound launches
-    // before this point would crawl under a saturated store stream.
-    if (spread && spread->fill_deferred) {
-        const int rc = fill_launch(p, *spread, st);
-        if (rc != PF_OK) return rc;
-    }
     const uint64_t cap = (uint64_t)p->sm_count * geo.per_sm;
     const uint64_t want = (n + kSimThreads / 32 - 1) / (kSimThreads / 32);
     const int grid = (int)(want < cap ? want : cap);
@@ -1088,15 +1081,12 @@ extern "C" int pf_simulate(pf_plan_t *p, const uint64_t *d_surv_idx, uint64_t n,
                            size_t workspace_bytes, void *stream)
 {
     return pf::simulate_run(p, d_surv_idx, n, d_n, jitter_seed, d_tput_sim, d_sim_status, k, d_topk_idx, d_topk_score,
-                            d_topk_count, d_workspace, workspace_bytes, (cudaStream_t)stream, nullptr);
+                            d_topk_count, d_workspace, workspace_bytes, (cudaStream_t)stream);
 }
 
-// spread (the search call): a split scoring call's constant slabs are started beside the simulator kernel and
-// joined before the re-ranking, which is a chain of short launches again.
 int pf::simulate_run(pf_plan_t *p, const uint64_t *d_surv_idx, uint64_t n, const uint64_t *d_n, uint32_t jitter_seed,
                      float *d_tput_sim, uint8_t *d_sim_status, uint32_t k, uint64_t *d_topk_idx, float *d_topk_score,
-                     uint32_t *d_topk_count, void *d_workspace, size_t workspace_bytes, cudaStream_t st,
-                     ScoreSpread *spread)
+                     uint32_t *d_topk_count, void *d_workspace, size_t workspace_bytes, cudaStream_t st)
 {
     if (!p || !d_surv_idx) return PF_EINVAL;
     if (p->dev.phase != PF_PHASE_TRAIN) return PF_EUNSUPPORTED;
@@ -1130,17 +1120,12 @@ int pf::simulate_run(pf_plan_t *p, const uint64_t *d_surv_idx, uint64_t n, const
     PF_CUDA_TRY(cudaMemsetAsync(ws + lay.off_ctrl, 0, kSimCtrlBytes, st), "pf_simulate: counter reset");
     if (n > 0) {
         int nk = 0;
-        rc = p->dev.wide ? launch_simulate<unsigned long long>(p, a, n, st, &nk, spread)
-                         : launch_simulate<uint32_t>(p, a, n, st, &nk, spread);
+        rc = p->dev.wide ? launch_simulate<unsigned long long>(p, a, n, st, &nk)
+                         : launch_simulate<uint32_t>(p, a, n, st, &nk);
         if (rc != PF_OK) return rc;
     }
-    if (spread) {
-        if (spread->fill_deferred) {   // nothing was simulated: the fills still have to go out
-            rc = fill_launch(p, *spread, st);
-            if (rc != PF_OK) return rc;
-        }
-        // the fill stream is joined by the caller, after the re-ranking below (which does not read the dense outputs)
-    }
+    // (inside a search call the fill stream is joined by the caller, after the re-ranking below, which does not read
+    // the dense outputs)
     if (k > 0) {
         int nk = 0;
         timing_begin(p, PF_T_TOPK, st);

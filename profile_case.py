@@ -5,7 +5,7 @@
 The cut keeps every axis of the benchmark's large space but three of its eleven expert-parallel degrees
 (49,065,984 candidates): 638 MB of dense outputs per call, larger than the 126 MB L2 but well under a few GB on the
 device, so that a multi-pass capture of one launch ends by itself quickly.  `search` runs the one-call search (the
-benchmark's step: scoring kernel, fill kernel beside the simulator kernel, selection, re-rank); the other stages run
+benchmark's step: scoring kernel, selection, simulator kernel and re-rank beside the fill kernel); the other stages run
 the separate entry points.
 """
 from __future__ import annotations
@@ -55,8 +55,7 @@ def main():
         span = plan.fill_span()
         fill = (span["n_blocks"] - span["scored_blocks"]) * span["block_candidates"]
         print(f"searched {plan.size} candidates; {int(bufs['surv_count'].item())} survivors; the fill kernel covers "
-              f"{fill} candidates ({span['n_blocks'] - span['scored_blocks']} of {span['n_blocks']} blocks, "
-              f"{span['early_fill_blocks']} of them in its first launch)")
+              f"{fill} candidates ({span['filled_blocks']} of {span['n_blocks']} blocks)")
     else:
         print(f"scored {plan.size} candidates; top-k holds {int(out['topk_count'].item())}"
               + (f"; {int(sel['surv_count'].item())} survivors" if sel is not None else ""))
