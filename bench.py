@@ -41,11 +41,11 @@ NOMINAL_HBM_GBS = 7700.0          # HGX B200 data-sheet figure, for context
 # DRAM traffic of the fill kernel (the dominant kernel of a step), from one ncu capture on the profiling slice
 # (profile_case.py: a 49 M-candidate cut of the same space; summary under profiles/): dram__bytes_read.sum +
 # dram__bytes_write.sum of one fill_tail_kernel launch there, and the candidates that launch covers.  The kernel
-# writes every byte once and reads nothing (0.1 MB read): the capture shows 543.1 MB of DRAM traffic for 602.1 MB
-# of dense outputs -- the difference, 59.0 MB, is what still sat dirty in the 126 MB L2 when the kernel ended, a
+# writes every byte once and reads nothing (0.1 MB read): the capture shows 542.4 MB of DRAM traffic for 602.1 MB
+# of dense outputs -- the difference, 59.7 MB, is what still sat dirty in the 126 MB L2 when the kernel ended, a
 # constant of the cache, not of the workload.  A full-space launch is therefore reported as its algorithmic bytes
 # minus that residue.
-FILL_KERNEL_SLICE_DRAM_BYTES = 543_096_576
+FILL_KERNEL_SLICE_DRAM_BYTES = 542_420_224
 FILL_KERNEL_SLICE_CANDIDATES = 46_313_472
 # thread-level instructions one simulated op needs at least: load the dependency's end, add the hand-over latency,
 # max with the rank's clock, add the duration, store the result, advance the cursor
