@@ -428,8 +428,13 @@ inline TopkLayout topk_layout(uint64_t n_keys_max, uint32_t k)
     l.off_ctrl = 0;
     l.off_keys_a = 256;
     size_t a = ((size_t)n_keys_max * 8 + 255) & ~(size_t)255;
+    // the second list: what pass 1 of the reduction leaves -- at most k keys from each of at most kFastKeys / k
+    // blocks, and never more keys than went in (the older, larger bound is kept so that workspace sizes stay put)
     size_t blocks = (n_keys_max + kReduceSeg - 1) / kReduceSeg;
-    size_t b = (blocks * kk * 8 + 255) & ~(size_t)255;
+    size_t keys_b = blocks * kk;
+    const size_t short_list = n_keys_max < (size_t)kFastKeys ? (size_t)n_keys_max : (size_t)kFastKeys;
+    if (keys_b < short_list) keys_b = short_list;
+    size_t b = (keys_b * 8 + 255) & ~(size_t)255;
     l.off_keys_b = l.off_keys_a + a;
     l.total = l.off_keys_b + b;
     return l;

@@ -788,7 +788,6 @@ struct ReduceArgs {
     unsigned long long *out;        // compact keys of the next pass (when not final)
     unsigned int *out_count;
     uint32_t k;
-    unsigned int seg;               // keys per block
     int final;                      // 1: write idx / score / count (gridDim.x == 1)
     uint64_t first;
     const uint64_t *idx_map;        // NULL: idx = first + rel; else idx = idx_map[rel]
@@ -797,11 +796,11 @@ struct ReduceArgs {
     uint32_t *topk_count;
 };
 
-// Block b walks keys [b*seg, (b+1)*seg) of the input one tile at a time, admitting only keys above its
-// running k-th best, and keeps the k best.  A tile's admissions are counted before they are appended, so the
-// buffer is pruned only when it would really overflow.
-// Pass 1: every block reduces one segment of kReduceSeg keys to its k best and appends them to the second list.
-// A producers' list of at most kFastKeys keys is left to the final kernel, which sorts it in one go.
+// Pass 1, for a producers' list longer than kFastKeys keys: the list is cut into as many segments as the grid has
+// blocks -- few enough that what the blocks leave (at most k keys each) fits the final kernel's one-go sort -- and
+// block b walks its segment one tile at a time, admitting only keys above its running k-th best, and keeps the k
+// best.  A tile's admissions are counted before they are appended, so the buffer is pruned only when it would
+// really overflow.  A shorter list is left to the final kernel as it is.
 __global__ void __launch_bounds__(kReduceThreads) reduce_kernel(const ReduceArgs A)
 {
     __shared__ unsigned long long s_buf[kTopkCap];
@@ -811,8 +810,9 @@ __global__ void __launch_bounds__(kReduceThreads) reduce_kernel(const ReduceArgs
     const int tid = threadIdx.x, k = (int)A.k;
     const unsigned int n = *A.in_count;
     if (n <= (unsigned int)kFastKeys) return;
-    const unsigned int lo = blockIdx.x * A.seg;
-    const unsigned int hi = min(lo + A.seg, n);
+    const unsigned int seg = (n + gridDim.x - 1) / gridDim.x;
+    const unsigned int lo = blockIdx.x * seg;
+    const unsigned int hi = min(lo + seg, n);
     if (lo >= hi) return;
     if (tid == 0) {
         s_count = 0;
@@ -849,12 +849,18 @@ __global__ void __launch_bounds__(kReduceThreads) reduce_final_kernel(const Redu
     __shared__ unsigned int s_need;
     __shared__ int s_stop;
     const int tid = threadIdx.x, k = (int)A.k;
-    const unsigned int n0 = *A.in0_count;
+    // the list to finish: the producers' own when it is short, else what pass 1 left of it (short by construction)
+    unsigned int n0 = *A.in0_count;
+    const unsigned long long *src0 = A.in0;
+    if (n0 > (unsigned int)kFastKeys) {
+        n0 = *A.in_count;
+        src0 = A.in;
+    }
     unsigned long long *s_out = s_big;
     int c;
     if (n0 <= (unsigned int)kFastKeys) {
         s_out = s_big + kFastKeys;
-        for (unsigned int i = tid; i < n0; i += kReduceThreads) s_big[i] = A.in0[i];
+        for (unsigned int i = tid; i < n0; i += kReduceThreads) s_big[i] = src0[i];
         if (tid == 0) {
             s_prefix = 0ull;
             s_need = (unsigned int)k;
@@ -969,15 +975,15 @@ int launch_topk_reduce(void *d_workspace, const TopkLayout &lay, uint64_t n_keys
     unsigned long long *in = (unsigned long long *)(ws + lay.off_keys_a);
     unsigned long long *out = (unsigned long long *)(ws + lay.off_keys_b);
     *n_kernels = 0;
-    // pass 1 spreads a long list over blocks of kReduceSeg keys; whatever it leaves (at most k keys per block) is
-    // finished by one block; a short list goes to that block directly
+    // pass 1 spreads a long list over so few blocks that what they leave (at most k keys each) is a short list;
+    // one block finishes a short list, the producers' own or that one
     ReduceArgs r;
     r.in = in; r.in_count = ctrl + 1; r.out = out; r.out_count = ctrl + 2;
     r.in0 = in; r.in0_count = ctrl + 1;
     r.k = k; r.final = 0; r.first = first; r.idx_map = d_idx_map;
-    r.seg = (unsigned int)kReduceSeg;
     r.topk_idx = d_topk_idx; r.topk_score = d_topk_score; r.topk_count = d_topk_count;
-    const uint64_t blocks = (n_keys_max + kReduceSeg - 1) / kReduceSeg;
+    uint64_t blocks = (uint64_t)kFastKeys / (k ? k : 1);
+    blocks = blocks < 1 ? 1 : (blocks > 256 ? 256 : blocks);
     if (n_keys_max > (uint64_t)kFastKeys) {
         reduce_kernel<<<(unsigned int)blocks, kReduceThreads, 0, st>>>(r);
         count_launch();
