@@ -47,6 +47,10 @@ NOMINAL_HBM_GBS = 7700.0          # HGX B200 data-sheet figure, for context
 # minus that residue.
 FILL_KERNEL_SLICE_DRAM_BYTES = 542_420_224
 FILL_KERNEL_SLICE_CANDIDATES = 46_313_472
+# thread-level instructions the scoring kernel issues per plan that goes through the memory model, the step-time
+# model and the price: smsp__thread_inst_executed.sum with the memory gate lifted minus with the gate on, over the
+# plans the gate had rejected (ncu, profile_case.py --config large_unconstrained --topk-only; summary under profiles/)
+COSTED_PLAN_THREAD_INSTRUCTIONS = 2780
 # thread-level instructions one simulated op needs at least: load the dependency's end, add the hand-over latency,
 # max with the rank's clock, add the duration, store the result, advance the cursor
 SIM_INSTR_PER_OP = 6
@@ -365,7 +369,13 @@ def _config_lines(torch, stream, hbm, peaks):
                 "t_alu_ms": t_alu * 1e3, "t_hbm_ms": t_hbm * 1e3, "score_kernel_ms": head_ms,
                 "note": "the scoring kernel of this call writes the evaluated blocks only; its ALU work is the feasible "
                         "candidates' cost model plus the rule tables",
-                "alu_frac_of_score_kernel": t_alu * 1e3 / head_ms if head_ms else None}
+                "alu_frac_of_score_kernel": t_alu * 1e3 / head_ms if head_ms else None,
+                # from the ncu capture summarised under profiles/ (score kernel, cost-heavy slice): what the
+                # compiled kernel issues per plan it takes through the cost model, and the issue-rate bound on that
+                "issued_thread_instructions_per_costed_plan": COSTED_PLAN_THREAD_INSTRUCTIONS,
+                "t_issue_ms": n_feas * COSTED_PLAN_THREAD_INSTRUCTIONS / peaks["logic"] * 1e3,
+                "issue_frac_of_score_kernel": (n_feas * COSTED_PLAN_THREAD_INSTRUCTIONS / peaks["logic"] * 1e3 / head_ms
+                                               if head_ms else None)}
         out[label] = line
         rig.close()
         del rig

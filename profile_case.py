@@ -1,6 +1,7 @@
 """A small, fixed workload for profiler captures (ncu): a cut of the large training space.
 
-  python profile_case.py [--launches 3] [--stage search|score|select|simulate] [--config large]
+  python profile_case.py [--launches 3] [--stage search|score|select|simulate] [--config large] [--lift-gate]
+                         [--topk-only]
 
 The cut keeps every axis of the benchmark's large space but three of its eleven expert-parallel degrees
 (49,065,984 candidates): 638 MB of dense outputs per call, larger than the 126 MB L2 but well under a few GB on the
@@ -37,15 +38,22 @@ def main():
     ap.add_argument("--launches", type=int, default=3)
     ap.add_argument("--stage", default="search", choices=("search", "score", "select", "simulate"))
     ap.add_argument("--config", default="large")
+    ap.add_argument("--lift-gate", action="store_true",
+                    help="raise the memory budget so that no plan is rejected by the gate (with --config "
+                         "large_unconstrained: every plan that passes the integer rules goes through the cost model)")
+    ap.add_argument("--topk-only", action="store_true", help="stage score: no dense outputs, top-k only")
     args = ap.parse_args()
 
-    plan = Plan(slice_config(args.config))
+    cfg = slice_config(args.config)
+    if args.lift_gate:
+        cfg["cluster"]["budget_bytes"] = 10 ** 15
+    plan = Plan(cfg)
     bufs = out = sel = None
     for _ in range(args.launches):
         if args.stage == "search":
             bufs = plan.search(1024, 1_000_000, 100, 4, bufs=bufs)
             continue
-        out = plan.score(k=1024)
+        out = plan.score(k=1024, dense=not args.topk_only)
         if args.stage in ("select", "simulate"):
             sel = plan.select_survivors(out["reason"], out["tput"], 1_000_000)
         if args.stage == "simulate":
