@@ -448,13 +448,23 @@ __global__ void __launch_bounds__(kThreads, 4) score_kernel(const __grid_constan
                         // the selection's first pass, done here for the few feasible plans inside the simulator's
                         // domain: score-bit histograms, the chunk's eligible count, the list of non-empty chunks
                         if (A.dg.hist1 && tput != 0.f && c.pp <= PF_SIM_MAX_RANKS && D.v_eff <= PF_SIM_MAX_V) {
+                            // lanes of the warp that add to the same word do it in one atomic (a slab's plans share
+                            // a chunk or two and most of their score's leading bits): where many plans are feasible
+                            // these atomics, issued under a saturated store stream, are what the drain waits for
                             const uint32_t bits = __float_as_uint(tput);
-                            atomicAdd(A.dg.hist1 + PF_AT(P.chk, bits >> 16, 65536, PF_SITE_DIGEST), 1u);
-                            atomicAdd(A.dg.coarse1 + PF_AT(P.chk, bits >> 24, 256, PF_SITE_DIGEST), 1u);
+                            const int lane2 = tid & 31;
+                            const unsigned here = __activemask();
                             const uint32_t n_chunks = (uint32_t)((A.count + A.dg.chunk - 1) / A.dg.chunk);
                             (void)n_chunks;
                             const uint32_t chunk = (uint32_t)PF_AT(P.chk, o / A.dg.chunk, n_chunks, PF_SITE_CHUNK);
-                            if (atomicAdd(A.dg.elig + chunk, 1u) == 0u)
+                            const unsigned p1 = __match_any_sync(here, bits >> 16);
+                            if (lane2 == __ffs(p1) - 1)
+                                atomicAdd(A.dg.hist1 + PF_AT(P.chk, bits >> 16, 65536, PF_SITE_DIGEST), (unsigned)__popc(p1));
+                            const unsigned p2 = __match_any_sync(here, bits >> 24);
+                            if (lane2 == __ffs(p2) - 1)
+                                atomicAdd(A.dg.coarse1 + PF_AT(P.chk, bits >> 24, 256, PF_SITE_DIGEST), (unsigned)__popc(p2));
+                            const unsigned p3 = __match_any_sync(here, chunk);
+                            if (lane2 == __ffs(p3) - 1 && atomicAdd(A.dg.elig + chunk, (unsigned)__popc(p3)) == 0u)
                                 A.dg.list[PF_AT(P.chk, atomicAdd(A.dg.n_list, 1u), n_chunks, PF_SITE_CHUNK)] = chunk;
                         }
                     }
