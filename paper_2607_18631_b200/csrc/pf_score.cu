@@ -1201,7 +1201,7 @@ int pf::score_run(pf_plan_t *p, uint64_t first, uint64_t count, uint8_t *d_reaso
         f.reason = d_reason; f.tput = d_tput; f.mem = (long long *)d_mem;
         f.order = a.order; f.order_hdr = a.order_hdr;
         f.ticket = p->d_fill_ctl; f.done = p->d_fill_ctl + 2;
-        f.sm_slots = p->d_fill_ctl + 16; f.per_sm = 1;
+        f.sm_slots = p->d_fill_ctl + 16; f.per_sm = kFillBlocksPerSm;
         PF_CUDA_TRY(cudaEventRecord(p->ev_fork3, st), "early fill fork");
         PF_CUDA_TRY(cudaStreamWaitEvent(p->fill_stream, p->ev_fork3, 0), "early fill fork");
     }

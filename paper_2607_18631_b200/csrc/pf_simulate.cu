@@ -10,9 +10,9 @@
 // Launch structure: a counting-sort pre-pass (classify, offsets, scatter) bins the survivors by
 // (timeline size class, lane-group width 8/16/32, schedule kind), then ONE simulate_kernel launch serves all
 // bins, largest timelines first.  Every warp owns a slice of the block's shared memory and runs its own
-// candidates there; the timeline is one signed 32-bit word per (stage stream, microbatch) -- 0 nothing
-// finished, +t forward ended at t, -t backward ended at t -- written by its owner lane and polled by the
-// neighbour.  No block barrier is used, and a warp whose lanes make no progress for 64 rounds reports its
+// candidates there; the timeline is one signed 32-bit word per (stage stream, microbatch), microbatch-major (word
+// j * streams + stream, so that the lanes of a group touch neighbouring words) -- 0 nothing finished, +t forward
+// ended at t, -t backward ended at t -- written by its owner lane and polled by the neighbour.  No block barrier is used, and a warp whose lanes make no progress for 64 rounds reports its
 // unfinished candidates as PF_SIM_STALL, so every loop is bounded by the op count.
 #include <cstdlib>
 #include <cstring>
@@ -448,9 +448,10 @@ __global__ void __launch_bounds__(256) sim_records_kernel(const __grid_constant_
 }
 
 // The round loops, one per schedule class (all candidates of a batch share the class).  The timeline has one
-// 32-bit word per (stage stream, microbatch): 0 = nothing finished, +t = forward ended at t, -t = backward ended
-// at t.  In every round a lane runs at most its next op, and only if the word it depends on already carries the
-// right sign; the body is branch-free apart from that test.  Every 64 rounds some lane of the warp must have
+// 32-bit word per (stage stream, microbatch), at index microbatch * streams + stream: 0 = nothing finished, +t =
+// forward ended at t, -t = backward ended at t.  In every round a lane runs at most its next op, and only if the
+// word it depends on already carries the right sign; a step's results are selected by that test, not branched
+// around.  Every 64 rounds some lane of the warp must have
 // advanced, otherwise the loop ends and the unfinished candidates are reported as stalled.
 #define PF_SIM_ROUND_END()                                               \
     if (!__any_sync(0xFFFFFFFFu, done < total_ops)) break;               \
