@@ -8,12 +8,15 @@
 // the backward of stage q+1; the op's own forward is already behind the lane's clock.
 //
 // Launch structure: a counting-sort pre-pass (classify, offsets, scatter) bins the survivors by
-// (timeline size class, lane-group width 8/16/32, schedule kind), then ONE simulate_kernel launch serves all
+// (timeline size class, lane-group width 4/8/16/32, round loop), then ONE simulate_kernel launch serves all
 // bins, largest timelines first.  Every warp owns a slice of the block's shared memory and runs its own
 // candidates there; the timeline is one signed 32-bit word per (stage stream, microbatch), microbatch-major (word
 // j * streams + stream, so that the lanes of a group touch neighbouring words) -- 0 nothing finished, +t forward
-// ended at t, -t backward ended at t -- written by its owner lane and polled by the neighbour.  No block barrier is used, and a warp whose lanes make no progress for 64 rounds reports its
-// unfinished candidates as PF_SIM_STALL, so every loop is bounded by the op count.
+// ended at t, -t backward ended at t -- written by its owner lane and polled by the neighbour.  In a large call
+// (kSimRingMinSurvivors) interleaved schedules run on a ring of 2 pp microbatch slots per stage stream instead
+// (tagged two-word slots), which lets more candidates share a warp, and pipelines of depth <= 4 take four lanes.
+// No block barrier is used, and a warp whose lanes make no progress for 64 rounds reports its unfinished
+// candidates as PF_SIM_STALL, so every loop is bounded by the op count.
 #include <cstdlib>
 #include <cstring>
 #include <vector>
@@ -182,12 +185,32 @@ __device__ __forceinline__ float jitter(uint32_t cand_hash, int q, int is_b)
 }
 
 constexpr int kSimClasses = 7;          // timeline sizes 256 << c entries (stage streams x microbatches)
-constexpr int kSimGroups = 3;           // lanes per candidate: 8, 16 or 32 (pipeline depth rounded up)
-constexpr int kSimKinds = 3;            // schedule class: candidates of one batch share the round loop
-constexpr int kSimBins = kSimClasses * kSimGroups * kSimKinds;
+constexpr int kSimGroups = 4;           // lanes per candidate: 4, 8, 16 or 32 (pipeline depth rounded up)
+constexpr int kSimKinds = 4;            // round loop of a batch: the three schedule classes, and the interleaved one
+                                        // on a ring timeline (kSimKindRing)
+constexpr int kSimKindRing = 3;
+constexpr int kSimBins = kSimClasses * kSimGroups * kSimKinds;   // 112
+constexpr int kSimTab = 128;            // queue tables: bins rounded up to four per lane
 constexpr int kSimThreads = 128;        // 4 warps per block, each with its own shared-memory slice
 __host__ __device__ inline int sim_class_entries(int c) { return 256 << c; }
-__host__ __device__ inline int sim_group_lanes(int g) { return 8 << g; }
+__host__ __device__ inline int sim_group_lanes(int g) { return 4 << g; }
+// (four-lane groups only in large calls, like ring timelines: see kSimRingMinSurvivors)
+__host__ __device__ inline int sim_group_of(int pp, bool narrow) { return (pp <= 4 && narrow) ? 0 : (pp <= 8 ? 1 : (pp <= 16 ? 2 : 3)); }
+// stages a lane group's duration tables must hold: the plan-wide bound, or what the group's ranks can carry
+__host__ __device__ inline int sim_group_stages(int lanes, int q_max)
+{
+    const int by_ranks = lanes * PF_SIM_MAX_V;
+    return by_ranks < q_max ? by_ranks : q_max;
+}
+// An interleaved schedule keeps few microbatches of a stage in flight, so its timeline can be a ring of W = 2 pp
+// microbatch slots per stage stream (a multiple of the order's window of pp microbatches) instead of one word per
+// microbatch; a slot is then two words, tag and time, so that a reader can tell the lap.  Worth it when that is at
+// least a size class smaller AND the call is large: a ring step costs a few instructions more than a full-timeline
+// step, which a call of few survivors (bound by its longest op chain, warps to spare) feels, whereas a large call is
+// bound by how many candidates a warp instruction serves (12,905 survivors: 0.147 ms full, 0.170 ms ring; 1e6: 6.6 ms
+// full, 5.0 ms ring).
+__host__ __device__ inline int sim_ring_slots(int pp) { return 2 * pp; }
+constexpr uint64_t kSimRingMinSurvivors = 32768;
 
 // What the simulator kernel needs about one survivor, worked out once by the pre-pass (one thread per survivor)
 // instead of by every lane of the group that simulates it: the per-layer times, the hand-over latency, the rest of
@@ -199,10 +222,11 @@ struct __align__(16) SimRec {
     uint32_t pad[4];
 };
 static_assert(sizeof(SimRec) == 64, "SimRec is read as four 16-byte words");
-// meta: pp - 1 (5 bits) | v - 1 (3 bits) << 5 | kind (2 bits) << 8 | m_sim (7 bits) << 10
-__device__ __forceinline__ uint32_t sim_meta(int pp, int v, int kind, int m_sim)
+// meta: pp - 1 (5 bits) | v - 1 (3 bits) << 5 | kind (2 bits) << 8 | m_sim (7 bits) << 10 | ring timeline << 17
+__device__ __forceinline__ uint32_t sim_meta(int pp, int v, int kind, int m_sim, bool ring)
 {
-    return (uint32_t)(pp - 1) | ((uint32_t)(v - 1) << 5) | ((uint32_t)kind << 8) | ((uint32_t)m_sim << 10);
+    return (uint32_t)(pp - 1) | ((uint32_t)(v - 1) << 5) | ((uint32_t)kind << 8) | ((uint32_t)m_sim << 10) |
+           ((uint32_t)(ring ? 1 : 0) << 17);
 }
 
 struct SimArgs {
@@ -216,8 +240,8 @@ struct SimArgs {
     unsigned int *bin_count;        // [kSimBins] survivors per bin
     unsigned int *bin_off;          // [kSimBins + 1] start of each bin in the record array
     unsigned int *bin_fill;         // [kSimBins] scatter cursors
-    unsigned int *bin_seq;          // [64] bins in the order the batch queue serves them
-    unsigned int *batch_pre;        // [65] batches before each position of that order; [64] = all batches
+    unsigned int *bin_seq;          // [kSimTab] bins in the order the batch queue serves them
+    unsigned int *batch_pre;        // [kSimTab + 1] batches before each position of that order; last = all batches
     uint8_t *bin_of;                // [n] bin of each survivor (0xFF: not simulated)
     SimRec *recs;                   // [n] records, grouped by bin
     const int32_t *vals;
@@ -283,6 +307,19 @@ __device__ __forceinline__ void sim_shape(const SimCand<RI> &S, int &m_sim, int 
     if (kind == PF_KIND_INTERLEAVED) m_sim = (m_sim / pp) * pp;
     streams = kind == PF_KIND_DUALPIPE ? pp : pp * S.D.v_eff;   // DualPipe-style: 2 directions x m/2
 }
+// timeline words of a shape and whether it goes on a ring (interleaved schedules only; see sim_ring_slots)
+__device__ __forceinline__ int sim_entries(int kind, int pp, int streams, int m_sim, uint64_t n_call, bool &ring)
+{
+    const int full = streams * m_sim;
+    ring = false;
+    if (kind != PF_KIND_INTERLEAVED || m_sim <= sim_ring_slots(pp) || n_call < kSimRingMinSurvivors) return full;
+    const int on_ring = streams * sim_ring_slots(pp) * 2;
+    int c_full = 0, c_ring = 0;
+    while (c_full < kSimClasses - 1 && sim_class_entries(c_full) < full) c_full++;
+    while (c_ring < kSimClasses - 1 && sim_class_entries(c_ring) < on_ring) c_ring++;
+    ring = c_ring < c_full;
+    return ring ? on_ring : full;
+}
 
 // Pre-pass 1, one thread per survivor: decode it, run the predicate again (the list may hold anything), and
 //   - infeasible: score 0, status UNSUPPORTED, written here;
@@ -309,13 +346,16 @@ __global__ void __launch_bounds__(256) sim_classify_kernel(const __grid_constant
         if (S.reason == 0) {
             int m_sim, streams;
             sim_shape<RI>(S, m_sim, streams);
-            const int pp = S.c.pp, entries = streams * m_sim;
+            const int pp = S.c.pp;
+            bool ring;
+            const int entries = sim_entries(S.D.kind, pp, streams, m_sim, n, ring);
             int cls = 0;
             while (cls < kSimClasses - 1 && sim_class_entries(cls) < entries) cls++;
             const bool table_ok = S.D.kind != PF_KIND_DUALPIPE || __ldg(A.dual_off + pp * 33 + m_sim / 2) >= 0;
             if (pp <= PF_SIM_MAX_RANKS && S.D.v_eff <= PF_SIM_MAX_V && cls <= A.cls_hi &&
-                sim_class_entries(cls) >= entries && streams <= A.q_max && table_ok) {
-                bin = (cls * kSimGroups + (pp <= 8 ? 0 : (pp <= 16 ? 1 : 2))) * kSimKinds + S.D.kind;
+                sim_class_entries(cls) >= entries && streams <= A.q_max &&
+                streams <= sim_group_stages(sim_group_lanes(sim_group_of(pp, n >= kSimRingMinSurvivors)), A.q_max) && table_ok) {
+                bin = (cls * kSimGroups + sim_group_of(pp, n >= kSimRingMinSurvivors)) * kSimKinds + (ring ? kSimKindRing : S.D.kind);
                 direct = false;
             } else {
                 train_times<RI>(P, S.c, S.D, S.M, S.T);
@@ -339,8 +379,8 @@ __global__ void __launch_bounds__(256) sim_classify_kernel(const __grid_constant
 // Pre-pass 2 (one warp): where each bin's records start, and the batch queue: bins are served interleaved
 // schedules first, then DualPipe-style, then 1F1B (the per-rank op chains of an interleaved schedule are v times
 // longer, so the longest simulations start first and the kernel's tail is short), larger timelines first within a
-// class; batches are numbered through in that order.  Lane l owns bins / queue positions l and l + 32, so every
-// global word is read once, all loads in flight together.
+// class; batches are numbered through in that order.  Lane l owns bins / queue positions l, l + 32, l + 64 and
+// l + 96, so every global word is read once, all loads in flight together.
 __device__ __forceinline__ unsigned int warp_incl_scan(unsigned int x, int lane)
 {
 #pragma unroll
@@ -352,40 +392,55 @@ __device__ __forceinline__ unsigned int warp_incl_scan(unsigned int x, int lane)
 }
 __global__ void __launch_bounds__(32) sim_offsets_kernel(const SimArgs A)
 {
+    constexpr int kQ = kSimTab / 32;   // table entries per lane: lane l owns entries l, l + 32, ...
     const int lane = threadIdx.x;
-    const unsigned int c_lo = A.bin_count[lane];
-    const unsigned int c_hi = lane + 32 < kSimBins ? A.bin_count[lane + 32] : 0u;
-    const unsigned int i_lo = warp_incl_scan(c_lo, lane), i_hi = warp_incl_scan(c_hi, lane);
-    const unsigned int t_lo = __shfl_sync(0xFFFFFFFFu, i_lo, 31);
-    A.bin_off[lane] = i_lo - c_lo;
-    A.bin_off[lane + 32] = t_lo + i_hi - c_hi;        // entry kSimBins (lane 31) = all records
-    unsigned int nb[2];
-    int bin_at[2];
+    unsigned int cnt[kQ], incl[kQ];
+    unsigned int carry = 0;
 #pragma unroll
-    for (int h = 0; h < 2; h++) {
+    for (int h = 0; h < kQ; h++) {
+        const int b = lane + 32 * h;
+        cnt[h] = b < kSimBins ? A.bin_count[b] : 0u;
+    }
+#pragma unroll
+    for (int h = 0; h < kQ; h++) {
+        incl[h] = warp_incl_scan(cnt[h], lane);
+        A.bin_off[lane + 32 * h] = carry + incl[h] - cnt[h];     // entries kSimBins .. kSimTab - 1 = all records
+        carry += __shfl_sync(0xFFFFFFFFu, incl[h], 31);
+    }
+    // queue order: interleaved schedules on full timelines, on ring timelines, DualPipe-style, 1F1B; larger
+    // timelines first within each; position -> bin
+    unsigned int nb[kQ];
+    int bin_at[kQ];
+#pragma unroll
+    for (int h = 0; h < kQ; h++) {
         const int pos = lane + 32 * h;
         const bool valid = pos < kSimBins;
         const int ko = pos / (kSimClasses * kSimGroups), rem = pos - ko * (kSimClasses * kSimGroups);
         const int cls = kSimClasses - 1 - rem / kSimGroups, gi = rem % kSimGroups;
-        const int kind = (ko + 1) % kSimKinds;        // 0 -> interleaved, 1 -> DualPipe-style, 2 -> 1F1B
+        const int kind = ko == 0 ? PF_KIND_INTERLEAVED : ko == 1 ? kSimKindRing : ko == 2 ? PF_KIND_DUALPIPE : PF_KIND_1F1B;
         const int bin = valid ? (cls * kSimGroups + gi) * kSimKinds + kind : 0;
-        const unsigned int from_lo = __shfl_sync(0xFFFFFFFFu, c_lo, bin & 31);
-        const unsigned int from_hi = __shfl_sync(0xFFFFFFFFu, c_hi, bin & 31);
-        const unsigned int cnt = bin < 32 ? from_lo : from_hi;
+        unsigned int c = 0;
+#pragma unroll
+        for (int hh = 0; hh < kQ; hh++) {
+            const unsigned int from = __shfl_sync(0xFFFFFFFFu, cnt[hh], bin & 31);
+            if ((bin >> 5) == hh) c = from;
+        }
         bin_at[h] = bin;
         nb[h] = 0u;
         if (valid && cls <= A.cls_hi) {
             const unsigned int per = (unsigned int)sim_bin_batch(bin, A.cls_hi);
-            nb[h] = (cnt + per - 1) / per;
+            nb[h] = (c + per - 1) / per;
         }
     }
-    const unsigned int b_lo = warp_incl_scan(nb[0], lane), b_hi = warp_incl_scan(nb[1], lane);
-    const unsigned int bt_lo = __shfl_sync(0xFFFFFFFFu, b_lo, 31);
-    A.bin_seq[lane] = (unsigned int)bin_at[0];
-    A.bin_seq[lane + 32] = (unsigned int)bin_at[1];
-    A.batch_pre[lane] = b_lo - nb[0];
-    A.batch_pre[lane + 32] = bt_lo + b_hi - nb[1];
-    if (lane == 31) A.batch_pre[64] = bt_lo + b_hi;   // all batches
+    carry = 0;
+#pragma unroll
+    for (int h = 0; h < kQ; h++) {
+        const unsigned int b_incl = warp_incl_scan(nb[h], lane);
+        A.bin_seq[lane + 32 * h] = (unsigned int)bin_at[h];
+        A.batch_pre[lane + 32 * h] = carry + b_incl - nb[h];
+        carry += __shfl_sync(0xFFFFFFFFu, b_incl, 31);
+    }
+    if (lane == 31) A.batch_pre[kSimTab] = carry;   // all batches
 }
 
 // Pre-pass 3, one thread per survivor again: the binned ones get their record -- every term the simulator kernel
@@ -425,6 +480,8 @@ __global__ void __launch_bounds__(256) sim_records_kernel(const __grid_constant_
     }
     int m_sim, streams;
     sim_shape<RI>(S, m_sim, streams);
+    bool ring;
+    (void)sim_entries(S.D.kind, c.pp, streams, m_sim, n, ring);
     SimRec r;
     r.F_l = T.F_l; r.B_l = T.B_l; r.F_ld = T.F_ld; r.B_ld = T.B_ld;
     r.headF = T.headF; r.p = T.p;
@@ -437,7 +494,7 @@ __global__ void __launch_bounds__(256) sim_records_kernel(const __grid_constant_
     r.denom = denom;
     r.hash = mix32(mix32(mix32(A.seed + 0x9e3779b9u) ^ (uint32_t)idx) ^ (uint32_t)(idx >> 32));
     r.w = (uint32_t)w;
-    r.meta = sim_meta(c.pp, S.D.v_eff, S.D.kind, m_sim);
+    r.meta = sim_meta(c.pp, S.D.v_eff, S.D.kind, m_sim, ring);
     r.m = (uint32_t)(S.D.m > (RI)0xFFFFFFFFu ? (RI)0xFFFFFFFFu : S.D.m);
     r.pad[0] = r.pad[1] = r.pad[2] = r.pad[3] = 0u;
     const uint4 *src = reinterpret_cast<const uint4 *>(&r);
@@ -646,6 +703,107 @@ __device__ __forceinline__ void sim_rounds_interleaved(volatile float *tl, const
     clock_out = clock;
     done_out = nF + nB;
 }
+
+// Interleaved on a ring timeline: W = 2 pp microbatch slots per stage stream, slot (j mod W) * Q + stage, two words
+// per slot: a tag (2 j + 1 once the forward of microbatch j has ended, 2 j + 2 once its backward has) and the time.
+// A reader takes a slot only when it carries exactly the tag it waits for, so a slot that was reused too early could
+// only ever make a reader wait for ever -- which the no-progress check reports as a stall -- never hand it a wrong
+// time.  The order's window of pp microbatches divides W, so a window never wraps inside: the ring row of unit
+// (window g, position w) is (g & 1) pp + w, and the cursor steps are those of the full timeline except when an odd
+// window is followed by an even one.
+__device__ __forceinline__ void sim_rounds_interleaved_ring(volatile unsigned long long *tl, const float *durF,
+                                                            const float *durB, int glane, int pp, int v, int U,
+                                                            int warm, int total_ops, float lat, int fonly,
+                                                            float &clock_out, int &done_out, unsigned int *chk,
+                                                            int w_lim, int r_lim, int q_lim)
+{
+    (void)chk; (void)w_lim; (void)r_lim; (void)q_lim;
+    const int Q = pp * v;
+    const bool active = total_ops > 0;
+    const int row = active ? glane : 0;
+    const int Ul = active ? U : 0;
+    int nF = 0, nB = 0, rounds = 0, seen = 0;
+    float clock = 0.f;
+    const int stepF_chunk = pp - (pp - 1) * Q, stepB_chunk = -pp - (pp - 1) * Q;
+    // next window: one ring row up, or from the last row back to the first
+    const int stepF_up = Q - (v - 1) * pp, stepF_wrap = -(2 * pp - 1) * Q - (v - 1) * pp;
+    const int stepB_up = Q + (v - 1) * pp, stepB_wrap = -(2 * pp - 1) * Q + (v - 1) * pp;
+    // slot of the next unit's own entry, its stage, its microbatch, countdowns, and whether its window is an odd one
+    int aF = row, qF = row, jF = 0, fw = pp - 1, fc = v - 1, oddF = 0;
+    int aB = (v - 1) * pp + row, qB = (v - 1) * pp + row, jB = 0, bw = pp - 1, bc = v - 1, oddB = 0;
+#define PF_RING_WORD(tag, t) (((unsigned long long)__float_as_uint(t) << 32) | (unsigned int)(tag))
+#define PF_SIM_FWD(e)                                                                                   \
+    {                                                                                                   \
+        const bool dep = qF > 0;                                                                        \
+        const bool ready = !dep || (unsigned int)(e) == (unsigned int)(2 * jF + 1);                     \
+        const bool go = nF < Ul && nF - nB <= warm && ready;                                            \
+        const float ev = __uint_as_float((unsigned int)((e) >> 32));                                    \
+        const float t = fmaxf(clock, dep ? ev + lat : 0.f) + durF[PF_AT(chk, qF, q_lim, PF_SITE_DURATION)]; \
+        if (go) tl[PF_AT(chk, aF, w_lim, PF_SITE_TIMELINE)] = PF_RING_WORD(2 * jF + 1, t);              \
+        clock = go ? t : clock;                                                                         \
+        const bool ww = fw == 0, wc = fc == 0;                                                          \
+        aF += go ? (ww ? (wc ? (oddF ? stepF_wrap : stepF_up) : stepF_chunk) : Q) : 0;                  \
+        jF += go ? (ww ? (wc ? 1 : -(pp - 1)) : 1) : 0;                                                 \
+        oddF ^= (go && ww && wc) ? 1 : 0;                                                               \
+        qF += (go && ww) ? (wc ? -(v - 1) * pp : pp) : 0;                                               \
+        fc = (go && ww) ? (wc ? v - 1 : fc - 1) : fc;                                                   \
+        fw = go ? (ww ? pp - 1 : fw - 1) : fw;                                                          \
+        nF += go ? 1 : 0;                                                                               \
+    }
+#define PF_SIM_BWD(e)                                                                                   \
+    {                                                                                                   \
+        const bool dep = qB < Q - 1;                                                                    \
+        const bool ready = !dep || (unsigned int)(e) == (unsigned int)(2 * jB + 2);                     \
+        const bool go = nB < Ul && (nF - nB > warm || nF == Ul) && ready;                               \
+        const float ev = __uint_as_float((unsigned int)((e) >> 32));                                    \
+        const float t = fmaxf(clock, dep ? ev + lat : 0.f) + durB[PF_AT(chk, qB, q_lim, PF_SITE_DURATION)]; \
+        if (go) tl[PF_AT(chk, aB, w_lim, PF_SITE_TIMELINE)] = PF_RING_WORD(2 * jB + 2, t);              \
+        clock = go ? t : clock;                                                                         \
+        const bool ww = bw == 0, wc = bc == 0;                                                          \
+        aB += go ? (ww ? (wc ? (oddB ? stepB_wrap : stepB_up) : stepB_chunk) : Q) : 0;                  \
+        jB += go ? (ww ? (wc ? 1 : -(pp - 1)) : 1) : 0;                                                 \
+        oddB ^= (go && ww && wc) ? 1 : 0;                                                               \
+        qB += (go && ww) ? (wc ? (v - 1) * pp : -pp) : 0;                                               \
+        bc = (go && ww) ? (wc ? v - 1 : bc - 1) : bc;                                                   \
+        bw = go ? (ww ? pp - 1 : bw - 1) : bw;                                                          \
+        nB += go ? 1 : 0;                                                                               \
+    }
+    // once a direction has run out of units its cursor rests on some slot of the ring: a valid word, never taken
+#define PF_SIM_POLL_F() tl[PF_AT(chk, aF - (qF > 0 ? 1 : 0), r_lim, PF_SITE_TIMELINE)]
+#define PF_SIM_POLL_B() tl[PF_AT(chk, aB + (qB < Q - 1 ? 1 : 0), r_lim, PF_SITE_TIMELINE)]
+    for (int i = 0; i < fonly; i++) {
+        const unsigned long long eF = PF_SIM_POLL_F();
+        PF_SIM_FWD(eF)
+    }
+    for (;;) {
+#pragma unroll
+        for (int rep = 0; rep < 2; rep++) {
+            const unsigned long long eF = PF_SIM_POLL_F();
+            const unsigned long long eB = PF_SIM_POLL_B();
+            PF_SIM_FWD(eF)
+            PF_SIM_BWD(eB)
+        }
+        PF_SIM_ITER_END(Ul)
+    }
+    while (__any_sync(0xFFFFFFFFu, nB < Ul)) {
+#pragma unroll
+        for (int rep = 0; rep < 4; rep++) {
+            const unsigned long long eB = PF_SIM_POLL_B();
+            PF_SIM_BWD(eB)
+        }
+        if ((++rounds & 15) == 0) {
+            if (!__any_sync(0xFFFFFFFFu, nF + nB != seen)) break;
+            seen = nF + nB;
+        }
+    }
+#undef PF_SIM_FWD
+#undef PF_SIM_BWD
+#undef PF_SIM_POLL_F
+#undef PF_SIM_POLL_B
+#undef PF_RING_WORD
+    clock_out = clock;
+    done_out = nF + nB;
+}
 #undef PF_SIM_ITER_END
 
 // DualPipe-style: two directions; the per-rank order comes from the host-built table
@@ -695,7 +853,7 @@ __device__ __forceinline__ void sim_rounds_dual(volatile float *tl, const float 
 // and the results are stored without waiting.  That matters inside a search call, where this kernel shares the GPU with a
 // saturated store stream under which every round trip to L2 takes microseconds.
 //
-// Inside a warp a candidate is run by a group of 8, 16 or 32 lanes, lane = pipeline rank; a warp takes as many
+// Inside a warp a candidate is run by a group of 4, 8, 16 or 32 lanes, lane = pipeline rank; a warp takes as many
 // candidates per batch as it has groups and its slice has room.  Each lane walks its rank's fixed op order and
 // computes  end(op) = max(rank clock, end(dependency) + latency) + duration.  A forward of stage q needs the
 // forward of stage q-1 of the same microbatch, a backward of stage q the backward of stage q+1 (the op's own
@@ -707,21 +865,26 @@ __device__ __forceinline__ void sim_rounds_dual(volatile float *tl, const float 
 // (and the groups of a warp) stay converged and a round costs one shared-memory poll plus one vote.  Every 64
 // rounds some lane of the warp must have advanced, otherwise its unfinished candidates are reported as
 // PF_SIM_STALL: the loop is bounded by the op count.
+// Two instances: kRings = true can serve ring-timeline bins too and is launched for the large calls that have them;
+// kRings = false is the same kernel without the ring loop (fewer registers, less code), for all other calls.
+template <bool kRings>
 __global__ void __launch_bounds__(kSimThreads, 4) simulate_kernel(const __grid_constant__ DevPlan P, const SimArgs A)
 {
     extern __shared__ __align__(16) float s_mem[];
-    __shared__ unsigned int s_seq[64], s_pre[65], s_off[kSimBins + 1], s_cnt[kSimBins];
+    // (1,016 bytes, and not one more: three blocks of this kernel -- 72 KB of timelines each -- and one block of the fill
+    // kernel fill an SM's shared memory to the last kilobyte)
+    __shared__ unsigned int s_pre[kSimBins + 1], s_off[kSimBins + 1];
+    __shared__ uint8_t s_seq[kSimBins];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int E_hi = sim_class_entries(A.cls_hi);
-    for (int i = threadIdx.x; i < 65; i += kSimThreads) {
-        if (i < 64) s_seq[i] = A.bin_seq[i];
-        s_pre[i] = A.batch_pre[i];
-        if (i <= kSimBins) s_off[i] = A.bin_off[i];
-        if (i < kSimBins) s_cnt[i] = A.bin_count[i];
+    for (int i = threadIdx.x; i <= kSimBins; i += kSimThreads) {
+        if (i < kSimBins) s_seq[i] = (uint8_t)A.bin_seq[i];
+        s_pre[i] = A.batch_pre[i];           // positions past the last bin hold no batches: entry kSimBins = all
+        s_off[i] = A.bin_off[i];
     }
     __syncthreads();
-    float *slice = s_mem + (size_t)warp * A.warp_floats;   // [E_hi] timelines, then 4 x (durF, durB)[q_max]
-    const unsigned int n_batches = s_pre[64];
+    float *slice = s_mem + (size_t)warp * A.warp_floats;   // [E_hi] timelines, then the groups' (durF, durB) tables
+    const unsigned int n_batches = s_pre[kSimBins];
 
     // a batch number -> its bin, its place in the bin, this lane's record
     struct Fetch {
@@ -734,15 +897,18 @@ __global__ void __launch_bounds__(kSimThreads, 4) simulate_kernel(const __grid_c
         f.have = false;
         if (t >= n_batches) return;
         // position in the queue's bin order: how many positions end at or before t
-        const unsigned c0 = __ballot_sync(0xFFFFFFFFu, s_pre[lane + 1] <= t);
-        const unsigned c1 = __ballot_sync(0xFFFFFFFFu, s_pre[lane + 33] <= t);
-        const int pos = __popc(c0) + __popc(c1);
+        int pos = 0;
+#pragma unroll
+        for (int h = 0; h < kSimTab / 32; h++) {
+            const int i = lane + 32 * h;
+            pos += __popc(__ballot_sync(0xFFFFFFFFu, i < kSimBins && s_pre[i + 1] <= t));
+        }
         f.bin = (int)s_seq[pos];
         const int gi = (f.bin / kSimKinds) % kSimGroups;
         const int g = sim_group_lanes(gi), batch = sim_bin_batch(f.bin, A.cls_hi);
         const unsigned int first = (t - s_pre[pos]) * (unsigned int)batch;
         const int gidx = lane / g;
-        f.have = gidx < batch && first + gidx < s_cnt[f.bin];
+        f.have = gidx < batch && first + gidx < s_off[f.bin + 1] - s_off[f.bin];
         if (f.have) {
             const uint4 *src = reinterpret_cast<const uint4 *>(
                 A.recs + PF_AT(P.chk, s_off[f.bin] + first + gidx, s_off[kSimBins], PF_SITE_RECORD));
@@ -769,7 +935,8 @@ __global__ void __launch_bounds__(kSimThreads, 4) simulate_kernel(const __grid_c
         const int gidx = lane / g, glane = lane - gidx * g;
         const bool group_on = gidx < batch;
         volatile float *tl = slice + (size_t)(group_on ? gidx : 0) * E;   // the timeline
-        float *durF = slice + E_hi + (size_t)(group_on ? gidx : 0) * 2 * A.q_max, *durB = durF + A.q_max;
+        const int qg = sim_group_stages(g, A.q_max);           // stages a group's duration tables hold
+        float *durF = slice + E_hi + (size_t)(group_on ? gidx : 0) * 2 * qg, *durB = durF + qg;
         const bool have = cur.have;                            // this group's candidate exists
 
         // ---- the group's candidate, from its record
@@ -782,12 +949,14 @@ __global__ void __launch_bounds__(kSimThreads, 4) simulate_kernel(const __grid_c
         const int pp = run ? (int)(meta & 31u) + 1 : 1, v = run ? (int)((meta >> 5) & 7u) + 1 : 1;
         const int kind = run ? (int)((meta >> 8) & 3u) : PF_KIND_1F1B;
         const int m_sim = run ? (int)((meta >> 10) & 127u) : 1;
+        const bool ring = run && ((meta >> 17) & 1u) != 0u;   // interleaved, on a ring timeline
         const bool dual = kind == PF_KIND_DUALPIPE;
         const int Q = dual ? pp : pp * v;
         const int nj = dual ? m_sim / 2 : m_sim;      // microbatches per stage stream
-        const int n_entries = (dual ? 2 * Q : Q) * nj;
+        const int n_entries = ring ? Q * sim_ring_slots(pp) * 2 : (dual ? 2 * Q : Q) * nj;   // timeline words
         // filed under a bin that cannot hold it: never happens for the pre-pass's records; reported, not overrun
-        bool stalled = run && (n_entries > E || Q > A.q_max || pp > g || kind != bin_kind);
+        bool stalled = run && (n_entries > E || Q > qg || pp > g || (ring ? kSimKindRing : kind) != bin_kind ||
+                              (ring && !kRings));
         if (stalled) run = false;
 
         // ---- stage durations (balanced layer split, head on the last stage, jitter), cleared timeline
@@ -800,7 +969,7 @@ __global__ void __launch_bounds__(kSimThreads, 4) simulate_kernel(const __grid_c
                 const int ndq = max(0, min(nq_i, P.L_dense - start));    // its leading dense layers
                 const float nq = (float)(nq_i - ndq), nd = (float)ndq;
                 const bool last = q == Q - 1;
-                const int qd = (int)PF_AT(P.chk, q, A.q_max, PF_SITE_DURATION);
+                const int qd = (int)PF_AT(P.chk, q, qg, PF_SITE_DURATION);
                 durF[qd] = (nq * F_l + nd * F_ld + (last ? headF : 0.f)) * jitter(cand_hash, q, 0);
                 durB[qd] = (nq * B_l + nd * B_ld + (last ? P.bwd_factor * headF : 0.f)) * jitter(cand_hash, q, 1);
             }
@@ -837,13 +1006,17 @@ __global__ void __launch_bounds__(kSimThreads, 4) simulate_kernel(const __grid_c
         int fonly = (run && !dual) ? Q - 1 : 0x7FFFFFFF;
         fonly = __reduce_min_sync(0xFFFFFFFFu, fonly);
         if (fonly == 0x7FFFFFFF) fonly = 0;
-        if (bin_kind == PF_KIND_1F1B)
+        if (kRings && bin_kind == kSimKindRing)
+            // (two-word slots: the limits count slots)
+            sim_rounds_interleaved_ring(reinterpret_cast<volatile unsigned long long *>(tl), durF, durB, glane, pp, v, U,
+                                        warm, total_ops, lat, fonly, clock, done, P.chk, w_lim >> 1, r_lim >> 1, qg);
+        else if (bin_kind == PF_KIND_1F1B)
             sim_rounds_1f1b(tl, durF, durB, glane, pp, nj, warm, total_ops, lat, fonly, clock, done, P.chk, w_lim, r_lim);
         else if (bin_kind == PF_KIND_INTERLEAVED)
             sim_rounds_interleaved(tl, durF, durB, glane, pp, v, nj, U, warm, total_ops, lat, fonly, clock, done, P.chk,
-                                   w_lim, r_lim, A.q_max);
+                                   w_lim, r_lim, qg);
         else
-            sim_rounds_dual(tl, durF, durB, glane, pp, nj, dops, total_ops, lat, clock, done, P.chk, w_lim, r_lim, A.q_max);
+            sim_rounds_dual(tl, durF, durB, glane, pp, nj, dops, total_ops, lat, clock, done, P.chk, w_lim, r_lim, qg);
         if (done < total_ops) stalled = true;
 
         // the next batch's records are requested before this batch's results are reduced and stored
@@ -975,7 +1148,8 @@ struct SimLayout {
     size_t off_ctrl, off_bin_of, off_recs, off_scores, off_topk, total;
     DenseTopkLayout dt;
 };
-constexpr size_t kSimCtrlBytes = 4096;   // work, bin_count, bin_off, bin_fill, bin_seq, batch_pre
+constexpr size_t kSimCtrlBytes = 4096;   // work (64 words), bin_count, bin_off, bin_fill, bin_seq (kSimTab each), batch_pre
+static_assert((64 + 5 * kSimTab + 1) * 4 <= 4096, "simulator control block");
 
 static SimLayout sim_layout(const pf_plan_t *p, uint64_t n, uint32_t k)
 {
@@ -1021,7 +1195,13 @@ static SimGeom sim_geom(int q_max)
     const int entries_max = q_max * PF_SIM_WINDOW;
     g.cls_hi = 0;
     while (g.cls_hi < kSimClasses - 1 && sim_class_entries(g.cls_hi) < entries_max) g.cls_hi++;
-    g.warp_floats = sim_class_entries(g.cls_hi) + 4 * 2 * q_max;
+    // a warp's slice: one timeline of the largest class, then the duration tables of as many lane groups as a warp holds
+    int dur_floats = 0;
+    for (int gi = 0; gi < kSimGroups; gi++) {
+        const int lanes = sim_group_lanes(gi), need = (32 / lanes) * 2 * sim_group_stages(lanes, q_max);
+        dur_floats = need > dur_floats ? need : dur_floats;
+    }
+    g.warp_floats = sim_class_entries(g.cls_hi) + ((dur_floats + 3) & ~3);
     g.pool = (size_t)(kSimThreads / 32) * g.warp_floats * sizeof(float);
     g.per_sm = (int)((size_t)(227 * 1024) / (g.pool + 1024 + 1280));
     g.per_sm = g.per_sm < 1 ? 1 : (g.per_sm > 12 ? 12 : g.per_sm);
@@ -1048,10 +1228,12 @@ static int launch_simulate(pf_plan_t *p, SimArgs a, uint64_t n, cudaStream_t st,
     const uint64_t want = (n + kSimThreads / 32 - 1) / (kSimThreads / 32);
     const int grid = (int)(want < cap ? want : cap);
     const int threads = kSimThreads;
-    PF_CUDA_TRY(cudaFuncSetAttribute(simulate_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)geo.pool),
+    // (the pre-pass puts survivors on ring timelines in calls of at least kSimRingMinSurvivors only)
+    const auto kernel = n >= kSimRingMinSurvivors ? simulate_kernel<true> : simulate_kernel<false>;
+    PF_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)geo.pool),
                 "simulate_kernel smem");
     timing_begin(p, PF_T_SIMULATE, st);
-    simulate_kernel<<<grid, threads, geo.pool, st>>>(p->dev, a);
+    kernel<<<grid, threads, geo.pool, st>>>(p->dev, a);
     count_launch();
     timing_end(p, PF_T_SIMULATE, 1, st);
     *n_kernels = 4;
@@ -1108,10 +1290,10 @@ int pf::simulate_run(pf_plan_t *p, const uint64_t *d_surv_idx, uint64_t n, const
     a.tput_sim = scores; a.status = d_sim_status;
     a.work = (unsigned int *)(ws + lay.off_ctrl);
     a.bin_count = a.work + 64;
-    a.bin_off = a.bin_count + 64;
-    a.bin_fill = a.bin_off + 64;
-    a.bin_seq = a.bin_fill + 64;
-    a.batch_pre = a.bin_seq + 64;
+    a.bin_off = a.bin_count + kSimTab;
+    a.bin_fill = a.bin_off + kSimTab;
+    a.bin_seq = a.bin_fill + kSimTab;
+    a.batch_pre = a.bin_seq + kSimTab;       // kSimTab + 1 words
     a.bin_of = ws + lay.off_bin_of;
     a.recs = (SimRec *)(ws + lay.off_recs);
     a.vals = p->d_vals; a.dual_ops = tab->d_ops; a.dual_off = tab->d_offset;

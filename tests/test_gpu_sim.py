@@ -168,6 +168,42 @@ def test_simulate_deep_pipelines_and_long_windows():
     assert np.all(status == 0)
 
 
+def test_simulate_every_interleaved_shape_of_the_large_space():
+    """Interleaved schedules keep their timelines on a ring of 2 pp microbatch slots per stage where that is smaller;
+    a ring that were too short for some shape would leave its readers waiting (status STALL).  Every interleaved
+    shape the large space offers -- pp 1..32, 1..8 virtual stages, every microbatch size, short and long windows --
+    must finish and agree with the oracle.  (The list is repeated so that the call is large enough for the rings to
+    be used: small calls keep full timelines, which are faster per simulated op.)"""
+    cfg = variant("large_unconstrained", cluster=dict(budget_bytes=10 ** 15))
+    for kn in cfg["kern"]:
+        kn["avail_mask"] = 255
+    orc = Oracle(cfg)
+    axes = dict(cfg["axes"])
+    picks = []
+    for v in axes["v"]:
+        for pp in (1, 2, 4, 8, 16, 32):
+            for mb in axes["mb"]:
+                for dp in (8, 32, 256):
+                    i = axis_index(cfg, kv=1, rec=0, sched=2, mb=mb, v=v, ep=8, pp=pp, tp=2, dp=dp)
+                    if orc.eval(i)["reason"] & 0x7F == 0:
+                        picks.append(i)
+    idx = np.unique(np.array(picks, dtype=np.uint64))
+    ds = [orc.eval(int(i)) for i in idx]
+    assert len(idx) > 300 and {d["kind"] for d in ds} == {1}
+    assert {d["v_eff"] for d in ds} == set(range(2, 9)) and {d["pp"] for d in ds} == {2, 4, 8, 16}
+    assert any(d["m"] >= 64 and d["pp"] * 2 < 64 for d in ds)          # rings that wrap
+    assert any(d["m"] <= 2 * d["pp"] for d in ds)                      # and windows too short to need one
+    _, status = _sim_parity(cfg, idx, k=64)                            # a small call: full timelines
+    assert np.all(status == 0)
+    big = np.tile(idx, 80)                                             # 40,320 entries: ring timelines
+    plan = _plan(cfg)
+    tput_big, status_big, _, _ = _simulate(plan, big, 4, 16)
+    plan.close()
+    want, want_st, _ = orc.simulate_list(idx, 4, threads=16)
+    assert np.all(status_big == 0)
+    np.testing.assert_allclose(tput_big, np.tile(want, 80), rtol=TPUT_RTOL, atol=0)
+
+
 def test_simulate_infeasible_and_out_of_domain_entries():
     cfg = variant("large_unconstrained", cluster=dict(budget_bytes=10 ** 15))
     cfg["model"]["L"] = 128
