@@ -3,6 +3,7 @@
 #pragma once
 
 #include <cuda_runtime.h>
+#include <utility>
 #include <stdint.h>
 
 #include "planfront.h"
@@ -178,6 +179,36 @@ void timing_end(pf_plan_t *p, int cls, int n_kernels, cudaStream_t st);
             return PF_ECUDA;                            \
         }                                               \
     } while (0)
+
+// ------------------------------------------------------------------ chained launches
+// The small kernels of a call form a chain on one stream, each reading what the one before wrote.  A plain launch
+// starts only after the kernel before it has completed and its launch has then been processed: a few microseconds
+// per link.  A chained launch (programmatic stream serialization) lets the GPU schedule the grid as soon as every
+// block of the kernel before it has passed chain_enter() or left, so that the launch itself overlaps that kernel;
+// the new grid's blocks then wait in chain_enter() until that kernel has completed and its writes are visible.
+// Rule for a kernel launched this way, and for the kernel in front of it: chain_enter() is its first statement
+// (nothing before it touches global memory).  In a kernel launched the plain way chain_enter() does nothing.
+__device__ __forceinline__ void chain_enter()
+{
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                  Args &&...args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(std::forward<Args>(args))...);
+}
 
 // ------------------------------------------------------------------ keys
 // A ranked candidate is one 64-bit key: (fp32 score bits << 32) | (0xFFFFFFFF - rel), rel = position in
@@ -442,10 +473,11 @@ inline TopkLayout topk_layout(uint64_t n_keys_max, uint32_t k)
 
 // host: reduce a compact key list (device count in ctrl[1], at most n_keys_max keys) to the final outputs.
 // idx_map (device, may be NULL): final index = idx_map[rel] instead of first + rel.
-// Returns the number of kernels launched through *n_kernels.
+// Returns the number of kernels launched through *n_kernels.  chained: the kernel that wrote the list is the operation
+// right before this call on the same stream (the first launch here is then a chained one).
 int launch_topk_reduce(void *d_workspace, const TopkLayout &lay, uint64_t n_keys_max, uint32_t k, uint64_t first,
                        const uint64_t *d_idx_map, uint64_t *d_topk_idx, float *d_topk_score, uint32_t *d_topk_count,
-                       cudaStream_t st, int *n_kernels);
+                       cudaStream_t st, int *n_kernels, bool chained = false);
 
 // host: top-k of a dense score array (entries with score <= 0 are skipped; ties go to the lower position).
 // The workspace is laid out by dense_topk_layout; idx_map as in launch_topk_reduce.
@@ -457,6 +489,8 @@ struct DenseTopkLayout {
 DenseTopkLayout dense_topk_layout(int sm_count, uint64_t n, uint32_t k);
 int launch_dense_topk(const float *d_score, uint64_t n, const uint64_t *d_n, uint32_t k, const uint64_t *d_idx_map,
                       void *d_workspace, const DenseTopkLayout &lay, uint64_t *d_topk_idx, float *d_topk_score,
-                      uint32_t *d_topk_count, cudaStream_t st, int *n_kernels);
+                      uint32_t *d_topk_count, cudaStream_t st, int *n_kernels, bool ctrl_cleared = false);
+// (ctrl_cleared: the caller has zeroed the first 256 bytes of the layout's control block earlier on the stream, so
+// that no memset stands between the kernel that wrote the scores and this one's first, chained, launch)
 
 }  // namespace pf

@@ -228,6 +228,7 @@ __device__ __noinline__ CostOut train_cost(const DevPlan &P, const TrainTuple c)
 template <typename RI>
 __global__ void __launch_bounds__(kThreads, 4) score_kernel(const __grid_constant__ DevPlan P, const ScoreArgs A)
 {
+    chain_enter();
     __shared__ unsigned long long s_buf[kTopkCap];
     __shared__ int s_count;
     __shared__ unsigned long long s_thr;
@@ -820,6 +821,7 @@ struct ReduceArgs {
 // really overflow.  A shorter list is left to the final kernel as it is.
 __global__ void __launch_bounds__(kReduceThreads) reduce_kernel(const ReduceArgs A)
 {
+    chain_enter();
     __shared__ unsigned long long s_buf[kTopkCap];
     __shared__ int s_count;
     __shared__ unsigned long long s_thr;
@@ -858,6 +860,7 @@ __global__ void __launch_bounds__(kReduceThreads) reduce_kernel(const ReduceArgs
 // prune-on-overflow.
 __global__ void __launch_bounds__(kReduceThreads) reduce_final_kernel(const ReduceArgs A)
 {
+    chain_enter();
     extern __shared__ __align__(16) unsigned long long s_big[];  // kFastKeys keys, then kTopkCap keys to sort in
     __shared__ int s_count;
     __shared__ unsigned long long s_thr;
@@ -985,7 +988,7 @@ __global__ void __launch_bounds__(kReduceThreads) reduce_final_kernel(const Redu
 
 int launch_topk_reduce(void *d_workspace, const TopkLayout &lay, uint64_t n_keys_max, uint32_t k, uint64_t first,
                        const uint64_t *d_idx_map, uint64_t *d_topk_idx, float *d_topk_score, uint32_t *d_topk_count,
-                       cudaStream_t st, int *n_kernels)
+                       cudaStream_t st, int *n_kernels, bool chained)
 {
     uint8_t *ws = (uint8_t *)d_workspace;
     unsigned int *ctrl = (unsigned int *)(ws + lay.off_ctrl);
@@ -1002,7 +1005,11 @@ int launch_topk_reduce(void *d_workspace, const TopkLayout &lay, uint64_t n_keys
     uint64_t blocks = (uint64_t)kFastKeys / (k ? k : 1);
     blocks = blocks < 1 ? 1 : (blocks > 256 ? 256 : blocks);
     if (n_keys_max > (uint64_t)kFastKeys) {
-        reduce_kernel<<<(unsigned int)blocks, kReduceThreads, 0, st>>>(r);
+        if (chained)
+            launch_chained(reduce_kernel, (unsigned int)blocks, kReduceThreads, 0, st, r);
+        else
+            reduce_kernel<<<(unsigned int)blocks, kReduceThreads, 0, st>>>(r);
+        chained = true;   // the next launch follows this kernel
         count_launch();
         (*n_kernels)++;
         PF_CUDA_TRY(cudaGetLastError(), "reduce_kernel launch");
@@ -1010,7 +1017,10 @@ int launch_topk_reduce(void *d_workspace, const TopkLayout &lay, uint64_t n_keys
     r.in = out; r.in_count = ctrl + 2; r.final = 1;
     PF_CUDA_TRY(cudaFuncSetAttribute(reduce_final_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      (kFastKeys + kTopkCap) * 8), "reduce_final_kernel smem");
-    reduce_final_kernel<<<1, kReduceThreads, (kFastKeys + kTopkCap) * 8, st>>>(r);
+    if (chained)
+        launch_chained(reduce_final_kernel, 1, kReduceThreads, (kFastKeys + kTopkCap) * 8, st, r);
+    else
+        reduce_final_kernel<<<1, kReduceThreads, (kFastKeys + kTopkCap) * 8, st>>>(r);
     count_launch();
     (*n_kernels)++;
     PF_CUDA_TRY(cudaGetLastError(), "reduce_final_kernel launch");
@@ -1273,8 +1283,9 @@ int pf::score_run(pf_plan_t *p, uint64_t first, uint64_t count, uint8_t *d_reaso
         }
         timing_begin(p, PF_T_TOPK, rs);
         int nk = 0;
+        // (on the caller's stream the scoring kernel is the operation right before: a chained launch)
         const int rc2 = launch_topk_reduce(ws, lay, (uint64_t)grid * k, k, first, nullptr, d_topk_idx, d_topk_score,
-                                           d_topk_count, rs, &nk);
+                                           d_topk_count, rs, &nk, rs == st && !split);
         timing_end(p, PF_T_TOPK, nk, rs);
         if (rs != st && cudaEventRecord(p->ev_join, rs) == cudaSuccess) sp.join_pending = true;
         if (rc == PF_OK) rc = rc2;

@@ -184,6 +184,7 @@ __device__ __forceinline__ void sel_hist_chunk(const DevPlan &P, const SelArgs &
 __global__ void __launch_bounds__(kSelThreads) sel_hist_kernel(const __grid_constant__ DevPlan P, const SelArgs A,
                                                                 const int32_t *vals, int pass)
 {
+    chain_enter();
     __shared__ unsigned int s_elig;
     if (pass == 0) {   // one block per chunk: the whole array is read, the more loads in flight the better
         sel_hist_chunk(P, A, vals, 0, blockIdx.x, &s_elig);
@@ -243,6 +244,7 @@ __device__ __forceinline__ unsigned long long block_prefix_256(unsigned long lon
 
 __global__ void __launch_bounds__(256) sel_scan_kernel(const SelArgs A, int pass)
 {
+    chain_enter();
     __shared__ unsigned long long s_warp[8];
     __shared__ unsigned long long s_total, s_above;
     __shared__ int s_group;
@@ -301,6 +303,7 @@ __global__ void __launch_bounds__(256) sel_scan_kernel(const SelArgs A, int pass
 __global__ void __launch_bounds__(kSelThreads) sel_count_kernel(const __grid_constant__ DevPlan P, const SelArgs A,
                                                                  const int32_t *vals)
 {
+    chain_enter();
     __shared__ unsigned int s_gt, s_eq;
     const unsigned int n_list = A.ctrl->n_elig;
     const bool all = A.ctrl->take_all != 0;
@@ -348,6 +351,7 @@ __global__ void __launch_bounds__(kSelThreads) sel_count_kernel(const __grid_con
 constexpr int kScanTiles = 16;
 __global__ void __launch_bounds__(1024) sel_blockscan_kernel(const SelArgs A, int nblocks)
 {
+    chain_enter();
     __shared__ unsigned long long s_warp[32];
     __shared__ unsigned long long s_tot[kScanTiles][33];   // warp totals per tile, then their exclusive prefixes
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -501,6 +505,7 @@ __device__ __forceinline__ void sel_write_chunk(const DevPlan &P, const SelArgs 
 __global__ void __launch_bounds__(kSelThreads) sel_write_kernel(const __grid_constant__ DevPlan P, const SelArgs A,
                                                                  const int32_t *vals)
 {
+    chain_enter();
     __shared__ unsigned int s_gt[kSelThreads / 32];   // warp totals of a tile's scan
     __shared__ unsigned long long s_run_gt, s_run_eq;
     const unsigned int n_list = A.ctrl->n_elig;
@@ -617,11 +622,11 @@ int pf::select_run(pf_plan_t *p, uint64_t first, uint64_t count, const uint8_t *
         launches++;
     }
     sel_scan_kernel<<<1, 256, 0, st>>>(a, 0);
-    sel_hist_kernel<<<list_grid, kSelThreads, 0, st>>>(p->dev, a, p->d_vals, 1);
-    sel_scan_kernel<<<1, 256, 0, st>>>(a, 1);
-    sel_count_kernel<<<list_grid, kSelThreads, 0, st>>>(p->dev, a, p->d_vals);
-    sel_blockscan_kernel<<<1, 1024, 0, st>>>(a, lay.nblocks);
-    sel_write_kernel<<<list_grid, kSelThreads, 0, st>>>(p->dev, a, p->d_vals);
+    launch_chained(sel_hist_kernel, list_grid, kSelThreads, 0, st, p->dev, a, p->d_vals, 1);
+    launch_chained(sel_scan_kernel, 1, 256, 0, st, a, 1);
+    launch_chained(sel_count_kernel, list_grid, kSelThreads, 0, st, p->dev, a, p->d_vals);
+    launch_chained(sel_blockscan_kernel, 1, 1024, 0, st, a, lay.nblocks);
+    launch_chained(sel_write_kernel, list_grid, kSelThreads, 0, st, p->dev, a, p->d_vals);
     timing_end(p, PF_T_SELECT, launches, st);
     for (int i = 0; i < launches; i++) count_launch();
     PF_CUDA_TRY(cudaGetLastError(), "pf_select_survivors launch");

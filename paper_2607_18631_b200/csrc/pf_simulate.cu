@@ -331,6 +331,7 @@ __device__ __forceinline__ int sim_entries(int kind, int pp, int streams, int m_
 template <typename RI>
 __global__ void __launch_bounds__(256) sim_classify_kernel(const __grid_constant__ DevPlan P, const SimArgs A)
 {
+    chain_enter();
     uint64_t n = A.n;
     if (A.d_n) {
         uint64_t dn = *A.d_n;
@@ -392,6 +393,7 @@ __device__ __forceinline__ unsigned int warp_incl_scan(unsigned int x, int lane)
 }
 __global__ void __launch_bounds__(32) sim_offsets_kernel(const SimArgs A)
 {
+    chain_enter();
     constexpr int kQ = kSimTab / 32;   // table entries per lane: lane l owns entries l, l + 32, ...
     const int lane = threadIdx.x;
     unsigned int cnt[kQ], incl[kQ];
@@ -448,6 +450,7 @@ __global__ void __launch_bounds__(32) sim_offsets_kernel(const SimArgs A)
 template <typename RI>
 __global__ void __launch_bounds__(256) sim_records_kernel(const __grid_constant__ DevPlan P, const SimArgs A)
 {
+    chain_enter();
     uint64_t n = A.n;
     if (A.d_n) {
         uint64_t dn = *A.d_n;
@@ -870,6 +873,7 @@ __device__ __forceinline__ void sim_rounds_dual(volatile float *tl, const float 
 template <bool kRings>
 __global__ void __launch_bounds__(kSimThreads, 4) simulate_kernel(const __grid_constant__ DevPlan P, const SimArgs A)
 {
+    chain_enter();
     extern __shared__ __align__(16) float s_mem[];
     // (1,016 bytes, and not one more: three blocks of this kernel -- 72 KB of timelines each -- and one block of the fill
     // kernel fill an SM's shared memory to the last kilobyte)
@@ -929,7 +933,9 @@ __global__ void __launch_bounds__(kSimThreads, 4) simulate_kernel(const __grid_c
         const int bin = cur.bin;
         const int cls = bin / (kSimGroups * kSimKinds), gi = (bin / kSimKinds) % kSimGroups;
         const int bin_kind = bin % kSimKinds;
-        const int g = sim_group_lanes(gi);
+        // (four-lane groups exist in the calls that have ring timelines only: the other instance is compiled for
+        // groups of eight lanes and more, and reports a narrower bin -- there is none -- as stalled)
+        const int g = kRings ? sim_group_lanes(gi) : max(sim_group_lanes(gi), 8);
         const int E = sim_class_entries(cls);
         const int batch = sim_bin_batch(bin, A.cls_hi);       // candidates this warp runs side by side
         const int gidx = lane / g, glane = lane - gidx * g;
@@ -956,7 +962,7 @@ __global__ void __launch_bounds__(kSimThreads, 4) simulate_kernel(const __grid_c
         const int n_entries = ring ? Q * sim_ring_slots(pp) * 2 : (dual ? 2 * Q : Q) * nj;   // timeline words
         // filed under a bin that cannot hold it: never happens for the pre-pass's records; reported, not overrun
         bool stalled = run && (n_entries > E || Q > qg || pp > g || (ring ? kSimKindRing : kind) != bin_kind ||
-                              (ring && !kRings));
+                              (!kRings && (ring || gi == 0)));
         if (stalled) run = false;
 
         // ---- stage durations (balanced layer split, head on the last stage, jitter), cleared timeline
@@ -977,6 +983,7 @@ __global__ void __launch_bounds__(kSimThreads, 4) simulate_kernel(const __grid_c
             {
                 float4 *tl4 = reinterpret_cast<float4 *>(const_cast<float *>(tl));
                 const int n4 = (n_entries + 3) >> 2;
+#pragma unroll 4
                 for (int i = glane; i < n4; i += g) tl4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
             }
         }
@@ -1077,6 +1084,7 @@ struct DenseTopkArgs {
 
 __global__ void __launch_bounds__(kThreads) dense_topk_kernel(const DenseTopkArgs A)
 {
+    chain_enter();
     __shared__ unsigned long long s_buf[kTopkCap];
     __shared__ int s_count;
     __shared__ unsigned long long s_thr;
@@ -1126,20 +1134,23 @@ DenseTopkLayout dense_topk_layout(int sm_count, uint64_t n, uint32_t k)
 
 int launch_dense_topk(const float *d_score, uint64_t n, const uint64_t *d_n, uint32_t k, const uint64_t *d_idx_map,
                       void *d_workspace, const DenseTopkLayout &lay, uint64_t *d_topk_idx, float *d_topk_score,
-                      uint32_t *d_topk_count, cudaStream_t st, int *n_kernels)
+                      uint32_t *d_topk_count, cudaStream_t st, int *n_kernels, bool ctrl_cleared)
 {
     uint8_t *tws = (uint8_t *)d_workspace;
-    PF_CUDA_TRY(cudaMemsetAsync(tws + lay.tk.off_ctrl, 0, 256, st), "dense top-k: counter reset");
+    if (!ctrl_cleared) PF_CUDA_TRY(cudaMemsetAsync(tws + lay.tk.off_ctrl, 0, 256, st), "dense top-k: counter reset");
     DenseTopkArgs t;
     t.score = d_score; t.n = n; t.d_n = d_n; t.k = k;
     t.keys = (unsigned long long *)(tws + lay.tk.off_keys_a);
     t.key_count = (unsigned int *)(tws + lay.tk.off_ctrl) + 1;
-    dense_topk_kernel<<<lay.blocks, kThreads, 0, st>>>(t);
+    if (ctrl_cleared)
+        launch_chained(dense_topk_kernel, lay.blocks, kThreads, 0, st, t);
+    else
+        dense_topk_kernel<<<lay.blocks, kThreads, 0, st>>>(t);
     count_launch();
     PF_CUDA_TRY(cudaGetLastError(), "dense_topk_kernel launch");
     int nk = 0;
     int rc = launch_topk_reduce(tws, lay.tk, lay.keys_max, k, 0, d_idx_map, d_topk_idx, d_topk_score, d_topk_count,
-                                st, &nk);
+                                st, &nk, true);
     *n_kernels = nk + 1;
     return rc;
 }
@@ -1219,8 +1230,8 @@ static int launch_simulate(pf_plan_t *p, SimArgs a, uint64_t n, cudaStream_t st,
     const unsigned int nb = (unsigned int)((n + 255) / 256);
     timing_begin(p, PF_T_SIMPREP, st);
     sim_classify_kernel<RI><<<nb, 256, 0, st>>>(p->dev, a);
-    sim_offsets_kernel<<<1, 32, 0, st>>>(a);
-    sim_records_kernel<RI><<<nb, 256, 0, st>>>(p->dev, a);
+    launch_chained(sim_offsets_kernel, 1, 32, 0, st, a);
+    launch_chained(sim_records_kernel<RI>, nb, 256, 0, st, p->dev, a);
     for (int i = 0; i < 3; i++) count_launch();
     timing_end(p, PF_T_SIMPREP, 3, st);
     PF_CUDA_TRY(cudaGetLastError(), "simulator pre-pass launch");
@@ -1233,7 +1244,7 @@ static int launch_simulate(pf_plan_t *p, SimArgs a, uint64_t n, cudaStream_t st,
     PF_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)geo.pool),
                 "simulate_kernel smem");
     timing_begin(p, PF_T_SIMULATE, st);
-    kernel<<<grid, threads, geo.pool, st>>>(p->dev, a);
+    launch_chained(kernel, grid, threads, geo.pool, st, p->dev, a);
     count_launch();
     timing_end(p, PF_T_SIMULATE, 1, st);
     *n_kernels = 4;
@@ -1301,6 +1312,9 @@ int pf::simulate_run(pf_plan_t *p, const uint64_t *d_surv_idx, uint64_t n, const
     a.cls_hi = 0;
     a.warp_floats = 0;
     PF_CUDA_TRY(cudaMemsetAsync(ws + lay.off_ctrl, 0, kSimCtrlBytes, st), "pf_simulate: counter reset");
+    // the re-ranking's counters too, here rather than in front of its kernel: nothing but kernels from here to the end,
+    // each launch chained to the one before
+    if (k > 0) PF_CUDA_TRY(cudaMemsetAsync(ws + lay.off_topk + lay.dt.tk.off_ctrl, 0, 256, st), "dense top-k: counter reset");
     if (n > 0) {
         int nk = 0;
         rc = p->dev.wide ? launch_simulate<unsigned long long>(p, a, n, st, &nk)
@@ -1313,7 +1327,7 @@ int pf::simulate_run(pf_plan_t *p, const uint64_t *d_surv_idx, uint64_t n, const
         int nk = 0;
         timing_begin(p, PF_T_TOPK, st);
         rc = launch_dense_topk(scores, n, d_n, k, d_surv_idx, ws + lay.off_topk, lay.dt, d_topk_idx, d_topk_score,
-                               d_topk_count, st, &nk);
+                               d_topk_count, st, &nk, true);
         timing_end(p, PF_T_TOPK, nk, st);
         return rc;
     }
