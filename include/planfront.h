@@ -424,7 +424,12 @@ int pf_compact(pf_plan_t *plan, uint64_t first, uint64_t count, const uint8_t *d
  * besides the two top-k lists -- on the 1.8e8-candidate space about 23 MB instead of 2.3 GB.
  * d_workspace: pf_search_compact_workspace() bytes of DEVICE memory.  Returns after all copies have completed
  * (the view is taken, and its copies start, as soon as the candidates are scored, beside the selection and the
- * simulator; host buffers should be pinned for the copies to overlap).  Errors as pf_search_host. */
+ * simulator).  Every host pointer may be pageable or page-locked memory.  The small results (histogram, count, top-k
+ * lists) pass through a page-locked block of the library's own.  h_mask and h_records are written directly: into
+ * page-locked memory beside the search, into pageable memory at its end.  A page-locked h_mask is moreover filled
+ * in two parts -- a copy of zeros to the whole of it that starts with the call, and, once the candidates are
+ * scored, device writes of the few 2 KB stretches that hold a feasible plan -- so its N / 8 bytes cross the host
+ * link beside the search instead of behind it.  Errors as pf_search_host. */
 size_t pf_search_compact_workspace(const pf_plan_t *plan, uint32_t k, uint64_t s_max, uint32_t k_sim,
                                    uint64_t record_cap);
 int pf_search_host_compact(pf_plan_t *plan, uint32_t k, uint64_t s_max, uint32_t k_sim, uint32_t jitter_seed,

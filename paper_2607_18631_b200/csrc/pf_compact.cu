@@ -279,6 +279,35 @@ __global__ void __launch_bounds__(kCmpThreads) compact_write_kernel(const Compac
     }
 }
 
+// The feasibility bits of the chunks that hold a feasible plan, written to `mask` -- which may be page-locked HOST
+// memory mapped into the device's address space: every other chunk's bits are zero and reach the host as one early
+// copy of zeros instead of crossing the bus behind the search.  Runs after compact_count_kernel (chunk counts).
+__global__ void __launch_bounds__(kCmpThreads) compact_mask_kernel(const CompactArgs A)
+{
+    const int tid = threadIdx.x;
+    const uint8_t *cls = cmp_guard_cls(A);
+    for (unsigned int chunk = blockIdx.x; chunk < A.n_chunks; chunk += gridDim.x) {
+        if (A.chunk_count[chunk] == 0u) continue;   // uniform across the block
+        const uint64_t lo = (uint64_t)chunk * kCmpChunk;
+#pragma unroll
+        for (int t = 0; t < kCmpTiles; t++) {
+            const uint64_t e = lo + (uint64_t)t * kCmpTile + (uint64_t)tid * 16;
+            const uint32_t m = e < A.count ? cmp_feasible16(cmp_reason16(A, cls, e)) : 0u;
+            // two neighbours share one 32-bit store (e / 8 is a multiple of 4 in even threads); a pair that reaches
+            // past the end of the range stores its bytes one by one
+            const uint32_t up = __shfl_down_sync(0xFFFFFFFFu, m, 1);
+            const uint64_t e_pair = e - (uint64_t)(tid & 1) * 16;
+            if (e_pair + 32 <= A.count) {
+                if ((tid & 1) == 0) *reinterpret_cast<uint32_t *>(A.mask + (e >> 3)) = m | (up << 16);
+            } else if (e < A.count) {
+                uint8_t *dst = A.mask + (e >> 3);
+                dst[0] = (uint8_t)(m & 0xFFu);
+                if (e + 8 < A.count) dst[1] = (uint8_t)(m >> 8);
+            }
+        }
+    }
+}
+
 struct CompactLayout {
     size_t off_count, off_pre, total;
     unsigned int n_chunks;
@@ -323,6 +352,26 @@ int compact_run(pf_plan_t *p, uint64_t first, uint64_t count, const uint8_t *d_r
     timing_end(p, PF_T_COMPACT, launches, st);
     for (int i = 0; i < launches; i++) count_launch();
     PF_CUDA_TRY(cudaGetLastError(), "pf_compact launch");
+    return PF_OK;
+}
+
+// The bits of the chunks with feasible plans, after compact_run on the same stream and workspace (see
+// compact_mask_kernel); `mask` is a device-visible address.
+int compact_mask_run(pf_plan_t *p, uint64_t first, uint64_t count, const uint8_t *d_reason, uint8_t *mask,
+                     void *d_workspace, cudaStream_t st, const FillGuard *guard)
+{
+    const CompactLayout lay = compact_layout(count);
+    uint8_t *ws = (uint8_t *)d_workspace;
+    CompactArgs a = {};
+    a.first = first; a.count = count; a.reason = d_reason; a.mask = mask;
+    a.chunk_count = (unsigned int *)(ws + lay.off_count);
+    a.chunk_pre = (unsigned long long *)(ws + lay.off_pre);
+    a.n_chunks = lay.n_chunks;
+    if (guard) a.guard = *guard;
+    const unsigned int grid = lay.n_chunks < (unsigned int)p->sm_count * 8 ? lay.n_chunks : (unsigned int)p->sm_count * 8;
+    compact_mask_kernel<<<grid, kCmpThreads, 0, st>>>(a);
+    count_launch();
+    PF_CUDA_TRY(cudaGetLastError(), "compact_mask_kernel launch");
     return PF_OK;
 }
 

@@ -428,6 +428,10 @@ struct ScoreSpread {
 int compact_run(pf_plan_t *p, uint64_t first, uint64_t count, const uint8_t *d_reason, const float *d_tput,
                 const int64_t *d_mem, uint64_t *d_hist, uint8_t *d_mask, pf_record_t *d_records, uint64_t record_cap,
                 uint64_t *d_n_feasible, void *d_workspace, cudaStream_t st, const FillGuard *guard);
+// after compact_run on the same stream and workspace: the feasibility bits of the chunks that hold a feasible plan
+// only, to a device-visible address (mapped host memory included); the rest of the mask is zero and not written
+int compact_mask_run(pf_plan_t *p, uint64_t first, uint64_t count, const uint8_t *d_reason, uint8_t *mask,
+                     void *d_workspace, cudaStream_t st, const FillGuard *guard);
 int simulate_run(pf_plan_t *p, const uint64_t *d_surv_idx, uint64_t n, const uint64_t *d_n, uint32_t jitter_seed,
                  float *d_tput_sim, uint8_t *d_sim_status, uint32_t k, uint64_t *d_topk_idx, float *d_topk_score,
                  uint32_t *d_topk_count, void *d_workspace, size_t workspace_bytes, cudaStream_t st);

@@ -3,9 +3,86 @@
 // and adds the copies.  Inside one call the scoring kernel also collects what the selection's first pass would
 // read the dense outputs for (score-bit histograms and per-chunk counts of the eligible plans), so the selection
 // starts at its second pass.
+#include <cstring>
+#include <mutex>
+#include <vector>
+
 #include "pf_internal.cuh"
 
 namespace pf {
+
+// Pinned staging for the small results of pf_search_host_compact.  The caller's result pointers may be pageable
+// memory, and a device-to-host copy into pageable memory blocks the host until the stream has reached it: in the
+// middle of a call that would stop the host from enqueueing the rest of the search (measured: the count of feasible
+// plans, copied right behind the compaction, held the selection's and the simulator's launches back by 0.2 ms).  The
+// small results therefore travel into a pinned block of the library's own and are handed over with memcpy once the
+// call's stream work is done.  Blocks are kept for reuse (pinning memory takes a fraction of a millisecond).
+namespace {
+constexpr size_t kStageBytes = 32768;
+constexpr size_t kStageKeep = 8;
+std::mutex g_stage_mu;
+std::vector<void *> g_stage_free;
+void *stage_acquire()
+{
+    {
+        std::lock_guard<std::mutex> lock(g_stage_mu);
+        if (!g_stage_free.empty()) {
+            void *b = g_stage_free.back();
+            g_stage_free.pop_back();
+            return b;
+        }
+    }
+    void *b = nullptr;
+    if (cudaHostAlloc(&b, kStageBytes, cudaHostAllocPortable) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return nullptr;
+    }
+    return b;
+}
+void stage_release(void *b)
+{
+    if (!b) return;
+    {
+        std::lock_guard<std::mutex> lock(g_stage_mu);
+        if (g_stage_free.size() < kStageKeep) {
+            g_stage_free.push_back(b);
+            return;
+        }
+    }
+    cudaFreeHost(b);
+}
+// page-locked host memory (a copy into it does not block the host)?
+bool host_pinned(const void *h)
+{
+    cudaPointerAttributes a;
+    if (cudaPointerGetAttributes(&a, h) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return false;
+    }
+    return a.type == cudaMemoryTypeHost;
+}
+// One stream per device for pf_search_host_compact's early copy of a zero mask, shared by all plans (their copies
+// share the bus anyway) and kept for the life of the process: creating and destroying a stream with every plan
+// costs more than the copy saves when a plan serves a single call.
+constexpr int kCopyDevices = 64;
+std::mutex g_copy_mu;
+cudaStream_t g_copy_stream[kCopyDevices];
+cudaStream_t copy_stream_of_current_device()
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kCopyDevices) return nullptr;
+    std::lock_guard<std::mutex> lock(g_copy_mu);
+    if (!g_copy_stream[dev] && cudaStreamCreateWithFlags(&g_copy_stream[dev], cudaStreamNonBlocking) != cudaSuccess) {
+        (void)cudaGetLastError();
+        g_copy_stream[dev] = nullptr;
+    }
+    return g_copy_stream[dev];
+}
+struct StageHold {   // releases the block on every return path
+    void *b;
+    ~StageHold() { stage_release(b); }
+};
+}  // namespace
 
 struct SearchLayout {
     size_t off_reason, off_tput, off_mem, off_topk_idx, off_topk_score, off_topk_count, off_surv, off_surv_count,
@@ -70,6 +147,10 @@ struct CompactJob {
     void *cws;
     uint64_t *h_hist, *h_nfeas;
     uint8_t *h_mask;
+    // sparse mode: the caller has a copy of zeros on its way to the whole host mask (done at `zeros_done`); only the
+    // bits of chunks with feasible plans are written, through this device-visible alias of the host buffer
+    uint8_t *mask_alias = nullptr;
+    cudaEvent_t zeros_done = nullptr;
     bool launched = false;   // out: enqueued; ev_count follows the copy of the count, ev_compact the copy of the bits
 };
 
@@ -115,8 +196,13 @@ static int search_device(pf_plan_t *p, uint32_t k, uint64_t s_max, uint32_t k_si
             e = cudaMemcpyAsync(cj->h_hist, cj->d_hist, PF_REASON_BINS * 8, cudaMemcpyDeviceToHost, cs);
             if (e == cudaSuccess) e = cudaMemcpyAsync(cj->h_nfeas, cj->d_nfeas, 8, cudaMemcpyDeviceToHost, cs);
             if (e == cudaSuccess) e = cudaEventRecord(p->ev_count, cs);
-            if (e == cudaSuccess && cj->h_mask)
+            if (e == cudaSuccess && cj->mask_alias) {
+                e = cudaStreamWaitEvent(cs, cj->zeros_done, 0);
+                if (e == cudaSuccess && compact_mask_run(p, 0, p->size, d_reason, cj->mask_alias, cj->cws, cs, guard) != PF_OK)
+                    rc2 = PF_ECUDA;
+            } else if (e == cudaSuccess && cj->h_mask) {
                 e = cudaMemcpyAsync(cj->h_mask, cj->d_mask, ((size_t)p->size + 7) / 8, cudaMemcpyDeviceToHost, cs);
+            }
             if (e == cudaSuccess) e = cudaEventRecord(p->ev_compact, cs);
             if (e == cudaSuccess) cj->launched = true;
         }
@@ -300,36 +386,76 @@ extern "C" int pf_search_host_compact(pf_plan_t *p, uint32_t k, uint64_t s_max, 
     uint64_t *d_hist = (uint64_t *)(ws + cl.off_hist), *d_nfeas = (uint64_t *)(ws + cl.off_nfeas);
     uint8_t *d_mask = h_mask ? ws + cl.off_mask : nullptr;
     pf_record_t *d_records = (pf_record_t *)(ws + cl.off_records);
+    // the small results go through a pinned block (see stage_acquire): [histogram | count | top-k lists | simulator lists]
+    StageHold hold{stage_acquire()};
+    if (!hold.b) {
+        set_cuda_error(cudaErrorMemoryAllocation, "pf_search_host_compact: pinned staging");
+        return PF_ECUDA;
+    }
+    uint8_t *stage = (uint8_t *)hold.b;
+    // two stretches of the device layout travel whole: the analytic top-k (indices, scores, count) and, past the
+    // survivor list, the survivor count with the simulator's top-k
+    const size_t tk_bytes = l.off_surv - l.off_topk_idx, sm_bytes = l.off_ws - l.off_surv_count;
+    const size_t so_hist = 0, so_nfeas = PF_REASON_BINS * 8, so_tk = 256, so_sm = so_tk + tk_bytes;
+    if (so_sm + sm_bytes > kStageBytes) return PF_EINVAL;   // (k, k_sim <= PF_K_MAX: 25.6 KB at most)
+    uint64_t *s_hist = (uint64_t *)(stage + so_hist), *s_nfeas = (uint64_t *)(stage + so_nfeas);
     CompactJob cj;
     cj.d_hist = d_hist; cj.d_nfeas = d_nfeas; cj.d_mask = d_mask; cj.d_records = d_records; cj.record_cap = record_cap;
     cj.cws = ws + cl.off_cws;
-    cj.h_hist = h_hist; cj.h_nfeas = h_n_feasible; cj.h_mask = h_mask;
+    // the bits travel beside the search only into pinned memory; a pageable buffer gets them at the end
+    const bool mask_early = h_mask && host_pinned(h_mask);
+    cj.h_hist = s_hist; cj.h_nfeas = s_nfeas; cj.h_mask = mask_early ? h_mask : nullptr;
+    // Nearly all of the mask is zero (a chunk of 16,384 candidates without a feasible plan: 22.5 MB for the large
+    // space, of which a few hundred KB are not).  Where the device can write the host buffer directly, a copy of
+    // zeros to the whole of it starts now, on a stream of its own, and crosses the bus beside the search; the
+    // compact view then writes only the chunks that hold feasible plans, straight into the host buffer.
+    // (Events: the plan's ev_count marks the entry for the copy stream and ev_compact the end of the zero copy; both
+    // are recorded again later in the call, on the second stream, which by then has waited for this record.)
+    bool zeros_forked = false;
+    cudaStream_t zs = (mask_early && sim && p->side_stream) ? copy_stream_of_current_device() : nullptr;
+    if (zs) {
+        void *alias = nullptr;
+        if (cudaHostGetDevicePointer(&alias, h_mask, 0) == cudaSuccess && alias) {
+            cudaError_t e = cudaEventRecord(p->ev_count, st);
+            if (e == cudaSuccess) e = cudaStreamWaitEvent(zs, p->ev_count, 0);
+            if (e == cudaSuccess) {
+                zeros_forked = true;   // from here on the copy stream is joined whatever happens
+                e = cudaMemsetAsync(d_mask, 0, (N + 7) / 8, zs);
+                if (e == cudaSuccess) e = cudaMemcpyAsync(h_mask, d_mask, (N + 7) / 8, cudaMemcpyDeviceToHost, zs);
+                const cudaError_t e2 = cudaEventRecord(p->ev_compact, zs);
+                if (e == cudaSuccess) e = e2;
+            }
+            if (e != cudaSuccess) {
+                set_cuda_error(e, "pf_search_host_compact: zero mask");
+                if (zeros_forked) cudaStreamSynchronize(zs);
+                return PF_ECUDA;
+            }
+            cj.mask_alias = (uint8_t *)alias;
+            cj.zeros_done = p->ev_compact;
+            cj.d_mask = nullptr;   // the compact view's kernels write no mask of their own
+        } else {
+            (void)cudaGetLastError();
+        }
+    }
     int rc = search_device(p, k, s_max, k_sim, jitter_seed, d_reason, d_tput, d_mem, d_tk_idx, d_tk_sc, d_tk_cnt,
                            d_surv, d_surv_cnt, d_sim_idx, d_sim_sc, d_sim_cnt, ws + l.off_ws, l.ws_bytes,
                            ws + l.off_ws_sel, l.ws_sel_bytes, st, &cj);
+    if (zeros_forked) {
+        // join the copy stream (ev_compact: the zero copy's end, or the compact view's, which waited for that)
+        if (cudaStreamWaitEvent(st, p->ev_compact, 0) != cudaSuccess && rc == PF_OK) rc = PF_ECUDA;
+        if (rc != PF_OK) cudaStreamSynchronize(st);   // nothing of this call touches the host buffers after it returns
+    }
     if (rc != PF_OK) return rc;
     if (!cj.launched) {
         // no second stream took the compact view (a serving space, or no simulator tier): after the search
         rc = pf_compact(p, 0, N, d_reason, d_tput, d_mem, d_hist, d_mask, d_records, record_cap, d_nfeas, ws + cl.off_cws,
                         cl.cws_bytes, stream);
         if (rc != PF_OK) return rc;
-        PF_CUDA_TRY(cudaMemcpyAsync(h_hist, d_hist, PF_REASON_BINS * 8, cudaMemcpyDeviceToHost, st), "copy histogram");
-        PF_CUDA_TRY(cudaMemcpyAsync(h_n_feasible, d_nfeas, 8, cudaMemcpyDeviceToHost, st), "copy count");
-        if (h_mask) PF_CUDA_TRY(cudaMemcpyAsync(h_mask, d_mask, (N + 7) / 8, cudaMemcpyDeviceToHost, st), "copy mask");
+        PF_CUDA_TRY(cudaMemcpyAsync(s_hist, d_hist, PF_REASON_BINS * 8, cudaMemcpyDeviceToHost, st), "copy histogram");
+        PF_CUDA_TRY(cudaMemcpyAsync(s_nfeas, d_nfeas, 8, cudaMemcpyDeviceToHost, st), "copy count");
     }
-    PF_CUDA_TRY(cudaMemcpyAsync(h_topk_idx, d_tk_idx, (size_t)k * 8, cudaMemcpyDeviceToHost, st), "copy top-k");
-    PF_CUDA_TRY(cudaMemcpyAsync(h_topk_score, d_tk_sc, (size_t)k * 4, cudaMemcpyDeviceToHost, st), "copy top-k");
-    PF_CUDA_TRY(cudaMemcpyAsync(h_topk_count, d_tk_cnt, 4, cudaMemcpyDeviceToHost, st), "copy top-k");
-    if (sim) {
-        PF_CUDA_TRY(cudaMemcpyAsync(h_sim_topk_idx, d_sim_idx, (size_t)k_sim * 8, cudaMemcpyDeviceToHost, st), "copy sim");
-        PF_CUDA_TRY(cudaMemcpyAsync(h_sim_topk_score, d_sim_sc, (size_t)k_sim * 4, cudaMemcpyDeviceToHost, st), "copy sim");
-        PF_CUDA_TRY(cudaMemcpyAsync(h_sim_topk_count, d_sim_cnt, 4, cudaMemcpyDeviceToHost, st), "copy sim");
-        if (h_surv_count)
-            PF_CUDA_TRY(cudaMemcpyAsync(h_surv_count, d_surv_cnt, 8, cudaMemcpyDeviceToHost, st), "copy count");
-    } else {
-        if (h_sim_topk_count) *h_sim_topk_count = 0;
-        if (h_surv_count) *h_surv_count = 0;
-    }
+    PF_CUDA_TRY(cudaMemcpyAsync(stage + so_tk, ws + l.off_topk_idx, tk_bytes, cudaMemcpyDeviceToHost, st), "copy top-k");
+    if (sim) PF_CUDA_TRY(cudaMemcpyAsync(stage + so_sm, ws + l.off_surv_count, sm_bytes, cudaMemcpyDeviceToHost, st), "copy sim");
     // the record count decides how many records travel: wait for it (with a second stream at work it has been on
     // the host since shortly after the scoring kernel ended), then copy exactly those
     if (cj.launched)
@@ -337,11 +463,30 @@ extern "C" int pf_search_host_compact(pf_plan_t *p, uint32_t k, uint64_t s_max, 
     else
         PF_CUDA_TRY(cudaStreamSynchronize(st), "pf_search_host_compact: synchronize");
     if (record_cap > 0) {
-        const uint64_t n = *h_n_feasible < record_cap ? *h_n_feasible : record_cap;
+        const uint64_t n = *s_nfeas < record_cap ? *s_nfeas : record_cap;
         if (n > 0)
             PF_CUDA_TRY(cudaMemcpyAsync(h_records, d_records, (size_t)n * sizeof(pf_record_t), cudaMemcpyDeviceToHost, st),
                         "copy records");
     }
+    // (a pageable h_mask or h_records makes its copy a blocking one; nothing is left to enqueue behind them)
+    if (h_mask && !(cj.launched && mask_early))
+        PF_CUDA_TRY(cudaMemcpyAsync(h_mask, d_mask, (N + 7) / 8, cudaMemcpyDeviceToHost, st), "copy mask");
     PF_CUDA_TRY(cudaStreamSynchronize(st), "pf_search_host_compact: synchronize");
+    // hand the small results over
+    memcpy(h_hist, s_hist, PF_REASON_BINS * 8);
+    *h_n_feasible = *s_nfeas;
+    const uint8_t *s_tk = stage + so_tk, *s_sm = stage + so_sm;
+    memcpy(h_topk_idx, s_tk, (size_t)k * 8);
+    memcpy(h_topk_score, s_tk + (l.off_topk_score - l.off_topk_idx), (size_t)k * 4);
+    memcpy(h_topk_count, s_tk + (l.off_topk_count - l.off_topk_idx), 4);
+    if (sim) {
+        memcpy(h_sim_topk_idx, s_sm + (l.off_sim_idx - l.off_surv_count), (size_t)k_sim * 8);
+        memcpy(h_sim_topk_score, s_sm + (l.off_sim_score - l.off_surv_count), (size_t)k_sim * 4);
+        memcpy(h_sim_topk_count, s_sm + (l.off_sim_count - l.off_surv_count), 4);
+        if (h_surv_count) memcpy(h_surv_count, s_sm, 8);
+    } else {
+        if (h_sim_topk_count) *h_sim_topk_count = 0;
+        if (h_surv_count) *h_surv_count = 0;
+    }
     return PF_OK;
 }

@@ -94,6 +94,20 @@ def test_search_host_compact_on_the_large_space():
         assert rp["n_records"] == r["n_records"]
         np.testing.assert_array_equal(rp["records"][:rp["n_records"]], r["records"][:r["n_records"]])
         np.testing.assert_array_equal(rp["sim_topk_idx"], r["sim_topk_idx"])
+    # pinned host buffers take the bits and the records beside the search (pageable ones, above, at its end)
+    from paper_2607_18631_b200 import binding
+    p_mask = torch.full(((N + 7) // 8,), 0xFF, dtype=torch.uint8).pin_memory()
+    p_recs = torch.zeros(cap * binding.RECORD_DTYPE.itemsize, dtype=torch.uint8).pin_memory()
+    ws.fill_(0x85)
+    rq = plan.search_host_compact(1024, 10 ** 6, 100, 4, ws, cap, h_mask=p_mask, h_records=p_recs)
+    np.testing.assert_array_equal(rq["hist"], r["hist"])
+    np.testing.assert_array_equal(p_mask.numpy(), h_mask)
+    assert rq["n_records"] == r["n_records"] and rq["n_survivors"] == r["n_survivors"]
+    q_recs = p_recs.numpy().view(binding.RECORD_DTYPE)[:rq["n_records"]]
+    np.testing.assert_array_equal(q_recs, r["records"][:r["n_records"]])
+    np.testing.assert_array_equal(rq["topk_idx"], r["topk_idx"])
+    np.testing.assert_array_equal(rq["sim_topk_idx"], r["sim_topk_idx"])
+    np.testing.assert_array_equal(rq["sim_topk_score"], r["sim_topk_score"])
     # records and mask are optional, and a short record buffer is filled from the front
     r2 = plan.search_host_compact(1024, 10 ** 6, 100, 4, ws, 1000)
     assert r2["n_feasible"] == 12_905 and r2["n_records"] == 1000
