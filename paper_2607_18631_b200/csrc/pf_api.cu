@@ -4,6 +4,7 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -87,7 +88,119 @@ void timing_end(pf_plan_t *p, int cls, int n_kernels, cudaStream_t st)
 using pf::DevPlan;
 
 namespace pf {
-int build_sim_tables(pf_plan_t *p);  // pf_simulate.cu: schedule-order tables for the simulator
+// ------------------------------------------------------------------ per-device caches of plan resources
+// A plan owns one block of device memory, two streams and six events.  Creating and releasing those through the
+// runtime takes 0.3 - 0.9 ms per plan (measured), several times the search of a large space, so released ones are
+// kept -- a few per device, blocks only up to kArenaKeepBytes -- and handed to the next plan.  A block is handed back
+// only after the device has gone idle (pf_plan_destroy), so nothing of its former plan can still touch it.
+namespace {
+constexpr size_t kArenaKeepBytes = 8u << 20;
+constexpr size_t kKeepPerDevice = 4;
+struct ArenaSlot {
+    int device;
+    void *base;
+    size_t cap;
+};
+struct StreamSlot {
+    int device;
+    cudaStream_t side, fill;
+    cudaEvent_t ev[6];
+};
+std::mutex g_cache_mu;
+std::vector<ArenaSlot> g_arenas;
+std::vector<StreamSlot> g_streams;
+}  // namespace
+
+void *arena_acquire(int device, size_t need, size_t *cap)
+{
+    {
+        std::lock_guard<std::mutex> lock(g_cache_mu);
+        for (size_t i = 0; i < g_arenas.size(); i++)
+            if (g_arenas[i].device == device && g_arenas[i].cap >= need) {
+                void *b = g_arenas[i].base;
+                *cap = g_arenas[i].cap;
+                g_arenas.erase(g_arenas.begin() + (long)i);
+                return b;
+            }
+    }
+    void *b = nullptr;
+    // (rounded up so that plans of similar spaces can take each other's blocks)
+    const size_t want = (need + 65535) & ~(size_t)65535;
+    if (cudaMalloc(&b, want) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return nullptr;
+    }
+    *cap = want;
+    return b;
+}
+
+void arena_release(int device, void *base, size_t cap)
+{
+    if (!base) return;
+    if (cap <= kArenaKeepBytes) {
+        std::lock_guard<std::mutex> lock(g_cache_mu);
+        size_t kept = 0;
+        for (const ArenaSlot &a : g_arenas) kept += a.device == device;
+        if (kept < kKeepPerDevice) {
+            g_arenas.push_back(ArenaSlot{device, base, cap});
+            return;
+        }
+    }
+    cudaFree(base);
+}
+
+cudaError_t streams_acquire(pf_plan_t *p)
+{
+    {
+        std::lock_guard<std::mutex> lock(g_cache_mu);
+        for (size_t i = 0; i < g_streams.size(); i++)
+            if (g_streams[i].device == p->device) {
+                const StreamSlot s = g_streams[i];
+                g_streams.erase(g_streams.begin() + (long)i);
+                p->side_stream = s.side; p->fill_stream = s.fill;
+                p->ev_fork = s.ev[0]; p->ev_join = s.ev[1]; p->ev_fill = s.ev[2];
+                p->ev_fork3 = s.ev[3]; p->ev_count = s.ev[4]; p->ev_compact = s.ev[5];
+                return cudaSuccess;
+            }
+    }
+    // the fill stream carries a long streaming kernel that should yield to everything else: lowest priority
+    int prio_lo = 0, prio_hi = 0;
+    cudaError_t e = cudaDeviceGetStreamPriorityRange(&prio_lo, &prio_hi);
+    if (e == cudaSuccess) e = cudaStreamCreateWithPriority(&p->side_stream, cudaStreamNonBlocking, prio_hi);
+    if (e == cudaSuccess) e = cudaStreamCreateWithPriority(&p->fill_stream, cudaStreamNonBlocking, prio_lo);
+    cudaEvent_t *evs[6] = {&p->ev_fork, &p->ev_join, &p->ev_fill, &p->ev_fork3, &p->ev_count, &p->ev_compact};
+    for (int i = 0; i < 6 && e == cudaSuccess; i++) e = cudaEventCreateWithFlags(evs[i], cudaEventDisableTiming);
+    return e;   // on failure pf_plan_destroy releases what was created
+}
+
+void streams_release(pf_plan_t *p)
+{
+    const bool complete = p->side_stream && p->fill_stream && p->ev_fork && p->ev_join && p->ev_fill && p->ev_fork3 &&
+                          p->ev_count && p->ev_compact;
+    if (complete) {
+        std::lock_guard<std::mutex> lock(g_cache_mu);
+        size_t kept = 0;
+        for (const StreamSlot &s : g_streams) kept += s.device == p->device;
+        if (kept < kKeepPerDevice) {
+            g_streams.push_back(StreamSlot{p->device, p->side_stream, p->fill_stream,
+                                           {p->ev_fork, p->ev_join, p->ev_fill, p->ev_fork3, p->ev_count, p->ev_compact}});
+            p->side_stream = p->fill_stream = nullptr;
+            p->ev_fork = p->ev_join = p->ev_fill = p->ev_fork3 = p->ev_count = p->ev_compact = nullptr;
+            return;
+        }
+    }
+    cudaEvent_t evs[6] = {p->ev_fork, p->ev_join, p->ev_fill, p->ev_fork3, p->ev_count, p->ev_compact};
+    for (cudaEvent_t ev : evs)
+        if (ev) cudaEventDestroy(ev);
+    if (p->side_stream) cudaStreamDestroy(p->side_stream);
+    if (p->fill_stream) cudaStreamDestroy(p->fill_stream);
+    p->side_stream = p->fill_stream = nullptr;
+    p->ev_fork = p->ev_join = p->ev_fill = p->ev_fork3 = p->ev_count = p->ev_compact = nullptr;
+}
+
+int build_sim_tables(pf_plan_t *p);  // pf_simulate.cu: schedule-order tables for the simulator (host part)
+size_t sim_tables_bytes(const pf_plan_t *p);
+void sim_tables_place(pf_plan_t *p, uint8_t *dev, uint8_t *image);
 void free_sim_tables(pf_plan_t *p);
 }
 
@@ -414,58 +527,67 @@ extern "C" int pf_plan_create(const pf_model_t *model, const pf_cluster_t *clust
         d.sim_domain_all = all_in ? 1 : 0;
     }
 
-    // device copies
-    cudaError_t e = cudaMalloc((void **)&p->d_vals, sizeof(int32_t) * (size_t)total_vals);
-    if (e == cudaSuccess)
-        e = cudaMemcpy(p->d_vals, p->h_vals, sizeof(int32_t) * (size_t)total_vals, cudaMemcpyHostToDevice);
-    if (e == cudaSuccess && phase == PF_PHASE_SERVE) {
-        size_t n = (size_t)workload->n_scen;
-        e = cudaMalloc((void **)&p->d_scen, sizeof(int32_t) * 2 * n);
-        if (e == cudaSuccess) e = cudaMemcpy(p->d_scen, workload->scen_P, sizeof(int32_t) * n, cudaMemcpyHostToDevice);
-        if (e == cudaSuccess)
-            e = cudaMemcpy(p->d_scen + n, workload->scen_O, sizeof(int32_t) * n, cudaMemcpyHostToDevice);
-    }
-    if (e == cudaSuccess) e = cudaMalloc((void **)&p->d_fill_ctl, 2048);
-    if (e == cudaSuccess) e = cudaMalloc((void **)&p->d_check, 64);
-    if (e == cudaSuccess) e = cudaMemset(p->d_check, 0, 64);
-    d.chk = p->d_check;
-    if (e == cudaSuccess) {
-        // room for the slab visiting order of one pf_score range (any alignment of its first candidate)
-        const uint64_t slabs = (p->size + d.slab - 1) / d.slab + 1;
-        p->order_cap = 0;
-        p->order_n_slabs = 0;
-        if (slabs <= (uint64_t)pf::kOrderMaxSlabs) {
-            e = cudaMalloc((void **)&p->d_order, 256 + (size_t)slabs * 5);
-            if (e == cudaSuccess) e = cudaMemset(p->d_order, 0, 256);
-            p->order_cap = (uint32_t)slabs;
-        }
-    }
-    if (e != cudaSuccess) {
-        pf::set_cuda_error(e, "pf_plan_create: upload");
-        pf_plan_destroy(p);
-        return PF_ECUDA;
-    }
+    // Device side: ONE block per plan -- [axis values | scenario lengths | fill-kernel control | check record |
+    // simulator order tables | order-table header] uploaded as one image, then the order table's body, which the
+    // first call builds.  The block comes from a small per-device cache (see arena_acquire), and so do the plan's
+    // streams and events: a plan that serves a single call would otherwise spend more time in the allocator
+    // than in the search.
     if (phase == PF_PHASE_TRAIN) {
-        // the fill stream carries long streaming-store kernels that should yield to everything else: lowest priority
-        int prio_lo = 0, prio_hi = 0;
-        e = cudaDeviceGetStreamPriorityRange(&prio_lo, &prio_hi);
-        if (e == cudaSuccess) e = cudaStreamCreateWithPriority(&p->side_stream, cudaStreamNonBlocking, prio_hi);
-        if (e == cudaSuccess) e = cudaStreamCreateWithPriority(&p->fill_stream, cudaStreamNonBlocking, prio_lo);
-        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->ev_fork, cudaEventDisableTiming);
-        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->ev_join, cudaEventDisableTiming);
-        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->ev_fill, cudaEventDisableTiming);
-        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->ev_fork3, cudaEventDisableTiming);
-        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->ev_count, cudaEventDisableTiming);
-        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->ev_compact, cudaEventDisableTiming);
-        if (e != cudaSuccess) {
-            pf::set_cuda_error(e, "pf_plan_create: side stream");
-            pf_plan_destroy(p);
-            return PF_ECUDA;
-        }
         int rc = pf::build_sim_tables(p);
         if (rc != PF_OK) {
             pf_plan_destroy(p);
             return rc;
+        }
+    }
+    auto up = [](size_t x) { return (x + 255) & ~(size_t)255; };
+    const size_t n_scen = phase == PF_PHASE_SERVE ? (size_t)workload->n_scen : 0;
+    const size_t o_vals = 0, o_scen = o_vals + up(sizeof(int32_t) * (size_t)total_vals);
+    const size_t o_fill = o_scen + up(sizeof(int32_t) * 2 * n_scen), o_check = o_fill + 2048, o_sim = o_check + 256;
+    const size_t o_order = o_sim + pf::sim_tables_bytes(p);
+    // room for the slab visiting order of one pf_score range (any alignment of its first candidate)
+    const uint64_t slabs = (p->size + d.slab - 1) / d.slab + 1;
+    const bool has_order = slabs <= (uint64_t)pf::kOrderMaxSlabs;
+    const size_t image_bytes = o_order + 256;
+    const size_t need = has_order ? o_order + up(256 + (size_t)slabs * 5) : image_bytes;
+    p->arena = pf::arena_acquire(dev, need, &p->arena_cap);
+    if (!p->arena) {
+        pf::set_cuda_error(cudaErrorMemoryAllocation, "pf_plan_create: device block");
+        pf_plan_destroy(p);
+        return PF_ECUDA;
+    }
+    uint8_t *base = (uint8_t *)p->arena;
+    p->d_vals = (int32_t *)(base + o_vals);
+    if (n_scen) p->d_scen = (int32_t *)(base + o_scen);
+    p->d_fill_ctl = (unsigned int *)(base + o_fill);
+    p->d_check = (unsigned int *)(base + o_check);
+    d.chk = p->d_check;
+    p->order_cap = 0;
+    p->order_n_slabs = 0;
+    if (has_order) {
+        p->d_order = (uint32_t *)(base + o_order);
+        p->order_cap = (uint32_t)slabs;
+    }
+    {
+        std::vector<uint8_t> image(image_bytes, 0);   // control words, check record and order header start as zeros
+        memcpy(image.data() + o_vals, p->h_vals, sizeof(int32_t) * (size_t)total_vals);
+        if (n_scen) {
+            memcpy(image.data() + o_scen, workload->scen_P, sizeof(int32_t) * n_scen);
+            memcpy(image.data() + o_scen + sizeof(int32_t) * n_scen, workload->scen_O, sizeof(int32_t) * n_scen);
+        }
+        pf::sim_tables_place(p, base + o_sim, image.data() + o_sim);
+        const cudaError_t e = cudaMemcpy(base, image.data(), image_bytes, cudaMemcpyHostToDevice);
+        if (e != cudaSuccess) {
+            pf::set_cuda_error(e, "pf_plan_create: upload");
+            pf_plan_destroy(p);
+            return PF_ECUDA;
+        }
+    }
+    if (phase == PF_PHASE_TRAIN) {
+        const cudaError_t e = pf::streams_acquire(p);
+        if (e != cudaSuccess) {
+            pf::set_cuda_error(e, "pf_plan_create: side stream");
+            pf_plan_destroy(p);
+            return PF_ECUDA;
         }
     }
     *out = p;
@@ -569,19 +691,16 @@ extern "C" void pf_plan_destroy(pf_plan_t *p)
         delete t;
     }
     pf::free_sim_tables(p);
-    if (p->d_vals) cudaFree(p->d_vals);
-    if (p->d_scen) cudaFree(p->d_scen);
-    if (p->d_order) cudaFree(p->d_order);
-    if (p->d_check) cudaFree(p->d_check);
-    if (p->d_fill_ctl) cudaFree(p->d_fill_ctl);
-    if (p->ev_fork) cudaEventDestroy(p->ev_fork);
-    if (p->ev_join) cudaEventDestroy(p->ev_join);
-    if (p->ev_fill) cudaEventDestroy(p->ev_fill);
-    if (p->ev_fork3) cudaEventDestroy(p->ev_fork3);
-    if (p->ev_count) cudaEventDestroy(p->ev_count);
-    if (p->ev_compact) cudaEventDestroy(p->ev_compact);
-    if (p->side_stream) cudaStreamDestroy(p->side_stream);
-    if (p->fill_stream) cudaStreamDestroy(p->fill_stream);
+    // The device block and the streams go back to their caches.  Work of this plan may still be in flight on a stream
+    // of the caller's; freeing the block would have waited for the device, so this does too.
+    if (p->arena || p->side_stream) {
+        int cur = -1;
+        const bool switched = cudaGetDevice(&cur) == cudaSuccess && cur != p->device && cudaSetDevice(p->device) == cudaSuccess;
+        cudaDeviceSynchronize();
+        if (switched) cudaSetDevice(cur);
+    }
+    pf::streams_release(p);
+    pf::arena_release(p->device, p->arena, p->arena_cap);
     free(p->h_vals);
     delete p;
 }

@@ -136,7 +136,9 @@ struct pf_plan {
     // host copies
     int32_t *h_vals;               // packed axis value lists
     int32_t axis_len[PF_MAX_AXES];
-    // device buffers owned by the handle
+    // device buffers owned by the handle: all inside one block (arena) from a per-device cache
+    void *arena;
+    size_t arena_cap;
     int32_t *d_vals;               // packed axis value lists
     int32_t *d_scen;               // serve: P[n_scen] then O[n_scen]
     // Slab visiting order of the most recent pf_score range (device: 64 header words, order_cap order words,

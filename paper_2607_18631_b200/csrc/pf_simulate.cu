@@ -29,11 +29,13 @@ namespace pf {
 // DualPipe-style order tables: for every (pp, m) in the domain a byte string per rank,
 // op = (j << 2) | (dir << 1) | is_backward, 2*m ops per rank.
 struct SimTables {
-    uint8_t *d_ops;                 // device copy of all tables
+    uint8_t *d_ops;                 // device copy of all tables (inside the plan's device block)
     int32_t *d_offset;              // [33][33]: offset of table (pp, m/2), -1 if absent
     std::vector<int32_t> h_offset;
+    std::vector<uint8_t> h_ops;     // host copy, until it has been placed in the plan's device block
     size_t bytes;
 };
+constexpr size_t kSimOffsetBytes = (sizeof(int32_t) * 33 * 33 + 255) & ~(size_t)255;
 
 // Host: nominal list scheduling that DEFINES the DualPipe-style order (F = 1 tick, B = 2 ticks, zero
 // latency).  At every event time each idle rank starts the ready op with the smallest
@@ -104,7 +106,8 @@ static bool build_dualpipe_table(int pp, int m, uint8_t *out /* [pp][2m] */)
     return true;
 }
 
-// Called once by pf_plan_create for training plans: builds and uploads the order tables.
+// Called once by pf_plan_create for training plans: builds the order tables on the host; sim_tables_place puts them
+// into the plan's device block.
 int build_sim_tables(pf_plan_t *p)
 {
     if (p->sim_tables) return PF_OK;
@@ -137,29 +140,37 @@ int build_sim_tables(pf_plan_t *p)
         }
     }
     t->bytes = ops.size();
-    cudaError_t e = cudaMalloc((void **)&t->d_offset, sizeof(int32_t) * 33 * 33);
-    if (e == cudaSuccess)
-        e = cudaMemcpy(t->d_offset, t->h_offset.data(), sizeof(int32_t) * 33 * 33, cudaMemcpyHostToDevice);
-    if (e == cudaSuccess) e = cudaMalloc((void **)&t->d_ops, ops.size() ? ops.size() : 16);
-    if (e == cudaSuccess && !ops.empty()) e = cudaMemcpy(t->d_ops, ops.data(), ops.size(), cudaMemcpyHostToDevice);
-    if (e != cudaSuccess) {
-        set_cuda_error(e, "simulator tables");
-        if (t->d_offset) cudaFree(t->d_offset);
-        if (t->d_ops) cudaFree(t->d_ops);
-        delete t;
-        return PF_ECUDA;
-    }
+    t->h_ops.swap(ops);
     p->sim_tables = t;
     return PF_OK;
+}
+
+// bytes of the plan's device block the tables take (both parts 256-byte aligned)
+size_t sim_tables_bytes(const pf_plan_t *p)
+{
+    const SimTables *t = (const SimTables *)p->sim_tables;
+    if (!t) return 0;
+    return kSimOffsetBytes + (((t->bytes ? t->bytes : 16) + 255) & ~(size_t)255);
+}
+
+// The tables live at `dev` in the plan's device block; their bytes are written to `image`, the host copy of that
+// stretch, which the caller uploads with the rest of the block.
+void sim_tables_place(pf_plan_t *p, uint8_t *dev, uint8_t *image)
+{
+    SimTables *t = (SimTables *)p->sim_tables;
+    if (!t) return;
+    t->d_offset = (int32_t *)dev;
+    t->d_ops = dev + kSimOffsetBytes;
+    memcpy(image, t->h_offset.data(), sizeof(int32_t) * 33 * 33);
+    if (!t->h_ops.empty()) memcpy(image + kSimOffsetBytes, t->h_ops.data(), t->h_ops.size());
+    std::vector<uint8_t>().swap(t->h_ops);
 }
 
 void free_sim_tables(pf_plan_t *p)
 {
     SimTables *t = (SimTables *)p->sim_tables;
     if (!t) return;
-    if (t->d_offset) cudaFree(t->d_offset);
-    if (t->d_ops) cudaFree(t->d_ops);
-    delete t;
+    delete t;   // (the device copy is part of the plan's device block)
     p->sim_tables = nullptr;
 }
 
