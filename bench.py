@@ -563,7 +563,8 @@ def run_ours(args):
     e2e = {"value": world * N / s_compact, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h_compact,
            "steps": e2e_steps, "ms_per_step": s_compact * 1e3,
            "mode": "pf_plan_create + pf_search_host_compact + pf_plan_destroy per step: reason histogram, feasibility "
-                   "bits, records of every feasible plan, both top-k lists"}
+                   "bits (a copy of zeros to the whole pinned mask beside the search + device writes of the 2 KB "
+                   "stretches that hold feasible plans), records of every feasible plan, both top-k lists"}
     if not args.no_dense_e2e:
         h_reason = torch.empty(N, dtype=torch.uint8, pin_memory=True)
         h_tput = torch.empty(N, dtype=torch.float32, pin_memory=True)
