@@ -83,3 +83,32 @@ def test_search_after_recycling_matches_a_fresh_process_result():
         else:
             for k in first:
                 np.testing.assert_array_equal(got[k], first[k])
+
+
+def test_plans_created_and_destroyed_from_several_threads():
+    """The caches are shared by every thread of the process (ctypes calls run without the interpreter lock)."""
+    import threading
+    import torch
+    cfgs = [make_config("mid"), make_config("tiny"), variant("mid", cluster=dict(budget_bytes=10 ** 15))]
+    refs = [_ref(c) for c in cfgs]
+    errors = []
+
+    def work(seed):
+        try:
+            torch.cuda.set_device(0)
+            stream = torch.cuda.Stream()
+            with torch.cuda.stream(stream):
+                for i in range(12):
+                    j = (seed + i) % len(cfgs)
+                    plan = _plan(cfgs[j])
+                    _parity(plan, cfgs[j], refs[j])
+                    plan.close()
+        except Exception as ex:   # noqa: BLE001 -- reported by the main thread
+            errors.append(repr(ex))
+
+    threads = [threading.Thread(target=work, args=(s,)) for s in range(4)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    assert not errors, errors
