@@ -415,7 +415,8 @@ extern "C" int pf_search_host_compact(pf_plan_t *p, uint32_t k, uint64_t s_max, 
     cudaStream_t zs = (mask_early && sim && p->side_stream) ? copy_stream_of_current_device() : nullptr;
     if (zs) {
         void *alias = nullptr;
-        if (cudaHostGetDevicePointer(&alias, h_mask, 0) == cudaSuccess && alias) {
+        // (the device writes 32-bit words: a buffer that is not 4-byte aligned takes the copy at the end instead)
+        if (cudaHostGetDevicePointer(&alias, h_mask, 0) == cudaSuccess && alias && ((uintptr_t)alias & 3) == 0) {
             cudaError_t e = cudaEventRecord(p->ev_count, st);
             if (e == cudaSuccess) e = cudaStreamWaitEvent(zs, p->ev_count, 0);
             if (e == cudaSuccess) {

@@ -108,6 +108,17 @@ def test_search_host_compact_on_the_large_space():
     np.testing.assert_array_equal(rq["topk_idx"], r["topk_idx"])
     np.testing.assert_array_equal(rq["sim_topk_idx"], r["sim_topk_idx"])
     np.testing.assert_array_equal(rq["sim_topk_score"], r["sim_topk_score"])
+    # the device writes into the pinned mask itself: nothing outside it may change, and a mask that starts at an odd
+    # address (the device writes whole words) must come out the same
+    nb = (N + 7) // 8
+    for lead in (64, 61):
+        guard = torch.full((lead + nb + 64,), 0xA5, dtype=torch.uint8).pin_memory()
+        ws.fill_(0)
+        rg = plan.search_host_compact(1024, 10 ** 6, 100, 4, ws, cap, h_mask=guard[lead:lead + nb], h_records=p_recs)
+        g = guard.numpy()
+        np.testing.assert_array_equal(g[lead:lead + nb], h_mask)
+        assert (g[:lead] == 0xA5).all() and (g[lead + nb:] == 0xA5).all()
+        np.testing.assert_array_equal(rg["hist"], r["hist"])
     # records and mask are optional, and a short record buffer is filled from the front
     r2 = plan.search_host_compact(1024, 10 ** 6, 100, 4, ws, 1000)
     assert r2["n_feasible"] == 12_905 and r2["n_records"] == 1000
