@@ -551,7 +551,7 @@ __global__ void __launch_bounds__(256) sim_records_kernel(const __grid_constant_
 __device__ __forceinline__ void sim_rounds_1f1b(volatile float *tl, const float *durF, const float *durB, int glane,
                                                 int pp, int nj, int warm, int total_ops, float lat, int fonly,
                                                 float &clock_out, int &done_out, unsigned int *chk, int w_lim,
-                                                int r_lim)
+                                                int r_lim, int sw)
 {
     (void)chk; (void)w_lim; (void)r_lim;
     // lanes beyond the pipeline depth take no part: they poll row 0 and never act
@@ -573,7 +573,7 @@ __device__ __forceinline__ void sim_rounds_1f1b(volatile float *tl, const float 
     {                                                                                        \
         const bool go = nF < njl && nF - nB <= warm && (!depF || (e) > 0.f);                 \
         const float t = fmaxf(clock, depF ? (e) + latF : 0.f) + dF;                          \
-        if (go) tl[PF_AT(chk, aF, w_lim, PF_SITE_TIMELINE)] = t;                             \
+        if (go) tl[PF_AT(chk, (aF) ^ sw, w_lim, PF_SITE_TIMELINE)] = t;                             \
         clock = go ? t : clock;                                                              \
         aF += go ? pp : 0;                                                                   \
         nF += go ? 1 : 0;                                                                    \
@@ -582,7 +582,7 @@ __device__ __forceinline__ void sim_rounds_1f1b(volatile float *tl, const float 
     {                                                                                        \
         const bool go = nB < njl && (nF - nB > warm || nF == njl) && (!depB || (e) < 0.f);   \
         const float t = fmaxf(clock, depB ? latB - (e) : 0.f) + dB;                          \
-        if (go) tl[PF_AT(chk, aB, w_lim, PF_SITE_TIMELINE)] = -t;                            \
+        if (go) tl[PF_AT(chk, (aB) ^ sw, w_lim, PF_SITE_TIMELINE)] = -t;                            \
         clock = go ? t : clock;                                                              \
         aB += go ? pp : 0;                                                                   \
         nB += go ? 1 : 0;                                                                    \
@@ -590,7 +590,7 @@ __device__ __forceinline__ void sim_rounds_1f1b(volatile float *tl, const float 
     // No backward can run before the first microbatch has crossed the shallowest pipeline of the warp: the first
     // `fonly` steps are forward steps only.
     for (int i = 0; i < fonly; i++) {
-        const float eF = tl[PF_AT(chk, aF + pF, r_lim, PF_SITE_TIMELINE)];
+        const float eF = tl[PF_AT(chk, (aF + pF) ^ sw, r_lim, PF_SITE_TIMELINE)];
         PF_SIM_FWD(eF)
     }
     for (;;) {
@@ -599,8 +599,8 @@ __device__ __forceinline__ void sim_rounds_1f1b(volatile float *tl, const float 
             // both polls are issued before either step runs, so that their shared-memory latencies overlap (the
             // backward step's dependency is another lane's word: reading it a few instructions early only means a
             // value that arrives in between is seen one iteration later)
-            const float eF = tl[PF_AT(chk, aF + pF, r_lim, PF_SITE_TIMELINE)];
-            const float eB = tl[PF_AT(chk, aB + pB, r_lim, PF_SITE_TIMELINE)];
+            const float eF = tl[PF_AT(chk, (aF + pF) ^ sw, r_lim, PF_SITE_TIMELINE)];
+            const float eB = tl[PF_AT(chk, (aB + pB) ^ sw, r_lim, PF_SITE_TIMELINE)];
             PF_SIM_FWD(eF)
             PF_SIM_BWD(eB)
         }
@@ -610,7 +610,7 @@ __device__ __forceinline__ void sim_rounds_1f1b(volatile float *tl, const float 
     while (__any_sync(0xFFFFFFFFu, nB < njl)) {
 #pragma unroll
         for (int rep = 0; rep < 4; rep++) {
-            const float eB = tl[PF_AT(chk, aB + pB, r_lim, PF_SITE_TIMELINE)];
+            const float eB = tl[PF_AT(chk, (aB + pB) ^ sw, r_lim, PF_SITE_TIMELINE)];
             PF_SIM_BWD(eB)
         }
         if ((++rounds & 15) == 0) {
@@ -633,7 +633,7 @@ __device__ __forceinline__ void sim_rounds_interleaved(volatile float *tl, const
                                                        int glane, int pp, int v, int nj, int U, int warm,
                                                        int total_ops, float lat, int fonly, float &clock_out,
                                                        int &done_out, unsigned int *chk, int w_lim, int r_lim,
-                                                       int q_lim)
+                                                       int q_lim, int sw)
 {
     (void)chk; (void)w_lim; (void)r_lim; (void)q_lim;
     const int Q = pp * v;
@@ -654,7 +654,7 @@ __device__ __forceinline__ void sim_rounds_interleaved(volatile float *tl, const
         const bool dep = qF > 0;                                                                        \
         const bool go = nF < Ul && nF - nB <= warm && (!dep || (e) > 0.f);                              \
         const float t = fmaxf(clock, dep ? (e) + lat : 0.f) + durF[PF_AT(chk, qF, q_lim, PF_SITE_DURATION)]; \
-        if (go) tl[PF_AT(chk, aF, w_lim, PF_SITE_TIMELINE)] = t;                                        \
+        if (go) tl[PF_AT(chk, (aF) ^ sw, w_lim, PF_SITE_TIMELINE)] = t;                                        \
         clock = go ? t : clock;                                                                         \
         const bool ww = fw == 0, wc = fc == 0;                                                          \
         aF += go ? (ww ? (wc ? stepF_window : stepF_chunk) : Q) : 0;                                    \
@@ -669,7 +669,7 @@ __device__ __forceinline__ void sim_rounds_interleaved(volatile float *tl, const
         const bool dep = qB < Q - 1;                                                                    \
         const bool go = nB < Ul && (nF - nB > warm || nF == Ul) && (!dep || (e) < 0.f);                 \
         const float t = fmaxf(clock, dep ? lat - (e) : 0.f) + durB[PF_AT(chk, qB, q_lim, PF_SITE_DURATION)]; \
-        if (go) tl[PF_AT(chk, aB, w_lim, PF_SITE_TIMELINE)] = -t;                                       \
+        if (go) tl[PF_AT(chk, (aB) ^ sw, w_lim, PF_SITE_TIMELINE)] = -t;                                       \
         clock = go ? t : clock;                                                                         \
         const bool ww = bw == 0, wc = bc == 0;                                                          \
         aB += go ? (ww ? (wc ? stepB_window : stepB_chunk) : Q) : 0;                                    \
@@ -680,8 +680,8 @@ __device__ __forceinline__ void sim_rounds_interleaved(volatile float *tl, const
     }
     // the words polled: one stage down / up from the own word (the own word when there is no dependency; once a
     // direction has run out of units its cursor rests up to Q words past the timeline, inside the warp's slice)
-#define PF_SIM_POLL_F() tl[PF_AT(chk, aF - (qF > 0 ? 1 : 0), r_lim, PF_SITE_TIMELINE)]
-#define PF_SIM_POLL_B() tl[PF_AT(chk, aB + (qB < Q - 1 ? 1 : 0), r_lim, PF_SITE_TIMELINE)]
+#define PF_SIM_POLL_F() tl[PF_AT(chk, (aF - (qF > 0 ? 1 : 0)) ^ sw, r_lim, PF_SITE_TIMELINE)]
+#define PF_SIM_POLL_B() tl[PF_AT(chk, (aB + (qB < Q - 1 ? 1 : 0)) ^ sw, r_lim, PF_SITE_TIMELINE)]
     // forward steps only until the first microbatch can have crossed the shallowest pipeline of the warp
     for (int i = 0; i < fonly; i++) {
         const float eF = PF_SIM_POLL_F();
@@ -729,7 +729,7 @@ __device__ __forceinline__ void sim_rounds_interleaved_ring(volatile unsigned lo
                                                             const float *durB, int glane, int pp, int v, int U,
                                                             int warm, int total_ops, float lat, int fonly,
                                                             float &clock_out, int &done_out, unsigned int *chk,
-                                                            int w_lim, int r_lim, int q_lim)
+                                                            int w_lim, int r_lim, int q_lim, int sw)
 {
     (void)chk; (void)w_lim; (void)r_lim; (void)q_lim;
     const int Q = pp * v;
@@ -753,7 +753,7 @@ __device__ __forceinline__ void sim_rounds_interleaved_ring(volatile unsigned lo
         const bool go = nF < Ul && nF - nB <= warm && ready;                                            \
         const float ev = __uint_as_float((unsigned int)((e) >> 32));                                    \
         const float t = fmaxf(clock, dep ? ev + lat : 0.f) + durF[PF_AT(chk, qF, q_lim, PF_SITE_DURATION)]; \
-        if (go) tl[PF_AT(chk, aF, w_lim, PF_SITE_TIMELINE)] = PF_RING_WORD(2 * jF + 1, t);              \
+        if (go) tl[PF_AT(chk, (aF) ^ sw, w_lim, PF_SITE_TIMELINE)] = PF_RING_WORD(2 * jF + 1, t);              \
         clock = go ? t : clock;                                                                         \
         const bool ww = fw == 0, wc = fc == 0;                                                          \
         aF += go ? (ww ? (wc ? (oddF ? stepF_wrap : stepF_up) : stepF_chunk) : Q) : 0;                  \
@@ -771,7 +771,7 @@ __device__ __forceinline__ void sim_rounds_interleaved_ring(volatile unsigned lo
         const bool go = nB < Ul && (nF - nB > warm || nF == Ul) && ready;                               \
         const float ev = __uint_as_float((unsigned int)((e) >> 32));                                    \
         const float t = fmaxf(clock, dep ? ev + lat : 0.f) + durB[PF_AT(chk, qB, q_lim, PF_SITE_DURATION)]; \
-        if (go) tl[PF_AT(chk, aB, w_lim, PF_SITE_TIMELINE)] = PF_RING_WORD(2 * jB + 2, t);              \
+        if (go) tl[PF_AT(chk, (aB) ^ sw, w_lim, PF_SITE_TIMELINE)] = PF_RING_WORD(2 * jB + 2, t);              \
         clock = go ? t : clock;                                                                         \
         const bool ww = bw == 0, wc = bc == 0;                                                          \
         aB += go ? (ww ? (wc ? (oddB ? stepB_wrap : stepB_up) : stepB_chunk) : Q) : 0;                  \
@@ -783,8 +783,8 @@ __device__ __forceinline__ void sim_rounds_interleaved_ring(volatile unsigned lo
         nB += go ? 1 : 0;                                                                               \
     }
     // once a direction has run out of units its cursor rests on some slot of the ring: a valid word, never taken
-#define PF_SIM_POLL_F() tl[PF_AT(chk, aF - (qF > 0 ? 1 : 0), r_lim, PF_SITE_TIMELINE)]
-#define PF_SIM_POLL_B() tl[PF_AT(chk, aB + (qB < Q - 1 ? 1 : 0), r_lim, PF_SITE_TIMELINE)]
+#define PF_SIM_POLL_F() tl[PF_AT(chk, (aF - (qF > 0 ? 1 : 0)) ^ sw, r_lim, PF_SITE_TIMELINE)]
+#define PF_SIM_POLL_B() tl[PF_AT(chk, (aB + (qB < Q - 1 ? 1 : 0)) ^ sw, r_lim, PF_SITE_TIMELINE)]
     for (int i = 0; i < fonly; i++) {
         const unsigned long long eF = PF_SIM_POLL_F();
         PF_SIM_FWD(eF)
@@ -824,7 +824,7 @@ __device__ __forceinline__ void sim_rounds_interleaved_ring(volatile unsigned lo
 __device__ __forceinline__ void sim_rounds_dual(volatile float *tl, const float *durF, const float *durB, int glane,
                                                 int pp, int nj, const uint8_t *ops, int total_ops, float lat,
                                                 float &clock_out, int &done_out, unsigned int *chk, int w_lim,
-                                                int r_lim, int q_lim)
+                                                int r_lim, int q_lim, int sw)
 {
     (void)chk; (void)w_lim; (void)r_lim; (void)q_lim;
     int done = 0, rounds = 0;
@@ -841,11 +841,11 @@ __device__ __forceinline__ void sim_rounds_dual(volatile float *tl, const float 
             const int sidx = d * pp + q;
             const bool dep = isb ? (q < pp - 1) : (q > 0);
             const int nb = dep ? (isb ? sidx + 1 : sidx - 1) : sidx;
-            const float e = tl[PF_AT(chk, j * 2 * pp + nb, r_lim, PF_SITE_TIMELINE)];
+            const float e = tl[PF_AT(chk, (j * 2 * pp + nb) ^ sw, r_lim, PF_SITE_TIMELINE)];
             const float dur = (isb ? durB : durF)[PF_AT(chk, q, q_lim, PF_SITE_DURATION)];
             if (!dep || (isb ? e < 0.f : e > 0.f)) {
                 clock = fmaxf(clock, dep ? fabsf(e) + lat : 0.f) + dur;
-                tl[PF_AT(chk, j * 2 * pp + sidx, w_lim, PF_SITE_TIMELINE)] = isb ? -clock : clock;
+                tl[PF_AT(chk, (j * 2 * pp + sidx) ^ sw, w_lim, PF_SITE_TIMELINE)] = isb ? -clock : clock;
                 done++;
                 moved = true;
             }
@@ -879,12 +879,23 @@ __device__ __forceinline__ void sim_rounds_dual(volatile float *tl, const float 
 // (and the groups of a warp) stay converged and a round costs one shared-memory poll plus one vote.  Every 64
 // rounds some lane of the warp must have advanced, otherwise its unfinished candidates are reported as
 // PF_SIM_STALL: the loop is bounded by the op count.
-// Two instances: kRings = true can serve ring-timeline bins too and is launched for the large calls that have them;
-// kRings = false is the same kernel without the ring loop (fewer registers, less code), for all other calls.
+// Two instances: kRings = true serves the large calls (at least kSimRingMinSurvivors actual survivors: ring-timeline
+// bins, four-lane groups, bank-permuted timelines); kRings = false is the same kernel without the ring loop and
+// the permutation (fewer registers, fewer instructions per step), for all other calls.
 template <bool kRings>
 __global__ void __launch_bounds__(kSimThreads, 4) simulate_kernel(const __grid_constant__ DevPlan P, const SimArgs A)
 {
     chain_enter();
+    // which instance serves the call is decided here, from the actual number of survivors (the host knows only the
+    // list's capacity and launches both when that is large)
+    {
+        uint64_t n_call = A.n;
+        if (A.d_n) {
+            const uint64_t dn = *A.d_n;
+            n_call = dn < n_call ? dn : n_call;
+        }
+        if ((n_call >= kSimRingMinSurvivors) != kRings) return;
+    }
     extern __shared__ __align__(16) float s_mem[];
     // (1,016 bytes, and not one more: three blocks of this kernel -- 72 KB of timelines each -- and one block of the fill
     // kernel fill an SM's shared memory to the last kilobyte)
@@ -952,6 +963,13 @@ __global__ void __launch_bounds__(kSimThreads, 4) simulate_kernel(const __grid_c
         const int gidx = lane / g, glane = lane - gidx * g;
         const bool group_on = gidx < batch;
         volatile float *tl = slice + (size_t)(group_on ? gidx : 0) * E;   // the timeline
+        // The groups' timelines start a multiple of 32 words apart and, candidates of one bin being alike, the groups
+        // tend to touch the same relative word at the same time: the same banks.  Every timeline index is therefore
+        // XORed with a constant of the group (a permutation of the 32-word stretches of its own timeline) that moves
+        // group i's lanes i * g * (words per lane) banks on: the groups of a warp then cover different banks.
+        // (large calls only: a small call is bound by instruction issue along its longest op chain, and the XOR costs
+        // it more than the conflicts do -- measured 0.151 against 0.139 ms)
+        const int sw = kRings ? (gidx * g * (bin_kind == kSimKindRing ? 2 : 1)) & 31 : 0;
         const int qg = sim_group_stages(g, A.q_max);           // stages a group's duration tables hold
         float *durF = slice + E_hi + (size_t)(group_on ? gidx : 0) * 2 * qg, *durB = durF + qg;
         const bool have = cur.have;                            // this group's candidate exists
@@ -993,7 +1011,7 @@ __global__ void __launch_bounds__(kSimThreads, 4) simulate_kernel(const __grid_c
             // clear the timeline with 16-byte stores (the slot is a multiple of four words, 16-byte aligned)
             {
                 float4 *tl4 = reinterpret_cast<float4 *>(const_cast<float *>(tl));
-                const int n4 = (n_entries + 3) >> 2;
+                const int n4 = ((n_entries + 31) & ~31) >> 2;   // whole 32-word stretches: what the permuted indices reach
 #pragma unroll 4
                 for (int i = glane; i < n4; i += g) tl4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
             }
@@ -1015,7 +1033,7 @@ __global__ void __launch_bounds__(kSimThreads, 4) simulate_kernel(const __grid_c
         const float lat = run ? lat_p : 0.f;
         // limits for the checked build: writes stay inside the candidate's own timeline, reads inside the warp's slice
         // (a lane that has run out of ops still polls one word past its row)
-        const int w_lim = run ? n_entries : 1;
+        const int w_lim = run ? ((n_entries + 31) & ~31) : 1;
         const int r_lim = A.warp_floats - (group_on ? gidx : 0) * E;
         // a batch's candidates share the schedule class of their bin: one specialised loop per class
         int done = 0;
@@ -1027,14 +1045,14 @@ __global__ void __launch_bounds__(kSimThreads, 4) simulate_kernel(const __grid_c
         if (kRings && bin_kind == kSimKindRing)
             // (two-word slots: the limits count slots)
             sim_rounds_interleaved_ring(reinterpret_cast<volatile unsigned long long *>(tl), durF, durB, glane, pp, v, U,
-                                        warm, total_ops, lat, fonly, clock, done, P.chk, w_lim >> 1, r_lim >> 1, qg);
+                                        warm, total_ops, lat, fonly, clock, done, P.chk, w_lim >> 1, r_lim >> 1, qg, sw >> 1);
         else if (bin_kind == PF_KIND_1F1B)
-            sim_rounds_1f1b(tl, durF, durB, glane, pp, nj, warm, total_ops, lat, fonly, clock, done, P.chk, w_lim, r_lim);
+            sim_rounds_1f1b(tl, durF, durB, glane, pp, nj, warm, total_ops, lat, fonly, clock, done, P.chk, w_lim, r_lim, sw);
         else if (bin_kind == PF_KIND_INTERLEAVED)
             sim_rounds_interleaved(tl, durF, durB, glane, pp, v, nj, U, warm, total_ops, lat, fonly, clock, done, P.chk,
-                                   w_lim, r_lim, qg);
+                                   w_lim, r_lim, qg, sw);
         else
-            sim_rounds_dual(tl, durF, durB, glane, pp, nj, dops, total_ops, lat, clock, done, P.chk, w_lim, r_lim, qg);
+            sim_rounds_dual(tl, durF, durB, glane, pp, nj, dops, total_ops, lat, clock, done, P.chk, w_lim, r_lim, qg, sw);
         if (done < total_ops) stalled = true;
 
         // the next batch's records are requested before this batch's results are reduced and stored
@@ -1250,15 +1268,23 @@ static int launch_simulate(pf_plan_t *p, SimArgs a, uint64_t n, cudaStream_t st,
     const uint64_t want = (n + kSimThreads / 32 - 1) / (kSimThreads / 32);
     const int grid = (int)(want < cap ? want : cap);
     const int threads = kSimThreads;
-    // (the pre-pass puts survivors on ring timelines in calls of at least kSimRingMinSurvivors only)
-    const auto kernel = n >= kSimRingMinSurvivors ? simulate_kernel<true> : simulate_kernel<false>;
-    PF_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)geo.pool),
+    // Two instances (see simulate_kernel): a list that can hold kSimRingMinSurvivors gets both launches, and the one
+    // that does not match the actual count ends at once.
+    const bool both = n >= kSimRingMinSurvivors;
+    PF_CUDA_TRY(cudaFuncSetAttribute(simulate_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)geo.pool),
                 "simulate_kernel smem");
+    if (both)
+        PF_CUDA_TRY(cudaFuncSetAttribute(simulate_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)geo.pool),
+                    "simulate_kernel smem");
     timing_begin(p, PF_T_SIMULATE, st);
-    launch_chained(kernel, grid, threads, geo.pool, st, p->dev, a);
+    if (both) {
+        launch_chained(simulate_kernel<true>, grid, threads, geo.pool, st, p->dev, a);
+        count_launch();
+    }
+    launch_chained(simulate_kernel<false>, grid, threads, geo.pool, st, p->dev, a);
     count_launch();
-    timing_end(p, PF_T_SIMULATE, 1, st);
-    *n_kernels = 4;
+    timing_end(p, PF_T_SIMULATE, both ? 2 : 1, st);
+    *n_kernels = both ? 5 : 4;
     PF_CUDA_TRY(cudaGetLastError(), "simulate_kernel launch");
     return PF_OK;
 }
