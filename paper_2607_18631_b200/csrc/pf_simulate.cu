@@ -8,13 +8,15 @@
 // the backward of stage q+1; the op's own forward is already behind the lane's clock.
 //
 // Launch structure: a counting-sort pre-pass (classify, offsets, scatter) bins the survivors by
-// (timeline size class, lane-group width 4/8/16/32, round loop), then ONE simulate_kernel launch serves all
-// bins, largest timelines first.  Every warp owns a slice of the block's shared memory and runs its own
+// (timeline size class, lane-group width 4/8/16/32, round loop), then ONE simulate_kernel grid serves all
+// bins, largest timelines first (of the kernel's two instances, for small and for large calls, the one that
+// matches the actual survivor count; the other, if launched, ends at once).  Every warp owns a slice of the block's shared memory and runs its own
 // candidates there; the timeline is one signed 32-bit word per (stage stream, microbatch), microbatch-major (word
 // j * streams + stream, so that the lanes of a group touch neighbouring words) -- 0 nothing finished, +t forward
 // ended at t, -t backward ended at t -- written by its owner lane and polled by the neighbour.  In a large call
 // (kSimRingMinSurvivors) interleaved schedules run on a ring of 2 pp microbatch slots per stage stream instead
-// (tagged two-word slots), which lets more candidates share a warp, and pipelines of depth <= 4 take four lanes.
+// (tagged two-word slots), which lets more candidates share a warp, pipelines of depth <= 4 take four lanes, and
+// timeline indices are XORed with a constant of the lane group so that the groups of a warp use different banks.
 // No block barrier is used, and a warp whose lanes make no progress for 64 rounds reports its unfinished
 // candidates as PF_SIM_STALL, so every loop is bounded by the op count.
 #include <cstdlib>
