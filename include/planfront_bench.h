@@ -3,7 +3,7 @@
  * (planfront.h): the paper has no counterpart for anything declared here and no scoring call depends on it.
  *
  * Two groups:
- *   - pf_timing_enable / pf_timing_read / pf_launch_count are exported by libplanfront.so itself, because they
+ *   - pf_timing_enable / pf_timing_classes / pf_timing_read / pf_launch_count are exported by libplanfront.so itself, because they
  *     instrument launches the library makes on streams of its own, which a caller's events cannot bracket;
  *   - pf_probe_alu / pf_probe_write are exported by a separate library, libplanfront_probe.so: micro-kernels that
  *     measure the denominators of the rooflines (instruction issue rates, the pure streaming-write rate).
@@ -33,6 +33,12 @@ enum {
 };
 int pf_timing_enable(pf_plan_t *plan, int on);
 int pf_timing_read(pf_plan_t *plan, float *ms, uint32_t *kernels);
+/* Restrict the timing to the classes whose bit (1 << PF_T_...) is set in `mask` (default: all) and to every
+ * `every`-th launch group of a class (default 1: all; 0 counts as 1).  An event between two kernels of a chain costs
+ * the chain its overlapped launches, and a timed event in front of the kernel a call waits for last costs the call
+ * microseconds, so a benchmark that needs one kernel's duration inside its timed region selects that class alone,
+ * samples it, and reads the other classes in a pass of their own.  PF_EINVAL: plan NULL. */
+int pf_timing_classes(pf_plan_t *plan, uint32_t mask, uint32_t every);
 
 /* Number of kernels this library has launched in this process (for launch accounting in benchmarks). */
 uint64_t pf_launch_count(void);

@@ -29,7 +29,7 @@ EXPORTS = ("pf_version", "pf_strerror", "pf_reason_str", "pf_last_cuda_error", "
            "pf_search_compact_workspace", "pf_search_host_compact", "pf_select_hist", "pf_select_cut",
            "pf_select_write")
 # measurement hooks of include/planfront_bench.h that this library exports (the probes live in probes.py)
-BENCH_EXPORTS = ("pf_launch_count", "pf_timing_enable", "pf_timing_read", "pf_bench_fill_span", "pf_check_read", "pf_check_selftest")
+BENCH_EXPORTS = ("pf_launch_count", "pf_timing_enable", "pf_timing_classes", "pf_timing_read", "pf_bench_fill_span", "pf_check_read", "pf_check_selftest")
 STATIC_SCRATCH_BYTES = 4 << 20
 T_CLASSES = ("score", "topk", "select", "simulate", "aggregate", "fill", "simprep", "compact")
 REASON_BINS = 16
@@ -161,6 +161,8 @@ def load_library(path: str | None = None):
     L.pf_launch_count.restype = u64
     L.pf_timing_enable.restype = C.c_int
     L.pf_timing_enable.argtypes = [vp, C.c_int]
+    L.pf_timing_classes.restype = C.c_int
+    L.pf_timing_classes.argtypes = [vp, C.c_uint32, C.c_uint32]
     L.pf_timing_read.restype = C.c_int
     L.pf_timing_read.argtypes = [vp, vp, vp]
     L.pf_check_selftest.restype = C.c_int
@@ -317,6 +319,11 @@ class Plan:
     # ---- pf_timing_enable / pf_timing_read
     def timing_enable(self, on: bool = True):
         _check(self._L.pf_timing_enable(self._h, 1 if on else 0), "pf_timing_enable")
+
+    def timing_classes(self, names=None, every: int = 1):
+        """pf_timing_classes: time only the named classes (names of T_CLASSES; None: all), every `every`-th time."""
+        mask = 0xFFFFFFFF if names is None else sum(1 << T_CLASSES.index(n) for n in names)
+        _check(self._L.pf_timing_classes(self._h, mask, every), "pf_timing_classes")
 
     def check_selftest(self) -> int:
         return int(self._L.pf_check_selftest(self._h))

@@ -39,6 +39,9 @@ struct TimingRec {
 };
 struct Timing {
     bool on = false;
+    uint32_t mask = ~0u;   // classes that are timed
+    uint32_t every = 1;    // ... in every `every`-th of their launch groups
+    uint32_t seen[PF_T_CLASSES] = {};
     std::vector<TimingRec> recs;
     std::vector<cudaEvent_t> pool;
     cudaEvent_t get()
@@ -57,7 +60,8 @@ struct Timing {
 void timing_begin(pf_plan_t *p, int cls, cudaStream_t st)
 {
     Timing *t = (Timing *)p->timing;
-    if (!t || !t->on) return;
+    if (!t || !t->on || !((t->mask >> cls) & 1u)) return;
+    if (t->seen[cls]++ % t->every != 0) return;   // (timing_end finds no open record of the class and does nothing)
     TimingRec r;
     r.cls = cls;
     r.n_kernels = 0;
@@ -71,7 +75,7 @@ void timing_begin(pf_plan_t *p, int cls, cudaStream_t st)
 void timing_end(pf_plan_t *p, int cls, int n_kernels, cudaStream_t st)
 {
     Timing *t = (Timing *)p->timing;
-    if (!t || !t->on) return;
+    if (!t || !t->on || !((t->mask >> cls) & 1u)) return;
     // the latest open record of this class (records of classes launched on other streams may lie in between)
     for (size_t i = t->recs.size(); i-- > 0;) {
         TimingRec &r = t->recs[i];
@@ -599,6 +603,17 @@ extern "C" int pf_timing_enable(pf_plan_t *p, int on)
     if (!p) return PF_EINVAL;
     if (!p->timing) p->timing = new pf::Timing;
     ((pf::Timing *)p->timing)->on = on != 0;
+    return PF_OK;
+}
+
+extern "C" int pf_timing_classes(pf_plan_t *p, uint32_t mask, uint32_t every)
+{
+    if (!p) return PF_EINVAL;
+    if (!p->timing) p->timing = new pf::Timing;
+    pf::Timing *t = (pf::Timing *)p->timing;
+    t->mask = mask;
+    t->every = every ? every : 1;
+    for (uint32_t &s : t->seen) s = 0;
     return PF_OK;
 }
 
