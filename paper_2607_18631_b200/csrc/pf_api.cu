@@ -92,6 +92,34 @@ void timing_end(pf_plan_t *p, int cls, int n_kernels, cudaStream_t st)
 using pf::DevPlan;
 
 namespace pf {
+// ------------------------------------------------------------------ dynamic shared-memory limits
+namespace {
+constexpr int kSmemDevices = 64;
+struct SmemLimit {
+    const void *kernel;
+    size_t have[kSmemDevices];
+};
+std::mutex g_smem_mu;
+std::vector<SmemLimit> g_smem;   // a handful of kernels: a linear search
+}  // namespace
+
+cudaError_t ensure_dynamic_smem(const void *kernel, int device, size_t bytes)
+{
+    if (device < 0 || device >= kSmemDevices) return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+    std::lock_guard<std::mutex> lock(g_smem_mu);
+    SmemLimit *l = nullptr;
+    for (SmemLimit &x : g_smem)
+        if (x.kernel == kernel) l = &x;
+    if (!l) {
+        g_smem.push_back(SmemLimit{kernel, {}});
+        l = &g_smem.back();
+    }
+    if (l->have[device] >= bytes) return cudaSuccess;
+    const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+    if (e == cudaSuccess) l->have[device] = bytes;
+    return e;
+}
+
 // ------------------------------------------------------------------ per-device caches of plan resources
 // A plan owns one block of device memory, two streams and six events.  Creating and releasing those through the
 // runtime takes 0.3 - 0.9 ms per plan (measured), several times the search of a large space, so released ones are

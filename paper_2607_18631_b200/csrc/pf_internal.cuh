@@ -170,6 +170,11 @@ void set_cuda_error(cudaError_t e, const char *where);
 // device would hand its kernels pointers of the plan's device: a fault on the GPU instead of an error code)
 int check_device(const pf_plan_t *p);
 void count_launch();
+// Make sure `kernel` may be launched with `bytes` of dynamic shared memory on the plan's device.  That limit is state
+// of the (kernel, device) pair, shared by every thread of the process: it is only ever RAISED, under a lock, so a
+// launch that needs less than another plan's call just asked for stays valid (two threads setting it back and
+// forth made the smaller setting win now and then: "invalid argument" at the other thread's launch).
+cudaError_t ensure_dynamic_smem(const void *kernel, int device, size_t bytes);
 // event pair around the launches of one kernel class; no-ops unless pf_timing_enable(plan, 1)
 void timing_begin(pf_plan_t *p, int cls, cudaStream_t st);
 void timing_end(pf_plan_t *p, int cls, int n_kernels, cudaStream_t st);

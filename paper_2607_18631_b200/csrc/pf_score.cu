@@ -1015,8 +1015,12 @@ int launch_topk_reduce(void *d_workspace, const TopkLayout &lay, uint64_t n_keys
         PF_CUDA_TRY(cudaGetLastError(), "reduce_kernel launch");
     }
     r.in = out; r.in_count = ctrl + 2; r.final = 1;
-    PF_CUDA_TRY(cudaFuncSetAttribute(reduce_final_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     (kFastKeys + kTopkCap) * 8), "reduce_final_kernel smem");
+    {
+        int dev = 0;
+        PF_CUDA_TRY(cudaGetDevice(&dev), "reduce_final_kernel device");
+        PF_CUDA_TRY(ensure_dynamic_smem((const void *)reduce_final_kernel, dev, (kFastKeys + kTopkCap) * 8),
+                    "reduce_final_kernel smem");
+    }
     if (chained)
         launch_chained(reduce_final_kernel, 1, kReduceThreads, (kFastKeys + kTopkCap) * 8, st, r);
     else
@@ -1226,12 +1230,9 @@ int pf::score_run(pf_plan_t *p, uint64_t first, uint64_t count, uint8_t *d_reaso
                                    ? (((size_t)p->dev.slab + 16 + 15) & ~(size_t)15) + kQueueCap * sizeof(uint16_t)
                                    : 0;
     // static + dynamic shared memory passes the 48 KB default for large slabs: opt in
-    if (p->dev.wide)
-        PF_CUDA_TRY(cudaFuncSetAttribute(score_kernel<unsigned long long>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)queue_bytes), "score_kernel smem");
-    else
-        PF_CUDA_TRY(cudaFuncSetAttribute(score_kernel<uint32_t>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)queue_bytes), "score_kernel smem");
+    PF_CUDA_TRY(ensure_dynamic_smem(p->dev.wide ? (const void *)score_kernel<unsigned long long>
+                                                : (const void *)score_kernel<uint32_t>,
+                                    p->device, queue_bytes), "score_kernel smem");
     if (p->dev.wide)
         score_kernel<unsigned long long><<<grid, kThreads, queue_bytes, st>>>(p->dev, a);
     else

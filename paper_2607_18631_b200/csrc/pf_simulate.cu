@@ -1273,11 +1273,9 @@ static int launch_simulate(pf_plan_t *p, SimArgs a, uint64_t n, cudaStream_t st,
     // Two instances (see simulate_kernel): a list that can hold kSimRingMinSurvivors gets both launches, and the one
     // that does not match the actual count ends at once.
     const bool both = n >= kSimRingMinSurvivors;
-    PF_CUDA_TRY(cudaFuncSetAttribute(simulate_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)geo.pool),
-                "simulate_kernel smem");
+    PF_CUDA_TRY(ensure_dynamic_smem((const void *)simulate_kernel<false>, p->device, geo.pool), "simulate_kernel smem");
     if (both)
-        PF_CUDA_TRY(cudaFuncSetAttribute(simulate_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)geo.pool),
-                    "simulate_kernel smem");
+        PF_CUDA_TRY(ensure_dynamic_smem((const void *)simulate_kernel<true>, p->device, geo.pool), "simulate_kernel smem");
     timing_begin(p, PF_T_SIMULATE, st);
     if (both) {
         launch_chained(simulate_kernel<true>, grid, threads, geo.pool, st, p->dev, a);

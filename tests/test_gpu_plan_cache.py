@@ -86,11 +86,23 @@ def test_search_after_recycling_matches_a_fresh_process_result():
 
 
 def test_plans_created_and_destroyed_from_several_threads():
-    """The caches are shared by every thread of the process (ctypes calls run without the interpreter lock)."""
+    """The caches, and the kernels' shared-memory limits, are shared by every thread of the process (ctypes calls run
+    without the interpreter lock): plans of different spaces scored and searched from four threads at once."""
     import threading
     import torch
     cfgs = [make_config("mid"), make_config("tiny"), variant("mid", cluster=dict(budget_bytes=10 ** 15))]
     refs = [_ref(c) for c in cfgs]
+
+    def search_result(cfg):
+        plan = _plan(cfg)
+        out = plan.search(64, 1000, 10, 3)
+        torch.cuda.current_stream().synchronize()
+        ns = int(out["sim_topk_count"].item())
+        res = (out["reason"].cpu().numpy().copy(), out["sim_topk_idx"][:ns].cpu().numpy().copy(),
+               out["sim_topk_score"][:ns].cpu().numpy().copy(), int(out["surv_count"].item()))
+        plan.close()
+        return res
+    searched = [search_result(c) for c in cfgs]
     errors = []
 
     def work(seed):
@@ -103,6 +115,9 @@ def test_plans_created_and_destroyed_from_several_threads():
                     plan = _plan(cfgs[j])
                     _parity(plan, cfgs[j], refs[j])
                     plan.close()
+                    got = search_result(cfgs[j])
+                    for x, y in zip(got, searched[j]):
+                        assert np.array_equal(x, y)
         except Exception as ex:   # noqa: BLE001 -- reported by the main thread
             errors.append(repr(ex))
 
