@@ -13,8 +13,9 @@
  *   - plain C, no exceptions; every call returns an int32 status (PF_OK = 0, negative = error).
  *   - "d_" pointers are DEVICE pointers owned by the caller; everything else is HOST memory.
  *   - the library allocates no output or workspace memory: the caller passes raw pointers and sizes.
- *     (pf_plan_create allocates a few KB of device memory for the plan's constant tables, freed by
- *     pf_plan_destroy.)
+ *     (pf_plan_create takes one block of device memory for the plan's tables -- tens of KB; 5 bytes per block of
+ *     candidates for the visiting order -- two streams and six events; pf_plan_destroy waits for the device and
+ *     hands them to a small per-device cache for the next plan instead of releasing them.)
  *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  All device work is
  *     enqueued on it and the calls do not synchronize; results are valid once the stream has been
  *     synchronized by the caller.  pf_search_host is the exception: it takes host buffers and returns
@@ -22,6 +23,8 @@
  *   - spec structs are copied by pf_plan_create; the caller may free them afterwards.
  *   - a handle may be used from one thread at a time, on the device that was current at create: every call
  *     that enqueues device work returns PF_EINVAL (nothing launched) when another device is current.
+ *     Different handles may be used from different threads at the same time (what they share -- the caches above,
+ *     the kernels' shared-memory limits -- is locked).
  *   - candidates are addressed by a linear index: idx = sum_a digit_a * prod_{b<a} len_b, axes listed
  *     least-significant first.  train axes: kv, rec, sched, mb, v, ep, pp, tp, dp, world [, shard];
  *     serve axes: kv, chunk, batch, dpa, ep, tp, scen.  An axis value list {0} for dp / world / v means
