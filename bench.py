@@ -430,7 +430,7 @@ def run_split(args, torch, dist, world, rank, local):
                 "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True,
                 "scaling": "strong", "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": cfgd,
                 "survivors": r["n_survivors_total"], "clocks": clocks, "gpu_launches": int(launches),
-                "collectives_per_step": {"all_reduce": 2, "all_reduce_bytes": 2 * 65536 * 8, "all_gather": 8,
+                "collectives_per_step": {"all_reduce": 2, "all_reduce_bytes": 2 * 65536 * 8, "all_gather": 4,
                                          "all_gather_bytes_per_rank": (K_TOP + K_SIM) * 12 + 8 + 16},
                 "note": "host-driven: per step one device-to-host read of the cut (48 bytes) sits between the "
                         "selection's passes; dense outputs and survivor lists stay on their ranks"}

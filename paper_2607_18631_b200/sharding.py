@@ -82,10 +82,20 @@ class CudaOps:
 
 def _fold(comm, merge, lists, k):
     """All-gather every rank's (idx, score, count) list and fold them into the global top-k on every rank."""
-    parts = [comm.all_gather(t) for t in lists]
-    acc = (parts[0][0], parts[1][0], parts[2][0])
+    import torch
+    idx, score, count = (t.contiguous() for t in lists)
+    if comm.world == 1:
+        return idx, score, count
+    # one collective instead of three: the list travels as one byte string (idx | score | count)
+    nb_i, nb_s = idx.numel() * idx.element_size(), score.numel() * score.element_size()
+    packed = torch.cat([idx.view(torch.uint8), score.view(torch.uint8), count.view(torch.uint8)])
+    parts = comm.all_gather(packed)
+
+    def unpack(buf):
+        return (buf[:nb_i].view(idx.dtype), buf[nb_i:nb_i + nb_s].view(score.dtype), buf[nb_i + nb_s:].view(count.dtype))
+    acc = unpack(parts[0])
     for r in range(1, comm.world):
-        acc = merge(k, acc, (parts[0][r], parts[1][r], parts[2][r]))
+        acc = merge(k, acc, unpack(parts[r]))
     return acc
 
 
