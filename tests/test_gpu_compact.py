@@ -127,3 +127,35 @@ def test_search_host_compact_on_the_large_space():
     r3 = plan.search_host_compact(1024, 10 ** 6, 100, 4, ws, 0)
     assert r3["n_feasible"] == 12_905 and r3["records"] is None
     plan.close()
+
+
+@pytest.mark.parametrize("name,k,s_max,k_sim", [("mid", 64, 1000, 10), ("tiny", 16, 100, 5), ("serve", 64, 0, 0)])
+def test_search_host_compact_small_spaces_pinned_and_pageable(name, k, s_max, k_sim):
+    """The host call's two ways of filling the mask (device writes into a pinned buffer over a copy of zeros; one copy
+    into a pageable one) on spaces whose last chunk is partial, with the mask at an even and at an odd address, on a
+    training space with and a serving space without the simulator tier."""
+    import torch
+    cfg = make_config(name)
+    plan, orc = _plan(cfg), Oracle(cfg)
+    N = plan.size
+    reason, _, _, _ = orc.score_range(threads=8)
+    feas = (reason & 0x7F) == 0
+    n_feas = int(feas.sum())
+    cap = n_feas + 10
+    ks = max(k_sim, 1) if s_max else 0
+    ws = torch.empty(plan.search_compact_workspace(k, s_max, ks, cap), dtype=torch.uint8, device="cuda")
+    nb = (N + 7) // 8
+    for pinned in (False, True):
+        for lead in (0, 3):
+            buf = torch.full((lead + nb + 8,), 0xA5, dtype=torch.uint8)
+            if pinned:
+                buf = buf.pin_memory()
+            ws.fill_(0x85)
+            r = plan.search_host_compact(k, s_max, ks, 4, ws, cap, h_mask=buf[lead:lead + nb])
+            g = buf.numpy()
+            bits = np.unpackbits(g[lead:lead + nb], bitorder="little")[:N].astype(bool)
+            np.testing.assert_array_equal(bits, feas)
+            assert (g[:lead] == 0xA5).all() and (g[lead + nb:] == 0xA5).all()
+            assert r["n_feasible"] == n_feas and r["n_records"] == n_feas
+            np.testing.assert_array_equal(r["records"][:n_feas]["idx"], np.nonzero(feas)[0].astype(np.uint64))
+    plan.close()
