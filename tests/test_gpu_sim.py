@@ -324,3 +324,31 @@ def test_one_million_survivors_against_the_oracle():
     check_topk(sim["topk_idx"].cpu().numpy().view(np.uint64)[:k], sim["topk_score"].cpu().numpy()[:k], ref_idx,
                ref_sc)
     plan.close()
+
+
+def test_both_simulator_instances_give_the_same_bits_at_the_threshold():
+    """A call of 32,767 survivors runs the small-call kernel (full timelines, eight-lane groups, plain indices), one
+    of 32,768 the large-call kernel (ring timelines, four-lane groups, permuted indices).  The arithmetic per
+    candidate is the same sequence of fp32 operations either way, so the survivors the two calls share must get the
+    same bits; and a list with room for more than it holds must be served by the instance its actual length asks
+    for."""
+    import torch
+    from paper_2607_18631_b200 import Plan
+    plan = Plan(make_config("large_unconstrained"))
+    b = plan.search(1024, 10 ** 6, 100, 4)
+    torch.cuda.synchronize()
+    ns = int(b["surv_count"].item())
+    surv = b["surv_idx"][:ns].clone()
+    T = 32768
+    assert ns > T
+    small = plan.simulate(surv[:T - 1].contiguous(), T - 1, 4)
+    large = plan.simulate(surv[:T].contiguous(), T, 4)
+    d_n = torch.tensor([T - 1], dtype=torch.int64, device="cuda")
+    roomy = plan.simulate(surv.contiguous(), ns, 4, d_n=d_n)
+    torch.cuda.synchronize()
+    s_small, s_large = small["tput_sim"].cpu().numpy(), large["tput_sim"][:T - 1].cpu().numpy()
+    assert (s_small > 0).all()
+    np.testing.assert_array_equal(s_small, s_large)
+    np.testing.assert_array_equal(small["sim_status"].cpu().numpy(), large["sim_status"][:T - 1].cpu().numpy())
+    np.testing.assert_array_equal(s_small, roomy["tput_sim"][:T - 1].cpu().numpy())
+    plan.close()
