@@ -180,12 +180,11 @@ def test_search_streams_constant_blocks_of_odd_size_exactly():
     plan.close()
 
 
-@pytest.mark.parametrize("name", ["large", "large_unconstrained"])
+@pytest.mark.parametrize("name", ["large"])
 def test_search_gives_the_same_bits_call_after_call(name):
     """Back-to-back calls overlap one call's last kernels with the next call's first ones on four streams (the
     caller's, two of the plan's, the chained launches in between); every output must come out bit for bit the
-    same, whatever the buffers held -- 12,905 survivors take the simulator's small-call kernel, 45,116 the
-    large-call one."""
+    same, whatever the buffers held."""
     import torch
     from paper_2607_18631_b200 import Plan
     plan = Plan(make_config(name))
