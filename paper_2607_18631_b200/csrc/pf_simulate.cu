@@ -1280,12 +1280,10 @@ static int launch_simulate(pf_plan_t *p, SimArgs a, uint64_t n, cudaStream_t st,
     if (both) {
         launch_chained(simulate_kernel<true>, grid, threads, geo.pool, st, p->dev, a);
         count_launch();
-        // a plain launch: chained, this instance's blocks would sit on the SMs waiting for as long as the other one
-        // runs (milliseconds in a large call)
-        simulate_kernel<false><<<grid, threads, geo.pool, st>>>(p->dev, a);
-    } else {
-        launch_chained(simulate_kernel<false>, grid, threads, geo.pool, st, p->dev, a);
     }
+    // (chained behind a running first instance, this one's blocks cannot land before blocks of that one leave: three
+    // blocks of either fill an SM's shared memory)
+    launch_chained(simulate_kernel<false>, grid, threads, geo.pool, st, p->dev, a);
     count_launch();
     timing_end(p, PF_T_SIMULATE, both ? 2 : 1, st);
     *n_kernels = both ? 5 : 4;
